@@ -1,0 +1,182 @@
+"""ORACLE — test infrastructure, not the product.
+
+A plain, slow CPU implementation (C, double precision) of what leaf evaluation computes:
+legal-move masks, input planes, the residual policy/value network and the masked softmax.
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this package; the
+CUDA library never does, and this package imports nothing of the CUDA library.
+
+The C sources are compiled on first use with the host's gcc (OpenMP for the per-position loop).
+"""
+import ctypes
+import hashlib
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SOURCES = ("chess_oracle.c", "net_oracle.c")
+_lib = None
+
+
+def _cpu_tag() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("flags"):
+                    return hashlib.sha1(line.encode()).hexdigest()[:8]
+    except OSError:
+        pass
+    return "generic"
+
+
+def build() -> str:
+    """Compile the oracle's C files into one shared library beside them; returns its path."""
+    h = hashlib.sha1()
+    for s in _SOURCES:
+        with open(os.path.join(_HERE, s), "rb") as f:
+            h.update(f.read())
+    out = os.path.join(_HERE, f"liboracle_{h.hexdigest()[:10]}_{_cpu_tag()}.so")
+    if not os.path.exists(out):
+        tmp = out + f".tmp{os.getpid()}"
+        cmd = ["gcc", "-O3", "-march=native", "-std=c11", "-fopenmp", "-shared", "-fPIC",
+               *[os.path.join(_HERE, s) for s in _SOURCES], "-lm", "-o", tmp]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, out)
+    return out
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        vp, ci = ctypes.c_void_p, ctypes.c_int
+        lib.orc_perft.restype = ctypes.c_uint64
+        lib.orc_perft.argtypes = [vp, ci]
+        lib.orc_legal_moves.restype = ci
+        lib.orc_legal_moves.argtypes = [vp, vp]
+        lib.orc_flat_count.restype = ci
+        lib.orc_policy_index.restype = ci
+        lib.orc_policy_index.argtypes = [ci] * 6
+        lib.orc_legal_masks.restype = ci
+        lib.orc_legal_masks.argtypes = [vp, ci, ci, ci, vp]
+        lib.orc_encode.restype = ci
+        lib.orc_encode.argtypes = [vp, ci, ci, ci, vp]
+        lib.orc_conv3x3.restype = None
+        lib.orc_conv3x3.argtypes = [vp, vp, ci, ci, vp]
+        lib.orc_masked_softmax.restype = None
+        lib.orc_masked_softmax.argtypes = [vp, vp, ci, vp]
+        lib.orc_forward.restype = ci
+        lib.orc_forward.argtypes = [vp, ctypes.c_size_t, vp, vp, ci, vp, vp, vp, vp, vp]
+        lib.orc_threads.restype = ci
+        _lib = lib
+    return _lib
+
+
+POLICY_SIZE = {0: 73 * 64, 1: 1858}
+MASK_WORDS = {0: 73, 1: 30}
+
+
+def _records(records):
+    rec = np.ascontiguousarray(records)
+    return rec, rec.dtype.itemsize, rec.shape[0] if rec.ndim else 1
+
+
+def perft(record, depth: int) -> int:
+    rec = np.ascontiguousarray(record)
+    return int(_load().orc_perft(rec.ctypes.data, depth))
+
+
+def legal_moves(record):
+    """Sorted (from, to, promo) triples; promo 0 none, 1 N, 2 B, 3 R, 4 Q; castling as the king's move."""
+    rec = np.ascontiguousarray(record)
+    buf = np.zeros(256 * 3, dtype=np.uint8)
+    n = _load().orc_legal_moves(rec.ctypes.data, buf.ctypes.data)
+    return sorted(tuple(int(v) for v in buf[3 * i:3 * i + 3]) for i in range(n))
+
+
+def flat_count() -> int:
+    return int(_load().orc_flat_count())
+
+
+def policy_index(head: int, stm: int, frm: int, to: int, promo: int = 0, castle: int = 0) -> int:
+    return int(_load().orc_policy_index(head, stm, frm, to, promo, castle))
+
+
+def legal_masks(records, head: int) -> np.ndarray:
+    """uint64 [n][73 or 30]: bit (i & 63) of word (i >> 6) set iff policy index i is legal."""
+    rec, stride, n = _records(records)
+    masks = np.zeros((n, MASK_WORDS[head]), dtype=np.uint64)
+    rc = _load().orc_legal_masks(rec.ctypes.data, stride, n, head, masks.ctypes.data)
+    if rc != 0:
+        raise RuntimeError("a legal move had no policy index")
+    return masks
+
+
+def encode(records, in_planes: int) -> np.ndarray:
+    """float64 [n][in_planes][8][8] input planes, mover-oriented."""
+    rec, stride, n = _records(records)
+    if in_planes == 112 and stride != 784:
+        raise ValueError("the 112-plane encoding needs records with history")
+    planes = np.zeros((n, in_planes, 8, 8), dtype=np.float64)
+    if _load().orc_encode(rec.ctypes.data, stride, n, in_planes, planes.ctypes.data) != 0:
+        raise ValueError("unsupported plane count")
+    return planes
+
+
+def conv3x3(weight: np.ndarray, x: np.ndarray) -> np.ndarray:
+    """weight float32 [cout][cin][3][3], x float64 [cin][8][8] -> float64 [cout][8][8]."""
+    w = np.ascontiguousarray(weight, dtype=np.float32)
+    xin = np.ascontiguousarray(x, dtype=np.float64)
+    cout, cin = w.shape[0], w.shape[1]
+    out = np.zeros((cout, 8, 8), dtype=np.float64)
+    _load().orc_conv3x3(w.ctypes.data, xin.ctypes.data, cin, cout, out.ctypes.data)
+    return out
+
+
+def masked_softmax(logits: np.ndarray, mask_words: np.ndarray) -> np.ndarray:
+    lg = np.ascontiguousarray(logits, dtype=np.float64)
+    mk = np.ascontiguousarray(mask_words, dtype=np.uint64)
+    out = np.zeros_like(lg)
+    _load().orc_masked_softmax(lg.ctypes.data, mk.ctypes.data, lg.shape[0], out.ctypes.data)
+    return out
+
+
+def forward(blob: np.ndarray, planes: np.ndarray, masks: np.ndarray, want_raw: bool = False,
+            want_tower: bool = False):
+    """Network + masked softmax on already-encoded planes.
+
+    Returns (policy [n][4672|1858], value [n][1|3]) and, on request, a dict with the raw logits,
+    the value head's pre-activation and the tower's final activations.
+    """
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    hdr = np.frombuffer(blob[8:36].tobytes(), dtype="<u4")
+    channels, policy_head, value_head = int(hdr[3]), int(hdr[4]), int(hdr[5])
+    pl = np.ascontiguousarray(planes, dtype=np.float64)
+    mk = np.ascontiguousarray(masks, dtype=np.uint64)
+    n = pl.shape[0]
+    npol, V = POLICY_SIZE[policy_head], 3 if value_head else 1
+    policy = np.zeros((n, npol), dtype=np.float64)
+    value = np.zeros((n, V), dtype=np.float64)
+    raw_l = np.zeros((n, npol), dtype=np.float64) if want_raw else None
+    raw_v = np.zeros((n, V), dtype=np.float64) if want_raw else None
+    tower = np.zeros((n, channels, 8, 8), dtype=np.float64) if want_tower else None
+    ptr = lambda a: a.ctypes.data if a is not None else None
+    rc = _load().orc_forward(blob.ctypes.data, blob.nbytes, pl.ctypes.data, mk.ctypes.data, n,
+                             policy.ctypes.data, value.ctypes.data, ptr(raw_l), ptr(raw_v), ptr(tower))
+    if rc != 0:
+        raise ValueError("malformed weight blob")
+    if want_raw or want_tower:
+        return policy, value, {"logits": raw_l, "value_pre": raw_v, "tower": tower}
+    return policy, value
+
+
+def evaluate(blob: np.ndarray, records, in_planes: int, policy_head: int, **kw):
+    """The whole path: masks from the rules, planes from the records, network, masked softmax."""
+    masks = legal_masks(records, policy_head)
+    planes = encode(records, in_planes)
+    return (masks, planes) + tuple(forward(blob, planes, masks, **kw))
+
+
+def threads() -> int:
+    return int(_load().orc_threads())
