@@ -1,0 +1,187 @@
+/*
+ * az_eval — batched evaluation of search-tree leaf positions on one NVIDIA B200 (sm_100a).
+ *
+ * The operation (Sec. 3.1 "At a new leaf, the network evaluates the position"; Sec. 3.3 requests
+ * of many games are grouped into one GPU batch; App. D.1 network input and output contract):
+ * a flat batch of independent chess positions goes in; for every position come out
+ *   - prior probabilities over its legal moves (illegal actions masked before the softmax), and
+ *   - a value for the player to move (win/draw/loss probabilities, or one tanh scalar).
+ * Steps, all executed by this library's own CUDA kernels on the caller's stream:
+ *   bitboards -> input planes -> 3x3 residual convolution tower (folded batch-norm, residual add,
+ *   ReLU) -> policy head and value head -> legal-move-masked softmax.
+ *
+ * Conventions
+ *   - Every function returns AZ_OK (0) or a negative AZ_ERR_* code; nothing throws or aborts.
+ *   - "dev" pointers are device memory of the device that was current at az_load_net; "host"
+ *     pointers are ordinary host memory.  The caller owns every buffer it passes and the stream.
+ *     The az_net owns its weights and a workspace sized for arch.max_batch (freed by az_free_net).
+ *   - Calls that take a stream are asynchronous on it.  Calls on one az_net must not overlap on
+ *     the GPU (they share the workspace): use one az_net per stream.
+ *   - There is no CPU fallback: without a usable CUDA device az_load_net fails with AZ_ERR_CUDA.
+ *
+ * Squares are numbered file + 8*rank (a1 = 0, b1 = 1, ..., h8 = 63).
+ */
+#ifndef AZ_EVAL_H
+#define AZ_EVAL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define AZ_ABI_VERSION 1
+
+enum {
+    AZ_OK = 0,
+    AZ_ERR_BAD_ARG = -1,          /* null pointer, negative size, misaligned buffer */
+    AZ_ERR_BAD_ARCH = -2,         /* unsupported combination in az_arch */
+    AZ_ERR_BAD_WEIGHTS = -3,      /* blob too short, wrong magic, header disagrees with az_arch, NaN/Inf */
+    AZ_ERR_BATCH_TOO_LARGE = -4,  /* batch > arch.max_batch */
+    AZ_ERR_CUDA = -5,             /* a CUDA runtime call failed (see az_last_cuda_error) */
+    AZ_ERR_DEVICE_TIMEOUT = -6,   /* a bounded device-side wait ran out (see az_device_status) */
+    AZ_ERR_NOT_CALIBRATED = -7,   /* FP8 tower used before az_calibrate */
+    AZ_ERR_UNSUPPORTED = -8       /* valid request that this build has no kernel for */
+};
+
+enum { AZ_POLICY_PLANES73 = 0, AZ_POLICY_FLAT1858 = 1 };
+enum { AZ_VALUE_TANH = 0, AZ_VALUE_WDL = 1 };
+enum { AZ_PREC_FP32 = 0, AZ_PREC_BF16 = 1, AZ_PREC_FP8_E4M3 = 2 };
+
+/* Network shape.  in_planes 19 or 112; blocks >= 0 residual blocks of `channels` channels
+ * (a multiple of 16); heads and precision as the enums above; max_batch sizes the workspace. */
+typedef struct {
+    uint32_t abi_version;   /* AZ_ABI_VERSION */
+    uint32_t in_planes;
+    uint32_t blocks;
+    uint32_t channels;
+    uint32_t policy_head;
+    uint32_t value_head;
+    uint32_t precision;
+    uint32_t max_batch;
+} az_arch;
+
+/* One position, 104 bytes.  pieces[] are absolute-colour bitboards in the order white P,N,B,R,Q,K
+ * then black P,N,B,R,Q,K.  ep_square is the square behind a pawn that has just advanced two ranks
+ * (64 if none).  halfmove is the fifty-move clock, repetitions the number of earlier occurrences
+ * of this position in its game; both saturate at 255. */
+typedef struct {
+    uint64_t pieces[12];
+    uint8_t stm;            /* 0 white to move, 1 black to move */
+    uint8_t castling;       /* bit0 white O-O, bit1 white O-O-O, bit2 black O-O, bit3 black O-O-O */
+    uint8_t ep_square;
+    uint8_t halfmove;
+    uint8_t repetitions;
+    uint8_t pad[3];
+} az_position;
+
+/* Position with the seven boards before it (784 bytes); consumed by 112-plane networks.
+ * hist_pieces[t-1] is the board t plies ago, n_hist (0..7) says how many are present. */
+typedef struct {
+    az_position cur;
+    uint64_t hist_pieces[7][12];
+    uint8_t hist_rep[7];
+    uint8_t n_hist;
+} az_position_h8;
+
+typedef struct az_net az_net;
+
+/* Size in bytes of one position record / of one position's outputs for a given arch. */
+size_t az_position_bytes(const az_arch *arch);      /* 104 (19 planes) or 784 (112 planes) */
+size_t az_policy_size(const az_arch *arch);         /* 4672 or 1858 floats per position */
+size_t az_mask_words(const az_arch *arch);          /* 73 or 30 uint64 words per position */
+size_t az_value_size(const az_arch *arch);          /* 1 or 3 floats per position */
+size_t az_plane_channels(const az_arch *arch);      /* channels of the encoded plane tensor: 32 or 128 */
+
+/*
+ * load_net(weights, arch)  (Sec. 3.3 publication hands the actors a network; Sec. 4.3.6 and
+ * App. D.3: batch-norm is folded into the convolutions on a deployment copy).
+ * weights_host: `nbytes` of host memory holding the blob: a 64-byte header (8-byte magic
+ * "AZNETv1\0", then uint32 version=1, in_planes, blocks, channels, policy_head, value_head,
+ * tensor_count, zero padding) followed by raw little-endian float32 tensors in this order:
+ *   input conv W[C][P][3][3], scale[C], bias[C];
+ *   per block W1[C][C][3][3], scale1[C], bias1[C], W2[C][C][3][3], scale2[C], bias2[C];
+ *   policy head: planes73 Wp[73][C], bp[73] | flat Wc[32][C], scale[32], bias[32], Wf[1858][2048], bf[1858];
+ *   value head Wc[32][C], scale[32], bias[32], W1[128][2048], b1[128], W2[V][128], b2[V] (V = 1 or 3).
+ * Convolution weights are [out][in][ky][kx]; "scale/bias" are the folded batch-norm
+ * (y = scale*conv + bias).  Fully-connected inputs are flattened channel-major (c*64 + square).
+ * The blob is copied; the caller may free it on return.  On success *out receives the network.
+ * Errors: BAD_ARG, BAD_ARCH, BAD_WEIGHTS, CUDA.
+ */
+int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az_net **out);
+
+/* Frees the network's device memory.  Null is allowed. */
+void az_free_net(az_net *net);
+
+/*
+ * evaluate(positions, legal_masks) -> (policy, value)   (Sec. 3.1, Sec. 3.6, App. D.1).
+ * positions_dev: `batch` records of az_position_bytes() each.
+ * legal_masks_dev: [batch][az_mask_words()] uint64; bit (i & 63) of word (i >> 6) is set iff
+ *   policy index i is a legal move (for the 73-plane head word p is plane p, bit s the origin).
+ * policy_dev: [batch][az_policy_size()] float32 out: softmax over the legal entries, exactly 0
+ *   elsewhere; a position whose mask is empty gets an all-zero row.
+ * value_dev: [batch][az_value_size()] float32 out: tanh scalar, or (win, draw, loss) for the
+ *   player to move.
+ * Errors: BAD_ARG, BATCH_TOO_LARGE, NOT_CALIBRATED, CUDA.  batch == 0 is a no-op.
+ */
+int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_masks_dev,
+                int batch, float *policy_dev, float *value_dev, void *cuda_stream);
+
+/*
+ * The encoder step alone (App. D.1: side-to-move canonical planes; for Black to move ranks are
+ * reflected and colours exchanged, files keep their order).  planes_dev receives
+ * [batch][64][az_plane_channels()] elements of the network's activation type (float32 for
+ * AZ_PREC_FP32, bfloat16 otherwise), square-major, channels beyond in_planes zero.
+ * 19 planes: 0-5 own P,N,B,R,Q,K; 6-11 opponent's; 12 one iff Black to move; 13-16 castling rights
+ * own king side, own queen side, opponent king side, opponent queen side; 17 min(halfmove,100)/100;
+ * 18 one iff repetitions >= 1.  112 planes: for t = 0..7 planes 13t..13t+11 the board t plies ago
+ * (own then opponent, oriented by the current mover) and 13t+12 its repetition flag, zero where
+ * there is no history; 104-107 castling as above; 108 one iff Black to move; 109 halfmove/100;
+ * 110 zeros; 111 ones.
+ */
+int az_encode(az_net *net, const void *positions_dev, int batch, void *planes_dev, void *cuda_stream);
+
+/*
+ * Encoder + convolution tower alone: tower_dev receives [batch][64][channels] elements of the
+ * activation type, the input of both heads (Sec. 3.5 shared backbone).  For layer-level checks.
+ */
+int az_tower(az_net *net, const void *positions_dev, int batch, void *tower_dev, void *cuda_stream);
+
+/*
+ * Legal-move masks from the rules of chess, computed on the GPU, in the layout az_evaluate
+ * takes.  Index maps (mover-oriented coordinates; App. D.1: castling is the king-to-own-rook
+ * pair, en passant the pawn's ordinary pair):
+ *   planes73: index = plane*64 + origin; planes 7*d + (distance-1) for directions d =
+ *     N,NE,E,SE,S,SW,W,NW; 56-63 knight jumps (1,2),(2,1),(2,-1),(1,-2),(-1,-2),(-2,-1),(-2,1),(-1,2)
+ *     as (file,rank) steps; 64 + 3*piece + dir for promotion to N,B,R, dir = capture to file-1,
+ *     straight, capture to file+1; queen promotion uses the one-step plane.
+ *   flat1858: every (origin, destination) a queen ray or knight jump apart, origin ascending then
+ *     destination ascending (1792), then for origins on the seventh rank the destinations
+ *     origin+7,+8,+9 on the board, each with N,B,R (66).
+ * position_stride is the byte distance between records (104 or 784).  No az_net is needed.
+ */
+int az_legal_masks(const void *positions_dev, size_t position_stride, int batch, int policy_head,
+                   uint64_t *masks_dev, void *cuda_stream);
+
+/*
+ * FP8 tower only (Sec. 4.3.6: ranges are fixed on a few hundred calibration positions): runs the
+ * bf16 tower on `n` positions, records per-channel activation ranges and fixes the e4m3 scales.
+ * Synchronises the stream.  Errors: BAD_ARG, BATCH_TOO_LARGE, CUDA, UNSUPPORTED (non-FP8 net).
+ */
+int az_calibrate(az_net *net, const void *positions_dev, int n, void *cuda_stream);
+
+/* Device-side status word of the last kernels (0 = clean).  Synchronises the given stream. */
+int az_device_status(az_net *net, void *cuda_stream, uint32_t *status_out);
+
+/* Number of kernel launches one az_evaluate of `batch` positions enqueues. */
+int az_launches_per_evaluate(const az_net *net, int batch);
+
+const char *az_strerror(int code);
+/* Text of the last CUDA runtime error seen by this thread inside the library ("" if none). */
+const char *az_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AZ_EVAL_H */

@@ -1,0 +1,203 @@
+"""Python binding of the az_eval C library (argument marshalling only).
+
+Every function has the name and meaning of the C entry point declared in include/az_eval.h; all
+computation happens in the library's CUDA kernels.  PyTorch supplies device memory and streams.
+There is no fallback: if libazeval.so is missing or fails to load, importing raises.
+"""
+import ctypes
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libazeval.so")
+
+AZ_ABI_VERSION = 1
+AZ_OK = 0
+AZ_ERR_BAD_ARG, AZ_ERR_BAD_ARCH, AZ_ERR_BAD_WEIGHTS, AZ_ERR_BATCH_TOO_LARGE = -1, -2, -3, -4
+AZ_ERR_CUDA, AZ_ERR_DEVICE_TIMEOUT, AZ_ERR_NOT_CALIBRATED, AZ_ERR_UNSUPPORTED = -5, -6, -7, -8
+AZ_POLICY_PLANES73, AZ_POLICY_FLAT1858 = 0, 1
+AZ_VALUE_TANH, AZ_VALUE_WDL = 0, 1
+AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3 = 0, 1, 2
+
+EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
+           "az_load_net", "az_free_net", "az_evaluate", "az_encode", "az_tower", "az_legal_masks",
+           "az_calibrate", "az_device_status", "az_launches_per_evaluate", "az_strerror",
+           "az_last_cuda_error")
+
+
+class az_arch(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint32) for n in ("abi_version", "in_planes", "blocks", "channels",
+                                               "policy_head", "value_head", "precision", "max_batch")]
+
+
+class AzError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        detail = _lib.az_last_cuda_error().decode() if code == AZ_ERR_CUDA else ""
+        super().__init__(f"{where}: {_lib.az_strerror(code).decode()} ({code}) {detail}".strip())
+
+
+def _load_library():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_37447_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, ci, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    ap = ctypes.POINTER(az_arch)
+    for name in ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels"):
+        getattr(lib, name).restype = sz
+        getattr(lib, name).argtypes = [ap]
+    lib.az_load_net.restype = ci
+    lib.az_load_net.argtypes = [ap, vp, sz, ctypes.POINTER(vp)]
+    lib.az_free_net.restype = None
+    lib.az_free_net.argtypes = [vp]
+    lib.az_evaluate.restype = ci
+    lib.az_evaluate.argtypes = [vp, vp, vp, ci, vp, vp, vp]
+    lib.az_encode.restype = ci
+    lib.az_encode.argtypes = [vp, vp, ci, vp, vp]
+    lib.az_tower.restype = ci
+    lib.az_tower.argtypes = [vp, vp, ci, vp, vp]
+    lib.az_legal_masks.restype = ci
+    lib.az_legal_masks.argtypes = [vp, sz, ci, ci, vp, vp]
+    lib.az_calibrate.restype = ci
+    lib.az_calibrate.argtypes = [vp, vp, ci, vp]
+    lib.az_device_status.restype = ci
+    lib.az_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.az_launches_per_evaluate.restype = ci
+    lib.az_launches_per_evaluate.argtypes = [vp, ci]
+    lib.az_strerror.restype = ctypes.c_char_p
+    lib.az_strerror.argtypes = [ci]
+    lib.az_last_cuda_error.restype = ctypes.c_char_p
+    lib.az_last_cuda_error.argtypes = []
+    return lib
+
+
+_lib = _load_library()
+
+
+def _check(code: int, where: str):
+    if code != AZ_OK:
+        raise AzError(code, where)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _dev_ptr(t: torch.Tensor, name: str) -> int:
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def make_arch(in_planes, blocks, channels, policy_head, value_head, precision, max_batch) -> az_arch:
+    return az_arch(AZ_ABI_VERSION, in_planes, blocks, channels, policy_head, value_head, precision, max_batch)
+
+
+def az_position_bytes(arch: az_arch) -> int:
+    return int(_lib.az_position_bytes(ctypes.byref(arch)))
+
+
+def az_policy_size(arch: az_arch) -> int:
+    return int(_lib.az_policy_size(ctypes.byref(arch)))
+
+
+def az_mask_words(arch: az_arch) -> int:
+    return int(_lib.az_mask_words(ctypes.byref(arch)))
+
+
+def az_value_size(arch: az_arch) -> int:
+    return int(_lib.az_value_size(ctypes.byref(arch)))
+
+
+def az_plane_channels(arch: az_arch) -> int:
+    return int(_lib.az_plane_channels(ctypes.byref(arch)))
+
+
+@dataclass
+class Net:
+    """Handle of a loaded network (owns device weights and workspace; call az_free_net when done)."""
+    handle: int
+    arch: az_arch
+
+    @property
+    def act_dtype(self):
+        return torch.float32 if self.arch.precision == AZ_PREC_FP32 else torch.bfloat16
+
+
+def az_load_net(arch: az_arch, weights_host) -> Net:
+    """weights_host: the weight blob as bytes / numpy uint8 array (host memory)."""
+    blob = np.ascontiguousarray(np.frombuffer(weights_host, dtype=np.uint8) if isinstance(weights_host, (bytes, bytearray))
+                                else weights_host, dtype=np.uint8)
+    out = ctypes.c_void_p()
+    _check(_lib.az_load_net(ctypes.byref(arch), blob.ctypes.data, blob.nbytes, ctypes.byref(out)), "az_load_net")
+    return Net(out.value, arch)
+
+
+def az_free_net(net: Net):
+    if net is not None and net.handle:
+        _lib.az_free_net(net.handle)
+        net.handle = 0
+
+
+def az_evaluate(net: Net, positions_dev, legal_masks_dev, batch, policy_dev, value_dev, stream=None):
+    """(positions, legal_masks) -> (policy, value), written into the caller's device tensors."""
+    _check(_lib.az_evaluate(net.handle, _dev_ptr(positions_dev, "positions"), _dev_ptr(legal_masks_dev, "legal_masks"),
+                            batch, _dev_ptr(policy_dev, "policy"), _dev_ptr(value_dev, "value"), _stream_ptr(stream)),
+           "az_evaluate")
+
+
+def az_encode(net: Net, positions_dev, batch, planes_dev, stream=None):
+    _check(_lib.az_encode(net.handle, _dev_ptr(positions_dev, "positions"), batch, _dev_ptr(planes_dev, "planes"),
+                          _stream_ptr(stream)), "az_encode")
+
+
+def az_tower(net: Net, positions_dev, batch, tower_dev, stream=None):
+    _check(_lib.az_tower(net.handle, _dev_ptr(positions_dev, "positions"), batch, _dev_ptr(tower_dev, "tower"),
+                         _stream_ptr(stream)), "az_tower")
+
+
+def az_legal_masks(positions_dev, position_stride, batch, policy_head, masks_dev, stream=None):
+    _check(_lib.az_legal_masks(_dev_ptr(positions_dev, "positions"), position_stride, batch, policy_head,
+                               _dev_ptr(masks_dev, "masks"), _stream_ptr(stream)), "az_legal_masks")
+
+
+def az_calibrate(net: Net, positions_dev, n, stream=None):
+    _check(_lib.az_calibrate(net.handle, _dev_ptr(positions_dev, "positions"), n, _stream_ptr(stream)), "az_calibrate")
+
+
+def az_device_status(net: Net, stream=None) -> int:
+    status = ctypes.c_uint32(0)
+    code = _lib.az_device_status(net.handle, _stream_ptr(stream), ctypes.byref(status))
+    if code not in (AZ_OK, AZ_ERR_DEVICE_TIMEOUT):
+        raise AzError(code, "az_device_status")
+    return int(status.value)
+
+
+def az_launches_per_evaluate(net: Net, batch: int) -> int:
+    return int(_lib.az_launches_per_evaluate(net.handle, batch))
+
+
+def az_strerror(code: int) -> str:
+    return _lib.az_strerror(code).decode()
+
+
+def az_last_cuda_error() -> str:
+    return _lib.az_last_cuda_error().decode()
+
+
+# ---- small marshalling helpers used by tests and the benchmark ----------------------------------
+
+def records_to_device(records: np.ndarray, device="cuda") -> torch.Tensor:
+    """A numpy record array (104- or 784-byte records) as a uint8 device tensor [n][record_bytes]."""
+    raw = np.ascontiguousarray(records).view(np.uint8).reshape(records.shape[0], -1)
+    return torch.from_numpy(raw.copy()).to(device)
+
+
+def masks_to_numpy(masks_dev: torch.Tensor) -> np.ndarray:
+    return masks_dev.cpu().numpy().view(np.uint64)

@@ -1,0 +1,380 @@
+// The C ABI of az_eval: argument checks, weight-blob parsing and repacking, workspace ownership,
+// and the sequence of kernel launches that makes up one evaluation.
+#include "common.cuh"
+
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+namespace az {
+
+static thread_local std::string g_cuda_error;
+
+void set_cuda_error(cudaError_t e, const char *what) {
+    g_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+}
+
+namespace {
+
+constexpr size_t kHeaderBytes = 64;
+
+struct BlobView {                       // float32 tensors of the blob, in file order
+    const float *in_w, *in_s, *in_b;
+    std::vector<const float *> w1, s1, b1, w2, s2, b2;
+    const float *p_w, *p_s, *p_b, *p_fw, *p_fb;
+    const float *v_cw, *v_cs, *v_cb, *v_w1, *v_b1, *v_w2, *v_b2;
+};
+
+bool arch_ok(const az_arch &a) {
+    if (a.abi_version != AZ_ABI_VERSION) return false;
+    if (a.in_planes != 19 && a.in_planes != 112) return false;
+    if (a.blocks > 64 || a.channels < 8 || a.channels > 512 || a.channels % 8) return false;
+    if (a.policy_head > 1 || a.value_head > 1 || a.precision > 2) return false;
+    if (a.max_batch == 0 || a.max_batch > (1u << 20)) return false;
+    return true;
+}
+
+int parse_blob(const az_arch &a, const unsigned char *blob, size_t nbytes, BlobView &v) {
+    if (nbytes < kHeaderBytes || memcmp(blob, "AZNETv1", 8) != 0) return AZ_ERR_BAD_WEIGHTS;
+    uint32_t h[7];
+    memcpy(h, blob + 8, sizeof h);
+    if (h[0] != 1 || h[1] != a.in_planes || h[2] != a.blocks || h[3] != a.channels ||
+        h[4] != a.policy_head || h[5] != a.value_head)
+        return AZ_ERR_BAD_WEIGHTS;
+    const size_t C = a.channels, P = a.in_planes, L = a.blocks;
+    const size_t V = a.value_head == AZ_VALUE_WDL ? 3 : 1;
+    size_t need = C * P * 9 + 2 * C + L * (2 * C * C * 9 + 4 * C);
+    need += a.policy_head == AZ_POLICY_PLANES73 ? (size_t)kPlanes73 * C + kPlanes73
+                                                : (size_t)kHeadChannels * C + 2 * kHeadChannels +
+                                                      (size_t)kFlatMoves * kHeadChannels * 64 + kFlatMoves;
+    need += (size_t)kHeadChannels * C + 2 * kHeadChannels + (size_t)kValueHidden * kHeadChannels * 64 +
+            kValueHidden + V * kValueHidden + V;
+    if (nbytes != kHeaderBytes + 4 * need) return AZ_ERR_BAD_WEIGHTS;
+    const float *p = reinterpret_cast<const float *>(blob + kHeaderBytes);
+    for (size_t i = 0; i < need; ++i)
+        if (!std::isfinite(p[i])) return AZ_ERR_BAD_WEIGHTS;
+    auto take = [&p](size_t n) { const float *q = p; p += n; return q; };
+    v.in_w = take(C * P * 9); v.in_s = take(C); v.in_b = take(C);
+    for (size_t b = 0; b < L; ++b) {
+        v.w1.push_back(take(C * C * 9)); v.s1.push_back(take(C)); v.b1.push_back(take(C));
+        v.w2.push_back(take(C * C * 9)); v.s2.push_back(take(C)); v.b2.push_back(take(C));
+    }
+    v.p_s = v.p_fw = v.p_fb = nullptr;
+    if (a.policy_head == AZ_POLICY_PLANES73) { v.p_w = take((size_t)kPlanes73 * C); v.p_b = take(kPlanes73); }
+    else {
+        v.p_w = take((size_t)kHeadChannels * C); v.p_s = take(kHeadChannels); v.p_b = take(kHeadChannels);
+        v.p_fw = take((size_t)kFlatMoves * kHeadChannels * 64); v.p_fb = take(kFlatMoves);
+    }
+    v.v_cw = take((size_t)kHeadChannels * C); v.v_cs = take(kHeadChannels); v.v_cb = take(kHeadChannels);
+    v.v_w1 = take((size_t)kValueHidden * kHeadChannels * 64); v.v_b1 = take(kValueHidden);
+    v.v_w2 = take(V * kValueHidden); v.v_b2 = take(V);
+    return AZ_OK;
+}
+
+// host float32 -> device buffer of the activation type (float32 or bfloat16, round to nearest even)
+int upload_act(const float *src, size_t n, bool bf16, void **dst) {
+    if (bf16) {
+        std::vector<__nv_bfloat16> tmp(n);
+        for (size_t i = 0; i < n; ++i) tmp[i] = __float2bfloat16_rn(src[i]);
+        AZ_CUDA(cudaMalloc(dst, n * sizeof(__nv_bfloat16)));
+        AZ_CUDA(cudaMemcpy(*dst, tmp.data(), n * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
+    } else {
+        AZ_CUDA(cudaMalloc(dst, n * sizeof(float)));
+        AZ_CUDA(cudaMemcpy(*dst, src, n * sizeof(float), cudaMemcpyHostToDevice));
+    }
+    return AZ_OK;
+}
+int upload_f32(const float *src, size_t n, float **dst) {
+    AZ_CUDA(cudaMalloc((void **)dst, n * sizeof(float)));
+    AZ_CUDA(cudaMemcpy(*dst, src, n * sizeof(float), cudaMemcpyHostToDevice));
+    return AZ_OK;
+}
+
+// [cout][cin][3][3] -> [tap][cin_pad][cout], zero rows for padded input channels
+int upload_conv_simt(const float *w, int cin, int cin_pad, int cout, bool bf16, void **dst) {
+    std::vector<float> t((size_t)9 * cin_pad * cout, 0.0f);
+    for (int co = 0; co < cout; ++co)
+        for (int ci = 0; ci < cin; ++ci)
+            for (int tap = 0; tap < 9; ++tap)
+                t[((size_t)tap * cin_pad + ci) * cout + co] = w[((size_t)co * cin + ci) * 9 + tap];
+    return upload_act(t.data(), t.size(), bf16, dst);
+}
+
+size_t act_bytes(const Net &n) { return n.bf16 ? 2 : 4; }
+
+int alloc_simt_buffers(Net &n) {
+    const size_t bytes = (size_t)n.arch.max_batch * 64 * n.arch.channels * act_bytes(n);
+    for (int i = 1; i < 3; ++i)
+        if (!n.act[i]) AZ_CUDA(cudaMalloc(&n.act[i], bytes));
+    return AZ_OK;
+}
+
+bool want_simt_tower() {
+    const char *e = getenv("AZ_EVAL_TOWER");
+    return e && strcmp(e, "simt") == 0;
+}
+
+int build_net(Net &n, const BlobView &v) {
+    const az_arch &a = n.arch;
+    const int C = (int)a.channels, L = (int)a.blocks;
+    n.bf16 = a.precision != AZ_PREC_FP32;
+    n.in_pad = a.in_planes == 19 ? 32 : 128;
+    n.n_conv = 1 + 2 * L;
+    int rc;
+
+    // tensor-core tower: bf16, 128 channels, 19-plane input
+    const bool tc_shape = a.precision == AZ_PREC_BF16 && C == 128 && n.in_pad == 32;
+    if (tc_shape && !want_simt_tower()) {
+        std::vector<const float *> w, s, b;
+        w.push_back(v.in_w); s.push_back(v.in_s); b.push_back(v.in_b);
+        for (int i = 0; i < L; ++i) {
+            w.push_back(v.w1[i]); s.push_back(v.s1[i]); b.push_back(v.b1[i]);
+            w.push_back(v.w2[i]); s.push_back(v.s2[i]); b.push_back(v.b2[i]);
+        }
+        const size_t bytes = tc_packed_weight_bytes(n.in_pad, C, n.n_conv);
+        std::vector<__nv_bfloat16> packed(bytes / sizeof(__nv_bfloat16));
+        tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, packed.data());
+        AZ_CUDA(cudaMalloc(&n.tc_weights, bytes));
+        AZ_CUDA(cudaMemcpy(n.tc_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
+        std::vector<float> bias((size_t)n.n_conv * C);
+        for (int l = 0; l < n.n_conv; ++l) memcpy(&bias[(size_t)l * C], b[l], sizeof(float) * C);
+        if ((rc = upload_f32(bias.data(), bias.size(), &n.tc_bias)) != AZ_OK) return rc;
+        n.tc_ready = true;
+    } else {
+        if ((rc = upload_conv_simt(v.in_w, (int)a.in_planes, n.in_pad, C, n.bf16, &n.conv_w[0])) != AZ_OK) return rc;
+        if ((rc = upload_f32(v.in_s, C, &n.conv_scale[0])) != AZ_OK) return rc;
+        if ((rc = upload_f32(v.in_b, C, &n.conv_bias[0])) != AZ_OK) return rc;
+        for (int i = 0; i < L; ++i) {
+            const int l1 = 1 + 2 * i, l2 = 2 + 2 * i;
+            if ((rc = upload_conv_simt(v.w1[i], C, C, C, n.bf16, &n.conv_w[l1])) != AZ_OK) return rc;
+            if ((rc = upload_f32(v.s1[i], C, &n.conv_scale[l1])) != AZ_OK) return rc;
+            if ((rc = upload_f32(v.b1[i], C, &n.conv_bias[l1])) != AZ_OK) return rc;
+            if ((rc = upload_conv_simt(v.w2[i], C, C, C, n.bf16, &n.conv_w[l2])) != AZ_OK) return rc;
+            if ((rc = upload_f32(v.s2[i], C, &n.conv_scale[l2])) != AZ_OK) return rc;
+            if ((rc = upload_f32(v.b2[i], C, &n.conv_bias[l2])) != AZ_OK) return rc;
+        }
+        if ((rc = alloc_simt_buffers(n)) != AZ_OK) return rc;
+    }
+
+    // heads
+    const int V = a.value_head == AZ_VALUE_WDL ? 3 : 1;
+    if (a.policy_head == AZ_POLICY_PLANES73) {
+        if ((rc = upload_act(v.p_w, (size_t)kPlanes73 * C, n.bf16, &n.p_w)) != AZ_OK) return rc;
+        if ((rc = upload_f32(v.p_b, kPlanes73, &n.p_bias)) != AZ_OK) return rc;
+    } else {
+        if ((rc = upload_act(v.p_w, (size_t)kHeadChannels * C, n.bf16, &n.p_w)) != AZ_OK) return rc;
+        if ((rc = upload_f32(v.p_s, kHeadChannels, &n.p_scale)) != AZ_OK) return rc;
+        if ((rc = upload_f32(v.p_b, kHeadChannels, &n.p_bias)) != AZ_OK) return rc;
+        if ((rc = upload_act(v.p_fw, (size_t)kFlatMoves * kHeadChannels * 64, n.bf16, &n.p_fw)) != AZ_OK) return rc;
+        if ((rc = upload_f32(v.p_fb, kFlatMoves, &n.p_fbias)) != AZ_OK) return rc;
+    }
+    if ((rc = upload_act(v.v_cw, (size_t)kHeadChannels * C, n.bf16, &n.v_cw)) != AZ_OK) return rc;
+    if ((rc = upload_f32(v.v_cs, kHeadChannels, &n.v_cscale)) != AZ_OK) return rc;
+    if ((rc = upload_f32(v.v_cb, kHeadChannels, &n.v_cbias)) != AZ_OK) return rc;
+    if ((rc = upload_act(v.v_w1, (size_t)kValueHidden * kHeadChannels * 64, n.bf16, &n.v_w1)) != AZ_OK) return rc;
+    if ((rc = upload_f32(v.v_b1, kValueHidden, &n.v_b1)) != AZ_OK) return rc;
+    if ((rc = upload_f32(v.v_w2, (size_t)V * kValueHidden, &n.v_w2)) != AZ_OK) return rc;
+    if ((rc = upload_f32(v.v_b2, V, &n.v_b2)) != AZ_OK) return rc;
+
+    // workspace
+    const size_t B = a.max_batch;
+    AZ_CUDA(cudaMalloc(&n.planes, B * 64 * n.in_pad * act_bytes(n)));
+    AZ_CUDA(cudaMalloc(&n.act[0], B * 64 * C * act_bytes(n)));
+    AZ_CUDA(cudaMalloc((void **)&n.logits, B * az_policy_size(&a) * sizeof(float)));
+    AZ_CUDA(cudaMalloc(&n.head_p, B * kHeadChannels * 64 * act_bytes(n)));
+    AZ_CUDA(cudaMalloc(&n.head_v, B * kHeadChannels * 64 * act_bytes(n)));
+    AZ_CUDA(cudaMalloc((void **)&n.hidden, B * kValueHidden * sizeof(float)));
+    AZ_CUDA(cudaMalloc((void **)&n.status_dev, sizeof(uint32_t)));
+    AZ_CUDA(cudaMemset(n.status_dev, 0, sizeof(uint32_t)));
+    return AZ_OK;
+}
+
+void free_net(Net *n) {
+    if (!n) return;
+    for (int i = 0; i < 1 + 2 * 64; ++i) { cudaFree(n->conv_w[i]); cudaFree(n->conv_scale[i]); cudaFree(n->conv_bias[i]); }
+    cudaFree(n->tc_weights); cudaFree(n->tc_bias);
+    cudaFree(n->p_w); cudaFree(n->p_scale); cudaFree(n->p_bias); cudaFree(n->p_fw); cudaFree(n->p_fbias);
+    cudaFree(n->v_cw); cudaFree(n->v_cscale); cudaFree(n->v_cbias); cudaFree(n->v_w1); cudaFree(n->v_b1);
+    cudaFree(n->v_w2); cudaFree(n->v_b2);
+    cudaFree(n->planes);
+    for (int i = 0; i < 3; ++i) cudaFree(n->act[i]);
+    cudaFree(n->logits); cudaFree(n->head_p); cudaFree(n->head_v); cudaFree(n->hidden); cudaFree(n->status_dev);
+    delete n;
+}
+
+// encoder + tower; *tower_out receives the buffer holding [batch][64][C]
+int run_tower(Net &n, const void *positions, int batch, void **tower_out, cudaStream_t s) {
+    int rc = launch_encode(positions, az_position_bytes(&n.arch), batch, (int)n.arch.in_planes, n.in_pad,
+                           n.bf16, n.planes, n.status_dev, s);
+    if (rc != AZ_OK) return rc;
+    const int C = (int)n.arch.channels;
+    if (n.tc_ready) {
+        *tower_out = n.act[0];
+        return launch_tower_tc(n, n.planes, batch, n.act[0], s);
+    }
+    void *x = n.act[0], *t = n.act[1], *y = n.act[2];
+    rc = launch_conv3x3_simt(n.planes, n.conv_w[0], n.conv_scale[0], n.conv_bias[0], nullptr, x, batch,
+                             n.in_pad, C, n.bf16, s);
+    if (rc != AZ_OK) return rc;
+    for (int b = 0; b < (int)n.arch.blocks; ++b) {
+        const int l1 = 1 + 2 * b, l2 = 2 + 2 * b;
+        rc = launch_conv3x3_simt(x, n.conv_w[l1], n.conv_scale[l1], n.conv_bias[l1], nullptr, t, batch, C, C, n.bf16, s);
+        if (rc != AZ_OK) return rc;
+        rc = launch_conv3x3_simt(t, n.conv_w[l2], n.conv_scale[l2], n.conv_bias[l2], x, y, batch, C, C, n.bf16, s);
+        if (rc != AZ_OK) return rc;
+        void *tmp = x; x = y; y = tmp;
+    }
+    *tower_out = x;
+    return AZ_OK;
+}
+
+}  // namespace
+}  // namespace az
+
+using az::Net;
+
+extern "C" {
+
+size_t az_position_bytes(const az_arch *a) { return a && a->in_planes == 112 ? sizeof(az_position_h8) : sizeof(az_position); }
+size_t az_policy_size(const az_arch *a) { return a && a->policy_head == AZ_POLICY_FLAT1858 ? az::kFlatMoves : az::kPlanes73 * 64; }
+size_t az_mask_words(const az_arch *a) { return a && a->policy_head == AZ_POLICY_FLAT1858 ? 30 : 73; }
+size_t az_value_size(const az_arch *a) { return a && a->value_head == AZ_VALUE_WDL ? 3 : 1; }
+size_t az_plane_channels(const az_arch *a) { return a && a->in_planes == 112 ? 128 : 32; }
+
+int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az_net **out) {
+    static_assert(sizeof(az_position) == 104 && sizeof(az_position_h8) == 784, "record layout");
+    if (!arch || !weights_host || !out) return AZ_ERR_BAD_ARG;
+    *out = nullptr;
+    if (!az::arch_ok(*arch)) return AZ_ERR_BAD_ARCH;
+    if (arch->precision == AZ_PREC_FP8_E4M3) return AZ_ERR_UNSUPPORTED;
+    az::BlobView view;
+    int rc = az::parse_blob(*arch, static_cast<const unsigned char *>(weights_host), nbytes, view);
+    if (rc != AZ_OK) return rc;
+    Net *n = new (std::nothrow) Net();
+    if (!n) return AZ_ERR_BAD_ARG;
+    n->arch = *arch;
+    cudaError_t e = cudaGetDevice(&n->device);
+    if (e != cudaSuccess) { az::set_cuda_error(e, "cudaGetDevice"); delete n; return AZ_ERR_CUDA; }
+    rc = az::build_net(*n, view);
+    if (rc != AZ_OK) { az::free_net(n); return rc; }
+    *out = reinterpret_cast<az_net *>(n);
+    return AZ_OK;
+}
+
+void az_free_net(az_net *net) { az::free_net(reinterpret_cast<Net *>(net)); }
+
+int az_encode(az_net *net, const void *positions_dev, int batch, void *planes_dev, void *cuda_stream) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n || batch < 0 || (batch > 0 && (!positions_dev || !planes_dev))) return AZ_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(positions_dev) & 7) || (reinterpret_cast<uintptr_t>(planes_dev) & 15)) return AZ_ERR_BAD_ARG;
+    if ((uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
+    return az::launch_encode(positions_dev, az_position_bytes(&n->arch), batch, (int)n->arch.in_planes,
+                             n->in_pad, n->bf16, planes_dev, n->status_dev, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int az_tower(az_net *net, const void *positions_dev, int batch, void *tower_dev, void *cuda_stream) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n || batch < 0 || (batch > 0 && (!positions_dev || !tower_dev))) return AZ_ERR_BAD_ARG;
+    if (reinterpret_cast<uintptr_t>(positions_dev) & 7) return AZ_ERR_BAD_ARG;
+    if ((uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
+    if (batch == 0) return AZ_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    void *x = nullptr;
+    int rc = az::run_tower(*n, positions_dev, batch, &x, s);
+    if (rc != AZ_OK) return rc;
+    AZ_CUDA(cudaMemcpyAsync(tower_dev, x, (size_t)batch * 64 * n->arch.channels * az::act_bytes(*n),
+                            cudaMemcpyDeviceToDevice, s));
+    return AZ_OK;
+}
+
+int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_masks_dev, int batch,
+                float *policy_dev, float *value_dev, void *cuda_stream) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n || batch < 0) return AZ_ERR_BAD_ARG;
+    if (batch == 0) return AZ_OK;
+    if (!positions_dev || !legal_masks_dev || !policy_dev || !value_dev) return AZ_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(positions_dev) & 7) || (reinterpret_cast<uintptr_t>(legal_masks_dev) & 7) ||
+        (reinterpret_cast<uintptr_t>(policy_dev) & 3) || (reinterpret_cast<uintptr_t>(value_dev) & 3))
+        return AZ_ERR_BAD_ARG;
+    if ((uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const az_arch &a = n->arch;
+    const int C = (int)a.channels;
+    void *h = nullptr;
+    int rc = az::run_tower(*n, positions_dev, batch, &h, s);
+    if (rc != AZ_OK) return rc;
+    if (a.policy_head == AZ_POLICY_PLANES73) {
+        rc = az::launch_conv1x1(h, n->p_w, nullptr, n->p_bias, batch, C, az::kPlanes73, false, n->bf16, n->logits, true, s);
+        if (rc != AZ_OK) return rc;
+    } else {
+        rc = az::launch_conv1x1(h, n->p_w, n->p_scale, n->p_bias, batch, C, az::kHeadChannels, true, n->bf16, n->head_p, !n->bf16, s);
+        if (rc != AZ_OK) return rc;
+        rc = az::launch_fc(n->head_p, n->p_fw, n->p_fbias, batch, az::kFlatMoves, az::kHeadChannels * 64, false, n->bf16, n->logits, true, s);
+        if (rc != AZ_OK) return rc;
+    }
+    rc = az::launch_conv1x1(h, n->v_cw, n->v_cscale, n->v_cbias, batch, C, az::kHeadChannels, true, n->bf16, n->head_v, !n->bf16, s);
+    if (rc != AZ_OK) return rc;
+    rc = az::launch_fc(n->head_v, n->v_w1, n->v_b1, batch, az::kValueHidden, az::kHeadChannels * 64, true, n->bf16, n->hidden, true, s);
+    if (rc != AZ_OK) return rc;
+    rc = az::launch_value_tail(n->hidden, n->v_w2, n->v_b2, batch, a.value_head == AZ_VALUE_WDL, value_dev, s);
+    if (rc != AZ_OK) return rc;
+    return az::launch_masked_softmax(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a), (int)az_mask_words(&a),
+                                     policy_dev, n->status_dev, s);
+}
+
+int az_legal_masks(const void *positions_dev, size_t position_stride, int batch, int policy_head,
+                   uint64_t *masks_dev, void *cuda_stream) {
+    if (batch < 0 || (policy_head != AZ_POLICY_PLANES73 && policy_head != AZ_POLICY_FLAT1858)) return AZ_ERR_BAD_ARG;
+    if (batch == 0) return AZ_OK;
+    if (!positions_dev || !masks_dev || position_stride < sizeof(az_position) || (position_stride & 7)) return AZ_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(positions_dev) & 7) || (reinterpret_cast<uintptr_t>(masks_dev) & 7)) return AZ_ERR_BAD_ARG;
+    return az::launch_legal_masks(positions_dev, position_stride, batch, policy_head, masks_dev,
+                                  static_cast<cudaStream_t>(cuda_stream));
+}
+
+int az_calibrate(az_net *net, const void *positions_dev, int n, void *cuda_stream) {
+    (void)positions_dev; (void)n; (void)cuda_stream;
+    if (!net) return AZ_ERR_BAD_ARG;
+    return AZ_ERR_UNSUPPORTED;
+}
+
+int az_device_status(az_net *net, void *cuda_stream, uint32_t *status_out) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n || !status_out) return AZ_ERR_BAD_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    AZ_CUDA(cudaMemcpyAsync(status_out, n->status_dev, sizeof(uint32_t), cudaMemcpyDeviceToHost, s));
+    AZ_CUDA(cudaMemsetAsync(n->status_dev, 0, sizeof(uint32_t), s));
+    AZ_CUDA(cudaStreamSynchronize(s));
+    return (*status_out & az::kStatusWaitTimeout) ? AZ_ERR_DEVICE_TIMEOUT : AZ_OK;
+}
+
+int az_launches_per_evaluate(const az_net *net, int batch) {
+    const Net *n = reinterpret_cast<const Net *>(net);
+    if (!n || batch <= 0) return 0;
+    const int tower = n->tc_ready ? az::tower_tc_launch_count() : n->n_conv;
+    const int policy = n->arch.policy_head == AZ_POLICY_PLANES73 ? 1 : 2;
+    return 1 /*encode*/ + tower + policy + 3 /*value*/ + 1 /*softmax*/;
+}
+
+const char *az_strerror(int code) {
+    switch (code) {
+        case AZ_OK: return "ok";
+        case AZ_ERR_BAD_ARG: return "bad argument";
+        case AZ_ERR_BAD_ARCH: return "unsupported network shape";
+        case AZ_ERR_BAD_WEIGHTS: return "malformed weight blob";
+        case AZ_ERR_BATCH_TOO_LARGE: return "batch exceeds max_batch";
+        case AZ_ERR_CUDA: return "CUDA runtime error";
+        case AZ_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+        case AZ_ERR_NOT_CALIBRATED: return "FP8 network not calibrated";
+        case AZ_ERR_UNSUPPORTED: return "not supported by this build";
+        default: return "unknown error";
+    }
+}
+
+const char *az_last_cuda_error(void) { return az::g_cuda_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,106 @@
+// Shared declarations of the az_eval library: the network object, error plumbing and the
+// launch functions each .cu file exports to api.cu.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "az_eval.h"
+
+namespace az {
+
+constexpr int kHeadChannels = 32;     // width of the 1x1 projections of the flat policy head and the value head
+constexpr int kValueHidden = 128;
+constexpr int kFlatMoves = 1858;
+constexpr int kPlanes73 = 73;
+
+// Device-side status bits (OR-ed into az_net::status_dev by kernels).
+enum : uint32_t {
+    kStatusEmptyMask = 1u << 0,       // a position had no legal move: all-zero policy row
+    kStatusWaitTimeout = 1u << 1,     // a bounded mbarrier wait ran out
+    kStatusBadRecord = 1u << 2,       // a position record without exactly one king per side
+};
+
+struct ConvLayerF32 {                 // fp32 path: weights [tap][cin][cout], folded scale / bias
+    float *w = nullptr, *scale = nullptr, *bias = nullptr;
+    int cin = 0, cout = 0;
+};
+
+struct Net {
+    az_arch arch{};
+    int device = 0;
+    int in_pad = 0;                   // channels of the encoded plane tensor (32 or 128)
+    int n_conv = 0;                   // 1 + 2*blocks
+    bool bf16 = false;                // activations stored as bf16 (true for BF16 and FP8 nets)
+
+    // ---- generic (SIMT) path: every conv as [tap][cin_pad][cout] in the activation type ----
+    void *conv_w[1 + 2 * 64] = {};    // element type = activation type
+    float *conv_scale[1 + 2 * 64] = {};
+    float *conv_bias[1 + 2 * 64] = {};
+
+    // ---- tensor-core tower (bf16, channels == 128) ----
+    void *tc_weights = nullptr;       // packed UMMA B-operand tiles, all layers
+    float *tc_bias = nullptr;         // [n_conv][C] folded bias (scales are folded into the weights)
+    bool tc_ready = false;
+
+    // ---- heads ----
+    void *p_w = nullptr;              // planes73: [73][C]; flat: 1x1 conv [32][C]      (activation type)
+    float *p_scale = nullptr, *p_bias = nullptr;
+    void *p_fw = nullptr;             // flat: [1858][2048] (activation type)
+    float *p_fbias = nullptr;
+    void *v_cw = nullptr;             // [32][C]
+    float *v_cscale = nullptr, *v_cbias = nullptr;
+    void *v_w1 = nullptr;             // [128][2048]
+    float *v_b1 = nullptr;
+    float *v_w2 = nullptr, *v_b2 = nullptr;   // [V][128], [V] fp32
+
+    // ---- workspace (sized for max_batch) ----
+    void *planes = nullptr;           // [B][64][in_pad]
+    void *act[3] = {};                // [B][64][C] x3 (SIMT tower ping-pong; act[0] doubles as tower output)
+    float *logits = nullptr;          // [B][policy_size]
+    void *head_p = nullptr;           // [B][2048] flat-policy projection (activation type)
+    void *head_v = nullptr;           // [B][2048] value projection
+    float *hidden = nullptr;          // [B][128]
+    uint32_t *status_dev = nullptr;
+};
+
+// ---- error plumbing ------------------------------------------------------------------------
+void set_cuda_error(cudaError_t e, const char *what);
+#define AZ_CUDA(call)                                                     \
+    do {                                                                  \
+        cudaError_t e__ = (call);                                         \
+        if (e__ != cudaSuccess) { az::set_cuda_error(e__, #call); return AZ_ERR_CUDA; } \
+    } while (0)
+#define AZ_LAUNCH_CHECK()                                                 \
+    do {                                                                  \
+        cudaError_t e__ = cudaGetLastError();                             \
+        if (e__ != cudaSuccess) { az::set_cuda_error(e__, "kernel launch"); return AZ_ERR_CUDA; } \
+    } while (0)
+
+// ---- kernels' launch functions (each returns AZ_OK or AZ_ERR_CUDA) ---------------------------
+int launch_encode(const void *positions, size_t stride, int batch, int in_planes, int in_pad,
+                  bool bf16, void *planes, uint32_t *status, cudaStream_t s);
+int launch_legal_masks(const void *positions, size_t stride, int batch, int head, uint64_t *masks,
+                       cudaStream_t s);
+int launch_conv3x3_simt(const void *in, const void *w, const float *scale, const float *bias,
+                        const void *residual, void *out, int batch, int cin, int cout, bool bf16,
+                        cudaStream_t s);
+int launch_conv1x1(const void *in, const void *w, const float *scale, const float *bias, int batch,
+                   int cin, int cout, bool relu, bool bf16_in, void *out, bool out_f32, cudaStream_t s);
+int launch_fc(const void *a, const void *w, const float *bias, int m, int n, int k, bool relu,
+              bool bf16_in, void *out, bool out_f32, cudaStream_t s);
+int launch_value_tail(const float *hidden, const float *w2, const float *b2, int batch, int wdl,
+                      float *value, cudaStream_t s);
+int launch_masked_softmax(const float *logits, const uint64_t *masks, int batch, int n, int words,
+                          float *policy, uint32_t *status, cudaStream_t s);
+
+// tensor-core tower (tower_tc.cu)
+size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv);
+void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
+                     int channels, int n_conv, __nv_bfloat16 *packed_host);
+int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, cudaStream_t s);
+int tower_tc_launch_count();
+
+}  // namespace az

@@ -1,0 +1,262 @@
+// Legal-move masks on the GPU (App. D.1: illegal actions are masked before the softmax; castling
+// is the king-to-own-rook pair, en passant the pawn's ordinary origin-destination pair).
+//
+// Bitboard move generation, one thread per position: pseudo-legal target sets per piece from
+// shift/ray arithmetic, each move tried on a copy of the bitboards and kept if the mover's king
+// is not attacked afterwards.  The mask row is built in registers/local memory and written once.
+// The work per position is a few thousand integer operations; the kernel is latency-bound and
+// runs off the timed path (masks are an input of az_evaluate).
+#include "common.cuh"
+
+#include <mutex>
+
+namespace az {
+namespace {
+
+typedef unsigned long long u64;
+
+constexpr u64 FILE_A = 0x0101010101010101ull;
+constexpr u64 FILE_B = FILE_A << 1;
+constexpr u64 FILE_G = FILE_A << 6;
+constexpr u64 FILE_H = FILE_A << 7;
+
+// flat-1858 index tables, built on the host once per device
+__device__ short g_flat_pair[64 * 64];
+__device__ short g_flat_promo[8 * 3];
+
+struct alignas(8) PosCur {
+    u64 pieces[12];
+    unsigned char stm, castling, ep_square, halfmove, repetitions, pad[3];
+};
+
+__device__ __forceinline__ u64 knight_set(u64 b) {
+    return ((b << 17) & ~FILE_A) | ((b << 15) & ~FILE_H) | ((b << 10) & ~(FILE_A | FILE_B)) |
+           ((b << 6) & ~(FILE_G | FILE_H)) | ((b >> 17) & ~FILE_H) | ((b >> 15) & ~FILE_A) |
+           ((b >> 10) & ~(FILE_G | FILE_H)) | ((b >> 6) & ~(FILE_A | FILE_B));
+}
+__device__ __forceinline__ u64 king_set(u64 b) {
+    return ((b << 1) & ~FILE_A) | ((b >> 1) & ~FILE_H) | (b << 8) | (b >> 8) | ((b << 9) & ~FILE_A) |
+           ((b << 7) & ~FILE_H) | ((b >> 7) & ~FILE_A) | ((b >> 9) & ~FILE_H);
+}
+// squares seen from sq along the four diagonal (diag) or four straight lines, stopping at (and
+// including) the first occupied square
+__device__ u64 ray_set(int sq, u64 occ, bool diag) {
+    u64 att = 0;
+#pragma unroll
+    for (int d = 0; d < 4; ++d) {
+        const int df = diag ? ((d & 1) ? -1 : 1) : (d == 0 ? 1 : d == 1 ? -1 : 0);
+        const int dr = diag ? ((d & 2) ? -1 : 1) : (d == 2 ? 1 : d == 3 ? -1 : 0);
+        int f = (sq & 7) + df, r = (sq >> 3) + dr;
+        while (f >= 0 && f < 8 && r >= 0 && r < 8) {
+            const u64 b = 1ull << (r * 8 + f);
+            att |= b;
+            if (occ & b) break;
+            f += df; r += dr;
+        }
+    }
+    return att;
+}
+// is `sq` attacked by side `by` (0 white, 1 black), given that side's bitboards bb[6] and the occupancy
+__device__ bool attacked(int sq, int by, const u64 *bb, u64 occ) {
+    const u64 b = 1ull << sq;
+    const u64 pawn_src = by == 0 ? (((b >> 9) & ~FILE_H) | ((b >> 7) & ~FILE_A))
+                                 : (((b << 9) & ~FILE_A) | ((b << 7) & ~FILE_H));
+    if (pawn_src & bb[0]) return true;
+    if (knight_set(b) & bb[1]) return true;
+    if (king_set(b) & bb[5]) return true;
+    if (ray_set(sq, occ, true) & (bb[2] | bb[4])) return true;
+    if (ray_set(sq, occ, false) & (bb[3] | bb[4])) return true;
+    return false;
+}
+
+template <int HEAD>
+__device__ __forceinline__ void set_move(u64 *row, int stm, int from, int to, int promo) {
+    // mover-oriented coordinates: reflect ranks for Black
+    if (stm) { from ^= 56; to ^= 56; }
+    int idx;
+    if (HEAD == AZ_POLICY_PLANES73) {
+        const int df = (to & 7) - (from & 7), dr = (to >> 3) - (from >> 3);
+        int plane;
+        if (promo) {                                     // under-promotion: 1 N, 2 B, 3 R
+            plane = 64 + 3 * (promo - 1) + (df + 1);
+        } else {
+            const int adf = df < 0 ? -df : df, adr = dr < 0 ? -dr : dr;
+            if (adf != adr && adf != 0 && adr != 0) {     // knight jump
+                // (1,2)=0 (2,1)=1 (2,-1)=2 (1,-2)=3 (-1,-2)=4 (-2,-1)=5 (-2,1)=6 (-1,2)=7
+                const int k = df > 0 ? (dr > 0 ? (adf == 1 ? 0 : 1) : (adf == 2 ? 2 : 3))
+                                     : (dr < 0 ? (adf == 1 ? 4 : 5) : (adf == 2 ? 6 : 7));
+                plane = 56 + k;
+            } else {
+                // N=0 NE=1 E=2 SE=3 S=4 SW=5 W=6 NW=7
+                const int d = df == 0 ? (dr > 0 ? 0 : 4)
+                            : df > 0 ? (dr > 0 ? 1 : dr == 0 ? 2 : 3)
+                                     : (dr < 0 ? 5 : dr == 0 ? 6 : 7);
+                plane = 7 * d + (adf > adr ? adf : adr) - 1;
+            }
+        }
+        idx = plane * 64 + from;
+    } else {
+        idx = promo ? g_flat_promo[(from & 7) * 3 + ((to & 7) - (from & 7) + 1)] + (promo - 1)
+                    : g_flat_pair[from * 64 + to];
+    }
+    row[idx >> 6] |= 1ull << (idx & 63);
+}
+
+template <int HEAD>
+__global__ void __launch_bounds__(64)
+legal_masks_kernel(const unsigned char *__restrict__ positions, size_t stride, int batch,
+                   u64 *__restrict__ masks) {
+    constexpr int WORDS = HEAD == AZ_POLICY_PLANES73 ? 73 : 30;
+    const int pos = blockIdx.x * blockDim.x + threadIdx.x;
+    if (pos >= batch) return;
+    const PosCur *r = reinterpret_cast<const PosCur *>(positions + (size_t)pos * stride);
+    u64 own[6], opp[6];
+    const int stm = r->stm & 1;
+#pragma unroll
+    for (int k = 0; k < 6; ++k) { own[k] = r->pieces[stm * 6 + k]; opp[k] = r->pieces[(stm ^ 1) * 6 + k]; }
+    u64 own_occ = 0, opp_occ = 0;
+#pragma unroll
+    for (int k = 0; k < 6; ++k) { own_occ |= own[k]; opp_occ |= opp[k]; }
+    const u64 occ = own_occ | opp_occ;
+    const int them = stm ^ 1;
+    const int king_sq = own[5] ? __ffsll((long long)own[5]) - 1 : 0;
+    const int ep = r->ep_square;
+
+    u64 row[WORDS];
+#pragma unroll 1
+    for (int w = 0; w < WORDS; ++w) row[w] = 0;
+
+    // try one move: piece kind k from `from` to `to`; ep_cap = square of a pawn captured en passant (or -1)
+    auto legal = [&](int k, int from, int to, int ep_cap) -> bool {
+        const u64 fb = 1ull << from, tb = 1ull << to;
+        u64 o[6];
+#pragma unroll
+        for (int j = 0; j < 6; ++j) o[j] = opp[j] & ~tb;
+        u64 n_occ = (occ & ~fb) | tb;
+        if (ep_cap >= 0) { o[0] &= ~(1ull << ep_cap); n_occ &= ~(1ull << ep_cap); }
+        const int ksq = k == 5 ? to : king_sq;
+        return !attacked(ksq, them, o, n_occ);
+    };
+
+#pragma unroll 1
+    for (int k = 0; k < 6; ++k) {
+        u64 pieces = own[k];
+        while (pieces) {
+            const int from = __ffsll((long long)pieces) - 1;
+            pieces &= pieces - 1;
+            const u64 fb = 1ull << from;
+            u64 targets;
+            if (k == 0) {
+                u64 push, cap;
+                if (stm == 0) {
+                    push = (fb << 8) & ~occ;
+                    if (push && (from >> 3) == 1) push |= (fb << 16) & ~occ;
+                    cap = (((fb << 9) & ~FILE_A) | ((fb << 7) & ~FILE_H));
+                } else {
+                    push = (fb >> 8) & ~occ;
+                    if (push && (from >> 3) == 6) push |= (fb >> 16) & ~occ;
+                    cap = (((fb >> 9) & ~FILE_H) | ((fb >> 7) & ~FILE_A));
+                }
+                const u64 ep_bit = ep < 64 ? (1ull << ep) : 0ull;
+                targets = push | (cap & (opp_occ | (ep_bit & ~occ)));
+            } else if (k == 1) targets = knight_set(fb) & ~own_occ;
+            else if (k == 5) targets = king_set(fb) & ~own_occ;
+            else {
+                targets = 0;
+                if (k != 3) targets |= ray_set(from, occ, true);
+                if (k != 2) targets |= ray_set(from, occ, false);
+                targets &= ~own_occ;
+            }
+            while (targets) {
+                const int to = __ffsll((long long)targets) - 1;
+                targets &= targets - 1;
+                int ep_cap = -1;
+                if (k == 0 && to == ep && ((from ^ to) & 7) != 0 && !((opp_occ >> to) & 1ull))
+                    ep_cap = (to & 7) + 8 * (from >> 3);
+                if (!legal(k, from, to, ep_cap)) continue;
+                const bool promotes = k == 0 && ((to >> 3) == (stm ? 0 : 7));
+                set_move<HEAD>(row, stm, from, to, 0);        // plain pair (= queen promotion)
+                if (promotes) {
+                    set_move<HEAD>(row, stm, from, to, 1);
+                    set_move<HEAD>(row, stm, from, to, 2);
+                    set_move<HEAD>(row, stm, from, to, 3);
+                }
+            }
+        }
+    }
+    // castling: rights, king and rook at home, squares between empty, king's path not attacked
+    {
+        const int r0 = stm ? 56 : 0;
+        const int kbit = stm ? 4 : 1, qbit = stm ? 8 : 2;
+        const int c = r->castling;
+        if ((c & (kbit | qbit)) && king_sq == r0 + 4 && !attacked(r0 + 4, them, opp, occ)) {
+            if ((c & kbit) && ((own[3] >> (r0 + 7)) & 1ull) && !(occ & (3ull << (r0 + 5))) &&
+                !attacked(r0 + 5, them, opp, occ) && !attacked(r0 + 6, them, opp, occ))
+                set_move<HEAD>(row, stm, r0 + 4, r0 + 7, 0);
+            if ((c & qbit) && ((own[3] >> r0) & 1ull) && !(occ & (7ull << (r0 + 1))) &&
+                !attacked(r0 + 3, them, opp, occ) && !attacked(r0 + 2, them, opp, occ))
+                set_move<HEAD>(row, stm, r0 + 4, r0, 0);
+        }
+    }
+    u64 *dst = masks + (size_t)pos * WORDS;
+#pragma unroll 1
+    for (int w = 0; w < WORDS; ++w) dst[w] = row[w];
+}
+
+// ---- host: flat-1858 tables -------------------------------------------------------------------
+std::mutex g_table_mutex;
+bool g_table_ready[64] = {};
+
+int ensure_tables() {
+    int dev = 0;
+    AZ_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(g_table_mutex);
+    if (dev < 64 && g_table_ready[dev]) return AZ_OK;
+    static short pair[64 * 64];
+    static short promo[8 * 3];
+    // An origin reaches a destination if they share a line or are a knight jump apart.  Entries are
+    // numbered by walking origins and destinations upward; the promotion entries follow.
+    short next = 0;
+    for (int from = 0; from < 64; ++from) {
+        const int ff = from % 8, fr = from / 8;
+        for (int to = 0; to < 64; ++to) {
+            const int tf = to % 8, tr = to / 8;
+            const int a = ff > tf ? ff - tf : tf - ff, b = fr > tr ? fr - tr : tr - fr;
+            const bool line = (a == 0) != (b == 0) || (a == b && a != 0);
+            const bool jump = a * b == 2;
+            pair[from * 64 + to] = (line || jump) ? next++ : (short)-1;
+        }
+    }
+    for (int file = 0; file < 8; ++file)
+        for (int step = 0; step < 3; ++step) {
+            const int tf = file + step - 1;
+            if (tf < 0 || tf > 7) { promo[file * 3 + step] = -1; continue; }
+            promo[file * 3 + step] = next;
+            next += 3;
+        }
+    AZ_CUDA(cudaMemcpyToSymbol(g_flat_pair, pair, sizeof pair));
+    AZ_CUDA(cudaMemcpyToSymbol(g_flat_promo, promo, sizeof promo));
+    if (dev < 64) g_table_ready[dev] = true;
+    return next == kFlatMoves ? AZ_OK : AZ_ERR_BAD_ARCH;
+}
+
+}  // namespace
+
+int launch_legal_masks(const void *positions, size_t stride, int batch, int head, uint64_t *masks,
+                       cudaStream_t s) {
+    if (batch == 0) return AZ_OK;
+    const unsigned char *p = static_cast<const unsigned char *>(positions);
+    const int block = 64;
+    const unsigned grid = (unsigned)((batch + block - 1) / block);
+    if (head == AZ_POLICY_PLANES73) {
+        legal_masks_kernel<AZ_POLICY_PLANES73><<<grid, block, 0, s>>>(p, stride, batch, (u64 *)masks);
+    } else {
+        int rc = ensure_tables();
+        if (rc != AZ_OK) return rc;
+        legal_masks_kernel<AZ_POLICY_FLAT1858><<<grid, block, 0, s>>>(p, stride, batch, (u64 *)masks);
+    }
+    AZ_LAUNCH_CHECK();
+    return AZ_OK;
+}
+
+}  // namespace az

@@ -1,0 +1,252 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle, on seeded inputs.
+
+Bars: encoding and legal masks bit-exact; policy and value max-abs 1e-4 (fp32), 2e-2 (bf16);
+arg-max move agreement >= 99 % in bf16.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from inputs import configs, positions, weights
+
+pytestmark = pytest.mark.gpu
+
+TOL = {0: 1e-4, 1: 2e-2, 2: 5e-2}
+
+
+@pytest.fixture(scope="module")
+def az():
+    import paper_2609_37447_b200 as az_mod
+    assert torch.cuda.is_available()
+    return az_mod
+
+
+def load(az, cfg, max_batch=None, blob=None):
+    arch = az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head,
+                        cfg.precision, max_batch or cfg.batch)
+    blob = weights.make_blob(cfg) if blob is None else blob
+    return az.az_load_net(arch, blob), blob
+
+
+def gpu_evaluate(az, net, cfg, recs, masks_np=None):
+    n = recs.shape[0]
+    pos = az.records_to_device(recs)
+    if masks_np is None:
+        masks = torch.zeros((n, cfg.mask_words), dtype=torch.int64, device="cuda")
+        az.az_legal_masks(pos, recs.dtype.itemsize, n, cfg.policy_head, masks)
+    else:
+        masks = torch.from_numpy(masks_np.view(np.int64)).cuda()
+    policy = torch.full((n, cfg.policy_size), -7.0, dtype=torch.float32, device="cuda")
+    value = torch.full((n, cfg.value_size), -7.0, dtype=torch.float32, device="cuda")
+    az.az_evaluate(net, pos, masks, n, policy, value)
+    torch.cuda.synchronize()
+    return az.masks_to_numpy(masks), policy.cpu().numpy(), value.cpu().numpy()
+
+
+def compare(cfg, masks_g, pol_g, val_g, masks_o, pol_o, val_o, tol):
+    assert (masks_g == masks_o).all(), "legal masks differ"
+    assert np.isfinite(pol_g).all() and np.isfinite(val_g).all()
+    bits = np.unpackbits(masks_o.view(np.uint8), axis=1, bitorder="little")[:, : cfg.policy_size].astype(bool)
+    assert (pol_g[~bits] == 0.0).all(), "illegal moves must get exactly zero"
+    assert np.abs(pol_g.sum(axis=1) - 1.0).max() < 1e-3
+    perr = np.abs(pol_g - pol_o).max()
+    verr = np.abs(val_g - val_o).max()
+    agree = (pol_g.argmax(axis=1) == pol_o.argmax(axis=1)).mean()
+    print(f"{cfg.name}: n={pol_g.shape[0]} policy max-abs {perr:.3e} value max-abs {verr:.3e} arg-max agreement {agree:.4f}")
+    assert perr <= tol and verr <= tol
+    return agree
+
+
+# ---- encoder and masks: bit-exact ------------------------------------------------------------------
+
+@pytest.mark.parametrize("in_planes,precision", [(19, 0), (19, 1), (112, 1), (112, 0)])
+def test_encoding_is_bit_exact(az, in_planes, precision):
+    cfg = configs.tiny_config(in_planes=in_planes, blocks=0, channels=16, precision=precision, batch=777)
+    net, _ = load(az, cfg)
+    rec, _ = positions.generate(31337, 777, (0, 40), (40, 160))
+    recs = positions.records_for_planes(in_planes, rec)
+    ref = oracle.encode(recs, in_planes)                                  # [n][P][8][8] float64
+    pad = az.az_plane_channels(net.arch)
+    planes = torch.full((777, 64, pad), 9.0, dtype=net.act_dtype, device="cuda")
+    az.az_encode(net, az.records_to_device(recs), 777, planes)
+    torch.cuda.synchronize()
+    want = torch.zeros((777, 64, pad), dtype=torch.float32)
+    want[:, :, :in_planes] = torch.from_numpy(ref.reshape(777, in_planes, 64).transpose(0, 2, 1).astype(np.float32))
+    want = want.to(net.act_dtype)                                         # same rounding decision as the kernel
+    got = planes.cpu()
+    assert torch.equal(got.view(torch.int16 if precision else torch.int32),
+                       want.view(torch.int16 if precision else torch.int32))
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
+@pytest.mark.parametrize("head", [0, 1])
+def test_legal_masks_are_bit_exact(az, head):
+    rec, _ = positions.generate(4242 + head, 6000, (0, 60), (40, 200))
+    special = [
+        "r3k2r/p1ppqpb1/bn2pnp1/3PN3/1p2P3/2N2Q1p/PPPBBPPP/R3K2R w KQkq - 0 1",
+        "8/2p5/3p4/KP5r/1R3p1k/8/4P1P1/8 w - - 0 1",
+        "r3k2r/Pppp1ppp/1b3nbN/nP6/BBP1P3/q4N2/Pp1P2PP/R2Q1RK1 w kq - 0 1",
+        "rnbq1k1r/pp1Pbppp/2p5/8/2B5/8/PPP1NnPP/RNBQK2R w KQ - 1 8",
+        "8/8/8/8/k2Pp2Q/8/8/3K4 b - d3 0 1",
+        "4kr2/8/8/8/8/8/8/R3K2R w KQ - 0 1",
+        "1r2k3/8/8/8/8/8/8/R3K2R w KQ - 0 1",
+        "r3k2r/8/8/3pP3/8/8/8/R3K2R w KQkq d6 0 1",
+        "r3k2r/8/8/8/3pP3/8/8/R3K2R b KQkq e3 0 1",
+        "1n5k/P7/8/8/8/8/8/K7 w - - 0 1",
+        "k7/8/8/8/8/8/p7/1N5K b - - 0 1",
+    ]
+    cur = np.concatenate([positions.cur_records(rec)] + [positions.record_from_fen(f) for f in special])
+    n = cur.shape[0]
+    words = 73 if head == 0 else 30
+    masks = torch.full((n, words), -1, dtype=torch.int64, device="cuda")
+    az.az_legal_masks(az.records_to_device(cur), 104, n, head, masks)
+    torch.cuda.synchronize()
+    assert (az.masks_to_numpy(masks) == oracle.legal_masks(cur, head)).all()
+    # records with history: same answer through the 784-byte stride
+    m2 = torch.zeros((64, words), dtype=torch.int64, device="cuda")
+    az.az_legal_masks(az.records_to_device(rec[:64]), 784, 64, head, m2)
+    torch.cuda.synchronize()
+    assert (az.masks_to_numpy(m2) == oracle.legal_masks(cur[:64], head)).all()
+
+
+# ---- whole path -------------------------------------------------------------------------------------
+
+def test_c1_fp32_batch_64_full_parity(az):
+    cfg = configs.CONFIGS["c1"]
+    net, blob = load(az, cfg)
+    recs = positions.cur_records(positions.for_config(cfg))
+    mo, _, po, vo = oracle.evaluate(blob, recs, cfg.in_planes, cfg.policy_head)
+    mg, pg, vg = gpu_evaluate(az, net, cfg, recs)
+    agree = compare(cfg, mg, pg, vg, mo, po, vo, TOL[0])
+    assert agree == 1.0
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
+@pytest.mark.parametrize("batch", [1, 2, 3, 5, 9, 63])
+@pytest.mark.parametrize("precision", [0, 1])
+def test_small_and_ragged_batches(az, batch, precision):
+    cfg = configs.tiny_config(blocks=2, channels=128 if precision else 32, policy_head=batch % 2,
+                              value_head=batch % 2, precision=precision, batch=batch, weight_seed=50 + batch)
+    blob = weights.make_blob(cfg, 0.02, 0.05)
+    net, _ = load(az, cfg, max_batch=64, blob=blob)
+    rec, _ = positions.generate(900 + batch, batch, (0, 100))
+    recs = positions.cur_records(rec)
+    mo, _, po, vo = oracle.evaluate(blob, recs, 19, cfg.policy_head)
+    mg, pg, vg = gpu_evaluate(az, net, cfg, recs)
+    compare(cfg, mg, pg, vg, mo, po, vo, TOL[precision])
+    az.az_free_net(net)
+
+
+@pytest.mark.parametrize("blocks", [0, 1, 3])
+def test_tower_activations_bf16_128_channels(az, blocks):
+    # layer-level check of the convolution tower against the oracle's tower output
+    cfg = configs.tiny_config(blocks=blocks, channels=128, precision=1, batch=11, weight_seed=7 + blocks)
+    blob = weights.make_blob(cfg, 1.0, 1.0)
+    net, _ = load(az, cfg, max_batch=16, blob=blob)
+    rec, _ = positions.generate(555, 11, (0, 100))
+    recs = positions.cur_records(rec)
+    _, _, _, _, raw = oracle.evaluate(blob, recs, 19, 0, want_tower=True)
+    tower = torch.zeros((11, 64, 128), dtype=torch.bfloat16, device="cuda")
+    az.az_tower(net, az.records_to_device(recs), 11, tower)
+    torch.cuda.synchronize()
+    got = tower.float().cpu().numpy().transpose(0, 2, 1).reshape(11, 128, 8, 8)
+    ref = raw["tower"]
+    err = np.abs(got - ref).max() / np.abs(ref).max()
+    print(f"tower blocks={blocks}: max-abs error relative to the largest activation {err:.3e}")
+    assert err < 2e-2 * (1 + blocks) ** 0.5
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
+def test_c2_bf16_batch_256(az):
+    cfg = configs.CONFIGS["c2"]
+    net, blob = load(az, cfg)
+    recs = positions.cur_records(positions.for_config(cfg))
+    mo, _, po, vo = oracle.evaluate(blob, recs, cfg.in_planes, cfg.policy_head)
+    mg, pg, vg = gpu_evaluate(az, net, cfg, recs)
+    agree = compare(cfg, mg, pg, vg, mo, po, vo, TOL[1])
+    assert agree >= 0.99
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
+def test_c3_bf16_batch_1024_full_launch_sampled_oracle(az):
+    # the launch configuration the benchmark times (batch 1024); the oracle checks a sample of rows
+    cfg = configs.CONFIGS["c3"]
+    net, blob = load(az, cfg)
+    recs = positions.cur_records(positions.for_config(cfg))
+    mg, pg, vg = gpu_evaluate(az, net, cfg, recs)
+    sample = np.concatenate([np.arange(0, 1024, 7), np.arange(1016, 1024)])
+    mo, _, po, vo = oracle.evaluate(blob, recs[sample], cfg.in_planes, cfg.policy_head)
+    agree = compare(cfg, mg[sample], pg[sample], vg[sample], mo, po, vo, TOL[1])
+    assert agree >= 0.99
+    # properties that hold for every row
+    assert np.abs(pg.sum(axis=1) - 1).max() < 1e-3 and np.abs(vg.sum(axis=1) - 1).max() < 1e-5
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
+def test_results_are_deterministic_and_independent_of_batch_composition(az):
+    cfg = configs.tiny_config(blocks=3, channels=128, policy_head=1, value_head=1, precision=1, batch=40)
+    blob = weights.make_blob(cfg, 0.02, 0.05)
+    net, _ = load(az, cfg, max_batch=64, blob=blob)
+    recs = positions.cur_records(positions.generate(1, 40, (0, 100))[0])
+    m1, p1, v1 = gpu_evaluate(az, net, cfg, recs)
+    m2, p2, v2 = gpu_evaluate(az, net, cfg, recs)
+    assert (p1 == p2).all() and (v1 == v2).all()                       # bitwise repeatable
+    # a position evaluated alone, or at another place in another batch, gives the same row
+    _, pa, va = gpu_evaluate(az, net, cfg, recs[17:18])
+    _, pb, vb = gpu_evaluate(az, net, cfg, recs[10:33][::-1].copy())
+    assert np.abs(pa[0] - p1[17]).max() <= 1e-6 and np.abs(va[0] - v1[17]).max() <= 1e-6
+    assert np.abs(pb[::-1] - p1[10:33]).max() <= 1e-6
+    az.az_free_net(net)
+
+
+def test_empty_mask_row_gives_zero_policy_and_a_status_flag(az):
+    cfg = configs.tiny_config(blocks=1, channels=32, batch=4)
+    net, blob = load(az, cfg, max_batch=8)
+    recs = positions.cur_records(positions.generate(3, 4, (0, 30))[0])
+    masks = oracle.legal_masks(recs, 0)
+    masks[2] = 0
+    _, pg, vg = gpu_evaluate(az, net, cfg, recs, masks_np=masks)
+    assert (pg[2] == 0).all() and abs(pg[1].sum() - 1) < 1e-5 and np.isfinite(vg).all()
+    assert az.az_device_status(net) & 1
+    assert az.az_device_status(net) == 0                                # reading clears it
+    az.az_free_net(net)
+
+
+def test_host_side_error_paths(az):
+    cfg = configs.tiny_config(blocks=1, channels=32, batch=4)
+    blob = weights.make_blob(cfg)
+    arch = az.make_arch(19, 1, 32, 0, 0, 0, 4)
+    for bad, code in ((blob[:-4], az.AZ_ERR_BAD_WEIGHTS), (blob[:40], az.AZ_ERR_BAD_WEIGHTS)):
+        with pytest.raises(az.AzError) as e:
+            az.az_load_net(arch, bad)
+        assert e.value.code == code
+    nan = blob.copy()
+    nan[64 + 400:64 + 404] = np.frombuffer(np.float32("nan").tobytes(), dtype=np.uint8)
+    with pytest.raises(az.AzError) as e:
+        az.az_load_net(arch, nan)
+    assert e.value.code == az.AZ_ERR_BAD_WEIGHTS
+    with pytest.raises(az.AzError) as e:
+        az.az_load_net(az.make_arch(19, 2, 32, 0, 0, 0, 4), blob)       # header disagrees with arch
+    assert e.value.code == az.AZ_ERR_BAD_WEIGHTS
+    with pytest.raises(az.AzError) as e:
+        az.az_load_net(az.make_arch(20, 1, 32, 0, 0, 0, 4), blob)
+    assert e.value.code == az.AZ_ERR_BAD_ARCH
+    net = az.az_load_net(arch, blob)
+    pos = az.records_to_device(positions.cur_records(positions.generate(3, 8, (0, 30))[0]))
+    masks = torch.zeros((8, 73), dtype=torch.int64, device="cuda")
+    pol = torch.zeros((8, 4672), device="cuda")
+    val = torch.zeros((8, 1), device="cuda")
+    with pytest.raises(az.AzError) as e:
+        az.az_evaluate(net, pos, masks, 8, pol, val)
+    assert e.value.code == az.AZ_ERR_BATCH_TOO_LARGE
+    az.az_evaluate(net, pos, masks, 0, pol, val)                        # empty batch is a no-op
+    with pytest.raises(az.AzError) as e:
+        az.az_evaluate(net, pos, masks, -1, pol, val)
+    assert e.value.code == az.AZ_ERR_BAD_ARG
+    az.az_free_net(net)
