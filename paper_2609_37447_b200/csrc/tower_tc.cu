@@ -1,8 +1,356 @@
-// placeholder until the tensor-core tower lands
+// The residual convolution tower on tcgen05 tensor cores (bf16 operands, fp32 accumulation in
+// TMEM), one persistent kernel for the whole tower (Sec. 3.5 shared residual backbone; block order
+// convolution, normalisation, activation, convolution, normalisation, residual addition,
+// activation, Sec. 4.3.6; batch-norm folded on the deployment copy, App. D.3).
+//
+// Boards are independent, so a CTA takes four boards and carries them through every layer without
+// leaving the SM: there is no grid-wide synchronisation and inter-layer activations never touch
+// HBM.  The 3x3 convolution is an implicit GEMM, M = 128 rows (2 boards x 64 squares, a "group"),
+// N = 128 output channels, K = 9 taps x input channels.
+//
+//  * A operand: the group's activations live in shared memory as a zero-bordered frame in the
+//    no-swizzle K-major core-matrix layout: for every 8-channel slice a plane of 16-byte slots,
+//    slot(y, b, x) = ((y+1)*2 + b)*9 + (x+1); slot 0 of every 9-slot strip and the strips y = -1
+//    and y = 8 are never written and stay zero.  Eight consecutive GEMM rows (one board row) are
+//    eight consecutive slots, row groups are 9 slots (144 B) apart, and a tap (dy, dx) is nothing
+//    but a start-address offset of (dy*18 + dx) slots: the implicit GEMM moves no data.
+//  * B operand: weights (batch-norm scale folded in, bf16) pre-packed on the host as ready-made
+//    core-matrix tiles, streamed L2 -> shared memory by bulk async copies through a 3-stage ring;
+//    one stage = 16 input channels x 9 taps x 128 outputs, shared by both groups of the CTA.
+//  * D: per group 128 TMEM columns H (the fp32 residual stream) and 128 columns ACC.  conv1 writes
+//    ACC; conv2 accumulates straight onto H, so the residual addition costs nothing and the
+//    residual stream is never re-rounded to bf16.
+//  * Epilogue (4 warps per group): bias + ReLU, fp32 back to H where needed, bf16 into the SAME
+//    shared-memory frame in place (all MMAs that read it have completed), 16 channels at a time, each
+//    slice handing the next layer's MMAs a "ready" mbarrier so that the tensor pipe restarts
+//    after the first slice instead of after the whole epilogue.
+// Warp roles: warp 0 weight producer, warp 1 MMA issuer, warps 2-5 / 6-9 epilogue of group 0 / 1.
+// Every mbarrier wait is bounded; on expiry the CTA raises a status bit, stops issuing work,
+// drains, frees its TMEM and exits.
 #include "common.cuh"
+#include "ptx.cuh"
+
 namespace az {
-size_t tc_packed_weight_bytes(int, int, int) { return 0; }
-void tc_pack_weights(const float *const *, const float *const *, int, int, int, int, __nv_bfloat16 *) {}
-int launch_tower_tc(const Net &, const void *, int, void *, cudaStream_t) { return AZ_ERR_UNSUPPORTED; }
-int tower_tc_launch_count() { return 1; }
+namespace {
+
+constexpr int kC = 128;                        // tower channels
+constexpr int kNB = 2;                         // boards per group
+constexpr int kGroups = 2;                     // groups per CTA
+constexpr int kBoardsPerCta = kNB * kGroups;
+constexpr int kSlots = 10 * kNB * 9 + 1;       // 181 sixteen-byte slots per 8-channel plane
+constexpr int kPlaneBytes = kSlots * 16;       // 2896
+constexpr int kFrameBytes = kPlaneBytes * (kC / 8);   // 46336 per group
+constexpr int kRowGroupBytes = 9 * 16;         // stride between 8-row groups (SBO)
+constexpr int kTileBytes = 128 * 16 * 2;       // one tap: N=128 x K=16 bf16 = 4096
+constexpr int kStageBytes = 9 * kTileBytes;    // 36864: 16 input channels, all taps
+constexpr int kStages = 3;
+constexpr int kThreads = 32 * (2 + 4 * kGroups);
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t kSpinLimit = 1u << 24;
+
+constexpr int kOffFrames = 0;
+constexpr int kOffWeights = kOffFrames + kGroups * kFrameBytes;          // 92672
+constexpr int kOffBars = kOffWeights + kStages * kStageBytes;            // 203264
+// barriers: w_full[3], w_empty[3], acc_full[2], a_ready[2][8], done
+constexpr int kNumBars = 2 * kStages + kGroups + kGroups * 8 + 1;
+constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
+constexpr int kOffAbort = kOffTmemPtr + 4;
+constexpr int kSmemBytes = kOffAbort + 4 + 8;
+
+struct TowerArgs {
+    const __nv_bfloat16 *planes;     // [batch][64][32]
+    const __nv_bfloat16 *weights;    // packed stages
+    const float *bias;               // [n_conv][128]
+    __nv_bfloat16 *out;              // [batch][64][128]
+    uint32_t *status;
+    int batch;
+    int n_conv;                      // 1 + 2*blocks
+    int in_kc;                       // 16-channel slices of the input layer (2)
+};
+
+// Bounded wait, called by all 32 lanes of a warp together.  Returns false (to every lane alike) if
+// the CTA has been aborted or this wait ran out; the latter raises the abort flag and the status bit.
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status) {
+    bool done = false;
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (ptx::mbar_try_wait(bar, parity)) { done = true; break; }
+        if ((i & 63u) == 63u && *abort_flag) break;
+    }
+    if (!done && !*abort_flag) {
+        *abort_flag = 1;
+        atomicOr(status, kStatusWaitTimeout);
+    }
+    return __all_sync(0xffffffffu, done);
 }
+
+__global__ void __launch_bounds__(kThreads, 1)
+tower_tc_kernel(const TowerArgs args) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = ptx::smem_addr(smem);
+    const uint32_t bars = smem_base + kOffBars;
+    auto bar_w_full = [&](int s) { return bars + 8u * s; };
+    auto bar_w_empty = [&](int s) { return bars + 8u * (kStages + s); };
+    auto bar_acc_full = [&](int g) { return bars + 8u * (2 * kStages + g); };
+    auto bar_a_ready = [&](int g, int kc) { return bars + 8u * (2 * kStages + kGroups + g * 8 + kc); };
+    const uint32_t bar_done = bars + 8u * (kNumBars - 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffAbort);
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + kOffTmemPtr);
+
+    // ---- set-up: zero the frames (their borders stay zero for the kernel's lifetime), barriers, TMEM
+    for (int i = threadIdx.x; i < kGroups * kFrameBytes / 16; i += kThreads)
+        reinterpret_cast<uint4 *>(smem + kOffFrames)[i] = make_uint4(0, 0, 0, 0);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { ptx::mbar_init(bar_w_full(s), 1); ptx::mbar_init(bar_w_empty(s), 1); }
+        for (int g = 0; g < kGroups; ++g) {
+            ptx::mbar_init(bar_acc_full(g), 1);
+            for (int kc = 0; kc < 8; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4);
+        }
+        ptx::mbar_init(bar_done, 1);
+        *abort_flag = 0;
+        ptx::fence_barrier_init();
+    }
+    ptx::fence_proxy_async_smem();
+    if (warp == 0) {
+        ptx::tmem_alloc(ptx::smem_addr(tmem_ptr_smem), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_ptr_smem;
+
+    const int n_units = (args.batch + kBoardsPerCta - 1) / kBoardsPerCta;
+    const int n_conv = args.n_conv;
+
+    if (warp == 0) {
+        // ================= weight producer =================
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t last_parity[kStages] = {0, 0, 0};
+        bool issued[kStages] = {false, false, false};
+        bool ok = true;
+        for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+            const unsigned char *src = reinterpret_cast<const unsigned char *>(args.weights);
+            for (int l = 0; l < n_conv && ok; ++l) {
+                const int nkc = l == 0 ? args.in_kc : kC / 16;
+                for (int kc = 0; kc < nkc; ++kc) {
+                    ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        ptx::mbar_arrive_expect_tx(bar_w_full(stage), kStageBytes);
+                        ptx::bulk_copy_g2s(smem_base + kOffWeights + stage * kStageBytes, src, kStageBytes, bar_w_full(stage));
+                    }
+                    issued[stage] = true; last_parity[stage] = phase;
+                    src += kStageBytes;
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    __syncwarp();
+                }
+            }
+        }
+        if (!ok) {
+            // copies already in flight must land before the CTA's shared memory is released
+            for (int s = 0; s < kStages; ++s)
+                if (issued[s])
+                    for (uint32_t i = 0; i < (1u << 20); ++i)
+                        if (ptx::mbar_try_wait(bar_w_full(s), last_parity[s])) break;
+        }
+    } else if (warp == 1) {
+        // ================= MMA issuer =================
+        constexpr uint32_t idesc = ptx::idesc_bf16_f32(128, 128);
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t a_phase[kGroups] = {0, 0};
+        bool ok = true;
+        for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+            for (int l = 0; l < n_conv && ok; ++l) {
+                const int nkc = l == 0 ? args.in_kc : kC / 16;
+                const bool conv2 = l >= 2 && (l & 1) == 0;             // accumulates onto the residual stream
+                const bool to_acc = (l & 1) == 1;                      // conv1 writes the ACC columns
+                for (int kc = 0; kc < nkc && ok; ++kc) {
+                    ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status);
+                    if (!ok) break;
+                    const uint32_t w_addr = smem_base + kOffWeights + stage * kStageBytes;
+                    for (int g = 0; g < kGroups; ++g) {
+                        ok = wait_bar(bar_a_ready(g, kc), (a_phase[g] >> kc) & 1u, abort_flag, args.status);
+                        if (!ok) break;
+                        a_phase[g] ^= 1u << kc;
+                        ptx::tc_fence_after();
+                        if (lane == 0) {
+                            const uint32_t d = tmem_base + (uint32_t)(g * 256 + (to_acc ? 128 : 0));
+                            // row m = (y*2 + b)*8 + x starts at slot (2 + 0)*9 + 1 = 19 for m = 0
+                            const uint32_t a_base = smem_base + kOffFrames + g * kFrameBytes + (2 * kc) * kPlaneBytes + (kNB * 9 + 1) * 16;
+#pragma unroll
+                            for (int tap = 0; tap < 9; ++tap) {
+                                const int dy = tap / 3 - 1, dx = tap % 3 - 1;
+                                const uint64_t adesc = ptx::smem_desc_kmajor_noswizzle(
+                                    a_base + (uint32_t)((dy * kNB * 9 + dx) * 16), kPlaneBytes, kRowGroupBytes);
+                                const uint64_t bdesc = ptx::smem_desc_kmajor_noswizzle(w_addr + tap * kTileBytes, 2048, 128);
+                                const uint32_t acc = (conv2 || kc > 0 || tap > 0) ? 1u : 0u;
+                                ptx::mma_bf16(d, adesc, bdesc, idesc, acc);
+                            }
+                            if (kc == nkc - 1) ptx::mma_commit(bar_acc_full(g));
+                        }
+                        __syncwarp();
+                    }
+                    if (!ok) break;
+                    if (lane == 0) ptx::mma_commit(bar_w_empty(stage));
+                    __syncwarp();
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+        // all issued MMAs must have completed before TMEM is freed
+        if (lane == 0) ptx::mma_commit(bar_done);
+        __syncwarp();
+        for (uint32_t i = 0; i < (1u << 22); ++i)
+            if (ptx::mbar_try_wait(bar_done, 0)) break;
+    } else {
+        // ================= epilogue: 4 warps per group =================
+        const int g = (warp - 2) >> 2;
+        const int q = warp & 3;                               // TMEM lane quarter this warp may access
+        const int m = q * 32 + lane;                          // GEMM row = TMEM lane
+        const int g8 = m >> 3, y = g8 >> 1, b = g8 & 1, x = m & 7;
+        const int slot = (g8 + kNB) * 9 + x + 1;
+        unsigned char *frame = smem + kOffFrames + g * kFrameBytes;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 256);
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+            const int board = unit * kBoardsPerCta + g * kNB + b;
+            const bool live = board < args.batch;
+            const int sq = y * 8 + x;
+            // ---- the unit's input planes -> frame slices 0..3 (32 channels)
+            {
+                const uint4 *src = reinterpret_cast<const uint4 *>(args.planes + ((size_t)board * 64 + sq) * 32);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint4 v = live ? __ldg(src + j) : make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = v;
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) { ptx::mbar_arrive(bar_a_ready(g, 0)); ptx::mbar_arrive(bar_a_ready(g, 1)); }
+            }
+            for (int l = 0; l < n_conv && ok; ++l) {
+                const bool from_acc = (l & 1) == 1;
+                const bool last = l == n_conv - 1;
+                ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status);
+                if (!ok) break;
+                acc_phase ^= 1u;
+                ptx::tc_fence_after();
+                const float *bias = args.bias + (size_t)l * kC;
+                __nv_bfloat16 *dst = args.out + ((size_t)board * 64 + sq) * kC;
+#pragma unroll 1
+                for (int kc = 0; kc < kC / 16; ++kc) {
+                    uint32_t r[16];
+                    ptx::tmem_ld16(t_lane + (uint32_t)((from_acc ? 128 : 0) + kc * 16), r);
+                    ptx::tmem_ld_wait();
+                    float v[16];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4) {
+                        const float4 bv = __ldg(reinterpret_cast<const float4 *>(bias + kc * 16 + i));
+                        v[i + 0] = fmaxf(__uint_as_float(r[i + 0]) + bv.x, 0.0f);
+                        v[i + 1] = fmaxf(__uint_as_float(r[i + 1]) + bv.y, 0.0f);
+                        v[i + 2] = fmaxf(__uint_as_float(r[i + 2]) + bv.z, 0.0f);
+                        v[i + 3] = fmaxf(__uint_as_float(r[i + 3]) + bv.w, 0.0f);
+                    }
+                    if (!from_acc && !last) {                  // keep the residual stream in fp32
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(v[i]);
+                        ptx::tmem_st16(t_lane + (uint32_t)(kc * 16), r);
+                    }
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+                        pk[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                    }
+                    if (last) {
+                        if (live) {
+                            reinterpret_cast<uint4 *>(dst + kc * 16)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            reinterpret_cast<uint4 *>(dst + kc * 16)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                        }
+                    } else {
+                        *reinterpret_cast<uint4 *>(frame + (2 * kc) * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        *reinterpret_cast<uint4 *>(frame + (2 * kc + 1) * kPlaneBytes + slot * 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                        if (!from_acc) ptx::tmem_st_wait();
+                        ptx::fence_proxy_async_smem();
+                        ptx::tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar_a_ready(g, kc));
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace
+
+// Packed layout: for layer l, 16-channel slice kc, tap, the N=128 x K=16 tile as core matrices
+// [k8 (2)][n-group (16)][n in group (8)][k in slice (8)] bf16, scale folded into the weights.
+size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv) {
+    const size_t stages = (size_t)in_pad / 16 + (size_t)(n_conv - 1) * (channels / 16);
+    return stages * kStageBytes;
+}
+
+void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
+                     int channels, int n_conv, __nv_bfloat16 *packed) {
+    __nv_bfloat16 *dst = packed;
+    for (int l = 0; l < n_conv; ++l) {
+        const int cin = l == 0 ? in_planes : channels;
+        const int nkc = (l == 0 ? in_pad : channels) / 16;
+        for (int kc = 0; kc < nkc; ++kc)
+            for (int tap = 0; tap < 9; ++tap)
+                for (int k8 = 0; k8 < 2; ++k8)
+                    for (int ng = 0; ng < channels / 8; ++ng)
+                        for (int r = 0; r < 8; ++r)
+                            for (int e = 0; e < 8; ++e) {
+                                const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
+                                float v = 0.0f;
+                                if (ci < cin) v = scale[l][n] * w[l][((size_t)n * cin + ci) * 9 + tap];
+                                *dst++ = __float2bfloat16_rn(v);
+                            }
+    }
+}
+
+int tower_tc_launch_count() { return 1; }
+
+int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, cudaStream_t s) {
+    if (batch == 0) return AZ_OK;
+    static int sm_count[64] = {};
+    int dev = 0;
+    AZ_CUDA(cudaGetDevice(&dev));
+    if (dev < 64 && sm_count[dev] == 0) {
+        int n = 0;
+        AZ_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        sm_count[dev] = n;
+    }
+    const int sms = dev < 64 ? sm_count[dev] : 148;
+    TowerArgs a;
+    a.planes = static_cast<const __nv_bfloat16 *>(planes);
+    a.weights = static_cast<const __nv_bfloat16 *>(net.tc_weights);
+    a.bias = net.tc_bias;
+    a.out = static_cast<__nv_bfloat16 *>(tower_out);
+    a.status = net.status_dev;
+    a.batch = batch;
+    a.n_conv = net.n_conv;
+    a.in_kc = net.in_pad / 16;
+    const int n_units = (batch + kBoardsPerCta - 1) / kBoardsPerCta;
+    const int grid = n_units < sms ? n_units : sms;
+    tower_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(a);
+    AZ_LAUNCH_CHECK();
+    return AZ_OK;
+}
+
+}  // namespace az
