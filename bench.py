@@ -1,0 +1,292 @@
+"""Benchmark of batched leaf evaluation: leaf evals/sec on the 20x128 bf16 batch-1024 workload.
+
+A step is one az_evaluate call (encode -> tower -> heads -> masked softmax) on one batch of
+synthetic positions that already sits in device memory.  One process per GPU; with N > 1
+(torchrun) every rank evaluates its own batch (weak scaling, no collective on the data path).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config c3] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from inputs import configs, positions, weights  # noqa: E402
+
+METRIC = "leaf evals/sec, 20x128 bf16 batch 1024"
+UNIT = "evals/s"
+WORKLOADS = {
+    "c1": "c1: 6x64 fp32 batch 64, 73-plane policy + tanh value",
+    "c2": "c2: 20x128 bf16 batch 256, 73-plane policy + tanh value",
+    "c3": "c3: 20x128 bf16 batch 1024, flat-1858 policy + WDL value",
+}
+DTYPE = {0: "f32", 1: "bf16", 2: "fp8_e4m3"}
+
+# DRAM bytes (read + write) of one tower-kernel launch at batch 1024 from an ncu capture; the
+# summary the figure comes from is profiles/tower_tc_kernel_c3.md.  None until captured.
+TOWER_TRAFFIC_BYTES = {"c3": None, "c2": None}
+
+
+def tower_flops_per_position(cfg) -> float:
+    """Dense convolution count 2*64*9*Cin*Cout per layer; channel padding is not counted."""
+    c = cfg.channels
+    return 2.0 * 64 * 9 * (cfg.in_planes * c + 2 * cfg.blocks * c * c)
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"bf16_tflops": float(p["bf16_tflops"]), "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+    except (OSError, KeyError, ValueError):
+        return {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._stop_event = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            pass
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonGpuIdle", 0x1): None,
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._stop_event.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if name and (r & bit):
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def stop(self):
+        self._stop_event.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def oracle_rate(cfg, blob, recs, sample: int):
+    """The CPU oracle, as it stands, on the first `sample` positions: (evals/s, seconds, threads)."""
+    import oracle
+    sub = recs[:sample]
+    t0 = time.perf_counter()
+    oracle.evaluate(blob, sub, cfg.in_planes, cfg.policy_head)
+    dt = time.perf_counter() - t0
+    return sub.shape[0] / dt, dt, oracle.threads()
+
+
+def run_reference(args, cfg):
+    """--impl reference: the oracle on the host cores; each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    blob = weights.make_blob(cfg)
+    recs = positions.records_for_planes(cfg.in_planes, positions.for_config(cfg))
+    sample = min(cfg.batch, 128)
+    for _ in range(args.warmup):
+        oracle_rate(cfg, blob, recs, min(sample, 16))
+    total_t, total_n, threads = 0.0, 0, 1
+    for _ in range(args.steps):
+        rate, dt, threads = oracle_rate(cfg, blob, recs, sample)
+        total_t += dt
+        total_n += sample
+    value = total_n / total_t
+    sample_txt = f"first {sample} positions of the {cfg.batch}-position batch per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOADS[cfg.name], "sample": sample_txt},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample_txt},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", default="c3", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    cfg = configs.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_37447_b200 as az
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    # ---- inputs: every rank evaluates its own batch of the same stream (weak scaling)
+    B = cfg.batch
+    rec = positions.for_config(cfg, B, first_index=rank * B)
+    recs = positions.records_for_planes(cfg.in_planes, rec)
+    blob = weights.make_blob(cfg)
+    arch = az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, B)
+    net = az.az_load_net(arch, blob)
+    pos_dev = az.records_to_device(recs)
+    masks_dev = torch.zeros((B, cfg.mask_words), dtype=torch.int64, device="cuda")
+    az.az_legal_masks(pos_dev, recs.dtype.itemsize, B, cfg.policy_head, masks_dev)
+    policy_dev = torch.zeros((B, cfg.policy_size), dtype=torch.float32, device="cuda")
+    value_dev = torch.zeros((B, cfg.value_size), dtype=torch.float32, device="cuda")
+    flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")   # > 126 MB L2
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: K steps, L2 flushed before each, each step bracketed by events
+    for _ in range(args.warmup):
+        az.az_evaluate(net, pos_dev, masks_dev, B, policy_dev, value_dev)
+    torch.cuda.synchronize()
+    az.az_profile_tower(net, True)
+    az.az_tower_time(net)
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    for i in range(args.steps):
+        flush.fill_(i & 0xFF)
+        starts[i].record()
+        az.az_evaluate(net, pos_dev, masks_dev, B, policy_dev, value_dev)
+        ends[i].record()
+    barrier()
+    clocks = sampler.stop()
+    step_ms = [s.elapsed_time(e) for s, e in zip(starts, ends)]
+    total_ms = float(sum(step_ms))
+    tower_ms, tower_passes = az.az_tower_time(net)
+    az.az_profile_tower(net, False)
+    status = az.az_device_status(net)
+
+    # ---- the same back to back without flushing (steady-state serving: weights stay in L2)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        az.az_evaluate(net, pos_dev, masks_dev, B, policy_dev, value_dev)
+    ev1.record()
+    barrier()
+    b2b_ms = ev0.elapsed_time(ev1)
+
+    # ---- end to end through the host-buffer entry point: pinned host in, pinned host out
+    pos_host = torch.from_numpy(np.ascontiguousarray(recs).view(np.uint8).reshape(B, -1).copy()).pin_memory()
+    masks_host = masks_dev.cpu().pin_memory()
+    policy_host = torch.zeros((B, cfg.policy_size), dtype=torch.float32).pin_memory()
+    value_host = torch.zeros((B, cfg.value_size), dtype=torch.float32).pin_memory()
+    for _ in range(3):
+        az.az_evaluate_host(net, pos_host, masks_host, B, policy_host, value_host)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        az.az_evaluate_host(net, pos_host, masks_host, B, policy_host, value_host)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    barrier()
+    h2d = pos_host.numel() + masks_host.numel() * 8
+    d2h = (policy_host.numel() + value_host.numel()) * 4
+    checksum = float(policy_host.sum())            # every row sums to one
+
+    # ---- max over ranks
+    t = torch.tensor([total_ms, b2b_ms, e2e_s * 1e3, tower_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, b2b_ms, e2e_ms, tower_ms_max = [float(x) for x in t.cpu()]
+
+    if rank == 0:
+        peaks = load_peaks()
+        evals = world * B * args.steps
+        flops = tower_flops_per_position(cfg) * B
+        tower_avg_ms = tower_ms / max(tower_passes, 1)
+        achieved = flops / (tower_avg_ms * 1e-3) / 1e12 if tower_passes else None
+        traffic = TOWER_TRAFFIC_BYTES.get(cfg.name)
+        out = {
+            "metric": METRIC, "value": evals / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": DTYPE[cfg.precision], "data": "synthetic",
+            "config": {"workload": WORKLOADS[cfg.name], "batch_per_gpu": B, "l2": "flushed before every step (256 MB write)",
+                       "timing": "CUDA events around each step on the launch stream, summed; max over ranks",
+                       "device_status": status, "policy_checksum": checksum},
+            "back_to_back": {"value": evals / (b2b_ms * 1e-3), "unit": UNIT, "ms_per_step": b2b_ms / args.steps,
+                             "note": "no L2 flush between steps"},
+            "e2e": {"value": evals / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                    "ms_per_step": e2e_ms / args.steps, "api": "az_evaluate_host, pinned host buffers"},
+            "gpu_launches": args.steps * az.az_launches_per_evaluate(net, B),
+            "clocks": clocks,
+            "roofline": {"kernel": "tower_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"],
+                         "unit": "TFLOP/s", "frac": (achieved / peaks["bf16_tflops"]) if achieved else None,
+                         "traffic": traffic, "peak_source": f"of {peaks['source']} (burst bf16 GEMM)",
+                         "avg_launch_ms": tower_avg_ms, "launches_timed": tower_passes,
+                         "flops_per_launch": flops},
+        }
+        if not args.no_cpu_baseline:
+            sample = 256 if cfg.channels >= 128 else cfg.batch
+            sample = min(sample, B)
+            rate, dt, threads = oracle_rate(cfg, blob, recs, sample)
+            out["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                   "sample": f"first {sample} positions of the batch, {dt:.1f} s"}
+        print(json.dumps(out))
+    az.az_free_net(net)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -129,6 +129,18 @@ int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_ma
                 int batch, float *policy_dev, float *value_dev, void *cuda_stream);
 
 /*
+ * The same evaluation for callers whose buffers live in HOST memory (Sec. 5.2: preallocated
+ * staging buffers, asynchronous copies and completion events between the search threads and the
+ * GPU).  positions_host / legal_masks_host are copied to device staging buffers owned by the
+ * az_net, the evaluation runs, policy_host / value_host receive the results, and the call returns
+ * after the stream has drained.  Pinned (page-locked) host buffers make the copies asynchronous
+ * with respect to other streams; pageable memory also works.  Layouts as in az_evaluate.
+ * Errors: as az_evaluate.
+ */
+int az_evaluate_host(az_net *net, const void *positions_host, const uint64_t *legal_masks_host,
+                     int batch, float *policy_host, float *value_host, void *cuda_stream);
+
+/*
  * The encoder step alone (App. D.1: side-to-move canonical planes; for Black to move ranks are
  * reflected and colours exchanged, files keep their order).  planes_dev receives
  * [batch][64][az_plane_channels()] elements of the network's activation type (float32 for
@@ -173,6 +185,16 @@ int az_calibrate(az_net *net, const void *positions_dev, int n, void *cuda_strea
 
 /* Device-side status word of the last kernels (0 = clean).  Synchronises the given stream. */
 int az_device_status(az_net *net, void *cuda_stream, uint32_t *status_out);
+
+/*
+ * Timing of the convolution tower alone, for roofline reports: while enabled, every evaluation
+ * brackets its tower kernel(s) with CUDA events on the caller's stream.  az_tower_time reads the
+ * events recorded since the last read (synchronising them), returns their summed duration in
+ * milliseconds and the number of bracketed tower passes, and starts afresh.  At most 4096 passes
+ * are kept between reads; later ones go untimed.
+ */
+int az_profile_tower(az_net *net, int enable);
+int az_tower_time(az_net *net, float *total_ms_out, int *passes_out);
 
 /* Number of kernel launches one az_evaluate of `batch` positions enqueues. */
 int az_launches_per_evaluate(const az_net *net, int batch);

@@ -23,8 +23,8 @@ AZ_VALUE_TANH, AZ_VALUE_WDL = 0, 1
 AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3 = 0, 1, 2
 
 EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
-           "az_load_net", "az_free_net", "az_evaluate", "az_encode", "az_tower", "az_legal_masks",
-           "az_calibrate", "az_device_status", "az_launches_per_evaluate", "az_strerror",
+           "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_host", "az_encode", "az_tower", "az_legal_masks",
+           "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error")
 
 
@@ -56,6 +56,12 @@ def _load_library():
     lib.az_free_net.argtypes = [vp]
     lib.az_evaluate.restype = ci
     lib.az_evaluate.argtypes = [vp, vp, vp, ci, vp, vp, vp]
+    lib.az_evaluate_host.restype = ci
+    lib.az_evaluate_host.argtypes = [vp, vp, vp, ci, vp, vp, vp]
+    lib.az_profile_tower.restype = ci
+    lib.az_profile_tower.argtypes = [vp, ci]
+    lib.az_tower_time.restype = ci
+    lib.az_tower_time.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ci)]
     lib.az_encode.restype = ci
     lib.az_encode.argtypes = [vp, vp, ci, vp, vp]
     lib.az_tower.restype = ci
@@ -150,6 +156,34 @@ def az_evaluate(net: Net, positions_dev, legal_masks_dev, batch, policy_dev, val
     _check(_lib.az_evaluate(net.handle, _dev_ptr(positions_dev, "positions"), _dev_ptr(legal_masks_dev, "legal_masks"),
                             batch, _dev_ptr(policy_dev, "policy"), _dev_ptr(value_dev, "value"), _stream_ptr(stream)),
            "az_evaluate")
+
+
+def _host_ptr(t, name: str) -> int:
+    if isinstance(t, torch.Tensor):
+        if t.is_cuda or not t.is_contiguous():
+            raise TypeError(f"{name} must be a contiguous host tensor")
+        return t.data_ptr()
+    if isinstance(t, np.ndarray) and t.flags["C_CONTIGUOUS"]:
+        return t.ctypes.data
+    raise TypeError(f"{name} must be a contiguous host tensor or numpy array")
+
+
+def az_evaluate_host(net: Net, positions_host, legal_masks_host, batch, policy_host, value_host, stream=None):
+    """az_evaluate with host buffers (pinned or pageable); returns after the results have landed."""
+    _check(_lib.az_evaluate_host(net.handle, _host_ptr(positions_host, "positions"), _host_ptr(legal_masks_host, "legal_masks"),
+                                 batch, _host_ptr(policy_host, "policy"), _host_ptr(value_host, "value"),
+                                 _stream_ptr(stream)), "az_evaluate_host")
+
+
+def az_profile_tower(net: Net, enable: bool):
+    _check(_lib.az_profile_tower(net.handle, 1 if enable else 0), "az_profile_tower")
+
+
+def az_tower_time(net: Net):
+    """(summed milliseconds, passes) of the tower since the last read."""
+    ms, n = ctypes.c_float(0), ctypes.c_int(0)
+    _check(_lib.az_tower_time(net.handle, ctypes.byref(ms), ctypes.byref(n)), "az_tower_time")
+    return float(ms.value), int(n.value)
 
 
 def az_encode(net: Net, positions_dev, batch, planes_dev, stream=None):

@@ -202,6 +202,9 @@ void free_net(Net *n) {
     cudaFree(n->v_w2); cudaFree(n->v_b2);
     cudaFree(n->planes);
     for (int i = 0; i < 3; ++i) cudaFree(n->act[i]);
+    cudaFree(n->stage_pos); cudaFree(n->stage_masks); cudaFree(n->stage_policy); cudaFree(n->stage_value);
+    if (n->ev_begin) for (int i = 0; i < kMaxProfiledPasses; ++i) { cudaEventDestroy(n->ev_begin[i]); cudaEventDestroy(n->ev_end[i]); }
+    delete[] n->ev_begin; delete[] n->ev_end;
     cudaFree(n->logits); cudaFree(n->head_p); cudaFree(n->head_v); cudaFree(n->hidden); cudaFree(n->status_dev);
     delete n;
 }
@@ -212,9 +215,13 @@ int run_tower(Net &n, const void *positions, int batch, void **tower_out, cudaSt
                            n.bf16, n.planes, n.status_dev, s);
     if (rc != AZ_OK) return rc;
     const int C = (int)n.arch.channels;
+    const bool timed = n.profile && n.n_events < kMaxProfiledPasses;
+    if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
     if (n.tc_ready) {
         *tower_out = n.act[0];
-        return launch_tower_tc(n, n.planes, batch, n.act[0], s);
+        rc = launch_tower_tc(n, n.planes, batch, n.act[0], s);
+        if (rc == AZ_OK && timed) AZ_CUDA(cudaEventRecord(n.ev_end[n.n_events++], s));
+        return rc;
     }
     void *x = n.act[0], *t = n.act[1], *y = n.act[2];
     rc = launch_conv3x3_simt(n.planes, n.conv_w[0], n.conv_scale[0], n.conv_bias[0], nullptr, x, batch,
@@ -229,6 +236,7 @@ int run_tower(Net &n, const void *positions, int batch, void **tower_out, cudaSt
         void *tmp = x; x = y; y = tmp;
     }
     *tower_out = x;
+    if (timed) AZ_CUDA(cudaEventRecord(n.ev_end[n.n_events++], s));
     return AZ_OK;
 }
 
@@ -324,6 +332,64 @@ int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_ma
     if (rc != AZ_OK) return rc;
     return az::launch_masked_softmax(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a), (int)az_mask_words(&a),
                                      policy_dev, n->status_dev, s);
+}
+
+int az_evaluate_host(az_net *net, const void *positions_host, const uint64_t *legal_masks_host, int batch,
+                     float *policy_host, float *value_host, void *cuda_stream) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n || batch < 0) return AZ_ERR_BAD_ARG;
+    if (batch == 0) return AZ_OK;
+    if (!positions_host || !legal_masks_host || !policy_host || !value_host) return AZ_ERR_BAD_ARG;
+    if ((uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const az_arch &a = n->arch;
+    const size_t B = a.max_batch, pb = az_position_bytes(&a), mw = az_mask_words(&a), ps = az_policy_size(&a), vs = az_value_size(&a);
+    if (!n->stage_pos) {
+        AZ_CUDA(cudaMalloc(&n->stage_pos, B * pb));
+        AZ_CUDA(cudaMalloc((void **)&n->stage_masks, B * mw * sizeof(uint64_t)));
+        AZ_CUDA(cudaMalloc((void **)&n->stage_policy, B * ps * sizeof(float)));
+        AZ_CUDA(cudaMalloc((void **)&n->stage_value, B * vs * sizeof(float)));
+    }
+    AZ_CUDA(cudaMemcpyAsync(n->stage_pos, positions_host, (size_t)batch * pb, cudaMemcpyHostToDevice, s));
+    AZ_CUDA(cudaMemcpyAsync(n->stage_masks, legal_masks_host, (size_t)batch * mw * sizeof(uint64_t), cudaMemcpyHostToDevice, s));
+    int rc = az_evaluate(net, n->stage_pos, n->stage_masks, batch, n->stage_policy, n->stage_value, cuda_stream);
+    if (rc != AZ_OK) return rc;
+    AZ_CUDA(cudaMemcpyAsync(policy_host, n->stage_policy, (size_t)batch * ps * sizeof(float), cudaMemcpyDeviceToHost, s));
+    AZ_CUDA(cudaMemcpyAsync(value_host, n->stage_value, (size_t)batch * vs * sizeof(float), cudaMemcpyDeviceToHost, s));
+    AZ_CUDA(cudaStreamSynchronize(s));
+    return AZ_OK;
+}
+
+int az_profile_tower(az_net *net, int enable) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n) return AZ_ERR_BAD_ARG;
+    if (enable && !n->ev_begin) {
+        n->ev_begin = new (std::nothrow) cudaEvent_t[az::kMaxProfiledPasses];
+        n->ev_end = new (std::nothrow) cudaEvent_t[az::kMaxProfiledPasses];
+        if (!n->ev_begin || !n->ev_end) return AZ_ERR_BAD_ARG;
+        for (int i = 0; i < az::kMaxProfiledPasses; ++i) {
+            AZ_CUDA(cudaEventCreate(&n->ev_begin[i]));
+            AZ_CUDA(cudaEventCreate(&n->ev_end[i]));
+        }
+    }
+    n->profile = enable != 0;
+    return AZ_OK;
+}
+
+int az_tower_time(az_net *net, float *total_ms_out, int *passes_out) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n || !total_ms_out || !passes_out) return AZ_ERR_BAD_ARG;
+    float total = 0.0f;
+    for (int i = 0; i < n->n_events; ++i) {
+        float ms = 0.0f;
+        AZ_CUDA(cudaEventSynchronize(n->ev_end[i]));
+        AZ_CUDA(cudaEventElapsedTime(&ms, n->ev_begin[i], n->ev_end[i]));
+        total += ms;
+    }
+    *total_ms_out = total;
+    *passes_out = n->n_events;
+    n->n_events = 0;
+    return AZ_OK;
 }
 
 int az_legal_masks(const void *positions_dev, size_t position_stride, int batch, int policy_head,

@@ -64,7 +64,18 @@ struct Net {
     void *head_v = nullptr;           // [B][2048] value projection
     float *hidden = nullptr;          // [B][128]
     uint32_t *status_dev = nullptr;
+
+    // ---- device staging for host-buffer calls (allocated on first use) ----
+    void *stage_pos = nullptr;
+    uint64_t *stage_masks = nullptr;
+    float *stage_policy = nullptr, *stage_value = nullptr;
+
+    // ---- optional event timing of the tower ----
+    bool profile = false;
+    int n_events = 0;                 // pairs recorded since the last read
+    cudaEvent_t *ev_begin = nullptr, *ev_end = nullptr;
 };
+constexpr int kMaxProfiledPasses = 4096;
 
 // ---- error plumbing ------------------------------------------------------------------------
 void set_cuda_error(cudaError_t e, const char *what);

@@ -55,6 +55,10 @@ def compare(cfg, masks_g, pol_g, val_g, masks_o, pol_o, val_o, tol):
     agree = (pol_g.argmax(axis=1) == pol_o.argmax(axis=1)).mean()
     print(f"{cfg.name}: n={pol_g.shape[0]} policy max-abs {perr:.3e} value max-abs {verr:.3e} arg-max agreement {agree:.4f}")
     assert perr <= tol and verr <= tol
+    if pol_g.shape[0] >= 32:
+        # scale-free guard: the value must follow the oracle's ups and downs, not merely sit near it
+        for k in range(val_o.shape[1]):
+            assert np.corrcoef(val_g[:, k], val_o[:, k])[0, 1] > 0.9
     return agree
 
 

@@ -16,8 +16,8 @@ def declared_functions():
 
 @pytest.fixture(scope="module")
 def lib():
-    from paper_2609_37447_b200 import build
-    return ctypes.CDLL(build.build())
+    import __graft_entry__
+    return ctypes.CDLL(__graft_entry__.load_build_module().build())
 
 
 def test_every_declared_entry_point_is_exported(lib):
