@@ -151,10 +151,14 @@ def main():
     ap.add_argument("--config", default="c3", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures on a smaller case)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     cfg = configs.CONFIGS[args.config]
+    if args.batch > 0:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, batch=args.batch)
     if args.impl == "reference":
         run_reference(args, cfg)
         return

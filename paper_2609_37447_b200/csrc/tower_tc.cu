@@ -24,11 +24,17 @@
 //    shared-memory frame in place (all MMAs that read it have completed), 16 channels at a time, each
 //    slice handing the next layer's MMAs a "ready" mbarrier so that the tensor pipe restarts
 //    after the first slice instead of after the whole epilogue.
-// Warp roles: warp 0 weight producer, warp 1 MMA issuer, warps 2-5 / 6-9 epilogue of group 0 / 1.
+// Warp roles: warp 0 weight producer, warps 1-2 MMA issuers of group 0 / 1, warps 3-6 / 7-10
+// epilogue of group 0 / 1.  The tensor pipe does not buffer work across gaps in the issuing
+// thread's instruction stream (measured: a stall of the issuer between two MMAs is pipe idle
+// time), so each group has its own issuer: while one waits on its barriers the other's MMAs run.
 // Every mbarrier wait is bounded; on expiry the CTA raises a status bit, stops issuing work,
 // drains, frees its TMEM and exits.
 #include "common.cuh"
 #include "ptx.cuh"
+
+#include <cstdio>
+#include <cstdlib>
 
 namespace az {
 namespace {
@@ -44,8 +50,15 @@ constexpr int kRowGroupBytes = 9 * 16;         // stride between 8-row groups (S
 constexpr int kTileBytes = 128 * 16 * 2;       // one tap: N=128 x K=16 bf16 = 4096
 constexpr int kStageBytes = 9 * kTileBytes;    // 36864: 16 input channels, all taps
 constexpr int kStages = 3;
-constexpr int kThreads = 32 * (2 + 4 * kGroups);
+constexpr int kThreads = 32 * (1 + kGroups + 4 * kGroups);   // producer, one MMA issuer per group, 4 epilogue warps per group
 constexpr uint32_t kTmemCols = 512;
+// high words of the shared-memory matrix descriptors (no swizzle, K-major): stride between 8-row
+// groups in bits 0-13, descriptor version 1 in bit 14; the low word carries the stride between the
+// two K core matrices in bits 16-29 above the start address.
+constexpr uint32_t kADescHi = (uint32_t)(kRowGroupBytes >> 4) | (1u << 14);
+constexpr uint32_t kBDescHi = (uint32_t)(128 >> 4) | (1u << 14);
+constexpr uint32_t kADescLbo = (uint32_t)(kPlaneBytes >> 4) << 16;
+constexpr uint32_t kBDescLbo = (uint32_t)(2048 >> 4) << 16;
 constexpr uint32_t kSpinLimit = 1u << 24;
 
 constexpr int kOffFrames = 0;
@@ -55,7 +68,10 @@ constexpr int kOffBars = kOffWeights + kStages * kStageBytes;            // 2032
 constexpr int kNumBars = 2 * kStages + kGroups + kGroups * 8 + 1;
 constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
 constexpr int kOffAbort = kOffTmemPtr + 4;
-constexpr int kSmemBytes = kOffAbort + 4 + 8;
+constexpr int kOffBias = (kOffAbort + 4 + 15) & ~15;                     // folded biases of every layer, fp32
+constexpr int kMaxSmem = 232448;
+constexpr int kMaxBiasLayers = (kMaxSmem - kOffBias) / (kC * 4);         // 56 layers fit beside everything else
+constexpr int kSmemBytesNoBias = kOffBias;
 
 struct TowerArgs {
     const __nv_bfloat16 *planes;     // [batch][64][32]
@@ -66,11 +82,15 @@ struct TowerArgs {
     int batch;
     int n_conv;                      // 1 + 2*blocks
     int in_kc;                       // 16-channel slices of the input layer (2)
+    int bias_in_smem;                // all biases staged in shared memory (n_conv <= kMaxBiasLayers)
+    int trace;                       // CTA 0 prints how long each role waited (debugging aid)
 };
 
 // Bounded wait, called by all 32 lanes of a warp together.  Returns false (to every lane alike) if
 // the CTA has been aborted or this wait ran out; the latter raises the abort flag and the status bit.
-__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status) {
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
+                                         long long *waited = nullptr) {
+    const long long t0 = waited ? clock64() : 0;
     bool done = false;
     for (uint32_t i = 0; i < kSpinLimit; ++i) {
         if (ptx::mbar_try_wait(bar, parity)) { done = true; break; }
@@ -80,6 +100,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
         *abort_flag = 1;
         atomicOr(status, kStatusWaitTimeout);
     }
+    if (waited) *waited += clock64() - t0;
     return __all_sync(0xffffffffu, done);
 }
 
@@ -100,13 +121,16 @@ tower_tc_kernel(const TowerArgs args) {
     // ---- set-up: zero the frames (their borders stay zero for the kernel's lifetime), barriers, TMEM
     for (int i = threadIdx.x; i < kGroups * kFrameBytes / 16; i += kThreads)
         reinterpret_cast<uint4 *>(smem + kOffFrames)[i] = make_uint4(0, 0, 0, 0);
+    if (args.bias_in_smem)
+        for (int i = threadIdx.x; i < args.n_conv * kC; i += kThreads)
+            reinterpret_cast<float *>(smem + kOffBias)[i] = args.bias[i];
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { ptx::mbar_init(bar_w_full(s), 1); ptx::mbar_init(bar_w_empty(s), 1); }
+        for (int s = 0; s < kStages; ++s) { ptx::mbar_init(bar_w_full(s), 1); ptx::mbar_init(bar_w_empty(s), kGroups); }
         for (int g = 0; g < kGroups; ++g) {
             ptx::mbar_init(bar_acc_full(g), 1);
             for (int kc = 0; kc < 8; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4);
         }
-        ptx::mbar_init(bar_done, 1);
+        ptx::mbar_init(bar_done, kGroups);
         *abort_flag = 0;
         ptx::fence_barrier_init();
     }
@@ -122,6 +146,10 @@ tower_tc_kernel(const TowerArgs args) {
 
     const int n_units = (args.batch + kBoardsPerCta - 1) / kBoardsPerCta;
     const int n_conv = args.n_conv;
+    const bool tr = args.trace && blockIdx.x == 0;
+    long long t_wait[3] = {0, 0, 0};
+    long long t_issue = 0;
+    const long long t_begin = clock64();
 
     if (warp == 0) {
         // ================= weight producer =================
@@ -135,11 +163,14 @@ tower_tc_kernel(const TowerArgs args) {
             for (int l = 0; l < n_conv && ok; ++l) {
                 const int nkc = l == 0 ? args.in_kc : kC / 16;
                 for (int kc = 0; kc < nkc; ++kc) {
-                    ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status);
+                    ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                     if (!ok) break;
                     if (lane == 0) {
+                        if (args.trace & 4) ptx::mbar_arrive(bar_w_full(stage));
+                        else {
                         ptx::mbar_arrive_expect_tx(bar_w_full(stage), kStageBytes);
                         ptx::bulk_copy_g2s(smem_base + kOffWeights + stage * kStageBytes, src, kStageBytes, bar_w_full(stage));
+                        }
                     }
                     issued[stage] = true; last_parity[stage] = phase;
                     src += kStageBytes;
@@ -155,47 +186,46 @@ tower_tc_kernel(const TowerArgs args) {
                     for (uint32_t i = 0; i < (1u << 20); ++i)
                         if (ptx::mbar_try_wait(bar_w_full(s), last_parity[s])) break;
         }
-    } else if (warp == 1) {
-        // ================= MMA issuer =================
+    } else if (warp <= kGroups) {
+        // ================= MMA issuer of group g =================
+        const int g = warp - 1;
         constexpr uint32_t idesc = ptx::idesc_bf16_f32(128, 128);
         int stage = 0;
         uint32_t phase = 0;
-        uint32_t a_phase[kGroups] = {0, 0};
+        uint32_t a_phase = 0;
         bool ok = true;
+        const uint32_t d_h = tmem_base + (uint32_t)(g * 256);
+        const uint32_t frame_lo = (((smem_base + kOffFrames + g * kFrameBytes) >> 4) + (uint32_t)(kNB * 9 + 1)) | kADescLbo;
         for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
             for (int l = 0; l < n_conv && ok; ++l) {
                 const int nkc = l == 0 ? args.in_kc : kC / 16;
                 const bool conv2 = l >= 2 && (l & 1) == 0;             // accumulates onto the residual stream
-                const bool to_acc = (l & 1) == 1;                      // conv1 writes the ACC columns
-                for (int kc = 0; kc < nkc && ok; ++kc) {
-                    ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status);
+                const uint32_t d = d_h + (((l & 1) == 1) ? 128u : 0u); // conv1 writes the ACC columns
+                for (int kc = 0; kc < nkc; ++kc) {
+                    ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                     if (!ok) break;
-                    const uint32_t w_addr = smem_base + kOffWeights + stage * kStageBytes;
-                    for (int g = 0; g < kGroups; ++g) {
-                        ok = wait_bar(bar_a_ready(g, kc), (a_phase[g] >> kc) & 1u, abort_flag, args.status);
-                        if (!ok) break;
-                        a_phase[g] ^= 1u << kc;
-                        ptx::tc_fence_after();
-                        if (lane == 0) {
-                            const uint32_t d = tmem_base + (uint32_t)(g * 256 + (to_acc ? 128 : 0));
-                            // row m = (y*2 + b)*8 + x starts at slot (2 + 0)*9 + 1 = 19 for m = 0
-                            const uint32_t a_base = smem_base + kOffFrames + g * kFrameBytes + (2 * kc) * kPlaneBytes + (kNB * 9 + 1) * 16;
+                    ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
+                    if (!ok) break;
+                    a_phase ^= 1u << kc;
+                    ptx::tc_fence_after();
+                    const long long ti0 = tr ? clock64() : 0;
+                    if (lane == 0) {
+                        // low descriptor words in 16-byte units; row m = 0 sits at slot 2*9 + 1 = 19
+                        const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
+                        const uint32_t b_lo = ((smem_base + kOffWeights + stage * kStageBytes) >> 4) | kBDescLbo;
+                        const uint32_t first = (conv2 || kc > 0) ? 1u : 0u;
 #pragma unroll
-                            for (int tap = 0; tap < 9; ++tap) {
-                                const int dy = tap / 3 - 1, dx = tap % 3 - 1;
-                                const uint64_t adesc = ptx::smem_desc_kmajor_noswizzle(
-                                    a_base + (uint32_t)((dy * kNB * 9 + dx) * 16), kPlaneBytes, kRowGroupBytes);
-                                const uint64_t bdesc = ptx::smem_desc_kmajor_noswizzle(w_addr + tap * kTileBytes, 2048, 128);
-                                const uint32_t acc = (conv2 || kc > 0 || tap > 0) ? 1u : 0u;
-                                ptx::mma_bf16(d, adesc, bdesc, idesc, acc);
-                            }
-                            if (kc == nkc - 1) ptx::mma_commit(bar_acc_full(g));
+                        for (int tap = 0; tap < 9; ++tap) {
+                            const int dy = tap / 3 - 1, dx = tap % 3 - 1;
+                            ptx::mma_bf16_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                                b_lo + (uint32_t)(tap * (kTileBytes / 16)), kBDescHi, idesc,
+                                                tap == 0 ? first : 1u);
                         }
-                        __syncwarp();
+                        if (kc == nkc - 1) ptx::mma_commit(bar_acc_full(g));
+                        ptx::mma_commit(bar_w_empty(stage));
                     }
-                    if (!ok) break;
-                    if (lane == 0) ptx::mma_commit(bar_w_empty(stage));
                     __syncwarp();
+                    if (tr) t_issue += clock64() - ti0;
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -207,7 +237,7 @@ tower_tc_kernel(const TowerArgs args) {
             if (ptx::mbar_try_wait(bar_done, 0)) break;
     } else {
         // ================= epilogue: 4 warps per group =================
-        const int g = (warp - 2) >> 2;
+        const int g = (warp - 1 - kGroups) >> 2;
         const int q = warp & 3;                               // TMEM lane quarter this warp may access
         const int m = q * 32 + lane;                          // GEMM row = TMEM lane
         const int g8 = m >> 3, y = g8 >> 1, b = g8 & 1, x = m & 7;
@@ -235,30 +265,33 @@ tower_tc_kernel(const TowerArgs args) {
             for (int l = 0; l < n_conv && ok; ++l) {
                 const bool from_acc = (l & 1) == 1;
                 const bool last = l == n_conv - 1;
-                ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status);
+                ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 acc_phase ^= 1u;
                 ptx::tc_fence_after();
-                const float *bias = args.bias + (size_t)l * kC;
+                const float *bias = args.bias_in_smem ? reinterpret_cast<const float *>(smem + kOffBias) + l * kC
+                                                      : args.bias + (size_t)l * kC;
                 __nv_bfloat16 *dst = args.out + ((size_t)board * 64 + sq) * kC;
-#pragma unroll 1
+                const uint32_t t_src = t_lane + (uint32_t)(from_acc ? 128 : 0);
+                const bool keep_h = !from_acc && !last;        // the residual stream stays in TMEM as fp32
+                uint32_t r[2][16];
+                const int hk = args.trace;
+                if (!(hk & 8)) ptx::tmem_ld16(t_src, r[0]);
+#pragma unroll
                 for (int kc = 0; kc < kC / 16; ++kc) {
-                    uint32_t r[16];
-                    ptx::tmem_ld16(t_lane + (uint32_t)((from_acc ? 128 : 0) + kc * 16), r);
+                    if (!(hk & 8)) {
                     ptx::tmem_ld_wait();
+                    if (kc + 1 < kC / 16) ptx::tmem_ld16(t_src + (uint32_t)((kc + 1) * 16), r[(kc + 1) & 1]);
+                    }
+                    uint32_t(&rr)[16] = r[kc & 1];
                     float v[16];
 #pragma unroll
                     for (int i = 0; i < 16; i += 4) {
-                        const float4 bv = __ldg(reinterpret_cast<const float4 *>(bias + kc * 16 + i));
-                        v[i + 0] = fmaxf(__uint_as_float(r[i + 0]) + bv.x, 0.0f);
-                        v[i + 1] = fmaxf(__uint_as_float(r[i + 1]) + bv.y, 0.0f);
-                        v[i + 2] = fmaxf(__uint_as_float(r[i + 2]) + bv.z, 0.0f);
-                        v[i + 3] = fmaxf(__uint_as_float(r[i + 3]) + bv.w, 0.0f);
-                    }
-                    if (!from_acc && !last) {                  // keep the residual stream in fp32
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(v[i]);
-                        ptx::tmem_st16(t_lane + (uint32_t)(kc * 16), r);
+                        const float4 bv = *reinterpret_cast<const float4 *>(bias + kc * 16 + i);
+                        v[i + 0] = fmaxf(__uint_as_float(rr[i + 0]) + bv.x, 0.0f);
+                        v[i + 1] = fmaxf(__uint_as_float(rr[i + 1]) + bv.y, 0.0f);
+                        v[i + 2] = fmaxf(__uint_as_float(rr[i + 2]) + bv.z, 0.0f);
+                        v[i + 3] = fmaxf(__uint_as_float(rr[i + 3]) + bv.w, 0.0f);
                     }
                     uint32_t pk[8];
 #pragma unroll
@@ -272,19 +305,33 @@ tower_tc_kernel(const TowerArgs args) {
                             reinterpret_cast<uint4 *>(dst + kc * 16)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                         }
                     } else {
+                        if (!(hk & 16)) {
                         *reinterpret_cast<uint4 *>(frame + (2 * kc) * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         *reinterpret_cast<uint4 *>(frame + (2 * kc + 1) * kPlaneBytes + slot * 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                        if (!from_acc) ptx::tmem_st_wait();
-                        ptx::fence_proxy_async_smem();
+                        }
+                        if (keep_h && !(hk & 16)) {
+                            // fp32 copy back to H.  Its completion is awaited once, after the loop: the next
+                            // reader of H is the conv2 two layers on, whose MMAs are gated by barriers these
+                            // same threads arrive on only after that wait.
+                            uint32_t w[16];
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) w[i] = __float_as_uint(v[i]);
+                            ptx::tmem_st16(t_lane + (uint32_t)(kc * 16), w);
+                        }
+                        if (!(hk & 32)) ptx::fence_proxy_async_smem();
                         ptx::tc_fence_before();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(bar_a_ready(g, kc));
                     }
                 }
+                if (keep_h) ptx::tmem_st_wait();
             }
         }
     }
 
+    if (tr && lane == 0 && (warp < 4 || warp == 7))
+        printf("tower trace: warp %d total %lld clk, waited %lld / %lld / %lld clk, issue %lld clk\n", warp, clock64() - t_begin,
+               t_wait[0], t_wait[1], t_wait[2], t_issue);
     // ---- teardown
     ptx::tc_fence_before();
     __syncthreads();
@@ -333,7 +380,7 @@ int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_o
     if (dev < 64 && sm_count[dev] == 0) {
         int n = 0;
         AZ_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
-        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
     const int sms = dev < 64 ? sm_count[dev] : 148;
@@ -346,9 +393,13 @@ int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_o
     a.batch = batch;
     a.n_conv = net.n_conv;
     a.in_kc = net.in_pad / 16;
+    a.bias_in_smem = net.n_conv <= kMaxBiasLayers ? 1 : 0;
+    static const bool trace = getenv("AZ_TOWER_TRACE") != nullptr;
+    a.trace = trace ? atoi(getenv("AZ_TOWER_TRACE")) : 0;
+    const int smem_bytes = kSmemBytesNoBias + (a.bias_in_smem ? net.n_conv * kC * 4 : 0);
     const int n_units = (batch + kBoardsPerCta - 1) / kBoardsPerCta;
     const int grid = n_units < sms ? n_units : sms;
-    tower_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(a);
+    tower_tc_kernel<<<grid, kThreads, smem_bytes, s>>>(a);
     AZ_LAUNCH_CHECK();
     return AZ_OK;
 }
