@@ -143,6 +143,34 @@ int build_net(Net &n, const BlobView &v) {
         std::vector<float> bias((size_t)n.n_conv * C);
         for (int l = 0; l < n.n_conv; ++l) memcpy(&bias[(size_t)l * C], b[l], sizeof(float) * C);
         if ((rc = upload_f32(bias.data(), bias.size(), &n.tc_bias)) != AZ_OK) return rc;
+        // fused head projections and tensor-core fully-connected layers
+        const bool flat = a.policy_head == AZ_POLICY_FLAT1858;
+        const int n_policy = flat ? kHeadChannels : kPlanes73, n_policy_pad = flat ? kHeadChannels : 80;
+        n.tc_head_n = n_policy_pad + kHeadChannels;
+        std::vector<__nv_bfloat16> hw(tc_head_weight_bytes(n.tc_head_n) / sizeof(__nv_bfloat16));
+        tc_pack_head(v.p_w, flat ? v.p_s : nullptr, n_policy, n_policy_pad, v.v_cw, v.v_cs, C, hw.data());
+        AZ_CUDA(cudaMalloc(&n.tc_head_w, hw.size() * sizeof(__nv_bfloat16)));
+        AZ_CUDA(cudaMemcpy(n.tc_head_w, hw.data(), hw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
+        std::vector<float> hb(n.tc_head_n, 0.0f);
+        for (int i = 0; i < n_policy; ++i) hb[i] = v.p_b[i];
+        for (int i = 0; i < kHeadChannels; ++i) hb[n_policy_pad + i] = v.v_cb[i];
+        if ((rc = upload_f32(hb.data(), hb.size(), &n.tc_head_bias)) != AZ_OK) return rc;
+        {
+            std::vector<__nv_bfloat16> fw(fc_tc_weight_bytes(kValueHidden) / sizeof(__nv_bfloat16));
+            fc_tc_pack_weights(v.v_w1, kValueHidden, fw.data());
+            AZ_CUDA(cudaMalloc(&n.fc_value_w, fw.size() * sizeof(__nv_bfloat16)));
+            AZ_CUDA(cudaMemcpy(n.fc_value_w, fw.data(), fw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
+        }
+        if (flat) {
+            std::vector<__nv_bfloat16> fw(fc_tc_weight_bytes(kFlatMoves) / sizeof(__nv_bfloat16));
+            fc_tc_pack_weights(v.p_fw, kFlatMoves, fw.data());
+            AZ_CUDA(cudaMalloc(&n.fc_policy_w, fw.size() * sizeof(__nv_bfloat16)));
+            AZ_CUDA(cudaMemcpy(n.fc_policy_w, fw.data(), fw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
+        }
+        const size_t u_bytes = (size_t)((a.max_batch + 127) / 128) * kHeadChannels * 64 * 128 * sizeof(__nv_bfloat16);
+        AZ_CUDA(cudaMalloc(&n.u_value, u_bytes));
+        AZ_CUDA(cudaMemset(n.u_value, 0, u_bytes));
+        if (flat) { AZ_CUDA(cudaMalloc(&n.u_policy, u_bytes)); AZ_CUDA(cudaMemset(n.u_policy, 0, u_bytes)); }
         n.tc_ready = true;
     } else {
         if ((rc = upload_conv_simt(v.in_w, (int)a.in_planes, n.in_pad, C, n.bf16, &n.conv_w[0])) != AZ_OK) return rc;
@@ -162,20 +190,21 @@ int build_net(Net &n, const BlobView &v) {
 
     // heads
     const int V = a.value_head == AZ_VALUE_WDL ? 3 : 1;
+    const bool simt_heads = !n.tc_ready;      // the tensor-core path carries its own packed head weights
     if (a.policy_head == AZ_POLICY_PLANES73) {
-        if ((rc = upload_act(v.p_w, (size_t)kPlanes73 * C, n.bf16, &n.p_w)) != AZ_OK) return rc;
+        if (simt_heads && (rc = upload_act(v.p_w, (size_t)kPlanes73 * C, n.bf16, &n.p_w)) != AZ_OK) return rc;
         if ((rc = upload_f32(v.p_b, kPlanes73, &n.p_bias)) != AZ_OK) return rc;
     } else {
-        if ((rc = upload_act(v.p_w, (size_t)kHeadChannels * C, n.bf16, &n.p_w)) != AZ_OK) return rc;
+        if (simt_heads && (rc = upload_act(v.p_w, (size_t)kHeadChannels * C, n.bf16, &n.p_w)) != AZ_OK) return rc;
         if ((rc = upload_f32(v.p_s, kHeadChannels, &n.p_scale)) != AZ_OK) return rc;
         if ((rc = upload_f32(v.p_b, kHeadChannels, &n.p_bias)) != AZ_OK) return rc;
-        if ((rc = upload_act(v.p_fw, (size_t)kFlatMoves * kHeadChannels * 64, n.bf16, &n.p_fw)) != AZ_OK) return rc;
+        if (simt_heads && (rc = upload_act(v.p_fw, (size_t)kFlatMoves * kHeadChannels * 64, n.bf16, &n.p_fw)) != AZ_OK) return rc;
         if ((rc = upload_f32(v.p_fb, kFlatMoves, &n.p_fbias)) != AZ_OK) return rc;
     }
-    if ((rc = upload_act(v.v_cw, (size_t)kHeadChannels * C, n.bf16, &n.v_cw)) != AZ_OK) return rc;
+    if (simt_heads && (rc = upload_act(v.v_cw, (size_t)kHeadChannels * C, n.bf16, &n.v_cw)) != AZ_OK) return rc;
     if ((rc = upload_f32(v.v_cs, kHeadChannels, &n.v_cscale)) != AZ_OK) return rc;
     if ((rc = upload_f32(v.v_cb, kHeadChannels, &n.v_cbias)) != AZ_OK) return rc;
-    if ((rc = upload_act(v.v_w1, (size_t)kValueHidden * kHeadChannels * 64, n.bf16, &n.v_w1)) != AZ_OK) return rc;
+    if (simt_heads && (rc = upload_act(v.v_w1, (size_t)kValueHidden * kHeadChannels * 64, n.bf16, &n.v_w1)) != AZ_OK) return rc;
     if ((rc = upload_f32(v.v_b1, kValueHidden, &n.v_b1)) != AZ_OK) return rc;
     if ((rc = upload_f32(v.v_w2, (size_t)V * kValueHidden, &n.v_w2)) != AZ_OK) return rc;
     if ((rc = upload_f32(v.v_b2, V, &n.v_b2)) != AZ_OK) return rc;
@@ -196,7 +225,8 @@ int build_net(Net &n, const BlobView &v) {
 void free_net(Net *n) {
     if (!n) return;
     for (int i = 0; i < 1 + 2 * 64; ++i) { cudaFree(n->conv_w[i]); cudaFree(n->conv_scale[i]); cudaFree(n->conv_bias[i]); }
-    cudaFree(n->tc_weights); cudaFree(n->tc_bias);
+    cudaFree(n->tc_weights); cudaFree(n->tc_bias); cudaFree(n->tc_head_w); cudaFree(n->tc_head_bias);
+    cudaFree(n->fc_policy_w); cudaFree(n->fc_value_w); cudaFree(n->u_policy); cudaFree(n->u_value);
     cudaFree(n->p_w); cudaFree(n->p_scale); cudaFree(n->p_bias); cudaFree(n->p_fw); cudaFree(n->p_fbias);
     cudaFree(n->v_cw); cudaFree(n->v_cscale); cudaFree(n->v_cbias); cudaFree(n->v_w1); cudaFree(n->v_b1);
     cudaFree(n->v_w2); cudaFree(n->v_b2);
@@ -209,8 +239,9 @@ void free_net(Net *n) {
     delete n;
 }
 
-// encoder + tower; *tower_out receives the buffer holding [batch][64][C]
-int run_tower(Net &n, const void *positions, int batch, void **tower_out, cudaStream_t s) {
+// encoder + tower; *tower_out receives the buffer holding [batch][64][C].  With `fused_heads` (tensor-core
+// path only) the tower kernel also runs the 1x1 head projections and leaves the activations on chip.
+int run_tower(Net &n, const void *positions, int batch, void **tower_out, bool fused_heads, cudaStream_t s) {
     int rc = launch_encode(positions, az_position_bytes(&n.arch), batch, (int)n.arch.in_planes, n.in_pad,
                            n.bf16, n.planes, n.status_dev, s);
     if (rc != AZ_OK) return rc;
@@ -218,8 +249,8 @@ int run_tower(Net &n, const void *positions, int batch, void **tower_out, cudaSt
     const bool timed = n.profile && n.n_events < kMaxProfiledPasses;
     if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
     if (n.tc_ready) {
-        *tower_out = n.act[0];
-        rc = launch_tower_tc(n, n.planes, batch, n.act[0], s);
+        *tower_out = fused_heads ? nullptr : n.act[0];
+        rc = launch_tower_tc(n, n.planes, batch, *tower_out, fused_heads, s);
         if (rc == AZ_OK && timed) AZ_CUDA(cudaEventRecord(n.ev_end[n.n_events++], s));
         return rc;
     }
@@ -292,7 +323,7 @@ int az_tower(az_net *net, const void *positions_dev, int batch, void *tower_dev,
     if (batch == 0) return AZ_OK;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     void *x = nullptr;
-    int rc = az::run_tower(*n, positions_dev, batch, &x, s);
+    int rc = az::run_tower(*n, positions_dev, batch, &x, false, s);
     if (rc != AZ_OK) return rc;
     AZ_CUDA(cudaMemcpyAsync(tower_dev, x, (size_t)batch * 64 * n->arch.channels * az::act_bytes(*n),
                             cudaMemcpyDeviceToDevice, s));
@@ -313,8 +344,16 @@ int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_ma
     const az_arch &a = n->arch;
     const int C = (int)a.channels;
     void *h = nullptr;
-    int rc = az::run_tower(*n, positions_dev, batch, &h, s);
+    int rc = az::run_tower(*n, positions_dev, batch, &h, n->tc_ready, s);
     if (rc != AZ_OK) return rc;
+    if (n->tc_ready) {
+        // the tower kernel has produced the 73-plane logits or the flat head's projection, and the value
+        // projection; one GEMM launch finishes both heads, the softmax follows
+        rc = az::launch_fc_tc(*n, batch, value_dev, s);
+        if (rc != AZ_OK) return rc;
+        return az::launch_masked_softmax(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a), (int)az_mask_words(&a),
+                                         policy_dev, n->status_dev, s);
+    }
     if (a.policy_head == AZ_POLICY_PLANES73) {
         rc = az::launch_conv1x1(h, n->p_w, nullptr, n->p_bias, batch, C, az::kPlanes73, false, n->bf16, n->logits, true, s);
         if (rc != AZ_OK) return rc;
@@ -421,9 +460,9 @@ int az_device_status(az_net *net, void *cuda_stream, uint32_t *status_out) {
 int az_launches_per_evaluate(const az_net *net, int batch) {
     const Net *n = reinterpret_cast<const Net *>(net);
     if (!n || batch <= 0) return 0;
-    const int tower = n->tc_ready ? az::tower_tc_launch_count() : n->n_conv;
+    if (n->tc_ready) return 1 /*encode*/ + az::tower_tc_launch_count() + 1 /*head GEMMs*/ + 1 /*softmax*/;
     const int policy = n->arch.policy_head == AZ_POLICY_PLANES73 ? 1 : 2;
-    return 1 /*encode*/ + tower + policy + 3 /*value*/ + 1 /*softmax*/;
+    return 1 /*encode*/ + n->n_conv + policy + 3 /*value*/ + 1 /*softmax*/;
 }
 
 const char *az_strerror(int code) {

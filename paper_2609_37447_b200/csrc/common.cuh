@@ -44,6 +44,13 @@ struct Net {
     void *tc_weights = nullptr;       // packed UMMA B-operand tiles, all layers
     float *tc_bias = nullptr;         // [n_conv][C] folded bias (scales are folded into the weights)
     bool tc_ready = false;
+    void *tc_head_w = nullptr;        // packed 1x1 head projections (policy | value), fused into the tower kernel
+    float *tc_head_bias = nullptr;
+    int tc_head_n = 0;                // 64 (flat policy head) or 112 (73-plane policy head)
+    void *fc_policy_w = nullptr;      // flat policy FC as GEMM B tiles (K permuted to square*32 + channel)
+    void *fc_value_w = nullptr;       // value FC1 as GEMM B tiles
+    void *u_policy = nullptr;         // head projections as GEMM A tiles [ceil(B/128)][256][16][8][8] bf16
+    void *u_value = nullptr;
 
     // ---- heads ----
     void *p_w = nullptr;              // planes73: [73][C]; flat: 1x1 conv [32][C]      (activation type)
@@ -111,7 +118,15 @@ int launch_masked_softmax(const float *logits, const uint64_t *masks, int batch,
 size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv);
 void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
                      int channels, int n_conv, __nv_bfloat16 *packed_host);
-int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, cudaStream_t s);
+int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, bool with_heads, cudaStream_t s);
 int tower_tc_launch_count();
+size_t tc_head_weight_bytes(int head_n);
+void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,
+                  int channels, __nv_bfloat16 *packed);
+
+// tensor-core fully-connected layers of the heads (fc_tc.cu)
+size_t fc_tc_weight_bytes(int n);
+void fc_tc_pack_weights(const float *w, int n, __nv_bfloat16 *packed);     // w[n][32*64], K permuted to square*32 + channel
+int launch_fc_tc(const Net &net, int batch, float *value_out, cudaStream_t s);
 
 }  // namespace az

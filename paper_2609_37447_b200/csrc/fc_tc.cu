@@ -1,0 +1,260 @@
+// Fully-connected layers of the heads on tcgen05 tensor cores (Sec. 4.3.1 dense policy head: a
+// small spatial projection flattened into the move logits; Sec. 4.3.4 / App. D.1 value head:
+// flatten, hidden layer, three logits, softmax giving win/draw/loss, or one tanh scalar).
+//
+//   policy  logits[b][n] = sum_k U_p[b][k] * Wp[n][k] + bp[n]          n < 1858, k < 2048
+//   value   hidden[b][j] = relu(sum_k U_v[b][k] * W1[j][k] + b1[j])    j < 128, then the 128 -> 1|3
+//           tail and tanh / softmax, all inside the epilogue of the value tile.
+//
+// One CTA per 128 x 128 output tile (blockIdx.x: the policy's column tiles, then one value tile;
+// blockIdx.y: tiles of 128 positions).  Both operands are bf16 and already sit in global memory
+// as ready-made no-swizzle K-major core-matrix tiles (the tower kernel writes U that way, the
+// weights are packed at load), so a pipeline stage of 64 k is two contiguous 16 KB bulk copies.
+// K runs over square*32 + channel; the weights are permuted to match at load time.
+// Bound: L2 -> shared-memory operand traffic (each CTA streams 1 MB for 4.3 us of MMA work).
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace az {
+namespace {
+
+constexpr int kK = kHeadChannels * 64;         // 2048
+constexpr int kStageK = 64;
+constexpr int kNumKStages = kK / kStageK;      // 32
+constexpr int kOperandStageBytes = 128 * kStageK * 2;   // 16384
+constexpr int kStages = 5;
+constexpr int kThreads = 32 * 6;               // producer, issuer, 4 epilogue warps
+constexpr uint32_t kTmemCols = 128;
+constexpr uint32_t kSpinLimit = 1u << 24;
+
+constexpr int kOffA = 0;
+constexpr int kOffB = kStages * kOperandStageBytes;
+constexpr int kOffBars = 2 * kStages * kOperandStageBytes;      // full[5], empty[5], acc
+constexpr int kOffTmemPtr = kOffBars + (2 * kStages + 1) * 8;
+constexpr int kOffAbort = kOffTmemPtr + 4;
+constexpr int kOffTail = (kOffAbort + 4 + 15) & ~15;           // value tail weights: w2[3][128], b2[3]
+constexpr int kSmemBytes = kOffTail + (3 * kValueHidden + 4) * 4;
+
+struct FcArgs {
+    const __nv_bfloat16 *u_policy, *u_value;    // A tiles [m_tile][256][16][8][8]
+    const __nv_bfloat16 *w_policy, *w_value;    // B tiles [n_tile][256][16][8][8]
+    const float *b_policy, *b_value;            // [1858], [128]
+    const float *w2, *b2;                       // value tail [V][128], [V]
+    float *logits;                              // [batch][1858]
+    float *value;                               // [batch][V]
+    uint32_t *status;
+    int batch, n_policy, n_policy_tiles, wdl;
+};
+
+__device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status) {
+    bool done = false;
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (ptx::mbar_try_wait(bar, parity)) { done = true; break; }
+        if ((i & 63u) == 63u && *abort_flag) break;
+    }
+    if (!done && !*abort_flag) {
+        *abort_flag = 1;
+        atomicOr(status, kStatusWaitTimeout);
+    }
+    return __all_sync(0xffffffffu, done);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+fc_tc_kernel(const FcArgs args) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t smem_base = ptx::smem_addr(smem);
+    const uint32_t bars = smem_base + kOffBars;
+    auto bar_full = [&](int s) { return bars + 8u * s; };
+    auto bar_empty = [&](int s) { return bars + 8u * (kStages + s); };
+    const uint32_t bar_acc = bars + 8u * (2 * kStages);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffAbort);
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + kOffTmemPtr);
+    float *tail = reinterpret_cast<float *>(smem + kOffTail);
+
+    const bool is_value = (int)blockIdx.x == args.n_policy_tiles;
+    const int n_tile = is_value ? 0 : blockIdx.x;
+    const int m_tile = blockIdx.y;
+    const int V = args.wdl ? 3 : 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { ptx::mbar_init(bar_full(s), 1); ptx::mbar_init(bar_empty(s), 1); }
+        ptx::mbar_init(bar_acc, 1);
+        *abort_flag = 0;
+        ptx::fence_barrier_init();
+    }
+    if (is_value)
+        for (int i = threadIdx.x; i < V * kValueHidden + V; i += kThreads)
+            tail[i] = i < V * kValueHidden ? args.w2[i] : args.b2[i - V * kValueHidden];
+    if (warp == 0) {
+        ptx::tmem_alloc(ptx::smem_addr(tmem_ptr_smem), kTmemCols);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_ptr_smem;
+
+    if (warp == 0) {
+        // ---- producer: two 16 KB bulk copies per stage
+        const unsigned char *a_src = reinterpret_cast<const unsigned char *>(is_value ? args.u_value : args.u_policy) +
+                                     (size_t)m_tile * (kK * 128 * 2);
+        const unsigned char *b_src = reinterpret_cast<const unsigned char *>(is_value ? args.w_value : args.w_policy) +
+                                     (size_t)n_tile * (kK * 128 * 2);
+        bool ok = true;
+        int issued = 0;
+        for (int ks = 0; ks < kNumKStages; ++ks) {
+            const int s = ks % kStages;
+            ok = wait_bar(bar_empty(s), ((ks / kStages) & 1) ^ 1u, abort_flag, args.status);
+            if (!ok) break;
+            if (lane == 0) {
+                ptx::mbar_arrive_expect_tx(bar_full(s), 2 * kOperandStageBytes);
+                ptx::bulk_copy_g2s(smem_base + kOffA + s * kOperandStageBytes, a_src + (size_t)ks * kOperandStageBytes, kOperandStageBytes, bar_full(s));
+                ptx::bulk_copy_g2s(smem_base + kOffB + s * kOperandStageBytes, b_src + (size_t)ks * kOperandStageBytes, kOperandStageBytes, bar_full(s));
+            }
+            issued = ks + 1;
+            __syncwarp();
+        }
+        if (!ok)   // let copies in flight land before the shared memory is released
+            for (int ks = issued > kStages ? issued - kStages : 0; ks < issued; ++ks)
+                for (uint32_t i = 0; i < (1u << 20); ++i)
+                    if (ptx::mbar_try_wait(bar_full(ks % kStages), (ks / kStages) & 1)) break;
+    } else if (warp == 1) {
+        // ---- MMA issuer: four K=16 steps per stage
+        constexpr uint32_t idesc = ptx::idesc_bf16_f32(128, 128);
+        constexpr uint32_t desc_hi = (uint32_t)(128 >> 4) | (1u << 14);        // 8-row groups 128 B apart
+        constexpr uint32_t lbo = (uint32_t)(2048 >> 4) << 16;                  // K core matrices 2048 B apart
+        bool ok = true;
+        for (int ks = 0; ks < kNumKStages && ok; ++ks) {
+            const int s = ks % kStages;
+            ok = wait_bar(bar_full(s), (ks / kStages) & 1, abort_flag, args.status);
+            if (!ok) break;
+            ptx::tc_fence_after();
+            if (lane == 0) {
+                const uint32_t a_lo = ((smem_base + kOffA + s * kOperandStageBytes) >> 4) | lbo;
+                const uint32_t b_lo = ((smem_base + kOffB + s * kOperandStageBytes) >> 4) | lbo;
+#pragma unroll
+                for (int j = 0; j < kStageK / 16; ++j)
+                    ptx::mma_bf16_split(tmem_base, a_lo + (uint32_t)(j * 256), desc_hi, b_lo + (uint32_t)(j * 256), desc_hi, idesc,
+                                        (ks > 0 || j > 0) ? 1u : 0u);
+                ptx::mma_commit(bar_empty(s));
+                if (ks == kNumKStages - 1) ptx::mma_commit(bar_acc);
+            }
+            __syncwarp();
+        }
+        if (!ok && lane == 0) ptx::mma_commit(bar_acc);      // lets the epilogue's bounded wait end early
+    } else {
+        // ---- epilogue
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const int m = m_tile * 128 + row;
+        const bool live = m < args.batch;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
+        bool ok = wait_bar(bar_acc, 0, abort_flag, args.status);
+        ptx::tc_fence_after();
+        if (ok) {
+            float z[3] = {0.0f, 0.0f, 0.0f};
+#pragma unroll 1
+            for (int j = 0; j < 8; ++j) {
+                uint32_t r[16];
+                ptx::tmem_ld16(t_lane + (uint32_t)(j * 16), r);
+                ptx::tmem_ld_wait();
+                if (is_value) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int n = j * 16 + i;
+                        const float h = fmaxf(__uint_as_float(r[i]) + __ldg(args.b_value + n), 0.0f);
+                        z[0] = fmaf(tail[n], h, z[0]);
+                        if (V == 3) { z[1] = fmaf(tail[kValueHidden + n], h, z[1]); z[2] = fmaf(tail[2 * kValueHidden + n], h, z[2]); }
+                    }
+                } else if (live) {
+                    float *dst = args.logits + (size_t)m * args.n_policy;
+#pragma unroll
+                    for (int i = 0; i < 16; i += 2) {
+                        const int n = n_tile * 128 + j * 16 + i;
+                        if (n + 1 < args.n_policy) {
+                            const float2 v = make_float2(__uint_as_float(r[i]) + __ldg(args.b_policy + n),
+                                                         __uint_as_float(r[i + 1]) + __ldg(args.b_policy + n + 1));
+                            *reinterpret_cast<float2 *>(dst + n) = v;
+                        } else if (n < args.n_policy) {
+                            dst[n] = __uint_as_float(r[i]) + __ldg(args.b_policy + n);
+                        }
+                    }
+                }
+            }
+            if (is_value && live) {
+                const float *b2 = tail + V * kValueHidden;
+                if (V == 1) args.value[m] = tanhf(z[0] + b2[0]);
+                else {
+                    const float a = z[0] + b2[0], b = z[1] + b2[1], c = z[2] + b2[2];
+                    const float mx = fmaxf(a, fmaxf(b, c));
+                    const float e0 = expf(a - mx), e1 = expf(b - mx), e2 = expf(c - mx);
+                    const float inv = 1.0f / (e0 + e1 + e2);
+                    args.value[(size_t)m * 3 + 0] = e0 * inv;
+                    args.value[(size_t)m * 3 + 1] = e1 * inv;
+                    args.value[(size_t)m * 3 + 2] = e2 * inv;
+                }
+            }
+        }
+    }
+    ptx::tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+}  // namespace
+
+size_t fc_tc_weight_bytes(int n) { return (size_t)((n + 127) / 128) * kK * 128 * 2; }
+
+// w[n][2048] with the input flattened channel-major (channel*64 + square)  ->  128-row tiles
+// [tile][8-wide K chunk (256)][row group (16)][row (8)][k (8)] with K = square*32 + channel.
+void fc_tc_pack_weights(const float *w, int n, __nv_bfloat16 *packed) {
+    const int tiles = (n + 127) / 128;
+    __nv_bfloat16 *dst = packed;
+    for (int t = 0; t < tiles; ++t)
+        for (int kc8 = 0; kc8 < kK / 8; ++kc8)
+            for (int ng = 0; ng < 16; ++ng)
+                for (int r = 0; r < 8; ++r)
+                    for (int e = 0; e < 8; ++e) {
+                        const int row = t * 128 + ng * 8 + r, k = kc8 * 8 + e;
+                        const int sq = k / kHeadChannels, c = k % kHeadChannels;
+                        *dst++ = __float2bfloat16_rn(row < n ? w[(size_t)row * kK + c * 64 + sq] : 0.0f);
+                    }
+}
+
+int launch_fc_tc(const Net &net, int batch, float *value_out, cudaStream_t s) {
+    if (batch == 0) return AZ_OK;
+    static bool configured[64] = {};
+    int dev = 0;
+    AZ_CUDA(cudaGetDevice(&dev));
+    if (dev < 64 && !configured[dev]) {
+        AZ_CUDA(cudaFuncSetAttribute(fc_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        configured[dev] = true;
+    }
+    const bool flat = net.arch.policy_head == AZ_POLICY_FLAT1858;
+    FcArgs a;
+    a.u_policy = static_cast<const __nv_bfloat16 *>(net.u_policy);
+    a.u_value = static_cast<const __nv_bfloat16 *>(net.u_value);
+    a.w_policy = static_cast<const __nv_bfloat16 *>(net.fc_policy_w);
+    a.w_value = static_cast<const __nv_bfloat16 *>(net.fc_value_w);
+    a.b_policy = net.p_fbias;
+    a.b_value = net.v_b1;
+    a.w2 = net.v_w2;
+    a.b2 = net.v_b2;
+    a.logits = net.logits;
+    a.value = value_out;
+    a.status = net.status_dev;
+    a.batch = batch;
+    a.n_policy = kFlatMoves;
+    a.n_policy_tiles = flat ? (kFlatMoves + 127) / 128 : 0;
+    a.wdl = net.arch.value_head == AZ_VALUE_WDL;
+    dim3 grid((unsigned)(a.n_policy_tiles + 1), (unsigned)((batch + 127) / 128));
+    fc_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(a);
+    AZ_LAUNCH_CHECK();
+    return AZ_OK;
+}
+
+}  // namespace az

@@ -84,6 +84,13 @@ struct TowerArgs {
     int in_kc;                       // 16-channel slices of the input layer (2)
     int bias_in_smem;                // all biases staged in shared memory (n_conv <= kMaxBiasLayers)
     int trace;                       // CTA 0 prints how long each role waited (debugging aid)
+    // fused 1x1 head projections (one extra MMA layer on the final activations); head_n == 0: none
+    int head_n;                      // 64: flat policy proj (32) | value proj (32); 112: 73 policy planes (+7 pad) | value proj (32)
+    const __nv_bfloat16 *head_w;     // packed [kc 8][k8 2][n-group head_n/8][8][8]
+    const float *head_bias;          // [head_n]
+    __nv_bfloat16 *u_policy;         // flat head: projection as GEMM A tiles, K index = square*32 + channel
+    __nv_bfloat16 *u_value;          // value projection, same layout
+    float *logits;                   // 73-plane head: [batch][73*64] fp32 logits, index = plane*64 + square
 };
 
 // Bounded wait, called by all 32 lanes of a warp together.  Returns false (to every lane alike) if
@@ -121,9 +128,12 @@ tower_tc_kernel(const TowerArgs args) {
     // ---- set-up: zero the frames (their borders stay zero for the kernel's lifetime), barriers, TMEM
     for (int i = threadIdx.x; i < kGroups * kFrameBytes / 16; i += kThreads)
         reinterpret_cast<uint4 *>(smem + kOffFrames)[i] = make_uint4(0, 0, 0, 0);
-    if (args.bias_in_smem)
+    if (args.bias_in_smem) {
         for (int i = threadIdx.x; i < args.n_conv * kC; i += kThreads)
             reinterpret_cast<float *>(smem + kOffBias)[i] = args.bias[i];
+        for (int i = threadIdx.x; i < args.head_n; i += kThreads)
+            reinterpret_cast<float *>(smem + kOffBias)[args.n_conv * kC + i] = args.head_bias[i];
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { ptx::mbar_init(bar_w_full(s), 1); ptx::mbar_init(bar_w_empty(s), kGroups); }
         for (int g = 0; g < kGroups; ++g) {
@@ -146,6 +156,7 @@ tower_tc_kernel(const TowerArgs args) {
 
     const int n_units = (args.batch + kBoardsPerCta - 1) / kBoardsPerCta;
     const int n_conv = args.n_conv;
+    const int head_n = args.head_n;
     const bool tr = args.trace && blockIdx.x == 0;
     long long t_wait[3] = {0, 0, 0};
     long long t_issue = 0;
@@ -166,17 +177,25 @@ tower_tc_kernel(const TowerArgs args) {
                     ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                     if (!ok) break;
                     if (lane == 0) {
-                        if (args.trace & 4) ptx::mbar_arrive(bar_w_full(stage));
-                        else {
                         ptx::mbar_arrive_expect_tx(bar_w_full(stage), kStageBytes);
                         ptx::bulk_copy_g2s(smem_base + kOffWeights + stage * kStageBytes, src, kStageBytes, bar_w_full(stage));
-                        }
                     }
                     issued[stage] = true; last_parity[stage] = phase;
                     src += kStageBytes;
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     __syncwarp();
                 }
+            }
+            if (head_n && ok) {                              // the head projections: one small stage
+                ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+                if (!ok) break;
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(bar_w_full(stage), (uint32_t)head_n * 256u);
+                    ptx::bulk_copy_g2s(smem_base + kOffWeights + stage * kStageBytes, args.head_w, (uint32_t)head_n * 256u, bar_w_full(stage));
+                }
+                issued[stage] = true; last_parity[stage] = phase;
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                __syncwarp();
             }
         }
         if (!ok) {
@@ -196,7 +215,17 @@ tower_tc_kernel(const TowerArgs args) {
         bool ok = true;
         const uint32_t d_h = tmem_base + (uint32_t)(g * 256);
         const uint32_t frame_lo = (((smem_base + kOffFrames + g * kFrameBytes) >> 4) + (uint32_t)(kNB * 9 + 1)) | kADescLbo;
+        const int n_layers = n_conv + (head_n ? 1 : 0);
+        uint32_t lead_parity = 0;                                      // parity of group 0's next layer-0 completion
         for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+            if (g == 1 && n_conv >= 3 && !(args.trace & 2)) {
+                // Start one (short) input layer behind group 0.  The groups then reach their layer
+                // boundaries at different times, so one group's wait for its epilogue is covered by
+                // the other's MMAs instead of idling the tensor pipe for both at once.
+                ok = wait_bar(bar_acc_full(0), lead_parity, abort_flag, args.status, tr ? &t_wait[2] : nullptr);
+                if (!ok) break;
+                lead_parity ^= (uint32_t)(n_layers & 1);
+            }
             for (int l = 0; l < n_conv && ok; ++l) {
                 const int nkc = l == 0 ? args.in_kc : kC / 16;
                 const bool conv2 = l >= 2 && (l & 1) == 0;             // accumulates onto the residual stream
@@ -228,6 +257,27 @@ tower_tc_kernel(const TowerArgs args) {
                     if (tr) t_issue += clock64() - ti0;
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
+            }
+            if (head_n && ok) {
+                // head projections: a 1x1 convolution = the centre tap only, N = head_n, into the ACC columns
+                const uint32_t idesc_h = ptx::idesc_bf16_f32(128, head_n);
+                ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+                if (!ok) break;
+                for (int kc = 0; kc < kC / 16; ++kc) {
+                    ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
+                    if (!ok) break;
+                    a_phase ^= 1u << kc;
+                    ptx::tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
+                        const uint32_t b_lo = (((smem_base + kOffWeights + stage * kStageBytes) >> 4) + (uint32_t)(kc * head_n * 2)) |
+                                              ((uint32_t)head_n << 16);          // K core matrices head_n*16 bytes apart
+                        ptx::mma_bf16_split(d_h + 128u, a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u);
+                        if (kc == kC / 16 - 1) { ptx::mma_commit(bar_acc_full(g)); ptx::mma_commit(bar_w_empty(stage)); }
+                    }
+                    __syncwarp();
+                }
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
         }
         // all issued MMAs must have completed before TMEM is freed
@@ -264,7 +314,8 @@ tower_tc_kernel(const TowerArgs args) {
             }
             for (int l = 0; l < n_conv && ok; ++l) {
                 const bool from_acc = (l & 1) == 1;
-                const bool last = l == n_conv - 1;
+                const bool last = l == n_conv - 1 && head_n == 0;        // nothing follows: results go to global only
+                const bool to_global = l == n_conv - 1 && args.out != nullptr;
                 ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 acc_phase ^= 1u;
@@ -273,16 +324,13 @@ tower_tc_kernel(const TowerArgs args) {
                                                       : args.bias + (size_t)l * kC;
                 __nv_bfloat16 *dst = args.out + ((size_t)board * 64 + sq) * kC;
                 const uint32_t t_src = t_lane + (uint32_t)(from_acc ? 128 : 0);
-                const bool keep_h = !from_acc && !last;        // the residual stream stays in TMEM as fp32
+                const bool keep_h = !from_acc && l != n_conv - 1;   // the residual stream stays in TMEM as fp32
                 uint32_t r[2][16];
-                const int hk = args.trace;
-                if (!(hk & 8)) ptx::tmem_ld16(t_src, r[0]);
+                ptx::tmem_ld16(t_src, r[0]);
 #pragma unroll
                 for (int kc = 0; kc < kC / 16; ++kc) {
-                    if (!(hk & 8)) {
                     ptx::tmem_ld_wait();
                     if (kc + 1 < kC / 16) ptx::tmem_ld16(t_src + (uint32_t)((kc + 1) * 16), r[(kc + 1) & 1]);
-                    }
                     uint32_t(&rr)[16] = r[kc & 1];
                     float v[16];
 #pragma unroll
@@ -299,17 +347,14 @@ tower_tc_kernel(const TowerArgs args) {
                         const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
                         pk[i] = *reinterpret_cast<const uint32_t *>(&h2);
                     }
-                    if (last) {
-                        if (live) {
-                            reinterpret_cast<uint4 *>(dst + kc * 16)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                            reinterpret_cast<uint4 *>(dst + kc * 16)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                        }
-                    } else {
-                        if (!(hk & 16)) {
+                    if (to_global && live) {
+                        reinterpret_cast<uint4 *>(dst + kc * 16)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        reinterpret_cast<uint4 *>(dst + kc * 16)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    }
+                    if (!last) {
                         *reinterpret_cast<uint4 *>(frame + (2 * kc) * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         *reinterpret_cast<uint4 *>(frame + (2 * kc + 1) * kPlaneBytes + slot * 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                        }
-                        if (keep_h && !(hk & 16)) {
+                        if (keep_h) {
                             // fp32 copy back to H.  Its completion is awaited once, after the loop: the next
                             // reader of H is the conv2 two layers on, whose MMAs are gated by barriers these
                             // same threads arrive on only after that wait.
@@ -318,13 +363,56 @@ tower_tc_kernel(const TowerArgs args) {
                             for (int i = 0; i < 16; ++i) w[i] = __float_as_uint(v[i]);
                             ptx::tmem_st16(t_lane + (uint32_t)(kc * 16), w);
                         }
-                        if (!(hk & 32)) ptx::fence_proxy_async_smem();
+                        ptx::fence_proxy_async_smem();
                         ptx::tc_fence_before();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(bar_a_ready(g, kc));
                     }
                 }
                 if (keep_h) ptx::tmem_st_wait();
+            }
+            if (head_n && ok) {
+                // ---- head projections out of the ACC columns
+                ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+                if (!ok) break;
+                acc_phase ^= 1u;
+                ptx::tc_fence_after();
+                const float *hb = args.bias_in_smem ? reinterpret_cast<const float *>(smem + kOffBias) + n_conv * kC : args.head_bias;
+                // this row's place in the GEMM A tiles: [tile of 128 boards][8-wide K chunk][board/8][board%8][8 k]
+                const size_t u_row = ((size_t)(board >> 7) * 256 * 16 + (size_t)((board & 127) >> 3)) * 128 + (size_t)(board & 7) * 16;
+                const int n_slices = head_n / 16;
+                const int value_slice0 = n_slices - 2;               // the value projection is the last 32 columns
+#pragma unroll 1
+                for (int j = 0; j < n_slices; ++j) {
+                    uint32_t rr[16];
+                    ptx::tmem_ld16(t_lane + 128u + (uint32_t)(j * 16), rr);
+                    ptx::tmem_ld_wait();
+                    float v[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(rr[i]) + hb[j * 16 + i];
+                    if (!live) {
+                        // rows past the end of the batch produce nothing
+                    } else if (head_n == 112 && j < value_slice0) {
+                        // 73 policy planes: raw logits, index = plane*64 + square
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const int plane = j * 16 + i;
+                            if (plane < kPlanes73) args.logits[(size_t)board * (kPlanes73 * 64) + plane * 64 + sq] = v[i];
+                        }
+                    } else {
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(fmaxf(v[2 * i], 0.0f), fmaxf(v[2 * i + 1], 0.0f));
+                            pk[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                        }
+                        const bool is_value = j >= value_slice0;
+                        const int c8 = 2 * (is_value ? j - value_slice0 : j);       // 8-channel chunk within the 32
+                        unsigned char *u = reinterpret_cast<unsigned char *>(is_value ? args.u_value : args.u_policy) + u_row;
+                        *reinterpret_cast<uint4 *>(u + (size_t)(sq * 4 + c8) * 2048) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        *reinterpret_cast<uint4 *>(u + (size_t)(sq * 4 + c8 + 1) * 2048) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    }
+                }
             }
         }
     }
@@ -372,7 +460,29 @@ void tc_pack_weights(const float *const *w, const float *const *scale, int in_pl
 
 int tower_tc_launch_count() { return 1; }
 
-int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, cudaStream_t s) {
+// Head projections as one N = head_n tile per 16-channel slice: rows [0, n_policy) the policy
+// projection (scaled where it has a folded batch-norm), zero rows up to n_policy_pad, then the 32
+// rows of the value projection.  Same core-matrix order as the tower's weight tiles.
+size_t tc_head_weight_bytes(int head_n) { return (size_t)head_n * 256; }
+
+void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,
+                  int channels, __nv_bfloat16 *packed) {
+    const int head_n = n_policy_pad + kHeadChannels;
+    __nv_bfloat16 *dst = packed;
+    for (int kc = 0; kc < channels / 16; ++kc)
+        for (int k8 = 0; k8 < 2; ++k8)
+            for (int ng = 0; ng < head_n / 8; ++ng)
+                for (int r = 0; r < 8; ++r)
+                    for (int e = 0; e < 8; ++e) {
+                        const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
+                        float v = 0.0f;
+                        if (n < n_policy) v = (sp ? sp[n] : 1.0f) * wp[(size_t)n * channels + ci];
+                        else if (n >= n_policy_pad) v = sv[n - n_policy_pad] * wv[(size_t)(n - n_policy_pad) * channels + ci];
+                        *dst++ = __float2bfloat16_rn(v);
+                    }
+}
+
+int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, bool with_heads, cudaStream_t s) {
     if (batch == 0) return AZ_OK;
     static int sm_count[64] = {};
     int dev = 0;
@@ -393,10 +503,16 @@ int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_o
     a.batch = batch;
     a.n_conv = net.n_conv;
     a.in_kc = net.in_pad / 16;
-    a.bias_in_smem = net.n_conv <= kMaxBiasLayers ? 1 : 0;
+    a.head_n = with_heads ? net.tc_head_n : 0;
+    a.head_w = static_cast<const __nv_bfloat16 *>(net.tc_head_w);
+    a.head_bias = net.tc_head_bias;
+    a.u_policy = static_cast<__nv_bfloat16 *>(net.u_policy);
+    a.u_value = static_cast<__nv_bfloat16 *>(net.u_value);
+    a.logits = net.logits;
+    a.bias_in_smem = net.n_conv + 1 <= kMaxBiasLayers ? 1 : 0;
     static const bool trace = getenv("AZ_TOWER_TRACE") != nullptr;
     a.trace = trace ? atoi(getenv("AZ_TOWER_TRACE")) : 0;
-    const int smem_bytes = kSmemBytesNoBias + (a.bias_in_smem ? net.n_conv * kC * 4 : 0);
+    const int smem_bytes = kSmemBytesNoBias + (a.bias_in_smem ? (net.n_conv + 1) * kC * 4 : 0);
     const int n_units = (batch + kBoardsPerCta - 1) / kBoardsPerCta;
     const int grid = n_units < sms ? n_units : sms;
     tower_tc_kernel<<<grid, kThreads, smem_bytes, s>>>(a);

@@ -177,17 +177,16 @@ def test_c2_bf16_batch_256(az):
     az.az_free_net(net)
 
 
-def test_c3_bf16_batch_1024_full_launch_sampled_oracle(az):
-    # the launch configuration the benchmark times (batch 1024); the oracle checks a sample of rows
+def test_c3_bf16_batch_1024_full_launch(az):
+    # the launch configuration the benchmark times (batch 1024); the oracle evaluates every row
+    # (a few seconds on the host cores), so the arg-max agreement is taken over 1024 positions
     cfg = configs.CONFIGS["c3"]
     net, blob = load(az, cfg)
     recs = positions.cur_records(positions.for_config(cfg))
     mg, pg, vg = gpu_evaluate(az, net, cfg, recs)
-    sample = np.concatenate([np.arange(0, 1024, 7), np.arange(1016, 1024)])
-    mo, _, po, vo = oracle.evaluate(blob, recs[sample], cfg.in_planes, cfg.policy_head)
-    agree = compare(cfg, mg[sample], pg[sample], vg[sample], mo, po, vo, TOL[1])
+    mo, _, po, vo = oracle.evaluate(blob, recs, cfg.in_planes, cfg.policy_head)
+    agree = compare(cfg, mg, pg, vg, mo, po, vo, TOL[1])
     assert agree >= 0.99
-    # properties that hold for every row
     assert np.abs(pg.sum(axis=1) - 1).max() < 1e-3 and np.abs(vg.sum(axis=1) - 1).max() < 1e-5
     assert az.az_device_status(net) == 0
     az.az_free_net(net)
