@@ -32,9 +32,13 @@ WORKLOADS = {
 }
 DTYPE = {0: "f32", 1: "bf16", 2: "fp8_e4m3"}
 
-# DRAM bytes (read + write) of one tower-kernel launch at batch 1024 from an ncu capture; the
-# summary the figure comes from is profiles/tower_tc_kernel_c3.md.  None until captured.
-TOWER_TRAFFIC_BYTES = {"c3": None, "c2": None}
+# DRAM bytes (read + write) of one tower-kernel launch, from the ncu capture summarised in
+# profiles/tower_tc_kernel_c3_batch592.md: 14.38 MB at batch 592, of which 11.87 MB are the weights
+# (read once whatever the batch) and the rest 4 KB of encoded planes per position.
+def tower_traffic_bytes(cfg, batch):
+    if cfg.channels != 128 or cfg.blocks != 20 or cfg.precision != 1:
+        return None
+    return 14.38e6 + (batch - 592) * 4096.0
 
 
 def tower_flops_per_position(cfg) -> float:
@@ -259,7 +263,7 @@ def main():
         flops = tower_flops_per_position(cfg) * B
         tower_avg_ms = tower_ms / max(tower_passes, 1)
         achieved = flops / (tower_avg_ms * 1e-3) / 1e12 if tower_passes else None
-        traffic = TOWER_TRAFFIC_BYTES.get(cfg.name)
+        traffic = tower_traffic_bytes(cfg, B)
         out = {
             "metric": METRIC, "value": evals / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
