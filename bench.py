@@ -171,6 +171,7 @@ def main():
     import torch.distributed as dist
 
     import paper_2609_37447_b200 as az
+    from paper_2609_37447_b200 import sharding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -181,7 +182,7 @@ def main():
 
     # ---- inputs: every rank evaluates its own batch of the same stream (weak scaling)
     B = cfg.batch
-    rec = positions.for_config(cfg, B, first_index=rank * B)
+    rec = positions.for_config(cfg, B, first_index=sharding.rank_first_index(rank, B))
     recs = positions.records_for_planes(cfg.in_planes, rec)
     blob = weights.make_blob(cfg)
     arch = az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, B)
@@ -252,10 +253,7 @@ def main():
     checksum = float(policy_host.sum())            # every row sums to one
 
     # ---- max over ranks
-    t = torch.tensor([total_ms, b2b_ms, e2e_s * 1e3, tower_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, b2b_ms, e2e_ms, tower_ms_max = [float(x) for x in t.cpu()]
+    total_ms, b2b_ms, e2e_ms, tower_ms_max = sharding.max_over_ranks([total_ms, b2b_ms, e2e_s * 1e3, tower_ms], device="cuda")
 
     if rank == 0:
         peaks = load_peaks()
