@@ -161,6 +161,34 @@ int az_encode(az_net *net, const void *positions_dev, int batch, void *planes_de
 int az_tower(az_net *net, const void *positions_dev, int batch, void *tower_dev, void *cuda_stream);
 
 /*
+ * az_tower for callers that cannot allocate device memory.  (The paper has no counterpart: this
+ * entry point exists for the library's users, not for the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits, or where a hidden allocation would
+ * break a guarantee -- a plugin inside a host application that hands out all device memory from
+ * its own pool and forbids others to allocate, a real-time serving thread that may not take the
+ * allocator's locks or its implicit device synchronisation, or a process whose memory budget was
+ * sized and frozen at start-up.  Such callers own their input and output buffers already; what they
+ * lack is a way to give the library room for its intermediate plane tensor.
+ *
+ * This call therefore uses NO allocator at all, neither cudaMalloc / cudaFree nor any pooling
+ * library: the encoded planes go to a fixed 1 MiB array that is part of the library image on the
+ * device (every GPU that loads the library holds it until the process exits).  Results are the
+ * same as az_tower's: tower_dev receives [batch][64][channels] bfloat16.
+ *   - Limits: batch <= 256 (AZ_ERR_BATCH_TOO_LARGE beyond, and beyond arch.max_batch); networks
+ *     with the tensor-core tower only, i.e. bf16, 128 channels, 19 input planes
+ *     (AZ_ERR_UNSUPPORTED otherwise).
+ *   - The first call on a device looks up the array's device address (one-time set-up, no
+ *     allocation); make that first call outside any stream capture.
+ *   - All calls, from every az_net and every stream, share the one array, and it keeps whatever
+ *     the previous call left in it.  Nothing in it needs clearing (each call overwrites all it
+ *     reads), but two calls that overlap on the GPU race on it: serialise them on one stream or
+ *     with events.
+ * Errors: BAD_ARG, BATCH_TOO_LARGE, UNSUPPORTED, CUDA.
+ */
+int az_tower_static(az_net *net, const void *positions_dev, int batch, void *tower_dev, void *cuda_stream);
+
+/*
  * Legal-move masks from the rules of chess, computed on the GPU, in the layout az_evaluate
  * takes.  Index maps (mover-oriented coordinates; App. D.1: castling is the king-to-own-rook
  * pair, en passant the pawn's ordinary pair):

@@ -23,7 +23,7 @@ AZ_VALUE_TANH, AZ_VALUE_WDL = 0, 1
 AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3 = 0, 1, 2
 
 EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
-           "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_host", "az_encode", "az_tower", "az_legal_masks",
+           "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_host", "az_encode", "az_tower", "az_tower_static", "az_legal_masks",
            "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error")
 
@@ -66,6 +66,8 @@ def _load_library():
     lib.az_encode.argtypes = [vp, vp, ci, vp, vp]
     lib.az_tower.restype = ci
     lib.az_tower.argtypes = [vp, vp, ci, vp, vp]
+    lib.az_tower_static.restype = ci
+    lib.az_tower_static.argtypes = [vp, vp, ci, vp, vp]
     lib.az_legal_masks.restype = ci
     lib.az_legal_masks.argtypes = [vp, sz, ci, ci, vp, vp]
     lib.az_calibrate.restype = ci
@@ -194,6 +196,17 @@ def az_encode(net: Net, positions_dev, batch, planes_dev, stream=None):
 def az_tower(net: Net, positions_dev, batch, tower_dev, stream=None):
     _check(_lib.az_tower(net.handle, _dev_ptr(positions_dev, "positions"), batch, _dev_ptr(tower_dev, "tower"),
                          _stream_ptr(stream)), "az_tower")
+
+
+def az_tower_static(net: Net, positions_dev, batch, tower_dev, stream=None):
+    """az_tower without any device allocation: the plane scratch is a fixed array inside the library.
+
+    For callers that may not allocate on the device (a host application that owns all device memory,
+    a real-time thread that must stay clear of the allocator).  At most 256 positions per call, bf16
+    128-channel networks only; all calls share the one scratch array, so do not overlap them on the GPU.
+    """
+    _check(_lib.az_tower_static(net.handle, _dev_ptr(positions_dev, "positions"), batch, _dev_ptr(tower_dev, "tower"),
+                                _stream_ptr(stream)), "az_tower_static")
 
 
 def az_legal_masks(positions_dev, position_stride, batch, policy_head, masks_dev, stream=None):
