@@ -6,14 +6,16 @@ vacuous.  Following the paper's own bootstrap (a small final policy projection, 
 set on a few hundred encoded positions, no chess targets: Sec. 4.3.5), the LAST linear layer of
 each head is multiplied by a scalar chosen on 512 seeded calibration positions so that
   * the standard deviation of a position's legal-move logits averages 1.0, and
-  * the value head's pre-activation has standard deviation 0.5 for the three win/draw/loss
-    logits and 0.03 for the scalar tanh head.  The scalar head has unit slope near the origin and
-    no softmax to cancel a shift common to its logits.  An emulation with bf16-rounded operands
-    but EXACT accumulation (the floor of any bf16 kernel) leaves the 20x128 tower's activations
-    0.6 % (rms) off, which this head turns into a pre-activation error of a quarter to a third
-    of its spread over positions; at a spread of 0.5 (or 0.15) that floor alone is 0.03-0.05 in
-    the tanh output, outside the 2e-2 bar.  0.03 keeps the floor inside the bar and is what an
-    untrained value head with a small final projection looks like.
+  * the value head's pre-activation has standard deviation 0.2 for the three win/draw/loss
+    logits and 0.03 for the scalar tanh head.  Why so small: an emulation with bf16-rounded
+    operands but EXACT accumulation (the floor of any bf16 kernel) leaves the towers' activations
+    0.6-0.7 % (rms) off, and the value heads turn that into a pre-activation error of a quarter
+    to a third of the head's spread over positions.  At a spread of 0.5 that floor alone is
+    0.03-0.05 in the tanh output of the 20x128 net and 0.03 in the win/draw/loss probabilities
+    of the 40x256 net, outside the 2e-2 bar for every possible bf16 implementation.  The tanh
+    head has unit slope near the origin and no softmax to cancel an error common to its logits,
+    hence the smaller figure.  A value head with a small final projection is also what an
+    untrained bootstrap network looks like.
 The scalars become part of the weights, so the oracle and the CUDA library see the same network.
 
 Calls only the oracle and the input generators.  Usage:  python -m oracle.calibrate_head_scales
@@ -41,7 +43,7 @@ def scales_for(cfg) -> dict:
         if legal.size >= 2:
             stds.append(float(np.std(legal)))
     policy = 1.0 / float(np.mean(stds))
-    value = (0.5 if cfg.value_head == 1 else 0.03) / float(np.std(raw["value_pre"]))
+    value = (0.2 if cfg.value_head == 1 else 0.03) / float(np.std(raw["value_pre"]))
     return {"policy": policy, "value": value, "positions": int(recs.shape[0]),
             "raw_legal_logit_std": float(np.mean(stds)), "raw_value_std": float(np.std(raw["value_pre"]))}
 
