@@ -30,6 +30,7 @@ class Config:
     position_seed: int
     weight_seed: int
     weights_like: str = ""       # name of the config whose weights (and head scales) this one reuses
+    branch_scale: float = 1.0    # factor folded into every block's second scale and bias (1/sqrt(blocks) in c4b)
     sweep: Tuple[int, ...] = field(default_factory=tuple)
 
     @property
@@ -54,6 +55,9 @@ CONFIGS = {
     "c2": Config("c2", 19, 20, 128, 0, 0, 1, 256, (0, 80), (0, 80), 20260939, 9370002),
     "c3": Config("c3", 19, 20, 128, 1, 1, 1, 1024, (0, 40), (40, 160), 20260940, 9370003),
     "c4": Config("c4", 19, 20, 128, 0, 0, 2, 4096, (0, 80), (0, 80), 20260941, 9370002, weights_like="c2"),
+    # c4 with the residual branches scaled by 1/sqrt(depth), the paper's quantisation-friendly block
+    # (Sec. 4.3.6), folded into the second convolution's scale and bias as the paper does at export
+    "c4b": Config("c4b", 19, 20, 128, 0, 0, 2, 4096, (0, 80), (0, 80), 20260941, 9370002, branch_scale=20 ** -0.5),
     "c5": Config("c5", 112, 40, 256, 1, 1, 1, 1024, (0, 80), (0, 80), 20260942, 9370005,
                  sweep=(16, 64, 256, 1024, 4096, 8192)),
 }

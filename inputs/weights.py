@@ -81,6 +81,10 @@ def draw_tensors(cfg: Config, policy_scale: float = None, value_scale: float = N
             fan_in = int(np.prod(shape[1:]))
             a = rng.normal(0.0, np.sqrt(2.0 / fan_in), size=shape)
         out[name] = a.astype(np.float32)
+    if cfg.branch_scale != 1.0:
+        for b in range(cfg.blocks):
+            for k in (f"b{b}.scale2", f"b{b}.bias2"):
+                out[k] = (out[k] * np.float32(cfg.branch_scale)).astype(np.float32)
     last_policy = ("p.w", "p.bias") if cfg.policy_head == 0 else ("p.fw", "p.fbias")
     for k in last_policy:
         out[k] = (out[k] * np.float32(policy_scale)).astype(np.float32)

@@ -29,6 +29,10 @@ struct BlobView {                       // float32 tensors of the blob, in file 
     const float *v_cw, *v_cs, *v_cb, *v_w1, *v_b1, *v_w2, *v_b2;
 };
 
+struct HostMaster {                     // fp32 tower parameters of an FP8 net, kept until az_calibrate has quantised them
+    std::vector<std::vector<float>> w, scale, bias;
+};
+
 bool arch_ok(const az_arch &a) {
     if (a.abi_version != AZ_ABI_VERSION) return false;
     if (a.in_planes != 19 && a.in_planes != 112) return false;
@@ -127,8 +131,10 @@ int build_net(Net &n, const BlobView &v) {
     int rc;
 
     // tensor-core tower: bf16, 128 channels, 19-plane input
-    const bool tc_shape = a.precision == AZ_PREC_BF16 && C == 128 && n.in_pad == 32;
-    if (tc_shape && !want_simt_tower()) {
+    n.fp8 = a.precision == AZ_PREC_FP8_E4M3;
+    const bool tc_shape = a.precision != AZ_PREC_FP32 && C == 128 && n.in_pad == 32;
+    if (n.fp8 && !tc_shape) return AZ_ERR_UNSUPPORTED;       // the FP8 tower exists for 128 channels, 19 planes
+    if (tc_shape && (n.fp8 || !want_simt_tower())) {
         std::vector<const float *> w, s, b;
         w.push_back(v.in_w); s.push_back(v.in_s); b.push_back(v.in_b);
         for (int i = 0; i < L; ++i) {
@@ -143,6 +149,17 @@ int build_net(Net &n, const BlobView &v) {
         std::vector<float> bias((size_t)n.n_conv * C);
         for (int l = 0; l < n.n_conv; ++l) memcpy(&bias[(size_t)l * C], b[l], sizeof(float) * C);
         if ((rc = upload_f32(bias.data(), bias.size(), &n.tc_bias)) != AZ_OK) return rc;
+        if (n.fp8) {
+            HostMaster *hm = new (std::nothrow) HostMaster();
+            if (!hm) return AZ_ERR_BAD_ARG;
+            n.host_master = hm;
+            for (int l = 0; l < n.n_conv; ++l) {
+                const size_t cin = l == 0 ? a.in_planes : C;
+                hm->w.emplace_back(w[l], w[l] + (size_t)C * cin * 9);
+                hm->scale.emplace_back(s[l], s[l] + C);
+                hm->bias.emplace_back(b[l], b[l] + C);
+            }
+        }
         // fused head projections and tensor-core fully-connected layers
         const bool flat = a.policy_head == AZ_POLICY_FLAT1858;
         const int n_policy = flat ? kHeadChannels : kPlanes73, n_policy_pad = flat ? kHeadChannels : 80;
@@ -226,6 +243,8 @@ void free_net(Net *n) {
     if (!n) return;
     for (int i = 0; i < 1 + 2 * 64; ++i) { cudaFree(n->conv_w[i]); cudaFree(n->conv_scale[i]); cudaFree(n->conv_bias[i]); }
     cudaFree(n->tc_weights); cudaFree(n->tc_bias); cudaFree(n->tc_head_w); cudaFree(n->tc_head_bias);
+    cudaFree(n->tc8_weights); cudaFree(n->tc8_lconst);
+    delete static_cast<HostMaster *>(n->host_master);
     cudaFree(n->fc_policy_w); cudaFree(n->fc_value_w); cudaFree(n->u_policy); cudaFree(n->u_value);
     cudaFree(n->p_w); cudaFree(n->p_scale); cudaFree(n->p_bias); cudaFree(n->p_fw); cudaFree(n->p_fbias);
     cudaFree(n->v_cw); cudaFree(n->v_cscale); cudaFree(n->v_cbias); cudaFree(n->v_w1); cudaFree(n->v_b1);
@@ -250,7 +269,7 @@ int run_tower(Net &n, const void *positions, int batch, void **tower_out, bool f
     if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
     if (n.tc_ready) {
         *tower_out = fused_heads ? nullptr : n.act[0];
-        rc = launch_tower_tc(n, n.planes, batch, *tower_out, fused_heads, s);
+        rc = launch_tower_tc(n, n.planes, batch, *tower_out, fused_heads, nullptr, s);
         if (rc == AZ_OK && timed) AZ_CUDA(cudaEventRecord(n.ev_end[n.n_events++], s));
         return rc;
     }
@@ -289,7 +308,6 @@ int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az
     if (!arch || !weights_host || !out) return AZ_ERR_BAD_ARG;
     *out = nullptr;
     if (!az::arch_ok(*arch)) return AZ_ERR_BAD_ARCH;
-    if (arch->precision == AZ_PREC_FP8_E4M3) return AZ_ERR_UNSUPPORTED;
     az::BlobView view;
     int rc = az::parse_blob(*arch, static_cast<const unsigned char *>(weights_host), nbytes, view);
     if (rc != AZ_OK) return rc;
@@ -321,6 +339,7 @@ int az_tower(az_net *net, const void *positions_dev, int batch, void *tower_dev,
     if (reinterpret_cast<uintptr_t>(positions_dev) & 7) return AZ_ERR_BAD_ARG;
     if ((uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
     if (batch == 0) return AZ_OK;
+    if (n->fp8 && !n->fp8_ready) return AZ_ERR_NOT_CALIBRATED;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     void *x = nullptr;
     int rc = az::run_tower(*n, positions_dev, batch, &x, false, s);
@@ -340,6 +359,7 @@ int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_ma
         (reinterpret_cast<uintptr_t>(policy_dev) & 3) || (reinterpret_cast<uintptr_t>(value_dev) & 3))
         return AZ_ERR_BAD_ARG;
     if ((uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
+    if (n->fp8 && !n->fp8_ready) return AZ_ERR_NOT_CALIBRATED;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const az_arch &a = n->arch;
     const int C = (int)a.channels;
@@ -441,10 +461,44 @@ int az_legal_masks(const void *positions_dev, size_t position_stride, int batch,
                                   static_cast<cudaStream_t>(cuda_stream));
 }
 
-int az_calibrate(az_net *net, const void *positions_dev, int n, void *cuda_stream) {
-    (void)positions_dev; (void)n; (void)cuda_stream;
-    if (!net) return AZ_ERR_BAD_ARG;
-    return AZ_ERR_UNSUPPORTED;
+int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_stream) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n || count <= 0 || !positions_dev || (reinterpret_cast<uintptr_t>(positions_dev) & 7)) return AZ_ERR_BAD_ARG;
+    if (!n->fp8 || !n->host_master) return AZ_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const int C = (int)n->arch.channels, L = n->n_conv;
+    const size_t pb = az_position_bytes(&n->arch);
+    // 1. bf16 tower over the calibration positions, recording every layer's per-channel output maximum
+    unsigned int *absmax_dev = nullptr;
+    AZ_CUDA(cudaMalloc((void **)&absmax_dev, (size_t)L * C * sizeof(unsigned int)));
+    cudaError_t e = cudaMemsetAsync(absmax_dev, 0, (size_t)L * C * sizeof(unsigned int), s);
+    int rc = AZ_OK;
+    for (int first = 0; first < count && rc == AZ_OK && e == cudaSuccess; first += (int)n->arch.max_batch) {
+        const int chunk = count - first < (int)n->arch.max_batch ? count - first : (int)n->arch.max_batch;
+        const unsigned char *p = static_cast<const unsigned char *>(positions_dev) + (size_t)first * pb;
+        rc = az::launch_encode(p, pb, chunk, (int)n->arch.in_planes, n->in_pad, true, n->planes, n->status_dev, s);
+        if (rc == AZ_OK) rc = az::launch_tower_tc(*n, n->planes, chunk, nullptr, false, absmax_dev, s);
+    }
+    std::vector<float> absmax((size_t)L * C);
+    if (rc == AZ_OK && e == cudaSuccess) e = cudaMemcpyAsync(absmax.data(), absmax_dev, absmax.size() * sizeof(float), cudaMemcpyDeviceToHost, s);
+    if (rc == AZ_OK && e == cudaSuccess) e = cudaStreamSynchronize(s);
+    cudaFree(absmax_dev);
+    if (rc != AZ_OK) return rc;
+    if (e != cudaSuccess) { az::set_cuda_error(e, "az_calibrate"); return AZ_ERR_CUDA; }
+    // 2. quantise the tower with those ranges
+    az::HostMaster *hm = static_cast<az::HostMaster *>(n->host_master);
+    std::vector<const float *> w, sc, bi;
+    for (int l = 0; l < L; ++l) { w.push_back(hm->w[l].data()); sc.push_back(hm->scale[l].data()); bi.push_back(hm->bias[l].data()); }
+    const size_t bytes = az::tc8_packed_weight_bytes(n->in_pad, C, L);
+    std::vector<unsigned char> packed(bytes);
+    std::vector<float> lconst((size_t)L * 4 * C);
+    az::tc8_pack(w.data(), sc.data(), bi.data(), absmax.data(), (int)n->arch.in_planes, n->in_pad, C, L, packed.data(), lconst.data());
+    if (!n->tc8_weights) AZ_CUDA(cudaMalloc(&n->tc8_weights, bytes));
+    if (!n->tc8_lconst) AZ_CUDA(cudaMalloc((void **)&n->tc8_lconst, lconst.size() * sizeof(float)));
+    AZ_CUDA(cudaMemcpy(n->tc8_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
+    AZ_CUDA(cudaMemcpy(n->tc8_lconst, lconst.data(), lconst.size() * sizeof(float), cudaMemcpyHostToDevice));
+    n->fp8_ready = true;
+    return AZ_OK;
 }
 
 int az_device_status(az_net *net, void *cuda_stream, uint32_t *status_out) {

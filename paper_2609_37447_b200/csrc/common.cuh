@@ -44,6 +44,11 @@ struct Net {
     void *tc_weights = nullptr;       // packed UMMA B-operand tiles, all layers
     float *tc_bias = nullptr;         // [n_conv][C] folded bias (scales are folded into the weights)
     bool tc_ready = false;
+    // FP8-e4m3 tower (weights and per-layer constants exist once az_calibrate has run)
+    bool fp8 = false, fp8_ready = false;
+    void *tc8_weights = nullptr;
+    float *tc8_lconst = nullptr;      // [n_conv][4][C]
+    void *host_master = nullptr;      // fp32 tower weights kept on the host until calibration (FP8 nets)
     void *tc_head_w = nullptr;        // packed 1x1 head projections (policy | value), fused into the tower kernel
     float *tc_head_bias = nullptr;
     int tc_head_n = 0;                // 64 (flat policy head) or 112 (73-plane policy head)
@@ -118,7 +123,11 @@ int launch_masked_softmax(const float *logits, const uint64_t *masks, int batch,
 size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv);
 void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
                      int channels, int n_conv, __nv_bfloat16 *packed_host);
-int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, bool with_heads, cudaStream_t s);
+int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, bool with_heads,
+                    unsigned int *absmax, cudaStream_t s);
+size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv);
+void tc8_pack(const float *const *w, const float *const *scale, const float *const *bias, const float *absmax,
+              int in_planes, int in_pad, int channels, int n_conv, unsigned char *packed, float *lconst);
 int tower_tc_launch_count();
 size_t tc_head_weight_bytes(int head_n);
 void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,

@@ -33,8 +33,12 @@
 #include "common.cuh"
 #include "ptx.cuh"
 
+#include <cuda_fp8.h>
+
+#include <cmath>
 #include <cstdio>
 #include <cstdlib>
+#include <vector>
 
 namespace az {
 namespace {
@@ -91,7 +95,14 @@ struct TowerArgs {
     __nv_bfloat16 *u_policy;         // flat head: projection as GEMM A tiles, K index = square*32 + channel
     __nv_bfloat16 *u_value;          // value projection, same layout
     float *logits;                   // 73-plane head: [batch][73*64] fp32 logits, index = plane*64 + square
+    // FP8 tower: per-layer channel constants [n_conv][4][128]: output scale, bias, 1/next activation
+    // scale, 1/(next conv2 weight scale) for the residual stream kept in TMEM
+    const float *lconst;
+    // calibration run (bf16 kernel): per-layer, per-channel maximum of the layer outputs, as float bits
+    unsigned int *absmax;            // [n_conv][128]
 };
+constexpr int kLconstFloats = 4 * kC;                       // per layer
+constexpr int kLconstSmemBytes = 4 * kGroups * kLconstFloats * 4;   // a private copy per epilogue warp: 16 KB
 
 // Bounded wait, called by all 32 lanes of a warp together.  Returns false (to every lane alike) if
 // the CTA has been aborted or this wait ran out; the latter raises the abort flag and the status bit.
@@ -111,6 +122,7 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     return __all_sync(0xffffffffu, done);
 }
 
+template <bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1)
 tower_tc_kernel(const TowerArgs args) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -128,7 +140,10 @@ tower_tc_kernel(const TowerArgs args) {
     // ---- set-up: zero the frames (their borders stay zero for the kernel's lifetime), barriers, TMEM
     for (int i = threadIdx.x; i < kGroups * kFrameBytes / 16; i += kThreads)
         reinterpret_cast<uint4 *>(smem + kOffFrames)[i] = make_uint4(0, 0, 0, 0);
-    if (args.bias_in_smem) {
+    if (kFp8) {
+        for (int i = threadIdx.x; i < args.head_n; i += kThreads)
+            reinterpret_cast<float *>(smem + kOffBias + kLconstSmemBytes)[i] = args.head_bias[i];
+    } else if (args.bias_in_smem) {
         for (int i = threadIdx.x; i < args.n_conv * kC; i += kThreads)
             reinterpret_cast<float *>(smem + kOffBias)[i] = args.bias[i];
         for (int i = threadIdx.x; i < args.head_n; i += kThreads)
@@ -172,7 +187,7 @@ tower_tc_kernel(const TowerArgs args) {
         for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
             const unsigned char *src = reinterpret_cast<const unsigned char *>(args.weights);
             for (int l = 0; l < n_conv && ok; ++l) {
-                const int nkc = l == 0 ? args.in_kc : kC / 16;
+                const int nkc = l == 0 ? args.in_kc : (kFp8 ? kC / 32 : kC / 16);     // K per MMA: 16 bf16 or 32 e4m3
                 for (int kc = 0; kc < nkc; ++kc) {
                     ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                     if (!ok) break;
@@ -209,6 +224,7 @@ tower_tc_kernel(const TowerArgs args) {
         // ================= MMA issuer of group g =================
         const int g = warp - 1;
         constexpr uint32_t idesc = ptx::idesc_bf16_f32(128, 128);
+        constexpr uint32_t idesc8 = ptx::idesc_e4m3_f32(128, 128);
         int stage = 0;
         uint32_t phase = 0;
         uint32_t a_phase = 0;
@@ -227,7 +243,8 @@ tower_tc_kernel(const TowerArgs args) {
                 lead_parity ^= (uint32_t)(n_layers & 1);
             }
             for (int l = 0; l < n_conv && ok; ++l) {
-                const int nkc = l == 0 ? args.in_kc : kC / 16;
+                const int nkc = l == 0 ? args.in_kc : (kFp8 ? kC / 32 : kC / 16);
+                const bool e4m3 = kFp8 && l > 0;                       // the input layer stays bf16
                 const bool conv2 = l >= 2 && (l & 1) == 0;             // accumulates onto the residual stream
                 const uint32_t d = d_h + (((l & 1) == 1) ? 128u : 0u); // conv1 writes the ACC columns
                 for (int kc = 0; kc < nkc; ++kc) {
@@ -246,9 +263,14 @@ tower_tc_kernel(const TowerArgs args) {
 #pragma unroll
                         for (int tap = 0; tap < 9; ++tap) {
                             const int dy = tap / 3 - 1, dx = tap % 3 - 1;
-                            ptx::mma_bf16_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                b_lo + (uint32_t)(tap * (kTileBytes / 16)), kBDescHi, idesc,
-                                                tap == 0 ? first : 1u);
+                            if (e4m3)
+                                ptx::mma_e4m3_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                                    b_lo + (uint32_t)(tap * (kTileBytes / 16)), kBDescHi, idesc8,
+                                                    tap == 0 ? first : 1u);
+                            else
+                                ptx::mma_bf16_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                                    b_lo + (uint32_t)(tap * (kTileBytes / 16)), kBDescHi, idesc,
+                                                    tap == 0 ? first : 1u);
                         }
                         if (kc == nkc - 1) ptx::mma_commit(bar_acc_full(g));
                         ptx::mma_commit(bar_w_empty(stage));
@@ -316,11 +338,27 @@ tower_tc_kernel(const TowerArgs args) {
                 const bool from_acc = (l & 1) == 1;
                 const bool last = l == n_conv - 1 && head_n == 0;        // nothing follows: results go to global only
                 const bool to_global = l == n_conv - 1 && args.out != nullptr;
+                const bool next_e4m3 = kFp8 && l + 1 < n_conv;           // the next layer reads e4m3 operands
+                const float *lc = nullptr;
+                if (kFp8) {
+                    // this layer's channel constants -> this warp's own copy in shared memory (every thread
+                    // needs all 128 channels; a private copy needs no cross-warp barrier, which could not
+                    // be bounded the way the mbarrier waits are)
+                    float *buf = reinterpret_cast<float *>(smem + kOffBias) + (warp - 1 - kGroups) * kLconstFloats;
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < kLconstFloats / 4 / 32; ++i)
+                        reinterpret_cast<float4 *>(buf)[i * 32 + lane] =
+                            __ldg(reinterpret_cast<const float4 *>(args.lconst + (size_t)l * kLconstFloats) + i * 32 + lane);
+                    __syncwarp();
+                    lc = buf;
+                }
                 ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 acc_phase ^= 1u;
                 ptx::tc_fence_after();
-                const float *bias = args.bias_in_smem ? reinterpret_cast<const float *>(smem + kOffBias) + l * kC
+                const float *bias = kFp8 ? lc + kC
+                                  : args.bias_in_smem ? reinterpret_cast<const float *>(smem + kOffBias) + l * kC
                                                       : args.bias + (size_t)l * kC;
                 __nv_bfloat16 *dst = args.out + ((size_t)board * 64 + sq) * kC;
                 const uint32_t t_src = t_lane + (uint32_t)(from_acc ? 128 : 0);
@@ -336,37 +374,79 @@ tower_tc_kernel(const TowerArgs args) {
 #pragma unroll
                     for (int i = 0; i < 16; i += 4) {
                         const float4 bv = *reinterpret_cast<const float4 *>(bias + kc * 16 + i);
-                        v[i + 0] = fmaxf(__uint_as_float(rr[i + 0]) + bv.x, 0.0f);
-                        v[i + 1] = fmaxf(__uint_as_float(rr[i + 1]) + bv.y, 0.0f);
-                        v[i + 2] = fmaxf(__uint_as_float(rr[i + 2]) + bv.z, 0.0f);
-                        v[i + 3] = fmaxf(__uint_as_float(rr[i + 3]) + bv.w, 0.0f);
+                        if (kFp8) {
+                            const float4 os = *reinterpret_cast<const float4 *>(lc + kc * 16 + i);
+                            v[i + 0] = fmaxf(fmaf(__uint_as_float(rr[i + 0]), os.x, bv.x), 0.0f);
+                            v[i + 1] = fmaxf(fmaf(__uint_as_float(rr[i + 1]), os.y, bv.y), 0.0f);
+                            v[i + 2] = fmaxf(fmaf(__uint_as_float(rr[i + 2]), os.z, bv.z), 0.0f);
+                            v[i + 3] = fmaxf(fmaf(__uint_as_float(rr[i + 3]), os.w, bv.w), 0.0f);
+                        } else {
+                            v[i + 0] = fmaxf(__uint_as_float(rr[i + 0]) + bv.x, 0.0f);
+                            v[i + 1] = fmaxf(__uint_as_float(rr[i + 1]) + bv.y, 0.0f);
+                            v[i + 2] = fmaxf(__uint_as_float(rr[i + 2]) + bv.z, 0.0f);
+                            v[i + 3] = fmaxf(__uint_as_float(rr[i + 3]) + bv.w, 0.0f);
+                        }
                     }
-                    uint32_t pk[8];
+                    if (!kFp8 && args.absmax != nullptr) {
+                        // calibration: largest output of this layer per channel over all rows of the warp
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-                        pk[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                        for (int i = 0; i < 16; ++i) {
+                            float mx = live ? v[i] : 0.0f;
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                            if (lane == i) atomicMax(args.absmax + l * kC + kc * 16 + i, __float_as_uint(mx));
+                        }
                     }
                     if (to_global && live) {
+                        uint32_t pk[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+                            pk[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                        }
                         reinterpret_cast<uint4 *>(dst + kc * 16)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         reinterpret_cast<uint4 *>(dst + kc * 16)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                     }
                     if (!last) {
-                        *reinterpret_cast<uint4 *>(frame + (2 * kc) * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                        *reinterpret_cast<uint4 *>(frame + (2 * kc + 1) * kPlaneBytes + slot * 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                        if (next_e4m3) {
+                            // 16 channels -> 16 e4m3 bytes (saturating, round to nearest even) = one slot of plane kc
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const float4 qs = *reinterpret_cast<const float4 *>(lc + 2 * kC + kc * 16 + 4 * i);
+                                const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(v[4 * i] * qs.x, v[4 * i + 1] * qs.y), __NV_SATFINITE, __NV_E4M3);
+                                const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(v[4 * i + 2] * qs.z, v[4 * i + 3] * qs.w), __NV_SATFINITE, __NV_E4M3);
+                                pk[i] = lo | (hi << 16);
+                            }
+                            *reinterpret_cast<uint4 *>(frame + kc * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        } else {
+                            uint32_t pk[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
+                                pk[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                            }
+                            *reinterpret_cast<uint4 *>(frame + (2 * kc) * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            *reinterpret_cast<uint4 *>(frame + (2 * kc + 1) * kPlaneBytes + slot * 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                        }
                         if (keep_h) {
-                            // fp32 copy back to H.  Its completion is awaited once, after the loop: the next
-                            // reader of H is the conv2 two layers on, whose MMAs are gated by barriers these
-                            // same threads arrive on only after that wait.
+                            // fp32 copy back to H (FP8: pre-divided by the next conv2's weight scale, so that
+                            // conv2 can accumulate its raw products straight onto it).  Its completion is
+                            // awaited once, after the loop: the next reader of H is the conv2 two layers on,
+                            // whose MMAs are gated by barriers these same threads arrive on only after that wait.
                             uint32_t w[16];
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) w[i] = __float_as_uint(v[i]);
+                            for (int i = 0; i < 16; ++i)
+                                w[i] = __float_as_uint(kFp8 ? v[i] * lc[3 * kC + kc * 16 + i] : v[i]);
                             ptx::tmem_st16(t_lane + (uint32_t)(kc * 16), w);
                         }
-                        ptx::fence_proxy_async_smem();
-                        ptx::tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(bar_a_ready(g, kc));
+                        // e4m3 layers consume 32 channels per MMA: one hand-off per two slices
+                        if (!next_e4m3 || (kc & 1)) {
+                            ptx::fence_proxy_async_smem();
+                            ptx::tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) ptx::mbar_arrive(bar_a_ready(g, next_e4m3 ? (kc >> 1) : kc));
+                        }
                     }
                 }
                 if (keep_h) ptx::tmem_st_wait();
@@ -377,7 +457,8 @@ tower_tc_kernel(const TowerArgs args) {
                 if (!ok) break;
                 acc_phase ^= 1u;
                 ptx::tc_fence_after();
-                const float *hb = args.bias_in_smem ? reinterpret_cast<const float *>(smem + kOffBias) + n_conv * kC : args.head_bias;
+                const float *hb = kFp8 ? reinterpret_cast<const float *>(smem + kOffBias + kLconstSmemBytes)
+                                : args.bias_in_smem ? reinterpret_cast<const float *>(smem + kOffBias) + n_conv * kC : args.head_bias;
                 // this row's place in the GEMM A tiles: [tile of 128 boards][8-wide K chunk][board/8][board%8][8 k]
                 const size_t u_row = ((size_t)(board >> 7) * 256 * 16 + (size_t)((board & 127) >> 3)) * 128 + (size_t)(board & 7) * 16;
                 const int n_slices = head_n / 16;
@@ -460,6 +541,62 @@ void tc_pack_weights(const float *const *w, const float *const *scale, int in_pl
 
 int tower_tc_launch_count() { return 1; }
 
+// ---- FP8-e4m3 tower (Sec. 4.3.6: trunk convolutions quantised, start block and heads at higher
+// precision, ranges fixed on calibration positions).  Layer 0 keeps bf16 operands.  For a layer
+// l >= 1 with input activation scale sa[ci] (calibration maximum / 448) the folded weight
+//     W'[co][ci][tap] = bn_scale[co] * W[co][ci][tap] * sa[ci]
+// is stored as e4m3 with one fp32 scale per output channel, ws[co] = max|W'[co]| / 448, so that
+//     conv = ws[co] * sum_k q_a[k] * q_w[co][k],   q_a = e4m3(a / sa), q_w = e4m3(W' / ws).
+// lconst[l] = { output scale ws (1 for layer 0), bias, 1/sa of the next layer, 1/ws of the next
+// conv2 (the residual stream sits in TMEM pre-divided by it) }.
+size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv) {
+    return ((size_t)in_pad / 16 + (size_t)(n_conv - 1) * (channels / 32)) * kStageBytes;
+}
+
+void tc8_pack(const float *const *w, const float *const *scale, const float *const *bias, const float *absmax,
+              int in_planes, int in_pad, int channels, int n_conv, unsigned char *packed, float *lconst) {
+    const int C = channels;
+    const float kMax = 448.0f, kTiny = 1e-30f;
+    std::vector<float> sa((size_t)n_conv * C, 1.0f), ws((size_t)n_conv * C, 1.0f);
+    for (int l = 1; l < n_conv; ++l)
+        for (int c = 0; c < C; ++c) sa[(size_t)l * C + c] = fmaxf(absmax[(size_t)(l - 1) * C + c], kTiny) / kMax;
+    // layer 0: bf16 tiles exactly as in the bf16 tower
+    tc_pack_weights(w, scale, in_planes, in_pad, C, 1, reinterpret_cast<__nv_bfloat16 *>(packed));
+    unsigned char *dst = packed + (size_t)(in_pad / 16) * kStageBytes;
+    std::vector<float> wf((size_t)C * C * 9);
+    for (int l = 1; l < n_conv; ++l) {
+        for (int co = 0; co < C; ++co) {
+            float mx = 0.0f;
+            for (int ci = 0; ci < C; ++ci)
+                for (int tap = 0; tap < 9; ++tap) {
+                    const float v = scale[l][co] * w[l][((size_t)co * C + ci) * 9 + tap] * sa[(size_t)l * C + ci];
+                    wf[((size_t)co * C + ci) * 9 + tap] = v;
+                    mx = fmaxf(mx, fabsf(v));
+                }
+            ws[(size_t)l * C + co] = fmaxf(mx, kTiny) / kMax;
+        }
+        for (int kc = 0; kc < C / 32; ++kc)
+            for (int tap = 0; tap < 9; ++tap)
+                for (int k16 = 0; k16 < 2; ++k16)
+                    for (int ng = 0; ng < C / 8; ++ng)
+                        for (int r = 0; r < 8; ++r)
+                            for (int e = 0; e < 16; ++e) {
+                                const int n = ng * 8 + r, ci = kc * 32 + k16 * 16 + e;
+                                const float v = wf[((size_t)n * C + ci) * 9 + tap] / ws[(size_t)l * C + n];
+                                *dst++ = (unsigned char)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
+                            }
+    }
+    for (int l = 0; l < n_conv; ++l) {
+        float *lc = lconst + (size_t)l * 4 * C;
+        for (int c = 0; c < C; ++c) {
+            lc[c] = l == 0 ? 1.0f : ws[(size_t)l * C + c];
+            lc[C + c] = bias[l][c];
+            lc[2 * C + c] = l + 1 < n_conv ? 1.0f / sa[(size_t)(l + 1) * C + c] : 1.0f;
+            lc[3 * C + c] = ((l & 1) == 0 && l + 2 < n_conv) ? 1.0f / ws[(size_t)(l + 2) * C + c] : 1.0f;
+        }
+    }
+}
+
 // Head projections as one N = head_n tile per 16-channel slice: rows [0, n_policy) the policy
 // projection (scaled where it has a folded batch-norm), zero rows up to n_policy_pad, then the 32
 // rows of the value projection.  Same core-matrix order as the tower's weight tiles.
@@ -482,7 +619,8 @@ void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_p
                     }
 }
 
-int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, bool with_heads, cudaStream_t s) {
+int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, bool with_heads,
+                    unsigned int *absmax, cudaStream_t s) {
     if (batch == 0) return AZ_OK;
     static int sm_count[64] = {};
     int dev = 0;
@@ -490,13 +628,15 @@ int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_o
     if (dev < 64 && sm_count[dev] == 0) {
         int n = 0;
         AZ_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
-        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
     const int sms = dev < 64 ? sm_count[dev] : 148;
+    const bool fp8 = net.fp8_ready && absmax == nullptr;      // the calibration pass itself runs in bf16
     TowerArgs a;
     a.planes = static_cast<const __nv_bfloat16 *>(planes);
-    a.weights = static_cast<const __nv_bfloat16 *>(net.tc_weights);
+    a.weights = static_cast<const __nv_bfloat16 *>(fp8 ? net.tc8_weights : net.tc_weights);
     a.bias = net.tc_bias;
     a.out = static_cast<__nv_bfloat16 *>(tower_out);
     a.status = net.status_dev;
@@ -509,13 +649,20 @@ int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_o
     a.u_policy = static_cast<__nv_bfloat16 *>(net.u_policy);
     a.u_value = static_cast<__nv_bfloat16 *>(net.u_value);
     a.logits = net.logits;
+    a.lconst = net.tc8_lconst;
+    a.absmax = absmax;
     a.bias_in_smem = net.n_conv + 1 <= kMaxBiasLayers ? 1 : 0;
     static const bool trace = getenv("AZ_TOWER_TRACE") != nullptr;
     a.trace = trace ? atoi(getenv("AZ_TOWER_TRACE")) : 0;
-    const int smem_bytes = kSmemBytesNoBias + (a.bias_in_smem ? (net.n_conv + 1) * kC * 4 : 0);
     const int n_units = (batch + kBoardsPerCta - 1) / kBoardsPerCta;
     const int grid = n_units < sms ? n_units : sms;
-    tower_tc_kernel<<<grid, kThreads, smem_bytes, s>>>(a);
+    if (fp8) {
+        const int smem_bytes = kSmemBytesNoBias + kLconstSmemBytes + kC * 4;
+        tower_tc_kernel<true><<<grid, kThreads, smem_bytes, s>>>(a);
+    } else {
+        const int smem_bytes = kSmemBytesNoBias + (a.bias_in_smem ? (net.n_conv + 1) * kC * 4 : 0);
+        tower_tc_kernel<false><<<grid, kThreads, smem_bytes, s>>>(a);
+    }
     AZ_LAUNCH_CHECK();
     return AZ_OK;
 }
