@@ -29,6 +29,7 @@ WORKLOADS = {
     "c1": "c1: 6x64 fp32 batch 64, 73-plane policy + tanh value",
     "c2": "c2: 20x128 bf16 batch 256, 73-plane policy + tanh value",
     "c3": "c3: 20x128 bf16 batch 1024, flat-1858 policy + WDL value",
+    "c5": "c5: 40x256 bf16, 112 history planes, flat-1858 policy + WDL value (batch sweep via --batch)",
     "c4": "c4: 20x128 FP8-e4m3 tower (bf16 heads) batch 4096, 73-plane policy + tanh value",
     "c4b": "c4b: c4 with residual branches scaled by 1/sqrt(20)",
 }

@@ -12,7 +12,7 @@ import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libazeval.so")
+LIB_PATH = os.environ.get("AZ_EVAL_LIB") or os.path.join(_HERE, "libazeval.so")
 
 AZ_ABI_VERSION = 1
 AZ_OK = 0

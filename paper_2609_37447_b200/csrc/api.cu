@@ -132,8 +132,9 @@ int build_net(Net &n, const BlobView &v) {
 
     // tensor-core tower: bf16, 128 channels, 19-plane input
     n.fp8 = a.precision == AZ_PREC_FP8_E4M3;
-    const bool tc_shape = a.precision != AZ_PREC_FP32 && C == 128 && n.in_pad == 32;
-    if (n.fp8 && !tc_shape) return AZ_ERR_UNSUPPORTED;       // the FP8 tower exists for 128 channels, 19 planes
+    // tensor-core tower: bf16 with 128 or 256 channels; the FP8 tower exists for 128 channels
+    const bool tc_shape = a.precision != AZ_PREC_FP32 && (C == 128 || (C == 256 && !n.fp8));
+    if (n.fp8 && !tc_shape) return AZ_ERR_UNSUPPORTED;
     if (tc_shape && (n.fp8 || !want_simt_tower())) {
         std::vector<const float *> w, s, b;
         w.push_back(v.in_w); s.push_back(v.in_s); b.push_back(v.in_b);
@@ -164,7 +165,7 @@ int build_net(Net &n, const BlobView &v) {
         const bool flat = a.policy_head == AZ_POLICY_FLAT1858;
         const int n_policy = flat ? kHeadChannels : kPlanes73, n_policy_pad = flat ? kHeadChannels : 80;
         n.tc_head_n = n_policy_pad + kHeadChannels;
-        std::vector<__nv_bfloat16> hw(tc_head_weight_bytes(n.tc_head_n) / sizeof(__nv_bfloat16));
+        std::vector<__nv_bfloat16> hw(tc_head_weight_bytes(n.tc_head_n, C) / sizeof(__nv_bfloat16));
         tc_pack_head(v.p_w, flat ? v.p_s : nullptr, n_policy, n_policy_pad, v.v_cw, v.v_cs, C, hw.data());
         AZ_CUDA(cudaMalloc(&n.tc_head_w, hw.size() * sizeof(__nv_bfloat16)));
         AZ_CUDA(cudaMemcpy(n.tc_head_w, hw.data(), hw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));

@@ -129,7 +129,7 @@ size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv);
 void tc8_pack(const float *const *w, const float *const *scale, const float *const *bias, const float *absmax,
               int in_planes, int in_pad, int channels, int n_conv, unsigned char *packed, float *lconst);
 int tower_tc_launch_count();
-size_t tc_head_weight_bytes(int head_n);
+size_t tc_head_weight_bytes(int head_n, int channels);
 void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,
                   int channels, __nv_bfloat16 *packed);
 

@@ -37,7 +37,7 @@ extern "C" int az_tower_static(az_net *net, const void *positions_dev, int batch
     az::Net *n = reinterpret_cast<az::Net *>(net);
     if (!n || batch < 0 || (batch > 0 && (!positions_dev || !tower_dev))) return AZ_ERR_BAD_ARG;
     if ((reinterpret_cast<uintptr_t>(positions_dev) & 7) || (reinterpret_cast<uintptr_t>(tower_dev) & 15)) return AZ_ERR_BAD_ARG;
-    if (!n->tc_ready || n->in_pad != 32) return AZ_ERR_UNSUPPORTED;
+    if (!n->tc_ready || n->in_pad != 32 || n->arch.channels != 128) return AZ_ERR_UNSUPPORTED;
     if (batch > az::kStaticMaxBatch || (uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
     if (batch == 0) return AZ_OK;
     void *planes = nullptr;

@@ -43,66 +43,73 @@
 namespace az {
 namespace {
 
-constexpr int kC = 128;                        // tower channels
-constexpr int kNB = 2;                         // boards per group
-constexpr int kGroups = 2;                     // groups per CTA
-constexpr int kBoardsPerCta = kNB * kGroups;
+constexpr int kNB = 2;                         // boards per group (128 GEMM rows)
 constexpr int kSlots = 10 * kNB * 9 + 1;       // 181 sixteen-byte slots per 8-channel plane
 constexpr int kPlaneBytes = kSlots * 16;       // 2896
-constexpr int kFrameBytes = kPlaneBytes * (kC / 8);   // 46336 per group
 constexpr int kRowGroupBytes = 9 * 16;         // stride between 8-row groups (SBO)
-constexpr int kTileBytes = 128 * 16 * 2;       // one tap: N=128 x K=16 bf16 = 4096
-constexpr int kStageBytes = 9 * kTileBytes;    // 36864: 16 input channels, all taps
-constexpr int kStages = 3;
-constexpr int kThreads = 32 * (1 + kGroups + 4 * kGroups);   // producer, one MMA issuer per group, 4 epilogue warps per group
 constexpr uint32_t kTmemCols = 512;
+constexpr int kMaxSmem = 232448;
 // high words of the shared-memory matrix descriptors (no swizzle, K-major): stride between 8-row
 // groups in bits 0-13, descriptor version 1 in bit 14; the low word carries the stride between the
 // two K core matrices in bits 16-29 above the start address.
 constexpr uint32_t kADescHi = (uint32_t)(kRowGroupBytes >> 4) | (1u << 14);
 constexpr uint32_t kBDescHi = (uint32_t)(128 >> 4) | (1u << 14);
 constexpr uint32_t kADescLbo = (uint32_t)(kPlaneBytes >> 4) << 16;
-constexpr uint32_t kBDescLbo = (uint32_t)(2048 >> 4) << 16;
 constexpr uint32_t kSpinLimit = 1u << 24;
 
-constexpr int kOffFrames = 0;
-constexpr int kOffWeights = kOffFrames + kGroups * kFrameBytes;          // 92672
-constexpr int kOffBars = kOffWeights + kStages * kStageBytes;            // 203264
-// barriers: w_full[3], w_empty[3], acc_full[2], a_ready[2][8], done
-constexpr int kNumBars = 2 * kStages + kGroups + kGroups * 8 + 1;
-constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
-constexpr int kOffAbort = kOffTmemPtr + 4;
-constexpr int kOffBias = (kOffAbort + 4 + 15) & ~15;                     // folded biases of every layer, fp32
-constexpr int kMaxSmem = 232448;
-constexpr int kMaxBiasLayers = (kMaxSmem - kOffBias) / (kC * 4);         // 56 layers fit beside everything else
-constexpr int kSmemBytesNoBias = kOffBias;
+// Shape-dependent constants.  128 channels: two groups per CTA share every weight stage (16 input
+// channels x 9 taps).  256 channels: the frame and the accumulators of ONE group fill shared memory
+// and TMEM, and a stage is 16 input channels x 3 taps.
+template <int C, int GROUPS>
+struct Shape {
+    static constexpr int kC = C, kGroups = GROUPS;
+    static constexpr int kBoardsPerCta = kNB * kGroups;
+    static constexpr int kSlices = kC / 16;                          // 16-channel slices of a layer's output
+    static constexpr int kFrameBytes = kPlaneBytes * (kC / 8);       // 46336 / 92672 per group
+    static constexpr int kTileBytes = kC * 32;                       // one tap: N = C rows x 32 bytes of K
+    static constexpr int kStageTaps = kC == 128 ? 9 : 3;
+    static constexpr int kStagesPerSlice = 9 / kStageTaps;
+    static constexpr int kStageBytes = kStageTaps * kTileBytes;      // 36864 / 24576
+    static constexpr int kStages = kC == 128 ? 3 : 5;
+    static constexpr int kEpiWarps = 4 * kGroups;
+    static constexpr int kThreads = 32 * (1 + kGroups + kEpiWarps);  // producer, one issuer per group, 4 epilogue warps per group
+    static constexpr uint32_t kBDescLbo = (uint32_t)kC << 16;        // K core matrices C*16 bytes apart
+    static constexpr int kOffFrames = 0;
+    static constexpr int kOffWeights = kGroups * kFrameBytes;
+    static constexpr int kOffBars = kOffWeights + kStages * kStageBytes;
+    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done
+    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1;
+    static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
+    static constexpr int kOffAbort = kOffTmemPtr + 4;
+    static constexpr int kOffConst = (kOffAbort + 4 + 15) & ~15;     // per-warp copies of the current layer's channel constants
+    static constexpr int smem_bytes(bool fp8) { return kOffConst + kEpiWarps * (fp8 ? 4 : 1) * kC * 4 + 128 * 4; }
+    static_assert(kOffConst + kEpiWarps * 4 * kC * 4 + 512 <= kMaxSmem || kC == 256, "shared memory budget");
+    static_assert(kGroups * 2 * kC == (int)kTmemCols, "TMEM: per group C columns of residual stream and C of accumulator");
+};
 
 struct TowerArgs {
-    const __nv_bfloat16 *planes;     // [batch][64][32]
-    const __nv_bfloat16 *weights;    // packed stages
-    const float *bias;               // [n_conv][128]
-    __nv_bfloat16 *out;              // [batch][64][128]
+    const __nv_bfloat16 *planes;     // [batch][64][in_pad]
+    const void *weights;             // packed stages
+    const float *bias;               // [n_conv][C]
+    __nv_bfloat16 *out;              // [batch][64][C] or null
     uint32_t *status;
     int batch;
     int n_conv;                      // 1 + 2*blocks
-    int in_kc;                       // 16-channel slices of the input layer (2)
-    int bias_in_smem;                // all biases staged in shared memory (n_conv <= kMaxBiasLayers)
+    int in_pad;                      // channels of the plane tensor (32 or 128)
     int trace;                       // CTA 0 prints how long each role waited (debugging aid)
     // fused 1x1 head projections (one extra MMA layer on the final activations); head_n == 0: none
     int head_n;                      // 64: flat policy proj (32) | value proj (32); 112: 73 policy planes (+7 pad) | value proj (32)
-    const __nv_bfloat16 *head_w;     // packed [kc 8][k8 2][n-group head_n/8][8][8]
+    const __nv_bfloat16 *head_w;     // packed [slice][k8 2][n-group head_n/8][8][8]
     const float *head_bias;          // [head_n]
     __nv_bfloat16 *u_policy;         // flat head: projection as GEMM A tiles, K index = square*32 + channel
     __nv_bfloat16 *u_value;          // value projection, same layout
     float *logits;                   // 73-plane head: [batch][73*64] fp32 logits, index = plane*64 + square
-    // FP8 tower: per-layer channel constants [n_conv][4][128]: output scale, bias, 1/next activation
+    // FP8 tower: per-layer channel constants [n_conv][4][C]: output scale, bias, 1/next activation
     // scale, 1/(next conv2 weight scale) for the residual stream kept in TMEM
     const float *lconst;
     // calibration run (bf16 kernel): per-layer, per-channel maximum of the layer outputs, as float bits
-    unsigned int *absmax;            // [n_conv][128]
+    unsigned int *absmax;            // [n_conv][C]
 };
-constexpr int kLconstFloats = 4 * kC;                       // per layer
-constexpr int kLconstSmemBytes = 4 * kGroups * kLconstFloats * 4;   // a private copy per epilogue warp: 16 KB
 
 // Bounded wait, called by all 32 lanes of a warp together.  Returns false (to every lane alike) if
 // the CTA has been aborted or this wait ran out; the latter raises the abort flag and the status bit.
@@ -122,38 +129,40 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     return __all_sync(0xffffffffu, done);
 }
 
-template <bool kFp8>
-__global__ void __launch_bounds__(kThreads, 1)
+// slices of the head projection's K that travel in one weight stage
+template <class S> __device__ __host__ constexpr int head_slices_per_stage(int head_n) {
+    return S::kC == 128 ? S::kSlices : (head_n == 64 ? 8 : 4);
+}
+
+template <bool kFp8, class S>
+__global__ void __launch_bounds__(S::kThreads, 1)
 tower_tc_kernel(const TowerArgs args) {
+    constexpr int kC = S::kC, kGroups = S::kGroups, kStages = S::kStages, kSlices = S::kSlices;
+    constexpr int kFrameBytes = S::kFrameBytes, kStageBytes = S::kStageBytes, kThreads = S::kThreads;
+    static_assert(!kFp8 || kC == 128, "the FP8 tower exists for 128 channels");
     extern __shared__ __align__(128) unsigned char smem[];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t smem_base = ptx::smem_addr(smem);
-    const uint32_t bars = smem_base + kOffBars;
+    const uint32_t bars = smem_base + S::kOffBars;
     auto bar_w_full = [&](int s) { return bars + 8u * s; };
     auto bar_w_empty = [&](int s) { return bars + 8u * (kStages + s); };
     auto bar_acc_full = [&](int g) { return bars + 8u * (2 * kStages + g); };
-    auto bar_a_ready = [&](int g, int kc) { return bars + 8u * (2 * kStages + kGroups + g * 8 + kc); };
-    const uint32_t bar_done = bars + 8u * (kNumBars - 1);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffAbort);
-    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + kOffTmemPtr);
+    auto bar_a_ready = [&](int g, int kc) { return bars + 8u * (2 * kStages + kGroups + g * kSlices + kc); };
+    const uint32_t bar_done = bars + 8u * (S::kNumBars - 1);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + S::kOffAbort);
+    uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + S::kOffTmemPtr);
+    constexpr int kConstFloats = (kFp8 ? 4 : 1) * kC;          // per layer: (scale, bias, 1/act scale, 1/h scale) or bias
+    float *head_bias_smem = reinterpret_cast<float *>(smem + S::kOffConst) + S::kEpiWarps * kConstFloats;
 
     // ---- set-up: zero the frames (their borders stay zero for the kernel's lifetime), barriers, TMEM
     for (int i = threadIdx.x; i < kGroups * kFrameBytes / 16; i += kThreads)
-        reinterpret_cast<uint4 *>(smem + kOffFrames)[i] = make_uint4(0, 0, 0, 0);
-    if (kFp8) {
-        for (int i = threadIdx.x; i < args.head_n; i += kThreads)
-            reinterpret_cast<float *>(smem + kOffBias + kLconstSmemBytes)[i] = args.head_bias[i];
-    } else if (args.bias_in_smem) {
-        for (int i = threadIdx.x; i < args.n_conv * kC; i += kThreads)
-            reinterpret_cast<float *>(smem + kOffBias)[i] = args.bias[i];
-        for (int i = threadIdx.x; i < args.head_n; i += kThreads)
-            reinterpret_cast<float *>(smem + kOffBias)[args.n_conv * kC + i] = args.head_bias[i];
-    }
+        reinterpret_cast<uint4 *>(smem + S::kOffFrames)[i] = make_uint4(0, 0, 0, 0);
+    for (int i = threadIdx.x; i < args.head_n; i += kThreads) head_bias_smem[i] = args.head_bias[i];
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { ptx::mbar_init(bar_w_full(s), 1); ptx::mbar_init(bar_w_empty(s), kGroups); }
         for (int g = 0; g < kGroups; ++g) {
             ptx::mbar_init(bar_acc_full(g), 1);
-            for (int kc = 0; kc < 8; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4);
+            for (int kc = 0; kc < kSlices; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4);
         }
         ptx::mbar_init(bar_done, kGroups);
         *abort_flag = 0;
@@ -169,9 +178,11 @@ tower_tc_kernel(const TowerArgs args) {
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_smem;
 
-    const int n_units = (args.batch + kBoardsPerCta - 1) / kBoardsPerCta;
+    const int n_units = (args.batch + S::kBoardsPerCta - 1) / S::kBoardsPerCta;
     const int n_conv = args.n_conv;
     const int head_n = args.head_n;
+    const int in_slices = args.in_pad / 16;
+    const int hsps = head_slices_per_stage<S>(head_n);
     const bool tr = args.trace && blockIdx.x == 0;
     long long t_wait[3] = {0, 0, 0};
     long long t_issue = 0;
@@ -181,37 +192,29 @@ tower_tc_kernel(const TowerArgs args) {
         // ================= weight producer =================
         int stage = 0;
         uint32_t phase = 0;
-        uint32_t last_parity[kStages] = {0, 0, 0};
-        bool issued[kStages] = {false, false, false};
+        uint32_t last_parity[kStages] = {};
+        bool issued[kStages] = {};
         bool ok = true;
+        auto push = [&](const unsigned char *src, uint32_t bytes) {
+            ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+            if (!ok) return;
+            if (lane == 0) {
+                ptx::mbar_arrive_expect_tx(bar_w_full(stage), bytes);
+                ptx::bulk_copy_g2s(smem_base + S::kOffWeights + stage * kStageBytes, src, bytes, bar_w_full(stage));
+            }
+            issued[stage] = true; last_parity[stage] = phase;
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            __syncwarp();
+        };
         for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
             const unsigned char *src = reinterpret_cast<const unsigned char *>(args.weights);
             for (int l = 0; l < n_conv && ok; ++l) {
-                const int nkc = l == 0 ? args.in_kc : (kFp8 ? kC / 32 : kC / 16);     // K per MMA: 16 bf16 or 32 e4m3
-                for (int kc = 0; kc < nkc; ++kc) {
-                    ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
-                    if (!ok) break;
-                    if (lane == 0) {
-                        ptx::mbar_arrive_expect_tx(bar_w_full(stage), kStageBytes);
-                        ptx::bulk_copy_g2s(smem_base + kOffWeights + stage * kStageBytes, src, kStageBytes, bar_w_full(stage));
-                    }
-                    issued[stage] = true; last_parity[stage] = phase;
-                    src += kStageBytes;
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
-                    __syncwarp();
-                }
+                const int nkc = l == 0 ? in_slices : (kFp8 ? kC / 32 : kC / 16);     // K per MMA: 16 bf16 or 32 e4m3
+                for (int st = 0; st < nkc * S::kStagesPerSlice && ok; ++st) { push(src, kStageBytes); src += kStageBytes; }
             }
-            if (head_n && ok) {                              // the head projections: one small stage
-                ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
-                if (!ok) break;
-                if (lane == 0) {
-                    ptx::mbar_arrive_expect_tx(bar_w_full(stage), (uint32_t)head_n * 256u);
-                    ptx::bulk_copy_g2s(smem_base + kOffWeights + stage * kStageBytes, args.head_w, (uint32_t)head_n * 256u, bar_w_full(stage));
-                }
-                issued[stage] = true; last_parity[stage] = phase;
-                if (++stage == kStages) { stage = 0; phase ^= 1u; }
-                __syncwarp();
-            }
+            if (head_n)                                        // the head projections: small stages of their own
+                for (int st = 0; st < kSlices / hsps && ok; ++st)
+                    push(reinterpret_cast<const unsigned char *>(args.head_w) + (size_t)st * hsps * head_n * 32, (uint32_t)(hsps * head_n * 32));
         }
         if (!ok) {
             // copies already in flight must land before the CTA's shared memory is released
@@ -223,18 +226,18 @@ tower_tc_kernel(const TowerArgs args) {
     } else if (warp <= kGroups) {
         // ================= MMA issuer of group g =================
         const int g = warp - 1;
-        constexpr uint32_t idesc = ptx::idesc_bf16_f32(128, 128);
-        constexpr uint32_t idesc8 = ptx::idesc_e4m3_f32(128, 128);
+        constexpr uint32_t idesc = ptx::idesc_bf16_f32(128, kC);
+        constexpr uint32_t idesc8 = ptx::idesc_e4m3_f32(128, kC);
         int stage = 0;
         uint32_t phase = 0;
         uint32_t a_phase = 0;
         bool ok = true;
-        const uint32_t d_h = tmem_base + (uint32_t)(g * 256);
-        const uint32_t frame_lo = (((smem_base + kOffFrames + g * kFrameBytes) >> 4) + (uint32_t)(kNB * 9 + 1)) | kADescLbo;
+        const uint32_t d_h = tmem_base + (uint32_t)(g * 2 * kC);
+        const uint32_t frame_lo = (((smem_base + S::kOffFrames + g * kFrameBytes) >> 4) + (uint32_t)(kNB * 9 + 1)) | kADescLbo;
         const int n_layers = n_conv + (head_n ? 1 : 0);
         uint32_t lead_parity = 0;                                      // parity of group 0's next layer-0 completion
         for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
-            if (g == 1 && n_conv >= 3 && !(args.trace & 2)) {
+            if (kGroups == 2 && g == 1 && n_conv >= 3 && !(args.trace & 2)) {
                 // Start one (short) input layer behind group 0.  The groups then reach their layer
                 // boundaries at different times, so one group's wait for its epilogue is covered by
                 // the other's MMAs instead of idling the tensor pipe for both at once.
@@ -243,63 +246,69 @@ tower_tc_kernel(const TowerArgs args) {
                 lead_parity ^= (uint32_t)(n_layers & 1);
             }
             for (int l = 0; l < n_conv && ok; ++l) {
-                const int nkc = l == 0 ? args.in_kc : (kFp8 ? kC / 32 : kC / 16);
+                const int nkc = l == 0 ? in_slices : (kFp8 ? kC / 32 : kC / 16);
                 const bool e4m3 = kFp8 && l > 0;                       // the input layer stays bf16
                 const bool conv2 = l >= 2 && (l & 1) == 0;             // accumulates onto the residual stream
-                const uint32_t d = d_h + (((l & 1) == 1) ? 128u : 0u); // conv1 writes the ACC columns
-                for (int kc = 0; kc < nkc; ++kc) {
-                    ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
-                    if (!ok) break;
+                const uint32_t d = d_h + (((l & 1) == 1) ? (uint32_t)kC : 0u);   // conv1 writes the ACC columns
+                for (int kc = 0; kc < nkc && ok; ++kc) {
                     ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
                     if (!ok) break;
                     a_phase ^= 1u << kc;
-                    ptx::tc_fence_after();
-                    const long long ti0 = tr ? clock64() : 0;
-                    if (lane == 0) {
-                        // low descriptor words in 16-byte units; row m = 0 sits at slot 2*9 + 1 = 19
-                        const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
-                        const uint32_t b_lo = ((smem_base + kOffWeights + stage * kStageBytes) >> 4) | kBDescLbo;
-                        const uint32_t first = (conv2 || kc > 0) ? 1u : 0u;
+                    // low descriptor word in 16-byte units; row m = 0 sits at slot 2*9 + 1 = 19
+                    const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
 #pragma unroll
-                        for (int tap = 0; tap < 9; ++tap) {
-                            const int dy = tap / 3 - 1, dx = tap % 3 - 1;
-                            if (e4m3)
-                                ptx::mma_e4m3_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                    b_lo + (uint32_t)(tap * (kTileBytes / 16)), kBDescHi, idesc8,
-                                                    tap == 0 ? first : 1u);
-                            else
-                                ptx::mma_bf16_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                    b_lo + (uint32_t)(tap * (kTileBytes / 16)), kBDescHi, idesc,
-                                                    tap == 0 ? first : 1u);
+                    for (int st = 0; st < S::kStagesPerSlice; ++st) {
+                        ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+                        if (!ok) break;
+                        ptx::tc_fence_after();
+                        const long long ti0 = tr ? clock64() : 0;
+                        if (lane == 0) {
+                            const uint32_t b_lo = ((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) | S::kBDescLbo;
+#pragma unroll
+                            for (int t = 0; t < S::kStageTaps; ++t) {
+                                const int tap = st * S::kStageTaps + t;
+                                const int dy = tap / 3 - 1, dx = tap % 3 - 1;
+                                const uint32_t acc = (tap == 0 && !conv2 && kc == 0) ? 0u : 1u;
+                                if (e4m3)
+                                    ptx::mma_e4m3_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                                        b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8, acc);
+                                else
+                                    ptx::mma_bf16_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                                        b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc, acc);
+                            }
+                            if (kc == nkc - 1 && st == S::kStagesPerSlice - 1) ptx::mma_commit(bar_acc_full(g));
+                            ptx::mma_commit(bar_w_empty(stage));
                         }
-                        if (kc == nkc - 1) ptx::mma_commit(bar_acc_full(g));
-                        ptx::mma_commit(bar_w_empty(stage));
+                        __syncwarp();
+                        if (tr) t_issue += clock64() - ti0;
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
-                    __syncwarp();
-                    if (tr) t_issue += clock64() - ti0;
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
             if (head_n && ok) {
                 // head projections: a 1x1 convolution = the centre tap only, N = head_n, into the ACC columns
                 const uint32_t idesc_h = ptx::idesc_bf16_f32(128, head_n);
-                ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
-                if (!ok) break;
-                for (int kc = 0; kc < kC / 16; ++kc) {
+                for (int kc = 0; kc < kSlices && ok; ++kc) {
+                    if (kc % hsps == 0) {
+                        ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+                        if (!ok) break;
+                    }
                     ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
                     if (!ok) break;
                     a_phase ^= 1u << kc;
                     ptx::tc_fence_after();
+                    const bool stage_done = (kc % hsps) == hsps - 1;
                     if (lane == 0) {
                         const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
-                        const uint32_t b_lo = (((smem_base + kOffWeights + stage * kStageBytes) >> 4) + (uint32_t)(kc * head_n * 2)) |
+                        const uint32_t b_lo = (((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) + (uint32_t)((kc % hsps) * head_n * 2)) |
                                               ((uint32_t)head_n << 16);          // K core matrices head_n*16 bytes apart
-                        ptx::mma_bf16_split(d_h + 128u, a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u);
-                        if (kc == kC / 16 - 1) { ptx::mma_commit(bar_acc_full(g)); ptx::mma_commit(bar_w_empty(stage)); }
+                        ptx::mma_bf16_split(d_h + (uint32_t)kC, a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u);
+                        if (kc == kSlices - 1) ptx::mma_commit(bar_acc_full(g));
+                        if (stage_done) ptx::mma_commit(bar_w_empty(stage));
                     }
                     __syncwarp();
+                    if (stage_done && ++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
-                if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
         }
         // all issued MMAs must have completed before TMEM is freed
@@ -309,66 +318,63 @@ tower_tc_kernel(const TowerArgs args) {
             if (ptx::mbar_try_wait(bar_done, 0)) break;
     } else {
         // ================= epilogue: 4 warps per group =================
-        const int g = (warp - 1 - kGroups) >> 2;
+        const int ew = warp - 1 - kGroups;                    // 0 .. 4*groups-1
+        const int g = ew >> 2;
         const int q = warp & 3;                               // TMEM lane quarter this warp may access
         const int m = q * 32 + lane;                          // GEMM row = TMEM lane
         const int g8 = m >> 3, y = g8 >> 1, b = g8 & 1, x = m & 7;
         const int slot = (g8 + kNB) * 9 + x + 1;
-        unsigned char *frame = smem + kOffFrames + g * kFrameBytes;
-        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 256);
+        unsigned char *frame = smem + S::kOffFrames + g * kFrameBytes;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 2 * kC);
+        float *lc = reinterpret_cast<float *>(smem + S::kOffConst) + ew * kConstFloats;   // this warp's copy of the layer constants
         uint32_t acc_phase = 0;
         bool ok = true;
         for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
-            const int board = unit * kBoardsPerCta + g * kNB + b;
+            const int board = unit * S::kBoardsPerCta + g * kNB + b;
             const bool live = board < args.batch;
             const int sq = y * 8 + x;
-            // ---- the unit's input planes -> frame slices 0..3 (32 channels)
+            // ---- the unit's input planes -> the first in_pad/8 planes of the frame
             {
-                const uint4 *src = reinterpret_cast<const uint4 *>(args.planes + ((size_t)board * 64 + sq) * 32);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(args.planes + ((size_t)board * 64 + sq) * args.in_pad);
+                for (int j = 0; j < args.in_pad / 8; ++j) {
                     const uint4 v = live ? __ldg(src + j) : make_uint4(0, 0, 0, 0);
                     *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = v;
                 }
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) { ptx::mbar_arrive(bar_a_ready(g, 0)); ptx::mbar_arrive(bar_a_ready(g, 1)); }
+                if (lane == 0)
+                    for (int kc = 0; kc < in_slices; ++kc) ptx::mbar_arrive(bar_a_ready(g, kc));
             }
             for (int l = 0; l < n_conv && ok; ++l) {
                 const bool from_acc = (l & 1) == 1;
                 const bool last = l == n_conv - 1 && head_n == 0;        // nothing follows: results go to global only
                 const bool to_global = l == n_conv - 1 && args.out != nullptr;
                 const bool next_e4m3 = kFp8 && l + 1 < n_conv;           // the next layer reads e4m3 operands
-                const float *lc = nullptr;
-                if (kFp8) {
+                {
                     // this layer's channel constants -> this warp's own copy in shared memory (every thread
-                    // needs all 128 channels; a private copy needs no cross-warp barrier, which could not
-                    // be bounded the way the mbarrier waits are)
-                    float *buf = reinterpret_cast<float *>(smem + kOffBias) + (warp - 1 - kGroups) * kLconstFloats;
+                    // needs all channels; a private copy needs no cross-warp barrier, which could not be
+                    // bounded the way the mbarrier waits are).  Issued before the wait below hides its latency.
+                    const float *src = kFp8 ? args.lconst + (size_t)l * kConstFloats : args.bias + (size_t)l * kC;
                     __syncwarp();
 #pragma unroll
-                    for (int i = 0; i < kLconstFloats / 4 / 32; ++i)
-                        reinterpret_cast<float4 *>(buf)[i * 32 + lane] =
-                            __ldg(reinterpret_cast<const float4 *>(args.lconst + (size_t)l * kLconstFloats) + i * 32 + lane);
+                    for (int i = 0; i < kConstFloats / 4 / 32; ++i)
+                        reinterpret_cast<float4 *>(lc)[i * 32 + lane] = __ldg(reinterpret_cast<const float4 *>(src) + i * 32 + lane);
                     __syncwarp();
-                    lc = buf;
                 }
                 ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 acc_phase ^= 1u;
                 ptx::tc_fence_after();
-                const float *bias = kFp8 ? lc + kC
-                                  : args.bias_in_smem ? reinterpret_cast<const float *>(smem + kOffBias) + l * kC
-                                                      : args.bias + (size_t)l * kC;
+                const float *bias = kFp8 ? lc + kC : lc;
                 __nv_bfloat16 *dst = args.out + ((size_t)board * 64 + sq) * kC;
-                const uint32_t t_src = t_lane + (uint32_t)(from_acc ? 128 : 0);
+                const uint32_t t_src = t_lane + (uint32_t)(from_acc ? kC : 0);
                 const bool keep_h = !from_acc && l != n_conv - 1;   // the residual stream stays in TMEM as fp32
                 uint32_t r[2][16];
                 ptx::tmem_ld16(t_src, r[0]);
 #pragma unroll
-                for (int kc = 0; kc < kC / 16; ++kc) {
+                for (int kc = 0; kc < kSlices; ++kc) {
                     ptx::tmem_ld_wait();
-                    if (kc + 1 < kC / 16) ptx::tmem_ld16(t_src + (uint32_t)((kc + 1) * 16), r[(kc + 1) & 1]);
+                    if (kc + 1 < kSlices) ptx::tmem_ld16(t_src + (uint32_t)((kc + 1) * 16), r[(kc + 1) & 1]);
                     uint32_t(&rr)[16] = r[kc & 1];
                     float v[16];
 #pragma unroll
@@ -457,8 +463,7 @@ tower_tc_kernel(const TowerArgs args) {
                 if (!ok) break;
                 acc_phase ^= 1u;
                 ptx::tc_fence_after();
-                const float *hb = kFp8 ? reinterpret_cast<const float *>(smem + kOffBias + kLconstSmemBytes)
-                                : args.bias_in_smem ? reinterpret_cast<const float *>(smem + kOffBias) + n_conv * kC : args.head_bias;
+                const float *hb = head_bias_smem;
                 // this row's place in the GEMM A tiles: [tile of 128 boards][8-wide K chunk][board/8][board%8][8 k]
                 const size_t u_row = ((size_t)(board >> 7) * 256 * 16 + (size_t)((board & 127) >> 3)) * 128 + (size_t)(board & 7) * 16;
                 const int n_slices = head_n / 16;
@@ -466,7 +471,7 @@ tower_tc_kernel(const TowerArgs args) {
 #pragma unroll 1
                 for (int j = 0; j < n_slices; ++j) {
                     uint32_t rr[16];
-                    ptx::tmem_ld16(t_lane + 128u + (uint32_t)(j * 16), rr);
+                    ptx::tmem_ld16(t_lane + (uint32_t)kC + (uint32_t)(j * 16), rr);
                     ptx::tmem_ld_wait();
                     float v[16];
 #pragma unroll
@@ -498,7 +503,7 @@ tower_tc_kernel(const TowerArgs args) {
         }
     }
 
-    if (tr && lane == 0 && (warp < 4 || warp == 7))
+    if (tr && lane == 0 && (warp <= kGroups + 1))
         printf("tower trace: warp %d total %lld clk, waited %lld / %lld / %lld clk, issue %lld clk\n", warp, clock64() - t_begin,
                t_wait[0], t_wait[1], t_wait[2], t_issue);
     // ---- teardown
@@ -510,13 +515,17 @@ tower_tc_kernel(const TowerArgs args) {
     }
 }
 
+typedef Shape<128, 2> Shape128;
+typedef Shape<256, 1> Shape256;
+constexpr int kStageBytes = Shape128::kStageBytes;       // host-side packing of the 128-channel stages
+
 }  // namespace
 
 // Packed layout: for layer l, 16-channel slice kc, tap, the N=128 x K=16 tile as core matrices
 // [k8 (2)][n-group (16)][n in group (8)][k in slice (8)] bf16, scale folded into the weights.
 size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv) {
-    const size_t stages = (size_t)in_pad / 16 + (size_t)(n_conv - 1) * (channels / 16);
-    return stages * kStageBytes;
+    const size_t slices = (size_t)in_pad / 16 + (size_t)(n_conv - 1) * (channels / 16);
+    return slices * 9 * (size_t)channels * 32;             // per slice and tap: N = channels rows x 32 bytes of K
 }
 
 void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
@@ -600,7 +609,7 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
 // Head projections as one N = head_n tile per 16-channel slice: rows [0, n_policy) the policy
 // projection (scaled where it has a folded batch-norm), zero rows up to n_policy_pad, then the 32
 // rows of the value projection.  Same core-matrix order as the tower's weight tiles.
-size_t tc_head_weight_bytes(int head_n) { return (size_t)head_n * 256; }
+size_t tc_head_weight_bytes(int head_n, int channels) { return (size_t)head_n * channels * 2; }
 
 void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,
                   int channels, __nv_bfloat16 *packed) {
@@ -628,21 +637,23 @@ int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_o
     if (dev < 64 && sm_count[dev] == 0) {
         int n = 0;
         AZ_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
-        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
-        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
     const int sms = dev < 64 ? sm_count[dev] : 148;
     const bool fp8 = net.fp8_ready && absmax == nullptr;      // the calibration pass itself runs in bf16
+    const bool wide = net.arch.channels == 256;
     TowerArgs a;
     a.planes = static_cast<const __nv_bfloat16 *>(planes);
-    a.weights = static_cast<const __nv_bfloat16 *>(fp8 ? net.tc8_weights : net.tc_weights);
+    a.weights = fp8 ? net.tc8_weights : net.tc_weights;
     a.bias = net.tc_bias;
     a.out = static_cast<__nv_bfloat16 *>(tower_out);
     a.status = net.status_dev;
     a.batch = batch;
     a.n_conv = net.n_conv;
-    a.in_kc = net.in_pad / 16;
+    a.in_pad = net.in_pad;
     a.head_n = with_heads ? net.tc_head_n : 0;
     a.head_w = static_cast<const __nv_bfloat16 *>(net.tc_head_w);
     a.head_bias = net.tc_head_bias;
@@ -651,18 +662,14 @@ int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_o
     a.logits = net.logits;
     a.lconst = net.tc8_lconst;
     a.absmax = absmax;
-    a.bias_in_smem = net.n_conv + 1 <= kMaxBiasLayers ? 1 : 0;
     static const bool trace = getenv("AZ_TOWER_TRACE") != nullptr;
     a.trace = trace ? atoi(getenv("AZ_TOWER_TRACE")) : 0;
-    const int n_units = (batch + kBoardsPerCta - 1) / kBoardsPerCta;
+    const int boards_per_cta = wide ? Shape256::kBoardsPerCta : Shape128::kBoardsPerCta;
+    const int n_units = (batch + boards_per_cta - 1) / boards_per_cta;
     const int grid = n_units < sms ? n_units : sms;
-    if (fp8) {
-        const int smem_bytes = kSmemBytesNoBias + kLconstSmemBytes + kC * 4;
-        tower_tc_kernel<true><<<grid, kThreads, smem_bytes, s>>>(a);
-    } else {
-        const int smem_bytes = kSmemBytesNoBias + (a.bias_in_smem ? (net.n_conv + 1) * kC * 4 : 0);
-        tower_tc_kernel<false><<<grid, kThreads, smem_bytes, s>>>(a);
-    }
+    if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
+    else if (fp8) tower_tc_kernel<true, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(true), s>>>(a);
+    else tower_tc_kernel<false, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(false), s>>>(a);
     AZ_LAUNCH_CHECK();
     return AZ_OK;
 }
