@@ -224,6 +224,15 @@ int az_device_status(az_net *net, void *cuda_stream, uint32_t *status_out);
 int az_profile_tower(az_net *net, int enable);
 int az_tower_time(az_net *net, float *total_ms_out, int *passes_out);
 
+/*
+ * Self-test of the failure path: launches a one-CTA kernel whose warps wait, through the same
+ * bounded wait as the tensor-core kernels, on a barrier nothing ever arrives on (poll limit a few
+ * tens of microseconds).  Returns AZ_ERR_DEVICE_TIMEOUT when the wait ran out, the kernel raised its
+ * status bit and still left through its normal teardown -- i.e. when failure detection works --
+ * and AZ_OK / another error otherwise.  Nothing hangs or traps; the context stays usable.
+ */
+int az_selftest_wait_timeout(void *cuda_stream);
+
 /* Number of kernel launches one az_evaluate of `batch` positions enqueues. */
 int az_launches_per_evaluate(const az_net *net, int batch);
 

@@ -24,7 +24,7 @@ AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3 = 0, 1, 2
 
 EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
            "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_host", "az_encode", "az_tower", "az_tower_static", "az_legal_masks",
-           "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_launches_per_evaluate", "az_strerror",
+           "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error")
 
 
@@ -74,6 +74,8 @@ def _load_library():
     lib.az_calibrate.argtypes = [vp, vp, ci, vp]
     lib.az_device_status.restype = ci
     lib.az_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.az_selftest_wait_timeout.restype = ci
+    lib.az_selftest_wait_timeout.argtypes = [vp]
     lib.az_launches_per_evaluate.restype = ci
     lib.az_launches_per_evaluate.argtypes = [vp, ci]
     lib.az_strerror.restype = ctypes.c_char_p
@@ -224,6 +226,11 @@ def az_device_status(net: Net, stream=None) -> int:
     if code not in (AZ_OK, AZ_ERR_DEVICE_TIMEOUT):
         raise AzError(code, "az_device_status")
     return int(status.value)
+
+
+def az_selftest_wait_timeout(stream=None) -> int:
+    """Returns the library's code: AZ_ERR_DEVICE_TIMEOUT means the bounded wait ran out as it should."""
+    return int(_lib.az_selftest_wait_timeout(_stream_ptr(stream)))
 
 
 def az_launches_per_evaluate(net: Net, batch: int) -> int:

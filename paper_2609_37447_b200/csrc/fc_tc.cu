@@ -47,16 +47,7 @@ struct FcArgs {
 };
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status) {
-    bool done = false;
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (ptx::mbar_try_wait(bar, parity)) { done = true; break; }
-        if ((i & 63u) == 63u && *abort_flag) break;
-    }
-    if (!done && !*abort_flag) {
-        *abort_flag = 1;
-        atomicOr(status, kStatusWaitTimeout);
-    }
-    return __all_sync(0xffffffffu, done);
+    return bounded_wait(bar, parity, abort_flag, status, kStatusWaitTimeout, kSpinLimit);
 }
 
 __global__ void __launch_bounds__(kThreads, 1)

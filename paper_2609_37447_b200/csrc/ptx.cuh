@@ -139,4 +139,25 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 }  // namespace ptx
+
+// Bounded mbarrier wait, called by all 32 lanes of a warp together.  Polls at most `limit` times.
+// Returns false (to every lane alike) if the CTA has been aborted or this wait ran out; the latter
+// raises the CTA's abort flag and ORs `timeout_bit` into the status word the host reads.  Callers
+// stop issuing work, drain what is in flight and leave through their normal teardown.
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
+                                             uint32_t timeout_bit, uint32_t limit, long long *waited = nullptr) {
+    const long long t0 = waited ? clock64() : 0;
+    bool done = false;
+    for (uint32_t i = 0; i < limit; ++i) {
+        if (ptx::mbar_try_wait(bar, parity)) { done = true; break; }
+        if ((i & 63u) == 63u && *abort_flag) break;
+    }
+    if (!done && !*abort_flag) {
+        *abort_flag = 1;
+        atomicOr(status, timeout_bit);
+    }
+    if (waited) *waited += clock64() - t0;
+    return __all_sync(0xffffffffu, done);
+}
+
 }  // namespace az

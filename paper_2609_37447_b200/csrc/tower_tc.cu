@@ -111,22 +111,9 @@ struct TowerArgs {
     unsigned int *absmax;            // [n_conv][C]
 };
 
-// Bounded wait, called by all 32 lanes of a warp together.  Returns false (to every lane alike) if
-// the CTA has been aborted or this wait ran out; the latter raises the abort flag and the status bit.
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
                                          long long *waited = nullptr) {
-    const long long t0 = waited ? clock64() : 0;
-    bool done = false;
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (ptx::mbar_try_wait(bar, parity)) { done = true; break; }
-        if ((i & 63u) == 63u && *abort_flag) break;
-    }
-    if (!done && !*abort_flag) {
-        *abort_flag = 1;
-        atomicOr(status, kStatusWaitTimeout);
-    }
-    if (waited) *waited += clock64() - t0;
-    return __all_sync(0xffffffffu, done);
+    return bounded_wait(bar, parity, abort_flag, status, kStatusWaitTimeout, kSpinLimit, waited);
 }
 
 // slices of the head projection's K that travel in one weight stage
