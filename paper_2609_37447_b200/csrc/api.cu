@@ -262,18 +262,21 @@ void free_net(Net *n) {
 // encoder + tower; *tower_out receives the buffer holding [batch][64][C].  With `fused_heads` (tensor-core
 // path only) the tower kernel also runs the 1x1 head projections and leaves the activations on chip.
 int run_tower(Net &n, const void *positions, int batch, void **tower_out, bool fused_heads, cudaStream_t s) {
-    int rc = launch_encode(positions, az_position_bytes(&n.arch), batch, (int)n.arch.in_planes, n.in_pad,
-                           n.bf16, n.planes, n.status_dev, s);
-    if (rc != AZ_OK) return rc;
+    int rc = AZ_OK;
     const int C = (int)n.arch.channels;
     const bool timed = n.profile && n.n_events < kMaxProfiledPasses;
-    if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
     if (n.tc_ready) {
+        // the tensor-core tower encodes its boards itself, straight into shared memory
+        if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
         *tower_out = fused_heads ? nullptr : n.act[0];
-        rc = launch_tower_tc(n, n.planes, batch, *tower_out, fused_heads, nullptr, s);
+        rc = launch_tower_tc(n, nullptr, positions, batch, *tower_out, fused_heads, nullptr, s);
         if (rc == AZ_OK && timed) AZ_CUDA(cudaEventRecord(n.ev_end[n.n_events++], s));
         return rc;
     }
+    rc = launch_encode(positions, az_position_bytes(&n.arch), batch, (int)n.arch.in_planes, n.in_pad,
+                       n.bf16, n.planes, n.status_dev, s);
+    if (rc != AZ_OK) return rc;
+    if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
     void *x = n.act[0], *t = n.act[1], *y = n.act[2];
     rc = launch_conv3x3_simt(n.planes, n.conv_w[0], n.conv_scale[0], n.conv_bias[0], nullptr, x, batch,
                              n.in_pad, C, n.bf16, s);
@@ -477,8 +480,7 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
     for (int first = 0; first < count && rc == AZ_OK && e == cudaSuccess; first += (int)n->arch.max_batch) {
         const int chunk = count - first < (int)n->arch.max_batch ? count - first : (int)n->arch.max_batch;
         const unsigned char *p = static_cast<const unsigned char *>(positions_dev) + (size_t)first * pb;
-        rc = az::launch_encode(p, pb, chunk, (int)n->arch.in_planes, n->in_pad, true, n->planes, n->status_dev, s);
-        if (rc == AZ_OK) rc = az::launch_tower_tc(*n, n->planes, chunk, nullptr, false, absmax_dev, s);
+        rc = az::launch_tower_tc(*n, nullptr, p, chunk, nullptr, false, absmax_dev, s);
     }
     std::vector<float> absmax((size_t)L * C);
     if (rc == AZ_OK && e == cudaSuccess) e = cudaMemcpyAsync(absmax.data(), absmax_dev, absmax.size() * sizeof(float), cudaMemcpyDeviceToHost, s);
@@ -515,7 +517,7 @@ int az_device_status(az_net *net, void *cuda_stream, uint32_t *status_out) {
 int az_launches_per_evaluate(const az_net *net, int batch) {
     const Net *n = reinterpret_cast<const Net *>(net);
     if (!n || batch <= 0) return 0;
-    if (n->tc_ready) return 1 /*encode*/ + az::tower_tc_launch_count() + 1 /*head GEMMs*/ + 1 /*softmax*/;
+    if (n->tc_ready) return az::tower_tc_launch_count() /*encoder + tower + head projections*/ + 1 /*head GEMMs*/ + 1 /*softmax*/;
     const int policy = n->arch.policy_head == AZ_POLICY_PLANES73 ? 1 : 2;
     return 1 /*encode*/ + n->n_conv + policy + 3 /*value*/ + 1 /*softmax*/;
 }

@@ -123,8 +123,9 @@ int launch_masked_softmax(const float *logits, const uint64_t *masks, int batch,
 size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv);
 void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
                      int channels, int n_conv, __nv_bfloat16 *packed_host);
-int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, bool with_heads,
-                    unsigned int *absmax, cudaStream_t s);
+// exactly one of `planes` (encoded plane tensor) and `positions` (records to encode in the kernel) is non-null
+int launch_tower_tc(const Net &net, const void *planes, const void *positions, int batch, void *tower_out,
+                    bool with_heads, unsigned int *absmax, cudaStream_t s);
 size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv);
 void tc8_pack(const float *const *w, const float *const *scale, const float *const *bias, const float *absmax,
               int in_planes, int in_pad, int channels, int n_conv, unsigned char *packed, float *lconst);

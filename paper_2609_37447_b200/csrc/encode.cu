@@ -8,70 +8,10 @@
 // read by all 64 threads of that position from the same words (broadcast through L1).
 // HBM-bound: per position 104 B (784 B with history) in, 64 * channels * sizeof(T) out.
 #include "common.cuh"
+#include "planes.cuh"
 
 namespace az {
 namespace {
-
-struct alignas(8) PosCur {
-    unsigned long long pieces[12];
-    unsigned char stm, castling, ep_square, halfmove, repetitions, pad[3];
-};
-struct alignas(8) PosH8 {
-    PosCur cur;
-    unsigned long long hist_pieces[7][12];
-    unsigned char hist_rep[7];
-    unsigned char n_hist;
-};
-
-template <typename T> __device__ __forceinline__ T to_act(float v);
-template <> __device__ __forceinline__ float to_act<float>(float v) { return v; }
-template <> __device__ __forceinline__ __nv_bfloat16 to_act<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
-
-// value of one channel of the 19-plane layout at absolute square s
-__device__ __forceinline__ float plane19(const PosCur *r, int ch, int s, float hm) {
-    const int stm = r->stm;
-    if (ch < 12) {
-        const int own = ch < 6;
-        const int idx = ((stm != 0) == (own != 0) ? 6 : 0) + (ch % 6);   // own pieces of Black sit at 6..11
-        return (float)((r->pieces[idx] >> s) & 1ull);
-    }
-    const int c = r->castling;
-    switch (ch) {
-        case 12: return (float)stm;
-        case 13: return (float)((c >> (stm ? 2 : 0)) & 1);
-        case 14: return (float)((c >> (stm ? 3 : 1)) & 1);
-        case 15: return (float)((c >> (stm ? 0 : 2)) & 1);
-        case 16: return (float)((c >> (stm ? 1 : 3)) & 1);
-        case 17: return hm;
-        case 18: return r->repetitions >= 1 ? 1.0f : 0.0f;
-        default: return 0.0f;
-    }
-}
-
-__device__ __forceinline__ float plane112(const PosH8 *h, int ch, int s, float hm) {
-    const PosCur *r = &h->cur;
-    const int stm = r->stm;
-    if (ch < 104) {
-        const int t = ch / 13, k = ch % 13;
-        if (t > h->n_hist) return 0.0f;
-        if (k == 12) return (t == 0 ? r->repetitions : h->hist_rep[t - 1]) >= 1 ? 1.0f : 0.0f;
-        const int own = k < 6;
-        const int idx = ((stm != 0) == (own != 0) ? 6 : 0) + (k % 6);
-        const unsigned long long bb = t == 0 ? r->pieces[idx] : h->hist_pieces[t - 1][idx];
-        return (float)((bb >> s) & 1ull);
-    }
-    const int c = r->castling;
-    switch (ch) {
-        case 104: return (float)((c >> (stm ? 2 : 0)) & 1);
-        case 105: return (float)((c >> (stm ? 3 : 1)) & 1);
-        case 106: return (float)((c >> (stm ? 0 : 2)) & 1);
-        case 107: return (float)((c >> (stm ? 1 : 3)) & 1);
-        case 108: return (float)stm;
-        case 109: return hm;
-        case 111: return 1.0f;
-        default: return 0.0f;
-    }
-}
 
 template <typename T, int IN_PLANES, int PAD>
 __global__ void __launch_bounds__(256)

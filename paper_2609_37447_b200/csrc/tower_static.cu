@@ -49,5 +49,5 @@ extern "C" int az_tower_static(az_net *net, const void *positions_dev, int batch
     rc = az::launch_encode(positions_dev, az_position_bytes(&n->arch), batch, (int)n->arch.in_planes, n->in_pad,
                            true, planes, n->status_dev, s);
     if (rc != AZ_OK) return rc;
-    return az::launch_tower_tc(*n, planes, batch, tower_dev, false, nullptr, s);
+    return az::launch_tower_tc(*n, planes, nullptr, batch, tower_dev, false, nullptr, s);
 }

@@ -31,6 +31,7 @@
 // Every mbarrier wait is bounded; on expiry the CTA raises a status bit, stops issuing work,
 // drains, frees its TMEM and exits.
 #include "common.cuh"
+#include "planes.cuh"
 #include "ptx.cuh"
 
 #include <cuda_fp8.h>
@@ -77,8 +78,8 @@ struct Shape {
     static constexpr int kOffFrames = 0;
     static constexpr int kOffWeights = kGroups * kFrameBytes;
     static constexpr int kOffBars = kOffWeights + kStages * kStageBytes;
-    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done
-    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1;
+    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done, lead[S]
+    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1 + kStages;
     static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
     static constexpr int kOffAbort = kOffTmemPtr + 4;
     static constexpr int kOffConst = (kOffAbort + 4 + 15) & ~15;     // per-warp copies of the current layer's channel constants
@@ -88,7 +89,10 @@ struct Shape {
 };
 
 struct TowerArgs {
-    const __nv_bfloat16 *planes;     // [batch][64][in_pad]
+    const __nv_bfloat16 *planes;     // [batch][64][in_pad] already encoded planes, or null:
+    const unsigned char *positions;  // then the boards are encoded here from their position records
+    size_t position_stride;
+    int in_planes;                   // 19 or 112
     const void *weights;             // packed stages
     const float *bias;               // [n_conv][C]
     __nv_bfloat16 *out;              // [batch][64][C] or null
@@ -135,7 +139,8 @@ tower_tc_kernel(const TowerArgs args) {
     auto bar_w_empty = [&](int s) { return bars + 8u * (kStages + s); };
     auto bar_acc_full = [&](int g) { return bars + 8u * (2 * kStages + g); };
     auto bar_a_ready = [&](int g, int kc) { return bars + 8u * (2 * kStages + kGroups + g * kSlices + kc); };
-    const uint32_t bar_done = bars + 8u * (S::kNumBars - 1);
+    const uint32_t bar_done = bars + 8u * (2 * kStages + kGroups + kGroups * kSlices);
+    auto bar_lead = [&](int s) { return bar_done + 8u * (1 + s); };   // group 0 has issued its MMAs on stage s
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + S::kOffAbort);
     uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + S::kOffTmemPtr);
     constexpr int kConstFloats = (kFp8 ? 4 : 1) * kC;          // per layer: (scale, bias, 1/act scale, 1/h scale) or bias
@@ -146,7 +151,11 @@ tower_tc_kernel(const TowerArgs args) {
         reinterpret_cast<uint4 *>(smem + S::kOffFrames)[i] = make_uint4(0, 0, 0, 0);
     for (int i = threadIdx.x; i < args.head_n; i += kThreads) head_bias_smem[i] = args.head_bias[i];
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) { ptx::mbar_init(bar_w_full(s), 1); ptx::mbar_init(bar_w_empty(s), kGroups); }
+        for (int s = 0; s < kStages; ++s) {
+            ptx::mbar_init(bar_w_full(s), 1);
+            ptx::mbar_init(bar_w_empty(s), kGroups);
+            ptx::mbar_init(bar_lead(s), 1);
+        }
         for (int g = 0; g < kGroups; ++g) {
             ptx::mbar_init(bar_acc_full(g), 1);
             for (int kc = 0; kc < kSlices; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4);
@@ -221,17 +230,13 @@ tower_tc_kernel(const TowerArgs args) {
         bool ok = true;
         const uint32_t d_h = tmem_base + (uint32_t)(g * 2 * kC);
         const uint32_t frame_lo = (((smem_base + S::kOffFrames + g * kFrameBytes) >> 4) + (uint32_t)(kNB * 9 + 1)) | kADescLbo;
-        const int n_layers = n_conv + (head_n ? 1 : 0);
-        uint32_t lead_parity = 0;                                      // parity of group 0's next layer-0 completion
+        // The two issuers take strict turns on every weight stage: group 1 issues its MMAs on a stage
+        // only after group 0 has issued its own (bar_lead).  While one issuer sits in its barrier round
+        // trips the other's MMAs keep the tensor pipe busy, and the groups reach their layer boundaries
+        // one stage apart instead of together.
+        const bool follow = kGroups == 2 && g == 1 && !(args.trace & 2);
+        const bool lead = kGroups == 2 && g == 0;
         for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
-            if (kGroups == 2 && g == 1 && n_conv >= 3 && !(args.trace & 2)) {
-                // Start one (short) input layer behind group 0.  The groups then reach their layer
-                // boundaries at different times, so one group's wait for its epilogue is covered by
-                // the other's MMAs instead of idling the tensor pipe for both at once.
-                ok = wait_bar(bar_acc_full(0), lead_parity, abort_flag, args.status, tr ? &t_wait[2] : nullptr);
-                if (!ok) break;
-                lead_parity ^= (uint32_t)(n_layers & 1);
-            }
             for (int l = 0; l < n_conv && ok; ++l) {
                 const int nkc = l == 0 ? in_slices : (kFp8 ? kC / 32 : kC / 16);
                 const bool e4m3 = kFp8 && l > 0;                       // the input layer stays bf16
@@ -247,6 +252,10 @@ tower_tc_kernel(const TowerArgs args) {
                     for (int st = 0; st < S::kStagesPerSlice; ++st) {
                         ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                         if (!ok) break;
+                        if (follow) {
+                            ok = wait_bar(bar_lead(stage), phase, abort_flag, args.status, tr ? &t_wait[2] : nullptr);
+                            if (!ok) break;
+                        }
                         ptx::tc_fence_after();
                         const long long ti0 = tr ? clock64() : 0;
                         if (lane == 0) {
@@ -265,6 +274,7 @@ tower_tc_kernel(const TowerArgs args) {
                             }
                             if (kc == nkc - 1 && st == S::kStagesPerSlice - 1) ptx::mma_commit(bar_acc_full(g));
                             ptx::mma_commit(bar_w_empty(stage));
+                            if (lead) ptx::mbar_arrive(bar_lead(stage));
                         }
                         __syncwarp();
                         if (tr) t_issue += clock64() - ti0;
@@ -279,6 +289,10 @@ tower_tc_kernel(const TowerArgs args) {
                     if (kc % hsps == 0) {
                         ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                         if (!ok) break;
+                        if (follow) {
+                            ok = wait_bar(bar_lead(stage), phase, abort_flag, args.status, tr ? &t_wait[2] : nullptr);
+                            if (!ok) break;
+                        }
                     }
                     ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
                     if (!ok) break;
@@ -291,7 +305,10 @@ tower_tc_kernel(const TowerArgs args) {
                                               ((uint32_t)head_n << 16);          // K core matrices head_n*16 bytes apart
                         ptx::mma_bf16_split(d_h + (uint32_t)kC, a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u);
                         if (kc == kSlices - 1) ptx::mma_commit(bar_acc_full(g));
-                        if (stage_done) ptx::mma_commit(bar_w_empty(stage));
+                        if (stage_done) {
+                            ptx::mma_commit(bar_w_empty(stage));
+                            if (lead) ptx::mbar_arrive(bar_lead(stage));
+                        }
                     }
                     __syncwarp();
                     if (stage_done && ++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -320,12 +337,33 @@ tower_tc_kernel(const TowerArgs args) {
             const int board = unit * S::kBoardsPerCta + g * kNB + b;
             const bool live = board < args.batch;
             const int sq = y * 8 + x;
-            // ---- the unit's input planes -> the first in_pad/8 planes of the frame
+            // ---- the unit's input planes -> the first in_pad/8 planes of the frame, either copied from an
+            // encoded plane tensor or encoded on the spot from the position record (App. D.1 conventions)
             {
-                const uint4 *src = reinterpret_cast<const uint4 *>(args.planes + ((size_t)board * 64 + sq) * args.in_pad);
-                for (int j = 0; j < args.in_pad / 8; ++j) {
-                    const uint4 v = live ? __ldg(src + j) : make_uint4(0, 0, 0, 0);
-                    *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = v;
+                if (args.planes != nullptr) {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(args.planes + ((size_t)board * 64 + sq) * args.in_pad);
+                    for (int j = 0; j < args.in_pad / 8; ++j) {
+                        const uint4 v = live ? __ldg(src + j) : make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = v;
+                    }
+                } else {
+                    const PosCur *rec = reinterpret_cast<const PosCur *>(args.positions + (size_t)(live ? board : 0) * args.position_stride);
+                    const int s_abs = rec->stm ? (sq ^ 56) : sq;            // reflect ranks for Black
+                    const float hm = halfmove_plane(rec);
+                    if (live && sq == 0 && (__popcll(rec->pieces[5]) != 1 || __popcll(rec->pieces[11]) != 1))
+                        atomicOr(args.status, kStatusBadRecord);
+                    if (args.in_planes == 19 && args.in_pad == 32) {
+                        uint4 v[4];
+                        planes19_bf16(rec, sq, v);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = live ? v[j] : make_uint4(0, 0, 0, 0);
+                    } else {
+                        for (int j = 0; j < args.in_pad / 8; ++j) {
+                            const uint4 v = live ? planes_chunk8_bf16(rec, args.in_planes, j * 8, s_abs, hm) : make_uint4(0, 0, 0, 0);
+                            *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = v;
+                        }
+                    }
                 }
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
@@ -615,8 +653,8 @@ void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_p
                     }
 }
 
-int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_out, bool with_heads,
-                    unsigned int *absmax, cudaStream_t s) {
+int launch_tower_tc(const Net &net, const void *planes, const void *positions, int batch, void *tower_out,
+                    bool with_heads, unsigned int *absmax, cudaStream_t s) {
     if (batch == 0) return AZ_OK;
     static int sm_count[64] = {};
     int dev = 0;
@@ -634,6 +672,9 @@ int launch_tower_tc(const Net &net, const void *planes, int batch, void *tower_o
     const bool wide = net.arch.channels == 256;
     TowerArgs a;
     a.planes = static_cast<const __nv_bfloat16 *>(planes);
+    a.positions = static_cast<const unsigned char *>(positions);
+    a.position_stride = az_position_bytes(&net.arch);
+    a.in_planes = (int)net.arch.in_planes;
     a.weights = fp8 ? net.tc8_weights : net.tc_weights;
     a.bias = net.tc_bias;
     a.out = static_cast<__nv_bfloat16 *>(tower_out);

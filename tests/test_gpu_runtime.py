@@ -74,7 +74,7 @@ def test_tower_event_timing_counts_passes(setup):
     assert passes == 5 and 0.0 < ms < 50.0
     az.az_evaluate(net, pos, masks, 96, pol, val)
     assert az.az_tower_time(net) == (0.0, 0)
-    assert az.az_launches_per_evaluate(net, 96) == 4
+    assert az.az_launches_per_evaluate(net, 96) == 3
 
 
 def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable(setup):
