@@ -64,7 +64,6 @@ constexpr uint32_t kSpinLimit = 1u << 24;
 template <int C, int GROUPS>
 struct Shape {
     static constexpr int kC = C, kGroups = GROUPS;
-    static constexpr int kBoardsPerCta = kNB * kGroups;
     static constexpr int kSlices = kC / 16;                          // 16-channel slices of a layer's output
     static constexpr int kFrameBytes = kPlaneBytes * (kC / 8);       // 46336 / 92672 per group
     static constexpr int kTileBytes = kC * 32;                       // one tap: N = C rows x 32 bytes of K
@@ -114,6 +113,38 @@ struct TowerArgs {
     // calibration run (bf16 kernel): per-layer, per-channel maximum of the layer outputs, as float bits
     unsigned int *absmax;            // [n_conv][C]
 };
+
+// One round of a CTA's work: which two-board groups sit in its slots (-1 = the slot idles).
+struct Round {
+    int group[2];
+    bool valid;
+};
+
+// Static schedule, computed identically by every warp.  G groups on P CTAs.  Full rounds give every CTA two
+// groups.  What is left for the last round is spread one group per CTA if there are CTAs enough (a CTA alone
+// with one group needs about 0.8 of a two-group round, measured), else paired onto as few CTAs as possible
+// (measured faster than mixing one- and two-group CTAs: the round lasts as long either way and fewer busy
+// SMs run at higher clocks under the power cap).
+template <class S>
+__device__ __forceinline__ Round get_round(int r, int cta, int P, int G) {
+    Round rd;
+    rd.group[0] = rd.group[1] = -1; rd.valid = false;
+    if (S::kGroups == 1) {
+        const int g = r * P + cta;
+        if (g < G) { rd.group[0] = g; rd.valid = true; }
+        return rd;
+    }
+    const int full = G / (2 * P), left = G - full * 2 * P, base = full * 2 * P;
+    if (r < full) { rd.group[0] = r * 2 * P + 2 * cta; rd.group[1] = rd.group[0] + 1; rd.valid = true; return rd; }
+    if (r > full || left == 0) return rd;
+    if (left <= P) {
+        if (cta < left) { rd.group[0] = base + cta; rd.valid = true; }
+    } else if (2 * cta < left) {
+        rd.group[0] = base + 2 * cta; rd.valid = true;
+        if (2 * cta + 1 < left) rd.group[1] = base + 2 * cta + 1;
+    }
+    return rd;
+}
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
                                          long long *waited = nullptr) {
@@ -174,11 +205,13 @@ tower_tc_kernel(const TowerArgs args) {
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_smem;
 
-    const int n_units = (args.batch + S::kBoardsPerCta - 1) / S::kBoardsPerCta;
+    const int n_groups = (args.batch + kNB - 1) / kNB;
     const int n_conv = args.n_conv;
     const int head_n = args.head_n;
     const int in_slices = args.in_pad / 16;
     const int hsps = head_slices_per_stage<S>(head_n);
+    auto round_of = [&](int r) { return get_round<S>(r, (int)blockIdx.x, (int)gridDim.x, n_groups); };
+    auto slices_of = [&](int l) { return l == 0 ? in_slices : (kFp8 ? kC / 32 : kC / 16); };   // K per MMA: 16 bf16 or 32 e4m3
     const bool tr = args.trace && blockIdx.x == 0;
     long long t_wait[3] = {0, 0, 0};
     long long t_issue = 0;
@@ -191,26 +224,28 @@ tower_tc_kernel(const TowerArgs args) {
         uint32_t last_parity[kStages] = {};
         bool issued[kStages] = {};
         bool ok = true;
-        auto push = [&](const unsigned char *src, uint32_t bytes) {
-            ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
-            if (!ok) return;
-            if (lane == 0) {
-                ptx::mbar_arrive_expect_tx(bar_w_full(stage), bytes);
-                ptx::bulk_copy_g2s(smem_base + S::kOffWeights + stage * kStageBytes, src, bytes, bar_w_full(stage));
+        for (int r = 0; ok; ++r) {
+            const Round rd = round_of(r);
+            if (!rd.valid) break;
+            int n_stages = 0;
+            for (int l = 0; l < n_conv; ++l) n_stages += slices_of(l) * S::kStagesPerSlice;
+            const int n_head_stages = head_n ? kSlices / hsps : 0;
+            for (int st = 0; st < n_stages + n_head_stages && ok; ++st) {
+                // tower stages are contiguous and equally sized; the head projections follow as small stages of their own
+                const bool head = st >= n_stages;
+                const unsigned char *src = head ? reinterpret_cast<const unsigned char *>(args.head_w) + (size_t)(st - n_stages) * hsps * head_n * 32
+                                                : reinterpret_cast<const unsigned char *>(args.weights) + (size_t)st * kStageBytes;
+                const uint32_t bytes = head ? (uint32_t)(hsps * head_n * 32) : (uint32_t)kStageBytes;
+                ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+                if (!ok) break;
+                if (lane == 0) {
+                    ptx::mbar_arrive_expect_tx(bar_w_full(stage), bytes);
+                    ptx::bulk_copy_g2s(smem_base + S::kOffWeights + stage * kStageBytes, src, bytes, bar_w_full(stage));
+                }
+                issued[stage] = true; last_parity[stage] = phase;
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                __syncwarp();
             }
-            issued[stage] = true; last_parity[stage] = phase;
-            if (++stage == kStages) { stage = 0; phase ^= 1u; }
-            __syncwarp();
-        };
-        for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
-            const unsigned char *src = reinterpret_cast<const unsigned char *>(args.weights);
-            for (int l = 0; l < n_conv && ok; ++l) {
-                const int nkc = l == 0 ? in_slices : (kFp8 ? kC / 32 : kC / 16);     // K per MMA: 16 bf16 or 32 e4m3
-                for (int st = 0; st < nkc * S::kStagesPerSlice && ok; ++st) { push(src, kStageBytes); src += kStageBytes; }
-            }
-            if (head_n)                                        // the head projections: small stages of their own
-                for (int st = 0; st < kSlices / hsps && ok; ++st)
-                    push(reinterpret_cast<const unsigned char *>(args.head_w) + (size_t)st * hsps * head_n * 32, (uint32_t)(hsps * head_n * 32));
         }
         if (!ok) {
             // copies already in flight must land before the CTA's shared memory is released
@@ -236,9 +271,26 @@ tower_tc_kernel(const TowerArgs args) {
         // one stage apart instead of together.
         const bool follow = kGroups == 2 && g == 1 && !(args.trace & 2);
         const bool lead = kGroups == 2 && g == 0;
-        for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+        for (int r = 0; ok; ++r) {
+            const Round rd = round_of(r);
+            if (!rd.valid) break;
+            if ((g == 0 ? rd.group[0] : rd.group[1]) < 0) {
+                // a slot without a group this round still takes part in the ring protocol: it waits for
+                // every stage of the round and releases it without issuing anything
+                int n_stages = head_n ? kSlices / hsps : 0;
+                for (int l = 0; l < n_conv; ++l) n_stages += slices_of(l) * S::kStagesPerSlice;
+                for (int st = 0; st < n_stages && ok; ++st) {
+                    ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status);
+                    if (ok && follow) ok = wait_bar(bar_lead(stage), phase, abort_flag, args.status);
+                    if (!ok) break;
+                    if (lane == 0) { ptx::mbar_arrive(bar_w_empty(stage)); if (lead) ptx::mbar_arrive(bar_lead(stage)); }
+                    __syncwarp();
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                continue;
+            }
             for (int l = 0; l < n_conv && ok; ++l) {
-                const int nkc = l == 0 ? in_slices : (kFp8 ? kC / 32 : kC / 16);
+                const int nkc = slices_of(l);
                 const bool e4m3 = kFp8 && l > 0;                       // the input layer stays bf16
                 const bool conv2 = l >= 2 && (l & 1) == 0;             // accumulates onto the residual stream
                 const uint32_t d = d_h + (((l & 1) == 1) ? (uint32_t)kC : 0u);   // conv1 writes the ACC columns
@@ -333,11 +385,14 @@ tower_tc_kernel(const TowerArgs args) {
         float *lc = reinterpret_cast<float *>(smem + S::kOffConst) + ew * kConstFloats;   // this warp's copy of the layer constants
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
-            const int board = unit * S::kBoardsPerCta + g * kNB + b;
+        for (int r = 0; ok; ++r) {
+            const Round rd = round_of(r);
+            if (!rd.valid) break;
+            if ((g == 0 ? rd.group[0] : rd.group[1]) < 0) continue;                     // this slot sits the round out
+            const int board = (g == 0 ? rd.group[0] : rd.group[1]) * kNB + b;
             const bool live = board < args.batch;
             const int sq = y * 8 + x;
-            // ---- the unit's input planes -> the first in_pad/8 planes of the frame, either copied from an
+            // ---- the group's input planes -> the first in_pad/8 planes of the frame, either copied from an
             // encoded plane tensor or encoded on the spot from the position record (App. D.1 conventions)
             {
                 if (args.planes != nullptr) {
@@ -438,6 +493,7 @@ tower_tc_kernel(const TowerArgs args) {
                         reinterpret_cast<uint4 *>(dst + kc * 16)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         reinterpret_cast<uint4 *>(dst + kc * 16)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                     }
+
                     if (!last) {
                         if (next_e4m3) {
                             // 16 channels -> 16 e4m3 bytes (saturating, round to nearest even) = one slot of plane kc
@@ -692,9 +748,9 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     a.absmax = absmax;
     static const bool trace = getenv("AZ_TOWER_TRACE") != nullptr;
     a.trace = trace ? atoi(getenv("AZ_TOWER_TRACE")) : 0;
-    const int boards_per_cta = wide ? Shape256::kBoardsPerCta : Shape128::kBoardsPerCta;
-    const int n_units = (batch + boards_per_cta - 1) / boards_per_cta;
-    const int grid = n_units < sms ? n_units : sms;
+    // one CTA per SM, or one per two-board group when there are fewer groups than SMs
+    const int n_groups = (batch + kNB - 1) / kNB;
+    const int grid = n_groups < sms ? n_groups : sms;
     if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
     else if (fp8) tower_tc_kernel<true, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(true), s>>>(a);
     else tower_tc_kernel<false, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(false), s>>>(a);
