@@ -36,18 +36,12 @@ WORKLOADS = {
 DTYPE = {0: "f32", 1: "bf16", 2: "fp8_e4m3"}
 
 # DRAM bytes (read + write) of one tower-kernel launch, from the ncu capture summarised in
-# profiles/tower_tc_kernel_c3_batch592.md: 14.38 MB at batch 592, of which 11.87 MB are the weights
-# (read once whatever the batch) and the rest 4 KB of encoded planes per position.
+# profiles/tower_tc_kernel_c3_batch592.md: 12.06 MB at batch 592, of which 11.87 MB are the weights
+# (read once whatever the batch) and the rest the 104-byte position records.
 def tower_traffic_bytes(cfg, batch):
     if cfg.channels != 128 or cfg.blocks != 20 or cfg.precision != 1:
         return None             # no capture yet for other shapes / the FP8 tower
-    return 14.38e6 + (batch - 592) * 4096.0
-
-
-def tower_flops_per_position(cfg) -> float:
-    """Dense convolution count 2*64*9*Cin*Cout per layer; channel padding is not counted."""
-    c = cfg.channels
-    return 2.0 * 64 * 9 * (cfg.in_planes * c + 2 * cfg.blocks * c * c)
+    return 12.06e6 + (batch - 592) * 104.0
 
 
 def load_peaks():
