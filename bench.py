@@ -44,6 +44,12 @@ def tower_traffic_bytes(cfg, batch):
     return 12.06e6 + (batch - 592) * 104.0
 
 
+def tower_flops_per_position(cfg) -> float:
+    """Dense convolution count 2*64*9*Cin*Cout per layer; channel padding is not counted."""
+    c = cfg.channels
+    return 2.0 * 64 * 9 * (cfg.in_planes * c + 2 * cfg.blocks * c * c)
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -250,10 +256,24 @@ def main():
     barrier()
     h2d = pos_host.numel() + masks_host.numel() * 8
     d2h = (policy_host.numel() + value_host.numel()) * 4
+    # the same with the policy returned over the legal moves only (1 KB per position instead of 7.4 KB)
+    legal_host = torch.zeros((B, az.AZ_MAX_LEGAL), dtype=torch.float32).pin_memory()
+    counts_host = torch.zeros((B,), dtype=torch.int32).pin_memory()
+    for _ in range(3):
+        az.az_evaluate_legal_host(net, pos_host, masks_host, B, legal_host, counts_host, value_host)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        az.az_evaluate_legal_host(net, pos_host, masks_host, B, legal_host, counts_host, value_host)
+    torch.cuda.synchronize()
+    e2e_legal_s = time.perf_counter() - t0
+    barrier()
+    d2h_legal = (legal_host.numel() + counts_host.numel() + value_host.numel()) * 4
     checksum = float(policy_host.sum())            # every row sums to one
 
     # ---- max over ranks
-    total_ms, b2b_ms, e2e_ms, tower_ms_max = sharding.max_over_ranks([total_ms, b2b_ms, e2e_s * 1e3, tower_ms], device="cuda")
+    total_ms, b2b_ms, e2e_ms, tower_ms_max, e2e_legal_ms = sharding.max_over_ranks(
+        [total_ms, b2b_ms, e2e_s * 1e3, tower_ms, e2e_legal_s * 1e3], device="cuda")
 
     if rank == 0:
         peaks = load_peaks()
@@ -277,6 +297,9 @@ def main():
                              "note": "no L2 flush between steps"},
             "e2e": {"value": evals / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "ms_per_step": e2e_ms / args.steps, "api": "az_evaluate_host, pinned host buffers"},
+            "e2e_legal_moves_only": {"value": evals / (e2e_legal_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                                     "d2h_bytes_per_step": int(d2h_legal), "ms_per_step": e2e_legal_ms / args.steps,
+                                     "api": "az_evaluate_legal_host, pinned host buffers"},
             "gpu_launches": args.steps * az.az_launches_per_evaluate(net, B),
             "clocks": clocks,
             "roofline": {"kernel": "tower_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peak_tf,

@@ -23,7 +23,7 @@ AZ_VALUE_TANH, AZ_VALUE_WDL = 0, 1
 AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3 = 0, 1, 2
 
 EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
-           "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_host", "az_encode", "az_tower", "az_tower_static", "az_legal_masks",
+           "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_encode", "az_tower", "az_tower_static", "az_legal_masks",
            "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error")
 
@@ -56,6 +56,10 @@ def _load_library():
     lib.az_free_net.argtypes = [vp]
     lib.az_evaluate.restype = ci
     lib.az_evaluate.argtypes = [vp, vp, vp, ci, vp, vp, vp]
+    lib.az_evaluate_legal.restype = ci
+    lib.az_evaluate_legal.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp]
+    lib.az_evaluate_legal_host.restype = ci
+    lib.az_evaluate_legal_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp]
     lib.az_evaluate_host.restype = ci
     lib.az_evaluate_host.argtypes = [vp, vp, vp, ci, vp, vp, vp]
     lib.az_profile_tower.restype = ci
@@ -177,6 +181,22 @@ def az_evaluate_host(net: Net, positions_host, legal_masks_host, batch, policy_h
     _check(_lib.az_evaluate_host(net.handle, _host_ptr(positions_host, "positions"), _host_ptr(legal_masks_host, "legal_masks"),
                                  batch, _host_ptr(policy_host, "policy"), _host_ptr(value_host, "value"),
                                  _stream_ptr(stream)), "az_evaluate_host")
+
+
+AZ_MAX_LEGAL = 256
+
+
+def az_evaluate_legal(net: Net, positions_dev, legal_masks_dev, batch, legal_policy_dev, legal_counts_dev, value_dev, stream=None):
+    """az_evaluate with the policy over the legal moves only: [batch][AZ_MAX_LEGAL] float32 + [batch] int32 counts."""
+    _check(_lib.az_evaluate_legal(net.handle, _dev_ptr(positions_dev, "positions"), _dev_ptr(legal_masks_dev, "legal_masks"),
+                                  batch, _dev_ptr(legal_policy_dev, "legal_policy"), _dev_ptr(legal_counts_dev, "legal_counts"),
+                                  _dev_ptr(value_dev, "value"), _stream_ptr(stream)), "az_evaluate_legal")
+
+
+def az_evaluate_legal_host(net: Net, positions_host, legal_masks_host, batch, legal_policy_host, legal_counts_host, value_host, stream=None):
+    _check(_lib.az_evaluate_legal_host(net.handle, _host_ptr(positions_host, "positions"), _host_ptr(legal_masks_host, "legal_masks"),
+                                       batch, _host_ptr(legal_policy_host, "legal_policy"), _host_ptr(legal_counts_host, "legal_counts"),
+                                       _host_ptr(value_host, "value"), _stream_ptr(stream)), "az_evaluate_legal_host")
 
 
 def az_profile_tower(net: Net, enable: bool):

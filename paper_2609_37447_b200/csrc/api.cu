@@ -253,6 +253,7 @@ void free_net(Net *n) {
     cudaFree(n->planes);
     for (int i = 0; i < 3; ++i) cudaFree(n->act[i]);
     cudaFree(n->stage_pos); cudaFree(n->stage_masks); cudaFree(n->stage_policy); cudaFree(n->stage_value);
+    cudaFree(n->stage_compact); cudaFree(n->stage_counts);
     if (n->ev_begin) for (int i = 0; i < kMaxProfiledPasses; ++i) { cudaEventDestroy(n->ev_begin[i]); cudaEventDestroy(n->ev_end[i]); }
     delete[] n->ev_begin; delete[] n->ev_end;
     cudaFree(n->logits); cudaFree(n->head_p); cudaFree(n->head_v); cudaFree(n->hidden); cudaFree(n->status_dev);
@@ -353,14 +354,17 @@ int az_tower(az_net *net, const void *positions_dev, int batch, void *tower_dev,
     return AZ_OK;
 }
 
-int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_masks_dev, int batch,
-                float *policy_dev, float *value_dev, void *cuda_stream) {
+// policy_dev (dense rows) or legal_dev + counts_dev (legal moves only): exactly one form is requested
+static int evaluate_impl(az_net *net, const void *positions_dev, const uint64_t *legal_masks_dev, int batch,
+                         float *policy_dev, float *legal_dev, int32_t *counts_dev, float *value_dev, void *cuda_stream) {
     Net *n = reinterpret_cast<Net *>(net);
     if (!n || batch < 0) return AZ_ERR_BAD_ARG;
     if (batch == 0) return AZ_OK;
-    if (!positions_dev || !legal_masks_dev || !policy_dev || !value_dev) return AZ_ERR_BAD_ARG;
+    const bool dense = policy_dev != nullptr;
+    if (!positions_dev || !legal_masks_dev || !value_dev || (!dense && (!legal_dev || !counts_dev))) return AZ_ERR_BAD_ARG;
     if ((reinterpret_cast<uintptr_t>(positions_dev) & 7) || (reinterpret_cast<uintptr_t>(legal_masks_dev) & 7) ||
-        (reinterpret_cast<uintptr_t>(policy_dev) & 3) || (reinterpret_cast<uintptr_t>(value_dev) & 3))
+        (reinterpret_cast<uintptr_t>(dense ? (void *)policy_dev : (void *)legal_dev) & 3) ||
+        (reinterpret_cast<uintptr_t>(counts_dev) & 3) || (reinterpret_cast<uintptr_t>(value_dev) & 3))
         return AZ_ERR_BAD_ARG;
     if ((uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
     if (n->fp8 && !n->fp8_ready) return AZ_ERR_NOT_CALIBRATED;
@@ -375,6 +379,9 @@ int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_ma
         // projection; one GEMM launch finishes both heads, the softmax follows
         rc = az::launch_fc_tc(*n, batch, value_dev, s);
         if (rc != AZ_OK) return rc;
+        if (!dense)
+            return az::launch_masked_softmax_compact(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a),
+                                                     (int)az_mask_words(&a), legal_dev, counts_dev, n->status_dev, s);
         return az::launch_masked_softmax(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a), (int)az_mask_words(&a),
                                          policy_dev, n->status_dev, s);
     }
@@ -393,8 +400,54 @@ int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_ma
     if (rc != AZ_OK) return rc;
     rc = az::launch_value_tail(n->hidden, n->v_w2, n->v_b2, batch, a.value_head == AZ_VALUE_WDL, value_dev, s);
     if (rc != AZ_OK) return rc;
+    if (!dense)
+        return az::launch_masked_softmax_compact(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a),
+                                                 (int)az_mask_words(&a), legal_dev, counts_dev, n->status_dev, s);
     return az::launch_masked_softmax(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a), (int)az_mask_words(&a),
                                      policy_dev, n->status_dev, s);
+}
+
+int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_masks_dev, int batch,
+                float *policy_dev, float *value_dev, void *cuda_stream) {
+    if (!policy_dev && batch > 0) return AZ_ERR_BAD_ARG;
+    return evaluate_impl(net, positions_dev, legal_masks_dev, batch, policy_dev, nullptr, nullptr, value_dev, cuda_stream);
+}
+
+int az_evaluate_legal(az_net *net, const void *positions_dev, const uint64_t *legal_masks_dev, int batch,
+                      float *legal_policy_dev, int32_t *legal_counts_dev, float *value_dev, void *cuda_stream) {
+    if ((!legal_policy_dev || !legal_counts_dev) && batch > 0) return AZ_ERR_BAD_ARG;
+    return evaluate_impl(net, positions_dev, legal_masks_dev, batch, nullptr, legal_policy_dev, legal_counts_dev, value_dev, cuda_stream);
+}
+
+int az_evaluate_legal_host(az_net *net, const void *positions_host, const uint64_t *legal_masks_host, int batch,
+                           float *legal_policy_host, int32_t *legal_counts_host, float *value_host, void *cuda_stream) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n || batch < 0) return AZ_ERR_BAD_ARG;
+    if (batch == 0) return AZ_OK;
+    if (!positions_host || !legal_masks_host || !legal_policy_host || !legal_counts_host || !value_host) return AZ_ERR_BAD_ARG;
+    if ((uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const az_arch &a = n->arch;
+    const size_t B = a.max_batch, pb = az_position_bytes(&a), mw = az_mask_words(&a), vs = az_value_size(&a);
+    if (!n->stage_pos) {
+        AZ_CUDA(cudaMalloc(&n->stage_pos, B * pb));
+        AZ_CUDA(cudaMalloc((void **)&n->stage_masks, B * mw * sizeof(uint64_t)));
+        AZ_CUDA(cudaMalloc((void **)&n->stage_policy, B * az_policy_size(&a) * sizeof(float)));
+        AZ_CUDA(cudaMalloc((void **)&n->stage_value, B * vs * sizeof(float)));
+    }
+    if (!n->stage_compact) {
+        AZ_CUDA(cudaMalloc((void **)&n->stage_compact, B * AZ_MAX_LEGAL * sizeof(float)));
+        AZ_CUDA(cudaMalloc((void **)&n->stage_counts, B * sizeof(int)));
+    }
+    AZ_CUDA(cudaMemcpyAsync(n->stage_pos, positions_host, (size_t)batch * pb, cudaMemcpyHostToDevice, s));
+    AZ_CUDA(cudaMemcpyAsync(n->stage_masks, legal_masks_host, (size_t)batch * mw * sizeof(uint64_t), cudaMemcpyHostToDevice, s));
+    int rc = az_evaluate_legal(net, n->stage_pos, n->stage_masks, batch, n->stage_compact, n->stage_counts, n->stage_value, cuda_stream);
+    if (rc != AZ_OK) return rc;
+    AZ_CUDA(cudaMemcpyAsync(legal_policy_host, n->stage_compact, (size_t)batch * AZ_MAX_LEGAL * sizeof(float), cudaMemcpyDeviceToHost, s));
+    AZ_CUDA(cudaMemcpyAsync(legal_counts_host, n->stage_counts, (size_t)batch * sizeof(int), cudaMemcpyDeviceToHost, s));
+    AZ_CUDA(cudaMemcpyAsync(value_host, n->stage_value, (size_t)batch * vs * sizeof(float), cudaMemcpyDeviceToHost, s));
+    AZ_CUDA(cudaStreamSynchronize(s));
+    return AZ_OK;
 }
 
 int az_evaluate_host(az_net *net, const void *positions_host, const uint64_t *legal_masks_host, int batch,

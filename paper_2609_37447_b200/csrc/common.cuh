@@ -15,6 +15,7 @@ constexpr int kHeadChannels = 32;     // width of the 1x1 projections of the fla
 constexpr int kValueHidden = 128;
 constexpr int kFlatMoves = 1858;
 constexpr int kPlanes73 = 73;
+constexpr int kMaxLegal = AZ_MAX_LEGAL;       // row stride of the legal-moves-only policy output
 
 // Device-side status bits (OR-ed into az_net::status_dev by kernels).
 enum : uint32_t {
@@ -81,6 +82,8 @@ struct Net {
     void *stage_pos = nullptr;
     uint64_t *stage_masks = nullptr;
     float *stage_policy = nullptr, *stage_value = nullptr;
+    float *stage_compact = nullptr;   // [max_batch][AZ_MAX_LEGAL]
+    int *stage_counts = nullptr;
 
     // ---- optional event timing of the tower ----
     bool profile = false;
@@ -116,6 +119,8 @@ int launch_fc(const void *a, const void *w, const float *bias, int m, int n, int
               bool bf16_in, void *out, bool out_f32, cudaStream_t s);
 int launch_value_tail(const float *hidden, const float *w2, const float *b2, int batch, int wdl,
                       float *value, cudaStream_t s);
+int launch_masked_softmax_compact(const float *logits, const uint64_t *masks, int batch, int n, int words,
+                                  float *out, int *counts, uint32_t *status, cudaStream_t s);
 int launch_masked_softmax(const float *logits, const uint64_t *masks, int batch, int n, int words,
                           float *policy, uint32_t *status, cudaStream_t s);
 

@@ -181,7 +181,87 @@ masked_softmax_kernel(const float *__restrict__ logits, const unsigned long long
     if (!any && tid == 0) atomicOr(status, kStatusEmptyMask);
 }
 
+// ---- masked softmax, legal moves only: one warp per position -------------------------------------
+// out[pos][j] = probability of the j-th legal move in ascending policy-index order (the order in which
+// a consumer walks the mask's set bits), j < counts[pos] <= kMaxLegal; entries beyond are not written.
+__global__ void __launch_bounds__(128)
+masked_softmax_compact_kernel(const float *__restrict__ logits, const unsigned long long *__restrict__ masks,
+                              int batch, int n, int words, float *__restrict__ out, int *__restrict__ counts,
+                              uint32_t *__restrict__ status) {
+    __shared__ float vals[4][kMaxLegal];
+    const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pos = blockIdx.x * 4 + wid;
+    if (pos >= batch) return;
+    const float *row = logits + (size_t)pos * n;
+    float *v = vals[wid];
+    // lane w owns mask words w, w+32, w+64; ranks of its bits come from a warp prefix sum of popcounts
+    unsigned long long mw[3];
+    int cnt = 0;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const int w = lane + 32 * k;
+        mw[k] = w < words ? masks[(size_t)pos * words + w] : 0ull;
+        // bits beyond the last policy index are ignored
+        if (w < words && (w + 1) * 64 > n) mw[k] &= (n - w * 64 >= 64) ? ~0ull : ((1ull << (n - w * 64)) - 1ull);
+    }
+    int base[3];
+    int total = 0;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        cnt = __popcll(mw[k]);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        base[k] = total + incl - cnt;
+        total += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    const int n_legal = total < kMaxLegal ? total : kMaxLegal;
+    float mx = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        unsigned long long bits = mw[k];
+        int j = base[k];
+        while (bits) {
+            const int bit = __ffsll((long long)bits) - 1;
+            bits &= bits - 1;
+            if (j < kMaxLegal) {
+                const float l = row[(lane + 32 * k) * 64 + bit];
+                v[j] = l;
+                mx = fmaxf(mx, l);
+            }
+            ++j;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    __syncwarp();
+    float sum = 0.0f;
+    for (int j = lane; j < n_legal; j += 32) { const float e = expf(v[j] - mx); v[j] = e; sum += e; }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float inv = n_legal > 0 ? 1.0f / sum : 0.0f;
+    float *dst = out + (size_t)pos * kMaxLegal;
+    for (int j = lane; j < n_legal; j += 32) dst[j] = v[j] * inv;
+    if (lane == 0) {
+        counts[pos] = n_legal;
+        if (n_legal == 0) atomicOr(status, kStatusEmptyMask);
+    }
+}
+
 }  // namespace
+
+int launch_masked_softmax_compact(const float *logits, const uint64_t *masks, int batch, int n, int words,
+                                  float *out, int *counts, uint32_t *status, cudaStream_t s) {
+    if (batch == 0) return AZ_OK;
+    if (words > 96) return AZ_ERR_BAD_ARCH;
+    masked_softmax_compact_kernel<<<(batch + 3) / 4, 128, 0, s>>>(
+        logits, reinterpret_cast<const unsigned long long *>(masks), batch, n, words, out, counts, status);
+    AZ_LAUNCH_CHECK();
+    return AZ_OK;
+}
 
 int launch_conv1x1(const void *in, const void *w, const float *scale, const float *bias, int batch,
                    int cin, int cout, bool relu, bool bf16_in, void *out, bool out_f32, cudaStream_t s) {

@@ -42,6 +42,33 @@ def test_host_buffer_entry_point_gives_the_same_results(setup):
     assert (pol_n == policy.cpu().numpy()).all() and (val_n == value.cpu().numpy()).all()
 
 
+def test_legal_moves_only_output_matches_the_dense_policy(setup):
+    az, net, recs, pos, masks, policy, value = setup
+    legal = torch.full((96, az.AZ_MAX_LEGAL), -1.0, device="cuda")
+    counts = torch.full((96,), -1, dtype=torch.int32, device="cuda")
+    val = torch.zeros_like(value)
+    az.az_evaluate_legal(net, pos, masks, 96, legal, counts, val)
+    torch.cuda.synchronize()
+    dense = policy.cpu().numpy()
+    bits = np.unpackbits(az.masks_to_numpy(masks).view(np.uint8), axis=1, bitorder="little")[:, :1858].astype(bool)
+    lg, cn = legal.cpu().numpy(), counts.cpu().numpy()
+    assert torch.equal(val, value)
+    for b in range(96):
+        idx = np.flatnonzero(bits[b])                      # ascending policy index = order of the mask's set bits
+        assert cn[b] == idx.size
+        assert np.abs(lg[b, :idx.size] - dense[b, idx]).max() < 1e-6
+        assert (lg[b, idx.size:] == -1.0).all()              # entries beyond the count are left alone
+    # host-buffer form
+    pos_h = torch.from_numpy(np.ascontiguousarray(recs).view(np.uint8).reshape(96, -1).copy()).pin_memory()
+    lg_h = torch.zeros((96, az.AZ_MAX_LEGAL)).pin_memory()
+    cn_h = torch.zeros((96,), dtype=torch.int32).pin_memory()
+    val_h = torch.zeros((96, 3)).pin_memory()
+    az.az_evaluate_legal_host(net, pos_h, masks.cpu().pin_memory(), 96, lg_h, cn_h, val_h)
+    assert torch.equal(cn_h, counts.cpu()) and torch.equal(val_h, value.cpu())
+    for b in range(96):
+        assert torch.equal(lg_h[b, :cn[b]], legal[b, :cn[b]].cpu())
+
+
 def test_evaluation_replays_from_a_cuda_graph(setup):
     az, net, recs, pos, masks, policy, value = setup
     pol_g = torch.zeros_like(policy)
