@@ -289,6 +289,37 @@ def test_results_are_deterministic_and_independent_of_batch_composition(az):
     az.az_free_net(net)
 
 
+@pytest.mark.parametrize("channels,in_planes", [(128, 19), (256, 112), (128, 112)])
+def test_work_schedule_is_invisible_in_the_results(az, channels, in_planes):
+    # The tower deals two-board groups out to CTAs in rounds and treats the last round specially
+    # (one group per CTA, or pairs on few CTAs).  Whatever the batch size, a position's outputs must
+    # not depend on where the schedule put it: every prefix of one big evaluation must reproduce.
+    cfg = configs.tiny_config(in_planes=in_planes, blocks=1, channels=channels, policy_head=0, value_head=1,
+                              precision=1, batch=1200, weight_seed=99)
+    blob = weights.make_blob(cfg, 0.05, 0.1)
+    net, _ = load(az, cfg, max_batch=1200, blob=blob)
+    rec, _ = positions.generate(321, 1200, (0, 60))
+    recs = positions.records_for_planes(in_planes, rec)
+    masks = oracle.legal_masks(positions.cur_records(rec), 0)
+    _, p_all, v_all = gpu_evaluate(az, net, cfg, recs, masks_np=masks)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    per_round = sms * (4 if channels == 128 else 2)           # positions one full round of all CTAs takes
+    sizes = sorted({1, 2, 3, 5, 2 * sms - 1, 2 * sms, 2 * sms + 1, per_round - 3, per_round, per_round + 2,
+                    per_round + 2 * sms, per_round + 2 * sms + 2, per_round + 3 * sms + 1, 2 * per_round - 2, 1199})
+    for n in sizes:
+        if n > 1200:
+            continue
+        _, p, v = gpu_evaluate(az, net, cfg, recs[:n], masks_np=masks[:n])
+        assert np.array_equal(p, p_all[:n]) and np.array_equal(v, v_all[:n]), n
+    # oracle spot check on rows that sit at the seams of the schedule
+    rows = np.array([0, 1, 2 * sms - 1, 2 * sms, per_round - 1, per_round, min(per_round + 2 * sms, 1199), 1199])
+    rows = rows[rows < 1200]
+    _, _, po, vo = oracle.evaluate(blob, recs[rows], in_planes, 0)
+    assert np.abs(p_all[rows] - po).max() <= TOL[1] and np.abs(v_all[rows] - vo).max() <= TOL[1]
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
 def test_empty_mask_row_gives_zero_policy_and_a_status_flag(az):
     cfg = configs.tiny_config(blocks=1, channels=32, batch=4)
     net, blob = load(az, cfg, max_batch=8)
