@@ -381,9 +381,9 @@ static int evaluate_impl(az_net *net, const void *positions_dev, const uint64_t 
         if (rc != AZ_OK) return rc;
         if (!dense)
             return az::launch_masked_softmax_compact(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a),
-                                                     (int)az_mask_words(&a), legal_dev, counts_dev, n->status_dev, s);
+                                                     (int)az_mask_words(&a), legal_dev, counts_dev, n->status_dev, true, s);
         return az::launch_masked_softmax(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a), (int)az_mask_words(&a),
-                                         policy_dev, n->status_dev, s);
+                                         policy_dev, n->status_dev, true, s);
     }
     if (a.policy_head == AZ_POLICY_PLANES73) {
         rc = az::launch_conv1x1(h, n->p_w, nullptr, n->p_bias, batch, C, az::kPlanes73, false, n->bf16, n->logits, true, s);
@@ -402,9 +402,9 @@ static int evaluate_impl(az_net *net, const void *positions_dev, const uint64_t 
     if (rc != AZ_OK) return rc;
     if (!dense)
         return az::launch_masked_softmax_compact(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a),
-                                                 (int)az_mask_words(&a), legal_dev, counts_dev, n->status_dev, s);
+                                                 (int)az_mask_words(&a), legal_dev, counts_dev, n->status_dev, false, s);
     return az::launch_masked_softmax(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a), (int)az_mask_words(&a),
-                                     policy_dev, n->status_dev, s);
+                                     policy_dev, n->status_dev, false, s);
 }
 
 int az_evaluate(az_net *net, const void *positions_dev, const uint64_t *legal_masks_dev, int batch,

@@ -105,6 +105,19 @@ void set_cuda_error(cudaError_t e, const char *what);
         if (e__ != cudaSuccess) { az::set_cuda_error(e__, "kernel launch"); return AZ_ERR_CUDA; } \
     } while (0)
 
+// Launch `kernel` so that it may begin (prologue only) before the previous kernel in the stream has
+// finished; the kernel itself must call ptx::grid_dependency_wait() before reading that kernel's output.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- kernels' launch functions (each returns AZ_OK or AZ_ERR_CUDA) ---------------------------
 int launch_encode(const void *positions, size_t stride, int batch, int in_planes, int in_pad,
                   bool bf16, void *planes, uint32_t *status, cudaStream_t s);
@@ -119,10 +132,11 @@ int launch_fc(const void *a, const void *w, const float *bias, int m, int n, int
               bool bf16_in, void *out, bool out_f32, cudaStream_t s);
 int launch_value_tail(const float *hidden, const float *w2, const float *b2, int batch, int wdl,
                       float *value, cudaStream_t s);
+// pdl: the logits come from the kernel launched just before on the same stream, and this launch may overlap its tail
 int launch_masked_softmax_compact(const float *logits, const uint64_t *masks, int batch, int n, int words,
-                                  float *out, int *counts, uint32_t *status, cudaStream_t s);
+                                  float *out, int *counts, uint32_t *status, bool pdl, cudaStream_t s);
 int launch_masked_softmax(const float *logits, const uint64_t *masks, int batch, int n, int words,
-                          float *policy, uint32_t *status, cudaStream_t s);
+                          float *policy, uint32_t *status, bool pdl, cudaStream_t s);
 
 // tensor-core tower (tower_tc.cu)
 size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv);

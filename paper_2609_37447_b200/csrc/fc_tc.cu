@@ -85,6 +85,10 @@ fc_tc_kernel(const FcArgs args) {
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_smem;
+    // everything above overlaps the tower kernel's tail; its output (U tiles, for 73-plane heads the logits)
+    // is read only below
+    ptx::grid_dependency_wait();
+    ptx::launch_dependents();
 
     if (warp == 0) {
         // ---- producer: two 16 KB bulk copies per stage
@@ -243,8 +247,7 @@ int launch_fc_tc(const Net &net, int batch, float *value_out, cudaStream_t s) {
     a.n_policy_tiles = flat ? (kFlatMoves + 127) / 128 : 0;
     a.wdl = net.arch.value_head == AZ_VALUE_WDL;
     dim3 grid((unsigned)(a.n_policy_tiles + 1), (unsigned)((batch + 127) / 128));
-    fc_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(a);
-    AZ_LAUNCH_CHECK();
+    AZ_CUDA(launch_dependent(fc_tc_kernel, grid, dim3(kThreads), kSmemBytes, s, a));
     return AZ_OK;
 }
 

@@ -133,16 +133,21 @@ value_tail_kernel(const float *__restrict__ hidden, const float *__restrict__ w2
     }
 }
 
+__device__ __forceinline__ void grid_dependency_wait_if(int pdl) {
+    if (pdl) asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- masked softmax: one CTA (128 threads) per position ----------------------------------------
 template <int ITEMS>       // elements per thread: ceil(n / 128)
 __global__ void __launch_bounds__(128)
 masked_softmax_kernel(const float *__restrict__ logits, const unsigned long long *__restrict__ masks,
-                      int n, int words, float *__restrict__ policy, uint32_t *__restrict__ status) {
+                      int n, int words, float *__restrict__ policy, uint32_t *__restrict__ status, int pdl) {
     __shared__ float red[4];
     __shared__ unsigned long long mw[80];
     const int pos = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     if (tid < words) mw[tid] = masks[(size_t)pos * words + tid];
     __syncthreads();
+    grid_dependency_wait_if(pdl);                   // the logits come from the previous kernel in the stream
     const float *row = logits + (size_t)pos * n;
     float v[ITEMS];
     float mx = -INFINITY;
@@ -187,10 +192,11 @@ masked_softmax_kernel(const float *__restrict__ logits, const unsigned long long
 __global__ void __launch_bounds__(128)
 masked_softmax_compact_kernel(const float *__restrict__ logits, const unsigned long long *__restrict__ masks,
                               int batch, int n, int words, float *__restrict__ out, int *__restrict__ counts,
-                              uint32_t *__restrict__ status) {
+                              uint32_t *__restrict__ status, int pdl) {
     __shared__ float vals[4][kMaxLegal];
     const int wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int pos = blockIdx.x * 4 + wid;
+    grid_dependency_wait_if(pdl);                   // the logits come from the previous kernel in the stream
     if (pos >= batch) return;
     const float *row = logits + (size_t)pos * n;
     float *v = vals[wid];
@@ -254,12 +260,17 @@ masked_softmax_compact_kernel(const float *__restrict__ logits, const unsigned l
 }  // namespace
 
 int launch_masked_softmax_compact(const float *logits, const uint64_t *masks, int batch, int n, int words,
-                                  float *out, int *counts, uint32_t *status, cudaStream_t s) {
+                                  float *out, int *counts, uint32_t *status, bool pdl, cudaStream_t s) {
     if (batch == 0) return AZ_OK;
     if (words > 96) return AZ_ERR_BAD_ARCH;
-    masked_softmax_compact_kernel<<<(batch + 3) / 4, 128, 0, s>>>(
-        logits, reinterpret_cast<const unsigned long long *>(masks), batch, n, words, out, counts, status);
-    AZ_LAUNCH_CHECK();
+    if (pdl)
+        AZ_CUDA(launch_dependent(masked_softmax_compact_kernel, dim3((batch + 3) / 4), dim3(128), 0, s, logits,
+                                 reinterpret_cast<const unsigned long long *>(masks), batch, n, words, out, counts, status, 1));
+    else {
+        masked_softmax_compact_kernel<<<(batch + 3) / 4, 128, 0, s>>>(
+            logits, reinterpret_cast<const unsigned long long *>(masks), batch, n, words, out, counts, status, 0);
+        AZ_LAUNCH_CHECK();
+    }
     return AZ_OK;
 }
 
@@ -296,12 +307,17 @@ int launch_value_tail(const float *hidden, const float *w2, const float *b2, int
 }
 
 int launch_masked_softmax(const float *logits, const uint64_t *masks, int batch, int n, int words,
-                          float *policy, uint32_t *status, cudaStream_t s) {
+                          float *policy, uint32_t *status, bool pdl, cudaStream_t s) {
     if (batch == 0) return AZ_OK;
     const unsigned long long *m = reinterpret_cast<const unsigned long long *>(masks);
-    if (n <= 128 * 15) masked_softmax_kernel<15><<<batch, 128, 0, s>>>(logits, m, n, words, policy, status);
-    else if (n <= 128 * 37) masked_softmax_kernel<37><<<batch, 128, 0, s>>>(logits, m, n, words, policy, status);
-    else return AZ_ERR_BAD_ARCH;
+    if (n > 128 * 37) return AZ_ERR_BAD_ARCH;
+    if (pdl) {
+        if (n <= 128 * 15) AZ_CUDA(launch_dependent(masked_softmax_kernel<15>, dim3(batch), dim3(128), 0, s, logits, m, n, words, policy, status, 1));
+        else AZ_CUDA(launch_dependent(masked_softmax_kernel<37>, dim3(batch), dim3(128), 0, s, logits, m, n, words, policy, status, 1));
+        return AZ_OK;
+    }
+    if (n <= 128 * 15) masked_softmax_kernel<15><<<batch, 128, 0, s>>>(logits, m, n, words, policy, status, 0);
+    else masked_softmax_kernel<37><<<batch, 128, 0, s>>>(logits, m, n, words, policy, status, 0);
     AZ_LAUNCH_CHECK();
     return AZ_OK;
 }

@@ -138,6 +138,14 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-stream-serialization
+// attribute may start while its predecessor in the stream is still running; it must call
+// grid_dependency_wait() before touching anything the predecessor writes (the call returns once the
+// predecessor has completed and its writes are visible).  launch_dependents() lets the successor's
+// CTAs be scheduled from this point on, wherever SMs are free.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 }  // namespace ptx
 
 // Bounded mbarrier wait, called by all 32 lanes of a warp together.  Polls at most `limit` times.

@@ -204,6 +204,7 @@ tower_tc_kernel(const TowerArgs args) {
     __syncthreads();
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_smem;
+    ptx::launch_dependents();        // the head GEMM kernel may set itself up on idle SMs; it waits for this grid before reading
 
     const int n_groups = (args.batch + kNB - 1) / kNB;
     const int n_conv = args.n_conv;
