@@ -61,9 +61,11 @@ constexpr uint32_t kSpinLimit = 1u << 24;
 // Shape-dependent constants.  128 channels: two groups per CTA share every weight stage (16 input
 // channels x 9 taps).  256 channels: the frame and the accumulators of ONE group fill shared memory
 // and TMEM, and a stage is 16 input channels x 3 taps.
-template <int C, int GROUPS>
+// SETS: how many sets of four epilogue warps share a group's layer (each set takes a contiguous run of
+// the 16-channel slices).  Two sets for the FP8 tower, whose MMAs are twice as fast as its epilogue needs.
+template <int C, int GROUPS, int SETS>
 struct Shape {
-    static constexpr int kC = C, kGroups = GROUPS;
+    static constexpr int kC = C, kGroups = GROUPS, kSets = SETS;
     static constexpr int kSlices = kC / 16;                          // 16-channel slices of a layer's output
     static constexpr int kFrameBytes = kPlaneBytes * (kC / 8);       // 46336 / 92672 per group
     static constexpr int kTileBytes = kC * 32;                       // one tap: N = C rows x 32 bytes of K
@@ -71,8 +73,8 @@ struct Shape {
     static constexpr int kStagesPerSlice = 9 / kStageTaps;
     static constexpr int kStageBytes = kStageTaps * kTileBytes;      // 36864 / 24576
     static constexpr int kStages = kC == 128 ? 3 : 5;
-    static constexpr int kEpiWarps = 4 * kGroups;
-    static constexpr int kThreads = 32 * (1 + kGroups + kEpiWarps);  // producer, one issuer per group, 4 epilogue warps per group
+    static constexpr int kEpiWarps = 4 * kGroups * kSets;
+    static constexpr int kThreads = 32 * (1 + kGroups + kEpiWarps);  // producer, one issuer per group, 4 epilogue warps per group and set
     static constexpr uint32_t kBDescLbo = (uint32_t)kC << 16;        // K core matrices C*16 bytes apart
     static constexpr int kOffFrames = 0;
     static constexpr int kOffWeights = kGroups * kFrameBytes;
@@ -82,8 +84,9 @@ struct Shape {
     static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
     static constexpr int kOffAbort = kOffTmemPtr + 4;
     static constexpr int kOffConst = (kOffAbort + 4 + 15) & ~15;     // per-warp copies of the current layer's channel constants
-    static constexpr int smem_bytes(bool fp8) { return kOffConst + kEpiWarps * (fp8 ? 4 : 1) * kC * 4 + 128 * 4; }
-    static_assert(kOffConst + kEpiWarps * 4 * kC * 4 + 512 <= kMaxSmem || kC == 256, "shared memory budget");
+    // per epilogue warp: the current layer's channel constants for the channels of its own slices
+    static constexpr int smem_bytes(bool fp8) { return kOffConst + kEpiWarps * (fp8 ? 4 : 1) * (kC / kSets) * 4 + 128 * 4; }
+    static_assert(kOffConst + kEpiWarps * 4 * (kC / kSets) * 4 + 512 <= kMaxSmem || kC == 256, "shared memory budget");
     static_assert(kGroups * 2 * kC == (int)kTmemCols, "TMEM: per group C columns of residual stream and C of accumulator");
 };
 
@@ -175,7 +178,9 @@ tower_tc_kernel(const TowerArgs args) {
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + S::kOffAbort);
     uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + S::kOffTmemPtr);
     constexpr int kConstFloats = (kFp8 ? 4 : 1) * kC;          // per layer: (scale, bias, 1/act scale, 1/h scale) or bias
-    float *head_bias_smem = reinterpret_cast<float *>(smem + S::kOffConst) + S::kEpiWarps * kConstFloats;
+    constexpr int kMyC = kC / S::kSets;                         // channels an epilogue warp is responsible for
+    constexpr int kMyConstFloats = (kFp8 ? 4 : 1) * kMyC;
+    float *head_bias_smem = reinterpret_cast<float *>(smem + S::kOffConst) + S::kEpiWarps * kMyConstFloats;
 
     // ---- set-up: zero the frames (their borders stay zero for the kernel's lifetime), barriers, TMEM
     for (int i = threadIdx.x; i < kGroups * kFrameBytes / 16; i += kThreads)
@@ -189,7 +194,7 @@ tower_tc_kernel(const TowerArgs args) {
         }
         for (int g = 0; g < kGroups; ++g) {
             ptx::mbar_init(bar_acc_full(g), 1);
-            for (int kc = 0; kc < kSlices; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4);
+            for (int kc = 0; kc < kSlices; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4 * S::kSets);
         }
         ptx::mbar_init(bar_done, kGroups);
         *abort_flag = 0;
@@ -313,17 +318,26 @@ tower_tc_kernel(const TowerArgs args) {
                         const long long ti0 = tr ? clock64() : 0;
                         if (lane == 0) {
                             const uint32_t b_lo = ((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) | S::kBDescLbo;
+                            // the operand type is chosen once per stage: a branch between consecutive MMAs
+                            // costs more than the MMA itself takes on the tensor pipe
+                            if (e4m3) {
 #pragma unroll
-                            for (int t = 0; t < S::kStageTaps; ++t) {
-                                const int tap = st * S::kStageTaps + t;
-                                const int dy = tap / 3 - 1, dx = tap % 3 - 1;
-                                const uint32_t acc = (tap == 0 && !conv2 && kc == 0) ? 0u : 1u;
-                                if (e4m3)
+                                for (int t = 0; t < S::kStageTaps; ++t) {
+                                    const int tap = st * S::kStageTaps + t;
+                                    const int dy = tap / 3 - 1, dx = tap % 3 - 1;
                                     ptx::mma_e4m3_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                        b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8, acc);
-                                else
+                                                        b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8,
+                                                        (tap == 0 && !conv2 && kc == 0) ? 0u : 1u);
+                                }
+                            } else {
+#pragma unroll
+                                for (int t = 0; t < S::kStageTaps; ++t) {
+                                    const int tap = st * S::kStageTaps + t;
+                                    const int dy = tap / 3 - 1, dx = tap % 3 - 1;
                                     ptx::mma_bf16_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                        b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc, acc);
+                                                        b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc,
+                                                        (tap == 0 && !conv2 && kc == 0) ? 0u : 1u);
+                                }
                             }
                             if (kc == nkc - 1 && st == S::kStagesPerSlice - 1) ptx::mma_commit(bar_acc_full(g));
                             ptx::mma_commit(bar_w_empty(stage));
@@ -374,16 +388,23 @@ tower_tc_kernel(const TowerArgs args) {
         for (uint32_t i = 0; i < (1u << 22); ++i)
             if (ptx::mbar_try_wait(bar_done, 0)) break;
     } else {
-        // ================= epilogue: 4 warps per group =================
-        const int ew = warp - 1 - kGroups;                    // 0 .. 4*groups-1
-        const int g = ew >> 2;
+        // ================= epilogue: 4 warps per group and set =================
+        // A set's last hand-off of a layer comes after its TMEM loads and stores of that layer have
+        // completed, and every later writer of those columns (an MMA two layers on) is gated, through the
+        // accumulator barrier of the layer between, by the hand-offs of ALL sets.
+        const int ew = warp - 1 - kGroups;                    // 0 .. 4*groups*sets-1
+        const int g = ew / (4 * S::kSets);
+        // this warp's share of every layer: the slices kc = ks * sets + set.  Interleaved, so that with two
+        // sets the two slices of the next layer's first 32-channel e4m3 step are produced side by side.
+        const int set = (ew >> 2) % S::kSets;
+        constexpr int kMySlices = kSlices / S::kSets;
         const int q = warp & 3;                               // TMEM lane quarter this warp may access
         const int m = q * 32 + lane;                          // GEMM row = TMEM lane
         const int g8 = m >> 3, y = g8 >> 1, b = g8 & 1, x = m & 7;
         const int slot = (g8 + kNB) * 9 + x + 1;
         unsigned char *frame = smem + S::kOffFrames + g * kFrameBytes;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 2 * kC);
-        float *lc = reinterpret_cast<float *>(smem + S::kOffConst) + ew * kConstFloats;   // this warp's copy of the layer constants
+        float *lc = reinterpret_cast<float *>(smem + S::kOffConst) + ew * kMyConstFloats;   // this warp's copy of the layer constants
         uint32_t acc_phase = 0;
         bool ok = true;
         for (int r = 0; ok; ++r) {
@@ -398,7 +419,7 @@ tower_tc_kernel(const TowerArgs args) {
             {
                 if (args.planes != nullptr) {
                     const uint4 *src = reinterpret_cast<const uint4 *>(args.planes + ((size_t)board * 64 + sq) * args.in_pad);
-                    for (int j = 0; j < args.in_pad / 8; ++j) {
+                    for (int j = set; j < args.in_pad / 8; j += S::kSets) {
                         const uint4 v = live ? __ldg(src + j) : make_uint4(0, 0, 0, 0);
                         *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = v;
                     }
@@ -413,9 +434,10 @@ tower_tc_kernel(const TowerArgs args) {
                         planes19_bf16(rec, sq, v);
 #pragma unroll
                         for (int j = 0; j < 4; ++j)
-                            *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = live ? v[j] : make_uint4(0, 0, 0, 0);
+                            if (S::kSets == 1 || (j % S::kSets) == set)
+                                *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = live ? v[j] : make_uint4(0, 0, 0, 0);
                     } else {
-                        for (int j = 0; j < args.in_pad / 8; ++j) {
+                        for (int j = set; j < args.in_pad / 8; j += S::kSets) {
                             const uint4 v = live ? planes_chunk8_bf16(rec, args.in_planes, j * 8, s_abs, hm) : make_uint4(0, 0, 0, 0);
                             *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = v;
                         }
@@ -438,31 +460,36 @@ tower_tc_kernel(const TowerArgs args) {
                     const float *src = kFp8 ? args.lconst + (size_t)l * kConstFloats : args.bias + (size_t)l * kC;
                     __syncwarp();
 #pragma unroll
-                    for (int i = 0; i < kConstFloats / 4 / 32; ++i)
-                        reinterpret_cast<float4 *>(lc)[i * 32 + lane] = __ldg(reinterpret_cast<const float4 *>(src) + i * 32 + lane);
+                    for (int i = 0; i < kMyConstFloats / 4 / 32; ++i) {
+                        // own copy: [vector][own slice ks][16 channels]
+                        const int idx = i * 32 + lane, vec = idx / (kMyC / 4), within = idx % (kMyC / 4);
+                        const int kc = (within >> 2) * S::kSets + set;
+                        reinterpret_cast<float4 *>(lc)[idx] = __ldg(reinterpret_cast<const float4 *>(src) + vec * (kC / 4) + kc * 4 + (within & 3));
+                    }
                     __syncwarp();
                 }
                 ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 acc_phase ^= 1u;
                 ptx::tc_fence_after();
-                const float *bias = kFp8 ? lc + kC : lc;
+                const float *bias = kFp8 ? lc + kMyC : lc;
                 __nv_bfloat16 *dst = args.out + ((size_t)board * 64 + sq) * kC;
                 const uint32_t t_src = t_lane + (uint32_t)(from_acc ? kC : 0);
                 const bool keep_h = !from_acc && l != n_conv - 1;   // the residual stream stays in TMEM as fp32
                 uint32_t r[2][16];
-                ptx::tmem_ld16(t_src, r[0]);
+                ptx::tmem_ld16(t_src + (uint32_t)(set * 16), r[0]);
 #pragma unroll
-                for (int kc = 0; kc < kSlices; ++kc) {
+                for (int ks = 0; ks < kMySlices; ++ks) {
+                    const int kc = ks * S::kSets + set;             // the slice; ks indexes this warp's constants
                     ptx::tmem_ld_wait();
-                    if (kc + 1 < kSlices) ptx::tmem_ld16(t_src + (uint32_t)((kc + 1) * 16), r[(kc + 1) & 1]);
-                    uint32_t(&rr)[16] = r[kc & 1];
+                    if (ks + 1 < kMySlices) ptx::tmem_ld16(t_src + (uint32_t)((kc + S::kSets) * 16), r[(ks + 1) & 1]);
+                    uint32_t(&rr)[16] = r[ks & 1];
                     float v[16];
 #pragma unroll
                     for (int i = 0; i < 16; i += 4) {
-                        const float4 bv = *reinterpret_cast<const float4 *>(bias + kc * 16 + i);
+                        const float4 bv = *reinterpret_cast<const float4 *>(bias + ks * 16 + i);
                         if (kFp8) {
-                            const float4 os = *reinterpret_cast<const float4 *>(lc + kc * 16 + i);
+                            const float4 os = *reinterpret_cast<const float4 *>(lc + ks * 16 + i);
                             v[i + 0] = fmaxf(fmaf(__uint_as_float(rr[i + 0]), os.x, bv.x), 0.0f);
                             v[i + 1] = fmaxf(fmaf(__uint_as_float(rr[i + 1]), os.y, bv.y), 0.0f);
                             v[i + 2] = fmaxf(fmaf(__uint_as_float(rr[i + 2]), os.z, bv.z), 0.0f);
@@ -501,7 +528,7 @@ tower_tc_kernel(const TowerArgs args) {
                             uint32_t pk[4];
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
-                                const float4 qs = *reinterpret_cast<const float4 *>(lc + 2 * kC + kc * 16 + 4 * i);
+                                const float4 qs = *reinterpret_cast<const float4 *>(lc + 2 * kMyC + ks * 16 + 4 * i);
                                 const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(v[4 * i] * qs.x, v[4 * i + 1] * qs.y), __NV_SATFINITE, __NV_E4M3);
                                 const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(v[4 * i + 2] * qs.z, v[4 * i + 3] * qs.w), __NV_SATFINITE, __NV_E4M3);
                                 pk[i] = lo | (hi << 16);
@@ -524,26 +551,40 @@ tower_tc_kernel(const TowerArgs args) {
                             // whose MMAs are gated by barriers these same threads arrive on only after that wait.
                             uint32_t w[16];
 #pragma unroll
-                            for (int i = 0; i < 16; ++i)
-                                w[i] = __float_as_uint(kFp8 ? v[i] * lc[3 * kC + kc * 16 + i] : v[i]);
+                            for (int i = 0; i < 16; i += 4) {
+                                float4 hs = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
+                                if (kFp8) hs = *reinterpret_cast<const float4 *>(lc + 3 * kMyC + ks * 16 + i);
+                                w[i + 0] = __float_as_uint(kFp8 ? v[i + 0] * hs.x : v[i + 0]);
+                                w[i + 1] = __float_as_uint(kFp8 ? v[i + 1] * hs.y : v[i + 1]);
+                                w[i + 2] = __float_as_uint(kFp8 ? v[i + 2] * hs.z : v[i + 2]);
+                                w[i + 3] = __float_as_uint(kFp8 ? v[i + 3] * hs.w : v[i + 3]);
+                            }
                             ptx::tmem_st16(t_lane + (uint32_t)(kc * 16), w);
+                            if (S::kSets > 1 && ks == kMySlices - 1) ptx::tmem_st_wait();
                         }
-                        // e4m3 layers consume 32 channels per MMA: one hand-off per two slices
-                        if (!next_e4m3 || (kc & 1)) {
+                        // e4m3 layers consume 32 channels per MMA: one hand-off per two slices.  With two sets
+                        // every barrier counts both sets' warps: a pair of slices is handed off by the four
+                        // warps of each set, and where the next layer reads 16-channel slices (the bf16 head)
+                        // each set also signs for its neighbour's slice once its own is written.
+                        if (S::kSets == 2 || !next_e4m3 || (kc & 1)) {
                             ptx::fence_proxy_async_smem();
                             ptx::tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) ptx::mbar_arrive(bar_a_ready(g, next_e4m3 ? (kc >> 1) : kc));
+                            if (lane == 0) {
+                                ptx::mbar_arrive(bar_a_ready(g, next_e4m3 ? (kc >> 1) : kc));
+                                if (S::kSets == 2 && !next_e4m3) ptx::mbar_arrive(bar_a_ready(g, kc ^ 1));
+                            }
                         }
                     }
                 }
-                if (keep_h) ptx::tmem_st_wait();
+                if (S::kSets == 1 && keep_h) ptx::tmem_st_wait();
             }
             if (head_n && ok) {
                 // ---- head projections out of the ACC columns
                 ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 acc_phase ^= 1u;
+                if (set != 0) continue;                               // the head's rows are few: set 0 writes them all
                 ptx::tc_fence_after();
                 const float *hb = head_bias_smem;
                 // this row's place in the GEMM A tiles: [tile of 128 boards][8-wide K chunk][board/8][board%8][8 k]
@@ -597,8 +638,12 @@ tower_tc_kernel(const TowerArgs args) {
     }
 }
 
-typedef Shape<128, 2> Shape128;
-typedef Shape<256, 1> Shape256;
+typedef Shape<128, 2, 1> Shape128;
+#ifndef AZ_FP8_EPI_SETS
+#define AZ_FP8_EPI_SETS 2
+#endif
+typedef Shape<128, 2, AZ_FP8_EPI_SETS> Shape128F8;
+typedef Shape<256, 1, 1> Shape256;
 constexpr int kStageBytes = Shape128::kStageBytes;       // host-side packing of the 128-channel stages
 
 }  // namespace
@@ -720,7 +765,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         int n = 0;
         AZ_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
-        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
@@ -753,7 +798,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     const int n_groups = (batch + kNB - 1) / kNB;
     const int grid = n_groups < sms ? n_groups : sms;
     if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
-    else if (fp8) tower_tc_kernel<true, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(true), s>>>(a);
+    else if (fp8) tower_tc_kernel<true, Shape128F8><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else tower_tc_kernel<false, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(false), s>>>(a);
     AZ_LAUNCH_CHECK();
     return AZ_OK;
