@@ -99,6 +99,35 @@ __device__ __forceinline__ void mma_bf16_split(uint32_t d_tmem, uint32_t a_lo, u
         "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n"
         "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate));
 }
+// The form the tower's issuer warps use: the whole warp executes the call, converged, and only the
+// lane whose `elected` is non-zero issues the MMA.  With no divergent region around it and every
+// descriptor input warp-uniform, the descriptor arithmetic runs on the uniform datapath and an MMA
+// costs the warp's scheduler one or two issue slots; as `if (lane == 0) mma(...)` the same loop fell
+// from 64 to 103 / 163 / 249 cycles per MMA with one / two / three arithmetic-busy warps on the
+// issuer's scheduler (measured on B200), i.e. the epilogue warps starved the tensor pipe.
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n"
+        ".reg .pred P;\n"
+        "elect.sync _|P, 0xffffffff;\n"
+        "selp.b32 %0, 1, 0, P;\n"
+        "}\n" : "=r"(pred));
+    return pred;
+}
+__device__ __forceinline__ void mma_bf16_elect(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                               uint32_t idesc, uint32_t accumulate, uint32_t elected) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 p, %6, 0;\n"
+        "setp.ne.b32 q, %7, 0;\n"
+        "mov.b64 da, {%1, %2};\n"
+        "mov.b64 db, {%3, %4};\n"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elected));
+}
 // Instruction descriptor, kind::f8f6f4: D fp32, A and B e4m3 (format code 0), both K-major, dense; K = 32 per MMA.
 __host__ __device__ constexpr uint32_t idesc_e4m3_f32(int m, int n) {
     return (1u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
@@ -114,6 +143,19 @@ __device__ __forceinline__ void mma_e4m3_split(uint32_t d_tmem, uint32_t a_lo, u
         "mov.b64 db, {%3, %4};\n"
         "tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %5, p;\n"
         "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate));
+}
+__device__ __forceinline__ void mma_e4m3_elect(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                               uint32_t idesc, uint32_t accumulate, uint32_t elected) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 p, %6, 0;\n"
+        "setp.ne.b32 q, %7, 0;\n"
+        "mov.b64 da, {%1, %2};\n"
+        "mov.b64 db, {%3, %4};\n"
+        "@q tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %5, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elected));
 }
 // mbarrier arrives once all MMAs issued so far by this thread have completed
 __device__ __forceinline__ void mma_commit(uint32_t bar) {

@@ -166,7 +166,9 @@ tower_tc_kernel(const TowerArgs args) {
     constexpr int kFrameBytes = S::kFrameBytes, kStageBytes = S::kStageBytes, kThreads = S::kThreads;
     static_assert(!kFp8 || kC == 128, "the FP8 tower exists for 128 channels");
     extern __shared__ __align__(128) unsigned char smem[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the warp index through a shuffle: the compiler then knows it is the same in all lanes, and role-
+    // dependent address arithmetic can stay on the uniform datapath
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const uint32_t smem_base = ptx::smem_addr(smem);
     const uint32_t bars = smem_base + S::kOffBars;
     auto bar_w_full = [&](int s) { return bars + 8u * s; };
@@ -277,6 +279,7 @@ tower_tc_kernel(const TowerArgs args) {
         // one stage apart instead of together.
         const bool follow = kGroups == 2 && g == 1 && !(args.trace & 2);
         const bool lead = kGroups == 2 && g == 0;
+        const uint32_t elected = ptx::elect_one();              // the lane that issues; the warp stays converged
         for (int r = 0; ok; ++r) {
             const Round rd = round_of(r);
             if (!rd.valid) break;
@@ -316,7 +319,7 @@ tower_tc_kernel(const TowerArgs args) {
                         }
                         ptx::tc_fence_after();
                         const long long ti0 = tr ? clock64() : 0;
-                        if (lane == 0) {
+                        {
                             const uint32_t b_lo = ((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) | S::kBDescLbo;
                             // the operand type is chosen once per stage: a branch between consecutive MMAs
                             // costs more than the MMA itself takes on the tensor pipe
@@ -325,23 +328,25 @@ tower_tc_kernel(const TowerArgs args) {
                                 for (int t = 0; t < S::kStageTaps; ++t) {
                                     const int tap = st * S::kStageTaps + t;
                                     const int dy = tap / 3 - 1, dx = tap % 3 - 1;
-                                    ptx::mma_e4m3_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                    ptx::mma_e4m3_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
                                                         b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8,
-                                                        (tap == 0 && !conv2 && kc == 0) ? 0u : 1u);
+                                                        (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
                                 }
                             } else {
 #pragma unroll
                                 for (int t = 0; t < S::kStageTaps; ++t) {
                                     const int tap = st * S::kStageTaps + t;
                                     const int dy = tap / 3 - 1, dx = tap % 3 - 1;
-                                    ptx::mma_bf16_split(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                    ptx::mma_bf16_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
                                                         b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc,
-                                                        (tap == 0 && !conv2 && kc == 0) ? 0u : 1u);
+                                                        (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
                                 }
                             }
-                            if (kc == nkc - 1 && st == S::kStagesPerSlice - 1) ptx::mma_commit(bar_acc_full(g));
-                            ptx::mma_commit(bar_w_empty(stage));
-                            if (lead) ptx::mbar_arrive(bar_lead(stage));
+                            if (elected) {
+                                if (kc == nkc - 1 && st == S::kStagesPerSlice - 1) ptx::mma_commit(bar_acc_full(g));
+                                ptx::mma_commit(bar_w_empty(stage));
+                                if (lead) ptx::mbar_arrive(bar_lead(stage));
+                            }
                         }
                         __syncwarp();
                         if (tr) t_issue += clock64() - ti0;
@@ -366,11 +371,13 @@ tower_tc_kernel(const TowerArgs args) {
                     a_phase ^= 1u << kc;
                     ptx::tc_fence_after();
                     const bool stage_done = (kc % hsps) == hsps - 1;
-                    if (lane == 0) {
+                    {
                         const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
                         const uint32_t b_lo = (((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) + (uint32_t)((kc % hsps) * head_n * 2)) |
                                               ((uint32_t)head_n << 16);          // K core matrices head_n*16 bytes apart
-                        ptx::mma_bf16_split(d_h + (uint32_t)kC, a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u);
+                        ptx::mma_bf16_elect(d_h + (uint32_t)kC, a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u, elected);
+                    }
+                    if (elected) {
                         if (kc == kSlices - 1) ptx::mma_commit(bar_acc_full(g));
                         if (stage_done) {
                             ptx::mma_commit(bar_w_empty(stage));
@@ -383,7 +390,7 @@ tower_tc_kernel(const TowerArgs args) {
             }
         }
         // all issued MMAs must have completed before TMEM is freed
-        if (lane == 0) ptx::mma_commit(bar_done);
+        if (elected) ptx::mma_commit(bar_done);
         __syncwarp();
         for (uint32_t i = 0; i < (1u << 22); ++i)
             if (ptx::mbar_try_wait(bar_done, 0)) break;
