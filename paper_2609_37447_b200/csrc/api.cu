@@ -547,7 +547,7 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
     for (int l = 0; l < L; ++l) { w.push_back(hm->w[l].data()); sc.push_back(hm->scale[l].data()); bi.push_back(hm->bias[l].data()); }
     const size_t bytes = az::tc8_packed_weight_bytes(n->in_pad, C, L);
     std::vector<unsigned char> packed(bytes);
-    std::vector<float> lconst((size_t)L * 4 * C);
+    std::vector<float> lconst((size_t)L * 3 * C);
     az::tc8_pack(w.data(), sc.data(), bi.data(), absmax.data(), (int)n->arch.in_planes, n->in_pad, C, L, packed.data(), lconst.data());
     if (!n->tc8_weights) AZ_CUDA(cudaMalloc(&n->tc8_weights, bytes));
     if (!n->tc8_lconst) AZ_CUDA(cudaMalloc((void **)&n->tc8_lconst, lconst.size() * sizeof(float)));

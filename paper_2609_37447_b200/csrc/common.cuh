@@ -48,7 +48,7 @@ struct Net {
     // FP8-e4m3 tower (weights and per-layer constants exist once az_calibrate has run)
     bool fp8 = false, fp8_ready = false;
     void *tc8_weights = nullptr;
-    float *tc8_lconst = nullptr;      // [n_conv][4][C]
+    float *tc8_lconst = nullptr;      // [n_conv][3][C]
     void *host_master = nullptr;      // fp32 tower weights kept on the host until calibration (FP8 nets)
     void *tc_head_w = nullptr;        // packed 1x1 head projections (policy | value), fused into the tower kernel
     float *tc_head_bias = nullptr;

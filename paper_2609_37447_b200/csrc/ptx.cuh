@@ -161,6 +161,18 @@ __device__ __forceinline__ void mma_e4m3_elect(uint32_t d_tmem, uint32_t a_lo, u
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// Two fp32 -> packed bf16x2 / e4m3x2 with the ReLU done by the conversion (negative inputs give +0);
+// `lo` lands in the low half.  Round to nearest even; e4m3 saturates to +-448.
+__device__ __forceinline__ uint32_t pack_bf16x2_relu(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.relu.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__device__ __forceinline__ uint32_t pack_e4m3x2_relu(float lo, float hi) {
+    unsigned short d;
+    asm("cvt.rn.satfinite.relu.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+    return (uint32_t)d;
+}
 // 16 consecutive fp32 columns of this thread's TMEM lane (warp-wide, lanes 32*(warp%4)..+31)
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile(

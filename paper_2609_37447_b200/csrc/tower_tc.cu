@@ -85,8 +85,8 @@ struct Shape {
     static constexpr int kOffAbort = kOffTmemPtr + 4;
     static constexpr int kOffConst = (kOffAbort + 4 + 15) & ~15;     // per-warp copies of the current layer's channel constants
     // per epilogue warp: the current layer's channel constants for the channels of its own slices
-    static constexpr int smem_bytes(bool fp8) { return kOffConst + kEpiWarps * (fp8 ? 4 : 1) * (kC / kSets) * 4 + 128 * 4; }
-    static_assert(kOffConst + kEpiWarps * 4 * (kC / kSets) * 4 + 512 <= kMaxSmem || kC == 256, "shared memory budget");
+    static constexpr int smem_bytes(bool fp8) { return kOffConst + kEpiWarps * (fp8 ? 3 : 1) * (kC / kSets) * 4 + 128 * 4; }
+    static_assert(kOffConst + kEpiWarps * 3 * (kC / kSets) * 4 + 512 <= kMaxSmem || kC == 256, "shared memory budget");
     static_assert(kGroups * 2 * kC == (int)kTmemCols, "TMEM: per group C columns of residual stream and C of accumulator");
 };
 
@@ -179,9 +179,9 @@ tower_tc_kernel(const TowerArgs args) {
     auto bar_lead = [&](int s) { return bar_done + 8u * (1 + s); };   // group 0 has issued its MMAs on stage s
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + S::kOffAbort);
     uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + S::kOffTmemPtr);
-    constexpr int kConstFloats = (kFp8 ? 4 : 1) * kC;          // per layer: (scale, bias, 1/act scale, 1/h scale) or bias
+    constexpr int kConstFloats = (kFp8 ? 3 : 1) * kC;          // per layer: (scale, bias, h ratio) or bias
     constexpr int kMyC = kC / S::kSets;                         // channels an epilogue warp is responsible for
-    constexpr int kMyConstFloats = (kFp8 ? 4 : 1) * kMyC;
+    constexpr int kMyConstFloats = (kFp8 ? 3 : 1) * kMyC;
     float *head_bias_smem = reinterpret_cast<float *>(smem + S::kOffConst) + S::kEpiWarps * kMyConstFloats;
 
     // ---- set-up: zero the frames (their borders stay zero for the kernel's lifetime), barriers, TMEM
@@ -467,9 +467,9 @@ tower_tc_kernel(const TowerArgs args) {
                     const float *src = kFp8 ? args.lconst + (size_t)l * kConstFloats : args.bias + (size_t)l * kC;
                     __syncwarp();
 #pragma unroll
-                    for (int i = 0; i < kMyConstFloats / 4 / 32; ++i) {
+                    for (int idx = lane; idx < kMyConstFloats / 4; idx += 32) {
                         // own copy: [vector][own slice ks][16 channels]
-                        const int idx = i * 32 + lane, vec = idx / (kMyC / 4), within = idx % (kMyC / 4);
+                        const int vec = idx / (kMyC / 4), within = idx % (kMyC / 4);
                         const int kc = (within >> 2) * S::kSets + set;
                         reinterpret_cast<float4 *>(lc)[idx] = __ldg(reinterpret_cast<const float4 *>(src) + vec * (kC / 4) + kc * 4 + (within & 3));
                     }
@@ -497,16 +497,22 @@ tower_tc_kernel(const TowerArgs args) {
                         const float4 bv = *reinterpret_cast<const float4 *>(bias + ks * 16 + i);
                         if (kFp8) {
                             const float4 os = *reinterpret_cast<const float4 *>(lc + ks * 16 + i);
-                            v[i + 0] = fmaxf(fmaf(__uint_as_float(rr[i + 0]), os.x, bv.x), 0.0f);
-                            v[i + 1] = fmaxf(fmaf(__uint_as_float(rr[i + 1]), os.y, bv.y), 0.0f);
-                            v[i + 2] = fmaxf(fmaf(__uint_as_float(rr[i + 2]), os.z, bv.z), 0.0f);
-                            v[i + 3] = fmaxf(fmaf(__uint_as_float(rr[i + 3]), os.w, bv.w), 0.0f);
+                            v[i + 0] = fmaf(__uint_as_float(rr[i + 0]), os.x, bv.x);
+                            v[i + 1] = fmaf(__uint_as_float(rr[i + 1]), os.y, bv.y);
+                            v[i + 2] = fmaf(__uint_as_float(rr[i + 2]), os.z, bv.z);
+                            v[i + 3] = fmaf(__uint_as_float(rr[i + 3]), os.w, bv.w);
                         } else {
-                            v[i + 0] = fmaxf(__uint_as_float(rr[i + 0]) + bv.x, 0.0f);
-                            v[i + 1] = fmaxf(__uint_as_float(rr[i + 1]) + bv.y, 0.0f);
-                            v[i + 2] = fmaxf(__uint_as_float(rr[i + 2]) + bv.z, 0.0f);
-                            v[i + 3] = fmaxf(__uint_as_float(rr[i + 3]) + bv.w, 0.0f);
+                            v[i + 0] = __uint_as_float(rr[i + 0]) + bv.x;
+                            v[i + 1] = __uint_as_float(rr[i + 1]) + bv.y;
+                            v[i + 2] = __uint_as_float(rr[i + 2]) + bv.z;
+                            v[i + 3] = __uint_as_float(rr[i + 3]) + bv.w;
                         }
+                    }
+                    // ReLU: a first convolution's output is only ever read as packed operands, and the
+                    // conversion clamps; elsewhere the fp32 value itself goes on (residual stream, output)
+                    if (!from_acc || (!kFp8 && args.absmax != nullptr)) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.0f);
                     }
                     if (!kFp8 && args.absmax != nullptr) {
                         // calibration: largest output of this layer per channel over all rows of the warp
@@ -521,10 +527,7 @@ tower_tc_kernel(const TowerArgs args) {
                     if (to_global && live) {
                         uint32_t pk[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-                            pk[i] = *reinterpret_cast<const uint32_t *>(&h2);
-                        }
+                        for (int i = 0; i < 8; ++i) pk[i] = ptx::pack_bf16x2_relu(v[2 * i], v[2 * i + 1]);
                         reinterpret_cast<uint4 *>(dst + kc * 16)[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         reinterpret_cast<uint4 *>(dst + kc * 16)[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                     }
@@ -534,20 +537,13 @@ tower_tc_kernel(const TowerArgs args) {
                             // 16 channels -> 16 e4m3 bytes (saturating, round to nearest even) = one slot of plane kc
                             uint32_t pk[4];
 #pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const float4 qs = *reinterpret_cast<const float4 *>(lc + 2 * kMyC + ks * 16 + 4 * i);
-                                const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(v[4 * i] * qs.x, v[4 * i + 1] * qs.y), __NV_SATFINITE, __NV_E4M3);
-                                const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(v[4 * i + 2] * qs.z, v[4 * i + 3] * qs.w), __NV_SATFINITE, __NV_E4M3);
-                                pk[i] = lo | (hi << 16);
-                            }
+                            for (int i = 0; i < 4; ++i)
+                                pk[i] = ptx::pack_e4m3x2_relu(v[4 * i], v[4 * i + 1]) | (ptx::pack_e4m3x2_relu(v[4 * i + 2], v[4 * i + 3]) << 16);
                             *reinterpret_cast<uint4 *>(frame + kc * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         } else {
                             uint32_t pk[8];
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) {
-                                const __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);
-                                pk[i] = *reinterpret_cast<const uint32_t *>(&h2);
-                            }
+                            for (int i = 0; i < 8; ++i) pk[i] = ptx::pack_bf16x2_relu(v[2 * i], v[2 * i + 1]);
                             *reinterpret_cast<uint4 *>(frame + (2 * kc) * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                             *reinterpret_cast<uint4 *>(frame + (2 * kc + 1) * kPlaneBytes + slot * 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                         }
@@ -560,7 +556,7 @@ tower_tc_kernel(const TowerArgs args) {
 #pragma unroll
                             for (int i = 0; i < 16; i += 4) {
                                 float4 hs = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
-                                if (kFp8) hs = *reinterpret_cast<const float4 *>(lc + 3 * kMyC + ks * 16 + i);
+                                if (kFp8) hs = *reinterpret_cast<const float4 *>(lc + 2 * kMyC + ks * 16 + i);
                                 w[i + 0] = __float_as_uint(kFp8 ? v[i + 0] * hs.x : v[i + 0]);
                                 w[i + 1] = __float_as_uint(kFp8 ? v[i + 1] * hs.y : v[i + 1]);
                                 w[i + 2] = __float_as_uint(kFp8 ? v[i + 2] * hs.z : v[i + 2]);
@@ -690,8 +686,11 @@ int tower_tc_launch_count() { return 1; }
 //     W'[co][ci][tap] = bn_scale[co] * W[co][ci][tap] * sa[ci]
 // is stored as e4m3 with one fp32 scale per output channel, ws[co] = max|W'[co]| / 448, so that
 //     conv = ws[co] * sum_k q_a[k] * q_w[co][k],   q_a = e4m3(a / sa), q_w = e4m3(W' / ws).
-// lconst[l] = { output scale ws (1 for layer 0), bias, 1/sa of the next layer, 1/ws of the next
-// conv2 (the residual stream sits in TMEM pre-divided by it) }.
+// With qs = 1/sa of the next layer (1 after the last), lconst[l] = { ws * qs (ws = 1 for layer 0),
+// bias * qs, 1 / (qs * ws of the next conv2) }: the epilogue forms v' = acc * lconst0 + lconst1, which is
+// the layer's output already divided by the next layer's activation scale, converts it to e4m3 (the
+// conversion clamps at zero: ReLU commutes with the positive scale), and on the residual stream writes
+// relu(v') * lconst2 back to TMEM, the stream pre-divided by the next conv2's weight scale.
 size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv) {
     return ((size_t)in_pad / 16 + (size_t)(n_conv - 1) * (channels / 32)) * kStageBytes;
 }
@@ -730,12 +729,13 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
                             }
     }
     for (int l = 0; l < n_conv; ++l) {
-        float *lc = lconst + (size_t)l * 4 * C;
+        float *lc = lconst + (size_t)l * 3 * C;
         for (int c = 0; c < C; ++c) {
-            lc[c] = l == 0 ? 1.0f : ws[(size_t)l * C + c];
-            lc[C + c] = bias[l][c];
-            lc[2 * C + c] = l + 1 < n_conv ? 1.0f / sa[(size_t)(l + 1) * C + c] : 1.0f;
-            lc[3 * C + c] = ((l & 1) == 0 && l + 2 < n_conv) ? 1.0f / ws[(size_t)(l + 2) * C + c] : 1.0f;
+            const float qs = l + 1 < n_conv ? 1.0f / sa[(size_t)(l + 1) * C + c] : 1.0f;
+            const float hs = ((l & 1) == 0 && l + 2 < n_conv) ? 1.0f / ws[(size_t)(l + 2) * C + c] : 1.0f;
+            lc[c] = (l == 0 ? 1.0f : ws[(size_t)l * C + c]) * qs;
+            lc[C + c] = bias[l][c] * qs;
+            lc[2 * C + c] = hs / qs;
         }
     }
 }
