@@ -43,7 +43,8 @@ enum {
     AZ_ERR_CUDA = -5,             /* a CUDA runtime call failed (see az_last_cuda_error) */
     AZ_ERR_DEVICE_TIMEOUT = -6,   /* a bounded device-side wait ran out (see az_device_status) */
     AZ_ERR_NOT_CALIBRATED = -7,   /* FP8 tower used before az_calibrate */
-    AZ_ERR_UNSUPPORTED = -8       /* valid request that this build has no kernel for */
+    AZ_ERR_UNSUPPORTED = -8,      /* valid request that this build has no kernel for */
+    AZ_ERR_BUSY = -9              /* az_submit_host: both in-flight slots are taken (az_wait_host first) */
 };
 
 enum { AZ_POLICY_PLANES73 = 0, AZ_POLICY_FLAT1858 = 1 };
@@ -156,6 +157,28 @@ int az_evaluate_legal_host(az_net *net, const void *positions_host, const uint64
  */
 int az_evaluate_host(az_net *net, const void *positions_host, const uint64_t *legal_masks_host,
                      int batch, float *policy_host, float *value_host, void *cuda_stream);
+
+/*
+ * Pipelined host entry (Sec. 5.2: double-buffered staging, asynchronous copies and completion
+ * events, so that the copies of one batch overlap the evaluation of the next).  az_submit_host
+ * queues one evaluation and returns at once with a ticket; az_wait_host blocks until that
+ * evaluation's results are in the caller's host buffers.  Up to AZ_HOST_SLOTS submissions may be
+ * in flight per az_net; they run in submission order on streams the az_net owns (created on the
+ * first call): the input copy of batch i+1 and the result copy of batch i-1 overlap the kernels of
+ * batch i.
+ *   - policy_host != NULL: dense output as az_evaluate_host (legal_policy_host / legal_counts_host
+ *     ignored); policy_host == NULL: legal-moves-only output as az_evaluate_legal_host.
+ *   - The host buffers must stay valid and untouched until az_wait_host returns for the ticket;
+ *     pinned memory is what makes the copies asynchronous.
+ *   - Tickets are small integers that are reused: wait for each ticket exactly once.
+ * Errors: az_submit_host BAD_ARG, BATCH_TOO_LARGE, NOT_CALIBRATED, BUSY (nothing queued), CUDA;
+ * az_wait_host BAD_ARG (no such ticket in flight), CUDA.
+ */
+#define AZ_HOST_SLOTS 2
+int az_submit_host(az_net *net, const void *positions_host, const uint64_t *legal_masks_host, int batch,
+                   float *policy_host, float *legal_policy_host, int32_t *legal_counts_host,
+                   float *value_host, int *ticket);
+int az_wait_host(az_net *net, int ticket);
 
 /*
  * The encoder step alone (App. D.1: side-to-move canonical planes; for Black to move ranks are

@@ -17,13 +17,14 @@ LIB_PATH = os.environ.get("AZ_EVAL_LIB") or os.path.join(_HERE, "libazeval.so")
 AZ_ABI_VERSION = 1
 AZ_OK = 0
 AZ_ERR_BAD_ARG, AZ_ERR_BAD_ARCH, AZ_ERR_BAD_WEIGHTS, AZ_ERR_BATCH_TOO_LARGE = -1, -2, -3, -4
-AZ_ERR_CUDA, AZ_ERR_DEVICE_TIMEOUT, AZ_ERR_NOT_CALIBRATED, AZ_ERR_UNSUPPORTED = -5, -6, -7, -8
+AZ_ERR_CUDA, AZ_ERR_DEVICE_TIMEOUT, AZ_ERR_NOT_CALIBRATED, AZ_ERR_UNSUPPORTED, AZ_ERR_BUSY = -5, -6, -7, -8, -9
+AZ_HOST_SLOTS = 2
 AZ_POLICY_PLANES73, AZ_POLICY_FLAT1858 = 0, 1
 AZ_VALUE_TANH, AZ_VALUE_WDL = 0, 1
 AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3 = 0, 1, 2
 
 EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
-           "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_encode", "az_tower", "az_tower_static", "az_legal_masks",
+           "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_submit_host", "az_wait_host", "az_encode", "az_tower", "az_tower_static", "az_legal_masks",
            "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error")
 
@@ -62,6 +63,10 @@ def _load_library():
     lib.az_evaluate_legal_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp]
     lib.az_evaluate_host.restype = ci
     lib.az_evaluate_host.argtypes = [vp, vp, vp, ci, vp, vp, vp]
+    lib.az_submit_host.restype = ci
+    lib.az_submit_host.argtypes = [vp, vp, vp, ci, vp, vp, vp, vp, ctypes.POINTER(ci)]
+    lib.az_wait_host.restype = ci
+    lib.az_wait_host.argtypes = [vp, ci]
     lib.az_profile_tower.restype = ci
     lib.az_profile_tower.argtypes = [vp, ci]
     lib.az_tower_time.restype = ci
@@ -197,6 +202,20 @@ def az_evaluate_legal_host(net: Net, positions_host, legal_masks_host, batch, le
     _check(_lib.az_evaluate_legal_host(net.handle, _host_ptr(positions_host, "positions"), _host_ptr(legal_masks_host, "legal_masks"),
                                        batch, _host_ptr(legal_policy_host, "legal_policy"), _host_ptr(legal_counts_host, "legal_counts"),
                                        _host_ptr(value_host, "value"), _stream_ptr(stream)), "az_evaluate_legal_host")
+
+
+def az_submit_host(net: Net, positions_host, legal_masks_host, batch, policy_host, legal_policy_host, legal_counts_host, value_host) -> int:
+    """Queues one evaluation on host buffers and returns its ticket (dense output if policy_host is given)."""
+    ticket = ctypes.c_int(-1)
+    opt = lambda t, name: None if t is None else _host_ptr(t, name)
+    _check(_lib.az_submit_host(net.handle, _host_ptr(positions_host, "positions"), _host_ptr(legal_masks_host, "legal_masks"), batch,
+                               opt(policy_host, "policy"), opt(legal_policy_host, "legal_policy"), opt(legal_counts_host, "legal_counts"),
+                               _host_ptr(value_host, "value"), ctypes.byref(ticket)), "az_submit_host")
+    return int(ticket.value)
+
+
+def az_wait_host(net: Net, ticket: int):
+    _check(_lib.az_wait_host(net.handle, ticket), "az_wait_host")
 
 
 def az_profile_tower(net: Net, enable: bool):

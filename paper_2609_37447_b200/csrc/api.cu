@@ -254,6 +254,15 @@ void free_net(Net *n) {
     for (int i = 0; i < 3; ++i) cudaFree(n->act[i]);
     cudaFree(n->stage_pos); cudaFree(n->stage_masks); cudaFree(n->stage_policy); cudaFree(n->stage_value);
     cudaFree(n->stage_compact); cudaFree(n->stage_counts);
+    for (Net::HostSlot &sl : n->slots) {
+        cudaFree(sl.pos); cudaFree(sl.masks); cudaFree(sl.policy); cudaFree(sl.value); cudaFree(sl.compact); cudaFree(sl.counts);
+        if (sl.in_ready) cudaEventDestroy(sl.in_ready);
+        if (sl.computed) cudaEventDestroy(sl.computed);
+        if (sl.out_ready) cudaEventDestroy(sl.out_ready);
+    }
+    if (n->s_in) cudaStreamDestroy(n->s_in);
+    if (n->s_compute) cudaStreamDestroy(n->s_compute);
+    if (n->s_out) cudaStreamDestroy(n->s_out);
     if (n->ev_begin) for (int i = 0; i < kMaxProfiledPasses; ++i) { cudaEventDestroy(n->ev_begin[i]); cudaEventDestroy(n->ev_end[i]); }
     delete[] n->ev_begin; delete[] n->ev_end;
     cudaFree(n->logits); cudaFree(n->head_p); cudaFree(n->head_v); cudaFree(n->hidden); cudaFree(n->status_dev);
@@ -476,6 +485,71 @@ int az_evaluate_host(az_net *net, const void *positions_host, const uint64_t *le
     return AZ_OK;
 }
 
+int az_submit_host(az_net *net, const void *positions_host, const uint64_t *legal_masks_host, int batch,
+                   float *policy_host, float *legal_policy_host, int32_t *legal_counts_host,
+                   float *value_host, int *ticket) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n || batch <= 0 || !ticket || !positions_host || !legal_masks_host || !value_host) return AZ_ERR_BAD_ARG;
+    const bool dense = policy_host != nullptr;
+    if (!dense && (!legal_policy_host || !legal_counts_host)) return AZ_ERR_BAD_ARG;
+    if ((uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
+    if (n->fp8 && !n->fp8_ready) return AZ_ERR_NOT_CALIBRATED;
+    const az_arch &a = n->arch;
+    const size_t B = a.max_batch, pb = az_position_bytes(&a), mw = az_mask_words(&a), ps = az_policy_size(&a), vs = az_value_size(&a);
+    if (!n->s_compute) {
+        AZ_CUDA(cudaStreamCreateWithFlags(&n->s_in, cudaStreamNonBlocking));
+        AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute, cudaStreamNonBlocking));
+        AZ_CUDA(cudaStreamCreateWithFlags(&n->s_out, cudaStreamNonBlocking));
+    }
+    Net::HostSlot &sl = n->slots[n->next_slot];
+    if (sl.busy) return AZ_ERR_BUSY;
+    if (!sl.pos) {
+        AZ_CUDA(cudaMalloc(&sl.pos, B * pb));
+        AZ_CUDA(cudaMalloc((void **)&sl.masks, B * mw * sizeof(uint64_t)));
+        AZ_CUDA(cudaMalloc((void **)&sl.value, B * vs * sizeof(float)));
+        AZ_CUDA(cudaEventCreateWithFlags(&sl.in_ready, cudaEventDisableTiming));
+        AZ_CUDA(cudaEventCreateWithFlags(&sl.computed, cudaEventDisableTiming));
+        AZ_CUDA(cudaEventCreateWithFlags(&sl.out_ready, cudaEventDisableTiming));
+    }
+    if (dense && !sl.policy) AZ_CUDA(cudaMalloc((void **)&sl.policy, B * ps * sizeof(float)));
+    if (!dense && !sl.compact) {
+        AZ_CUDA(cudaMalloc((void **)&sl.compact, B * AZ_MAX_LEGAL * sizeof(float)));
+        AZ_CUDA(cudaMalloc((void **)&sl.counts, B * sizeof(int)));
+    }
+    // A slot is handed out again only after az_wait_host saw its result copy finish, and that copy was
+    // ordered after the slot's kernels: neither the staging inputs nor the outputs are still in use.
+    AZ_CUDA(cudaMemcpyAsync(sl.pos, positions_host, (size_t)batch * pb, cudaMemcpyHostToDevice, n->s_in));
+    AZ_CUDA(cudaMemcpyAsync(sl.masks, legal_masks_host, (size_t)batch * mw * sizeof(uint64_t), cudaMemcpyHostToDevice, n->s_in));
+    AZ_CUDA(cudaEventRecord(sl.in_ready, n->s_in));
+    AZ_CUDA(cudaStreamWaitEvent(n->s_compute, sl.in_ready, 0));
+    const int rc = dense ? az_evaluate(net, sl.pos, sl.masks, batch, sl.policy, sl.value, n->s_compute)
+                         : az_evaluate_legal(net, sl.pos, sl.masks, batch, sl.compact, sl.counts, sl.value, n->s_compute);
+    if (rc != AZ_OK) return rc;
+    AZ_CUDA(cudaEventRecord(sl.computed, n->s_compute));
+    AZ_CUDA(cudaStreamWaitEvent(n->s_out, sl.computed, 0));
+    if (dense) {
+        AZ_CUDA(cudaMemcpyAsync(policy_host, sl.policy, (size_t)batch * ps * sizeof(float), cudaMemcpyDeviceToHost, n->s_out));
+    } else {
+        AZ_CUDA(cudaMemcpyAsync(legal_policy_host, sl.compact, (size_t)batch * AZ_MAX_LEGAL * sizeof(float), cudaMemcpyDeviceToHost, n->s_out));
+        AZ_CUDA(cudaMemcpyAsync(legal_counts_host, sl.counts, (size_t)batch * sizeof(int), cudaMemcpyDeviceToHost, n->s_out));
+    }
+    AZ_CUDA(cudaMemcpyAsync(value_host, sl.value, (size_t)batch * vs * sizeof(float), cudaMemcpyDeviceToHost, n->s_out));
+    AZ_CUDA(cudaEventRecord(sl.out_ready, n->s_out));
+    sl.busy = true;
+    *ticket = n->next_slot;
+    n->next_slot = (n->next_slot + 1) % AZ_HOST_SLOTS;
+    return AZ_OK;
+}
+
+int az_wait_host(az_net *net, int ticket) {
+    Net *n = reinterpret_cast<Net *>(net);
+    if (!n || ticket < 0 || ticket >= AZ_HOST_SLOTS || !n->slots[ticket].busy) return AZ_ERR_BAD_ARG;
+    Net::HostSlot &sl = n->slots[ticket];
+    sl.busy = false;
+    AZ_CUDA(cudaEventSynchronize(sl.out_ready));
+    return AZ_OK;
+}
+
 int az_profile_tower(az_net *net, int enable) {
     Net *n = reinterpret_cast<Net *>(net);
     if (!n) return AZ_ERR_BAD_ARG;
@@ -586,6 +660,7 @@ const char *az_strerror(int code) {
         case AZ_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
         case AZ_ERR_NOT_CALIBRATED: return "FP8 network not calibrated";
         case AZ_ERR_UNSUPPORTED: return "not supported by this build";
+        case AZ_ERR_BUSY: return "all in-flight slots are taken";
         default: return "unknown error";
     }
 }

@@ -85,6 +85,19 @@ struct Net {
     float *stage_compact = nullptr;   // [max_batch][AZ_MAX_LEGAL]
     int *stage_counts = nullptr;
 
+    // ---- pipelined host entry: per-slot staging, the az_net's own streams and events ----
+    struct HostSlot {
+        void *pos = nullptr;
+        uint64_t *masks = nullptr;
+        float *policy = nullptr, *value = nullptr, *compact = nullptr;
+        int *counts = nullptr;
+        cudaEvent_t in_ready = nullptr, computed = nullptr, out_ready = nullptr;
+        bool busy = false;
+    };
+    HostSlot slots[AZ_HOST_SLOTS];
+    cudaStream_t s_in = nullptr, s_compute = nullptr, s_out = nullptr;
+    int next_slot = 0;
+
     // ---- optional event timing of the tower ----
     bool profile = false;
     int n_events = 0;                 // pairs recorded since the last read

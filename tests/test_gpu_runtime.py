@@ -42,6 +42,49 @@ def test_host_buffer_entry_point_gives_the_same_results(setup):
     assert (pol_n == policy.cpu().numpy()).all() and (val_n == value.cpu().numpy()).all()
 
 
+def test_pipelined_host_entry_matches_and_bounds_its_queue(setup):
+    az, net, recs, pos, masks, policy, value = setup
+    pos_h = torch.from_numpy(np.ascontiguousarray(recs).view(np.uint8).reshape(96, -1).copy()).pin_memory()
+    masks_h = masks.cpu().pin_memory()
+    # six batches of different sizes through two slots; every result must equal the synchronous one
+    sizes = [96, 17, 64, 96, 1, 50]
+    outs = [(torch.full((96, 1858), -1.0).pin_memory(), torch.full((96, 3), -1.0).pin_memory()) for _ in sizes]
+    tickets = []
+    for i, n in enumerate(sizes):
+        if len(tickets) == az.AZ_HOST_SLOTS:
+            az.az_wait_host(net, tickets.pop(0))
+        tickets.append(az.az_submit_host(net, pos_h, masks_h, n, outs[i][0], None, None, outs[i][1]))
+    for t in tickets:
+        az.az_wait_host(net, t)
+    for (pol_h, val_h), n in zip(outs, sizes):
+        assert torch.equal(pol_h[:n], policy.cpu()[:n]) and torch.equal(val_h[:n], value.cpu()[:n])
+        assert (pol_h[n:] == -1.0).all()
+    # legal-moves-only output through the same queue
+    legal_ref = torch.zeros((96, az.AZ_MAX_LEGAL), device="cuda")
+    counts_ref = torch.zeros((96,), dtype=torch.int32, device="cuda")
+    az.az_evaluate_legal(net, pos, masks, 96, legal_ref, counts_ref, torch.zeros_like(value))
+    torch.cuda.synchronize()
+    legal_h = torch.zeros((96, az.AZ_MAX_LEGAL)).pin_memory()
+    counts_h = torch.zeros((96,), dtype=torch.int32).pin_memory()
+    val_h = torch.zeros((96, 3)).pin_memory()
+    az.az_wait_host(net, az.az_submit_host(net, pos_h, masks_h, 96, None, legal_h, counts_h, val_h))
+    assert torch.equal(counts_h, counts_ref.cpu()) and torch.equal(val_h, value.cpu())
+    for b in range(96):
+        assert torch.equal(legal_h[b, :counts_h[b]], legal_ref.cpu()[b, :counts_h[b]])
+    # a third submission while two are in flight is refused and queues nothing; a stale ticket is an error
+    t0 = az.az_submit_host(net, pos_h, masks_h, 96, outs[0][0], None, None, outs[0][1])
+    t1 = az.az_submit_host(net, pos_h, masks_h, 96, outs[1][0], None, None, outs[1][1])
+    with pytest.raises(az.AzError) as err:
+        az.az_submit_host(net, pos_h, masks_h, 96, outs[2][0], None, None, outs[2][1])
+    assert err.value.code == az.AZ_ERR_BUSY
+    az.az_wait_host(net, t0)
+    az.az_wait_host(net, t1)
+    with pytest.raises(az.AzError) as err:
+        az.az_wait_host(net, t0)
+    assert err.value.code == az.AZ_ERR_BAD_ARG
+    assert az.az_device_status(net) == 0
+
+
 def test_legal_moves_only_output_matches_the_dense_policy(setup):
     az, net, recs, pos, masks, policy, value = setup
     legal = torch.full((96, az.AZ_MAX_LEGAL), -1.0, device="cuda")
