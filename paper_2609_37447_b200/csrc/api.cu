@@ -8,6 +8,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <utility>
 #include <vector>
 
 namespace az {
@@ -261,8 +262,9 @@ void free_net(Net *n) {
         if (sl.out_ready) cudaEventDestroy(sl.out_ready);
     }
     if (n->s_in) cudaStreamDestroy(n->s_in);
-    if (n->s_compute) cudaStreamDestroy(n->s_compute);
+    for (cudaStream_t s : n->s_compute) if (s) cudaStreamDestroy(s);
     if (n->s_out) cudaStreamDestroy(n->s_out);
+    cudaFree(n->alt_u_policy); cudaFree(n->alt_u_value); cudaFree(n->alt_logits);
     if (n->ev_begin) for (int i = 0; i < kMaxProfiledPasses; ++i) { cudaEventDestroy(n->ev_begin[i]); cudaEventDestroy(n->ev_end[i]); }
     delete[] n->ev_begin; delete[] n->ev_end;
     cudaFree(n->logits); cudaFree(n->head_p); cudaFree(n->head_v); cudaFree(n->hidden); cudaFree(n->status_dev);
@@ -496,13 +498,26 @@ int az_submit_host(az_net *net, const void *positions_host, const uint64_t *lega
     if (n->fp8 && !n->fp8_ready) return AZ_ERR_NOT_CALIBRATED;
     const az_arch &a = n->arch;
     const size_t B = a.max_batch, pb = az_position_bytes(&a), mw = az_mask_words(&a), ps = az_policy_size(&a), vs = az_value_size(&a);
-    if (!n->s_compute) {
+    if (!n->s_in) {
         AZ_CUDA(cudaStreamCreateWithFlags(&n->s_in, cudaStreamNonBlocking));
-        AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute, cudaStreamNonBlocking));
         AZ_CUDA(cudaStreamCreateWithFlags(&n->s_out, cudaStreamNonBlocking));
+        AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute[0], cudaStreamNonBlocking));
+        // The tensor-core path keeps nothing else between its kernels than the head GEMM's operands and
+        // the logits; with a second copy of those, odd slots run on a stream of their own.  The other
+        // paths share one workspace, so all their slots take turns on one stream.
+        if (n->tc_ready) {
+            const size_t u_bytes = (size_t)((a.max_batch + 127) / 128) * az::kHeadChannels * 64 * 128 * sizeof(__nv_bfloat16);
+            AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute[1], cudaStreamNonBlocking));
+            AZ_CUDA(cudaMalloc(&n->alt_u_value, u_bytes));
+            AZ_CUDA(cudaMemset(n->alt_u_value, 0, u_bytes));
+            if (n->u_policy) { AZ_CUDA(cudaMalloc(&n->alt_u_policy, u_bytes)); AZ_CUDA(cudaMemset(n->alt_u_policy, 0, u_bytes)); }
+            AZ_CUDA(cudaMalloc((void **)&n->alt_logits, B * ps * sizeof(float)));
+        }
     }
     Net::HostSlot &sl = n->slots[n->next_slot];
     if (sl.busy) return AZ_ERR_BUSY;
+    const bool alt = n->s_compute[1] != nullptr && (n->next_slot & 1);
+    cudaStream_t sc = alt ? n->s_compute[1] : n->s_compute[0];
     if (!sl.pos) {
         AZ_CUDA(cudaMalloc(&sl.pos, B * pb));
         AZ_CUDA(cudaMalloc((void **)&sl.masks, B * mw * sizeof(uint64_t)));
@@ -521,11 +536,15 @@ int az_submit_host(az_net *net, const void *positions_host, const uint64_t *lega
     AZ_CUDA(cudaMemcpyAsync(sl.pos, positions_host, (size_t)batch * pb, cudaMemcpyHostToDevice, n->s_in));
     AZ_CUDA(cudaMemcpyAsync(sl.masks, legal_masks_host, (size_t)batch * mw * sizeof(uint64_t), cudaMemcpyHostToDevice, n->s_in));
     AZ_CUDA(cudaEventRecord(sl.in_ready, n->s_in));
-    AZ_CUDA(cudaStreamWaitEvent(n->s_compute, sl.in_ready, 0));
-    const int rc = dense ? az_evaluate(net, sl.pos, sl.masks, batch, sl.policy, sl.value, n->s_compute)
-                         : az_evaluate_legal(net, sl.pos, sl.masks, batch, sl.compact, sl.counts, sl.value, n->s_compute);
+    AZ_CUDA(cudaStreamWaitEvent(sc, sl.in_ready, 0));
+    // kernel arguments are captured when a kernel is launched: pointing the net at the other copy for
+    // the duration of the (asynchronous) launches is all it takes
+    if (alt) { std::swap(n->u_policy, n->alt_u_policy); std::swap(n->u_value, n->alt_u_value); std::swap(n->logits, n->alt_logits); }
+    const int rc = dense ? az_evaluate(net, sl.pos, sl.masks, batch, sl.policy, sl.value, sc)
+                         : az_evaluate_legal(net, sl.pos, sl.masks, batch, sl.compact, sl.counts, sl.value, sc);
+    if (alt) { std::swap(n->u_policy, n->alt_u_policy); std::swap(n->u_value, n->alt_u_value); std::swap(n->logits, n->alt_logits); }
     if (rc != AZ_OK) return rc;
-    AZ_CUDA(cudaEventRecord(sl.computed, n->s_compute));
+    AZ_CUDA(cudaEventRecord(sl.computed, sc));
     AZ_CUDA(cudaStreamWaitEvent(n->s_out, sl.computed, 0));
     if (dense) {
         AZ_CUDA(cudaMemcpyAsync(policy_host, sl.policy, (size_t)batch * ps * sizeof(float), cudaMemcpyDeviceToHost, n->s_out));

@@ -95,8 +95,13 @@ struct Net {
         bool busy = false;
     };
     HostSlot slots[AZ_HOST_SLOTS];
-    cudaStream_t s_in = nullptr, s_compute = nullptr, s_out = nullptr;
+    cudaStream_t s_in = nullptr, s_compute[AZ_HOST_SLOTS] = {}, s_out = nullptr;
     int next_slot = 0;
+    // second copy of what the tensor-core path keeps between its three kernels, so that the second
+    // slot's evaluation can run beside the first's: the tail of one tower launch (the last, partly
+    // filled round of board groups) overlaps the head of the next
+    void *alt_u_policy = nullptr, *alt_u_value = nullptr;
+    float *alt_logits = nullptr;
 
     // ---- optional event timing of the tower ----
     bool profile = false;
