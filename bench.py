@@ -55,9 +55,10 @@ def load_peaks():
     try:
         with open(path) as f:
             p = json.load(f)
-        return {"bf16_tflops": float(p["bf16_tflops"]), "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
+        return {"bf16_tflops": float(p["bf16_tflops"]), "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
     except (OSError, KeyError, ValueError):
-        return {"bf16_tflops": 1590.0, "hbm_gbs": 6650.0, "source": "fallback"}
+        return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
 
 
 class ClockSampler(threading.Thread):
@@ -315,8 +316,13 @@ def main():
         achieved = flops / (tower_avg_ms * 1e-3) / 1e12 if tower_passes else None
         traffic = tower_traffic_bytes(cfg, B)
         # FP8 contraction: the measured bf16 peak times the nominal e4m3/bf16 ratio of 2 (4.5 / 2.25 PFLOP/s)
-        peak_tf = peaks["bf16_tflops"] * (2.0 if cfg.precision == 2 else 1.0)
-        peak_note = f"of {peaks['source']} (burst bf16 GEMM" + (" x 2, nominal e4m3/bf16 ratio)" if cfg.precision == 2 else ")")
+        # a tower launch of a few hundred microseconds between L2 flushes is a burst; launches of
+        # milliseconds back to back for the whole timed region run under the power cap like the sustained GEMM
+        sustained = tower_avg_ms >= 2.0
+        peak_tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"] * (2.0 if cfg.precision == 2 else 1.0)
+        peak_note = (f"of {peaks['source']} ({'sustained' if sustained else 'burst'} bf16 GEMM"
+                     + (" x 2, nominal e4m3/bf16 ratio" if cfg.precision == 2 else "")
+                     + "; sustained is used when a tower launch takes 2 ms or more)")
         out = {
             "metric": METRIC, "value": evals / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
