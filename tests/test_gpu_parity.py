@@ -207,6 +207,28 @@ def test_c5_40x256_history_planes_bf16(az, batch):
     az.az_free_net(net)
 
 
+@pytest.mark.parametrize("batch", [1024, 8192])
+def test_c5_large_batches_on_sampled_rows(az, batch):
+    # the sizes bench.py times: the whole batch runs on the GPU (several rounds of the persistent
+    # kernel, a ragged last one), the oracle checks rows spread over it, first and last included;
+    # properties that hold at any size cover the rest
+    import dataclasses
+    cfg = dataclasses.replace(configs.CONFIGS["c5"], batch=batch)
+    net, blob = load(az, cfg)
+    recs = positions.for_config(cfg, batch)
+    mg, pg, vg = gpu_evaluate(az, net, cfg, recs)
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+    rows = np.unique(np.concatenate([[0, 1, 295, 296, 297, batch - 2, batch - 1],
+                                     np.random.default_rng(batch).integers(0, batch, 9)]))
+    mo, _, po, vo = oracle.evaluate(blob, recs[rows], cfg.in_planes, cfg.policy_head)
+    compare(cfg, mg[rows], pg[rows], vg[rows], mo, po, vo, TOL[1])
+    bits = np.unpackbits(mg.view(np.uint8), axis=1, bitorder="little")[:, : cfg.policy_size].astype(bool)
+    assert np.isfinite(pg).all() and np.isfinite(vg).all()
+    assert (pg[~bits] == 0.0).all() and (pg[bits] > 0.0).all()
+    assert np.abs(pg.sum(axis=1) - 1.0).max() < 1e-3 and np.abs(vg.sum(axis=1) - 1.0).max() < 1e-5
+
+
 def fp8_run(az, name, batch, oracle_rows):
     """Load the FP8 net, calibrate it on the 512 seeded calibration positions, evaluate `batch`
     positions, and return GPU and oracle results on `oracle_rows` of them, plus tower outputs."""
