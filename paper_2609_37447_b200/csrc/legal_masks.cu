@@ -1,11 +1,12 @@
 // Legal-move masks on the GPU (App. D.1: illegal actions are masked before the softmax; castling
 // is the king-to-own-rook pair, en passant the pawn's ordinary origin-destination pair).
 //
-// Bitboard move generation, one thread per position: pseudo-legal target sets per piece from
-// shift/ray arithmetic, each move tried on a copy of the bitboards and kept if the mover's king
-// is not attacked afterwards.  The mask row is built in registers/local memory and written once.
-// The work per position is a few thousand integer operations; the kernel is latency-bound and
-// runs off the timed path (masks are an input of az_evaluate).
+// Bitboard move generation, one warp per position: pseudo-legal target sets per piece from
+// shift/ray arithmetic (one lane per square pair), then every listed move tried on a copy of the
+// bitboards (moves dealt out over the lanes) and kept if the mover's king is not attacked
+// afterwards.  The mask row is built in shared memory and written once.  The work per position is
+// a few thousand integer operations; masks are an input of az_evaluate, so the kernel runs off
+// that call's timed path.
 #include "common.cuh"
 
 #include <mutex>
@@ -99,16 +100,27 @@ __device__ __forceinline__ void set_move(u64 *row, int stm, int from, int to, in
         idx = promo ? g_flat_promo[(from & 7) * 3 + ((to & 7) - (from & 7) + 1)] + (promo - 1)
                     : g_flat_pair[from * 64 + to];
     }
-    row[idx >> 6] |= 1ull << (idx & 63);
+    atomicOr(row + (idx >> 6), 1ull << (idx & 63));          // the row sits in shared memory, lanes share it
 }
 
+// One warp per position.  Step 1: lane L looks at squares L and L + 32; if one of the mover's pieces
+// stands there it lists that piece's pseudo-legal moves in shared memory.  Step 2: the listed moves
+// are dealt out over the 32 lanes; each is tried on a copy of the bitboards and, if the mover's king
+// is not attacked afterwards, its bit (four bits for a promotion) is set in the shared mask row.
+constexpr int kWarpsPerBlock = 4;
+constexpr int kMaxListed = 384;            // pseudo-legal moves of one position (218 legal at most in chess)
+
 template <int HEAD>
-__global__ void __launch_bounds__(64)
+__global__ void __launch_bounds__(32 * kWarpsPerBlock)
 legal_masks_kernel(const unsigned char *__restrict__ positions, size_t stride, int batch,
                    u64 *__restrict__ masks) {
     constexpr int WORDS = HEAD == AZ_POLICY_PLANES73 ? 73 : 30;
-    const int pos = blockIdx.x * blockDim.x + threadIdx.x;
-    if (pos >= batch) return;
+    __shared__ u64 s_row[kWarpsPerBlock][WORDS];
+    __shared__ unsigned s_list[kWarpsPerBlock][kMaxListed];
+    __shared__ int s_count[kWarpsPerBlock];
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pos = blockIdx.x * kWarpsPerBlock + w;
+    if (pos >= batch) return;                                // whole warps leave together
     const PosCur *r = reinterpret_cast<const PosCur *>(positions + (size_t)pos * stride);
     u64 own[6], opp[6];
     const int stm = r->stm & 1;
@@ -121,86 +133,94 @@ legal_masks_kernel(const unsigned char *__restrict__ positions, size_t stride, i
     const int them = stm ^ 1;
     const int king_sq = own[5] ? __ffsll((long long)own[5]) - 1 : 0;
     const int ep = r->ep_square;
+    u64 *row = s_row[w];
+    unsigned *list = s_list[w];
+    for (int i = lane; i < WORDS; i += 32) row[i] = 0;
+    if (lane == 0) s_count[w] = 0;
+    __syncwarp();
 
-    u64 row[WORDS];
+    // ---- step 1: pseudo-legal moves, entry = kind | from << 3 | to << 9
 #pragma unroll 1
-    for (int w = 0; w < WORDS; ++w) row[w] = 0;
+    for (int half = 0; half < 2; ++half) {
+        const int from = lane + 32 * half;
+        const u64 fb = 1ull << from;
+        if (!(own_occ & fb)) continue;
+        int k = 0;
+#pragma unroll
+        for (int j = 1; j < 6; ++j) if (own[j] & fb) k = j;
+        u64 targets;
+        if (k == 0) {
+            u64 push, cap;
+            if (stm == 0) {
+                push = (fb << 8) & ~occ;
+                if (push && (from >> 3) == 1) push |= (fb << 16) & ~occ;
+                cap = (((fb << 9) & ~FILE_A) | ((fb << 7) & ~FILE_H));
+            } else {
+                push = (fb >> 8) & ~occ;
+                if (push && (from >> 3) == 6) push |= (fb >> 16) & ~occ;
+                cap = (((fb >> 9) & ~FILE_H) | ((fb >> 7) & ~FILE_A));
+            }
+            const u64 ep_bit = ep < 64 ? (1ull << ep) : 0ull;
+            targets = push | (cap & (opp_occ | (ep_bit & ~occ)));
+        } else if (k == 1) targets = knight_set(fb) & ~own_occ;
+        else if (k == 5) targets = king_set(fb) & ~own_occ;
+        else {
+            targets = 0;
+            if (k != 3) targets |= ray_set(from, occ, true);
+            if (k != 2) targets |= ray_set(from, occ, false);
+            targets &= ~own_occ;
+        }
+        int at = atomicAdd(&s_count[w], __popcll(targets));
+        while (targets) {
+            const int to = __ffsll((long long)targets) - 1;
+            targets &= targets - 1;
+            if (at < kMaxListed) list[at] = (unsigned)k | ((unsigned)from << 3) | ((unsigned)to << 9);
+            ++at;
+        }
+    }
+    __syncwarp();
+    const int listed = min(s_count[w], kMaxListed);
 
-    // try one move: piece kind k from `from` to `to`; ep_cap = square of a pawn captured en passant (or -1)
-    auto legal = [&](int k, int from, int to, int ep_cap) -> bool {
+    // ---- step 2: keep the moves that do not leave the mover's king attacked
+    for (int i = lane; i < listed; i += 32) {
+        const unsigned e = list[i];
+        const int k = e & 7, from = (e >> 3) & 63, to = (e >> 9) & 63;
         const u64 fb = 1ull << from, tb = 1ull << to;
         u64 o[6];
 #pragma unroll
         for (int j = 0; j < 6; ++j) o[j] = opp[j] & ~tb;
         u64 n_occ = (occ & ~fb) | tb;
-        if (ep_cap >= 0) { o[0] &= ~(1ull << ep_cap); n_occ &= ~(1ull << ep_cap); }
-        const int ksq = k == 5 ? to : king_sq;
-        return !attacked(ksq, them, o, n_occ);
-    };
-
-#pragma unroll 1
-    for (int k = 0; k < 6; ++k) {
-        u64 pieces = own[k];
-        while (pieces) {
-            const int from = __ffsll((long long)pieces) - 1;
-            pieces &= pieces - 1;
-            const u64 fb = 1ull << from;
-            u64 targets;
-            if (k == 0) {
-                u64 push, cap;
-                if (stm == 0) {
-                    push = (fb << 8) & ~occ;
-                    if (push && (from >> 3) == 1) push |= (fb << 16) & ~occ;
-                    cap = (((fb << 9) & ~FILE_A) | ((fb << 7) & ~FILE_H));
-                } else {
-                    push = (fb >> 8) & ~occ;
-                    if (push && (from >> 3) == 6) push |= (fb >> 16) & ~occ;
-                    cap = (((fb >> 9) & ~FILE_H) | ((fb >> 7) & ~FILE_A));
-                }
-                const u64 ep_bit = ep < 64 ? (1ull << ep) : 0ull;
-                targets = push | (cap & (opp_occ | (ep_bit & ~occ)));
-            } else if (k == 1) targets = knight_set(fb) & ~own_occ;
-            else if (k == 5) targets = king_set(fb) & ~own_occ;
-            else {
-                targets = 0;
-                if (k != 3) targets |= ray_set(from, occ, true);
-                if (k != 2) targets |= ray_set(from, occ, false);
-                targets &= ~own_occ;
-            }
-            while (targets) {
-                const int to = __ffsll((long long)targets) - 1;
-                targets &= targets - 1;
-                int ep_cap = -1;
-                if (k == 0 && to == ep && ((from ^ to) & 7) != 0 && !((opp_occ >> to) & 1ull))
-                    ep_cap = (to & 7) + 8 * (from >> 3);
-                if (!legal(k, from, to, ep_cap)) continue;
-                const bool promotes = k == 0 && ((to >> 3) == (stm ? 0 : 7));
-                set_move<HEAD>(row, stm, from, to, 0);        // plain pair (= queen promotion)
-                if (promotes) {
-                    set_move<HEAD>(row, stm, from, to, 1);
-                    set_move<HEAD>(row, stm, from, to, 2);
-                    set_move<HEAD>(row, stm, from, to, 3);
-                }
-            }
+        if (k == 0 && to == ep && ((from ^ to) & 7) != 0 && !((opp_occ >> to) & 1ull)) {
+            const int ep_cap = (to & 7) + 8 * (from >> 3);   // the pawn taken en passant leaves the board too
+            o[0] &= ~(1ull << ep_cap);
+            n_occ &= ~(1ull << ep_cap);
+        }
+        if (attacked(k == 5 ? to : king_sq, them, o, n_occ)) continue;
+        set_move<HEAD>(row, stm, from, to, 0);               // plain pair (= queen promotion)
+        if (k == 0 && ((to >> 3) == (stm ? 0 : 7))) {
+            set_move<HEAD>(row, stm, from, to, 1);
+            set_move<HEAD>(row, stm, from, to, 2);
+            set_move<HEAD>(row, stm, from, to, 3);
         }
     }
     // castling: rights, king and rook at home, squares between empty, king's path not attacked
-    {
+    // (lane 0 the king side, lane 1 the queen side)
+    if (lane < 2) {
         const int r0 = stm ? 56 : 0;
         const int kbit = stm ? 4 : 1, qbit = stm ? 8 : 2;
         const int c = r->castling;
         if ((c & (kbit | qbit)) && king_sq == r0 + 4 && !attacked(r0 + 4, them, opp, occ)) {
-            if ((c & kbit) && ((own[3] >> (r0 + 7)) & 1ull) && !(occ & (3ull << (r0 + 5))) &&
+            if (lane == 0 && (c & kbit) && ((own[3] >> (r0 + 7)) & 1ull) && !(occ & (3ull << (r0 + 5))) &&
                 !attacked(r0 + 5, them, opp, occ) && !attacked(r0 + 6, them, opp, occ))
                 set_move<HEAD>(row, stm, r0 + 4, r0 + 7, 0);
-            if ((c & qbit) && ((own[3] >> r0) & 1ull) && !(occ & (7ull << (r0 + 1))) &&
+            if (lane == 1 && (c & qbit) && ((own[3] >> r0) & 1ull) && !(occ & (7ull << (r0 + 1))) &&
                 !attacked(r0 + 3, them, opp, occ) && !attacked(r0 + 2, them, opp, occ))
                 set_move<HEAD>(row, stm, r0 + 4, r0, 0);
         }
     }
+    __syncwarp();
     u64 *dst = masks + (size_t)pos * WORDS;
-#pragma unroll 1
-    for (int w = 0; w < WORDS; ++w) dst[w] = row[w];
+    for (int i = lane; i < WORDS; i += 32) dst[i] = row[i];
 }
 
 // ---- host: flat-1858 tables -------------------------------------------------------------------
@@ -246,8 +266,8 @@ int launch_legal_masks(const void *positions, size_t stride, int batch, int head
                        cudaStream_t s) {
     if (batch == 0) return AZ_OK;
     const unsigned char *p = static_cast<const unsigned char *>(positions);
-    const int block = 64;
-    const unsigned grid = (unsigned)((batch + block - 1) / block);
+    const int block = 32 * kWarpsPerBlock;
+    const unsigned grid = (unsigned)((batch + kWarpsPerBlock - 1) / kWarpsPerBlock);
     if (head == AZ_POLICY_PLANES73) {
         legal_masks_kernel<AZ_POLICY_PLANES73><<<grid, block, 0, s>>>(p, stride, batch, (u64 *)masks);
     } else {
