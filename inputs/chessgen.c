@@ -51,6 +51,16 @@ typedef struct {
     uint8_t n_hist;
 } RecH8;
 
+/* Record with the last eight moves instead of the last seven boards (128 bytes): the input of
+ * the 52-plane encoder (App. D.1, Table D.1: recent moves as origin / destination squares,
+ * castling recorded as the king's own move). */
+typedef struct {
+    RecCur cur;
+    uint8_t move_from[8], move_to[8]; /* absolute squares, most recent move first */
+    uint8_t n_moves;                  /* how many of the eight exist */
+    uint8_t pad[7];
+} RecM8;
+
 /* ---- random stream ------------------------------------------------------- */
 typedef struct { uint64_t s[4]; } Rng;
 static uint64_t splitmix64(uint64_t *x) {
@@ -277,60 +287,99 @@ static int same_position(const Board *a, const Board *b) {
  * [lo_even, hi_even], odd ones from [lo_odd, hi_odd].  plies_out (optional)
  * receives each record's ply count.  Returns 0, or -1 on bad arguments.
  */
+static int play_one(uint64_t base_seed, int64_t index, int lo_even, int hi_even, int lo_odd, int hi_odd,
+                    Board *game, int *reps, Move *played)
+{
+    Rng rng; rng_seed(&rng, base_seed ^ (uint64_t)index);
+    int lo = (index & 1) ? lo_odd : lo_even, hi = (index & 1) ? hi_odd : hi_even;
+    int n;
+    for (;;) {
+        n = lo + (int)(rng_next(&rng) % (uint64_t)(hi - lo + 1));
+        board_start(&game[0]); reps[0] = 0;
+        int ply = 0, ok = 1;
+        Move list[256];
+        for (; ply < n; ++ply) {
+            int k = legal_moves(&game[ply], list);
+            if (k == 0) { ok = 0; break; }
+            qsort(list, (size_t)k, sizeof(Move), cmp_move);
+            Move m = list[rng_next(&rng) % (uint64_t)k];
+            played[ply] = m;
+            game[ply + 1] = game[ply];
+            make_move(&game[ply + 1], m);
+            int r = 0;
+            for (int j = 0; j <= ply; ++j) r += same_position(&game[j], &game[ply + 1]);
+            reps[ply + 1] = r;
+        }
+        if (ok) {
+            Move tmp[256];
+            if (legal_moves(&game[n], tmp) > 0) break; /* emitted positions are never terminal */
+        }
+    }
+    return n;
+}
+
+static void fill_cur(RecCur *cur, const Board *b, int reps)
+{
+    board_bitboards(b, cur->pieces);
+    cur->stm = b->stm;
+    cur->castling = b->castling;
+    cur->ep_square = b->ep;
+    cur->halfmove = (uint8_t)(b->halfmove > 255 ? 255 : b->halfmove);
+    cur->repetitions = (uint8_t)(reps > 255 ? 255 : reps);
+}
+
+static int generate(uint64_t base_seed, int64_t first_index, int count,
+                    int lo_even, int hi_even, int lo_odd, int hi_odd,
+                    void *records_out, int32_t *plies_out, int with_moves)
+{
+    if (count < 0 || !records_out || lo_even < 0 || lo_odd < 0 || hi_even < lo_even ||
+        hi_odd < lo_odd || hi_even >= MAX_PLIES || hi_odd >= MAX_PLIES) return -1;
+    Board *game = (Board *)malloc(sizeof(Board) * (MAX_PLIES + 1));
+    int *reps = (int *)malloc(sizeof(int) * (MAX_PLIES + 1));
+    Move *played = (Move *)malloc(sizeof(Move) * (MAX_PLIES + 1));
+    if (!game || !reps || !played) { free(game); free(reps); free(played); return -1; }
+    for (int i = 0; i < count; ++i) {
+        int n = play_one(base_seed, first_index + i, lo_even, hi_even, lo_odd, hi_odd, game, reps, played);
+        if (with_moves) {
+            RecM8 *rec = &((RecM8 *)records_out)[i];
+            memset(rec, 0, sizeof *rec);
+            fill_cur(&rec->cur, &game[n], reps[n]);
+            int nm = n < 8 ? n : 8;
+            rec->n_moves = (uint8_t)nm;
+            for (int t = 0; t < nm; ++t) {
+                rec->move_from[t] = played[n - 1 - t].from;
+                rec->move_to[t] = played[n - 1 - t].to;
+            }
+        } else {
+            RecH8 *rec = &((RecH8 *)records_out)[i];
+            memset(rec, 0, sizeof *rec);
+            fill_cur(&rec->cur, &game[n], reps[n]);
+            int nh = n < 7 ? n : 7;
+            rec->n_hist = (uint8_t)nh;
+            for (int t = 1; t <= nh; ++t) {
+                board_bitboards(&game[n - t], rec->hist_pieces[t - 1]);
+                rec->hist_rep[t - 1] = (uint8_t)(reps[n - t] > 255 ? 255 : reps[n - t]);
+            }
+        }
+        if (plies_out) plies_out[i] = n;
+    }
+    free(game); free(reps); free(played);
+    return 0;
+}
+
 int azgen_positions(uint64_t base_seed, int64_t first_index, int count,
                     int lo_even, int hi_even, int lo_odd, int hi_odd,
                     void *records_out, int32_t *plies_out)
 {
-    if (count < 0 || !records_out || lo_even < 0 || lo_odd < 0 || hi_even < lo_even ||
-        hi_odd < lo_odd || hi_even >= MAX_PLIES || hi_odd >= MAX_PLIES) return -1;
-    RecH8 *out = (RecH8 *)records_out;
-    Board *game = (Board *)malloc(sizeof(Board) * (MAX_PLIES + 1));
-    int *reps = (int *)malloc(sizeof(int) * (MAX_PLIES + 1));
-    if (!game || !reps) { free(game); free(reps); return -1; }
-    for (int i = 0; i < count; ++i) {
-        int64_t index = first_index + i;
-        Rng rng; rng_seed(&rng, base_seed ^ (uint64_t)index);
-        int lo = (index & 1) ? lo_odd : lo_even, hi = (index & 1) ? hi_odd : hi_even;
-        int n;
-        for (;;) {
-            n = lo + (int)(rng_next(&rng) % (uint64_t)(hi - lo + 1));
-            board_start(&game[0]); reps[0] = 0;
-            int ply = 0, ok = 1;
-            Move list[256];
-            for (; ply < n; ++ply) {
-                int k = legal_moves(&game[ply], list);
-                if (k == 0) { ok = 0; break; }
-                qsort(list, (size_t)k, sizeof(Move), cmp_move);
-                Move m = list[rng_next(&rng) % (uint64_t)k];
-                game[ply + 1] = game[ply];
-                make_move(&game[ply + 1], m);
-                int r = 0;
-                for (int j = 0; j <= ply; ++j) r += same_position(&game[j], &game[ply + 1]);
-                reps[ply + 1] = r;
-            }
-            if (ok) {
-                Move tmp[256];
-                if (legal_moves(&game[n], tmp) > 0) break; /* emitted positions are never terminal */
-            }
-        }
-        RecH8 *rec = &out[i];
-        memset(rec, 0, sizeof *rec);
-        board_bitboards(&game[n], rec->cur.pieces);
-        rec->cur.stm = game[n].stm;
-        rec->cur.castling = game[n].castling;
-        rec->cur.ep_square = game[n].ep;
-        rec->cur.halfmove = (uint8_t)(game[n].halfmove > 255 ? 255 : game[n].halfmove);
-        rec->cur.repetitions = (uint8_t)(reps[n] > 255 ? 255 : reps[n]);
-        int nh = n < 7 ? n : 7;
-        rec->n_hist = (uint8_t)nh;
-        for (int t = 1; t <= nh; ++t) {
-            board_bitboards(&game[n - t], rec->hist_pieces[t - 1]);
-            rec->hist_rep[t - 1] = (uint8_t)(reps[n - t] > 255 ? 255 : reps[n - t]);
-        }
-        if (plies_out) plies_out[i] = n;
-    }
-    free(game); free(reps);
-    return 0;
+    return generate(base_seed, first_index, count, lo_even, hi_even, lo_odd, hi_odd, records_out, plies_out, 0);
+}
+
+/* The same positions (same seeds, same playouts) as 128-byte records with the last eight moves. */
+int azgen_positions_moves(uint64_t base_seed, int64_t first_index, int count,
+                          int lo_even, int hi_even, int lo_odd, int hi_odd,
+                          void *records_out, int32_t *plies_out)
+{
+    return generate(base_seed, first_index, count, lo_even, hi_even, lo_odd, hi_odd, records_out, plies_out, 1);
 }
 
 /* Legal moves of one 104-byte position record, sorted by (from, to, promotion);
@@ -353,3 +402,4 @@ int azgen_legal_moves(const void *record, uint8_t *moves_out)
 }
 
 int azgen_record_bytes(void) { return (int)sizeof(RecH8); }
+int azgen_move_record_bytes(void) { return (int)sizeof(RecM8); }

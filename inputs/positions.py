@@ -23,7 +23,12 @@ H8_DTYPE = np.dtype([
     ("hist_rep", "u1", (7,)),
     ("n_hist", "u1"),
 ])
-assert CUR_DTYPE.itemsize == 104 and H8_DTYPE.itemsize == 784
+M8_DTYPE = np.dtype([
+    ("cur", CUR_DTYPE),
+    ("move_from", "u1", (8,)), ("move_to", "u1", (8,)),
+    ("n_moves", "u1"), ("pad", "u1", (7,)),
+])
+assert CUR_DTYPE.itemsize == 104 and H8_DTYPE.itemsize == 784 and M8_DTYPE.itemsize == 128
 
 _lib = None
 
@@ -38,6 +43,9 @@ def _load():
         lib.azgen_positions.argtypes = [ctypes.c_uint64, ctypes.c_int64, ctypes.c_int,
                                         ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                         ctypes.c_void_p, ctypes.c_void_p]
+        lib.azgen_positions_moves.restype = ctypes.c_int
+        lib.azgen_positions_moves.argtypes = lib.azgen_positions.argtypes
+        assert lib.azgen_move_record_bytes() == M8_DTYPE.itemsize
         lib.azgen_legal_moves.restype = ctypes.c_int
         lib.azgen_legal_moves.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
         assert lib.azgen_record_bytes() == H8_DTYPE.itemsize
@@ -60,6 +68,19 @@ def generate(seed: int, count: int, plies_even=(0, 80), plies_odd=None, first_in
                                  plies_odd[0], plies_odd[1], rec.ctypes.data, plies.ctypes.data)
     if rc != 0:
         raise ValueError("azgen_positions rejected its arguments")
+    return rec, plies
+
+
+def generate_moves(seed: int, count: int, plies_even=(0, 80), plies_odd=None, first_index: int = 0):
+    """The same positions as `generate`, as 128-byte records with the last eight moves (most recent
+    first, castling as the king's own move) instead of the last seven boards."""
+    plies_odd = plies_odd or plies_even
+    rec = np.zeros(count, dtype=M8_DTYPE)
+    plies = np.zeros(count, dtype=np.int32)
+    rc = _load().azgen_positions_moves(seed, first_index, count, plies_even[0], plies_even[1],
+                                       plies_odd[0], plies_odd[1], rec.ctypes.data, plies.ctypes.data)
+    if rc != 0:
+        raise ValueError("azgen_positions_moves rejected its arguments")
     return rec, plies
 
 

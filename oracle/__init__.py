@@ -62,6 +62,8 @@ def _load():
         lib.orc_legal_masks.argtypes = [vp, ci, ci, ci, vp]
         lib.orc_encode.restype = ci
         lib.orc_encode.argtypes = [vp, ci, ci, ci, vp]
+        lib.orc_encode52.restype = ci
+        lib.orc_encode52.argtypes = [vp, ci, ci, vp]
         lib.orc_conv3x3.restype = None
         lib.orc_conv3x3.argtypes = [vp, vp, ci, ci, vp]
         lib.orc_masked_softmax.restype = None
@@ -121,6 +123,17 @@ def encode(records, in_planes: int) -> np.ndarray:
     planes = np.zeros((n, in_planes, 8, 8), dtype=np.float64)
     if _load().orc_encode(rec.ctypes.data, stride, n, in_planes, planes.ctypes.data) != 0:
         raise ValueError("unsupported plane count")
+    return planes
+
+
+def encode52(records) -> np.ndarray:
+    """float64 [n][52][8][8]: the input planes of the paper's network (App. D.1, Table D.1) from
+    128-byte records that carry the last eight moves."""
+    rec, stride, n = _records(records)
+    if stride != 128:
+        raise ValueError("the 52-plane encoding needs 128-byte records with the last eight moves")
+    planes = np.zeros((n, 52, 8, 8), dtype=np.float64)
+    _load().orc_encode52(rec.ctypes.data, stride, n, planes.ctypes.data)
     return planes
 
 

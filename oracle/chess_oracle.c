@@ -408,3 +408,99 @@ int orc_encode(const void *records, int stride, int n, int in_planes, double *pl
     }
     return 0;
 }
+
+/* ---- the 52 input planes of the paper's network (App. D.1, Table D.1) -----------------------
+ * records: 128-byte records = the 104-byte position, then move_from[8], move_to[8] (absolute
+ * squares, most recent move first, castling as the king's own move), n_moves, padding.
+ * planes_out: [n][52][64] doubles in mover orientation (Black to move: ranks reflected, colours
+ * exchanged, files kept; row 0 = the mover's home rank, column 0 = file a).
+ *   0-5 own P N B R Q K, 6-11 opponent's; 12-15 castling rights own K-side, own Q-side, opponent
+ *   K-side, opponent Q-side; 16 all own pieces, 17 all opponent pieces; 18 the opponent pieces
+ *   that give check; 19 the en-passant target square; 20 / 21 one iff the position occurred at
+ *   least once / twice before; 22+2t, 23+2t origin and destination of the move t plies back
+ *   (t = 0..7, zero where the game is shorter); 38 checkerboard fixed in these coordinates, the
+ *   a1 corner (row 0, column 0) set; 39 one iff each side has exactly one bishop and the two stand
+ *   on squares of different colour; 40-45 own minus opponent count of P N B R Q K; 46 halfmove
+ *   clock capped at 100, as a count; 47-51 own count of P N B R Q.
+ * Readings where the table is silent: plane 19 is set whenever the record carries an en-passant
+ * square (the square behind a pawn that has just advanced two ranks), whether or not a capture
+ * there is legal; counts and the clock are plain integers, not normalised. */
+typedef struct {
+    PosRecord cur;
+    uint8_t move_from[8], move_to[8];
+    uint8_t n_moves;
+    uint8_t pad[7];
+} PosRecordM8;                    /* 128 bytes */
+
+static int popcount64(uint64_t v) { int n = 0; while (v) { v &= v - 1; ++n; } return n; }
+
+int orc_encode52(const void *records, int stride, int n, double *planes_out) {
+    for (int i = 0; i < n; ++i) {
+        const PosRecordM8 *m8 = (const PosRecordM8 *)((const char *)records + (size_t)i * stride);
+        const PosRecord *r = &m8->cur;
+        double *pl = planes_out + (size_t)i * 52 * 64;
+        memset(pl, 0, sizeof(double) * 52 * 64);
+        const int stm = r->stm;
+        const int flip = stm ? 56 : 0;
+        const int ownK = stm ? 4 : 1, ownQ = stm ? 8 : 2, oppK = stm ? 1 : 4, oppQ = stm ? 2 : 8;
+        put_board(pl, 0, r->pieces, stm);
+        if (r->castling & ownK) fill(pl, 12, 1.0);
+        if (r->castling & ownQ) fill(pl, 13, 1.0);
+        if (r->castling & oppK) fill(pl, 14, 1.0);
+        if (r->castling & oppQ) fill(pl, 15, 1.0);
+        for (int k = 0; k < 6; ++k)
+            for (int s = 0; s < 64; ++s) {
+                if (pl[k * 64 + s] != 0.0) pl[16 * 64 + s] = 1.0;
+                if (pl[(6 + k) * 64 + s] != 0.0) pl[17 * 64 + s] = 1.0;
+            }
+        /* checkers: walk from the mover's king outwards and see which enemy piece looks back */
+        {
+            MBoard b; load_record(r, &b);
+            const int km = find_king(&b, stm);
+            const int eb = stm ? 0 : 6;        /* enemy piece codes eb+1 .. eb+6 */
+            if (km) {
+                /* an enemy pawn checks from the two squares diagonally in front of the king (seen from the mover) */
+                const int fwd = stm ? -10 : 10;
+                for (int d = -1; d <= 1; d += 2)
+                    if (b.sq[km + fwd + d] == eb + 1) pl[18 * 64 + (sq64(km + fwd + d) ^ flip)] = 1.0;
+                for (int j = 0; j < 8; ++j)
+                    if (b.sq[km + N_OFF[j]] == eb + 2) pl[18 * 64 + (sq64(km + N_OFF[j]) ^ flip)] = 1.0;
+                for (int j = 0; j < 4; ++j) {
+                    int t = km + B_OFF[j];
+                    while (b.sq[t] == EMPTY) t += B_OFF[j];
+                    if (b.sq[t] == eb + 3 || b.sq[t] == eb + 5) pl[18 * 64 + (sq64(t) ^ flip)] = 1.0;
+                    t = km + R_OFF[j];
+                    while (b.sq[t] == EMPTY) t += R_OFF[j];
+                    if (b.sq[t] == eb + 4 || b.sq[t] == eb + 5) pl[18 * 64 + (sq64(t) ^ flip)] = 1.0;
+                }
+            }
+        }
+        if (r->ep_square < 64) pl[19 * 64 + (r->ep_square ^ flip)] = 1.0;
+        if (r->repetitions >= 1) fill(pl, 20, 1.0);
+        if (r->repetitions >= 2) fill(pl, 21, 1.0);
+        for (int t = 0; t < 8 && t < m8->n_moves; ++t) {
+            pl[(22 + 2 * t) * 64 + (m8->move_from[t] ^ flip)] = 1.0;
+            pl[(23 + 2 * t) * 64 + (m8->move_to[t] ^ flip)] = 1.0;
+        }
+        for (int row = 0; row < 8; ++row)
+            for (int col = 0; col < 8; ++col)
+                if (((row + col) & 1) == 0) pl[38 * 64 + row * 8 + col] = 1.0;
+        int own_n[6], opp_n[6];
+        for (int k = 0; k < 6; ++k) {
+            own_n[k] = popcount64(r->pieces[(stm ? 6 : 0) + k]);
+            opp_n[k] = popcount64(r->pieces[(stm ? 0 : 6) + k]);
+        }
+        if (own_n[2] == 1 && opp_n[2] == 1) {
+            int a = 0, c = 0;
+            for (int s = 0; s < 64; ++s) {
+                if ((r->pieces[(stm ? 6 : 0) + 2] >> s) & 1ULL) a = ((s & 7) + (s >> 3)) & 1;
+                if ((r->pieces[(stm ? 0 : 6) + 2] >> s) & 1ULL) c = ((s & 7) + (s >> 3)) & 1;
+            }
+            if (a != c) fill(pl, 39, 1.0);
+        }
+        for (int k = 0; k < 6; ++k) fill(pl, 40 + k, (double)(own_n[k] - opp_n[k]));
+        fill(pl, 46, (double)(r->halfmove > 100 ? 100 : r->halfmove));
+        for (int k = 0; k < 5; ++k) fill(pl, 47 + k, (double)own_n[k]);
+    }
+    return 0;
+}
