@@ -159,6 +159,25 @@ int az_evaluate_host(az_net *net, const void *positions_host, const uint64_t *le
                      int batch, float *policy_host, float *value_host, void *cuda_stream);
 
 /*
+ * The encoder of the paper's own network (App. D.1, Table D.1: 52 planes).  positions_dev holds
+ * 128-byte records: the 104-byte az_position, then move_from[8] and move_to[8] (absolute squares of
+ * the last eight moves, most recent first, castling as the king's own move), n_moves (0..8) and
+ * seven bytes of padding.  planes_dev receives [batch][64][64] float32 (bf16 == 0) or bfloat16:
+ * square-major in the mover's orientation (Black to move: ranks reflected, colours exchanged,
+ * files kept), channel c of the table at index c, channels 52..63 zero.
+ *   0-5 own P N B R Q K, 6-11 opponent's; 12-15 castling rights own K-side, own Q-side, opponent
+ *   K-side, opponent Q-side; 16, 17 all own / all opponent pieces; 18 the pieces that give check;
+ *   19 the en-passant target square (set whenever the record carries one); 20, 21 one iff the
+ *   position occurred at least once / twice before; 22+2t, 23+2t origin and destination of the
+ *   move t plies back; 38 a checkerboard fixed in tensor coordinates with corner (0,0) set; 39 one
+ *   iff each side has exactly one bishop and they stand on different colours; 40-45 own minus
+ *   opponent count of P N B R Q K; 46 halfmove clock capped at 100 (a count, not normalised);
+ *   47-51 own count of P N B R Q.  Every value is an integer that both output types hold exactly.
+ * No az_net is involved.  Errors: BAD_ARG (null or misaligned pointer: positions 8, planes 16), CUDA.
+ */
+int az_encode52(const void *positions_dev, int batch, int bf16, void *planes_dev, void *cuda_stream);
+
+/*
  * Pipelined host entry (Sec. 5.2: double-buffered staging, asynchronous copies and completion
  * events, so that the copies of one batch overlap the evaluation of the next).  az_submit_host
  * queues one evaluation and returns at once with a ticket; az_wait_host blocks until that

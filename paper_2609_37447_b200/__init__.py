@@ -24,7 +24,7 @@ AZ_VALUE_TANH, AZ_VALUE_WDL = 0, 1
 AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3 = 0, 1, 2
 
 EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
-           "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_submit_host", "az_wait_host", "az_encode", "az_tower", "az_tower_static", "az_legal_masks",
+           "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_submit_host", "az_wait_host", "az_encode", "az_encode52", "az_tower", "az_tower_static", "az_legal_masks",
            "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error")
 
@@ -73,6 +73,8 @@ def _load_library():
     lib.az_tower_time.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ci)]
     lib.az_encode.restype = ci
     lib.az_encode.argtypes = [vp, vp, ci, vp, vp]
+    lib.az_encode52.restype = ci
+    lib.az_encode52.argtypes = [vp, ci, ci, vp, vp]
     lib.az_tower.restype = ci
     lib.az_tower.argtypes = [vp, vp, ci, vp, vp]
     lib.az_tower_static.restype = ci
@@ -232,6 +234,15 @@ def az_tower_time(net: Net):
 def az_encode(net: Net, positions_dev, batch, planes_dev, stream=None):
     _check(_lib.az_encode(net.handle, _dev_ptr(positions_dev, "positions"), batch, _dev_ptr(planes_dev, "planes"),
                           _stream_ptr(stream)), "az_encode")
+
+
+def az_encode52(positions_dev, batch, planes_dev, stream=None):
+    """128-byte move-history records -> [batch][64][64] planes (float32 or bfloat16 by the tensor's dtype)."""
+    bf16 = 1 if planes_dev.dtype == torch.bfloat16 else 0
+    if not bf16 and planes_dev.dtype != torch.float32:
+        raise TypeError("planes must be float32 or bfloat16")
+    _check(_lib.az_encode52(_dev_ptr(positions_dev, "positions"), batch, bf16, _dev_ptr(planes_dev, "planes"),
+                            _stream_ptr(stream)), "az_encode52")
 
 
 def az_tower(net: Net, positions_dev, batch, tower_dev, stream=None):

@@ -349,6 +349,12 @@ int az_encode(az_net *net, const void *positions_dev, int batch, void *planes_de
                              n->in_pad, n->bf16, planes_dev, n->status_dev, static_cast<cudaStream_t>(cuda_stream));
 }
 
+int az_encode52(const void *positions_dev, int batch, int bf16, void *planes_dev, void *cuda_stream) {
+    if (batch < 0 || (batch > 0 && (!positions_dev || !planes_dev))) return AZ_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(positions_dev) & 7) || (reinterpret_cast<uintptr_t>(planes_dev) & 15)) return AZ_ERR_BAD_ARG;
+    return az::launch_encode52(positions_dev, batch, bf16 != 0, planes_dev, static_cast<cudaStream_t>(cuda_stream));
+}
+
 int az_tower(az_net *net, const void *positions_dev, int batch, void *tower_dev, void *cuda_stream) {
     Net *n = reinterpret_cast<Net *>(net);
     if (!n || batch < 0 || (batch > 0 && (!positions_dev || !tower_dev))) return AZ_ERR_BAD_ARG;

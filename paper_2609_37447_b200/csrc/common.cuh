@@ -137,6 +137,7 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 }
 
 // ---- kernels' launch functions (each returns AZ_OK or AZ_ERR_CUDA) ---------------------------
+int launch_encode52(const void *positions, int batch, bool bf16, void *planes, cudaStream_t s);
 int launch_encode(const void *positions, size_t stride, int batch, int in_planes, int in_pad,
                   bool bf16, void *planes, uint32_t *status, cudaStream_t s);
 int launch_legal_masks(const void *positions, size_t stride, int batch, int head, uint64_t *masks,
