@@ -15,7 +15,7 @@ import subprocess
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SOURCES = ("chess_oracle.c", "net_oracle.c")
+_SOURCES = ("chess_oracle.c", "net_oracle.c", "pnet_oracle.c")
 _lib = None
 
 
@@ -64,6 +64,8 @@ def _load():
         lib.orc_encode.argtypes = [vp, ci, ci, ci, vp]
         lib.orc_encode52.restype = ci
         lib.orc_encode52.argtypes = [vp, ci, ci, vp]
+        lib.orc_pnet_forward.restype = ci
+        lib.orc_pnet_forward.argtypes = [vp, ctypes.c_size_t, vp, vp, ci, vp, vp, vp, vp]
         lib.orc_conv3x3.restype = None
         lib.orc_conv3x3.argtypes = [vp, vp, ci, ci, vp]
         lib.orc_masked_softmax.restype = None
@@ -76,7 +78,7 @@ def _load():
 
 
 POLICY_SIZE = {0: 73 * 64, 1: 1858}
-MASK_WORDS = {0: 73, 1: 30}
+MASK_WORDS = {0: 73, 1: 30, 2: 30}
 
 
 def _records(records):
@@ -106,7 +108,8 @@ def policy_index(head: int, stm: int, frm: int, to: int, promo: int = 0, castle:
 
 
 def legal_masks(records, head: int) -> np.ndarray:
-    """uint64 [n][73 or 30]: bit (i & 63) of word (i >> 6) set iff policy index i is legal."""
+    """uint64 [n][73 or 30]: bit (i & 63) of word (i >> 6) set iff policy index i is legal.
+    head 0: 73 move planes, 1: flat 1,858 list, 2: the paper's 1,880 actions (30 words)."""
     rec, stride, n = _records(records)
     masks = np.zeros((n, MASK_WORDS[head]), dtype=np.uint64)
     rc = _load().orc_legal_masks(rec.ctypes.data, stride, n, head, masks.ctypes.data)
@@ -135,6 +138,37 @@ def encode52(records) -> np.ndarray:
     planes = np.zeros((n, 52, 8, 8), dtype=np.float64)
     _load().orc_encode52(rec.ctypes.data, stride, n, planes.ctypes.data)
     return planes
+
+
+def pnet_forward(blob: np.ndarray, planes: np.ndarray, masks: np.ndarray, want_raw=False, want_tower=False):
+    """The paper's network on encoded planes [n][52][8][8] and 1,880-action masks [n][30]:
+    (policy [n][1880], value [n][3] win/draw/loss) and, on request, a dict with the raw policy
+    logits and the backbone's output [n][C][8][8]."""
+    b = np.ascontiguousarray(blob, dtype=np.uint8)
+    pl = np.ascontiguousarray(planes, dtype=np.float64)
+    mk = np.ascontiguousarray(masks, dtype=np.uint64)
+    n = pl.shape[0]
+    channels = int(np.frombuffer(b[16:20].tobytes(), dtype="<u4")[0])
+    policy = np.zeros((n, 1880), dtype=np.float64)
+    value = np.zeros((n, 3), dtype=np.float64)
+    raw = np.zeros((n, 1880), dtype=np.float64) if want_raw else None
+    tower = np.zeros((n, channels, 8, 8), dtype=np.float64) if want_tower else None
+    rc = _load().orc_pnet_forward(b.ctypes.data, b.size, pl.ctypes.data, mk.ctypes.data, n, policy.ctypes.data,
+                                  value.ctypes.data, raw.ctypes.data if want_raw else None,
+                                  tower.ctypes.data if want_tower else None)
+    if rc != 0:
+        raise ValueError("malformed network blob")
+    if want_raw or want_tower:
+        return policy, value, {"logits": raw, "tower": tower}
+    return policy, value
+
+
+def pnet_evaluate(blob: np.ndarray, records, **kw):
+    """Records with the last eight moves -> (masks, planes, policy, value[, extras]) of the paper's network."""
+    masks = legal_masks(np.ascontiguousarray(records["cur"]), 2)
+    planes = encode52(records)
+    out = pnet_forward(blob, planes, masks, **kw)
+    return (masks, planes) + tuple(out)
 
 
 def conv3x3(weight: np.ndarray, x: np.ndarray) -> np.ndarray:

@@ -312,16 +312,39 @@ static int index_flat(int from, int to, int promo) {
 
 int orc_flat_count(void) { if (!flat_ready) build_flat(); return flat_count; }
 
+/* The paper's own action list (Sec. 3.2, App. D.1): the same 1,792 origin-destination pairs, in
+ * the same order, then 88 explicit promotions: origins on the seventh rank ascending, destinations
+ * origin+7, +8, +9 that stay on the board ascending, pieces in the order queen, rook, bishop,
+ * knight (22 x 4).  A promoting pawn move has ONLY its promotion action; the plain pair of the
+ * same two squares belongs to the other pieces that can make that step. */
+static int index_fromto(int from, int to, int promo) {
+    if (!flat_ready) build_flat();
+    if (promo >= 1 && promo <= 4) {
+        int step = (to & 7) - (from & 7);
+        if ((from >> 3) != 6 || (to >> 3) != 7 || step < -1 || step > 1) return -1;
+        int slot = 0;                       /* how many (file, step) combinations come before this one */
+        for (int file = 0; file < 8; ++file)
+            for (int st = -1; st <= 1; ++st) {
+                if (file + st < 0 || file + st > 7) continue;
+                if (file == (from & 7) && st == step) return 1792 + 4 * slot + (4 - promo);
+                ++slot;
+            }
+        return -1;
+    }
+    return flat_pair[from][to];
+}
+
 /* Policy index of a move given in ABSOLUTE squares for the side `stm`; `castle` 0 none,
  * 1 short, 2 long.  Returns -1 if the move has no index. */
 int orc_policy_index(int head, int stm, int from, int to, int promo, int castle) {
     if (castle) to = (stm ? 56 : 0) + (castle == 1 ? 7 : 0);   /* king takes the own-rook square */
     if (stm) { from ^= 56; to ^= 56; }                          /* reflect ranks for Black */
-    return head == 0 ? index73(from, to, promo) : index_flat(from, to, promo);
+    return head == 0 ? index73(from, to, promo) : head == 1 ? index_flat(from, to, promo) : index_fromto(from, to, promo);
 }
 
 /* Legal-move masks: bit (i & 63) of word (i >> 6) is set iff policy index i is a legal move.
- * words = 73 (head 0) or 30 (head 1) per position.  Returns 0, or -1 if a move had no index. */
+ * words = 73 (head 0) or 30 (head 1: 1,858 moves; head 2: the paper's 1,880 actions) per position.
+ * Returns 0, or -1 if a move had no index. */
 int orc_legal_masks(const void *records, int stride, int n, int head, uint64_t *masks) {
     int words = head == 0 ? 73 : 30, bad = 0;
     for (int i = 0; i < n; ++i) {

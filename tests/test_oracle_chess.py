@@ -150,6 +150,39 @@ def test_index_maps_are_injective(head, size):
         assert plain == sorted(plain) and plain == list(range(1792))   # (from, to) ascending order
 
 
+def test_the_papers_1880_action_list():
+    # Sec. 3.2 / App. D.1: 1,792 ray-or-knight pairs plus 88 promotions with four pieces each
+    moves = [m for m in geometric_moves() if m[2] == 0]
+    promos = [(f, t, p) for f in range(48, 56) for t in (f + 7, f + 8, f + 9)
+              if abs((t & 7) - (f & 7)) <= 1 and t < 64 for p in (4, 3, 2, 1)]      # queen, rook, bishop, knight
+    assert len(moves) == 1792 and len(promos) == 88
+    idx = [oracle.policy_index(2, 0, f, t, p, 0) for f, t, p in moves + promos]
+    assert idx == list(range(1880))                   # this very order, no gaps, nothing twice
+    # plain pairs are numbered as in the 1,858 list
+    assert [oracle.policy_index(1, 0, f, t, 0, 0) for f, t, _ in moves] == idx[:1792]
+    # by hand: a7-a8=Q is the first promotion action, h7-h8=N the last; b7xa8=R: a-file has 2 combinations
+    assert oracle.policy_index(2, 0, sq("a7"), sq("a8"), 4, 0) == 1792
+    assert oracle.policy_index(2, 0, sq("h7"), sq("h8"), 1, 0) == 1879
+    assert oracle.policy_index(2, 0, sq("b7"), sq("a8"), 3, 0) == 1792 + 4 * 2 + 1
+    # Black's promotion is the mover's promotion; a promotion from anywhere else has no action
+    assert oracle.policy_index(2, 1, sq("a2"), sq("a1"), 4, 0) == 1792
+    assert oracle.policy_index(2, 0, sq("a6"), sq("a7"), 4, 0) == -1
+    # masks: one bit per legal move, promotions on their own actions and not on the plain pair
+    rec, _ = positions.generate(23, 1200, (0, 200))
+    cur = positions.cur_records(rec)
+    m2 = oracle.legal_masks(cur, 2)
+    n = np.array([len(oracle.legal_moves(cur[i])) for i in range(cur.shape[0])])
+    assert (popcounts(m2) == n).all()
+    promo_rec = positions.record_from_fen("1r2k3/P7/8/8/8/8/8/4K3 w - - 0 1")
+    bits = mask_bits(oracle.legal_masks(promo_rec, 2)[0], 1920)
+    assert not bits[1880:].any()
+    for to in ("a8", "b8"):
+        for piece in (1, 2, 3, 4):
+            assert bits[oracle.policy_index(2, 0, sq("a7"), sq(to), piece, 0)]
+        assert not bits[oracle.policy_index(2, 0, sq("a7"), sq(to), 0, 0)]
+    assert bits.sum() == len(oracle.legal_moves(promo_rec)) == 8 + 5
+
+
 def test_index_73_plane_examples_by_hand():
     # plane = 7*direction + distance-1 with directions N, NE, E, SE, S, SW, W, NW; index = plane*64 + from
     assert oracle.policy_index(0, 0, sq("e2"), sq("e4"), 0, 0) == (7 * 0 + 1) * 64 + sq("e2")
