@@ -47,12 +47,14 @@ enum {
     AZ_ERR_BUSY = -9              /* az_submit_host: both in-flight slots are taken (az_wait_host first) */
 };
 
-enum { AZ_POLICY_PLANES73 = 0, AZ_POLICY_FLAT1858 = 1 };
+enum { AZ_POLICY_PLANES73 = 0, AZ_POLICY_FLAT1858 = 1, AZ_POLICY_FROMTO1880 = 2 };
 enum { AZ_VALUE_TANH = 0, AZ_VALUE_WDL = 1 };
 enum { AZ_PREC_FP32 = 0, AZ_PREC_BF16 = 1, AZ_PREC_FP8_E4M3 = 2 };
 
 /* Network shape.  in_planes 19 or 112; blocks >= 0 residual blocks of `channels` channels
- * (a multiple of 16); heads and precision as the enums above; max_batch sizes the workspace. */
+ * (a multiple of 16); heads and precision as the enums above; max_batch sizes the workspace.
+ * in_planes 52 selects the paper's own network (Sec. 3.2, 4.3, App. D.1): it goes with
+ * policy_head AZ_POLICY_FROMTO1880 and value_head AZ_VALUE_WDL, see az_load_net. */
 typedef struct {
     uint32_t abi_version;   /* AZ_ABI_VERSION */
     uint32_t in_planes;
@@ -87,14 +89,25 @@ typedef struct {
     uint8_t n_hist;
 } az_position_h8;
 
+/* Position with the last eight moves (128 bytes); consumed by the paper's 52-plane network.
+ * move_from[t] / move_to[t]: absolute squares of the move t plies back (castling as the king's own
+ * move), n_moves (0..8) says how many are present. */
+typedef struct {
+    az_position cur;
+    uint8_t move_from[8];
+    uint8_t move_to[8];
+    uint8_t n_moves;
+    uint8_t pad[7];
+} az_position_m8;
+
 typedef struct az_net az_net;
 
 /* Size in bytes of one position record / of one position's outputs for a given arch. */
-size_t az_position_bytes(const az_arch *arch);      /* 104 (19 planes) or 784 (112 planes) */
-size_t az_policy_size(const az_arch *arch);         /* 4672 or 1858 floats per position */
+size_t az_position_bytes(const az_arch *arch);      /* 104 (19 planes), 784 (112 planes) or 128 (52 planes) */
+size_t az_policy_size(const az_arch *arch);         /* 4672, 1858 or 1880 floats per position */
 size_t az_mask_words(const az_arch *arch);          /* 73 or 30 uint64 words per position */
 size_t az_value_size(const az_arch *arch);          /* 1 or 3 floats per position */
-size_t az_plane_channels(const az_arch *arch);      /* channels of the encoded plane tensor: 32 or 128 */
+size_t az_plane_channels(const az_arch *arch);      /* channels of the encoded plane tensor: 32, 128 or 64 */
 
 /*
  * load_net(weights, arch)  (Sec. 3.3 publication hands the actors a network; Sec. 4.3.6 and
@@ -109,7 +122,26 @@ size_t az_plane_channels(const az_arch *arch);      /* channels of the encoded p
  * Convolution weights are [out][in][ky][kx]; "scale/bias" are the folded batch-norm
  * (y = scale*conv + bias).  Fully-connected inputs are flattened channel-major (c*64 + square).
  * The blob is copied; the caller may free it on return.  On success *out receives the network.
- * Errors: BAD_ARG, BAD_ARCH, BAD_WEIGHTS, CUDA.
+ *
+ * The paper's own network (arch.in_planes == 52; Sec. 3.2, 4.3.3, 4.3.6, App. D.1): input planes as
+ * az_encode52; scaled post-activation blocks, act(z) = min(max(z, 0), 6), the branch scale
+ * 1/sqrt(blocks) already folded into scale2 / bias2; in blocks 1, 3, 5, ... the last C/4 output
+ * channels of the first convolution are activated, averaged and maximised over the board, mapped
+ * (means first, then maxima) by gw to 3C/4 values that are added to the other channels before their
+ * activation, and the second convolution reads those 3C/4 channels only; policy = tokens (1x1
+ * convolution with bias, no activation), queries and keys (linear maps of the token), score
+ * q_origin . k_destination / sqrt(128) for the 1,792 pair actions, plus an offset (linear map of the
+ * origin's token, one per piece: queen, rook, bishop, knight) for the 88 promotion actions, which
+ * follow the pairs: origins on the seventh rank ascending, destinations origin+7, +8, +9 on the board,
+ * then the piece; a promoting pawn move has only its promotion actions; value = 2-channel 1x1
+ * convolution, folded normalisation, ReLU, 48 hidden units with ReLU, three logits, softmax.
+ * Blob: 64-byte header ("AZPNET1\0", uint32 version = 1, blocks, channels, 128, 2, 48, tensor count),
+ * then in.w[C][52][3][3] in.scale in.bias; per block w1[C][C][3][3] scale1 bias1, (odd blocks)
+ * gw[3C/4][C/2], w2[C][C or 3C/4][3][3] scale2 bias2; t.w[128][C] t.b; q.w[128][128] q.b; k.w k.b;
+ * o.w[4][128] o.b; v.cw[2][C] v.cscale v.cbias; v.w1[48][128] v.b1; v.w2[3][48] v.b2.
+ * Built for channels == 128 in bf16 (AZ_ERR_UNSUPPORTED otherwise); az_evaluate_legal and the
+ * FP8 / fp32 precisions are not available for it.
+ * Errors: BAD_ARG, BAD_ARCH, BAD_WEIGHTS, UNSUPPORTED, CUDA.
  */
 int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az_net **out);
 
@@ -258,7 +290,10 @@ int az_tower_static(az_net *net, const void *positions_dev, int batch, void *tow
  *   flat1858: every (origin, destination) a queen ray or knight jump apart, origin ascending then
  *     destination ascending (1792), then for origins on the seventh rank the destinations
  *     origin+7,+8,+9 on the board, each with N,B,R (66).
- * position_stride is the byte distance between records (104 or 784).  No az_net is needed.
+ *   fromto1880 (Sec. 3.2, App. D.1): the same 1792 pairs, then the 88 promotion actions: origins on
+ *     the seventh rank ascending, destinations origin+7,+8,+9 on the board, each with Q,R,B,N; a
+ *     promoting pawn move sets only its four promotion actions, not the plain pair.  30 words.
+ * position_stride is the byte distance between records (104, 784 or 128).  No az_net is needed.
  */
 int az_legal_masks(const void *positions_dev, size_t position_stride, int batch, int policy_head,
                    uint64_t *masks_dev, void *cuda_stream);

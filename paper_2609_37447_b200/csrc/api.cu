@@ -36,9 +36,12 @@ struct HostMaster {                     // fp32 tower parameters of an FP8 net, 
 
 bool arch_ok(const az_arch &a) {
     if (a.abi_version != AZ_ABI_VERSION) return false;
-    if (a.in_planes != 19 && a.in_planes != 112) return false;
+    if (a.in_planes != 19 && a.in_planes != 112 && a.in_planes != 52) return false;
     if (a.blocks > 64 || a.channels < 8 || a.channels > 512 || a.channels % 8) return false;
-    if (a.policy_head > 1 || a.value_head > 1 || a.precision > 2) return false;
+    if (a.policy_head > 2 || a.value_head > 1 || a.precision > 2) return false;
+    // the paper's own network: 52 planes go with the 1,880-action head and the win/draw/loss value, and only with them
+    if ((a.in_planes == 52) != (a.policy_head == AZ_POLICY_FROMTO1880)) return false;
+    if (a.in_planes == 52 && a.value_head != AZ_VALUE_WDL) return false;
     if (a.max_batch == 0 || a.max_batch > (1u << 20)) return false;
     return true;
 }
@@ -265,6 +268,7 @@ void free_net(Net *n) {
     for (cudaStream_t s : n->s_compute) if (s) cudaStreamDestroy(s);
     if (n->s_out) cudaStreamDestroy(n->s_out);
     cudaFree(n->alt_u_policy); cudaFree(n->alt_u_value); cudaFree(n->alt_logits);
+    cudaFree(n->pnet_gw); cudaFree(n->pnet_qk); cudaFree(n->pnet_small); cudaFree(n->pnet_actions);
     if (n->ev_begin) for (int i = 0; i < kMaxProfiledPasses; ++i) { cudaEventDestroy(n->ev_begin[i]); cudaEventDestroy(n->ev_end[i]); }
     delete[] n->ev_begin; delete[] n->ev_end;
     cudaFree(n->logits); cudaFree(n->head_p); cudaFree(n->head_v); cudaFree(n->hidden); cudaFree(n->status_dev);
@@ -277,6 +281,16 @@ int run_tower(Net &n, const void *positions, int batch, void **tower_out, bool f
     int rc = AZ_OK;
     const int C = (int)n.arch.channels;
     const bool timed = n.profile && n.n_events < kMaxProfiledPasses;
+    if (n.pnet) {
+        // the paper's network: its 52 planes come from the stand-alone encoder, the tower reads them
+        rc = launch_encode52(positions, batch, true, n.planes, s);
+        if (rc != AZ_OK) return rc;
+        if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
+        *tower_out = n.act[0];
+        rc = launch_tower_tc(n, n.planes, positions, batch, n.act[0], fused_heads, nullptr, s);
+        if (rc == AZ_OK && timed) AZ_CUDA(cudaEventRecord(n.ev_end[n.n_events++], s));
+        return rc;
+    }
     if (n.tc_ready) {
         // the tensor-core tower encodes its boards itself, straight into shared memory
         if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
@@ -313,26 +327,34 @@ using az::Net;
 
 extern "C" {
 
-size_t az_position_bytes(const az_arch *a) { return a && a->in_planes == 112 ? sizeof(az_position_h8) : sizeof(az_position); }
-size_t az_policy_size(const az_arch *a) { return a && a->policy_head == AZ_POLICY_FLAT1858 ? az::kFlatMoves : az::kPlanes73 * 64; }
-size_t az_mask_words(const az_arch *a) { return a && a->policy_head == AZ_POLICY_FLAT1858 ? 30 : 73; }
+size_t az_position_bytes(const az_arch *a) {
+    return a && a->in_planes == 112 ? sizeof(az_position_h8) : a && a->in_planes == 52 ? sizeof(az_position_m8) : sizeof(az_position);
+}
+size_t az_policy_size(const az_arch *a) {
+    return a && a->policy_head == AZ_POLICY_FLAT1858 ? az::kFlatMoves : a && a->policy_head == AZ_POLICY_FROMTO1880 ? 1880 : az::kPlanes73 * 64;
+}
+size_t az_mask_words(const az_arch *a) { return a && a->policy_head != AZ_POLICY_PLANES73 ? 30 : 73; }
 size_t az_value_size(const az_arch *a) { return a && a->value_head == AZ_VALUE_WDL ? 3 : 1; }
-size_t az_plane_channels(const az_arch *a) { return a && a->in_planes == 112 ? 128 : 32; }
+size_t az_plane_channels(const az_arch *a) { return a && a->in_planes == 112 ? 128 : a && a->in_planes == 52 ? 64 : 32; }
 
 int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az_net **out) {
-    static_assert(sizeof(az_position) == 104 && sizeof(az_position_h8) == 784, "record layout");
+    static_assert(sizeof(az_position) == 104 && sizeof(az_position_h8) == 784 && sizeof(az_position_m8) == 128, "record layout");
     if (!arch || !weights_host || !out) return AZ_ERR_BAD_ARG;
     *out = nullptr;
     if (!az::arch_ok(*arch)) return AZ_ERR_BAD_ARCH;
+    const bool pnet = arch->in_planes == 52;
+    // of the paper's network ladder the 128-channel size is built, in bf16
+    if (pnet && (arch->channels != 128 || arch->precision != AZ_PREC_BF16)) return AZ_ERR_UNSUPPORTED;
     az::BlobView view;
-    int rc = az::parse_blob(*arch, static_cast<const unsigned char *>(weights_host), nbytes, view);
+    int rc = AZ_OK;
+    if (!pnet) rc = az::parse_blob(*arch, static_cast<const unsigned char *>(weights_host), nbytes, view);
     if (rc != AZ_OK) return rc;
     Net *n = new (std::nothrow) Net();
     if (!n) return AZ_ERR_BAD_ARG;
     n->arch = *arch;
     cudaError_t e = cudaGetDevice(&n->device);
     if (e != cudaSuccess) { az::set_cuda_error(e, "cudaGetDevice"); delete n; return AZ_ERR_CUDA; }
-    rc = az::build_net(*n, view);
+    rc = pnet ? az::build_pnet(*n, static_cast<const unsigned char *>(weights_host), nbytes) : az::build_net(*n, view);
     if (rc != AZ_OK) { az::free_net(n); return rc; }
     *out = reinterpret_cast<az_net *>(n);
     return AZ_OK;
@@ -345,6 +367,7 @@ int az_encode(az_net *net, const void *positions_dev, int batch, void *planes_de
     if (!n || batch < 0 || (batch > 0 && (!positions_dev || !planes_dev))) return AZ_ERR_BAD_ARG;
     if ((reinterpret_cast<uintptr_t>(positions_dev) & 7) || (reinterpret_cast<uintptr_t>(planes_dev) & 15)) return AZ_ERR_BAD_ARG;
     if ((uint32_t)batch > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
+    if (n->pnet) return az::launch_encode52(positions_dev, batch, true, planes_dev, static_cast<cudaStream_t>(cuda_stream));
     return az::launch_encode(positions_dev, az_position_bytes(&n->arch), batch, (int)n->arch.in_planes,
                              n->in_pad, n->bf16, planes_dev, n->status_dev, static_cast<cudaStream_t>(cuda_stream));
 }
@@ -391,6 +414,10 @@ static int evaluate_impl(az_net *net, const void *positions_dev, const uint64_t 
     void *h = nullptr;
     int rc = az::run_tower(*n, positions_dev, batch, &h, n->tc_ready, s);
     if (rc != AZ_OK) return rc;
+    if (n->pnet) {
+        if (!dense) return AZ_ERR_UNSUPPORTED;
+        return az::launch_pnet_finish(*n, legal_masks_dev, batch, policy_dev, value_dev, s);
+    }
     if (n->tc_ready) {
         // the tower kernel has produced the 73-plane logits or the flat head's projection, and the value
         // projection; one GEMM launch finishes both heads, the softmax follows
@@ -511,7 +538,7 @@ int az_submit_host(az_net *net, const void *positions_host, const uint64_t *lega
         // The tensor-core path keeps nothing else between its kernels than the head GEMM's operands and
         // the logits; with a second copy of those, odd slots run on a stream of their own.  The other
         // paths share one workspace, so all their slots take turns on one stream.
-        if (n->tc_ready) {
+        if (n->tc_ready && !n->pnet) {
             const size_t u_bytes = (size_t)((a.max_batch + 127) / 128) * az::kHeadChannels * 64 * 128 * sizeof(__nv_bfloat16);
             AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute[1], cudaStreamNonBlocking));
             AZ_CUDA(cudaMalloc(&n->alt_u_value, u_bytes));
@@ -609,7 +636,7 @@ int az_tower_time(az_net *net, float *total_ms_out, int *passes_out) {
 
 int az_legal_masks(const void *positions_dev, size_t position_stride, int batch, int policy_head,
                    uint64_t *masks_dev, void *cuda_stream) {
-    if (batch < 0 || (policy_head != AZ_POLICY_PLANES73 && policy_head != AZ_POLICY_FLAT1858)) return AZ_ERR_BAD_ARG;
+    if (batch < 0 || policy_head < AZ_POLICY_PLANES73 || policy_head > AZ_POLICY_FROMTO1880) return AZ_ERR_BAD_ARG;
     if (batch == 0) return AZ_OK;
     if (!positions_dev || !masks_dev || position_stride < sizeof(az_position) || (position_stride & 7)) return AZ_ERR_BAD_ARG;
     if ((reinterpret_cast<uintptr_t>(positions_dev) & 7) || (reinterpret_cast<uintptr_t>(masks_dev) & 7)) return AZ_ERR_BAD_ARG;

@@ -103,6 +103,13 @@ struct Net {
     void *alt_u_policy = nullptr, *alt_u_value = nullptr;
     float *alt_logits = nullptr;
 
+    // ---- the paper's own network (52 planes, pooled context, query-key policy head) ----
+    bool pnet = false;
+    float *pnet_gw = nullptr;         // [pooled block][3C/4][C/2]
+    void *pnet_qk = nullptr;          // [max_batch][64][256] fp32: queries | keys
+    float *pnet_small = nullptr;      // the finishing kernel's fp32 parameters, see pnet.cu
+    unsigned char *pnet_actions = nullptr;   // [1880][4]: origin, destination, promotion piece + 1 (0 none), pad
+
     // ---- optional event timing of the tower ----
     bool profile = false;
     int n_events = 0;                 // pairs recorded since the last read
@@ -138,6 +145,12 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 
 // ---- kernels' launch functions (each returns AZ_OK or AZ_ERR_CUDA) ---------------------------
 int launch_encode52(const void *positions, int batch, bool bf16, void *planes, cudaStream_t s);
+int build_pnet(Net &n, const unsigned char *blob, size_t nbytes);
+int launch_pnet_finish(const Net &n, const uint64_t *masks, int batch, float *policy, float *value, cudaStream_t s);
+size_t tc_packed_layers_bytes(const int *cin_pad, int channels, int n_conv);
+void tc_pack_layers(const float *const *w, const float *const *scale, const int *cin, const int *cin_pad,
+                    int channels, int n_conv, __nv_bfloat16 *packed);
+void tc_pack_qk(const float *wq, const float *wk, int channels, __nv_bfloat16 *packed);
 int launch_encode(const void *positions, size_t stride, int batch, int in_planes, int in_pad,
                   bool bf16, void *planes, uint32_t *status, cudaStream_t s);
 int launch_legal_masks(const void *positions, size_t stride, int batch, int head, uint64_t *masks,

@@ -96,8 +96,13 @@ __device__ __forceinline__ void set_move(u64 *row, int stm, int from, int to, in
             }
         }
         idx = plane * 64 + from;
-    } else {
+    } else if (HEAD == AZ_POLICY_FLAT1858) {
         idx = promo ? g_flat_promo[(from & 7) * 3 + ((to & 7) - (from & 7) + 1)] + (promo - 1)
+                    : g_flat_pair[from * 64 + to];
+    } else {
+        // the paper's 1,880 actions: the same pairs, then four promotion pieces per (file, direction) in the
+        // order queen, rook, bishop, knight (promo 4, 3, 2, 1); the 1,858 table numbers three per combination
+        idx = promo ? 1792 + 4 * ((g_flat_promo[(from & 7) * 3 + ((to & 7) - (from & 7) + 1)] - 1792) / 3) + (4 - promo)
                     : g_flat_pair[from * 64 + to];
     }
     atomicOr(row + (idx >> 6), 1ull << (idx & 63));          // the row sits in shared memory, lanes share it
@@ -196,8 +201,17 @@ legal_masks_kernel(const unsigned char *__restrict__ positions, size_t stride, i
             n_occ &= ~(1ull << ep_cap);
         }
         if (attacked(k == 5 ? to : king_sq, them, o, n_occ)) continue;
+        const bool promotes = k == 0 && ((to >> 3) == (stm ? 0 : 7));
+        if (HEAD == AZ_POLICY_FROMTO1880 && promotes) {
+            // a promoting move has only its four promotion actions
+            set_move<HEAD>(row, stm, from, to, 1);
+            set_move<HEAD>(row, stm, from, to, 2);
+            set_move<HEAD>(row, stm, from, to, 3);
+            set_move<HEAD>(row, stm, from, to, 4);
+            continue;
+        }
         set_move<HEAD>(row, stm, from, to, 0);               // plain pair (= queen promotion)
-        if (k == 0 && ((to >> 3) == (stm ? 0 : 7))) {
+        if (promotes) {
             set_move<HEAD>(row, stm, from, to, 1);
             set_move<HEAD>(row, stm, from, to, 2);
             set_move<HEAD>(row, stm, from, to, 3);
@@ -273,7 +287,8 @@ int launch_legal_masks(const void *positions, size_t stride, int batch, int head
     } else {
         int rc = ensure_tables();
         if (rc != AZ_OK) return rc;
-        legal_masks_kernel<AZ_POLICY_FLAT1858><<<grid, block, 0, s>>>(p, stride, batch, (u64 *)masks);
+        if (head == AZ_POLICY_FLAT1858) legal_masks_kernel<AZ_POLICY_FLAT1858><<<grid, block, 0, s>>>(p, stride, batch, (u64 *)masks);
+        else legal_masks_kernel<AZ_POLICY_FROMTO1880><<<grid, block, 0, s>>>(p, stride, batch, (u64 *)masks);
     }
     AZ_LAUNCH_CHECK();
     return AZ_OK;

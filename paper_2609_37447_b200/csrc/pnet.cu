@@ -1,0 +1,340 @@
+// The paper's own inference network (Sec. 3.2, 4.3, App. D.1) on top of the tensor-core tower:
+// loading (blob -> packed tiles), and the finishing kernel that turns the tower's outputs into the
+// policy over the 1,880 actions and the win/draw/loss value.
+//
+// What runs where.  az_encode52's kernel writes the 52 planes (bf16, 64 channels per square); the
+// tower kernel's paper-network instantiation runs the input convolution, the scaled post-activation
+// blocks (activations capped at six, pooled context in blocks 1, 3, 5, ...) and, as its fused head
+// layer, the query and key maps of every square.  The token projection has no activation, so query,
+// key and promotion-offset maps are linear in the backbone's features and are composed with it at
+// load (W_q' = W_q W_t / sqrt(K), b_q' = (W_q b_t + b_q) / sqrt(K), and likewise for keys and
+// offsets, without the 1/sqrt(K)).  The finishing kernel, one CTA per position, computes
+//   - the value head: 2-channel 1x1 convolution + folded normalisation + ReLU, 48 hidden units with
+//     ReLU, three logits, softmax (fp32 ALU: 22 k multiply-adds per position);
+//   - the logits of the LEGAL actions only, q_origin . k_destination (+ the promotion piece's offset,
+//     a 128-long dot product with the origin square's features), and the softmax over them; illegal
+//     actions get exactly zero.
+// Shares nothing with oracle/.
+#include "common.cuh"
+#include "ptx.cuh"
+
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+namespace az {
+namespace {
+
+constexpr int kPlanes52 = 52, kActions = 1880, kKey = 128, kVC = 2, kVH = 48;
+
+// offsets (in floats) into Net::pnet_small
+struct Small {
+    static constexpr int o_w = 0;                       // [4][C]
+    static constexpr int o_b = o_w + 4 * 128;           // [4]
+    static constexpr int v_cw = o_b + 4;                // [2][C]
+    static constexpr int v_cs = v_cw + kVC * 128;       // [2]
+    static constexpr int v_cb = v_cs + kVC;             // [2]
+    static constexpr int v_w1 = v_cb + kVC;             // [48][128]
+    static constexpr int v_b1 = v_w1 + kVH * kVC * 64;  // [48]
+    static constexpr int v_w2 = v_b1 + kVH;             // [3][48]
+    static constexpr int v_b2 = v_w2 + 3 * kVH;         // [3]
+    static constexpr int total = v_b2 + 3;
+};
+
+__device__ __forceinline__ float dot128_f32(const float *a, const float *b) {
+    const float4 *pa = reinterpret_cast<const float4 *>(a), *pb = reinterpret_cast<const float4 *>(b);
+    float acc = 0.0f;
+#pragma unroll 8
+    for (int i = 0; i < 32; ++i) {
+        const float4 x = __ldg(pa + i), y = __ldg(pb + i);
+        acc = fmaf(x.x, y.x, acc); acc = fmaf(x.y, y.y, acc);
+        acc = fmaf(x.z, y.z, acc); acc = fmaf(x.w, y.w, acc);
+    }
+    return acc;
+}
+__device__ __forceinline__ float dot128_f32_bf16(const float *w, const __nv_bfloat16 *h) {
+    const uint4 *ph = reinterpret_cast<const uint4 *>(h);
+    float acc = 0.0f;
+#pragma unroll 4
+    for (int i = 0; i < 16; ++i) {
+        const uint4 y = __ldg(ph + i);
+        const uint32_t ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float2 fy = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&ys[j]));
+            acc = fmaf(w[i * 8 + 2 * j], fy.x, acc);
+            acc = fmaf(w[i * 8 + 2 * j + 1], fy.y, acc);
+        }
+    }
+    return acc;
+}
+
+constexpr int kFinishThreads = 128;
+constexpr int kPerThread = (kActions + kFinishThreads - 1) / kFinishThreads;   // 15
+
+__device__ __forceinline__ float block_reduce(float v, bool is_max, float *scratch) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float t = __shfl_xor_sync(0xffffffffu, v, o);
+        v = is_max ? fmaxf(v, t) : v + t;
+    }
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = scratch[0];
+#pragma unroll
+    for (int w = 1; w < kFinishThreads / 32; ++w) r = is_max ? fmaxf(r, scratch[w]) : r + scratch[w];
+    return r;
+}
+
+__global__ void __launch_bounds__(kFinishThreads)
+pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict__ qk,
+                   const uint64_t *__restrict__ masks, const float *__restrict__ small,
+                   const uchar4 *__restrict__ actions, int batch, float *__restrict__ policy,
+                   float *__restrict__ value, uint32_t *__restrict__ status) {
+    ptx::grid_dependency_wait();                     // the tower's outputs must be complete
+    const int pos = blockIdx.x, tid = threadIdx.x;
+    if (pos >= batch) return;
+    __shared__ float v_s[kVC * 64], hid_s[kVH], red[kFinishThreads / 32];
+    const __nv_bfloat16 *hp = h + (size_t)pos * 64 * 128;
+    const float *qkp = qk + (size_t)pos * 64 * 256;
+
+    // ---- value head
+    {
+        const int c = tid >> 6, sq = tid & 63;
+        const float d = dot128_f32_bf16(small + Small::v_cw + c * 128, hp + sq * 128);
+        v_s[c * 64 + sq] = fmaxf(fmaf(small[Small::v_cs + c], d, small[Small::v_cb + c]), 0.0f);
+    }
+    __syncthreads();
+    if (tid < kVH) {
+        const float *w = small + Small::v_w1 + tid * (kVC * 64);
+        float acc = small[Small::v_b1 + tid];
+#pragma unroll 8
+        for (int i = 0; i < kVC * 64; ++i) acc = fmaf(w[i], v_s[i], acc);
+        hid_s[tid] = fmaxf(acc, 0.0f);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        float z[3], m = -INFINITY, sum = 0.0f;
+#pragma unroll
+        for (int c = 0; c < 3; ++c) {
+            float acc = small[Small::v_b2 + c];
+            for (int j = 0; j < kVH; ++j) acc = fmaf(small[Small::v_w2 + c * kVH + j], hid_s[j], acc);
+            z[c] = acc;
+            m = fmaxf(m, acc);
+        }
+#pragma unroll
+        for (int c = 0; c < 3; ++c) { z[c] = __expf(z[c] - m); sum += z[c]; }
+#pragma unroll
+        for (int c = 0; c < 3; ++c) value[(size_t)pos * 3 + c] = z[c] / sum;
+    }
+
+    // ---- policy: logits of the legal actions, softmax over them
+    float lg[kPerThread];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kPerThread; ++j) {
+        const int i = tid + j * kFinishThreads;
+        lg[j] = -INFINITY;
+        if (i < kActions && ((masks[(size_t)pos * 30 + (i >> 6)] >> (i & 63)) & 1ull)) {
+            const uchar4 a = actions[i];                                   // origin, destination, piece + 1
+            float s = dot128_f32(qkp + a.x * 256, qkp + a.y * 256 + 128);
+            if (a.z) s += dot128_f32_bf16(small + Small::o_w + (a.z - 1) * 128, hp + a.x * 128) + small[Small::o_b + a.z - 1];
+            lg[j] = s;
+            mx = fmaxf(mx, s);
+        }
+    }
+    mx = block_reduce(mx, true, red);
+    float sum = 0.0f;
+#pragma unroll
+    for (int j = 0; j < kPerThread; ++j) {
+        lg[j] = lg[j] == -INFINITY ? 0.0f : __expf(lg[j] - mx);
+        sum += lg[j];
+    }
+    sum = block_reduce(sum, false, red);
+    if (!(sum > 0.0f)) {                                                   // no legal action: an all-zero row and a status bit
+        if (tid == 0) atomicOr(status, kStatusEmptyMask);
+        sum = 1.0f;
+    }
+    const float inv = 1.0f / sum;
+#pragma unroll
+    for (int j = 0; j < kPerThread; ++j) {
+        const int i = tid + j * kFinishThreads;
+        if (i < kActions) policy[(size_t)pos * kActions + i] = lg[j] * inv;
+    }
+}
+
+struct PBlob {
+    int L, C;
+    const float *in_w, *in_s, *in_b;
+    std::vector<const float *> w1, s1, b1, gw, w2, s2, b2;
+    const float *t_w, *t_b, *q_w, *q_b, *k_w, *k_b, *o_w, *o_b;
+    const float *v_cw, *v_cs, *v_cb, *v_w1, *v_b1, *v_w2, *v_b2;
+};
+
+int parse_pnet(const az_arch &a, const unsigned char *blob, size_t nbytes, PBlob &v) {
+    if (nbytes < 64 || memcmp(blob, "AZPNET1", 8) != 0) return AZ_ERR_BAD_WEIGHTS;
+    uint32_t h[7];
+    memcpy(h, blob + 8, sizeof h);
+    if (h[0] != 1 || h[1] != a.blocks || h[2] != a.channels || h[3] != (uint32_t)kKey || h[4] != (uint32_t)kVC ||
+        h[5] != (uint32_t)kVH)
+        return AZ_ERR_BAD_WEIGHTS;
+    const size_t C = a.channels, L = a.blocks, P = C / 4, R = C - P;
+    size_t need = C * kPlanes52 * 9 + 2 * C;
+    for (size_t b = 0; b < L; ++b) need += C * C * 9 + 2 * C + ((b & 1) ? R * 2 * P + C * R * 9 : C * C * 9) + 2 * C;
+    need += (size_t)kKey * C + kKey + 2 * ((size_t)kKey * kKey + kKey) + 4 * kKey + 4;
+    need += (size_t)kVC * C + 2 * kVC + (size_t)kVH * kVC * 64 + kVH + 3 * kVH + 3;
+    if (nbytes != 64 + 4 * need) return AZ_ERR_BAD_WEIGHTS;
+    const float *p = reinterpret_cast<const float *>(blob + 64);
+    for (size_t i = 0; i < need; ++i)
+        if (!std::isfinite(p[i])) return AZ_ERR_BAD_WEIGHTS;
+    auto take = [&p](size_t n) { const float *q = p; p += n; return q; };
+    v.L = (int)L; v.C = (int)C;
+    v.in_w = take(C * kPlanes52 * 9); v.in_s = take(C); v.in_b = take(C);
+    for (size_t b = 0; b < L; ++b) {
+        v.w1.push_back(take(C * C * 9)); v.s1.push_back(take(C)); v.b1.push_back(take(C));
+        v.gw.push_back((b & 1) ? take(R * 2 * P) : nullptr);
+        v.w2.push_back(take(C * ((b & 1) ? R : C) * 9)); v.s2.push_back(take(C)); v.b2.push_back(take(C));
+    }
+    v.t_w = take((size_t)kKey * C); v.t_b = take(kKey);
+    v.q_w = take((size_t)kKey * kKey); v.q_b = take(kKey);
+    v.k_w = take((size_t)kKey * kKey); v.k_b = take(kKey);
+    v.o_w = take(4 * kKey); v.o_b = take(4);
+    v.v_cw = take((size_t)kVC * C); v.v_cs = take(kVC); v.v_cb = take(kVC);
+    v.v_w1 = take((size_t)kVH * kVC * 64); v.v_b1 = take(kVH);
+    v.v_w2 = take(3 * kVH); v.v_b2 = take(3);
+    return AZ_OK;
+}
+
+// out[rows][C] = m[rows][K] * t_w[K][C] * f,  out_b[rows] = (m * t_b + b) * f   (double accumulation)
+void compose(const float *m, const float *b, int rows, const float *t_w, const float *t_b, int C, double f,
+             std::vector<float> &out, std::vector<float> &out_b) {
+    out.assign((size_t)rows * C, 0.0f);
+    out_b.assign(rows, 0.0f);
+    for (int r = 0; r < rows; ++r) {
+        for (int c = 0; c < C; ++c) {
+            double acc = 0.0;
+            for (int k = 0; k < kKey; ++k) acc += (double)m[(size_t)r * kKey + k] * (double)t_w[(size_t)k * C + c];
+            out[(size_t)r * C + c] = (float)(acc * f);
+        }
+        double acc = b[r];
+        for (int k = 0; k < kKey; ++k) acc += (double)m[(size_t)r * kKey + k] * (double)t_b[k];
+        out_b[r] = (float)(acc * f);
+    }
+}
+
+}  // namespace
+
+// Builds the device side of a paper-network az_net: 128 channels, bf16 (other sizes of the paper's
+// ladder are not built yet and are refused by the caller).
+int build_pnet(Net &n, const unsigned char *blob, size_t nbytes) {
+    const az_arch &a = n.arch;
+    PBlob v;
+    int rc = parse_pnet(a, blob, nbytes, v);
+    if (rc != AZ_OK) return rc;
+    const int C = v.C, L = v.L, P = C / 4, R = C - P;
+    n.bf16 = true;
+    n.pnet = true;
+    n.in_pad = 64;
+    n.n_conv = 1 + 2 * L;
+    // tower tiles
+    std::vector<const float *> w, s;
+    std::vector<int> cin, cin_pad;
+    std::vector<float> bias((size_t)n.n_conv * C);
+    w.push_back(v.in_w); s.push_back(v.in_s); cin.push_back(kPlanes52); cin_pad.push_back(64);
+    memcpy(&bias[0], v.in_b, sizeof(float) * C);
+    for (int b = 0; b < L; ++b) {
+        w.push_back(v.w1[b]); s.push_back(v.s1[b]); cin.push_back(C); cin_pad.push_back(C);
+        memcpy(&bias[(size_t)(1 + 2 * b) * C], v.b1[b], sizeof(float) * C);
+        w.push_back(v.w2[b]); s.push_back(v.s2[b]); cin.push_back((b & 1) ? R : C); cin_pad.push_back((b & 1) ? R : C);
+        memcpy(&bias[(size_t)(2 + 2 * b) * C], v.b2[b], sizeof(float) * C);
+    }
+    const size_t bytes = tc_packed_layers_bytes(cin_pad.data(), C, n.n_conv);
+    std::vector<__nv_bfloat16> packed(bytes / sizeof(__nv_bfloat16));
+    tc_pack_layers(w.data(), s.data(), cin.data(), cin_pad.data(), C, n.n_conv, packed.data());
+    AZ_CUDA(cudaMalloc(&n.tc_weights, bytes));
+    AZ_CUDA(cudaMemcpy(n.tc_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
+    AZ_CUDA(cudaMalloc((void **)&n.tc_bias, bias.size() * sizeof(float)));
+    AZ_CUDA(cudaMemcpy(n.tc_bias, bias.data(), bias.size() * sizeof(float), cudaMemcpyHostToDevice));
+    // pooled-context maps of blocks 1, 3, 5, ...
+    {
+        std::vector<float> gw;
+        for (int b = 1; b < L; b += 2) gw.insert(gw.end(), v.gw[b], v.gw[b] + (size_t)R * 2 * P);
+        if (gw.empty()) gw.push_back(0.0f);
+        AZ_CUDA(cudaMalloc((void **)&n.pnet_gw, gw.size() * sizeof(float)));
+        AZ_CUDA(cudaMemcpy(n.pnet_gw, gw.data(), gw.size() * sizeof(float), cudaMemcpyHostToDevice));
+    }
+    // head layer: queries and keys composed with the token projection, 1/sqrt(K) folded into the queries
+    std::vector<float> wq, bq, wk, bk, wo, bo;
+    compose(v.q_w, v.q_b, kKey, v.t_w, v.t_b, C, 1.0 / std::sqrt((double)kKey), wq, bq);
+    compose(v.k_w, v.k_b, kKey, v.t_w, v.t_b, C, 1.0, wk, bk);
+    compose(v.o_w, v.o_b, 4, v.t_w, v.t_b, C, 1.0, wo, bo);
+    n.tc_head_n = 256;
+    std::vector<__nv_bfloat16> hw((size_t)256 * C);
+    tc_pack_qk(wq.data(), wk.data(), C, hw.data());
+    AZ_CUDA(cudaMalloc(&n.tc_head_w, hw.size() * sizeof(__nv_bfloat16)));
+    AZ_CUDA(cudaMemcpy(n.tc_head_w, hw.data(), hw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
+    std::vector<float> hb(256);
+    for (int i = 0; i < 128; ++i) { hb[i] = bq[i]; hb[128 + i] = bk[i]; }
+    AZ_CUDA(cudaMalloc((void **)&n.tc_head_bias, hb.size() * sizeof(float)));
+    AZ_CUDA(cudaMemcpy(n.tc_head_bias, hb.data(), hb.size() * sizeof(float), cudaMemcpyHostToDevice));
+    // the finishing kernel's parameters
+    std::vector<float> small(Small::total);
+    memcpy(&small[Small::o_w], wo.data(), sizeof(float) * 4 * C);
+    memcpy(&small[Small::o_b], bo.data(), sizeof(float) * 4);
+    memcpy(&small[Small::v_cw], v.v_cw, sizeof(float) * kVC * C);
+    memcpy(&small[Small::v_cs], v.v_cs, sizeof(float) * kVC);
+    memcpy(&small[Small::v_cb], v.v_cb, sizeof(float) * kVC);
+    memcpy(&small[Small::v_w1], v.v_w1, sizeof(float) * kVH * kVC * 64);
+    memcpy(&small[Small::v_b1], v.v_b1, sizeof(float) * kVH);
+    memcpy(&small[Small::v_w2], v.v_w2, sizeof(float) * 3 * kVH);
+    memcpy(&small[Small::v_b2], v.v_b2, sizeof(float) * 3);
+    AZ_CUDA(cudaMalloc((void **)&n.pnet_small, small.size() * sizeof(float)));
+    AZ_CUDA(cudaMemcpy(n.pnet_small, small.data(), small.size() * sizeof(float), cudaMemcpyHostToDevice));
+    // the action list (Sec. 3.2, App. D.1), generated: 1,792 origin-destination pairs a queen ray or a knight
+    // jump apart, origins then destinations ascending; then, for origins on the seventh rank ascending and the
+    // destinations origin+7, +8, +9 that stay on the board, the pieces queen, rook, bishop, knight
+    {
+        std::vector<unsigned char> act((size_t)kActions * 4, 0);
+        int next = 0;
+        for (int from = 0; from < 64; ++from)
+            for (int to = 0; to < 64; ++to) {
+                const int df = abs((to & 7) - (from & 7)), dr = abs((to >> 3) - (from >> 3));
+                if (from == to) continue;
+                if (df == 0 || dr == 0 || df == dr || df * dr == 2) {
+                    act[4 * next] = (unsigned char)from; act[4 * next + 1] = (unsigned char)to; ++next;
+                }
+            }
+        for (int from = 48; from < 56; ++from)
+            for (int to = from + 7; to <= from + 9; ++to) {
+                if (to > 63 || abs((to & 7) - (from & 7)) > 1) continue;
+                for (int piece = 0; piece < 4; ++piece) {
+                    act[4 * next] = (unsigned char)from; act[4 * next + 1] = (unsigned char)to;
+                    act[4 * next + 2] = (unsigned char)(piece + 1); ++next;
+                }
+            }
+        if (next != kActions) return AZ_ERR_BAD_ARCH;
+        AZ_CUDA(cudaMalloc((void **)&n.pnet_actions, act.size()));
+        AZ_CUDA(cudaMemcpy(n.pnet_actions, act.data(), act.size(), cudaMemcpyHostToDevice));
+    }
+    // workspace: planes, tower output, queries and keys, status
+    const size_t B = a.max_batch;
+    AZ_CUDA(cudaMalloc(&n.planes, B * 64 * 64 * sizeof(__nv_bfloat16)));
+    AZ_CUDA(cudaMalloc(&n.act[0], B * 64 * C * sizeof(__nv_bfloat16)));
+    AZ_CUDA(cudaMalloc(&n.pnet_qk, B * 64 * 256 * sizeof(float)));
+    AZ_CUDA(cudaMalloc((void **)&n.status_dev, sizeof(uint32_t)));
+    AZ_CUDA(cudaMemset(n.status_dev, 0, sizeof(uint32_t)));
+    n.tc_ready = true;
+    return AZ_OK;
+}
+
+int launch_pnet_finish(const Net &n, const uint64_t *masks, int batch, float *policy, float *value, cudaStream_t s) {
+    if (batch == 0) return AZ_OK;
+    AZ_CUDA(launch_dependent(pnet_finish_kernel, dim3((unsigned)batch), dim3(kFinishThreads), 0, s,
+                             static_cast<const __nv_bfloat16 *>(n.act[0]), static_cast<const float *>(n.pnet_qk), masks,
+                             static_cast<const float *>(n.pnet_small), reinterpret_cast<const uchar4 *>(n.pnet_actions), batch,
+                             policy, value, n.status_dev));
+    return AZ_OK;
+}
+
+}  // namespace az

@@ -79,14 +79,19 @@ struct Shape {
     static constexpr int kOffFrames = 0;
     static constexpr int kOffWeights = kGroups * kFrameBytes;
     static constexpr int kOffBars = kOffWeights + kStages * kStageBytes;
-    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done, lead[S]
-    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1 + kStages;
+    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done, lead[S], pool[G]
+    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1 + kStages + kGroups;
     static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
     static constexpr int kOffAbort = kOffTmemPtr + 4;
     static constexpr int kOffConst = (kOffAbort + 4 + 15) & ~15;     // per-warp copies of the current layer's channel constants
     // per epilogue warp: the current layer's channel constants for the channels of its own slices
-    static constexpr int smem_bytes(bool fp8) { return kOffConst + kEpiWarps * (fp8 ? 3 : 1) * (kC / kSets) * 4 + 128 * 4; }
-    static_assert(kOffConst + kEpiWarps * 3 * (kC / kSets) * 4 + 512 <= kMaxSmem || kC == 256, "shared memory budget");
+    // after the constants: head biases (up to 256), then the pooled-context scratch of the paper's network
+    // per group: partial sums and maxima [4 warps][2 boards][C/4], pooled vector [2][C/2], context [2][3C/4]
+    static constexpr int kPoolFloats = kGroups * (2 * 4 * 2 * (kC / 4) + 2 * (kC / 2) + 2 * (3 * kC / 4));
+    static constexpr int smem_bytes(bool fp8, bool pnet = false) {
+        return kOffConst + kEpiWarps * (fp8 ? 3 : 1) * (kC / kSets) * 4 + 256 * 4 + (pnet ? kPoolFloats * 4 : 0);
+    }
+    static_assert(kOffConst + kEpiWarps * 3 * (kC / kSets) * 4 + 1024 <= kMaxSmem || kC == 256, "shared memory budget");
     static_assert(kGroups * 2 * kC == (int)kTmemCols, "TMEM: per group C columns of residual stream and C of accumulator");
 };
 
@@ -115,6 +120,10 @@ struct TowerArgs {
     const float *lconst;
     // calibration run (bf16 kernel): per-layer, per-channel maximum of the layer outputs, as float bits
     unsigned int *absmax;            // [n_conv][C]
+    // the paper's own network (kPnet instantiation; Sec. 3.2, 4.3.3, 4.3.6, App. D.1): activations capped
+    // at six, pooled context in blocks 1, 3, 5, ..., query / key projections as the fused head layer
+    const float *gw;                 // [pooled block][3C/4][C/2] fp32: pooled vector -> context
+    float *qk_out;                   // [batch][64][256] fp32: queries (128) then keys (128) per square
 };
 
 // One round of a CTA's work: which two-board groups sit in its slots (-1 = the slot idles).
@@ -156,12 +165,13 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
 
 // slices of the head projection's K that travel in one weight stage
 template <class S> __device__ __host__ constexpr int head_slices_per_stage(int head_n) {
-    return S::kC == 128 ? S::kSlices : (head_n == 64 ? 8 : 4);
+    return S::kC == 128 ? (head_n == 256 ? 4 : S::kSlices) : (head_n == 64 ? 8 : 4);
 }
 
-template <bool kFp8, class S>
+template <bool kFp8, class S, bool kPnet = false>
 __global__ void __launch_bounds__(S::kThreads, 1)
 tower_tc_kernel(const TowerArgs args) {
+    static_assert(!kPnet || (!kFp8 && S::kC == 128 && S::kSets == 1), "the paper's network runs on the bf16 128-channel shape");
     constexpr int kC = S::kC, kGroups = S::kGroups, kStages = S::kStages, kSlices = S::kSlices;
     constexpr int kFrameBytes = S::kFrameBytes, kStageBytes = S::kStageBytes, kThreads = S::kThreads;
     static_assert(!kFp8 || kC == 128, "the FP8 tower exists for 128 channels");
@@ -177,6 +187,7 @@ tower_tc_kernel(const TowerArgs args) {
     auto bar_a_ready = [&](int g, int kc) { return bars + 8u * (2 * kStages + kGroups + g * kSlices + kc); };
     const uint32_t bar_done = bars + 8u * (2 * kStages + kGroups + kGroups * kSlices);
     auto bar_lead = [&](int s) { return bar_done + 8u * (1 + s); };   // group 0 has issued its MMAs on stage s
+    auto bar_pool = [&](int g) { return bar_done + 8u * (1 + kStages + g); };   // the four epilogue warps of group g meet here
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + S::kOffAbort);
     uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + S::kOffTmemPtr);
     constexpr int kConstFloats = (kFp8 ? 3 : 1) * kC;          // per layer: (scale, bias, h ratio) or bias
@@ -196,6 +207,7 @@ tower_tc_kernel(const TowerArgs args) {
         }
         for (int g = 0; g < kGroups; ++g) {
             ptx::mbar_init(bar_acc_full(g), 1);
+            ptx::mbar_init(bar_pool(g), 4);
             for (int kc = 0; kc < kSlices; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4 * S::kSets);
         }
         ptx::mbar_init(bar_done, kGroups);
@@ -218,8 +230,14 @@ tower_tc_kernel(const TowerArgs args) {
     const int head_n = args.head_n;
     const int in_slices = args.in_pad / 16;
     const int hsps = head_slices_per_stage<S>(head_n);
+    // the paper's network: the first convolution of blocks 1, 3, 5, ... (layers 3, 7, 11, ...) feeds the pooled
+    // context, and the second convolution of those blocks (layers 4, 8, 12, ...) reads 3C/4 channels only
+    auto pool_layer = [&](int l) { return kPnet && (l & 3) == 3; };
+    auto short_layer = [&](int l) { return kPnet && l >= 4 && (l & 3) == 0; };
     auto round_of = [&](int r) { return get_round<S>(r, (int)blockIdx.x, (int)gridDim.x, n_groups); };
-    auto slices_of = [&](int l) { return l == 0 ? in_slices : (kFp8 ? kC / 32 : kC / 16); };   // K per MMA: 16 bf16 or 32 e4m3
+    auto slices_of = [&](int l) {                                                               // K per MMA: 16 bf16 or 32 e4m3
+        return l == 0 ? in_slices : short_layer(l) ? 3 * kC / 64 : (kFp8 ? kC / 32 : kC / 16);
+    };
     const bool tr = args.trace && blockIdx.x == 0;
     long long t_wait[3] = {0, 0, 0};
     long long t_issue = 0;
@@ -357,6 +375,15 @@ tower_tc_kernel(const TowerArgs args) {
             if (head_n && ok) {
                 // head projections: a 1x1 convolution = the centre tap only, N = head_n, into the ACC columns
                 const uint32_t idesc_h = ptx::idesc_bf16_f32(128, head_n);
+                if (kPnet) {
+                    // 256 output columns = the residual stream's columns and the accumulator's: the last
+                    // layer's epilogue must have read all of them before the first MMA overwrites any
+                    for (int kc = 0; kc < kSlices && ok; ++kc) {
+                        ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
+                        a_phase ^= 1u << kc;
+                    }
+                    if (!ok) break;
+                }
                 for (int kc = 0; kc < kSlices && ok; ++kc) {
                     if (kc % hsps == 0) {
                         ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
@@ -366,16 +393,18 @@ tower_tc_kernel(const TowerArgs args) {
                             if (!ok) break;
                         }
                     }
-                    ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
-                    if (!ok) break;
-                    a_phase ^= 1u << kc;
+                    if (!kPnet) {
+                        ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
+                        if (!ok) break;
+                        a_phase ^= 1u << kc;
+                    }
                     ptx::tc_fence_after();
                     const bool stage_done = (kc % hsps) == hsps - 1;
                     {
                         const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
                         const uint32_t b_lo = (((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) + (uint32_t)((kc % hsps) * head_n * 2)) |
                                               ((uint32_t)head_n << 16);          // K core matrices head_n*16 bytes apart
-                        ptx::mma_bf16_elect(d_h + (uint32_t)kC, a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u, elected);
+                        ptx::mma_bf16_elect(d_h + (kPnet ? 0u : (uint32_t)kC), a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u, elected);
                     }
                     if (elected) {
                         if (kc == kSlices - 1) ptx::mma_commit(bar_acc_full(g));
@@ -412,6 +441,12 @@ tower_tc_kernel(const TowerArgs args) {
         unsigned char *frame = smem + S::kOffFrames + g * kFrameBytes;
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 2 * kC);
         float *lc = reinterpret_cast<float *>(smem + S::kOffConst) + ew * kMyConstFloats;   // this warp's copy of the layer constants
+        // pooled-context scratch of this group (paper's network only)
+        constexpr int kPoolC = kC / 4, kRegC = kC - kC / 4;
+        float *pool_part = head_bias_smem + 256 + g * (S::kPoolFloats / kGroups);   // [sum|max][warp q][board][kPoolC]
+        float *pool_vec = pool_part + 2 * 4 * 2 * kPoolC;                          // [board][2 * kPoolC]: means, then maxima
+        float *pool_ctx = pool_vec + 2 * 2 * kPoolC;                               // [board][kRegC]
+        uint32_t pool_phase = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
         for (int r = 0; ok; ++r) {
@@ -484,12 +519,85 @@ tower_tc_kernel(const TowerArgs args) {
                 const uint32_t t_src = t_lane + (uint32_t)(from_acc ? kC : 0);
                 const bool keep_h = !from_acc && l != n_conv - 1;   // the residual stream stays in TMEM as fp32
                 uint32_t r[2][16];
+                const bool pooled = pool_layer(l);
+                if (kPnet && pooled) {
+                    // ---- pooled context (Sec. 3.2, 4.3.3): the last C/4 channels of this first convolution are
+                    // activated, averaged and maximised over each board's 64 squares, mapped to 3C/4 values and
+                    // added to the other channels before THEIR activation.
+                    // (1) this warp's 32 rows: 16 of board 0 (lanes with bit 3 clear) and 16 of board 1
+#pragma unroll
+                    for (int ps = 0; ps < kPoolC / 16; ++ps) {
+                        ptx::tmem_ld16(t_src + (uint32_t)(kRegC + ps * 16), r[0]);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            const float a = live ? fminf(fmaxf(__uint_as_float(r[0][i]) + bias[kRegC + ps * 16 + i], 0.0f), 6.0f) : 0.0f;
+                            float sm = a, mx = a;
+#pragma unroll
+                            for (int o = 1; o <= 16; o <<= 1) {
+                                if (o == 8) continue;                          // bit 3 of the lane tells the boards apart
+                                sm += __shfl_xor_sync(0xffffffffu, sm, o);
+                                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                            }
+                            if ((lane & 23) == 0) {                            // lanes 0 and 8: one per board
+                                pool_part[(q * 2 + b) * kPoolC + ps * 16 + i] = sm;
+                                pool_part[4 * 2 * kPoolC + (q * 2 + b) * kPoolC + ps * 16 + i] = mx;
+                            }
+                        }
+                    }
+                    auto meet = [&]() -> bool {                                // the group's four warps, bounded
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(bar_pool(g));
+                        const bool met = wait_bar(bar_pool(g), pool_phase, abort_flag, args.status);
+                        pool_phase ^= 1u;
+                        return met;
+                    };
+                    ok = meet();
+                    if (!ok) break;
+                    // (2) the four warps' partial results -> the pooled vector: one entry per thread
+                    {
+                        const int e = q * 32 + lane;                           // 0..127 = board * 64 + entry
+                        const int pb = e >> 6, j = e & 63, c = j % kPoolC;
+                        const float *src = pool_part + (j >= kPoolC ? 4 * 2 * kPoolC : 0);
+                        float acc = src[(0 * 2 + pb) * kPoolC + c];
+#pragma unroll
+                        for (int w4 = 1; w4 < 4; ++w4) {
+                            const float t = src[(w4 * 2 + pb) * kPoolC + c];
+                            acc = j >= kPoolC ? fmaxf(acc, t) : acc + t;
+                        }
+                        pool_vec[pb * 2 * kPoolC + j] = j >= kPoolC ? acc : acc * (1.0f / 64.0f);
+                    }
+                    ok = meet();
+                    if (!ok) break;
+                    // (3) context = gw . pooled vector: 2 boards x 3C/4 outputs over the group's 128 threads
+                    {
+                        const float *gw = args.gw + (size_t)((l - 3) >> 2) * kRegC * 2 * kPoolC;
+                        for (int e = q * 32 + lane; e < 2 * kRegC; e += 128) {
+                            const int pb = e / kRegC, rr0 = e % kRegC;
+                            const float4 *wrow = reinterpret_cast<const float4 *>(gw + (size_t)rr0 * 2 * kPoolC);
+                            const float4 *vec = reinterpret_cast<const float4 *>(pool_vec + pb * 2 * kPoolC);
+                            float acc = 0.0f;
+#pragma unroll
+                            for (int j = 0; j < 2 * kPoolC / 4; ++j) {
+                                const float4 wv = __ldg(wrow + j), pv = vec[j];
+                                acc = fmaf(wv.x, pv.x, acc); acc = fmaf(wv.y, pv.y, acc);
+                                acc = fmaf(wv.z, pv.z, acc); acc = fmaf(wv.w, pv.w, acc);
+                            }
+                            pool_ctx[pb * kRegC + rr0] = acc;
+                        }
+                    }
+                    ok = meet();
+                    if (!ok) break;
+                }
+                const float *ctx = pool_ctx + b * kRegC;                       // this row's board
+                const int n_my = (kPnet && pooled) ? kRegC / 16 : kMySlices;   // the pooled channels are not handed on
                 ptx::tmem_ld16(t_src + (uint32_t)(set * 16), r[0]);
 #pragma unroll
                 for (int ks = 0; ks < kMySlices; ++ks) {
+                    if (kPnet && ks >= n_my) break;
                     const int kc = ks * S::kSets + set;             // the slice; ks indexes this warp's constants
                     ptx::tmem_ld_wait();
-                    if (ks + 1 < kMySlices) ptx::tmem_ld16(t_src + (uint32_t)((kc + S::kSets) * 16), r[(ks + 1) & 1]);
+                    if (ks + 1 < n_my) ptx::tmem_ld16(t_src + (uint32_t)((kc + S::kSets) * 16), r[(ks + 1) & 1]);
                     uint32_t(&rr)[16] = r[ks & 1];
                     float v[16];
 #pragma unroll
@@ -508,11 +616,19 @@ tower_tc_kernel(const TowerArgs args) {
                             v[i + 3] = __uint_as_float(rr[i + 3]) + bv.w;
                         }
                     }
+                    if (kPnet && pooled) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] += ctx[ks * 16 + i];
+                    }
                     // ReLU: a first convolution's output is only ever read as packed operands, and the
                     // conversion clamps; elsewhere the fp32 value itself goes on (residual stream, output)
                     if (!from_acc || (!kFp8 && args.absmax != nullptr)) {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.0f);
+                    }
+                    if (kPnet) {                                     // activations capped at six (Sec. 4.3.6)
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = fminf(v[i], 6.0f);
                     }
                     if (!kFp8 && args.absmax != nullptr) {
                         // calibration: largest output of this layer per channel over all rows of the warp
@@ -597,13 +713,18 @@ tower_tc_kernel(const TowerArgs args) {
 #pragma unroll 1
                 for (int j = 0; j < n_slices; ++j) {
                     uint32_t rr[16];
-                    ptx::tmem_ld16(t_lane + (uint32_t)kC + (uint32_t)(j * 16), rr);
+                    ptx::tmem_ld16(t_lane + (kPnet ? 0u : (uint32_t)kC) + (uint32_t)(j * 16), rr);
                     ptx::tmem_ld_wait();
                     float v[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(rr[i]) + hb[j * 16 + i];
                     if (!live) {
                         // rows past the end of the batch produce nothing
+                    } else if (kPnet) {
+                        // queries (columns 0..127) and keys (128..255) of this square, fp32 as accumulated, row-major
+                        float4 *qk = reinterpret_cast<float4 *>(args.qk_out + ((size_t)board * 64 + sq) * 256 + j * 16);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) qk[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
                     } else if (head_n == 112 && j < value_slice0) {
                         // 73 policy planes: raw logits, index = plane*64 + square
 #pragma unroll
@@ -676,6 +797,47 @@ void tc_pack_weights(const float *const *w, const float *const *scale, int in_pl
                                 *dst++ = __float2bfloat16_rn(v);
                             }
     }
+}
+
+// The same tiles for a tower whose layers read different numbers of input channels (the paper's
+// network: 52 planes padded to 64 into the input layer, 3C/4 channels into the second convolution
+// of every pooled block).  cin[l] real input channels, cin_pad[l] a multiple of 16.
+size_t tc_packed_layers_bytes(const int *cin_pad, int channels, int n_conv) {
+    size_t slices = 0;
+    for (int l = 0; l < n_conv; ++l) slices += (size_t)cin_pad[l] / 16;
+    return slices * 9 * (size_t)channels * 32;
+}
+
+void tc_pack_layers(const float *const *w, const float *const *scale, const int *cin, const int *cin_pad,
+                    int channels, int n_conv, __nv_bfloat16 *packed) {
+    __nv_bfloat16 *dst = packed;
+    for (int l = 0; l < n_conv; ++l)
+        for (int kc = 0; kc < cin_pad[l] / 16; ++kc)
+            for (int tap = 0; tap < 9; ++tap)
+                for (int k8 = 0; k8 < 2; ++k8)
+                    for (int ng = 0; ng < channels / 8; ++ng)
+                        for (int r = 0; r < 8; ++r)
+                            for (int e = 0; e < 8; ++e) {
+                                const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
+                                float v = 0.0f;
+                                if (ci < cin[l]) v = scale[l][n] * w[l][((size_t)n * cin[l] + ci) * 9 + tap];
+                                *dst++ = __float2bfloat16_rn(v);
+                            }
+}
+
+// Head layer of the paper's network: one N = 256 tile per 16-channel slice, rows 0..127 the query
+// map, rows 128..255 the key map (both already composed with the token projection).
+void tc_pack_qk(const float *wq, const float *wk, int channels, __nv_bfloat16 *packed) {
+    __nv_bfloat16 *dst = packed;
+    for (int kc = 0; kc < channels / 16; ++kc)
+        for (int k8 = 0; k8 < 2; ++k8)
+            for (int ng = 0; ng < 256 / 8; ++ng)
+                for (int r = 0; r < 8; ++r)
+                    for (int e = 0; e < 8; ++e) {
+                        const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
+                        const float v = n < 128 ? wq[(size_t)n * channels + ci] : wk[(size_t)(n - 128) * channels + ci];
+                        *dst++ = __float2bfloat16_rn(v);
+                    }
 }
 
 int tower_tc_launch_count() { return 1; }
@@ -774,6 +936,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
     const int sms = dev < 64 ? sm_count[dev] : 148;
@@ -799,12 +962,15 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     a.logits = net.logits;
     a.lconst = net.tc8_lconst;
     a.absmax = absmax;
+    a.gw = net.pnet_gw;
+    a.qk_out = static_cast<float *>(net.pnet_qk);
     static const bool trace = getenv("AZ_TOWER_TRACE") != nullptr;
     a.trace = trace ? atoi(getenv("AZ_TOWER_TRACE")) : 0;
     // one CTA per SM, or one per two-board group when there are fewer groups than SMs
     const int n_groups = (batch + kNB - 1) / kNB;
     const int grid = n_groups < sms ? n_groups : sms;
-    if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
+    if (net.pnet) tower_tc_kernel<false, Shape128, true><<<grid, Shape128::kThreads, Shape128::smem_bytes(false, true), s>>>(a);
+    else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
     else if (fp8) tower_tc_kernel<true, Shape128F8><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else tower_tc_kernel<false, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(false), s>>>(a);
     AZ_LAUNCH_CHECK();
