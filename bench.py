@@ -21,7 +21,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from inputs import configs, positions, weights  # noqa: E402
+from inputs import configs, pnet_weights, positions, weights  # noqa: E402
 
 METRIC = "leaf evals/sec, 20x128 bf16 batch 1024"
 UNIT = "evals/s"
@@ -32,14 +32,35 @@ WORKLOADS = {
     "c5": "c5: 40x256 bf16, 112 history planes, flat-1858 policy + WDL value (batch sweep via --batch)",
     "c4": "c4: 20x128 FP8-e4m3 tower (bf16 heads) batch 4096, 73-plane policy + tanh value",
     "c4b": "c4b: c4 with residual branches scaled by 1/sqrt(20)",
+    "p12": "p12: the paper's own network, 12x128 bf16 batch 1024 (52 planes, capped scaled blocks, pooled context, "
+           "query-key policy over 1,880 actions, WDL value)",
 }
+
+
+def is_pnet(cfg) -> bool:
+    return cfg.in_planes == 52
+
+
+def get_config(name: str):
+    return pnet_weights.PNET_CONFIGS[name] if name in pnet_weights.PNET_CONFIGS else configs.CONFIGS[name]
+
+
+def make_records(cfg, count, first_index=0):
+    """Position records of the workload, in the layout its network consumes."""
+    if is_pnet(cfg):
+        return positions.generate_moves(cfg.position_seed, count, cfg.plies, first_index=first_index)[0]
+    return positions.records_for_planes(cfg.in_planes, positions.for_config(cfg, count, first_index=first_index))
+
+
+def make_blob(cfg):
+    return pnet_weights.make_blob(cfg) if is_pnet(cfg) else weights.make_blob(cfg)
 DTYPE = {0: "f32", 1: "bf16", 2: "fp8_e4m3"}
 
 # DRAM bytes (read + write) of one tower-kernel launch, from the ncu capture summarised in
 # profiles/tower_tc_kernel_c3_batch592.md: 12.06 MB at batch 592, of which 11.87 MB are the weights
 # (read once whatever the batch) and the rest the 104-byte position records.
 def tower_traffic_bytes(cfg, batch):
-    if cfg.channels != 128 or cfg.blocks != 20 or cfg.precision != 1:
+    if is_pnet(cfg) or cfg.channels != 128 or cfg.blocks != 20 or cfg.precision != 1:
         return None             # no capture yet for other shapes / the FP8 tower
     return 12.06e6 + (batch - 592) * 104.0
 
@@ -47,6 +68,11 @@ def tower_traffic_bytes(cfg, batch):
 def tower_flops_per_position(cfg) -> float:
     """Dense convolution count 2*64*9*Cin*Cout per layer; channel padding is not counted."""
     c = cfg.channels
+    if is_pnet(cfg):
+        # second convolutions of the pooled blocks (1, 3, 5, ...) read 3C/4 channels; the fused query/key
+        # layer (a 1x1 convolution C -> 256) is part of the kernel's work
+        pooled = cfg.blocks // 2
+        return 2.0 * 64 * (9 * (cfg.in_planes * c + (2 * cfg.blocks - pooled) * c * c + pooled * c * (3 * c // 4)) + c * 256)
     return 2.0 * 64 * 9 * (cfg.in_planes * c + 2 * cfg.blocks * c * c)
 
 
@@ -118,7 +144,10 @@ def oracle_rate(cfg, blob, recs, sample: int):
     import oracle
     sub = recs[:sample]
     t0 = time.perf_counter()
-    oracle.evaluate(blob, sub, cfg.in_planes, cfg.policy_head)
+    if is_pnet(cfg):
+        oracle.pnet_evaluate(blob, sub)
+    else:
+        oracle.evaluate(blob, sub, cfg.in_planes, cfg.policy_head)
     dt = time.perf_counter() - t0
     return sub.shape[0] / dt, dt, oracle.threads()
 
@@ -128,8 +157,8 @@ def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    blob = weights.make_blob(cfg)
-    recs = positions.records_for_planes(cfg.in_planes, positions.for_config(cfg))
+    blob = make_blob(cfg)
+    recs = make_records(cfg, cfg.batch)
     sample = min(cfg.batch, 128)
     for _ in range(args.warmup):
         oracle_rate(cfg, blob, recs, min(sample, 16))
@@ -163,7 +192,7 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    cfg = configs.CONFIGS[args.config]
+    cfg = get_config(args.config)
     if args.batch > 0:
         import dataclasses
         cfg = dataclasses.replace(cfg, batch=args.batch)
@@ -186,9 +215,8 @@ def main():
 
     # ---- inputs: every rank evaluates its own batch of the same stream (weak scaling)
     B = cfg.batch
-    rec = positions.for_config(cfg, B, first_index=sharding.rank_first_index(rank, B))
-    recs = positions.records_for_planes(cfg.in_planes, rec)
-    blob = weights.make_blob(cfg)
+    recs = make_records(cfg, B, first_index=sharding.rank_first_index(rank, B))
+    blob = make_blob(cfg)
     arch = az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, B)
     net = az.az_load_net(arch, blob)
     if cfg.precision == 2:      # FP8 tower: fix the activation ranges on the seeded calibration positions first

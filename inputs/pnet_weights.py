@@ -39,6 +39,15 @@ class PNetConfig:
     value_hidden: int = 48
     plies: tuple = (0, 160)
 
+    # the same vocabulary as the other workloads' Config, so that callers can treat both alike
+    in_planes = PLANES
+    policy_head = 2
+    value_head = 1
+    precision = 1
+    policy_size = ACTIONS
+    value_size = 3
+    mask_words = MASK_WORDS
+
 
 # the paper's network ladder (App. D.3): 12 x 128 and 14 x 160 (the reported checkpoint's size)
 PNET_CONFIGS = {

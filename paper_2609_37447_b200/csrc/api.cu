@@ -414,10 +414,7 @@ static int evaluate_impl(az_net *net, const void *positions_dev, const uint64_t 
     void *h = nullptr;
     int rc = az::run_tower(*n, positions_dev, batch, &h, n->tc_ready, s);
     if (rc != AZ_OK) return rc;
-    if (n->pnet) {
-        if (!dense) return AZ_ERR_UNSUPPORTED;
-        return az::launch_pnet_finish(*n, legal_masks_dev, batch, policy_dev, value_dev, s);
-    }
+    if (n->pnet) return az::launch_pnet_finish(*n, legal_masks_dev, batch, policy_dev, legal_dev, counts_dev, value_dev, s);
     if (n->tc_ready) {
         // the tower kernel has produced the 73-plane logits or the flat head's projection, and the value
         // projection; one GEMM launch finishes both heads, the softmax follows

@@ -105,7 +105,7 @@ struct Net {
 
     // ---- the paper's own network (52 planes, pooled context, query-key policy head) ----
     bool pnet = false;
-    float *pnet_gw = nullptr;         // [pooled block][3C/4][C/2]
+    float *pnet_gw = nullptr;         // [pooled block][C/2][3C/4] (transposed)
     void *pnet_qk = nullptr;          // [max_batch][64][256] fp32: queries | keys
     float *pnet_small = nullptr;      // the finishing kernel's fp32 parameters, see pnet.cu
     unsigned char *pnet_actions = nullptr;   // [1880][4]: origin, destination, promotion piece + 1 (0 none), pad
@@ -146,7 +146,8 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 // ---- kernels' launch functions (each returns AZ_OK or AZ_ERR_CUDA) ---------------------------
 int launch_encode52(const void *positions, int batch, bool bf16, void *planes, cudaStream_t s);
 int build_pnet(Net &n, const unsigned char *blob, size_t nbytes);
-int launch_pnet_finish(const Net &n, const uint64_t *masks, int batch, float *policy, float *value, cudaStream_t s);
+int launch_pnet_finish(const Net &n, const uint64_t *masks, int batch, float *policy, float *legal, int *counts,
+                       float *value, cudaStream_t s);
 size_t tc_packed_layers_bytes(const int *cin_pad, int channels, int n_conv);
 void tc_pack_layers(const float *const *w, const float *const *scale, const int *cin, const int *cin_pad,
                     int channels, int n_conv, __nv_bfloat16 *packed);

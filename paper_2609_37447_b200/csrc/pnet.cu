@@ -91,6 +91,7 @@ __global__ void __launch_bounds__(kFinishThreads)
 pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict__ qk,
                    const uint64_t *__restrict__ masks, const float *__restrict__ small,
                    const uchar4 *__restrict__ actions, int batch, float *__restrict__ policy,
+                   float *__restrict__ legal, int *__restrict__ counts,
                    float *__restrict__ value, uint32_t *__restrict__ status) {
     ptx::grid_dependency_wait();                     // the tower's outputs must be complete
     const int pos = blockIdx.x, tid = threadIdx.x;
@@ -157,10 +158,28 @@ pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict_
         sum = 1.0f;
     }
     const float inv = 1.0f / sum;
+    if (policy != nullptr) {
 #pragma unroll
-    for (int j = 0; j < kPerThread; ++j) {
-        const int i = tid + j * kFinishThreads;
-        if (i < kActions) policy[(size_t)pos * kActions + i] = lg[j] * inv;
+        for (int j = 0; j < kPerThread; ++j) {
+            const int i = tid + j * kFinishThreads;
+            if (i < kActions) policy[(size_t)pos * kActions + i] = lg[j] * inv;
+        }
+    } else {
+        // legal actions only, in ascending action index: an action's place is the number of legal ones before it
+        const uint64_t *row = masks + (size_t)pos * 30;
+#pragma unroll
+        for (int j = 0; j < kPerThread; ++j) {
+            const int i = tid + j * kFinishThreads;
+            if (i >= kActions || !((row[i >> 6] >> (i & 63)) & 1ull)) continue;
+            int place = __popcll(row[i >> 6] & ((1ull << (i & 63)) - 1ull));
+            for (int w = 0; w < (i >> 6); ++w) place += __popcll(row[w]);
+            if (place < AZ_MAX_LEGAL) legal[(size_t)pos * AZ_MAX_LEGAL + place] = lg[j] * inv;
+        }
+        if (tid == 0) {
+            int n = 0;
+            for (int w = 0; w < 30; ++w) n += __popcll(row[w]);
+            counts[pos] = n < AZ_MAX_LEGAL ? n : AZ_MAX_LEGAL;
+        }
     }
 }
 
@@ -259,7 +278,9 @@ int build_pnet(Net &n, const unsigned char *blob, size_t nbytes) {
     // pooled-context maps of blocks 1, 3, 5, ...
     {
         std::vector<float> gw;
-        for (int b = 1; b < L; b += 2) gw.insert(gw.end(), v.gw[b], v.gw[b] + (size_t)R * 2 * P);
+        for (int b = 1; b < L; b += 2)                       // stored transposed: [entry of the pooled vector][output]
+            for (int j = 0; j < 2 * P; ++j)
+                for (int r = 0; r < R; ++r) gw.push_back(v.gw[b][(size_t)r * 2 * P + j]);
         if (gw.empty()) gw.push_back(0.0f);
         AZ_CUDA(cudaMalloc((void **)&n.pnet_gw, gw.size() * sizeof(float)));
         AZ_CUDA(cudaMemcpy(n.pnet_gw, gw.data(), gw.size() * sizeof(float), cudaMemcpyHostToDevice));
@@ -328,12 +349,13 @@ int build_pnet(Net &n, const unsigned char *blob, size_t nbytes) {
     return AZ_OK;
 }
 
-int launch_pnet_finish(const Net &n, const uint64_t *masks, int batch, float *policy, float *value, cudaStream_t s) {
+int launch_pnet_finish(const Net &n, const uint64_t *masks, int batch, float *policy, float *legal, int *counts,
+                       float *value, cudaStream_t s) {
     if (batch == 0) return AZ_OK;
     AZ_CUDA(launch_dependent(pnet_finish_kernel, dim3((unsigned)batch), dim3(kFinishThreads), 0, s,
                              static_cast<const __nv_bfloat16 *>(n.act[0]), static_cast<const float *>(n.pnet_qk), masks,
                              static_cast<const float *>(n.pnet_small), reinterpret_cast<const uchar4 *>(n.pnet_actions), batch,
-                             policy, value, n.status_dev));
+                             policy, legal, counts, value, n.status_dev));
     return AZ_OK;
 }
 

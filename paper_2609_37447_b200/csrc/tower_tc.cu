@@ -122,7 +122,7 @@ struct TowerArgs {
     unsigned int *absmax;            // [n_conv][C]
     // the paper's own network (kPnet instantiation; Sec. 3.2, 4.3.3, 4.3.6, App. D.1): activations capped
     // at six, pooled context in blocks 1, 3, 5, ..., query / key projections as the fused head layer
-    const float *gw;                 // [pooled block][3C/4][C/2] fp32: pooled vector -> context
+    const float *gw;                 // [pooled block][C/2][3C/4] fp32, transposed: pooled vector -> context
     float *qk_out;                   // [batch][64][256] fp32: queries (128) then keys (128) per square
 };
 
@@ -449,6 +449,15 @@ tower_tc_kernel(const TowerArgs args) {
         uint32_t pool_phase = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
+        if (kPnet) {
+            // the pooled-context maps are read in the middle of a layer's hand-over, where a miss to DRAM would
+            // sit on the critical path: ask for all of them now (148 CTAs ask for the same lines; L2 merges them)
+            const int n_pooled = (n_conv - 1) / 4;
+            const char *gwb = reinterpret_cast<const char *>(args.gw);
+            const size_t bytes = (size_t)n_pooled * kRegC * 2 * kPoolC * sizeof(float);
+            for (size_t off = (size_t)(ew * 32 + lane) * 128; off < bytes; off += (size_t)S::kEpiWarps * 32 * 128)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(gwb + off));
+        }
         for (int r = 0; ok; ++r) {
             const Round rd = round_of(r);
             if (!rd.valid) break;
@@ -524,25 +533,43 @@ tower_tc_kernel(const TowerArgs args) {
                     // ---- pooled context (Sec. 3.2, 4.3.3): the last C/4 channels of this first convolution are
                     // activated, averaged and maximised over each board's 64 squares, mapped to 3C/4 values and
                     // added to the other channels before THEIR activation.
-                    // (1) this warp's 32 rows: 16 of board 0 (lanes with bit 3 clear) and 16 of board 1
+                    // (1) this warp's 32 rows: 16 of board 0 (lanes with bit 3 clear) and 16 of board 1.  Sixteen
+                    // channels are reduced over eight lanes by a halving butterfly (a lane passes on the half of its
+                    // values that its partner keeps): 8 + 4 + 2 exchanges, after which lane k of each eight holds
+                    // channels 2k', 2k'+1 (k' = k with its bits reversed); one more exchange joins the board's two
+                    // row groups.  Sums and maxima travel together.
 #pragma unroll
                     for (int ps = 0; ps < kPoolC / 16; ++ps) {
                         ptx::tmem_ld16(t_src + (uint32_t)(kRegC + ps * 16), r[0]);
                         ptx::tmem_ld_wait();
+                        float sm[16], mx[16];
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
-                            const float a = live ? fminf(fmaxf(__uint_as_float(r[0][i]) + bias[kRegC + ps * 16 + i], 0.0f), 6.0f) : 0.0f;
-                            float sm = a, mx = a;
+                            sm[i] = live ? fminf(fmaxf(__uint_as_float(r[0][i]) + bias[kRegC + ps * 16 + i], 0.0f), 6.0f) : 0.0f;
+                            mx[i] = sm[i];
+                        }
 #pragma unroll
-                            for (int o = 1; o <= 16; o <<= 1) {
-                                if (o == 8) continue;                          // bit 3 of the lane tells the boards apart
-                                sm += __shfl_xor_sync(0xffffffffu, sm, o);
-                                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+                        for (int step = 0; step < 3; ++step) {
+                            const int half = 8 >> step;                    // values kept after this step
+                            const bool upper = (lane >> step) & 1;         // this lane keeps the upper half
+#pragma unroll
+                            for (int i = 0; i < half; ++i) {
+                                const float give_s = upper ? sm[i] : sm[half + i], keep_s = upper ? sm[half + i] : sm[i];
+                                const float give_m = upper ? mx[i] : mx[half + i], keep_m = upper ? mx[half + i] : mx[i];
+                                sm[i] = keep_s + __shfl_xor_sync(0xffffffffu, give_s, 1 << step);
+                                mx[i] = fmaxf(keep_m, __shfl_xor_sync(0xffffffffu, give_m, 1 << step));
                             }
-                            if ((lane & 23) == 0) {                            // lanes 0 and 8: one per board
-                                pool_part[(q * 2 + b) * kPoolC + ps * 16 + i] = sm;
-                                pool_part[4 * 2 * kPoolC + (q * 2 + b) * kPoolC + ps * 16 + i] = mx;
-                            }
+                        }
+                        // sm[0], mx[0] now cover channel c0 = 8*(lane&1) + 4*((lane>>1)&1) + 2*((lane>>2)&1), sm[1], mx[1] c0 + 1
+                        sm[0] += __shfl_xor_sync(0xffffffffu, sm[0], 16);
+                        sm[1] += __shfl_xor_sync(0xffffffffu, sm[1], 16);
+                        mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], 16));
+                        mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], 16));
+                        if (lane < 16) {                                   // lanes 0-7 board 0, lanes 8-15 board 1
+                            const int c0 = ps * 16 + 8 * (lane & 1) + 4 * ((lane >> 1) & 1) + 2 * ((lane >> 2) & 1);
+                            float *ds = pool_part + (q * 2 + b) * kPoolC + c0;
+                            ds[0] = sm[0]; ds[1] = sm[1];
+                            ds[4 * 2 * kPoolC] = mx[0]; ds[4 * 2 * kPoolC + 1] = mx[1];
                         }
                     }
                     auto meet = [&]() -> bool {                                // the group's four warps, bounded
@@ -569,21 +596,21 @@ tower_tc_kernel(const TowerArgs args) {
                     }
                     ok = meet();
                     if (!ok) break;
-                    // (3) context = gw . pooled vector: 2 boards x 3C/4 outputs over the group's 128 threads
+                    // (3) context = gw . pooled vector: 2 boards x 3C/4 outputs over the group's 128 threads.  The map
+                    // is stored transposed, [entry of the pooled vector][output], so that neighbouring threads read
+                    // neighbouring words.
                     {
-                        const float *gw = args.gw + (size_t)((l - 3) >> 2) * kRegC * 2 * kPoolC;
+                        const float *gwt = args.gw + (size_t)((l - 3) >> 2) * kRegC * 2 * kPoolC;
                         for (int e = q * 32 + lane; e < 2 * kRegC; e += 128) {
                             const int pb = e / kRegC, rr0 = e % kRegC;
-                            const float4 *wrow = reinterpret_cast<const float4 *>(gw + (size_t)rr0 * 2 * kPoolC);
-                            const float4 *vec = reinterpret_cast<const float4 *>(pool_vec + pb * 2 * kPoolC);
-                            float acc = 0.0f;
-#pragma unroll
-                            for (int j = 0; j < 2 * kPoolC / 4; ++j) {
-                                const float4 wv = __ldg(wrow + j), pv = vec[j];
-                                acc = fmaf(wv.x, pv.x, acc); acc = fmaf(wv.y, pv.y, acc);
-                                acc = fmaf(wv.z, pv.z, acc); acc = fmaf(wv.w, pv.w, acc);
+                            const float *vec = pool_vec + pb * 2 * kPoolC;
+                            float acc0 = 0.0f, acc1 = 0.0f;
+#pragma unroll 16
+                            for (int j = 0; j < 2 * kPoolC; j += 2) {
+                                acc0 = fmaf(__ldg(gwt + (size_t)j * kRegC + rr0), vec[j], acc0);
+                                acc1 = fmaf(__ldg(gwt + (size_t)(j + 1) * kRegC + rr0), vec[j + 1], acc1);
                             }
-                            pool_ctx[pb * kRegC + rr0] = acc;
+                            pool_ctx[pb * kRegC + rr0] = acc0 + acc1;
                         }
                     }
                     ok = meet();
