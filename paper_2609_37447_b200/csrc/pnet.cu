@@ -70,7 +70,6 @@ __device__ __forceinline__ float dot128_f32_bf16(const float *w, const __nv_bflo
 }
 
 constexpr int kFinishThreads = 128;
-constexpr int kPerThread = (kActions + kFinishThreads - 1) / kFinishThreads;   // 15
 
 __device__ __forceinline__ float block_reduce(float v, bool is_max, float *scratch) {
 #pragma unroll
@@ -87,16 +86,37 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float *scrat
     return r;
 }
 
+// One CTA per position.  The legal actions are first listed (ascending action index, which is also
+// the order of the legal-moves-only output), then each gets a thread for its 128-long dot product.
 __global__ void __launch_bounds__(kFinishThreads)
 pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict__ qk,
                    const uint64_t *__restrict__ masks, const float *__restrict__ small,
                    const uchar4 *__restrict__ actions, int batch, float *__restrict__ policy,
                    float *__restrict__ legal, int *__restrict__ counts,
                    float *__restrict__ value, uint32_t *__restrict__ status) {
-    ptx::grid_dependency_wait();                     // the tower's outputs must be complete
     const int pos = blockIdx.x, tid = threadIdx.x;
-    if (pos >= batch) return;
-    __shared__ float v_s[kVC * 64], hid_s[kVH], red[kFinishThreads / 32];
+    __shared__ float v_s[kVC * 64], hid_s[kVH], red[kFinishThreads / 32], lg_s[AZ_MAX_LEGAL];
+    __shared__ unsigned short list_s[AZ_MAX_LEGAL];
+    __shared__ int first_s[31];
+    // ---- the legal actions, from the mask alone (before the tower's results are needed)
+    const uint64_t *row = masks + (size_t)pos * 30;
+    if (tid < 30) first_s[tid + 1] = __popcll(row[tid]);
+    __syncthreads();
+    if (tid == 0) {
+        first_s[0] = 0;
+        for (int w = 1; w <= 30; ++w) first_s[w] += first_s[w - 1];
+    }
+    __syncthreads();
+    const int n_legal = min(first_s[30], AZ_MAX_LEGAL);
+    if (tid < 30) {
+        uint64_t bits = row[tid];
+        int at = first_s[tid];
+        while (bits && at < AZ_MAX_LEGAL) {
+            list_s[at++] = (unsigned short)(tid * 64 + __ffsll((long long)bits) - 1);
+            bits &= bits - 1;
+        }
+    }
+    ptx::grid_dependency_wait();                     // from here on the tower's outputs are read
     const __nv_bfloat16 *hp = h + (size_t)pos * 64 * 128;
     const float *qkp = qk + (size_t)pos * 64 * 256;
 
@@ -108,13 +128,25 @@ pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict_
     }
     __syncthreads();
     if (tid < kVH) {
-        const float *w = small + Small::v_w1 + tid * (kVC * 64);
-        float acc = small[Small::v_b1 + tid];
-#pragma unroll 8
-        for (int i = 0; i < kVC * 64; ++i) acc = fmaf(w[i], v_s[i], acc);
-        hid_s[tid] = fmaxf(acc, 0.0f);
+        const float *w = small + Small::v_w1 + tid;  // stored [input][hidden unit]: neighbouring threads, neighbouring words
+        float acc0 = small[Small::v_b1 + tid], acc1 = 0.0f;
+#pragma unroll 16
+        for (int i = 0; i < kVC * 64; i += 2) {
+            acc0 = fmaf(__ldg(w + i * kVH), v_s[i], acc0);
+            acc1 = fmaf(__ldg(w + (i + 1) * kVH), v_s[i + 1], acc1);
+        }
+        hid_s[tid] = fmaxf(acc0 + acc1, 0.0f);
     }
-    __syncthreads();
+    // ---- policy: one thread per legal action
+    float mx = -INFINITY;
+    for (int t = tid; t < n_legal; t += kFinishThreads) {
+        const uchar4 a = actions[list_s[t]];                                   // origin, destination, piece + 1
+        float s = dot128_f32(qkp + a.x * 256, qkp + a.y * 256 + 128);
+        if (a.z) s += dot128_f32_bf16(small + Small::o_w + (a.z - 1) * 128, hp + a.x * 128) + small[Small::o_b + a.z - 1];
+        lg_s[t] = s;
+        mx = fmaxf(mx, s);
+    }
+    mx = block_reduce(mx, true, red);                                      // (its barriers also publish hid_s and lg_s)
     if (tid == 0) {
         float z[3], m = -INFINITY, sum = 0.0f;
 #pragma unroll
@@ -129,57 +161,26 @@ pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict_
 #pragma unroll
         for (int c = 0; c < 3; ++c) value[(size_t)pos * 3 + c] = z[c] / sum;
     }
-
-    // ---- policy: logits of the legal actions, softmax over them
-    float lg[kPerThread];
-    float mx = -INFINITY;
-#pragma unroll
-    for (int j = 0; j < kPerThread; ++j) {
-        const int i = tid + j * kFinishThreads;
-        lg[j] = -INFINITY;
-        if (i < kActions && ((masks[(size_t)pos * 30 + (i >> 6)] >> (i & 63)) & 1ull)) {
-            const uchar4 a = actions[i];                                   // origin, destination, piece + 1
-            float s = dot128_f32(qkp + a.x * 256, qkp + a.y * 256 + 128);
-            if (a.z) s += dot128_f32_bf16(small + Small::o_w + (a.z - 1) * 128, hp + a.x * 128) + small[Small::o_b + a.z - 1];
-            lg[j] = s;
-            mx = fmaxf(mx, s);
-        }
-    }
-    mx = block_reduce(mx, true, red);
     float sum = 0.0f;
-#pragma unroll
-    for (int j = 0; j < kPerThread; ++j) {
-        lg[j] = lg[j] == -INFINITY ? 0.0f : __expf(lg[j] - mx);
-        sum += lg[j];
+    for (int t = tid; t < n_legal; t += kFinishThreads) {
+        const float e = __expf(lg_s[t] - mx);
+        lg_s[t] = e;
+        sum += e;
     }
     sum = block_reduce(sum, false, red);
-    if (!(sum > 0.0f)) {                                                   // no legal action: an all-zero row and a status bit
+    if (n_legal == 0) {                                                    // no legal action: an all-zero row and a status bit
         if (tid == 0) atomicOr(status, kStatusEmptyMask);
         sum = 1.0f;
     }
     const float inv = 1.0f / sum;
     if (policy != nullptr) {
-#pragma unroll
-        for (int j = 0; j < kPerThread; ++j) {
-            const int i = tid + j * kFinishThreads;
-            if (i < kActions) policy[(size_t)pos * kActions + i] = lg[j] * inv;
-        }
+        float *out = policy + (size_t)pos * kActions;
+        for (int i = tid; i < kActions / 4; i += kFinishThreads) reinterpret_cast<float4 *>(out)[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        __syncthreads();
+        for (int t = tid; t < n_legal; t += kFinishThreads) out[list_s[t]] = lg_s[t] * inv;
     } else {
-        // legal actions only, in ascending action index: an action's place is the number of legal ones before it
-        const uint64_t *row = masks + (size_t)pos * 30;
-#pragma unroll
-        for (int j = 0; j < kPerThread; ++j) {
-            const int i = tid + j * kFinishThreads;
-            if (i >= kActions || !((row[i >> 6] >> (i & 63)) & 1ull)) continue;
-            int place = __popcll(row[i >> 6] & ((1ull << (i & 63)) - 1ull));
-            for (int w = 0; w < (i >> 6); ++w) place += __popcll(row[w]);
-            if (place < AZ_MAX_LEGAL) legal[(size_t)pos * AZ_MAX_LEGAL + place] = lg[j] * inv;
-        }
-        if (tid == 0) {
-            int n = 0;
-            for (int w = 0; w < 30; ++w) n += __popcll(row[w]);
-            counts[pos] = n < AZ_MAX_LEGAL ? n : AZ_MAX_LEGAL;
-        }
+        for (int t = tid; t < n_legal; t += kFinishThreads) legal[(size_t)pos * AZ_MAX_LEGAL + t] = lg_s[t] * inv;
+        if (tid == 0) counts[pos] = n_legal;
     }
 }
 
@@ -306,7 +307,8 @@ int build_pnet(Net &n, const unsigned char *blob, size_t nbytes) {
     memcpy(&small[Small::v_cw], v.v_cw, sizeof(float) * kVC * C);
     memcpy(&small[Small::v_cs], v.v_cs, sizeof(float) * kVC);
     memcpy(&small[Small::v_cb], v.v_cb, sizeof(float) * kVC);
-    memcpy(&small[Small::v_w1], v.v_w1, sizeof(float) * kVH * kVC * 64);
+    for (int j = 0; j < kVH; ++j)                        // stored [input][hidden unit]
+        for (int i = 0; i < kVC * 64; ++i) small[Small::v_w1 + (size_t)i * kVH + j] = v.v_w1[(size_t)j * kVC * 64 + i];
     memcpy(&small[Small::v_b1], v.v_b1, sizeof(float) * kVH);
     memcpy(&small[Small::v_w2], v.v_w2, sizeof(float) * 3 * kVH);
     memcpy(&small[Small::v_b2], v.v_b2, sizeof(float) * 3);
