@@ -97,6 +97,64 @@ def test_p12_batch_1024():
         assert np.corrcoef(vg[:, k], vo[:, k])[0, 1] > 0.7
 
 
+def test_other_entry_points_serve_the_papers_network_too():
+    # legal-moves-only output, the pipelined host entry, CUDA-graph replay and the stand-alone encoder entry
+    import paper_2609_37447_b200 as az
+    cfg = pw.PNetConfig("t3", 3, 128, 48, 20260972, 4477)
+    blob = pw.make_blob(cfg, 0.1, 0.6)
+    rec, _ = positions.generate_moves(cfg.position_seed, 48, (0, 160))
+    net = load(az, cfg, blob, 64)
+    mg, pg, vg, _ = gpu_run(az, net, cfg, rec)
+    pos = az.records_to_device(rec)
+    masks = torch.from_numpy(mg.view(np.int64)).cuda()
+    legal = torch.full((48, az.AZ_MAX_LEGAL), -1.0, device="cuda")
+    counts = torch.full((48,), -1, dtype=torch.int32, device="cuda")
+    val = torch.zeros((48, 3), device="cuda")
+    az.az_evaluate_legal(net, pos, masks, 48, legal, counts, val)
+    torch.cuda.synchronize()
+    bits = np.unpackbits(mg.view(np.uint8), axis=1, bitorder="little")[:, :pw.ACTIONS].astype(bool)
+    lg, cn = legal.cpu().numpy(), counts.cpu().numpy()
+    assert (val.cpu().numpy() == vg).all()
+    for b in range(48):
+        idx = np.flatnonzero(bits[b])
+        assert cn[b] == idx.size and (lg[b, :idx.size] == pg[b, idx]).all() and (lg[b, idx.size:] == -1.0).all()
+    # pipelined host entry
+    pos_h = torch.from_numpy(np.ascontiguousarray(rec).view(np.uint8).reshape(48, -1).copy()).pin_memory()
+    masks_h = masks.cpu().pin_memory()
+    outs = [(torch.zeros((48, pw.ACTIONS)).pin_memory(), torch.zeros((48, 3)).pin_memory()) for _ in range(3)]
+    tickets = []
+    for pol_h, val_h in outs:
+        if len(tickets) == az.AZ_HOST_SLOTS:
+            az.az_wait_host(net, tickets.pop(0))
+        tickets.append(az.az_submit_host(net, pos_h, masks_h, 48, pol_h, None, None, val_h))
+    for t in tickets:
+        az.az_wait_host(net, t)
+    for pol_h, val_h in outs:
+        assert (pol_h.numpy() == pg).all() and (val_h.numpy() == vg).all()
+    # CUDA-graph replay
+    policy = torch.zeros((48, pw.ACTIONS), device="cuda")
+    value = torch.zeros((48, 3), device="cuda")
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(stream):
+        az.az_evaluate(net, pos, masks, 48, policy, value, stream=stream)
+        stream.synchronize()
+        with torch.cuda.graph(graph, stream=stream):
+            az.az_evaluate(net, pos, masks, 48, policy, value, stream=stream)
+    policy.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert (policy.cpu().numpy() == pg).all() and (value.cpu().numpy() == vg).all()
+    # az_encode of such a net is the 52-plane encoder
+    planes = torch.zeros((48, 64, 64), dtype=torch.bfloat16, device="cuda")
+    az.az_encode(net, pos, 48, planes)
+    torch.cuda.synchronize()
+    want = oracle.encode52(rec).reshape(48, 52, 64).transpose(0, 2, 1)
+    assert (planes.float().cpu().numpy()[:, :, :52] == want).all()
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
 def test_unsupported_sizes_are_refused():
     import paper_2609_37447_b200 as az
     cfg = pw.PNET_CONFIGS["p14"]
