@@ -282,12 +282,10 @@ int run_tower(Net &n, const void *positions, int batch, void **tower_out, bool f
     const int C = (int)n.arch.channels;
     const bool timed = n.profile && n.n_events < kMaxProfiledPasses;
     if (n.pnet) {
-        // the paper's network: its 52 planes come from the stand-alone encoder, the tower reads them
-        rc = launch_encode52(positions, batch, true, n.planes, s);
-        if (rc != AZ_OK) return rc;
+        // the paper's network: the tower encodes the 52 planes itself, as the other tensor-core towers do
         if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
         *tower_out = n.act[0];
-        rc = launch_tower_tc(n, n.planes, positions, batch, n.act[0], fused_heads, nullptr, s);
+        rc = launch_tower_tc(n, nullptr, positions, batch, n.act[0], fused_heads, nullptr, s);
         if (rc == AZ_OK && timed) AZ_CUDA(cudaEventRecord(n.ev_end[n.n_events++], s));
         return rc;
     }
@@ -693,6 +691,7 @@ int az_device_status(az_net *net, void *cuda_stream, uint32_t *status_out) {
 int az_launches_per_evaluate(const az_net *net, int batch) {
     const Net *n = reinterpret_cast<const Net *>(net);
     if (!n || batch <= 0) return 0;
+    if (n->pnet) return az::tower_tc_launch_count() /*encoder + tower + query/key maps*/ + 1 /*scores, softmax, value head*/;
     if (n->tc_ready) return az::tower_tc_launch_count() /*encoder + tower + head projections*/ + 1 /*head GEMMs*/ + 1 /*softmax*/;
     const int policy = n->arch.policy_head == AZ_POLICY_PLANES73 ? 1 : 2;
     return 1 /*encode*/ + n->n_conv + policy + 3 /*value*/ + 1 /*softmax*/;

@@ -474,6 +474,24 @@ tower_tc_kernel(const TowerArgs args) {
                         const uint4 v = live ? __ldg(src + j) : make_uint4(0, 0, 0, 0);
                         *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) = v;
                     }
+                } else if (kPnet) {
+                    // the paper's 52 planes (64 channels = 8 planes of the frame) from the 128-byte record
+                    const PosM8 *rec = reinterpret_cast<const PosM8 *>(args.positions + (size_t)(live ? board : 0) * args.position_stride);
+                    if (live && sq == 0 && (__popcll(rec->pieces[5]) != 1 || __popcll(rec->pieces[11]) != 1))
+                        atomicOr(args.status, kStatusBadRecord);
+                    float pv[64];
+                    planes52_square(rec, sq, pv);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const __nv_bfloat162 h2 = __floats2bfloat162_rn(pv[8 * j + 2 * i], pv[8 * j + 2 * i + 1]);
+                            w[i] = *reinterpret_cast<const uint32_t *>(&h2);
+                        }
+                        *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) =
+                            live ? make_uint4(w[0], w[1], w[2], w[3]) : make_uint4(0, 0, 0, 0);
+                    }
                 } else {
                     const PosCur *rec = reinterpret_cast<const PosCur *>(args.positions + (size_t)(live ? board : 0) * args.position_stride);
                     const int s_abs = rec->stm ? (sq ^ 56) : sq;            // reflect ranks for Black
