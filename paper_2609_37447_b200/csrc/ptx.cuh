@@ -161,6 +161,14 @@ __device__ __forceinline__ void mma_e4m3_elect(uint32_t d_tmem, uint32_t a_lo, u
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// 8 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(taddr)
+        : "memory");
+}
 // Two fp32 -> packed bf16x2 / e4m3x2 with the ReLU done by the conversion (negative inputs give +0);
 // `lo` lands in the low half.  Round to nearest even; e4m3 saturates to +-448.
 __device__ __forceinline__ uint32_t pack_bf16x2_relu(float lo, float hi) {

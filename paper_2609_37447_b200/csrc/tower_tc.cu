@@ -87,7 +87,8 @@ struct Shape {
     // per epilogue warp: the current layer's channel constants for the channels of its own slices
     // after the constants: head biases (up to 256), then the pooled-context scratch of the paper's network
     // per group: partial sums and maxima [4 warps][2 boards][C/4], pooled vector [2][C/2], context [2][3C/4]
-    static constexpr int kPoolFloats = kGroups * (2 * 4 * 2 * (kC / 4) + 2 * (kC / 2) + 2 * (3 * kC / 4));
+    static constexpr int kCtxStride = (3 * kC / 4 + 15) & ~15;      // context entries per board, padded with zeros to whole slices
+    static constexpr int kPoolFloats = kGroups * (2 * 4 * 2 * (kC / 4) + 2 * (kC / 2) + 2 * kCtxStride);
     static constexpr int smem_bytes(bool fp8, bool pnet = false) {
         return kOffConst + kEpiWarps * (fp8 ? 3 : 1) * (kC / kSets) * 4 + 256 * 4 + (pnet ? kPoolFloats * 4 : 0);
     }
@@ -234,9 +235,10 @@ tower_tc_kernel(const TowerArgs args) {
     // context, and the second convolution of those blocks (layers 4, 8, 12, ...) reads 3C/4 channels only
     auto pool_layer = [&](int l) { return kPnet && (l & 3) == 3; };
     auto short_layer = [&](int l) { return kPnet && l >= 4 && (l & 3) == 0; };
+    constexpr int kShortSlices = (3 * kC / 4 + 15) / 16;      // slices that hold the 3C/4 channels a pooled block hands on
     auto round_of = [&](int r) { return get_round<S>(r, (int)blockIdx.x, (int)gridDim.x, n_groups); };
     auto slices_of = [&](int l) {                                                               // K per MMA: 16 bf16 or 32 e4m3
-        return l == 0 ? in_slices : short_layer(l) ? 3 * kC / 64 : (kFp8 ? kC / 32 : kC / 16);
+        return l == 0 ? in_slices : short_layer(l) ? kShortSlices : (kFp8 ? kC / 32 : kC / 16);
     };
     const bool tr = args.trace && blockIdx.x == 0;
     long long t_wait[3] = {0, 0, 0};
@@ -445,7 +447,8 @@ tower_tc_kernel(const TowerArgs args) {
         constexpr int kPoolC = kC / 4, kRegC = kC - kC / 4;
         float *pool_part = head_bias_smem + 256 + g * (S::kPoolFloats / kGroups);   // [sum|max][warp q][board][kPoolC]
         float *pool_vec = pool_part + 2 * 4 * 2 * kPoolC;                          // [board][2 * kPoolC]: means, then maxima
-        float *pool_ctx = pool_vec + 2 * 2 * kPoolC;                               // [board][kRegC]
+        float *pool_ctx = pool_vec + 2 * 2 * kPoolC;                               // [board][kCtxStride], zero beyond kRegC
+        constexpr int kCtxStride = S::kCtxStride;
         uint32_t pool_phase = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -551,24 +554,25 @@ tower_tc_kernel(const TowerArgs args) {
                     // ---- pooled context (Sec. 3.2, 4.3.3): the last C/4 channels of this first convolution are
                     // activated, averaged and maximised over each board's 64 squares, mapped to 3C/4 values and
                     // added to the other channels before THEIR activation.
-                    // (1) this warp's 32 rows: 16 of board 0 (lanes with bit 3 clear) and 16 of board 1.  Sixteen
-                    // channels are reduced over eight lanes by a halving butterfly (a lane passes on the half of its
-                    // values that its partner keeps): 8 + 4 + 2 exchanges, after which lane k of each eight holds
-                    // channels 2k', 2k'+1 (k' = k with its bits reversed); one more exchange joins the board's two
-                    // row groups.  Sums and maxima travel together.
+                    // (1) this warp's 32 rows: 16 of board 0 (lanes with bit 3 clear) and 16 of board 1.  Eight
+                    // channels at a time are reduced over eight lanes by a halving butterfly (a lane passes on the
+                    // half of its values that its partner keeps): 4 + 2 + 1 exchanges, after which every lane of
+                    // the eight holds one channel; one more exchange joins the board's two row groups.  Sums and
+                    // maxima travel together.
 #pragma unroll
-                    for (int ps = 0; ps < kPoolC / 16; ++ps) {
-                        ptx::tmem_ld16(t_src + (uint32_t)(kRegC + ps * 16), r[0]);
+                    for (int pc = 0; pc < kPoolC / 8; ++pc) {
+                        uint32_t r8[8];
+                        ptx::tmem_ld8(t_src + (uint32_t)(kRegC + pc * 8), r8);
                         ptx::tmem_ld_wait();
-                        float sm[16], mx[16];
+                        float sm[8], mx[8];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            sm[i] = live ? fminf(fmaxf(__uint_as_float(r[0][i]) + bias[kRegC + ps * 16 + i], 0.0f), 6.0f) : 0.0f;
+                        for (int i = 0; i < 8; ++i) {
+                            sm[i] = live ? fminf(fmaxf(__uint_as_float(r8[i]) + bias[kRegC + pc * 8 + i], 0.0f), 6.0f) : 0.0f;
                             mx[i] = sm[i];
                         }
 #pragma unroll
                         for (int step = 0; step < 3; ++step) {
-                            const int half = 8 >> step;                    // values kept after this step
+                            const int half = 4 >> step;                    // values kept after this step
                             const bool upper = (lane >> step) & 1;         // this lane keeps the upper half
 #pragma unroll
                             for (int i = 0; i < half; ++i) {
@@ -578,16 +582,12 @@ tower_tc_kernel(const TowerArgs args) {
                                 mx[i] = fmaxf(keep_m, __shfl_xor_sync(0xffffffffu, give_m, 1 << step));
                             }
                         }
-                        // sm[0], mx[0] now cover channel c0 = 8*(lane&1) + 4*((lane>>1)&1) + 2*((lane>>2)&1), sm[1], mx[1] c0 + 1
                         sm[0] += __shfl_xor_sync(0xffffffffu, sm[0], 16);
-                        sm[1] += __shfl_xor_sync(0xffffffffu, sm[1], 16);
                         mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], 16));
-                        mx[1] = fmaxf(mx[1], __shfl_xor_sync(0xffffffffu, mx[1], 16));
                         if (lane < 16) {                                   // lanes 0-7 board 0, lanes 8-15 board 1
-                            const int c0 = ps * 16 + 8 * (lane & 1) + 4 * ((lane >> 1) & 1) + 2 * ((lane >> 2) & 1);
-                            float *ds = pool_part + (q * 2 + b) * kPoolC + c0;
-                            ds[0] = sm[0]; ds[1] = sm[1];
-                            ds[4 * 2 * kPoolC] = mx[0]; ds[4 * 2 * kPoolC + 1] = mx[1];
+                            const int c0 = pc * 8 + 4 * (lane & 1) + 2 * ((lane >> 1) & 1) + ((lane >> 2) & 1);
+                            pool_part[(q * 2 + b) * kPoolC + c0] = sm[0];
+                            pool_part[4 * 2 * kPoolC + (q * 2 + b) * kPoolC + c0] = mx[0];
                         }
                     }
                     auto meet = [&]() -> bool {                                // the group's four warps, bounded
@@ -600,9 +600,8 @@ tower_tc_kernel(const TowerArgs args) {
                     ok = meet();
                     if (!ok) break;
                     // (2) the four warps' partial results -> the pooled vector: one entry per thread
-                    {
-                        const int e = q * 32 + lane;                           // 0..127 = board * 64 + entry
-                        const int pb = e >> 6, j = e & 63, c = j % kPoolC;
+                    for (int e = q * 32 + lane; e < 2 * 2 * kPoolC; e += 128) {   // e = board * 2 * kPoolC + entry
+                        const int pb = e / (2 * kPoolC), j = e % (2 * kPoolC), c = j % kPoolC;
                         const float *src = pool_part + (j >= kPoolC ? 4 * 2 * kPoolC : 0);
                         float acc = src[(0 * 2 + pb) * kPoolC + c];
 #pragma unroll
@@ -612,6 +611,9 @@ tower_tc_kernel(const TowerArgs args) {
                         }
                         pool_vec[pb * 2 * kPoolC + j] = j >= kPoolC ? acc : acc * (1.0f / 64.0f);
                     }
+                    if (kCtxStride > kRegC)                                    // the padding of the context stays zero
+                        for (int z = q * 32 + lane; z < 2 * (kCtxStride - kRegC); z += 128)
+                            pool_ctx[(z / (kCtxStride - kRegC)) * kCtxStride + kRegC + z % (kCtxStride - kRegC)] = 0.0f;
                     ok = meet();
                     if (!ok) break;
                     // (3) context = gw . pooled vector: 2 boards x 3C/4 outputs over the group's 128 threads.  The map
@@ -628,14 +630,14 @@ tower_tc_kernel(const TowerArgs args) {
                                 acc0 = fmaf(__ldg(gwt + (size_t)j * kRegC + rr0), vec[j], acc0);
                                 acc1 = fmaf(__ldg(gwt + (size_t)(j + 1) * kRegC + rr0), vec[j + 1], acc1);
                             }
-                            pool_ctx[pb * kRegC + rr0] = acc0 + acc1;
+                            pool_ctx[pb * kCtxStride + rr0] = acc0 + acc1;
                         }
                     }
                     ok = meet();
                     if (!ok) break;
                 }
-                const float *ctx = pool_ctx + b * kRegC;                       // this row's board
-                const int n_my = (kPnet && pooled) ? kRegC / 16 : kMySlices;   // the pooled channels are not handed on
+                const float *ctx = pool_ctx + b * kCtxStride;                  // this row's board
+                const int n_my = (kPnet && pooled) ? kShortSlices : kMySlices; // the pooled channels are not handed on
                 ptx::tmem_ld16(t_src + (uint32_t)(set * 16), r[0]);
 #pragma unroll
                 for (int ks = 0; ks < kMySlices; ++ks) {
