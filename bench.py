@@ -34,6 +34,8 @@ WORKLOADS = {
     "c4b": "c4b: c4 with residual branches scaled by 1/sqrt(20)",
     "p12": "p12: the paper's own network, 12x128 bf16 batch 1024 (52 planes, capped scaled blocks, pooled context, "
            "query-key policy over 1,880 actions, WDL value)",
+    "p14": "p14: the paper's own network at its reported size, 14x160 bf16, batch 320 as the paper serves it "
+           "(App. D.3); --batch for other sizes",
 }
 
 

@@ -341,8 +341,8 @@ int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az
     *out = nullptr;
     if (!az::arch_ok(*arch)) return AZ_ERR_BAD_ARCH;
     const bool pnet = arch->in_planes == 52;
-    // of the paper's network ladder the 128-channel size is built, in bf16
-    if (pnet && (arch->channels != 128 || arch->precision != AZ_PREC_BF16)) return AZ_ERR_UNSUPPORTED;
+    // of the paper's network ladder the 128- and 160-channel sizes are built, in bf16
+    if (pnet && ((arch->channels != 128 && arch->channels != 160) || arch->precision != AZ_PREC_BF16)) return AZ_ERR_UNSUPPORTED;
     az::BlobView view;
     int rc = AZ_OK;
     if (!pnet) rc = az::parse_blob(*arch, static_cast<const unsigned char *>(weights_host), nbytes, view);

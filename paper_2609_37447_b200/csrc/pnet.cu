@@ -27,18 +27,21 @@ namespace {
 
 constexpr int kPlanes52 = 52, kActions = 1880, kKey = 128, kVC = 2, kVH = 48;
 
-// offsets (in floats) into Net::pnet_small
+// offsets (in floats) into Net::pnet_small for a backbone of C channels
 struct Small {
-    static constexpr int o_w = 0;                       // [4][C]
-    static constexpr int o_b = o_w + 4 * 128;           // [4]
-    static constexpr int v_cw = o_b + 4;                // [2][C]
-    static constexpr int v_cs = v_cw + kVC * 128;       // [2]
-    static constexpr int v_cb = v_cs + kVC;             // [2]
-    static constexpr int v_w1 = v_cb + kVC;             // [48][128]
-    static constexpr int v_b1 = v_w1 + kVH * kVC * 64;  // [48]
-    static constexpr int v_w2 = v_b1 + kVH;             // [3][48]
-    static constexpr int v_b2 = v_w2 + 3 * kVH;         // [3]
-    static constexpr int total = v_b2 + 3;
+    int o_w, o_b, v_cw, v_cs, v_cb, v_w1, v_b1, v_w2, v_b2, total;
+    __host__ __device__ explicit Small(int C) {
+        o_w = 0;                        // [4][C]
+        o_b = o_w + 4 * C;              // [4]
+        v_cw = o_b + 4;                 // [2][C]
+        v_cs = v_cw + kVC * C;          // [2]
+        v_cb = v_cs + kVC;              // [2]
+        v_w1 = v_cb + kVC;              // [128][48] (input-major)
+        v_b1 = v_w1 + kVH * kVC * 64;   // [48]
+        v_w2 = v_b1 + kVH;              // [3][48]
+        v_b2 = v_w2 + 3 * kVH;          // [3]
+        total = v_b2 + 3;
+    }
 };
 
 __device__ __forceinline__ float dot128_f32(const float *a, const float *b) {
@@ -52,11 +55,12 @@ __device__ __forceinline__ float dot128_f32(const float *a, const float *b) {
     }
     return acc;
 }
-__device__ __forceinline__ float dot128_f32_bf16(const float *w, const __nv_bfloat16 *h) {
+// fp32 weights . bf16 features, n a multiple of 8
+__device__ __forceinline__ float dot_f32_bf16(const float *w, const __nv_bfloat16 *h, int n) {
     const uint4 *ph = reinterpret_cast<const uint4 *>(h);
     float acc = 0.0f;
 #pragma unroll 4
-    for (int i = 0; i < 16; ++i) {
+    for (int i = 0; i < n / 8; ++i) {
         const uint4 y = __ldg(ph + i);
         const uint32_t ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
@@ -91,10 +95,11 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float *scrat
 __global__ void __launch_bounds__(kFinishThreads)
 pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict__ qk,
                    const uint64_t *__restrict__ masks, const float *__restrict__ small,
-                   const uchar4 *__restrict__ actions, int batch, float *__restrict__ policy,
+                   const uchar4 *__restrict__ actions, int batch, int C, float *__restrict__ policy,
                    float *__restrict__ legal, int *__restrict__ counts,
                    float *__restrict__ value, uint32_t *__restrict__ status) {
     const int pos = blockIdx.x, tid = threadIdx.x;
+    const Small S(C);
     __shared__ float v_s[kVC * 64], hid_s[kVH], red[kFinishThreads / 32], lg_s[AZ_MAX_LEGAL];
     __shared__ unsigned short list_s[AZ_MAX_LEGAL];
     __shared__ int first_s[31];
@@ -117,19 +122,19 @@ pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict_
         }
     }
     ptx::grid_dependency_wait();                     // from here on the tower's outputs are read
-    const __nv_bfloat16 *hp = h + (size_t)pos * 64 * 128;
+    const __nv_bfloat16 *hp = h + (size_t)pos * 64 * C;
     const float *qkp = qk + (size_t)pos * 64 * 256;
 
     // ---- value head
     {
         const int c = tid >> 6, sq = tid & 63;
-        const float d = dot128_f32_bf16(small + Small::v_cw + c * 128, hp + sq * 128);
-        v_s[c * 64 + sq] = fmaxf(fmaf(small[Small::v_cs + c], d, small[Small::v_cb + c]), 0.0f);
+        const float d = dot_f32_bf16(small + S.v_cw + c * C, hp + sq * C, C);
+        v_s[c * 64 + sq] = fmaxf(fmaf(small[S.v_cs + c], d, small[S.v_cb + c]), 0.0f);
     }
     __syncthreads();
     if (tid < kVH) {
-        const float *w = small + Small::v_w1 + tid;  // stored [input][hidden unit]: neighbouring threads, neighbouring words
-        float acc0 = small[Small::v_b1 + tid], acc1 = 0.0f;
+        const float *w = small + S.v_w1 + tid;       // stored [input][hidden unit]: neighbouring threads, neighbouring words
+        float acc0 = small[S.v_b1 + tid], acc1 = 0.0f;
 #pragma unroll 16
         for (int i = 0; i < kVC * 64; i += 2) {
             acc0 = fmaf(__ldg(w + i * kVH), v_s[i], acc0);
@@ -142,7 +147,7 @@ pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict_
     for (int t = tid; t < n_legal; t += kFinishThreads) {
         const uchar4 a = actions[list_s[t]];                                   // origin, destination, piece + 1
         float s = dot128_f32(qkp + a.x * 256, qkp + a.y * 256 + 128);
-        if (a.z) s += dot128_f32_bf16(small + Small::o_w + (a.z - 1) * 128, hp + a.x * 128) + small[Small::o_b + a.z - 1];
+        if (a.z) s += dot_f32_bf16(small + S.o_w + (a.z - 1) * C, hp + a.x * C, C) + small[S.o_b + a.z - 1];
         lg_s[t] = s;
         mx = fmaxf(mx, s);
     }
@@ -151,8 +156,8 @@ pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict_
         float z[3], m = -INFINITY, sum = 0.0f;
 #pragma unroll
         for (int c = 0; c < 3; ++c) {
-            float acc = small[Small::v_b2 + c];
-            for (int j = 0; j < kVH; ++j) acc = fmaf(small[Small::v_w2 + c * kVH + j], hid_s[j], acc);
+            float acc = small[S.v_b2 + c];
+            for (int j = 0; j < kVH; ++j) acc = fmaf(small[S.v_w2 + c * kVH + j], hid_s[j], acc);
             z[c] = acc;
             m = fmaxf(m, acc);
         }
@@ -245,8 +250,8 @@ void compose(const float *m, const float *b, int rows, const float *t_w, const f
 
 }  // namespace
 
-// Builds the device side of a paper-network az_net: 128 channels, bf16 (other sizes of the paper's
-// ladder are not built yet and are refused by the caller).
+// Builds the device side of a paper-network az_net: 128 or 160 channels, bf16 (the caller refuses
+// other sizes).
 int build_pnet(Net &n, const unsigned char *blob, size_t nbytes) {
     const az_arch &a = n.arch;
     PBlob v;
@@ -266,7 +271,7 @@ int build_pnet(Net &n, const unsigned char *blob, size_t nbytes) {
     for (int b = 0; b < L; ++b) {
         w.push_back(v.w1[b]); s.push_back(v.s1[b]); cin.push_back(C); cin_pad.push_back(C);
         memcpy(&bias[(size_t)(1 + 2 * b) * C], v.b1[b], sizeof(float) * C);
-        w.push_back(v.w2[b]); s.push_back(v.s2[b]); cin.push_back((b & 1) ? R : C); cin_pad.push_back((b & 1) ? R : C);
+        w.push_back(v.w2[b]); s.push_back(v.s2[b]); cin.push_back((b & 1) ? R : C); cin_pad.push_back((b & 1) ? ((R + 15) & ~15) : C);
         memcpy(&bias[(size_t)(2 + 2 * b) * C], v.b2[b], sizeof(float) * C);
     }
     const size_t bytes = tc_packed_layers_bytes(cin_pad.data(), C, n.n_conv);
@@ -301,17 +306,18 @@ int build_pnet(Net &n, const unsigned char *blob, size_t nbytes) {
     AZ_CUDA(cudaMalloc((void **)&n.tc_head_bias, hb.size() * sizeof(float)));
     AZ_CUDA(cudaMemcpy(n.tc_head_bias, hb.data(), hb.size() * sizeof(float), cudaMemcpyHostToDevice));
     // the finishing kernel's parameters
-    std::vector<float> small(Small::total);
-    memcpy(&small[Small::o_w], wo.data(), sizeof(float) * 4 * C);
-    memcpy(&small[Small::o_b], bo.data(), sizeof(float) * 4);
-    memcpy(&small[Small::v_cw], v.v_cw, sizeof(float) * kVC * C);
-    memcpy(&small[Small::v_cs], v.v_cs, sizeof(float) * kVC);
-    memcpy(&small[Small::v_cb], v.v_cb, sizeof(float) * kVC);
+    const Small S(C);
+    std::vector<float> small(S.total);
+    memcpy(&small[S.o_w], wo.data(), sizeof(float) * 4 * C);
+    memcpy(&small[S.o_b], bo.data(), sizeof(float) * 4);
+    memcpy(&small[S.v_cw], v.v_cw, sizeof(float) * kVC * C);
+    memcpy(&small[S.v_cs], v.v_cs, sizeof(float) * kVC);
+    memcpy(&small[S.v_cb], v.v_cb, sizeof(float) * kVC);
     for (int j = 0; j < kVH; ++j)                        // stored [input][hidden unit]
-        for (int i = 0; i < kVC * 64; ++i) small[Small::v_w1 + (size_t)i * kVH + j] = v.v_w1[(size_t)j * kVC * 64 + i];
-    memcpy(&small[Small::v_b1], v.v_b1, sizeof(float) * kVH);
-    memcpy(&small[Small::v_w2], v.v_w2, sizeof(float) * 3 * kVH);
-    memcpy(&small[Small::v_b2], v.v_b2, sizeof(float) * 3);
+        for (int i = 0; i < kVC * 64; ++i) small[S.v_w1 + (size_t)i * kVH + j] = v.v_w1[(size_t)j * kVC * 64 + i];
+    memcpy(&small[S.v_b1], v.v_b1, sizeof(float) * kVH);
+    memcpy(&small[S.v_w2], v.v_w2, sizeof(float) * 3 * kVH);
+    memcpy(&small[S.v_b2], v.v_b2, sizeof(float) * 3);
     AZ_CUDA(cudaMalloc((void **)&n.pnet_small, small.size() * sizeof(float)));
     AZ_CUDA(cudaMemcpy(n.pnet_small, small.data(), small.size() * sizeof(float), cudaMemcpyHostToDevice));
     // the action list (Sec. 3.2, App. D.1), generated: 1,792 origin-destination pairs a queen ray or a knight
@@ -357,7 +363,7 @@ int launch_pnet_finish(const Net &n, const uint64_t *masks, int batch, float *po
     AZ_CUDA(launch_dependent(pnet_finish_kernel, dim3((unsigned)batch), dim3(kFinishThreads), 0, s,
                              static_cast<const __nv_bfloat16 *>(n.act[0]), static_cast<const float *>(n.pnet_qk), masks,
                              static_cast<const float *>(n.pnet_small), reinterpret_cast<const uchar4 *>(n.pnet_actions), batch,
-                             policy, legal, counts, value, n.status_dev));
+                             (int)n.arch.channels, policy, legal, counts, value, n.status_dev));
     return AZ_OK;
 }
 

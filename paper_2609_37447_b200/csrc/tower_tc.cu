@@ -60,7 +60,8 @@ constexpr uint32_t kSpinLimit = 1u << 24;
 
 // Shape-dependent constants.  128 channels: two groups per CTA share every weight stage (16 input
 // channels x 9 taps).  256 channels: the frame and the accumulators of ONE group fill shared memory
-// and TMEM, and a stage is 16 input channels x 3 taps.
+// and TMEM, and a stage is 16 input channels x 3 taps.  160 channels (the paper's 14 x 160 network):
+// one group as well (two would need 640 TMEM columns), stages of 9 taps.
 // SETS: how many sets of four epilogue warps share a group's layer (each set takes a contiguous run of
 // the 16-channel slices).  Two sets for the FP8 tower, whose MMAs are twice as fast as its epilogue needs.
 template <int C, int GROUPS, int SETS>
@@ -69,10 +70,10 @@ struct Shape {
     static constexpr int kSlices = kC / 16;                          // 16-channel slices of a layer's output
     static constexpr int kFrameBytes = kPlaneBytes * (kC / 8);       // 46336 / 92672 per group
     static constexpr int kTileBytes = kC * 32;                       // one tap: N = C rows x 32 bytes of K
-    static constexpr int kStageTaps = kC == 128 ? 9 : 3;
+    static constexpr int kStageTaps = kC == 256 ? 3 : 9;
     static constexpr int kStagesPerSlice = 9 / kStageTaps;
     static constexpr int kStageBytes = kStageTaps * kTileBytes;      // 36864 / 24576
-    static constexpr int kStages = kC == 128 ? 3 : 5;
+    static constexpr int kStages = kC == 256 ? 5 : 3;
     static constexpr int kEpiWarps = 4 * kGroups * kSets;
     static constexpr int kThreads = 32 * (1 + kGroups + kEpiWarps);  // producer, one issuer per group, 4 epilogue warps per group and set
     static constexpr uint32_t kBDescLbo = (uint32_t)kC << 16;        // K core matrices C*16 bytes apart
@@ -93,7 +94,7 @@ struct Shape {
         return kOffConst + kEpiWarps * (fp8 ? 3 : 1) * (kC / kSets) * 4 + 256 * 4 + (pnet ? kPoolFloats * 4 : 0);
     }
     static_assert(kOffConst + kEpiWarps * 3 * (kC / kSets) * 4 + 1024 <= kMaxSmem || kC == 256, "shared memory budget");
-    static_assert(kGroups * 2 * kC == (int)kTmemCols, "TMEM: per group C columns of residual stream and C of accumulator");
+    static_assert(kGroups * 2 * kC <= (int)kTmemCols, "TMEM: per group C columns of residual stream and C of accumulator");
 };
 
 struct TowerArgs {
@@ -166,13 +167,13 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
 
 // slices of the head projection's K that travel in one weight stage
 template <class S> __device__ __host__ constexpr int head_slices_per_stage(int head_n) {
-    return S::kC == 128 ? (head_n == 256 ? 4 : S::kSlices) : (head_n == 64 ? 8 : 4);
+    return S::kC == 128 ? (head_n == 256 ? 4 : S::kSlices) : S::kC == 160 ? 5 : (head_n == 64 ? 8 : 4);
 }
 
 template <bool kFp8, class S, bool kPnet = false>
 __global__ void __launch_bounds__(S::kThreads, 1)
 tower_tc_kernel(const TowerArgs args) {
-    static_assert(!kPnet || (!kFp8 && S::kC == 128 && S::kSets == 1), "the paper's network runs on the bf16 128-channel shape");
+    static_assert(!kPnet || (!kFp8 && (S::kC == 128 || S::kC == 160) && S::kSets == 1), "the paper's network runs on the bf16 128- and 160-channel shapes");
     constexpr int kC = S::kC, kGroups = S::kGroups, kStages = S::kStages, kSlices = S::kSlices;
     constexpr int kFrameBytes = S::kFrameBytes, kStageBytes = S::kStageBytes, kThreads = S::kThreads;
     static_assert(!kFp8 || kC == 128, "the FP8 tower exists for 128 channels");
@@ -815,6 +816,7 @@ typedef Shape<128, 2, 1> Shape128;
 #endif
 typedef Shape<128, 2, AZ_FP8_EPI_SETS> Shape128F8;
 typedef Shape<256, 1, 1> Shape256;
+typedef Shape<160, 1, 1> Shape160;
 constexpr int kStageBytes = Shape128::kStageBytes;       // host-side packing of the 128-channel stages
 
 }  // namespace
@@ -984,6 +986,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape160, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
     const int sms = dev < 64 ? sm_count[dev] : 148;
@@ -1016,7 +1019,8 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     // one CTA per SM, or one per two-board group when there are fewer groups than SMs
     const int n_groups = (batch + kNB - 1) / kNB;
     const int grid = n_groups < sms ? n_groups : sms;
-    if (net.pnet) tower_tc_kernel<false, Shape128, true><<<grid, Shape128::kThreads, Shape128::smem_bytes(false, true), s>>>(a);
+    if (net.pnet && net.arch.channels == 160) tower_tc_kernel<false, Shape160, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(false, true), s>>>(a);
+    else if (net.pnet) tower_tc_kernel<false, Shape128, true><<<grid, Shape128::kThreads, Shape128::smem_bytes(false, true), s>>>(a);
     else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
     else if (fp8) tower_tc_kernel<true, Shape128F8><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else tower_tc_kernel<false, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(false), s>>>(a);

@@ -48,10 +48,11 @@ def test_masks_of_the_1880_action_list_are_bit_exact():
     assert bits[:, 1792:1880].sum() > 0 and not bits[:, 1880:].any()
 
 
+@pytest.mark.parametrize("channels", [128, 160])
 @pytest.mark.parametrize("blocks,batch", [(0, 5), (1, 7), (2, 9), (4, 33)])
-def test_small_networks_layer_by_layer(blocks, batch):
+def test_small_networks_layer_by_layer(blocks, batch, channels):
     import paper_2609_37447_b200 as az
-    cfg = pw.PNetConfig(f"t{blocks}", blocks, 128, batch, 20260971, 4400 + blocks)
+    cfg = pw.PNetConfig(f"t{blocks}", blocks, channels, batch, 20260971, 4400 + blocks)
     blob = pw.make_blob(cfg, 0.1, 0.6)
     rec, _ = positions.generate_moves(cfg.position_seed, batch, (0, 160))
     net = load(az, cfg, blob, 64)
@@ -59,7 +60,7 @@ def test_small_networks_layer_by_layer(blocks, batch):
     az.az_free_net(net)
     mo, _, po, vo, extra = oracle.pnet_evaluate(blob, rec, want_tower=True)
     assert (mg == mo).all()
-    want = extra["tower"].reshape(batch, 128, 64).transpose(0, 2, 1)
+    want = extra["tower"].reshape(batch, channels, 64).transpose(0, 2, 1)
     rel = float(np.sqrt(((tg - want) ** 2).mean() / (want ** 2).mean()))
     print(f"blocks {blocks}: backbone rms error {rel:.3e}, policy {np.abs(pg - po).max():.3e}, value {np.abs(vg - vo).max():.3e}")
     assert rel < 1.5e-2
@@ -95,6 +96,28 @@ def test_p12_batch_1024():
     assert perr <= TOL and verr <= TOL and agree >= 0.975 and agree_clear == 1.0
     for k in range(3):
         assert np.corrcoef(vg[:, k], vo[:, k])[0, 1] > 0.7
+
+
+def test_p14_the_reported_checkpoints_size_batch_320_and_a_ragged_multiple():
+    # 14 x 160 at the batch the paper serves with (App. D.3) and at 299 positions (two rounds of the
+    # persistent kernel with a half-filled last group); the oracle checks rows spread over the batch
+    import paper_2609_37447_b200 as az
+    cfg = pw.PNET_CONFIGS["p14"]
+    blob = pw.make_blob(cfg)
+    net = load(az, cfg, blob, 320)
+    for batch in (320, 299):
+        rec, _ = positions.generate_moves(cfg.position_seed, batch, cfg.plies)
+        mg, pg, vg, _ = gpu_run(az, net, cfg, rec)
+        rows = np.unique(np.concatenate([[0, 1, 147, 148, 149, 295, 296, batch - 2, batch - 1], np.arange(3, batch, 7)]))
+        mo, _, po, vo = oracle.pnet_evaluate(blob, rec[rows])
+        assert (mg[rows] == mo).all()
+        perr, verr = np.abs(pg[rows] - po).max(), np.abs(vg[rows] - vo).max()
+        agree = (pg[rows].argmax(axis=1) == po.argmax(axis=1)).mean()
+        print(f"p14: n={rows.size} of {batch} policy max-abs {perr:.3e} value max-abs {verr:.3e} arg-max agreement {agree:.4f}")
+        assert perr <= TOL and verr <= TOL and agree >= 0.95
+        bits = np.unpackbits(mg.view(np.uint8), axis=1, bitorder="little")[:, :pw.ACTIONS].astype(bool)
+        assert np.isfinite(pg).all() and (pg[~bits] == 0.0).all() and np.abs(pg.sum(axis=1) - 1).max() < 1e-3
+    az.az_free_net(net)
 
 
 def test_other_entry_points_serve_the_papers_network_too():
@@ -157,9 +180,9 @@ def test_other_entry_points_serve_the_papers_network_too():
 
 def test_unsupported_sizes_are_refused():
     import paper_2609_37447_b200 as az
-    cfg = pw.PNET_CONFIGS["p14"]
+    cfg = pw.PNetConfig("p19", 2, 176, 16, 1, 1)                      # the ladder's 176-channel size is not built
     with pytest.raises(az.AzError) as e:
-        load(az, cfg, pw.make_blob(cfg), 16)
+        load(az, cfg, pw.make_blob(cfg, 1.0, 1.0), 16)
     assert e.value.code == az.AZ_ERR_UNSUPPORTED
     with pytest.raises(az.AzError) as e:
         az.az_load_net(az.make_arch(52, 2, 128, 1, 1, 1, 16), pw.make_blob(pw.PNetConfig("x", 2, 128, 8, 1, 1)))
