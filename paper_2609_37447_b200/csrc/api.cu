@@ -268,6 +268,7 @@ void free_net(Net *n) {
     for (cudaStream_t s : n->s_compute) if (s) cudaStreamDestroy(s);
     if (n->s_out) cudaStreamDestroy(n->s_out);
     cudaFree(n->alt_u_policy); cudaFree(n->alt_u_value); cudaFree(n->alt_logits);
+    cudaFree(n->alt_act0); cudaFree(n->alt_pnet_qk);
     cudaFree(n->pnet_gw); cudaFree(n->pnet_qk); cudaFree(n->pnet_small); cudaFree(n->pnet_actions);
     if (n->ev_begin) for (int i = 0; i < kMaxProfiledPasses; ++i) { cudaEventDestroy(n->ev_begin[i]); cudaEventDestroy(n->ev_end[i]); }
     delete[] n->ev_begin; delete[] n->ev_end;
@@ -533,7 +534,12 @@ int az_submit_host(az_net *net, const void *positions_host, const uint64_t *lega
         // The tensor-core path keeps nothing else between its kernels than the head GEMM's operands and
         // the logits; with a second copy of those, odd slots run on a stream of their own.  The other
         // paths share one workspace, so all their slots take turns on one stream.
-        if (n->tc_ready && !n->pnet) {
+        if (n->pnet) {
+            // the paper's network keeps the backbone's output and the queries/keys between its two kernels
+            AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute[1], cudaStreamNonBlocking));
+            AZ_CUDA(cudaMalloc(&n->alt_act0, B * 64 * a.channels * sizeof(__nv_bfloat16)));
+            AZ_CUDA(cudaMalloc(&n->alt_pnet_qk, B * 64 * 256 * sizeof(float)));
+        } else if (n->tc_ready) {
             const size_t u_bytes = (size_t)((a.max_batch + 127) / 128) * az::kHeadChannels * 64 * 128 * sizeof(__nv_bfloat16);
             AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute[1], cudaStreamNonBlocking));
             AZ_CUDA(cudaMalloc(&n->alt_u_value, u_bytes));
@@ -567,10 +573,14 @@ int az_submit_host(az_net *net, const void *positions_host, const uint64_t *lega
     AZ_CUDA(cudaStreamWaitEvent(sc, sl.in_ready, 0));
     // kernel arguments are captured when a kernel is launched: pointing the net at the other copy for
     // the duration of the (asynchronous) launches is all it takes
-    if (alt) { std::swap(n->u_policy, n->alt_u_policy); std::swap(n->u_value, n->alt_u_value); std::swap(n->logits, n->alt_logits); }
+    auto swap_workspace = [&]() {
+        if (n->pnet) { std::swap(n->act[0], n->alt_act0); std::swap(n->pnet_qk, n->alt_pnet_qk); }
+        else { std::swap(n->u_policy, n->alt_u_policy); std::swap(n->u_value, n->alt_u_value); std::swap(n->logits, n->alt_logits); }
+    };
+    if (alt) swap_workspace();
     const int rc = dense ? az_evaluate(net, sl.pos, sl.masks, batch, sl.policy, sl.value, sc)
                          : az_evaluate_legal(net, sl.pos, sl.masks, batch, sl.compact, sl.counts, sl.value, sc);
-    if (alt) { std::swap(n->u_policy, n->alt_u_policy); std::swap(n->u_value, n->alt_u_value); std::swap(n->logits, n->alt_logits); }
+    if (alt) swap_workspace();
     if (rc != AZ_OK) return rc;
     AZ_CUDA(cudaEventRecord(sl.computed, sc));
     AZ_CUDA(cudaStreamWaitEvent(n->s_out, sl.computed, 0));

@@ -102,6 +102,7 @@ struct Net {
     // filled round of board groups) overlaps the head of the next
     void *alt_u_policy = nullptr, *alt_u_value = nullptr;
     float *alt_logits = nullptr;
+    void *alt_act0 = nullptr, *alt_pnet_qk = nullptr;   // the paper's network: backbone output, queries and keys
 
     // ---- the paper's own network (52 planes, pooled context, query-key policy head) ----
     bool pnet = false;
