@@ -32,6 +32,7 @@ WORKLOADS = {
     "c5": "c5: 40x256 bf16, 112 history planes, flat-1858 policy + WDL value (batch sweep via --batch)",
     "c4": "c4: 20x128 FP8-e4m3 tower (bf16 heads) batch 4096, 73-plane policy + tanh value",
     "c4b": "c4b: c4 with residual branches scaled by 1/sqrt(20)",
+    "c4i": "c4i: c4b with the tower in int8 (u8 activations x s8 weights, int32 accumulation), batch 4096",
     "p12": "p12: the paper's own network, 12x128 bf16 batch 1024 (52 planes, capped scaled blocks, pooled context, "
            "query-key policy over 1,880 actions, WDL value)",
     "p14": "p14: the paper's own network at its reported size, 14x160 bf16, batch 320 as the paper serves it "
@@ -56,7 +57,7 @@ def make_records(cfg, count, first_index=0):
 
 def make_blob(cfg):
     return pnet_weights.make_blob(cfg) if is_pnet(cfg) else weights.make_blob(cfg)
-DTYPE = {0: "f32", 1: "bf16", 2: "fp8_e4m3"}
+DTYPE = {0: "f32", 1: "bf16", 2: "fp8_e4m3", 3: "int8"}
 
 # DRAM bytes (read + write) of one tower-kernel launch, from the ncu capture summarised in
 # profiles/tower_tc_kernel_c3_batch592.md: 12.06 MB at batch 592, of which 11.87 MB are the weights
@@ -221,7 +222,7 @@ def main():
     blob = make_blob(cfg)
     arch = az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, B)
     net = az.az_load_net(arch, blob)
-    if cfg.precision == 2:      # FP8 tower: fix the activation ranges on the seeded calibration positions first
+    if cfg.precision >= 2:      # 8-bit tower: fix the activation ranges on the seeded calibration positions first
         cal = positions.records_for_planes(cfg.in_planes, positions.for_config(cfg, calibration=True))
         az.az_calibrate(net, az.records_to_device(cal), cal.shape[0])
     pos_dev = az.records_to_device(recs)
@@ -349,9 +350,9 @@ def main():
         # a tower launch of a few hundred microseconds between L2 flushes is a burst; launches of
         # milliseconds back to back for the whole timed region run under the power cap like the sustained GEMM
         sustained = tower_avg_ms >= 2.0
-        peak_tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"] * (2.0 if cfg.precision == 2 else 1.0)
+        peak_tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"] * (2.0 if cfg.precision >= 2 else 1.0)
         peak_note = (f"of {peaks['source']} ({'sustained' if sustained else 'burst'} bf16 GEMM"
-                     + (" x 2, nominal e4m3/bf16 ratio" if cfg.precision == 2 else "")
+                     + (" x 2, nominal 8-bit/bf16 ratio" if cfg.precision >= 2 else "")
                      + "; sustained is used when a tower launch takes 2 ms or more)")
         out = {
             "metric": METRIC, "value": evals / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,

@@ -49,7 +49,7 @@ enum {
 
 enum { AZ_POLICY_PLANES73 = 0, AZ_POLICY_FLAT1858 = 1, AZ_POLICY_FROMTO1880 = 2 };
 enum { AZ_VALUE_TANH = 0, AZ_VALUE_WDL = 1 };
-enum { AZ_PREC_FP32 = 0, AZ_PREC_BF16 = 1, AZ_PREC_FP8_E4M3 = 2 };
+enum { AZ_PREC_FP32 = 0, AZ_PREC_BF16 = 1, AZ_PREC_FP8_E4M3 = 2, AZ_PREC_INT8 = 3 };
 
 /* Network shape.  in_planes 19 or 112; blocks >= 0 residual blocks of `channels` channels
  * (a multiple of 16); heads and precision as the enums above; max_batch sizes the workspace.
@@ -298,9 +298,14 @@ int az_legal_masks(const void *positions_dev, size_t position_stride, int batch,
                    uint64_t *masks_dev, void *cuda_stream);
 
 /*
- * FP8 tower only (Sec. 4.3.6: ranges are fixed on a few hundred calibration positions): runs the
- * bf16 tower on `n` positions, records per-channel activation ranges and fixes the e4m3 scales.
- * Synchronises the stream.  Errors: BAD_ARG, BATCH_TOO_LARGE, CUDA, UNSUPPORTED (non-FP8 net).
+ * 8-bit towers only (AZ_PREC_FP8_E4M3, AZ_PREC_INT8; Sec. 4.3.6: ranges are fixed on a few hundred
+ * calibration positions): runs the bf16 tower on `n` positions, records per-channel activation
+ * ranges and fixes the scales.  FP8: e4m3 activations (range / 448 per input channel, folded into
+ * the weights) and e4m3 weights (one fp32 scale per output channel).  INT8, the precision the paper
+ * deploys: unsigned 8-bit activations (range / 255; they are never negative), signed 8-bit weights
+ * (max / 127 per output channel), int32 accumulation, the residual stream kept as int32 in the
+ * second convolution's units; input layer and heads in bf16 in both.
+ * Synchronises the stream.  Errors: BAD_ARG, BATCH_TOO_LARGE, CUDA, UNSUPPORTED (not an 8-bit net).
  */
 int az_calibrate(az_net *net, const void *positions_dev, int n, void *cuda_stream);
 

@@ -3,7 +3,7 @@
 Pure data.  `arch` fields use the same integer codes as the library's arch struct:
 policy_head 0 = 73 move planes (4672 logits), 1 = flat 1858-move list;
 value_head 0 = scalar tanh, 1 = win/draw/loss softmax;
-precision 0 = fp32, 1 = bf16, 2 = FP8-e4m3 tower (heads bf16).
+precision 0 = fp32, 1 = bf16, 2 = FP8-e4m3 tower (heads bf16), 3 = int8 tower (heads bf16).
 """
 from dataclasses import dataclass, field
 from typing import Tuple
@@ -58,6 +58,10 @@ CONFIGS = {
     # c4 with the residual branches scaled by 1/sqrt(depth), the paper's quantisation-friendly block
     # (Sec. 4.3.6), folded into the second convolution's scale and bias as the paper does at export
     "c4b": Config("c4b", 19, 20, 128, 0, 0, 2, 4096, (0, 80), (0, 80), 20260941, 9370002, branch_scale=20 ** -0.5),
+    # the same network with the tower in int8 (unsigned 8-bit activations, signed 8-bit weights), the
+    # precision the paper deploys (Sec. 4.3.6); precision code 3
+    "c4i": Config("c4i", 19, 20, 128, 0, 0, 3, 4096, (0, 80), (0, 80), 20260941, 9370002, weights_like="c4b",
+                  branch_scale=20 ** -0.5),
     "c5": Config("c5", 112, 40, 256, 1, 1, 1, 1024, (0, 80), (0, 80), 20260942, 9370005,
                  sweep=(16, 64, 256, 1024, 4096, 8192)),
 }

@@ -46,7 +46,8 @@ struct Net {
     float *tc_bias = nullptr;         // [n_conv][C] folded bias (scales are folded into the weights)
     bool tc_ready = false;
     // FP8-e4m3 tower (weights and per-layer constants exist once az_calibrate has run)
-    bool fp8 = false, fp8_ready = false;
+    bool fp8 = false, fp8_ready = false;   // 8-bit tower (FP8-e4m3 or int8) and whether it has been calibrated
+    bool int8 = false;                      // the 8-bit tower's operands are u8 activations x s8 weights
     void *tc8_weights = nullptr;
     float *tc8_lconst = nullptr;      // [n_conv][3][C]
     void *host_master = nullptr;      // fp32 tower weights kept on the host until calibration (FP8 nets)
@@ -181,7 +182,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
                     bool with_heads, unsigned int *absmax, cudaStream_t s);
 size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv);
 void tc8_pack(const float *const *w, const float *const *scale, const float *const *bias, const float *absmax,
-              int in_planes, int in_pad, int channels, int n_conv, unsigned char *packed, float *lconst);
+              int in_planes, int in_pad, int channels, int n_conv, bool int8, unsigned char *packed, float *lconst);
 int tower_tc_launch_count();
 size_t tc_head_weight_bytes(int head_n, int channels);
 void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,

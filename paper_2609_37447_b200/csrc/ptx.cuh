@@ -157,6 +157,30 @@ __device__ __forceinline__ void mma_e4m3_elect(uint32_t d_tmem, uint32_t a_lo, u
         "@q tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], da, db, %5, p;\n"
         "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elected));
 }
+// Instruction descriptor, kind::i8: D int32 (format code 2), A unsigned 8-bit (0), B signed 8-bit (1),
+// both K-major, dense; K = 32 per MMA.
+__host__ __device__ constexpr uint32_t idesc_u8s8_s32(int m, int n) {
+    return (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void mma_i8_elect(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                             uint32_t idesc, uint32_t accumulate, uint32_t elected) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 p, %6, 0;\n"
+        "setp.ne.b32 q, %7, 0;\n"
+        "mov.b64 da, {%1, %2};\n"
+        "mov.b64 db, {%3, %4};\n"
+        "@q tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elected));
+}
+// fp32 -> unsigned 8-bit, round to nearest even, saturating to [0, 255] (so it also clamps at zero)
+__device__ __forceinline__ uint32_t cvt_u8_sat(float v) {
+    uint32_t d;
+    asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(d) : "f"(v));
+    return d;
+}
 // mbarrier arrives once all MMAs issued so far by this thread have completed
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");

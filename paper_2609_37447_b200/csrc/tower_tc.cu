@@ -170,9 +170,13 @@ template <class S> __device__ __host__ constexpr int head_slices_per_stage(int h
     return S::kC == 128 ? (head_n == 256 ? 4 : S::kSlices) : S::kC == 160 ? 5 : (head_n == 64 ? 8 : 4);
 }
 
-template <bool kFp8, class S, bool kPnet = false>
+// kFp8: the 8-bit tower (layers after the input layer read 8-bit operands, 32 channels per MMA); with
+// kInt8 those operands are unsigned 8-bit activations and signed 8-bit weights (kind::i8, int32
+// accumulators, the residual stream kept as int32 in the same units), else e4m3 (kind::f8f6f4).
+template <bool kFp8, class S, bool kPnet = false, bool kInt8 = false>
 __global__ void __launch_bounds__(S::kThreads, 1)
 tower_tc_kernel(const TowerArgs args) {
+    static_assert(!kInt8 || kFp8, "the int8 tower is a form of the 8-bit tower");
     static_assert(!kPnet || (!kFp8 && (S::kC == 128 || S::kC == 160) && S::kSets == 1), "the paper's network runs on the bf16 128- and 160-channel shapes");
     constexpr int kC = S::kC, kGroups = S::kGroups, kStages = S::kStages, kSlices = S::kSlices;
     constexpr int kFrameBytes = S::kFrameBytes, kStageBytes = S::kStageBytes, kThreads = S::kThreads;
@@ -287,7 +291,7 @@ tower_tc_kernel(const TowerArgs args) {
         // ================= MMA issuer of group g =================
         const int g = warp - 1;
         constexpr uint32_t idesc = ptx::idesc_bf16_f32(128, kC);
-        constexpr uint32_t idesc8 = ptx::idesc_e4m3_f32(128, kC);
+        constexpr uint32_t idesc8 = kInt8 ? ptx::idesc_u8s8_s32(128, kC) : ptx::idesc_e4m3_f32(128, kC);
         int stage = 0;
         uint32_t phase = 0;
         uint32_t a_phase = 0;
@@ -349,9 +353,14 @@ tower_tc_kernel(const TowerArgs args) {
                                 for (int t = 0; t < S::kStageTaps; ++t) {
                                     const int tap = st * S::kStageTaps + t;
                                     const int dy = tap / 3 - 1, dx = tap % 3 - 1;
-                                    ptx::mma_e4m3_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                        b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8,
-                                                        (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
+                                    if (kInt8)
+                                        ptx::mma_i8_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                                          b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8,
+                                                          (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
+                                    else
+                                        ptx::mma_e4m3_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                                            b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8,
+                                                            (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
                                 }
                             } else {
 #pragma unroll
@@ -653,10 +662,16 @@ tower_tc_kernel(const TowerArgs args) {
                         const float4 bv = *reinterpret_cast<const float4 *>(bias + ks * 16 + i);
                         if (kFp8) {
                             const float4 os = *reinterpret_cast<const float4 *>(lc + ks * 16 + i);
-                            v[i + 0] = fmaf(__uint_as_float(rr[i + 0]), os.x, bv.x);
-                            v[i + 1] = fmaf(__uint_as_float(rr[i + 1]), os.y, bv.y);
-                            v[i + 2] = fmaf(__uint_as_float(rr[i + 2]), os.z, bv.z);
-                            v[i + 3] = fmaf(__uint_as_float(rr[i + 3]), os.w, bv.w);
+                            // int8 tower: layers after the input layer accumulate in int32 (the input layer's MMAs are bf16 -> fp32)
+                            const bool ints = kInt8 && l > 0;
+                            const float a0 = ints ? __int2float_rn((int)rr[i + 0]) : __uint_as_float(rr[i + 0]);
+                            const float a1 = ints ? __int2float_rn((int)rr[i + 1]) : __uint_as_float(rr[i + 1]);
+                            const float a2 = ints ? __int2float_rn((int)rr[i + 2]) : __uint_as_float(rr[i + 2]);
+                            const float a3 = ints ? __int2float_rn((int)rr[i + 3]) : __uint_as_float(rr[i + 3]);
+                            v[i + 0] = fmaf(a0, os.x, bv.x);
+                            v[i + 1] = fmaf(a1, os.y, bv.y);
+                            v[i + 2] = fmaf(a2, os.z, bv.z);
+                            v[i + 3] = fmaf(a3, os.w, bv.w);
                         } else {
                             v[i + 0] = __uint_as_float(rr[i + 0]) + bv.x;
                             v[i + 1] = __uint_as_float(rr[i + 1]) + bv.y;
@@ -701,8 +716,13 @@ tower_tc_kernel(const TowerArgs args) {
                             // 16 channels -> 16 e4m3 bytes (saturating, round to nearest even) = one slot of plane kc
                             uint32_t pk[4];
 #pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                pk[i] = ptx::pack_e4m3x2_relu(v[4 * i], v[4 * i + 1]) | (ptx::pack_e4m3x2_relu(v[4 * i + 2], v[4 * i + 3]) << 16);
+                            for (int i = 0; i < 4; ++i) {
+                                if (kInt8)      // unsigned 8-bit, saturating: clamps at zero (ReLU) and at 255
+                                    pk[i] = ptx::cvt_u8_sat(v[4 * i]) | (ptx::cvt_u8_sat(v[4 * i + 1]) << 8) |
+                                            (ptx::cvt_u8_sat(v[4 * i + 2]) << 16) | (ptx::cvt_u8_sat(v[4 * i + 3]) << 24);
+                                else
+                                    pk[i] = ptx::pack_e4m3x2_relu(v[4 * i], v[4 * i + 1]) | (ptx::pack_e4m3x2_relu(v[4 * i + 2], v[4 * i + 3]) << 16);
+                            }
                             *reinterpret_cast<uint4 *>(frame + kc * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         } else {
                             uint32_t pk[8];
@@ -721,10 +741,17 @@ tower_tc_kernel(const TowerArgs args) {
                             for (int i = 0; i < 16; i += 4) {
                                 float4 hs = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
                                 if (kFp8) hs = *reinterpret_cast<const float4 *>(lc + 2 * kMyC + ks * 16 + i);
-                                w[i + 0] = __float_as_uint(kFp8 ? v[i + 0] * hs.x : v[i + 0]);
-                                w[i + 1] = __float_as_uint(kFp8 ? v[i + 1] * hs.y : v[i + 1]);
-                                w[i + 2] = __float_as_uint(kFp8 ? v[i + 2] * hs.z : v[i + 2]);
-                                w[i + 3] = __float_as_uint(kFp8 ? v[i + 3] * hs.w : v[i + 3]);
+                                if (kInt8) {    // the stream in the next second convolution's integer units, rounded
+                                    w[i + 0] = (uint32_t)__float2int_rn(v[i + 0] * hs.x);
+                                    w[i + 1] = (uint32_t)__float2int_rn(v[i + 1] * hs.y);
+                                    w[i + 2] = (uint32_t)__float2int_rn(v[i + 2] * hs.z);
+                                    w[i + 3] = (uint32_t)__float2int_rn(v[i + 3] * hs.w);
+                                } else {
+                                    w[i + 0] = __float_as_uint(kFp8 ? v[i + 0] * hs.x : v[i + 0]);
+                                    w[i + 1] = __float_as_uint(kFp8 ? v[i + 1] * hs.y : v[i + 1]);
+                                    w[i + 2] = __float_as_uint(kFp8 ? v[i + 2] * hs.z : v[i + 2]);
+                                    w[i + 3] = __float_as_uint(kFp8 ? v[i + 3] * hs.w : v[i + 3]);
+                                }
                             }
                             ptx::tmem_st16(t_lane + (uint32_t)(kc * 16), w);
                             if (S::kSets > 1 && ks == kMySlices - 1) ptx::tmem_st_wait();
@@ -906,10 +933,13 @@ size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv) {
     return ((size_t)in_pad / 16 + (size_t)(n_conv - 1) * (channels / 32)) * kStageBytes;
 }
 
+// int8 form (the paper's deployed precision, Sec. 4.3.6): activations unsigned 8-bit with sa =
+// calibration maximum / 255 (they are never negative), weights signed 8-bit with ws = max|W'| / 127,
+// round to nearest; same constants, same layout.
 void tc8_pack(const float *const *w, const float *const *scale, const float *const *bias, const float *absmax,
-              int in_planes, int in_pad, int channels, int n_conv, unsigned char *packed, float *lconst) {
+              int in_planes, int in_pad, int channels, int n_conv, bool int8, unsigned char *packed, float *lconst) {
     const int C = channels;
-    const float kMax = 448.0f, kTiny = 1e-30f;
+    const float kMax = int8 ? 255.0f : 448.0f, kMaxW = int8 ? 127.0f : 448.0f, kTiny = 1e-30f;
     std::vector<float> sa((size_t)n_conv * C, 1.0f), ws((size_t)n_conv * C, 1.0f);
     for (int l = 1; l < n_conv; ++l)
         for (int c = 0; c < C; ++c) sa[(size_t)l * C + c] = fmaxf(absmax[(size_t)(l - 1) * C + c], kTiny) / kMax;
@@ -926,7 +956,7 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
                     wf[((size_t)co * C + ci) * 9 + tap] = v;
                     mx = fmaxf(mx, fabsf(v));
                 }
-            ws[(size_t)l * C + co] = fmaxf(mx, kTiny) / kMax;
+            ws[(size_t)l * C + co] = fmaxf(mx, kTiny) / kMaxW;
         }
         for (int kc = 0; kc < C / 32; ++kc)
             for (int tap = 0; tap < 9; ++tap)
@@ -936,7 +966,12 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
                             for (int e = 0; e < 16; ++e) {
                                 const int n = ng * 8 + r, ci = kc * 32 + k16 * 16 + e;
                                 const float v = wf[((size_t)n * C + ci) * 9 + tap] / ws[(size_t)l * C + n];
-                                *dst++ = (unsigned char)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
+                                if (int8) {
+                                    const float q = fminf(fmaxf(nearbyintf(v), -127.0f), 127.0f);
+                                    *dst++ = (unsigned char)(signed char)q;
+                                } else {
+                                    *dst++ = (unsigned char)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
+                                }
                             }
     }
     for (int l = 0; l < n_conv; ++l) {
@@ -984,6 +1019,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape160, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
@@ -1022,6 +1058,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     if (net.pnet && net.arch.channels == 160) tower_tc_kernel<false, Shape160, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(false, true), s>>>(a);
     else if (net.pnet) tower_tc_kernel<false, Shape128, true><<<grid, Shape128::kThreads, Shape128::smem_bytes(false, true), s>>>(a);
     else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
+    else if (fp8 && net.int8) tower_tc_kernel<true, Shape128F8, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else if (fp8) tower_tc_kernel<true, Shape128F8><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else tower_tc_kernel<false, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(false), s>>>(a);
     AZ_LAUNCH_CHECK();

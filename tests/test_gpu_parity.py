@@ -295,6 +295,15 @@ def test_c4b_fp8_with_scaled_residual_branches(az):
     assert verr <= TOL[2] and perr < 0.1
 
 
+def test_c4i_int8_tower_meets_the_bar_of_the_quantised_configs(az):
+    # the tower in int8, the precision the paper deploys (Sec. 4.3.6), on the branch-scaled weights: unsigned
+    # 8-bit activations carry one bit more than e4m3's mantissa does over most of their range
+    rows = np.arange(0, 4096, 16)
+    perr, verr, agree, tower_err = fp8_run(az, "c4i", 4096, rows)
+    assert tower_err < 2.5e-2
+    assert perr <= TOL[2] and verr <= TOL[2]
+
+
 def test_results_are_deterministic_and_independent_of_batch_composition(az):
     cfg = configs.tiny_config(blocks=3, channels=128, policy_head=1, value_head=1, precision=1, batch=40)
     blob = weights.make_blob(cfg, 0.02, 0.05)
