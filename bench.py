@@ -35,6 +35,7 @@ WORKLOADS = {
     "c4i": "c4i: c4b with the tower in int8 (u8 activations x s8 weights, int32 accumulation), batch 4096",
     "p12": "p12: the paper's own network, 12x128 bf16 batch 1024 (52 planes, capped scaled blocks, pooled context, "
            "query-key policy over 1,880 actions, WDL value)",
+    "p12i": "p12i: p12 with the backbone's convolutions in int8 (pooled context and heads in floating point), batch 1024",
     "p14": "p14: the paper's own network at its reported size, 14x160 bf16, batch 320 as the paper serves it "
            "(App. D.3); --batch for other sizes",
 }
@@ -223,7 +224,10 @@ def main():
     arch = az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, B)
     net = az.az_load_net(arch, blob)
     if cfg.precision >= 2:      # 8-bit tower: fix the activation ranges on the seeded calibration positions first
-        cal = positions.records_for_planes(cfg.in_planes, positions.for_config(cfg, calibration=True))
+        if is_pnet(cfg):
+            cal = positions.generate_moves(cfg.position_seed + configs.CALIBRATION_SEED_OFFSET, configs.CALIBRATION_COUNT, cfg.plies)[0]
+        else:
+            cal = positions.records_for_planes(cfg.in_planes, positions.for_config(cfg, calibration=True))
         az.az_calibrate(net, az.records_to_device(cal), cal.shape[0])
     pos_dev = az.records_to_device(recs)
     masks_dev = torch.zeros((B, cfg.mask_words), dtype=torch.int64, device="cuda")

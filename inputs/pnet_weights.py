@@ -38,12 +38,13 @@ class PNetConfig:
     value_channels: int = 2
     value_hidden: int = 48
     plies: tuple = (0, 160)
+    precision: int = 1           # 1 = bf16, 3 = int8 tower (heads and pooled context in floating point)
+    weights_like: str = ""       # name of the configuration whose head scales this one reuses
 
     # the same vocabulary as the other workloads' Config, so that callers can treat both alike
     in_planes = PLANES
     policy_head = 2
     value_head = 1
-    precision = 1
     policy_size = ACTIONS
     value_size = 3
     mask_words = MASK_WORDS
@@ -53,6 +54,8 @@ class PNetConfig:
 PNET_CONFIGS = {
     "p12": PNetConfig("p12", 12, 128, 1024, 20260961, 9371201),
     "p14": PNetConfig("p14", 14, 160, 320, 20260962, 9371401),
+    # p12 with the backbone's convolutions in int8, the precision the paper deploys (Sec. 4.3.6)
+    "p12i": PNetConfig("p12i", 12, 128, 1024, 20260961, 9371201, precision=3, weights_like="p12"),
 }
 
 
@@ -99,7 +102,7 @@ def head_scales(name: str):
 
 def draw_tensors(cfg: PNetConfig, policy_scale: float = None, value_scale: float = None):
     if policy_scale is None or value_scale is None:
-        ps, vs = head_scales(cfg.name)
+        ps, vs = head_scales(cfg.weights_like or cfg.name)
         policy_scale = ps if policy_scale is None else policy_scale
         value_scale = vs if value_scale is None else value_scale
     rng = np.random.Generator(np.random.PCG64(cfg.weight_seed))

@@ -61,4 +61,4 @@ def main(names):
 
 
 if __name__ == "__main__":
-    main(sys.argv[1:] or list(pw.PNET_CONFIGS))
+    main(sys.argv[1:] or [n for n, c in pw.PNET_CONFIGS.items() if not c.weights_like])

@@ -271,6 +271,7 @@ void free_net(Net *n) {
     cudaFree(n->alt_u_policy); cudaFree(n->alt_u_value); cudaFree(n->alt_logits);
     cudaFree(n->alt_act0); cudaFree(n->alt_pnet_qk);
     cudaFree(n->pnet_gw); cudaFree(n->pnet_qk); cudaFree(n->pnet_small); cudaFree(n->pnet_actions);
+    free_pnet_master(n->pnet_master);
     if (n->ev_begin) for (int i = 0; i < kMaxProfiledPasses; ++i) { cudaEventDestroy(n->ev_begin[i]); cudaEventDestroy(n->ev_end[i]); }
     delete[] n->ev_begin; delete[] n->ev_end;
     cudaFree(n->logits); cudaFree(n->head_p); cudaFree(n->head_v); cudaFree(n->hidden); cudaFree(n->status_dev);
@@ -343,8 +344,10 @@ int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az
     *out = nullptr;
     if (!az::arch_ok(*arch)) return AZ_ERR_BAD_ARCH;
     const bool pnet = arch->in_planes == 52;
-    // of the paper's network ladder the 128- and 160-channel sizes are built, in bf16
-    if (pnet && ((arch->channels != 128 && arch->channels != 160) || arch->precision != AZ_PREC_BF16)) return AZ_ERR_UNSUPPORTED;
+    // of the paper's network ladder the 128- and 160-channel sizes are built in bf16, the 128-channel one also in int8
+    if (pnet && !((arch->precision == AZ_PREC_BF16 && (arch->channels == 128 || arch->channels == 160)) ||
+                  (arch->precision == AZ_PREC_INT8 && arch->channels == 128)))
+        return AZ_ERR_UNSUPPORTED;
     az::BlobView view;
     int rc = AZ_OK;
     if (!pnet) rc = az::parse_blob(*arch, static_cast<const unsigned char *>(weights_host), nbytes, view);
@@ -653,7 +656,8 @@ int az_legal_masks(const void *positions_dev, size_t position_stride, int batch,
 int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_stream) {
     Net *n = reinterpret_cast<Net *>(net);
     if (!n || count <= 0 || !positions_dev || (reinterpret_cast<uintptr_t>(positions_dev) & 7)) return AZ_ERR_BAD_ARG;
-    if (!n->fp8 || !n->host_master) return AZ_ERR_UNSUPPORTED;
+    if (!n->fp8 || (!n->host_master && !n->pnet_master)) return AZ_ERR_UNSUPPORTED;
+    if (n->pnet && n->fp8_ready) return AZ_ERR_UNSUPPORTED;   // its context maps were rescaled by the first calibration
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const int C = (int)n->arch.channels, L = n->n_conv;
     const size_t pb = az_position_bytes(&n->arch);
@@ -674,6 +678,7 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
     if (rc != AZ_OK) return rc;
     if (e != cudaSuccess) { az::set_cuda_error(e, "az_calibrate"); return AZ_ERR_CUDA; }
     // 2. quantise the tower with those ranges
+    if (n->pnet) return az::quantise_pnet(*n, absmax.data());
     az::HostMaster *hm = static_cast<az::HostMaster *>(n->host_master);
     std::vector<const float *> w, sc, bi;
     for (int l = 0; l < L; ++l) { w.push_back(hm->w[l].data()); sc.push_back(hm->scale[l].data()); bi.push_back(hm->bias[l].data()); }

@@ -111,6 +111,7 @@ struct Net {
     void *pnet_qk = nullptr;          // [max_batch][64][256] fp32: queries | keys
     float *pnet_small = nullptr;      // the finishing kernel's fp32 parameters, see pnet.cu
     unsigned char *pnet_actions = nullptr;   // [1880][4]: origin, destination, promotion piece + 1 (0 none), pad
+    void *pnet_master = nullptr;      // int8 form: the fp32 tower parameters, kept until az_calibrate has quantised them
 
     // ---- optional event timing of the tower ----
     bool profile = false;
@@ -148,6 +149,8 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
 // ---- kernels' launch functions (each returns AZ_OK or AZ_ERR_CUDA) ---------------------------
 int launch_encode52(const void *positions, int batch, bool bf16, void *planes, cudaStream_t s);
 int build_pnet(Net &n, const unsigned char *blob, size_t nbytes);
+int quantise_pnet(Net &n, const float *absmax);      // int8 form, after the calibration pass ([n_conv][C] output maxima)
+void free_pnet_master(void *master);
 int launch_pnet_finish(const Net &n, const uint64_t *masks, int batch, float *policy, float *legal, int *counts,
                        float *value, cudaStream_t s);
 size_t tc_packed_layers_bytes(const int *cin_pad, int channels, int n_conv);

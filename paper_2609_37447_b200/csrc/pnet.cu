@@ -20,6 +20,7 @@
 
 #include <cmath>
 #include <cstring>
+#include <new>
 #include <vector>
 
 namespace az {
@@ -248,7 +249,98 @@ void compose(const float *m, const float *b, int rows, const float *t_w, const f
     }
 }
 
+// fp32 master copy of the tower for the int8 form (quantised once the calibration ranges are known)
+struct PnetMaster {
+    std::vector<std::vector<float>> w, scale, bias;   // per convolution layer
+    std::vector<int> cin;                             // input channels of each layer
+    std::vector<std::vector<float>> gw;               // per pooled block: [3C/4][C/2]
+};
+
 }  // namespace
+
+void free_pnet_master(void *master) { delete static_cast<PnetMaster *>(master); }
+
+// int8 form of the paper's tower (Sec. 4.3.6: the trunk's convolutions in INT8, the pooled context and
+// the heads in floating point).  As in the plain int8 tower: layer l >= 1 reads unsigned 8-bit
+// activations with a per-input-channel scale sa (calibration maximum / 255, folded into the weight
+// rows) and signed 8-bit weights with a per-output-channel scale ws (max / 127).  Per layer four
+// constant vectors: os * qs, bias * qs, hs / qs, 6 * qs, where os = ws (1 for the input layer), qs =
+// 1 / sa of the next layer for the channels that are handed on and 1 for the pooled ones (so that
+// their values stay in real units), hs = 1 / ws of the next second convolution on the residual
+// stream.  The context map's rows are multiplied by the same qs, since the context is added to
+// values that are already in those units.
+int quantise_pnet(Net &n, const float *absmax) {
+    const PnetMaster *m = static_cast<const PnetMaster *>(n.pnet_master);
+    if (!m) return AZ_ERR_UNSUPPORTED;
+    const int C = (int)n.arch.channels, L = n.n_conv, P = C / 4, R = C - P;
+    const float kTiny = 1e-30f;
+    constexpr int kStage = 9 * 128 * 32;              // bytes of one weight stage: 9 taps x 128 outputs x 32 bytes of K
+    std::vector<float> sa((size_t)L * C, 1.0f), ws((size_t)L * C, 1.0f);
+    for (int l = 1; l < L; ++l)
+        for (int c = 0; c < m->cin[l]; ++c) sa[(size_t)l * C + c] = fmaxf(absmax[(size_t)(l - 1) * C + c], kTiny) / 255.0f;
+    size_t bytes = (size_t)(n.in_pad / 16) * kStage;
+    for (int l = 1; l < L; ++l) bytes += (size_t)((m->cin[l] + 31) / 32) * kStage;
+    std::vector<unsigned char> packed(bytes, 0);
+    // input layer: bf16 tiles as in the bf16 tower
+    {
+        const float *w0 = m->w[0].data(), *s0 = m->scale[0].data();
+        const int cin0 = m->cin[0], pad0 = n.in_pad;
+        tc_pack_layers(&w0, &s0, &cin0, &pad0, C, 1, reinterpret_cast<__nv_bfloat16 *>(packed.data()));
+    }
+    unsigned char *dst = packed.data() + (size_t)(n.in_pad / 16) * kStage;
+    for (int l = 1; l < L; ++l) {
+        const int cin = m->cin[l];
+        std::vector<float> wf((size_t)C * cin * 9);
+        for (int co = 0; co < C; ++co) {
+            float mx = 0.0f;
+            for (int ci = 0; ci < cin; ++ci)
+                for (int tap = 0; tap < 9; ++tap) {
+                    const float v = m->scale[l][co] * m->w[l][((size_t)co * cin + ci) * 9 + tap] * sa[(size_t)l * C + ci];
+                    wf[((size_t)co * cin + ci) * 9 + tap] = v;
+                    mx = fmaxf(mx, fabsf(v));
+                }
+            ws[(size_t)l * C + co] = fmaxf(mx, kTiny) / 127.0f;
+        }
+        for (int kc = 0; kc < (cin + 31) / 32; ++kc)
+            for (int tap = 0; tap < 9; ++tap)
+                for (int k16 = 0; k16 < 2; ++k16)
+                    for (int ng = 0; ng < C / 8; ++ng)
+                        for (int r = 0; r < 8; ++r)
+                            for (int e = 0; e < 16; ++e) {
+                                const int co = ng * 8 + r, ci = kc * 32 + k16 * 16 + e;
+                                float q = 0.0f;
+                                if (ci < cin) q = fminf(fmaxf(nearbyintf(wf[((size_t)co * cin + ci) * 9 + tap] / ws[(size_t)l * C + co]), -127.0f), 127.0f);
+                                *dst++ = (unsigned char)(signed char)q;
+                            }
+    }
+    std::vector<float> lconst((size_t)L * 4 * C), gwt;
+    for (int l = 0; l < L; ++l) {
+        float *lc = lconst.data() + (size_t)l * 4 * C;
+        const int next_cin = l + 1 < L ? m->cin[l + 1] : 0;       // channels of this layer's output that are handed on as 8-bit
+        for (int c = 0; c < C; ++c) {
+            const float qs = c < next_cin ? 1.0f / sa[(size_t)(l + 1) * C + c] : 1.0f;
+            const float hs = ((l & 1) == 0 && l + 2 < L) ? 1.0f / ws[(size_t)(l + 2) * C + c] : 1.0f;
+            lc[c] = (l == 0 ? 1.0f : ws[(size_t)l * C + c]) * qs;
+            lc[C + c] = m->bias[l][c] * qs;
+            lc[2 * C + c] = hs / qs;
+            lc[3 * C + c] = 6.0f * qs;
+        }
+        if ((l & 3) == 3) {                                          // first convolution of a pooled block: its context map
+            const std::vector<float> &g = m->gw[(l - 3) / 4];
+            for (int j = 0; j < 2 * P; ++j)
+                for (int r = 0; r < R; ++r) gwt.push_back(g[(size_t)r * 2 * P + j] / sa[(size_t)(l + 1) * C + r]);
+        }
+    }
+    if (gwt.empty()) gwt.push_back(0.0f);
+    if (!n.tc8_weights) AZ_CUDA(cudaMalloc(&n.tc8_weights, bytes));
+    if (!n.tc8_lconst) AZ_CUDA(cudaMalloc((void **)&n.tc8_lconst, lconst.size() * sizeof(float)));
+    AZ_CUDA(cudaMemcpy(n.tc8_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
+    AZ_CUDA(cudaMemcpy(n.tc8_lconst, lconst.data(), lconst.size() * sizeof(float), cudaMemcpyHostToDevice));
+    // the scaled context maps replace the plain ones (the calibration pass, which needed those, is over)
+    AZ_CUDA(cudaMemcpy(n.pnet_gw, gwt.data(), gwt.size() * sizeof(float), cudaMemcpyHostToDevice));
+    n.fp8_ready = true;
+    return AZ_OK;
+}
 
 // Builds the device side of a paper-network az_net: 128 or 160 channels, bf16 (the caller refuses
 // other sizes).
@@ -260,6 +352,8 @@ int build_pnet(Net &n, const unsigned char *blob, size_t nbytes) {
     const int C = v.C, L = v.L, P = C / 4, R = C - P;
     n.bf16 = true;
     n.pnet = true;
+    n.int8 = a.precision == AZ_PREC_INT8;
+    n.fp8 = n.int8;                                      // the 8-bit tower; usable after az_calibrate
     n.in_pad = 64;
     n.n_conv = 1 + 2 * L;
     // tower tiles
@@ -273,6 +367,18 @@ int build_pnet(Net &n, const unsigned char *blob, size_t nbytes) {
         memcpy(&bias[(size_t)(1 + 2 * b) * C], v.b1[b], sizeof(float) * C);
         w.push_back(v.w2[b]); s.push_back(v.s2[b]); cin.push_back((b & 1) ? R : C); cin_pad.push_back((b & 1) ? ((R + 15) & ~15) : C);
         memcpy(&bias[(size_t)(2 + 2 * b) * C], v.b2[b], sizeof(float) * C);
+    }
+    if (n.int8) {
+        PnetMaster *m = new (std::nothrow) PnetMaster();
+        if (!m) return AZ_ERR_BAD_ARG;
+        n.pnet_master = m;
+        for (int l = 0; l < n.n_conv; ++l) {
+            m->w.emplace_back(w[l], w[l] + (size_t)C * cin[l] * 9);
+            m->scale.emplace_back(s[l], s[l] + C);
+            m->bias.emplace_back(&bias[(size_t)l * C], &bias[(size_t)l * C] + C);
+            m->cin.push_back(cin[l]);
+        }
+        for (int b = 1; b < L; b += 2) m->gw.emplace_back(v.gw[b], v.gw[b] + (size_t)R * 2 * P);
     }
     const size_t bytes = tc_packed_layers_bytes(cin_pad.data(), C, n.n_conv);
     std::vector<__nv_bfloat16> packed(bytes / sizeof(__nv_bfloat16));

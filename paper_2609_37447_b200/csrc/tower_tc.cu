@@ -91,9 +91,9 @@ struct Shape {
     static constexpr int kCtxStride = (3 * kC / 4 + 15) & ~15;      // context entries per board, padded with zeros to whole slices
     static constexpr int kPoolFloats = kGroups * (2 * 4 * 2 * (kC / 4) + 2 * (kC / 2) + 2 * kCtxStride);
     static constexpr int smem_bytes(bool fp8, bool pnet = false) {
-        return kOffConst + kEpiWarps * (fp8 ? 3 : 1) * (kC / kSets) * 4 + 256 * 4 + (pnet ? kPoolFloats * 4 : 0);
+        return kOffConst + kEpiWarps * (fp8 ? (pnet ? 4 : 3) : 1) * (kC / kSets) * 4 + 256 * 4 + (pnet ? kPoolFloats * 4 : 0);
     }
-    static_assert(kOffConst + kEpiWarps * 3 * (kC / kSets) * 4 + 1024 <= kMaxSmem || kC == 256, "shared memory budget");
+    static_assert(kOffConst + kEpiWarps * 4 * (kC / kSets) * 4 + 1024 + kPoolFloats * 4 <= kMaxSmem || kC == 256, "shared memory budget");
     static_assert(kGroups * 2 * kC <= (int)kTmemCols, "TMEM: per group C columns of residual stream and C of accumulator");
 };
 
@@ -177,7 +177,8 @@ template <bool kFp8, class S, bool kPnet = false, bool kInt8 = false>
 __global__ void __launch_bounds__(S::kThreads, 1)
 tower_tc_kernel(const TowerArgs args) {
     static_assert(!kInt8 || kFp8, "the int8 tower is a form of the 8-bit tower");
-    static_assert(!kPnet || (!kFp8 && (S::kC == 128 || S::kC == 160) && S::kSets == 1), "the paper's network runs on the bf16 128- and 160-channel shapes");
+    static_assert(!kPnet || ((S::kC == 128 || S::kC == 160) && S::kSets == 1), "the paper's network runs on the one-set 128- and 160-channel shapes");
+    static_assert(!(kPnet && kFp8) || (kInt8 && S::kC == 128), "of the 8-bit towers the int8 one carries the paper's network, at 128 channels");
     constexpr int kC = S::kC, kGroups = S::kGroups, kStages = S::kStages, kSlices = S::kSlices;
     constexpr int kFrameBytes = S::kFrameBytes, kStageBytes = S::kStageBytes, kThreads = S::kThreads;
     static_assert(!kFp8 || kC == 128, "the FP8 tower exists for 128 channels");
@@ -196,9 +197,10 @@ tower_tc_kernel(const TowerArgs args) {
     auto bar_pool = [&](int g) { return bar_done + 8u * (1 + kStages + g); };   // the four epilogue warps of group g meet here
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + S::kOffAbort);
     uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + S::kOffTmemPtr);
-    constexpr int kConstFloats = (kFp8 ? 3 : 1) * kC;          // per layer: (scale, bias, h ratio) or bias
+    constexpr int kVecs = kFp8 ? (kPnet ? 4 : 3) : 1;           // per layer: (scale, bias, h ratio[, cap]) or bias
+    constexpr int kConstFloats = kVecs * kC;
     constexpr int kMyC = kC / S::kSets;                         // channels an epilogue warp is responsible for
-    constexpr int kMyConstFloats = (kFp8 ? 3 : 1) * kMyC;
+    constexpr int kMyConstFloats = kVecs * kMyC;
     float *head_bias_smem = reinterpret_cast<float *>(smem + S::kOffConst) + S::kEpiWarps * kMyConstFloats;
 
     // ---- set-up: zero the frames (their borders stay zero for the kernel's lifetime), barriers, TMEM
@@ -243,7 +245,7 @@ tower_tc_kernel(const TowerArgs args) {
     constexpr int kShortSlices = (3 * kC / 4 + 15) / 16;      // slices that hold the 3C/4 channels a pooled block hands on
     auto round_of = [&](int r) { return get_round<S>(r, (int)blockIdx.x, (int)gridDim.x, n_groups); };
     auto slices_of = [&](int l) {                                                               // K per MMA: 16 bf16 or 32 e4m3
-        return l == 0 ? in_slices : short_layer(l) ? kShortSlices : (kFp8 ? kC / 32 : kC / 16);
+        return l == 0 ? in_slices : short_layer(l) ? (kFp8 ? kShortSlices / 2 : kShortSlices) : (kFp8 ? kC / 32 : kC / 16);
     };
     const bool tr = args.trace && blockIdx.x == 0;
     long long t_wait[3] = {0, 0, 0};
@@ -577,7 +579,11 @@ tower_tc_kernel(const TowerArgs args) {
                         float sm[8], mx[8];
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            sm[i] = live ? fminf(fmaxf(__uint_as_float(r8[i]) + bias[kRegC + pc * 8 + i], 0.0f), 6.0f) : 0.0f;
+                            // (8-bit tower: int32 accumulator times the weight scale; these channels are not handed on,
+                            // so their constants carry no activation scale and the value is in real units)
+                            const float pre = kFp8 ? fmaf(__int2float_rn((int)r8[i]), lc[kRegC + pc * 8 + i], bias[kRegC + pc * 8 + i])
+                                                   : __uint_as_float(r8[i]) + bias[kRegC + pc * 8 + i];
+                            sm[i] = live ? fminf(fmaxf(pre, 0.0f), 6.0f) : 0.0f;
                             mx[i] = sm[i];
                         }
 #pragma unroll
@@ -621,9 +627,10 @@ tower_tc_kernel(const TowerArgs args) {
                         }
                         pool_vec[pb * 2 * kPoolC + j] = j >= kPoolC ? acc : acc * (1.0f / 64.0f);
                     }
+                    constexpr int kCtxPad = kCtxStride > kRegC ? kCtxStride - kRegC : 1;
                     if (kCtxStride > kRegC)                                    // the padding of the context stays zero
-                        for (int z = q * 32 + lane; z < 2 * (kCtxStride - kRegC); z += 128)
-                            pool_ctx[(z / (kCtxStride - kRegC)) * kCtxStride + kRegC + z % (kCtxStride - kRegC)] = 0.0f;
+                        for (int z = q * 32 + lane; z < 2 * kCtxPad; z += 128)
+                            pool_ctx[(z / kCtxPad) * kCtxStride + kRegC + z % kCtxPad] = 0.0f;
                     ok = meet();
                     if (!ok) break;
                     // (3) context = gw . pooled vector: 2 boards x 3C/4 outputs over the group's 128 threads.  The map
@@ -691,7 +698,7 @@ tower_tc_kernel(const TowerArgs args) {
                     }
                     if (kPnet) {                                     // activations capped at six (Sec. 4.3.6)
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = fminf(v[i], 6.0f);
+                        for (int i = 0; i < 16; ++i) v[i] = fminf(v[i], kFp8 ? lc[3 * kMyC + ks * 16 + i] : 6.0f);   // six, in the layer's output units
                     }
                     if (!kFp8 && args.absmax != nullptr) {
                         // calibration: largest output of this layer per channel over all rows of the warp
@@ -1023,6 +1030,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape160, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
     const int sms = dev < 64 ? sm_count[dev] : 148;
@@ -1056,6 +1064,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     const int n_groups = (batch + kNB - 1) / kNB;
     const int grid = n_groups < sms ? n_groups : sms;
     if (net.pnet && net.arch.channels == 160) tower_tc_kernel<false, Shape160, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(false, true), s>>>(a);
+    else if (net.pnet && fp8) tower_tc_kernel<true, Shape128, true, true><<<grid, Shape128::kThreads, Shape128::smem_bytes(true, true), s>>>(a);
     else if (net.pnet) tower_tc_kernel<false, Shape128, true><<<grid, Shape128::kThreads, Shape128::smem_bytes(false, true), s>>>(a);
     else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
     else if (fp8 && net.int8) tower_tc_kernel<true, Shape128F8, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);

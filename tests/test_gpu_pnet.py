@@ -13,7 +13,7 @@ TOL = 2e-2
 
 
 def load(az, cfg, blob, max_batch):
-    arch = az.make_arch(52, cfg.blocks, cfg.channels, 2, 1, 1, max_batch)
+    arch = az.make_arch(52, cfg.blocks, cfg.channels, 2, 1, cfg.precision, max_batch)
     return az.az_load_net(arch, blob)
 
 
@@ -118,6 +118,38 @@ def test_p14_the_reported_checkpoints_size_batch_320_and_a_ragged_multiple():
         bits = np.unpackbits(mg.view(np.uint8), axis=1, bitorder="little")[:, :pw.ACTIONS].astype(bool)
         assert np.isfinite(pg).all() and (pg[~bits] == 0.0).all() and np.abs(pg.sum(axis=1) - 1).max() < 1e-3
     az.az_free_net(net)
+
+
+def test_p12_with_an_int8_backbone():
+    # Sec. 4.3.6: the backbone's convolutions in INT8, pooled context and heads in floating point, ranges fixed
+    # on calibration positions; the bar is the quantised configs' 5e-2
+    import paper_2609_37447_b200 as az
+    cfg = pw.PNET_CONFIGS["p12i"]
+    blob = pw.make_blob(cfg)
+    rec, _ = positions.generate_moves(cfg.position_seed, cfg.batch, cfg.plies)
+    cal, _ = positions.generate_moves(cfg.position_seed + 777_000_000, 512, cfg.plies)
+    net = load(az, cfg, blob, cfg.batch)
+    pos = az.records_to_device(rec)
+    masks = torch.zeros((cfg.batch, 30), dtype=torch.int64, device="cuda")
+    az.az_legal_masks(pos, 128, cfg.batch, 2, masks)
+    policy = torch.zeros((cfg.batch, pw.ACTIONS), device="cuda")
+    value = torch.zeros((cfg.batch, 3), device="cuda")
+    with pytest.raises(az.AzError) as e:                      # refuses to run before its ranges are fixed
+        az.az_evaluate(net, pos, masks, cfg.batch, policy, value)
+    assert e.value.code == az.AZ_ERR_NOT_CALIBRATED
+    az.az_calibrate(net, az.records_to_device(cal), 512)
+    mg, pg, vg, tg = gpu_run(az, net, cfg, rec, tower=True)
+    az.az_free_net(net)
+    rows = np.arange(0, cfg.batch, 4)
+    mo, _, po, vo, extra = oracle.pnet_evaluate(blob, rec[rows], want_tower=True)
+    assert (mg[rows] == mo).all()
+    want = extra["tower"].reshape(rows.size, 128, 64).transpose(0, 2, 1)
+    rel = float(np.sqrt(((tg[rows] - want) ** 2).mean() / (want ** 2).mean()))
+    perr, verr = np.abs(pg[rows] - po).max(), np.abs(vg[rows] - vo).max()
+    agree = (pg[rows].argmax(axis=1) == po.argmax(axis=1)).mean()
+    print(f"p12i: n={rows.size} of {cfg.batch} policy max-abs {perr:.3e} value max-abs {verr:.3e} arg-max agreement {agree:.4f} backbone rms {rel:.3e}")
+    assert perr <= 5e-2 and verr <= 5e-2 and rel < 3e-2
+    assert tg.min() >= 0.0 and tg.max() <= 6.0
 
 
 def test_other_entry_points_serve_the_papers_network_too():
