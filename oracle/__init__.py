@@ -64,6 +64,8 @@ def _load():
         lib.orc_encode.argtypes = [vp, ci, ci, ci, vp]
         lib.orc_encode52.restype = ci
         lib.orc_encode52.argtypes = [vp, ci, ci, vp]
+        lib.orc_apply_moves.restype = ci
+        lib.orc_apply_moves.argtypes = [vp, ci, ci, ci, vp, vp]
         lib.orc_pnet_forward.restype = ci
         lib.orc_pnet_forward.argtypes = [vp, ctypes.c_size_t, vp, vp, ci, vp, vp, vp, vp]
         lib.orc_conv3x3.restype = None
@@ -127,6 +129,16 @@ def encode(records, in_planes: int) -> np.ndarray:
     if _load().orc_encode(rec.ctypes.data, stride, n, in_planes, planes.ctypes.data) != 0:
         raise ValueError("unsupported plane count")
     return planes
+
+
+def apply_moves(records, head: int, actions) -> np.ndarray:
+    """Successor records (same layout) of `records` after the legal actions `actions` (policy indices of `head`)."""
+    rec, stride, n = _records(records)
+    act = np.ascontiguousarray(actions, dtype=np.int32)
+    out = np.zeros_like(rec)
+    if _load().orc_apply_moves(rec.ctypes.data, stride, n, head, act.ctypes.data, out.ctypes.data) != 0:
+        raise ValueError("an action is not a legal move of its position")
+    return out
 
 
 def encode52(records) -> np.ndarray:

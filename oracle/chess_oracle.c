@@ -527,3 +527,65 @@ int orc_encode52(const void *records, int stride, int n, double *planes_out) {
     }
     return 0;
 }
+
+/* ---- applying an action to a position (the step a search tree takes from a node to its child) ----
+ * actions[i] is a policy index of `head` (0: 73 planes, 1: 1,858 list, 2: 1,880 list) that is legal
+ * in records[i]; out[i] receives the successor in the same record layout (stride 104, 784 or 128):
+ * bitboards, side to move, castling rights (lost when the king or a rook leaves its home square or a
+ * rook is captured there), en-passant square (set behind a pawn that advanced two ranks, else 64),
+ * halfmove clock (0 after a pawn move or a capture, else one more, saturating at 255), repetitions 0
+ * (a successor built this way does not know its game's earlier positions).  Records with history
+ * get the old position pushed onto their seven boards, records with moves the move pushed onto
+ * their eight (castling as the king's own move).  In the 73-plane and 1,858 lists a pawn that
+ * reaches the last rank through a plain action becomes a queen.  Returns 0, or -1 if an action is
+ * not a legal move of its position. */
+int orc_apply_moves(const void *records, int stride, int n, int head, const int32_t *actions, void *out) {
+    for (int i = 0; i < n; ++i) {
+        const PosRecord *r = (const PosRecord *)((const char *)records + (size_t)i * stride);
+        char *dst = (char *)out + (size_t)i * stride;
+        MBoard b; load_record(r, &b);
+        MMove list[256];
+        int k = gen_legal(&b, list), found = -1;
+        for (int j = 0; j < k && found < 0; ++j) {
+            int castle = list[j].flag == 3 ? 1 : list[j].flag == 4 ? 2 : 0;
+            if (orc_policy_index(head, b.stm, list[j].from, list[j].to, list[j].promo, castle) == actions[i]) found = j;
+        }
+        if (found < 0) return -1;
+        const MMove mv = list[found];
+        const int piece = b.sq[mb(mv.from)];
+        const int pawn = piece == 1 || piece == 7;
+        const int capture = b.sq[mb(mv.to)] != EMPTY || mv.flag == 2;
+        play(&b, &mv);
+        memcpy(dst, r, (size_t)stride);
+        PosRecord *o = (PosRecord *)dst;
+        memset(o->pieces, 0, sizeof o->pieces);
+        for (int s = 0; s < 64; ++s) {
+            int p = b.sq[mb(s)];
+            if (p != EMPTY) o->pieces[p - 1] |= 1ULL << s;
+        }
+        o->stm = (uint8_t)b.stm;
+        o->castling = (uint8_t)b.castling;
+        o->ep_square = (uint8_t)(b.ep ? sq64(b.ep) : 64);
+        o->halfmove = (uint8_t)((pawn || capture) ? 0 : (r->halfmove < 255 ? r->halfmove + 1 : 255));
+        o->repetitions = 0;
+        if (stride == (int)sizeof(PosRecordH8)) {
+            const PosRecordH8 *h = (const PosRecordH8 *)r;
+            PosRecordH8 *oh = (PosRecordH8 *)dst;
+            for (int t = 6; t >= 1; --t) {
+                memcpy(oh->hist_pieces[t], h->hist_pieces[t - 1], sizeof h->hist_pieces[0]);
+                oh->hist_rep[t] = h->hist_rep[t - 1];
+            }
+            memcpy(oh->hist_pieces[0], r->pieces, sizeof r->pieces);
+            oh->hist_rep[0] = r->repetitions;
+            oh->n_hist = (uint8_t)(h->n_hist < 7 ? h->n_hist + 1 : 7);
+        } else if (stride == (int)sizeof(PosRecordM8)) {
+            const PosRecordM8 *m = (const PosRecordM8 *)r;
+            PosRecordM8 *om = (PosRecordM8 *)dst;
+            for (int t = 7; t >= 1; --t) { om->move_from[t] = m->move_from[t - 1]; om->move_to[t] = m->move_to[t - 1]; }
+            om->move_from[0] = (uint8_t)mv.from;
+            om->move_to[0] = (uint8_t)mv.to;
+            om->n_moves = (uint8_t)(m->n_moves < 8 ? m->n_moves + 1 : 8);
+        }
+    }
+    return 0;
+}
