@@ -15,7 +15,7 @@ import subprocess
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SOURCES = ("chess_oracle.c", "net_oracle.c", "pnet_oracle.c")
+_SOURCES = ("chess_oracle.c", "net_oracle.c", "pnet_oracle.c", "mcts_oracle.c")
 _lib = None
 
 
@@ -39,7 +39,7 @@ def build() -> str:
     out = os.path.join(_HERE, f"liboracle_{h.hexdigest()[:10]}_{_cpu_tag()}.so")
     if not os.path.exists(out):
         tmp = out + f".tmp{os.getpid()}"
-        cmd = ["gcc", "-O3", "-march=native", "-std=c11", "-fopenmp", "-shared", "-fPIC",
+        cmd = ["gcc", "-O3", "-march=native", "-std=c11", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC",
                *[os.path.join(_HERE, s) for s in _SOURCES], "-lm", "-o", tmp]
         subprocess.run(cmd, check=True)
         os.replace(tmp, out)
@@ -66,6 +66,13 @@ def _load():
         lib.orc_encode52.argtypes = [vp, ci, ci, vp]
         lib.orc_apply_moves.restype = ci
         lib.orc_apply_moves.argtypes = [vp, ci, ci, ci, vp, vp]
+        lib.orc_in_check.restype = ci
+        lib.orc_in_check.argtypes = [vp]
+        lib.orc_synth_eval.restype = ci
+        lib.orc_synth_eval.argtypes = [vp, ci, ctypes.c_uint64, vp, vp, vp]
+        lib.orc_mcts_search.restype = ci
+        lib.orc_mcts_search.argtypes = [vp, ci, ci, ci, ci, ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_uint64,
+                                        ci, ci, vp, vp, vp, vp, vp, vp, vp]
         lib.orc_pnet_forward.restype = ci
         lib.orc_pnet_forward.argtypes = [vp, ctypes.c_size_t, vp, vp, ci, vp, vp, vp, vp]
         lib.orc_conv3x3.restype = None
@@ -139,6 +146,42 @@ def apply_moves(records, head: int, actions) -> np.ndarray:
     if _load().orc_apply_moves(rec.ctypes.data, stride, n, head, act.ctypes.data, out.ctypes.data) != 0:
         raise ValueError("an action is not a legal move of its position")
     return out
+
+
+def synth_eval(record, head: int, seed: int):
+    """The stand-in evaluator of the search tests: (actions, priors float32, value float32) of one position."""
+    rec = np.ascontiguousarray(record)
+    actions = np.zeros(256, dtype=np.int32)
+    priors = np.zeros(256, dtype=np.float32)
+    value = np.zeros(1, dtype=np.float32)
+    k = _load().orc_synth_eval(rec.ctypes.data, head, seed, actions.ctypes.data, priors.ctypes.data, value.ctypes.data)
+    if k < 0:
+        raise RuntimeError("a legal move had no policy index")
+    return actions[:k].copy(), priors[:k].copy(), float(value[0])
+
+
+def mcts_search(record, head: int, simulations: int, leaves: int = 1, c_puct: float = 1.5, fpu_reduction: float = 0.2,
+                discount: float = 0.99, seed: int = 0, node_cap: int | None = None, edge_cap: int | None = None) -> dict:
+    """Sequential tree search of one game with the stand-in evaluator (Eq. 1; constants of App. D.2)."""
+    rec, stride, n = _records(record)
+    assert n == 1
+    node_cap = node_cap or simulations * leaves + 2
+    edge_cap = edge_cap or node_cap * 64
+    actions = np.zeros(256, dtype=np.int32)
+    visits = np.zeros(256, dtype=np.int32)
+    w = np.zeros(256, dtype=np.float32)
+    prior = np.zeros(256, dtype=np.float32)
+    counts = np.zeros(4, dtype=np.int32)
+    nvis = np.zeros(node_cap, dtype=np.int32)
+    wsum = np.zeros(node_cap, dtype=np.float32)
+    k = _load().orc_mcts_search(rec.ctypes.data, stride, head, simulations, leaves, c_puct, fpu_reduction, discount, seed,
+                                node_cap, edge_cap, actions.ctypes.data, visits.ctypes.data, w.ctypes.data,
+                                prior.ctypes.data, counts.ctypes.data, nvis.ctypes.data, wsum.ctypes.data)
+    if k < 0:
+        raise ValueError("bad search arguments")
+    return {"actions": actions[:k].copy(), "visits": visits[:k].copy(), "w": w[:k].copy(), "prior": prior[:k].copy(),
+            "n_nodes": int(counts[0]), "n_edges": int(counts[1]), "flags": int(counts[2]), "idle": int(counts[3]),
+            "node_nvis": nvis[:counts[0]].copy(), "node_wsum": wsum[:counts[0]].copy()}
 
 
 def encode52(records) -> np.ndarray:

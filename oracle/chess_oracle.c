@@ -589,3 +589,9 @@ int orc_apply_moves(const void *records, int stride, int n, int head, const int3
     }
     return 0;
 }
+
+/* 1 iff the side to move of `record` is in check. */
+int orc_in_check(const void *record) {
+    MBoard b; load_record((const PosRecord *)record, &b);
+    return is_attacked(&b, find_king(&b, b.stm), b.stm ^ 1);
+}

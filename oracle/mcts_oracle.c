@@ -1,0 +1,216 @@
+/* TEST INFRASTRUCTURE: a plain, sequential tree search (Sec. 3.4 "Search and self-play", Eq. 1;
+ * Sec. 4.1 parallel leaves; App. D.2 search constants), one game at a time, against which the GPU
+ * search driver is compared.  Only tests, the smoke check and the benchmark's CPU baseline may use it.
+ *
+ * Readings of the paper taken here (the paper gives the rule and the constants, not the bookkeeping):
+ *  - statistics live on the edges: N(s,a), W(s,a), Q = W/N; N(s) of Eq. 1 is the sum of N(s,a) over
+ *    the node's edges (the form in which max(1, N) matters);
+ *  - an edge without visits takes Q = V(s) - 0.2, V(s) the mean of all values backed up through s
+ *    (its own evaluation included) from the point of view of the player to move at s;
+ *  - a backed-up value changes sign and is multiplied by the discount at every ply it climbs;
+ *  - a reservation (parallel leaves) counts on its edges as one visit that lost: N + m visits,
+ *    W - m value; it is removed when the traversal's result arrives.  A traversal that runs into a
+ *    node still waiting for its evaluation is given up (its reservations are removed, its slot idles);
+ *  - a node is terminal if the mover has no legal move (value -1 in check, else 0) or the halfmove
+ *    clock has reached 100 (value 0); repetitions are not tracked inside the tree;
+ *  - the root's evaluation is a step of its own before the counted simulations.
+ * Every decision (the arg-max of Eq. 1) is taken in float32 with one rounding per operation, in the
+ * order written below, ties to the lower action index.
+ *
+ * The evaluator is the deterministic stand-in described at synth_eval(): priors and value are pure
+ * functions of the position and a seed, in arithmetic that rounds the same way everywhere. */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#include <math.h>
+
+int orc_legal_masks(const void *records, int stride, int n, int head, uint64_t *masks);
+int orc_apply_moves(const void *records, int stride, int n, int head, const int32_t *actions, void *out);
+int orc_in_check(const void *record);
+
+#define MAX_STRIDE 784
+#define MAX_DEPTH 128
+
+typedef struct {
+    uint64_t pieces[12];
+    uint8_t stm, castling, ep_square, halfmove, repetitions, pad[3];
+} Cur;
+
+typedef struct { int action, child, n, m; float prior, w; } Edge;
+typedef struct {
+    int edge_begin, n_edges;      /* n_edges < 0: waiting for its evaluation */
+    int terminal; float tvalue;
+    int nvis; float wsum;         /* values backed up through the node, its own first */
+    int nsum;                     /* sum over edges of N + m */
+    unsigned char rec[MAX_STRIDE];
+} Node;
+
+static uint64_t mix64(uint64_t x) {
+    x ^= x >> 30; x *= 0xbf58476d1ce4e5b9ULL;
+    x ^= x >> 27; x *= 0x94d049bb133111ebULL;
+    x ^= x >> 31;
+    return x;
+}
+
+/* Stand-in evaluator: key = hash of the twelve bitboards, side to move, castling rights and en-passant
+ * square under `seed`.  Legal action a gets the integer weight 1 + r*r/64, r the top ten bits of
+ * mix64(key + (a + 1) * 0x9e3779b97f4a7c15); its prior is weight / sum of weights (one float32 division).
+ * The value is 0.75 * (t * 2^-23 - 1), t the top 24 bits of mix64(key ^ 0x5851f42d4c957f2d). */
+static uint64_t position_key(const Cur *c, uint64_t seed) {
+    uint64_t h = mix64(seed);
+    for (int i = 0; i < 12; ++i) h = mix64(h ^ c->pieces[i]);
+    return mix64(h ^ ((uint64_t)c->stm | (uint64_t)c->castling << 8 | (uint64_t)c->ep_square << 16));
+}
+static int synth_weight(uint64_t key, int action) {
+    const int r = (int)(mix64(key + (uint64_t)(action + 1) * 0x9e3779b97f4a7c15ULL) >> 54);
+    return 1 + r * r / 64;
+}
+static float synth_value(uint64_t key) {
+    const int t = (int)(mix64(key ^ 0x5851f42d4c957f2dULL) >> 40);
+    const float u = (float)t * 0x1p-23f - 1.0f;
+    return u * 0.75f;
+}
+
+int orc_synth_eval(const void *record, int head, uint64_t seed, int32_t *actions, float *priors, float *value) {
+    uint64_t mask[73];
+    const int words = head == 0 ? 73 : 30;
+    if (orc_legal_masks(record, 104, 1, head, mask) != 0) return -1;
+    const uint64_t key = position_key((const Cur *)record, seed);
+    int k = 0, sum = 0, w[256];
+    for (int i = 0; i < words * 64 && k < 256; ++i)
+        if (mask[i >> 6] >> (i & 63) & 1) { actions[k] = i; w[k] = synth_weight(key, i); sum += w[k]; ++k; }
+    for (int i = 0; i < k; ++i) priors[i] = (float)w[i] / (float)sum;
+    *value = synth_value(key);
+    return k;
+}
+
+typedef struct {
+    Node *nodes; Edge *edges;
+    int n_nodes, n_edges, node_cap, edge_cap;
+    int stride, head;
+    float c_puct, fpu_reduction, discount;
+    uint64_t seed;
+    uint32_t flags;               /* 1: node pool full, 2: edge pool full, 4: depth limit */
+    int root_submitted, idle;     /* idle: traversals given up (collisions, full pools) */
+} Tree;
+
+typedef struct { int kind, leaf, depth; int path_e[MAX_DEPTH], path_n[MAX_DEPTH]; } Slot;
+enum { SLOT_NONE = 0, SLOT_EVAL = 1, SLOT_TERMINAL = 2 };
+
+static void undo(Tree *t, Slot *s) {
+    for (int d = 0; d < s->depth; ++d) { t->edges[s->path_e[d]].m -= 1; t->nodes[s->path_n[d]].nsum -= 1; }
+    s->kind = SLOT_NONE;
+    t->idle += 1;
+}
+
+static void descend(Tree *t, Slot *s) {
+    int node = 0;
+    s->depth = 0; s->kind = SLOT_NONE; s->leaf = -1;
+    if (!t->root_submitted) {                 /* the root's own evaluation, once; the step's other slots idle */
+        t->root_submitted = 1; s->kind = SLOT_EVAL; s->leaf = 0;
+        return;
+    }
+    for (;;) {
+        Node *nd = &t->nodes[node];
+        if (nd->terminal) { s->kind = SLOT_TERMINAL; s->leaf = node; return; }
+        if (nd->n_edges < 0) { undo(t, s); return; }
+        if (s->depth == MAX_DEPTH) { t->flags |= 4; undo(t, s); return; }
+        const float sqrt_n = sqrtf((float)(nd->nsum > 1 ? nd->nsum : 1));
+        const float fpu = nd->wsum / (float)nd->nvis - t->fpu_reduction;
+        int best = -1; float best_score = 0.0f;
+        for (int i = 0; i < nd->n_edges; ++i) {
+            const Edge *e = &t->edges[nd->edge_begin + i];
+            const int n = e->n + e->m;
+            const float q = n > 0 ? (e->w - (float)e->m) / (float)n : fpu;
+            float u = t->c_puct * e->prior;
+            u = u * sqrt_n;
+            u = u / (float)(1 + n);
+            const float score = q + u;
+            if (best < 0 || score > best_score) { best = i; best_score = score; }
+        }
+        Edge *e = &t->edges[nd->edge_begin + best];
+        e->m += 1; nd->nsum += 1;
+        s->path_e[s->depth] = nd->edge_begin + best; s->path_n[s->depth] = node; s->depth += 1;
+        if (e->child < 0) {
+            if (t->n_nodes == t->node_cap) { t->flags |= 1; undo(t, s); return; }
+            const int child = t->n_nodes++;
+            Node *c = &t->nodes[child];
+            memset(c, 0, sizeof *c);
+            c->n_edges = -1;
+            int32_t a = e->action;
+            orc_apply_moves(nd->rec, t->stride, 1, t->head, &a, c->rec);
+            e->child = child;
+            s->kind = SLOT_EVAL; s->leaf = child;
+            return;
+        }
+        node = e->child;
+    }
+}
+
+static void finish(Tree *t, Slot *s) {
+    if (s->kind == SLOT_NONE) return;
+    Node *nd = &t->nodes[s->leaf];
+    float v;
+    if (s->kind == SLOT_EVAL) {
+        int32_t actions[256]; float priors[256], value;
+        const int k = orc_synth_eval(nd->rec, t->head, t->seed, actions, priors, &value);
+        const Cur *c = (const Cur *)nd->rec;
+        nd->nsum = 0;
+        if (k == 0) { nd->terminal = 1; nd->tvalue = orc_in_check(nd->rec) ? -1.0f : 0.0f; nd->n_edges = 0; }
+        else if (c->halfmove >= 100) { nd->terminal = 1; nd->tvalue = 0.0f; nd->n_edges = 0; }
+        else if (t->n_edges + k > t->edge_cap) { t->flags |= 2; nd->terminal = 1; nd->tvalue = value; nd->n_edges = 0; }
+        else {
+            nd->edge_begin = t->n_edges; nd->n_edges = k; t->n_edges += k;
+            for (int i = 0; i < k; ++i) {
+                Edge *e = &t->edges[nd->edge_begin + i];
+                e->action = actions[i]; e->prior = priors[i]; e->child = -1; e->n = 0; e->m = 0; e->w = 0.0f;
+            }
+        }
+        v = nd->terminal ? nd->tvalue : value;
+    } else {
+        v = nd->tvalue;
+    }
+    nd->nvis += 1; nd->wsum += v;
+    for (int d = s->depth - 1; d >= 0; --d) {
+        v = -v * t->discount;
+        Edge *e = &t->edges[s->path_e[d]];
+        e->n += 1; e->w += v; e->m -= 1;
+        Node *p = &t->nodes[s->path_n[d]];
+        p->nvis += 1; p->wsum += v;
+    }
+}
+
+/* One search from `root_record`: the root's evaluation, then `simulations` steps of `leaves` traversals each
+ * (all traversals of a step choose their paths before any of the step's results arrive).
+ * Out: the root's edges (action, visits, value sum, prior; at most 256), the counts of nodes and edges,
+ * per node (node_cap entries) its visit count and value sum, and the flags.  Returns the root's edge count. */
+int orc_mcts_search(const void *root_record, int stride, int head, int simulations, int leaves,
+                    float c_puct, float fpu_reduction, float discount, uint64_t seed, int node_cap, int edge_cap,
+                    int32_t *root_actions, int32_t *root_visits, float *root_w, float *root_prior,
+                    int32_t *counts /* n_nodes, n_edges, flags, idle */, int32_t *node_nvis, float *node_wsum) {
+    if (stride > MAX_STRIDE || leaves < 1 || leaves > 64) return -1;
+    Tree t;
+    memset(&t, 0, sizeof t);
+    t.nodes = (Node *)calloc((size_t)node_cap, sizeof(Node));
+    t.edges = (Edge *)calloc((size_t)edge_cap, sizeof(Edge));
+    t.node_cap = node_cap; t.edge_cap = edge_cap; t.stride = stride; t.head = head;
+    t.c_puct = c_puct; t.fpu_reduction = fpu_reduction; t.discount = discount; t.seed = seed;
+    memcpy(t.nodes[0].rec, root_record, (size_t)stride);
+    t.nodes[0].n_edges = -1;
+    t.n_nodes = 1;
+    Slot *slots = (Slot *)calloc((size_t)leaves, sizeof(Slot));
+    for (int step = -1; step < simulations; ++step) {
+        for (int j = 0; j < leaves; ++j) descend(&t, &slots[j]);
+        for (int j = 0; j < leaves; ++j) finish(&t, &slots[j]);
+    }
+    const Node *root = &t.nodes[0];
+    for (int i = 0; i < root->n_edges && i < 256; ++i) {
+        const Edge *e = &t.edges[root->edge_begin + i];
+        root_actions[i] = e->action; root_visits[i] = e->n; root_w[i] = e->w; root_prior[i] = e->prior;
+    }
+    counts[0] = t.n_nodes; counts[1] = t.n_edges; counts[2] = (int32_t)t.flags; counts[3] = t.idle;
+    for (int i = 0; i < t.n_nodes; ++i) { node_nvis[i] = t.nodes[i].nvis; node_wsum[i] = t.nodes[i].wsum; }
+    const int k = root->n_edges;
+    free(slots); free(t.nodes); free(t.edges);
+    return k;
+}

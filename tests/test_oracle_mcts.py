@@ -1,0 +1,133 @@
+"""Pins of the oracle's tree search (Eq. 1, Sec. 3.4; constants of App. D.2) and of the stand-in evaluator
+it searches with: bookkeeping invariants, the first two selections recomputed by hand from Eq. 1, forced
+mates whose backed-up value the discount fixes, and the accounting of parallel leaves."""
+import numpy as np
+import pytest
+
+import oracle
+from inputs import positions
+
+START = "rnbqkbnr/pppppppp/8/8/8/8/PPPPPPPP/RNBQKBNR w KQkq - 0 1"
+MATE_IN_1 = "6k1/5ppp/8/8/8/8/8/R3K3 w Q - 0 1"          # Ra8 mates
+MATE_IN_2 = "7k/8/5K2/8/8/8/8/6R1 w - - 0 1"             # king and rook against a cornered king: mate in two, none in one
+
+
+def sq(name):
+    return (ord(name[0]) - 97) + 8 * (int(name[1]) - 1)
+
+
+def test_stand_in_evaluator_is_a_distribution_over_the_legal_actions():
+    rec, _ = positions.generate(5, 30, (2, 80))
+    cur = np.ascontiguousarray(rec["cur"])
+    values = []
+    for i in range(30):
+        for head, size in ((1, 1858), (2, 1880)):
+            a, p, v = oracle.synth_eval(cur[i], head, 7)
+            mask = oracle.legal_masks(cur[i:i + 1], head)[0]
+            bits = np.flatnonzero(np.unpackbits(mask.view(np.uint8), bitorder="little")[:size])
+            assert (a == bits).all() and (p > 0).all() and abs(float(p.astype(np.float64).sum()) - 1) < 1e-5
+            assert -0.75 <= v < 0.75
+        a2, p2, v2 = oracle.synth_eval(cur[i], 2, 8)
+        assert v2 != v or not np.array_equal(p2, p)          # the seed matters
+        values.append(v)
+    assert len(set(values)) > 25 and min(values) < -0.3 and max(values) > 0.3
+    a, p, v = oracle.synth_eval(cur[0], 2, 7)
+    b, q, w = oracle.synth_eval(cur[0], 2, 7)
+    assert np.array_equal(p, q) and v == w
+
+
+@pytest.mark.parametrize("head", [1, 2])
+def test_bookkeeping_invariants(head):
+    rec = positions.record_from_fen(START)
+    r = oracle.mcts_search(rec, head, 300)
+    assert r["flags"] == 0 and r["idle"] == 0
+    assert r["visits"].sum() == 300 and r["n_nodes"] == 301          # every traversal ends in a new node here
+    assert r["node_nvis"][0] == 301 and (r["node_nvis"][1:] >= 1).all()
+    assert len(r["actions"]) == 20 and abs(float(r["prior"].sum()) - 1) < 1e-5
+    # a node's visits = its own evaluation + the traversals that went on through it: the sum over all nodes
+    # counts each traversal once per node of its path
+    assert r["node_nvis"].sum() > 2 * 300
+    q = r["w"][r["visits"] > 0] / r["visits"][r["visits"] > 0]
+    assert (np.abs(q) <= 0.99 * 0.75 + 1e-6).all()                    # |value| <= 0.75, one ply of discount at least
+
+
+def test_first_two_selections_follow_eq_1():
+    rec, _ = positions.generate(11, 24, (2, 60))
+    cur = np.ascontiguousarray(rec["cur"])
+    checked = 0
+    for i in range(24):
+        a, p, v0 = oracle.synth_eval(cur[i], 1, 3)
+        if len(a) < 2:
+            continue
+        one = oracle.mcts_search(cur[i:i + 1], 1, 1, seed=3)
+        first = int(np.argmax(p))                                      # all Q equal: the largest prior wins, first of equals
+        assert one["visits"][first] == 1 and one["visits"].sum() == 1
+        child = oracle.apply_moves(cur[i:i + 1], 1, [int(a[first])])
+        ca, cp, v1 = oracle.synth_eval(child[0], 1, 3)
+        if len(ca) == 0 or child[0]["halfmove"] >= 100:
+            continue
+        w1 = -0.99 * v1
+        assert abs(float(one["w"][first]) - w1) < 1e-6
+        fpu = (v0 + w1) / 2 - 0.2
+        score = fpu + 1.5 * p.astype(np.float64) * 1.0 / 1.0           # sqrt(max(1, N(s))) with N(s) = 1
+        score[first] = w1 + 1.5 * float(p[first]) * 1.0 / 2.0
+        order = np.sort(score)
+        if order[-1] - order[-2] < 1e-5:
+            continue                                                    # too close to call in float64
+        second = int(np.argmax(score))
+        two = oracle.mcts_search(cur[i:i + 1], 1, 2, seed=3)
+        want = np.zeros(len(a), dtype=np.int32)
+        want[first] += 1
+        want[second] += 1
+        assert (two["visits"] == want).all()
+        checked += 1
+    assert checked >= 15
+
+
+def test_forced_mates_back_up_the_discounted_result():
+    rec = positions.record_from_fen(MATE_IN_1)
+    r = oracle.mcts_search(rec, 2, 400)
+    mate = oracle.policy_index(2, 0, sq("a1"), sq("a8"))
+    i = int(np.flatnonzero(r["actions"] == mate)[0])
+    assert r["visits"][i] > 200 and abs(float(r["w"][i]) / int(r["visits"][i]) - 0.99) < 1e-5
+    assert r["n_nodes"] < 400                                           # visits of the mated node open no new node
+    rec = positions.record_from_fen(MATE_IN_2)
+    r = oracle.mcts_search(rec, 2, 4000)
+    # White mates by force but not in one move: the search settles on a winning line, and no root move can be
+    # worth more than a mate three plies below it
+    i = int(np.argmax(r["visits"]))
+    assert r["visits"][i] > 2000
+    q = r["w"].astype(np.float64) / np.maximum(r["visits"], 1)
+    assert 0.85 < q[i] and (q <= 0.99 ** 3 + 1e-6).all()
+
+
+def test_stalemate_and_fifty_move_leaves_are_draws():
+    # Black to move is stalemated: the root itself is terminal, every traversal ends there with value 0
+    r = oracle.mcts_search(positions.record_from_fen("7k/5Q2/6K1/8/8/8/8/8 b - - 0 1"), 2, 10)
+    assert len(r["actions"]) == 0 and r["n_nodes"] == 1 and r["node_nvis"][0] == 11 and r["node_wsum"][0] == 0
+    # halfmove clock 99: every quiet successor is a fifty-move draw, captures and pawn moves are not
+    r = oracle.mcts_search(positions.record_from_fen("4k3/8/8/8/8/8/4P3/4K3 w - - 99 80"), 2, 50)
+    pawn = {oracle.policy_index(2, 0, sq("e2"), sq("e3")), oracle.policy_index(2, 0, sq("e2"), sq("e4"))}
+    for a, n, w in zip(r["actions"], r["visits"], r["w"]):
+        if int(a) not in pawn and n > 0:
+            assert w == 0
+
+
+@pytest.mark.parametrize("leaves", [2, 8])
+def test_parallel_leaves_accounting(leaves):
+    rec = positions.record_from_fen(START)
+    r = oracle.mcts_search(rec, 2, 100, leaves=leaves)
+    # the root's step idles its other slots; afterwards every traversal is either counted or given up
+    assert r["visits"].sum() + r["idle"] == 100 * leaves + (leaves - 1)
+    assert r["n_nodes"] == 1 + r["visits"].sum()
+    # the traversals of the first counted step take different root moves: a reservation counts as a lost visit
+    one = oracle.mcts_search(rec, 2, 1, leaves=leaves)
+    assert one["visits"].max() == 1 and one["visits"].sum() == leaves
+
+
+def test_pools_that_fill_up_are_reported():
+    rec = positions.record_from_fen(START)
+    r = oracle.mcts_search(rec, 2, 100, node_cap=40, edge_cap=40 * 64)
+    assert r["flags"] & 1 and r["n_nodes"] == 40 and r["visits"].sum() + r["idle"] == 100
+    r = oracle.mcts_search(rec, 2, 100, node_cap=128, edge_cap=300)
+    assert r["flags"] & 2 and r["n_edges"] <= 300 and r["visits"].sum() == 100
