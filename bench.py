@@ -38,7 +38,14 @@ WORKLOADS = {
     "p12i": "p12i: p12 with the backbone's convolutions in int8 (pooled context and heads in floating point), batch 1024",
     "p14": "p14: the paper's own network at its reported size, 14x160 bf16, batch 320 as the paper serves it "
            "(App. D.3); --batch for other sizes",
+    "s14": "s14: batched tree search (Eq. 1, c 1.5, first-play reduction 0.2, discount 0.99) over the paper's 14x160 "
+           "network: two groups of games, each step one batch of leaf positions per group (320 rows as the paper "
+           "serves, App. D.3; --batch for other sizes), one traversal per game and step",
+    "s12": "s12: the same search over the 12x128 network",
 }
+SEARCH_NETS = {"s14": "p14", "s12": "p12"}
+SEARCH_METRIC = "searches/sec (tree traversals with their leaf evaluation)"
+SEARCH_UNIT = "searches/s"
 
 
 def is_pnet(cfg) -> bool:
@@ -46,6 +53,7 @@ def is_pnet(cfg) -> bool:
 
 
 def get_config(name: str):
+    name = SEARCH_NETS.get(name, name)
     return pnet_weights.PNET_CONFIGS[name] if name in pnet_weights.PNET_CONFIGS else configs.CONFIGS[name]
 
 
@@ -184,6 +192,163 @@ def run_reference(args, cfg):
     }))
 
 
+def oracle_search_rate(recs, sims: int, games: int):
+    """The oracle's sequential search with its stand-in evaluator (no network) on `games` roots: (searches/s, seconds)."""
+    import oracle
+    t0 = time.perf_counter()
+    for g in range(games):
+        oracle.mcts_search(recs[g:g + 1], 2, sims, seed=1)
+    dt = time.perf_counter() - t0
+    return games * sims / dt, dt
+
+
+def run_search_reference(args, name):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = get_config(name)
+    recs = make_records(cfg, 64)
+    for _ in range(args.warmup):
+        oracle_search_rate(recs, 50, 2)
+    total_t, total_n = 0.0, 0
+    for _ in range(args.steps):
+        rate, dt = oracle_search_rate(recs, 400, 8)
+        total_t += dt
+        total_n += 8 * 400
+    value = total_n / total_t
+    sample_txt = ("8 games x 400 traversals per step, sequential, the oracle's stand-in evaluator in place of the network "
+                  "(the oracle has no network-backed search: an upper bound of its search rate)")
+    print(json.dumps({
+        "impl": "reference", "metric": SEARCH_METRIC, "value": value, "unit": SEARCH_UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOADS[name], "sample": sample_txt},
+        "cpu_baseline": {"value": value, "unit": SEARCH_UNIT, "cores": 1, "kind": "oracle", "sample": sample_txt},
+        "e2e": {"value": value, "unit": SEARCH_UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def run_search(args, name):
+    """Search workloads: a step is one search step of every game (one leaf batch per group)."""
+    import torch
+    import torch.distributed as dist
+
+    import paper_2609_37447_b200 as az
+    from paper_2609_37447_b200 import sharding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    cfg = get_config(name)
+    rows = args.batch if args.batch > 0 else 320
+    leaves = max(1, args.leaves)
+    games = 2 * rows // leaves
+    recs = make_records(cfg, games, first_index=sharding.rank_first_index(rank, games))
+    blob = make_blob(cfg)
+    net = az.az_load_net(az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, rows), blob)
+    nodes = (args.steps + args.warmup) * leaves + 2
+
+    def new_search():
+        sc = az.make_search_config(games, 2, 128, leaves=leaves, groups=2, max_nodes=nodes, max_edges=48 * nodes)
+        s = az.az_search_create(net, sc)
+        az.az_search_set_roots(s, recs)
+        return s
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    actions = np.zeros((games, az.AZ_MAX_LEGAL), dtype=np.int32)
+    visits = np.zeros((games, az.AZ_MAX_LEGAL), dtype=np.int32)
+    counts = np.zeros(games, dtype=np.int32)
+
+    def done(s):
+        az.az_search_root_visits(s, actions, visits, counts)
+        return int(sum(int(visits[g, :counts[g]].sum()) for g in range(games)))
+
+    # ---- device-timed: warm-up steps, then K steps queued in one call, timed by events on the search's stream
+    s = new_search()
+    az.az_search_run(s, args.warmup)
+    before = done(s)
+    az.az_profile_tower(net, True)
+    az.az_tower_time(net)
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    ms = az.az_search_run(s, args.steps)
+    barrier()
+    clocks = sampler.stop()
+    tower_ms, tower_passes = az.az_tower_time(net)
+    az.az_profile_tower(net, False)
+    searched = done(s) - before
+    flags = 0
+    for g in range(games):
+        flags |= int(az.az_search_tree(s, g, nodes=False)[0][2])
+    launches = az.az_search_launches_per_step(s) * 2 * args.steps
+    az.az_search_destroy(s)
+
+    # ---- end to end: roots from host memory, K steps (plus the roots' own), the root visit counts back to the host
+    s = new_search()
+    az.az_search_run(s, 3)
+    az.az_search_destroy(s)
+    barrier()
+    t0 = time.perf_counter()
+    s = new_search()
+    az.az_search_run(s, args.steps)
+    searched_e2e = done(s)
+    e2e_s = time.perf_counter() - t0
+    barrier()
+    az.az_search_destroy(s)
+    status = az.az_device_status(net)
+
+    ms_max, e2e_ms = sharding.max_over_ranks([ms, e2e_s * 1e3], device="cuda")
+    if rank == 0:
+        peaks = load_peaks()
+        flops = tower_flops_per_position(cfg) * rows
+        total_s = ms_max * 1e-3
+        achieved = flops * 2 * args.steps / total_s / 1e12
+        sustained = total_s >= 1.0
+        peak_tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"]
+        out = {
+            "metric": SEARCH_METRIC, "value": world * searched / total_s, "unit": SEARCH_UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_max / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": DTYPE[cfg.precision], "data": "synthetic",
+            "config": {"workload": WORKLOADS[name], "games_per_gpu": games, "rows_per_batch": rows, "leaves": leaves,
+                       "l2": "not flushed: the steps run back to back on the device without returning to the host; the trees "
+                             f"({games * nodes * (160 + 48 * 24) / 1e6:.0f} MB) exceed L2",
+                       "timing": "CUDA events around the queued steps on the search's stream; max over ranks",
+                       "device_status": status, "tree_flags": flags, "evaluations": rows * 2 * args.steps},
+            "e2e": {"value": world * searched_e2e / (e2e_ms * 1e-3), "unit": SEARCH_UNIT,
+                    "h2d_bytes_per_step": int(recs.nbytes / args.steps), "d2h_bytes_per_step": int((actions.nbytes + visits.nbytes + counts.nbytes) / args.steps),
+                    "ms_per_step": e2e_ms / args.steps,
+                    "api": "az_search_create + az_search_set_roots (roots from host memory) + az_search_run + az_search_root_visits "
+                           "(root visit counts to host memory); bytes are per step of the K-step search"},
+            "gpu_launches": launches,
+            "clocks": clocks,
+            "roofline": {"kernel": "tower_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
+                         "frac": achieved / peak_tf, "traffic": None,
+                         "peak_source": f"of {peaks['source']} ({'sustained' if sustained else 'burst'} bf16 GEMM)",
+                         "note": "whole-loop figure: the tower's flops of all leaf batches over the search's elapsed time (the two "
+                                 "groups' launches overlap, so a per-launch duration would count the shared time twice)",
+                         "avg_launch_ms_overlapped": tower_ms / max(tower_passes, 1), "launches_timed": tower_passes,
+                         "flops_per_launch": flops},
+        }
+        if not args.no_cpu_baseline:
+            rate, dt = oracle_search_rate(recs, 400, 16)
+            out["cpu_baseline"] = {"value": rate, "unit": SEARCH_UNIT, "cores": 1, "kind": "oracle",
+                                   "sample": f"16 games x 400 traversals, sequential, stand-in evaluator in place of the network "
+                                             f"(the oracle has no network-backed search), {dt:.1f} s"}
+        print(json.dumps(out))
+    az.az_free_net(net)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -193,9 +358,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures on a smaller case)")
+    ap.add_argument("--leaves", type=int, default=1, help="search workloads: traversals per tree and step")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.config in SEARCH_NETS:
+        if args.impl == "reference":
+            run_search_reference(args, args.config)
+        else:
+            run_search(args, args.config)
+        return
     cfg = get_config(args.config)
     if args.batch > 0:
         import dataclasses

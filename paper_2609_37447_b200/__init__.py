@@ -26,12 +26,26 @@ AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3 = 0, 1, 2
 EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
            "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_submit_host", "az_wait_host", "az_encode", "az_encode52", "az_tower", "az_tower_static", "az_legal_masks",
            "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
-           "az_last_cuda_error")
+           "az_last_cuda_error",
+           "az_apply_moves", "az_standin_evaluate", "az_search_create", "az_search_destroy", "az_search_set_roots",
+           "az_search_run", "az_search_root", "az_search_root_visits", "az_search_tree", "az_search_launches_per_step")
 
 
 class az_arch(ctypes.Structure):
     _fields_ = [(n, ctypes.c_uint32) for n in ("abi_version", "in_planes", "blocks", "channels",
                                                "policy_head", "value_head", "precision", "max_batch")]
+
+
+class az_search_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint32) for n in ("games", "leaves", "groups", "max_nodes", "max_edges", "evaluator",
+                                               "policy_head", "position_bytes")] + \
+               [("c_puct", ctypes.c_float), ("fpu_reduction", ctypes.c_float), ("discount", ctypes.c_float),
+                ("reserved", ctypes.c_uint32), ("seed", ctypes.c_uint64)]
+
+
+AZ_SEARCH_EVAL_NET, AZ_SEARCH_EVAL_STANDIN = 0, 1
+AZ_SEARCH_MAX_LEAVES, AZ_SEARCH_MAX_DEPTH = 16, 128
+AZ_SEARCH_FLAG_NODES_FULL, AZ_SEARCH_FLAG_EDGES_FULL, AZ_SEARCH_FLAG_DEPTH, AZ_SEARCH_FLAG_BAD_ACTION = 1, 2, 4, 8
 
 
 class AzError(RuntimeError):
@@ -93,6 +107,26 @@ def _load_library():
     lib.az_strerror.argtypes = [ci]
     lib.az_last_cuda_error.restype = ctypes.c_char_p
     lib.az_last_cuda_error.argtypes = []
+    lib.az_apply_moves.restype = ci
+    lib.az_apply_moves.argtypes = [vp, sz, ci, ci, vp, vp, vp, vp]
+    lib.az_standin_evaluate.restype = ci
+    lib.az_standin_evaluate.argtypes = [vp, sz, vp, ci, ci, ctypes.c_uint64, vp, vp, vp, vp]
+    lib.az_search_create.restype = ci
+    lib.az_search_create.argtypes = [vp, ctypes.POINTER(az_search_config), ctypes.POINTER(vp)]
+    lib.az_search_destroy.restype = None
+    lib.az_search_destroy.argtypes = [vp]
+    lib.az_search_set_roots.restype = ci
+    lib.az_search_set_roots.argtypes = [vp, vp]
+    lib.az_search_run.restype = ci
+    lib.az_search_run.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_float)]
+    lib.az_search_root.restype = ci
+    lib.az_search_root.argtypes = [vp, ci, vp, vp, vp, vp, ctypes.POINTER(ctypes.c_int32)]
+    lib.az_search_root_visits.restype = ci
+    lib.az_search_root_visits.argtypes = [vp, vp, vp, vp]
+    lib.az_search_tree.restype = ci
+    lib.az_search_tree.argtypes = [vp, ci, vp, vp, vp]
+    lib.az_search_launches_per_step.restype = ci
+    lib.az_search_launches_per_step.argtypes = [vp]
     return lib
 
 
@@ -296,6 +330,98 @@ def az_last_cuda_error() -> str:
 
 
 # ---- small marshalling helpers used by tests and the benchmark ----------------------------------
+
+def az_apply_moves(positions_dev, position_stride, batch, policy_head, actions_dev, out_positions_dev, status_dev=None, stream=None):
+    _check(_lib.az_apply_moves(_dev_ptr(positions_dev, "positions"), position_stride, batch, policy_head,
+                               _dev_ptr(actions_dev, "actions"), _dev_ptr(out_positions_dev, "out_positions"),
+                               _dev_ptr(status_dev, "status") if status_dev is not None else None, _stream_ptr(stream)),
+           "az_apply_moves")
+
+
+def az_standin_evaluate(positions_dev, position_stride, legal_masks_dev, batch, policy_head, seed, legal_policy_dev,
+                        legal_counts_dev, value_dev, stream=None):
+    _check(_lib.az_standin_evaluate(_dev_ptr(positions_dev, "positions"), position_stride, _dev_ptr(legal_masks_dev, "legal_masks"),
+                                    batch, policy_head, seed, _dev_ptr(legal_policy_dev, "legal_policy"),
+                                    _dev_ptr(legal_counts_dev, "legal_counts"), _dev_ptr(value_dev, "value"), _stream_ptr(stream)),
+           "az_standin_evaluate")
+
+
+@dataclass
+class Search:
+    """Handle of a batched tree search (owns the trees in device memory; call az_search_destroy when done)."""
+    handle: int
+    config: az_search_config
+
+
+def make_search_config(games, policy_head, position_bytes, leaves=1, groups=2, max_nodes=1024, max_edges=None,
+                       evaluator=AZ_SEARCH_EVAL_NET, c_puct=1.5, fpu_reduction=0.2, discount=0.99, seed=0) -> az_search_config:
+    return az_search_config(games, leaves, groups, max_nodes, max_edges or 64 * max_nodes, evaluator, policy_head,
+                            position_bytes, c_puct, fpu_reduction, discount, 0, seed)
+
+
+def az_search_create(net, config: az_search_config) -> Search:
+    out = ctypes.c_void_p()
+    _check(_lib.az_search_create(net.handle if net is not None else None, ctypes.byref(config), ctypes.byref(out)), "az_search_create")
+    return Search(out.value, config)
+
+
+def az_search_destroy(search: Search):
+    if search is not None and search.handle:
+        _lib.az_search_destroy(search.handle)
+        search.handle = 0
+
+
+def az_search_set_roots(search: Search, positions_host: np.ndarray):
+    rec = np.ascontiguousarray(positions_host)
+    if rec.nbytes != search.config.games * search.config.position_bytes:
+        raise ValueError("positions_host must hold one record per game")
+    _check(_lib.az_search_set_roots(search.handle, rec.ctypes.data), "az_search_set_roots")
+
+
+def az_search_run(search: Search, simulations: int) -> float:
+    """Runs `simulations` steps on every tree; returns the device time in milliseconds."""
+    ms = ctypes.c_float(0)
+    _check(_lib.az_search_run(search.handle, simulations, ctypes.byref(ms)), "az_search_run")
+    return float(ms.value)
+
+
+def az_search_root(search: Search, game: int):
+    """(actions, visits, value sums, priors) of the root's edges of one game."""
+    a = np.zeros(AZ_MAX_LEGAL, dtype=np.int32)
+    n = np.zeros(AZ_MAX_LEGAL, dtype=np.int32)
+    w = np.zeros(AZ_MAX_LEGAL, dtype=np.float32)
+    p = np.zeros(AZ_MAX_LEGAL, dtype=np.float32)
+    k = ctypes.c_int32(0)
+    _check(_lib.az_search_root(search.handle, game, a.ctypes.data, n.ctypes.data, w.ctypes.data, p.ctypes.data, ctypes.byref(k)),
+           "az_search_root")
+    return a[:k.value].copy(), n[:k.value].copy(), w[:k.value].copy(), p[:k.value].copy()
+
+
+def az_search_root_visits(search: Search, actions_host: np.ndarray, visits_host: np.ndarray, counts_host: np.ndarray):
+    """Root actions and visit counts of all games into int32 host arrays [games][AZ_MAX_LEGAL] (x2) and [games]."""
+    g = search.config.games
+    for arr, shape in ((actions_host, (g, AZ_MAX_LEGAL)), (visits_host, (g, AZ_MAX_LEGAL)), (counts_host, (g,))):
+        if arr.dtype != np.int32 or arr.shape != shape or not arr.flags.c_contiguous:
+            raise TypeError("int32 C-contiguous arrays of [games][AZ_MAX_LEGAL], [games][AZ_MAX_LEGAL], [games] expected")
+    _check(_lib.az_search_root_visits(search.handle, actions_host.ctypes.data, visits_host.ctypes.data, counts_host.ctypes.data),
+           "az_search_root_visits")
+
+
+def az_search_tree(search: Search, game: int, nodes: bool = True):
+    """counts (nodes, edges, flags, traversals given up) and, with nodes=True, per-node visit counts and value sums."""
+    counts = np.zeros(4, dtype=np.int32)
+    if not nodes:
+        _check(_lib.az_search_tree(search.handle, game, counts.ctypes.data, None, None), "az_search_tree")
+        return counts, None, None
+    nvis = np.zeros(search.config.max_nodes, dtype=np.int32)
+    wsum = np.zeros(search.config.max_nodes, dtype=np.float32)
+    _check(_lib.az_search_tree(search.handle, game, counts.ctypes.data, nvis.ctypes.data, wsum.ctypes.data), "az_search_tree")
+    return counts, nvis[:counts[0]].copy(), wsum[:counts[0]].copy()
+
+
+def az_search_launches_per_step(search: Search) -> int:
+    return int(_lib.az_search_launches_per_step(search.handle))
+
 
 def records_to_device(records: np.ndarray, device="cuda") -> torch.Tensor:
     """A numpy record array (104- or 784-byte records) as a uint8 device tensor [n][record_bytes]."""

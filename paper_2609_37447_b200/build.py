@@ -17,7 +17,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
 
 def _digest() -> str:
     h = hashlib.sha1(" ".join(NVCC_FLAGS).encode())
-    for path in sorted(glob.glob(os.path.join(CSRC, "*")) + [os.path.join(ROOT, "include", "az_eval.h")]):
+    for path in sorted(glob.glob(os.path.join(CSRC, "*")) + glob.glob(os.path.join(ROOT, "include", "*.h"))):
         with open(path, "rb") as f:
             h.update(path.encode() + f.read())
     return h.hexdigest()

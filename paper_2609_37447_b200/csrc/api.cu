@@ -322,6 +322,39 @@ int run_tower(Net &n, const void *positions, int batch, void **tower_out, bool f
 }
 
 }  // namespace
+
+// Second copy of what an evaluation keeps between its kernels, so that two evaluations of one az_net can
+// run side by side on two streams.  The tensor-core path keeps the head GEMM's operands and the logits,
+// the paper's network its backbone output and the queries/keys; the other paths have one workspace only.
+int ensure_second_workspace(Net &n, bool *available) {
+    const az_arch &a = n.arch;
+    const size_t B = a.max_batch;
+    *available = false;
+    if (n.pnet) {
+        if (!n.alt_act0) {
+            AZ_CUDA(cudaMalloc(&n.alt_act0, B * 64 * a.channels * sizeof(__nv_bfloat16)));
+            AZ_CUDA(cudaMalloc(&n.alt_pnet_qk, B * 64 * 256 * sizeof(float)));
+        }
+        *available = true;
+    } else if (n.tc_ready) {
+        if (!n.alt_u_value) {
+            const size_t u_bytes = (size_t)((a.max_batch + 127) / 128) * kHeadChannels * 64 * 128 * sizeof(__nv_bfloat16);
+            AZ_CUDA(cudaMalloc(&n.alt_u_value, u_bytes));
+            AZ_CUDA(cudaMemset(n.alt_u_value, 0, u_bytes));
+            if (n.u_policy) { AZ_CUDA(cudaMalloc(&n.alt_u_policy, u_bytes)); AZ_CUDA(cudaMemset(n.alt_u_policy, 0, u_bytes)); }
+            AZ_CUDA(cudaMalloc((void **)&n.alt_logits, B * az_policy_size(&a) * sizeof(float)));
+        }
+        *available = true;
+    }
+    return AZ_OK;
+}
+// Kernel arguments are captured when a kernel is launched: pointing the net at the other copy for the
+// duration of the (asynchronous) launches is all it takes.
+void swap_workspace(Net &n) {
+    if (n.pnet) { std::swap(n.act[0], n.alt_act0); std::swap(n.pnet_qk, n.alt_pnet_qk); }
+    else { std::swap(n.u_policy, n.alt_u_policy); std::swap(n.u_value, n.alt_u_value); std::swap(n.logits, n.alt_logits); }
+}
+
 }  // namespace az
 
 using az::Net;
@@ -535,22 +568,12 @@ int az_submit_host(az_net *net, const void *positions_host, const uint64_t *lega
         AZ_CUDA(cudaStreamCreateWithFlags(&n->s_in, cudaStreamNonBlocking));
         AZ_CUDA(cudaStreamCreateWithFlags(&n->s_out, cudaStreamNonBlocking));
         AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute[0], cudaStreamNonBlocking));
-        // The tensor-core path keeps nothing else between its kernels than the head GEMM's operands and
-        // the logits; with a second copy of those, odd slots run on a stream of their own.  The other
-        // paths share one workspace, so all their slots take turns on one stream.
-        if (n->pnet) {
-            // the paper's network keeps the backbone's output and the queries/keys between its two kernels
-            AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute[1], cudaStreamNonBlocking));
-            AZ_CUDA(cudaMalloc(&n->alt_act0, B * 64 * a.channels * sizeof(__nv_bfloat16)));
-            AZ_CUDA(cudaMalloc(&n->alt_pnet_qk, B * 64 * 256 * sizeof(float)));
-        } else if (n->tc_ready) {
-            const size_t u_bytes = (size_t)((a.max_batch + 127) / 128) * az::kHeadChannels * 64 * 128 * sizeof(__nv_bfloat16);
-            AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute[1], cudaStreamNonBlocking));
-            AZ_CUDA(cudaMalloc(&n->alt_u_value, u_bytes));
-            AZ_CUDA(cudaMemset(n->alt_u_value, 0, u_bytes));
-            if (n->u_policy) { AZ_CUDA(cudaMalloc(&n->alt_u_policy, u_bytes)); AZ_CUDA(cudaMemset(n->alt_u_policy, 0, u_bytes)); }
-            AZ_CUDA(cudaMalloc((void **)&n->alt_logits, B * ps * sizeof(float)));
-        }
+        // with a second copy of the workspace odd slots run on a stream of their own; the paths that share
+        // one workspace take turns on one stream
+        bool second = false;
+        const int rc2 = az::ensure_second_workspace(*n, &second);
+        if (rc2 != AZ_OK) return rc2;
+        if (second) AZ_CUDA(cudaStreamCreateWithFlags(&n->s_compute[1], cudaStreamNonBlocking));
     }
     Net::HostSlot &sl = n->slots[n->next_slot];
     if (sl.busy) return AZ_ERR_BUSY;
@@ -577,14 +600,10 @@ int az_submit_host(az_net *net, const void *positions_host, const uint64_t *lega
     AZ_CUDA(cudaStreamWaitEvent(sc, sl.in_ready, 0));
     // kernel arguments are captured when a kernel is launched: pointing the net at the other copy for
     // the duration of the (asynchronous) launches is all it takes
-    auto swap_workspace = [&]() {
-        if (n->pnet) { std::swap(n->act[0], n->alt_act0); std::swap(n->pnet_qk, n->alt_pnet_qk); }
-        else { std::swap(n->u_policy, n->alt_u_policy); std::swap(n->u_value, n->alt_u_value); std::swap(n->logits, n->alt_logits); }
-    };
-    if (alt) swap_workspace();
+    if (alt) az::swap_workspace(*n);
     const int rc = dense ? az_evaluate(net, sl.pos, sl.masks, batch, sl.policy, sl.value, sc)
                          : az_evaluate_legal(net, sl.pos, sl.masks, batch, sl.compact, sl.counts, sl.value, sc);
-    if (alt) swap_workspace();
+    if (alt) az::swap_workspace(*n);
     if (rc != AZ_OK) return rc;
     AZ_CUDA(cudaEventRecord(sl.computed, sc));
     AZ_CUDA(cudaStreamWaitEvent(n->s_out, sl.computed, 0));

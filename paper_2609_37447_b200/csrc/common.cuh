@@ -146,6 +146,10 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// second evaluation workspace (api.cu)
+int ensure_second_workspace(Net &n, bool *available);
+void swap_workspace(Net &n);
+
 // ---- kernels' launch functions (each returns AZ_OK or AZ_ERR_CUDA) ---------------------------
 int launch_encode52(const void *positions, int batch, bool bf16, void *planes, cudaStream_t s);
 int build_pnet(Net &n, const unsigned char *blob, size_t nbytes);

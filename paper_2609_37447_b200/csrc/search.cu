@@ -1,0 +1,797 @@
+// Batched tree search on the GPU (Sec. 3.4, Eq. 1; Sec. 4.1 parallel leaves; Sec. 5.1: many games
+// interleaved, two batches outstanding; App. D.2 constants).  The trees of all games live in device
+// memory; one step of a group of games is: select (one warp per game walks Eq. 1 from the root to an
+// edge without a child, reserving its path, and builds the successor position), the legal-move masks
+// of the new positions, their evaluation, expand-and-backup (one warp per game).  Nothing returns
+// to the host between steps.
+//
+// Every decision is float32 arithmetic with one rounding per operation (__fmul_rn and friends keep
+// the compiler from contracting them), so that a sequential host implementation of the same rules
+// reproduces the trees bit for bit.
+#include "common.cuh"
+#include "chess.cuh"
+#include "az_search.h"
+
+#include <mutex>
+#include <new>
+
+namespace az {
+namespace {
+
+constexpr int kWarps = 4;                        // warps (games, positions) per block
+constexpr int kMaxDepth = AZ_SEARCH_MAX_DEPTH;
+
+enum : int { kSlotNone = 0, kSlotEval = 1, kSlotTerminal = 2 };
+
+struct alignas(8) Edge {                         // 24 bytes
+    int action, child, n, m;
+    float prior, w;
+};
+struct alignas(16) Node {                        // 32 bytes
+    int edge_begin, n_edges;                     // n_edges < 0: waiting for its evaluation
+    int terminal; float tvalue;
+    int nvis; float wsum;                        // values backed up through the node, its own first
+    int nsum;                                    // sum over the edges of N + m
+    int pad;
+};
+struct GameState { int n_nodes, n_edges, flags, idle, root_submitted, pad[3]; };
+
+// inverse of the from-to numbering: pair number -> origin | destination << 6 (mover's orientation);
+// promotion combination -> origin file | destination file << 3
+__device__ unsigned short g_inv_pair[1792];
+__device__ unsigned char g_inv_promo[22];
+
+struct Move { int from, to, promo; };
+
+// policy index -> move in the mover's orientation (promo 0 none, 1 N, 2 B, 3 R, 4 Q)
+__device__ Move decode_action(int head, int action) {
+    Move mv{0, 0, 0};
+    if (head == AZ_POLICY_PLANES73) {
+        const int plane = action >> 6;
+        mv.from = action & 63;
+        int df, dr;
+        if (plane < 56) {
+            const int d = plane / 7, dist = plane % 7 + 1;         // N NE E SE S SW W NW
+            df = (d == 1 || d == 2 || d == 3) ? dist : (d == 5 || d == 6 || d == 7) ? -dist : 0;
+            dr = (d == 0 || d == 1 || d == 7) ? dist : (d == 3 || d == 4 || d == 5) ? -dist : 0;
+        } else if (plane < 64) {
+            const int k = plane - 56;                              // (1,2) (2,1) (2,-1) (1,-2) (-1,-2) (-2,-1) (-2,1) (-1,2)
+            const int adf = (k == 0 || k == 3 || k == 4 || k == 7) ? 1 : 2;
+            df = k < 4 ? adf : -adf;
+            dr = (k == 0 || k == 1 || k == 6 || k == 7) ? 3 - adf : adf - 3;
+        } else {
+            mv.promo = (plane - 64) / 3 + 1;
+            df = (plane - 64) % 3 - 1;
+            dr = 1;
+        }
+        mv.to = mv.from + df + 8 * dr;
+    } else if (action < 1792) {
+        const unsigned e = g_inv_pair[action];
+        mv.from = e & 63; mv.to = e >> 6;
+    } else {
+        const int per = head == AZ_POLICY_FLAT1858 ? 3 : 4;
+        const int k = (action - 1792) / per, j = (action - 1792) % per;
+        const unsigned e = g_inv_promo[k < 22 ? k : 0];
+        mv.from = 48 + (e & 7); mv.to = 56 + (e >> 3);
+        mv.promo = head == AZ_POLICY_FLAT1858 ? j + 1 : 4 - j;     // 1,858: N B R; 1,880: Q R B N
+    }
+    return mv;
+}
+
+// The warp writes the successor of record `in` under `action` to `out` (global memory, distinct from in).
+// Returns false (all lanes) if the action's origin holds no piece of the mover; out is then a copy.
+__device__ bool apply_action_warp(const unsigned char *in, unsigned char *out, int stride, int head, int action, int lane) {
+    const u64 *iw = reinterpret_cast<const u64 *>(in);
+    u64 *ow = reinterpret_cast<u64 *>(out);
+    // ---- the new current position, computed by every lane alike
+    const u64 tail = iw[12];
+    const int stm = (int)(tail & 1), castling = (int)((tail >> 8) & 0xff), halfmove = (int)((tail >> 24) & 0xff);
+    const int reps = (int)((tail >> 32) & 0xff);
+    u64 own[6], opp[6];
+#pragma unroll
+    for (int j = 0; j < 6; ++j) { const u64 wh = iw[j], bl = iw[6 + j]; own[j] = stm ? bl : wh; opp[j] = stm ? wh : bl; }
+    Move mv = decode_action(head, action);
+    int from = mv.from & 63, to = mv.to & 63;
+    if (stm) { from ^= 56; to ^= 56; }
+    const u64 fb = 1ull << from, tb = 1ull << to;
+    int k = -1;
+#pragma unroll
+    for (int j = 0; j < 6; ++j) if (own[j] & fb) k = j;
+    const bool ok = k >= 0;
+    int moved_to = to;                                             // the king's destination when castling
+    bool capture = false;
+    if (ok) {
+        if (k == 5 && (own[3] & tb)) {                             // the king "takes" its own rook: castling
+            const int r0 = stm ? 56 : 0;
+            const bool king_side = to > from;
+            moved_to = r0 + (king_side ? 6 : 2);
+            own[5] = 1ull << moved_to;
+            own[3] = (own[3] & ~tb) | (1ull << (r0 + (king_side ? 5 : 3)));
+        } else {
+#pragma unroll
+            for (int j = 0; j < 6; ++j) { if (opp[j] & tb) capture = true; opp[j] &= ~tb; }
+            if (k == 0 && ((from ^ to) & 7) != 0 && !capture) {    // en passant: the pawn taken stands beside the origin
+                opp[0] &= ~(1ull << ((to & 7) + 8 * (from >> 3)));
+                capture = true;
+            }
+            const bool promotes = k == 0 && (to >> 3) == (stm ? 0 : 7);
+            const int dest = promotes ? (mv.promo ? mv.promo : 4) : k;
+#pragma unroll
+            for (int j = 0; j < 6; ++j) { if (j == k) own[j] &= ~fb; if (j == dest) own[j] |= tb; }
+        }
+    }
+    int rights = castling;
+    if (ok) {
+        const int a = from, b = to;
+        const int lose = (a == 4 || b == 4 ? 3 : 0) | (a == 7 || b == 7 ? 1 : 0) | (a == 0 || b == 0 ? 2 : 0) |
+                         (a == 60 || b == 60 ? 12 : 0) | (a == 63 || b == 63 ? 4 : 0) | (a == 56 || b == 56 ? 8 : 0);
+        rights &= ~lose;
+    }
+    const int dist = to > from ? to - from : from - to;
+    const int ep = ok && k == 0 && dist == 16 ? (from + to) >> 1 : 64;
+    const int hm = (k == 0 || capture) ? 0 : (halfmove < 255 ? halfmove + 1 : 255);
+    u64 new_tail = tail;
+    if (ok) new_tail = (tail & 0xffffff0000000000ull) | (u64)(stm ^ 1) | ((u64)rights << 8) | ((u64)ep << 16) | ((u64)hm << 24);
+    // ---- write: the current position by lanes 0..12, then what the record carries besides it
+    {
+        u64 val = new_tail;
+        const int own_base = stm * 6, opp_base = 6 - own_base;
+#pragma unroll
+        for (int j = 0; j < 6; ++j) { if (lane == own_base + j) val = own[j]; if (lane == opp_base + j) val = opp[j]; }
+        if (lane < 13) ow[lane] = val;
+    }
+    if (stride == 784) {
+        // seven earlier boards: the old current position enters at the front, the oldest leaves
+        for (int i = lane; i < 84; i += 32) ow[13 + i] = !ok ? iw[13 + i] : i < 12 ? iw[i] : iw[13 + i - 12];
+        if (lane == 13) {
+            const u64 old = iw[97];                                // hist_rep[7] | n_hist << 56
+            const u64 n_hist = old >> 56;
+            ow[97] = !ok ? old : (((old << 8) | (u64)reps) & 0x00ffffffffffffffull) | ((n_hist < 7 ? n_hist + 1 : 7) << 56);
+        }
+    } else if (stride == 128) {
+        if (lane == 13) ow[13] = !ok ? iw[13] : (iw[13] << 8) | (u64)from;
+        if (lane == 14) ow[14] = !ok ? iw[14] : (iw[14] << 8) | (u64)moved_to;
+        if (lane == 15) {
+            const u64 old = iw[15];
+            const u64 n = old & 0xff;
+            ow[15] = !ok ? old : (old & ~0xffull) | (n < 8 ? n + 1 : 8);
+        }
+    }
+    return ok;
+}
+
+__global__ void __launch_bounds__(32 * kWarps)
+apply_moves_kernel(const unsigned char *__restrict__ positions, int stride, int batch, int head,
+                   const int *__restrict__ actions, unsigned char *__restrict__ out, uint32_t *status) {
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * kWarps + w;
+    if (i >= batch) return;
+    const bool ok = apply_action_warp(positions + (size_t)i * stride, out + (size_t)i * stride, stride, head, actions[i], lane);
+    if (!ok && lane == 0 && status) atomicOr(status, AZ_SEARCH_FLAG_BAD_ACTION);
+}
+
+// ---- the stand-in evaluator ---------------------------------------------------------------------
+__device__ __forceinline__ u64 mix64(u64 x) {
+    x ^= x >> 30; x *= 0xbf58476d1ce4e5b9ull;
+    x ^= x >> 27; x *= 0x94d049bb133111ebull;
+    x ^= x >> 31;
+    return x;
+}
+__device__ u64 position_key(const u64 *rec, u64 seed) {
+    u64 h = mix64(seed);
+#pragma unroll
+    for (int i = 0; i < 12; ++i) h = mix64(h ^ rec[i]);
+    const u64 tail = rec[12];
+    return mix64(h ^ (tail & 0xffffffull));                        // side to move | castling << 8 | en-passant square << 16
+}
+
+// The set bits of a mask row in ascending order, dealt over the warp: lane L owns words L, L + 32, L + 64.
+// Calls f(action, rank) for every set bit, rank = the number of set bits before it; returns the total.
+template <typename F>
+__device__ __forceinline__ int for_each_legal(const u64 *__restrict__ row, int words, int lane, F f) {
+    int base = 0;
+    for (int r = 0; r * 32 < words; ++r) {
+        const int wi = r * 32 + lane;
+        u64 bits = wi < words ? row[wi] : 0ull;
+        const int c = __popcll(bits);
+        int incl = c;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) { const int t = __shfl_up_sync(0xffffffffu, incl, d); if (lane >= d) incl += t; }
+        int rank = base + incl - c;
+        while (bits) {
+            const int b = __ffsll((long long)bits) - 1;
+            bits &= bits - 1;
+            f(wi * 64 + b, rank++);
+        }
+        base += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    return base;
+}
+
+__global__ void __launch_bounds__(32 * kWarps)
+standin_eval_kernel(const unsigned char *__restrict__ positions, int stride, const u64 *__restrict__ masks, int words,
+                    int batch, u64 seed, float *__restrict__ legal, int *__restrict__ counts, float *__restrict__ value, int vs) {
+    __shared__ int s_w[kWarps][AZ_MAX_LEGAL];
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * kWarps + w;
+    if (i >= batch) return;
+    const u64 key = position_key(reinterpret_cast<const u64 *>(positions + (size_t)i * stride), seed);
+    int sum = 0;
+    int *wt = s_w[w];
+    const int n = for_each_legal(masks + (size_t)i * words, words, lane, [&](int action, int rank) {
+        const int r = (int)(mix64(key + (u64)(action + 1) * 0x9e3779b97f4a7c15ull) >> 54);
+        const int weight = 1 + r * r / 64;
+        if (rank < AZ_MAX_LEGAL) wt[rank] = weight;
+        sum += weight;
+    });
+#pragma unroll
+    for (int d = 16; d; d >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, d);
+    __syncwarp();
+    const int cnt = n < AZ_MAX_LEGAL ? n : AZ_MAX_LEGAL;
+    for (int j = lane; j < cnt; j += 32) legal[(size_t)i * AZ_MAX_LEGAL + j] = __fdiv_rn((float)wt[j], (float)sum);
+    if (lane == 0) {
+        counts[i] = cnt;
+        const int t = (int)(mix64(key ^ 0x5851f42d4c957f2dull) >> 40);
+        const float u = __fsub_rn(__fmul_rn((float)t, 0x1p-23f), 1.0f);
+        value[(size_t)i * vs] = __fmul_rn(u, 0.75f);
+    }
+}
+
+// ---- the trees ------------------------------------------------------------------------------------
+struct Trees {
+    Node *nodes; Edge *edges; unsigned char *node_pos; GameState *games;
+    int node_cap, edge_cap, stride, head, leaves;
+    float c_puct, fpu_reduction, discount;
+};
+struct Batch {                                   // one group's step
+    unsigned char *pos;                          // [rows][stride]
+    int *kind, *leaf, *depth;                    // [rows]
+    int *path_e, *path_n;                        // [rows][kMaxDepth]
+};
+
+// Removes the reservations of the first `depth` levels of a path (all lanes call).
+__device__ __forceinline__ void undo_path(const Trees &t, Edge *edges, Node *nodes, const int *pe, const int *pn, int depth, int lane) {
+    for (int d = lane; d < depth; d += 32) { edges[pe[d]].m -= 1; nodes[pn[d]].nsum -= 1; }
+}
+
+// select: one warp per game, `leaves` traversals one after the other
+__global__ void __launch_bounds__(32 * kWarps)
+search_select_kernel(Trees t, Batch b, int game0, int n_games) {
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gl = blockIdx.x * kWarps + w;
+    if (gl >= n_games) return;
+    const int g = game0 + gl;
+    Node *nodes = t.nodes + (size_t)g * t.node_cap;
+    Edge *edges = t.edges + (size_t)g * t.edge_cap;
+    unsigned char *npos = t.node_pos + (size_t)g * t.node_cap * t.stride;
+    GameState *gs = t.games + g;
+    for (int j = 0; j < t.leaves; ++j) {
+        const int row = gl * t.leaves + j;
+        int *pe = b.path_e + (size_t)row * kMaxDepth, *pn = b.path_n + (size_t)row * kMaxDepth;
+        int kind = kSlotNone, leaf = -1, depth = 0;
+        if (!gs->root_submitted) {
+            // the root's own evaluation, once; the step's other rows idle
+            __syncwarp();
+            if (lane == 0) gs->root_submitted = 1;
+            __syncwarp();
+            kind = kSlotEval; leaf = 0;
+            const u64 *src = reinterpret_cast<const u64 *>(npos);
+            u64 *dst = reinterpret_cast<u64 *>(b.pos + (size_t)row * t.stride);
+            for (int i = lane; i < t.stride / 8; i += 32) dst[i] = src[i];
+        } else {
+            int node = 0;
+            bool given_up = false;
+            for (;;) {
+                const Node nd = nodes[node];
+                if (nd.terminal) { kind = kSlotTerminal; leaf = node; break; }
+                if (nd.n_edges < 0) { given_up = true; break; }
+                if (depth == kMaxDepth) { if (lane == 0) gs->flags |= AZ_SEARCH_FLAG_DEPTH; given_up = true; break; }
+                const float sqrt_n = __fsqrt_rn((float)(nd.nsum > 1 ? nd.nsum : 1));
+                const float fpu = __fsub_rn(__fdiv_rn(nd.wsum, (float)nd.nvis), t.fpu_reduction);
+                float best_score = 0.0f; int best = -1;
+                for (int i = lane; i < nd.n_edges; i += 32) {
+                    const Edge e = edges[nd.edge_begin + i];
+                    const int n = e.n + e.m;
+                    const float q = n > 0 ? __fdiv_rn(__fsub_rn(e.w, (float)e.m), (float)n) : fpu;
+                    float u = __fmul_rn(t.c_puct, e.prior);
+                    u = __fmul_rn(u, sqrt_n);
+                    u = __fdiv_rn(u, (float)(1 + n));
+                    const float score = __fadd_rn(q, u);
+                    if (best < 0 || score > best_score) { best = i; best_score = score; }
+                }
+#pragma unroll
+                for (int d = 16; d; d >>= 1) {
+                    const float os = __shfl_xor_sync(0xffffffffu, best_score, d);
+                    const int ob = __shfl_xor_sync(0xffffffffu, best, d);
+                    // the larger score wins, of equal scores the lower index; a lane without edges never wins
+                    if (ob >= 0 && (best < 0 || os > best_score || (os == best_score && ob < best))) { best = ob; best_score = os; }
+                }
+                const int ei = nd.edge_begin + best;
+                const Edge chosen = edges[ei];
+                __syncwarp();
+                if (lane == 0) {
+                    edges[ei].m = chosen.m + 1;
+                    nodes[node].nsum = nd.nsum + 1;
+                    pe[depth] = ei; pn[depth] = node;
+                }
+                ++depth;
+                __syncwarp();
+                if (chosen.child < 0) {
+                    const int child = gs->n_nodes;
+                    if (child >= t.node_cap) { if (lane == 0) gs->flags |= AZ_SEARCH_FLAG_NODES_FULL; given_up = true; break; }
+                    __syncwarp();
+                    if (lane == 0) {
+                        gs->n_nodes = child + 1;
+                        edges[ei].child = child;
+                        Node c{};
+                        c.n_edges = -1;
+                        nodes[child] = c;
+                    }
+                    unsigned char *cpos = npos + (size_t)child * t.stride;
+                    apply_action_warp(npos + (size_t)node * t.stride, cpos, t.stride, t.head, chosen.action, lane);
+                    __syncwarp();
+                    const u64 *src = reinterpret_cast<const u64 *>(cpos);
+                    u64 *dst = reinterpret_cast<u64 *>(b.pos + (size_t)row * t.stride);
+                    for (int i = lane; i < t.stride / 8; i += 32) dst[i] = src[i];
+                    kind = kSlotEval; leaf = child;
+                    break;
+                }
+                node = chosen.child;
+            }
+            if (given_up) {
+                __syncwarp();
+                undo_path(t, edges, nodes, pe, pn, depth, lane);
+                if (lane == 0) gs->idle += 1;
+                kind = kSlotNone;
+            }
+        }
+        __syncwarp();
+        if (lane == 0) { b.kind[row] = kind; b.leaf[row] = leaf; b.depth[row] = depth; }
+        __syncwarp();
+    }
+}
+
+// expand and back up: one warp per game, the step's rows in order
+__global__ void __launch_bounds__(32 * kWarps)
+search_finish_kernel(Trees t, Batch b, int game0, int n_games, const u64 *__restrict__ masks, int words,
+                     const float *__restrict__ legal, const int *__restrict__ counts, const float *__restrict__ value, int vs) {
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int gl = blockIdx.x * kWarps + w;
+    if (gl >= n_games) return;
+    const int g = game0 + gl;
+    Node *nodes = t.nodes + (size_t)g * t.node_cap;
+    Edge *edges = t.edges + (size_t)g * t.edge_cap;
+    GameState *gs = t.games + g;
+    for (int j = 0; j < t.leaves; ++j) {
+        const int row = gl * t.leaves + j;
+        const int kind = b.kind[row];
+        if (kind == kSlotNone) continue;
+        const int leaf = b.leaf[row], depth = b.depth[row];
+        float v;
+        if (kind == kSlotEval) {
+            const int cnt = counts[row];
+            const float net_v = vs == 3 ? __fsub_rn(value[(size_t)row * 3], value[(size_t)row * 3 + 2]) : value[row];
+            const u64 *rec = reinterpret_cast<const u64 *>(b.pos + (size_t)row * t.stride);
+            const int halfmove = (int)((rec[12] >> 24) & 0xff);
+            Node nd = nodes[leaf];
+            nd.nsum = 0; nd.n_edges = 0;
+            if (cnt == 0) {
+                // no legal move: mated if the mover's king is attacked, else stalemate
+                const int stm = (int)(rec[12] & 1);
+                u64 opp[6], occ = 0;
+#pragma unroll
+                for (int k = 0; k < 6; ++k) { opp[k] = rec[(stm ^ 1) * 6 + k]; occ |= opp[k] | rec[stm * 6 + k]; }
+                const u64 king = rec[stm * 6 + 5];
+                const bool check = king && attacked(__ffsll((long long)king) - 1, stm ^ 1, opp, occ);
+                nd.terminal = 1; nd.tvalue = check ? -1.0f : 0.0f;
+            } else if (halfmove >= 100) {
+                nd.terminal = 1; nd.tvalue = 0.0f;
+            } else if (gs->n_edges + cnt > t.edge_cap) {
+                if (lane == 0) gs->flags |= AZ_SEARCH_FLAG_EDGES_FULL;
+                nd.terminal = 1; nd.tvalue = net_v;
+            } else {
+                const int begin = gs->n_edges;
+                nd.edge_begin = begin; nd.n_edges = cnt;
+                const float *pr = legal + (size_t)row * AZ_MAX_LEGAL;
+                for_each_legal(masks + (size_t)row * words, words, lane, [&](int action, int rank) {
+                    if (rank < cnt) {
+                        Edge e;
+                        e.action = action; e.child = -1; e.n = 0; e.m = 0; e.prior = pr[rank]; e.w = 0.0f;
+                        edges[begin + rank] = e;
+                    }
+                });
+                __syncwarp();
+                if (lane == 0) gs->n_edges = begin + cnt;
+            }
+            v = nd.terminal ? nd.tvalue : net_v;
+            nd.nvis = 1; nd.wsum = v;
+            __syncwarp();
+            if (lane == 0) nodes[leaf] = nd;
+        } else {
+            const Node nd = nodes[leaf];
+            v = nd.tvalue;
+            __syncwarp();
+            if (lane == 0) { nodes[leaf].nvis = nd.nvis + 1; nodes[leaf].wsum = __fadd_rn(nd.wsum, v); }
+        }
+        __syncwarp();
+        // up the path: level d takes the value after depth - d sign changes and discounts; the levels touch
+        // different edges and nodes, so the lanes update them side by side
+        const int *pe = b.path_e + (size_t)row * kMaxDepth, *pn = b.path_n + (size_t)row * kMaxDepth;
+        for (int base = 0; base < depth; base += 32) {
+            const int up = base + lane;                            // 0: the edge into the leaf
+            float x = v;
+            for (int s = 0; s <= up && s < depth; ++s) x = __fmul_rn(-x, t.discount);
+            if (up < depth) {
+                const int d = depth - 1 - up;
+                Edge *e = edges + pe[d];
+                e->n += 1; e->w = __fadd_rn(e->w, x); e->m -= 1;
+                Node *p = nodes + pn[d];
+                p->nvis += 1; p->wsum = __fadd_rn(p->wsum, x);
+            }
+        }
+        __syncwarp();
+    }
+}
+
+std::mutex g_inv_mutex;
+bool g_inv_ready[64] = {};
+
+int ensure_inverse_tables() {
+    int dev = 0;
+    AZ_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(g_inv_mutex);
+    if (dev < 64 && g_inv_ready[dev]) return AZ_OK;
+    static short pair[64 * 64];
+    static short promo[8 * 3];
+    static unsigned short inv_pair[1792];
+    static unsigned char inv_promo[22];
+    if (build_flat_tables(pair, promo) != kFlatMoves) return AZ_ERR_BAD_ARCH;
+    for (int from = 0; from < 64; ++from)
+        for (int to = 0; to < 64; ++to)
+            if (pair[from * 64 + to] >= 0) {
+                if (pair[from * 64 + to] >= 1792) return AZ_ERR_BAD_ARCH;
+                inv_pair[pair[from * 64 + to]] = (unsigned short)(from | to << 6);
+            }
+    for (int file = 0; file < 8; ++file)
+        for (int step = 0; step < 3; ++step)
+            if (promo[file * 3 + step] >= 0) {
+                const int k = (promo[file * 3 + step] - 1792) / 3;
+                if (k < 0 || k >= 22) return AZ_ERR_BAD_ARCH;
+                inv_promo[k] = (unsigned char)(file | (file + step - 1) << 3);
+            }
+    AZ_CUDA(cudaMemcpyToSymbol(g_inv_pair, inv_pair, sizeof inv_pair));
+    AZ_CUDA(cudaMemcpyToSymbol(g_inv_promo, inv_promo, sizeof inv_promo));
+    if (dev < 64) g_inv_ready[dev] = true;
+    return AZ_OK;
+}
+
+struct Group {
+    cudaStream_t owned = nullptr;                // null: the group takes turns with group 0 on that group's stream
+    cudaStream_t stream = nullptr;               // the stream its steps are queued on
+    int game0 = 0, n_games = 0, rows = 0;
+    Batch batch{};
+    uint64_t *masks = nullptr;
+    float *legal = nullptr, *value = nullptr;
+    int *counts = nullptr;
+    cudaEvent_t done = nullptr;
+};
+
+struct Search {
+    az_search_config cfg{};
+    Net *net = nullptr;
+    int device = 0;
+    int words = 0, vs = 1;
+    Trees trees{};
+    Group groups[2];
+    int n_groups = 1;
+    bool second_workspace = false;
+    cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
+    unsigned char *roots_stage = nullptr;        // device copy of the root records
+    int *out_actions = nullptr, *out_visits = nullptr, *out_counts = nullptr;   // read-out of all roots
+};
+
+void free_search(Search *s) {
+    if (!s) return;
+    cudaFree(s->trees.nodes); cudaFree(s->trees.edges); cudaFree(s->trees.node_pos); cudaFree(s->trees.games);
+    cudaFree(s->roots_stage);
+    cudaFree(s->out_actions); cudaFree(s->out_visits); cudaFree(s->out_counts);
+    for (Group &g : s->groups) {
+        cudaFree(g.batch.pos); cudaFree(g.batch.kind); cudaFree(g.batch.leaf); cudaFree(g.batch.depth);
+        cudaFree(g.batch.path_e); cudaFree(g.batch.path_n);
+        cudaFree(g.masks); cudaFree(g.legal); cudaFree(g.value); cudaFree(g.counts);
+        if (g.done) cudaEventDestroy(g.done);
+        if (g.owned) cudaStreamDestroy(g.owned);
+    }
+    if (s->ev_begin) cudaEventDestroy(s->ev_begin);
+    if (s->ev_end) cudaEventDestroy(s->ev_end);
+    delete s;
+}
+
+__global__ void reset_trees_kernel(Trees t, const unsigned char *__restrict__ roots, int games) {
+    const int g = blockIdx.x;
+    if (g >= games) return;
+    if (threadIdx.x == 0) {
+        GameState gs{};
+        gs.n_nodes = 1;
+        t.games[g] = gs;
+        Node root{};
+        root.n_edges = -1;
+        t.nodes[(size_t)g * t.node_cap] = root;
+    }
+    const u64 *src = reinterpret_cast<const u64 *>(roots + (size_t)g * t.stride);
+    u64 *dst = reinterpret_cast<u64 *>(t.node_pos + (size_t)g * t.node_cap * t.stride);
+    for (int i = threadIdx.x; i < t.stride / 8; i += blockDim.x) dst[i] = src[i];
+}
+
+// root actions and visit counts of every game, in rows of AZ_MAX_LEGAL
+__global__ void gather_roots_kernel(Trees t, int games, int *__restrict__ actions, int *__restrict__ visits, int *__restrict__ counts) {
+    const int g = blockIdx.x;
+    if (g >= games) return;
+    const Node root = t.nodes[(size_t)g * t.node_cap];
+    const int k = root.n_edges > 0 ? (root.n_edges < AZ_MAX_LEGAL ? root.n_edges : AZ_MAX_LEGAL) : 0;
+    const Edge *e = t.edges + (size_t)g * t.edge_cap + root.edge_begin;
+    for (int i = threadIdx.x; i < k; i += blockDim.x) {
+        actions[(size_t)g * AZ_MAX_LEGAL + i] = e[i].action;
+        visits[(size_t)g * AZ_MAX_LEGAL + i] = e[i].n;
+    }
+    if (threadIdx.x == 0) counts[g] = k;
+}
+
+// one step of one group: four launches (five with the paper's network or a tensor-core net: their
+// evaluation is two or three kernels)
+int queue_step(Search &s, int gi) {
+    Group &g = s.groups[gi];
+    const unsigned blocks = (unsigned)((g.n_games + kWarps - 1) / kWarps);
+    search_select_kernel<<<blocks, 32 * kWarps, 0, g.stream>>>(s.trees, g.batch, g.game0, g.n_games);
+    AZ_LAUNCH_CHECK();
+    int rc = launch_legal_masks(g.batch.pos, (size_t)s.trees.stride, g.rows, s.trees.head, g.masks, g.stream);
+    if (rc != AZ_OK) return rc;
+    if (s.cfg.evaluator == AZ_SEARCH_EVAL_STANDIN) {
+        standin_eval_kernel<<<(unsigned)((g.rows + kWarps - 1) / kWarps), 32 * kWarps, 0, g.stream>>>(
+            g.batch.pos, s.trees.stride, (const u64 *)g.masks, s.words, g.rows, s.cfg.seed, g.legal, g.counts, g.value, s.vs);
+        AZ_LAUNCH_CHECK();
+    } else {
+        const bool alt = s.second_workspace && gi == 1;
+        if (alt) swap_workspace(*s.net);
+        rc = az_evaluate_legal(reinterpret_cast<az_net *>(s.net), g.batch.pos, g.masks, g.rows, g.legal, g.counts, g.value, g.stream);
+        if (alt) swap_workspace(*s.net);
+        if (rc != AZ_OK) return rc;
+    }
+    search_finish_kernel<<<blocks, 32 * kWarps, 0, g.stream>>>(s.trees, g.batch, g.game0, g.n_games, (const u64 *)g.masks, s.words,
+                                                               g.legal, g.counts, g.value, s.vs);
+    AZ_LAUNCH_CHECK();
+    return AZ_OK;
+}
+
+}  // namespace
+}  // namespace az
+
+using az::Search;
+
+extern "C" {
+
+int az_apply_moves(const void *positions_dev, size_t position_stride, int batch, int policy_head,
+                   const int32_t *actions_dev, void *out_positions_dev, uint32_t *status_dev, void *cuda_stream) {
+    if (batch < 0 || policy_head < 0 || policy_head > AZ_POLICY_FROMTO1880) return AZ_ERR_BAD_ARG;
+    if (position_stride != 104 && position_stride != 784 && position_stride != 128) return AZ_ERR_BAD_ARG;
+    if (batch == 0) return AZ_OK;
+    if (!positions_dev || !actions_dev || !out_positions_dev || positions_dev == out_positions_dev) return AZ_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(positions_dev) & 7) || (reinterpret_cast<uintptr_t>(out_positions_dev) & 7) ||
+        (reinterpret_cast<uintptr_t>(actions_dev) & 3) || (reinterpret_cast<uintptr_t>(status_dev) & 3))
+        return AZ_ERR_BAD_ARG;
+    int rc = az::ensure_inverse_tables();
+    if (rc != AZ_OK) return rc;
+    az::apply_moves_kernel<<<(unsigned)((batch + az::kWarps - 1) / az::kWarps), 32 * az::kWarps, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        static_cast<const unsigned char *>(positions_dev), (int)position_stride, batch, policy_head, actions_dev,
+        static_cast<unsigned char *>(out_positions_dev), status_dev);
+    AZ_LAUNCH_CHECK();
+    return AZ_OK;
+}
+
+int az_standin_evaluate(const void *positions_dev, size_t position_stride, const uint64_t *legal_masks_dev, int batch,
+                        int policy_head, uint64_t seed, float *legal_policy_dev, int32_t *legal_counts_dev,
+                        float *value_dev, void *cuda_stream) {
+    if (batch < 0 || policy_head < 0 || policy_head > AZ_POLICY_FROMTO1880 || position_stride < 104 || (position_stride & 7)) return AZ_ERR_BAD_ARG;
+    if (batch == 0) return AZ_OK;
+    if (!positions_dev || !legal_masks_dev || !legal_policy_dev || !legal_counts_dev || !value_dev) return AZ_ERR_BAD_ARG;
+    if ((reinterpret_cast<uintptr_t>(positions_dev) & 7) || (reinterpret_cast<uintptr_t>(legal_masks_dev) & 7)) return AZ_ERR_BAD_ARG;
+    const int words = policy_head == AZ_POLICY_PLANES73 ? 73 : 30;
+    az::standin_eval_kernel<<<(unsigned)((batch + az::kWarps - 1) / az::kWarps), 32 * az::kWarps, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        static_cast<const unsigned char *>(positions_dev), (int)position_stride, (const az::u64 *)legal_masks_dev, words, batch,
+        seed, legal_policy_dev, legal_counts_dev, value_dev, 1);
+    AZ_LAUNCH_CHECK();
+    return AZ_OK;
+}
+
+int az_search_create(az_net *net, const az_search_config *c, az_search **out) {
+    if (!c || !out) return AZ_ERR_BAD_ARG;
+    *out = nullptr;
+    if (c->games < 1 || c->leaves < 1 || c->leaves > AZ_SEARCH_MAX_LEAVES || c->groups < 1 || c->groups > 2 ||
+        c->max_nodes < 2 || c->max_edges < 1 || c->evaluator > AZ_SEARCH_EVAL_STANDIN || c->policy_head > AZ_POLICY_FROMTO1880)
+        return AZ_ERR_BAD_ARG;
+    if (c->position_bytes != 104 && c->position_bytes != 784 && c->position_bytes != 128) return AZ_ERR_BAD_ARG;
+    if (!(c->c_puct >= 0.0f) || !(c->discount > 0.0f && c->discount <= 1.0f) || !(c->fpu_reduction >= 0.0f)) return AZ_ERR_BAD_ARG;
+    az::Net *n = reinterpret_cast<az::Net *>(net);
+    if (c->evaluator == AZ_SEARCH_EVAL_NET) {
+        if (!n) return AZ_ERR_BAD_ARG;
+        if (n->arch.policy_head != c->policy_head || az_position_bytes(&n->arch) != c->position_bytes) return AZ_ERR_BAD_ARCH;
+        if (n->fp8 && !n->fp8_ready) return AZ_ERR_NOT_CALIBRATED;
+    }
+    const int n_groups = c->games >= 2 ? (int)c->groups : 1;
+    const int per_group = (int)((c->games + n_groups - 1) / n_groups);
+    if (c->evaluator == AZ_SEARCH_EVAL_NET && (uint64_t)per_group * c->leaves > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
+    if (n) AZ_CUDA(cudaSetDevice(n->device));
+    int rc = az::ensure_inverse_tables();
+    if (rc != AZ_OK) return rc;
+    Search *s = new (std::nothrow) Search();
+    if (!s) return AZ_ERR_BAD_ARG;
+    s->cfg = *c;
+    s->net = c->evaluator == AZ_SEARCH_EVAL_NET ? n : nullptr;
+    s->n_groups = n_groups;
+    s->words = c->policy_head == AZ_POLICY_PLANES73 ? 73 : 30;
+    s->vs = s->net ? (int)az_value_size(&s->net->arch) : 1;
+    az::Trees &t = s->trees;
+    t.node_cap = (int)c->max_nodes; t.edge_cap = (int)c->max_edges; t.stride = (int)c->position_bytes;
+    t.head = (int)c->policy_head; t.leaves = (int)c->leaves;
+    t.c_puct = c->c_puct; t.fpu_reduction = c->fpu_reduction; t.discount = c->discount;
+    const size_t G = c->games;
+#define AZ_SEARCH_ALLOC(ptr, bytes)                                                          \
+    do {                                                                                     \
+        cudaError_t e__ = cudaMalloc((void **)&(ptr), (bytes));                              \
+        if (e__ != cudaSuccess) { az::set_cuda_error(e__, "cudaMalloc (search)"); az::free_search(s); return AZ_ERR_CUDA; } \
+    } while (0)
+    AZ_SEARCH_ALLOC(t.nodes, G * t.node_cap * sizeof(az::Node));
+    AZ_SEARCH_ALLOC(t.edges, G * t.edge_cap * sizeof(az::Edge));
+    AZ_SEARCH_ALLOC(t.node_pos, G * t.node_cap * (size_t)t.stride);
+    AZ_SEARCH_ALLOC(t.games, G * sizeof(az::GameState));
+    AZ_SEARCH_ALLOC(s->roots_stage, G * (size_t)t.stride);
+    AZ_SEARCH_ALLOC(s->out_actions, G * AZ_MAX_LEGAL * sizeof(int));
+    AZ_SEARCH_ALLOC(s->out_visits, G * AZ_MAX_LEGAL * sizeof(int));
+    AZ_SEARCH_ALLOC(s->out_counts, G * sizeof(int));
+    cudaMemset(s->out_actions, 0, G * AZ_MAX_LEGAL * sizeof(int));
+    cudaMemset(s->out_visits, 0, G * AZ_MAX_LEGAL * sizeof(int));
+    if (s->net && n_groups == 2) {
+        rc = az::ensure_second_workspace(*s->net, &s->second_workspace);
+        if (rc != AZ_OK) { az::free_search(s); return rc; }
+    }
+    for (int gi = 0; gi < n_groups; ++gi) {
+        az::Group &g = s->groups[gi];
+        g.game0 = gi * per_group;
+        g.n_games = (int)G - g.game0 < per_group ? (int)G - g.game0 : per_group;
+        g.rows = g.n_games * (int)c->leaves;
+        // without a second evaluation workspace both groups take turns on one stream
+        if (gi == 1 && s->net && !s->second_workspace) g.stream = s->groups[0].stream;
+        else {
+            if (cudaStreamCreateWithFlags(&g.owned, cudaStreamNonBlocking) != cudaSuccess) { az::free_search(s); return AZ_ERR_CUDA; }
+            g.stream = g.owned;
+        }
+        if (cudaEventCreateWithFlags(&g.done, cudaEventDisableTiming) != cudaSuccess) { az::free_search(s); return AZ_ERR_CUDA; }
+        const size_t R = (size_t)g.rows;
+        AZ_SEARCH_ALLOC(g.batch.pos, R * t.stride);
+        AZ_SEARCH_ALLOC(g.batch.kind, R * sizeof(int));
+        AZ_SEARCH_ALLOC(g.batch.leaf, R * sizeof(int));
+        AZ_SEARCH_ALLOC(g.batch.depth, R * sizeof(int));
+        AZ_SEARCH_ALLOC(g.batch.path_e, R * az::kMaxDepth * sizeof(int));
+        AZ_SEARCH_ALLOC(g.batch.path_n, R * az::kMaxDepth * sizeof(int));
+        AZ_SEARCH_ALLOC(g.masks, R * s->words * sizeof(uint64_t));
+        AZ_SEARCH_ALLOC(g.legal, R * AZ_MAX_LEGAL * sizeof(float));
+        AZ_SEARCH_ALLOC(g.value, R * s->vs * sizeof(float));
+        AZ_SEARCH_ALLOC(g.counts, R * sizeof(int));
+    }
+#undef AZ_SEARCH_ALLOC
+    if (cudaEventCreate(&s->ev_begin) != cudaSuccess || cudaEventCreate(&s->ev_end) != cudaSuccess) { az::free_search(s); return AZ_ERR_CUDA; }
+    *out = reinterpret_cast<az_search *>(s);
+    return AZ_OK;
+}
+
+void az_search_destroy(az_search *search) { az::free_search(reinterpret_cast<Search *>(search)); }
+
+int az_search_set_roots(az_search *search, const void *positions_host) {
+    Search *s = reinterpret_cast<Search *>(search);
+    if (!s || !positions_host) return AZ_ERR_BAD_ARG;
+    const az::Trees &t = s->trees;
+    cudaStream_t st = s->groups[0].stream;
+    AZ_CUDA(cudaMemcpyAsync(s->roots_stage, positions_host, (size_t)s->cfg.games * t.stride, cudaMemcpyHostToDevice, st));
+    az::reset_trees_kernel<<<s->cfg.games, 32, 0, st>>>(t, s->roots_stage, (int)s->cfg.games);
+    AZ_LAUNCH_CHECK();
+    // the rows of every group's batch must hold valid records from the first step on (rows that idle are still evaluated)
+    for (int gi = 0; gi < s->n_groups; ++gi) {
+        az::Group &g = s->groups[gi];
+        for (uint32_t j = 0; j < s->cfg.leaves; ++j)
+            AZ_CUDA(cudaMemcpy2DAsync(g.batch.pos + (size_t)j * t.stride, (size_t)t.stride * s->cfg.leaves,
+                                      s->roots_stage + (size_t)g.game0 * t.stride, (size_t)t.stride, (size_t)t.stride,
+                                      (size_t)g.n_games, cudaMemcpyDeviceToDevice, st));
+    }
+    AZ_CUDA(cudaStreamSynchronize(st));
+    return AZ_OK;
+}
+
+int az_search_run(az_search *search, int simulations, float *elapsed_ms_out) {
+    Search *s = reinterpret_cast<Search *>(search);
+    if (!s || simulations < 0) return AZ_ERR_BAD_ARG;
+    cudaStream_t s0 = s->groups[0].stream;
+    cudaStream_t s1 = s->n_groups == 2 ? s->groups[1].stream : s0;
+    AZ_CUDA(cudaEventRecord(s->ev_begin, s0));
+    if (s1 != s0) AZ_CUDA(cudaStreamWaitEvent(s1, s->ev_begin, 0));
+    // a tree whose root has not been evaluated spends its first step on that; give every tree that step
+    az::GameState first{};
+    AZ_CUDA(cudaMemcpy(&first, s->trees.games, sizeof first, cudaMemcpyDeviceToHost));
+    const int steps = simulations + (first.root_submitted ? 0 : 1);
+    for (int step = 0; step < steps; ++step)
+        for (int gi = 0; gi < s->n_groups; ++gi) {
+            const int rc = az::queue_step(*s, gi);
+            if (rc != AZ_OK) return rc;
+        }
+    if (s1 != s0) {
+        AZ_CUDA(cudaEventRecord(s->groups[1].done, s1));
+        AZ_CUDA(cudaStreamWaitEvent(s0, s->groups[1].done, 0));
+    }
+    AZ_CUDA(cudaEventRecord(s->ev_end, s0));
+    AZ_CUDA(cudaEventSynchronize(s->ev_end));
+    if (elapsed_ms_out) AZ_CUDA(cudaEventElapsedTime(elapsed_ms_out, s->ev_begin, s->ev_end));
+    if (s->net) {
+        uint32_t status = 0;
+        AZ_CUDA(cudaMemcpy(&status, s->net->status_dev, sizeof status, cudaMemcpyDeviceToHost));
+        if (status & az::kStatusWaitTimeout) return AZ_ERR_DEVICE_TIMEOUT;
+    }
+    return AZ_OK;
+}
+
+int az_search_root(az_search *search, int game, int32_t *actions_host, int32_t *visits_host, float *w_host,
+                   float *prior_host, int32_t *count_out) {
+    Search *s = reinterpret_cast<Search *>(search);
+    if (!s || game < 0 || (uint32_t)game >= s->cfg.games || !actions_host || !visits_host || !w_host || !prior_host || !count_out)
+        return AZ_ERR_BAD_ARG;
+    az::Node root;
+    AZ_CUDA(cudaMemcpy(&root, s->trees.nodes + (size_t)game * s->trees.node_cap, sizeof root, cudaMemcpyDeviceToHost));
+    const int k = root.n_edges > 0 ? (root.n_edges < AZ_MAX_LEGAL ? root.n_edges : AZ_MAX_LEGAL) : 0;
+    *count_out = k;
+    if (k == 0) return AZ_OK;
+    az::Edge e[AZ_MAX_LEGAL];
+    AZ_CUDA(cudaMemcpy(e, s->trees.edges + (size_t)game * s->trees.edge_cap + root.edge_begin, (size_t)k * sizeof(az::Edge), cudaMemcpyDeviceToHost));
+    for (int i = 0; i < k; ++i) { actions_host[i] = e[i].action; visits_host[i] = e[i].n; w_host[i] = e[i].w; prior_host[i] = e[i].prior; }
+    return AZ_OK;
+}
+
+int az_search_root_visits(az_search *search, int32_t *actions_host, int32_t *visits_host, int32_t *counts_host) {
+    Search *s = reinterpret_cast<Search *>(search);
+    if (!s || !actions_host || !visits_host || !counts_host) return AZ_ERR_BAD_ARG;
+    cudaStream_t st = s->groups[0].stream;
+    const size_t G = s->cfg.games;
+    az::gather_roots_kernel<<<(unsigned)G, 64, 0, st>>>(s->trees, (int)G, s->out_actions, s->out_visits, s->out_counts);
+    AZ_LAUNCH_CHECK();
+    AZ_CUDA(cudaMemcpyAsync(counts_host, s->out_counts, G * sizeof(int), cudaMemcpyDeviceToHost, st));
+    AZ_CUDA(cudaMemcpyAsync(actions_host, s->out_actions, G * AZ_MAX_LEGAL * sizeof(int), cudaMemcpyDeviceToHost, st));
+    AZ_CUDA(cudaMemcpyAsync(visits_host, s->out_visits, G * AZ_MAX_LEGAL * sizeof(int), cudaMemcpyDeviceToHost, st));
+    AZ_CUDA(cudaStreamSynchronize(st));
+    return AZ_OK;
+}
+
+int az_search_tree(az_search *search, int game, int32_t *counts_out, int32_t *node_visits_host, float *node_value_sum_host) {
+    Search *s = reinterpret_cast<Search *>(search);
+    if (!s || game < 0 || (uint32_t)game >= s->cfg.games || !counts_out) return AZ_ERR_BAD_ARG;
+    az::GameState gs;
+    AZ_CUDA(cudaMemcpy(&gs, s->trees.games + game, sizeof gs, cudaMemcpyDeviceToHost));
+    counts_out[0] = gs.n_nodes; counts_out[1] = gs.n_edges; counts_out[2] = gs.flags; counts_out[3] = gs.idle;
+    if (node_visits_host || node_value_sum_host) {
+        az::Node *host = new (std::nothrow) az::Node[(size_t)gs.n_nodes];
+        if (!host) return AZ_ERR_BAD_ARG;
+        cudaError_t e = cudaMemcpy(host, s->trees.nodes + (size_t)game * s->trees.node_cap, (size_t)gs.n_nodes * sizeof(az::Node), cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) { delete[] host; az::set_cuda_error(e, "cudaMemcpy (tree)"); return AZ_ERR_CUDA; }
+        for (int i = 0; i < gs.n_nodes; ++i) {
+            if (node_visits_host) node_visits_host[i] = host[i].nvis;
+            if (node_value_sum_host) node_value_sum_host[i] = host[i].wsum;
+        }
+        delete[] host;
+    }
+    return AZ_OK;
+}
+
+int az_search_launches_per_step(const az_search *search) {
+    const Search *s = reinterpret_cast<const Search *>(search);
+    if (!s) return 0;
+    const int eval = s->net ? az_launches_per_evaluate(reinterpret_cast<const az_net *>(s->net), s->groups[0].rows) : 1;
+    return 3 + eval;
+}
+
+}  // extern "C"

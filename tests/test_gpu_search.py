@@ -1,0 +1,259 @@
+"""The GPU search driver (Eq. 1, Sec. 3.4, 4.1, 5.1; App. D.2) against the oracle's sequential search:
+successor positions bit-exact, the stand-in evaluator bit-exact, and with that evaluator whole trees equal
+node by node (visit counts as integers, value sums as float32 bit patterns).  With a network as evaluator the
+trees cannot be compared across precisions; the bookkeeping invariants and the root priors are checked."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from inputs import pnet_weights as pw
+from inputs import positions
+
+pytestmark = pytest.mark.gpu
+
+START = "rnbqkbnr/pppppppp/8/8/8/8/PPPPPPPP/RNBQKBNR w KQkq - 0 1"
+SPECIAL = [START,
+           "r3k2r/p1ppqpb1/bn2pnp1/3PN3/1p2P3/2N2Q1p/PPPBBPPP/R3K2R w KQkq - 0 1",
+           "6k1/5ppp/8/8/8/8/8/R3K3 w Q - 0 1",
+           "7k/8/5K2/8/8/8/8/6R1 w - - 0 1",
+           "7k/5Q2/6K1/8/8/8/8/8 b - - 0 1",
+           "4k3/8/8/8/8/8/4P3/4K3 w - - 99 80",
+           "1r2k3/P7/8/8/8/8/8/4K3 w - - 5 1",
+           "4k3/8/8/3pP3/8/8/8/4K3 w - d6 0 1"]
+SIZE = {0: 4672, 1: 1858, 2: 1880}
+
+
+def records(head, stride, n, seed):
+    """n generated records of the given layout, the special positions in front."""
+    if stride == 128:
+        rec, _ = positions.generate_moves(seed, n, (0, 160))
+    else:
+        rec, _ = positions.generate(seed, n, (0, 160))
+        if stride == 104:
+            rec = positions.cur_records(rec)
+    rec = rec.copy()
+    for i, fen in enumerate(SPECIAL):
+        cur = positions.record_from_fen(fen)[0]
+        if stride == 104:
+            rec[i] = cur
+        else:
+            rec[i] = np.zeros((), dtype=rec.dtype)
+            rec[i]["cur"] = cur
+    return rec
+
+
+def cur_of(rec):
+    return np.ascontiguousarray(rec["cur"]) if rec.dtype.names and "cur" in rec.dtype.names else rec
+
+
+@pytest.mark.parametrize("head,stride", [(0, 784), (1, 104), (2, 128), (0, 104), (1, 784)])
+def test_successor_positions_are_bit_exact(head, stride):
+    import paper_2609_37447_b200 as az
+    rec = records(head, stride, 400, 20260980 + head)
+    masks = oracle.legal_masks(cur_of(rec), head)
+    bits = np.unpackbits(masks.view(np.uint8), axis=1, bitorder="little")[:, :SIZE[head]].astype(bool)
+    parent, action = np.nonzero(bits)
+    assert len(parent) > 8000
+    src = np.ascontiguousarray(rec[parent])
+    want = oracle.apply_moves(src, head, action.astype(np.int32))
+    pos = az.records_to_device(src)
+    out = torch.zeros_like(pos)
+    act = torch.from_numpy(action.astype(np.int32)).cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    az.az_apply_moves(pos, stride, len(parent), head, act, out, status)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy().view(np.uint8).reshape(len(parent), stride)
+    ref = want.view(np.uint8).reshape(len(parent), stride)
+    bad = np.flatnonzero((got != ref).any(axis=1))
+    assert len(bad) == 0, (len(bad), parent[bad[:5]], action[bad[:5]])
+    assert int(status.item()) == 0
+    # an action whose origin is empty leaves a copy and raises the flag
+    empty = torch.full((1,), int(oracle.policy_index(head, 0, 27, 35)), dtype=torch.int32, device="cuda")
+    az.az_apply_moves(pos[:1], stride, 1, head, empty, out[:1], status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == az.AZ_SEARCH_FLAG_BAD_ACTION and (out[:1].cpu() == pos[:1].cpu()).all()
+
+
+@pytest.mark.parametrize("head,stride", [(1, 104), (2, 128)])
+def test_stand_in_evaluator_is_bit_exact(head, stride):
+    import paper_2609_37447_b200 as az
+    rec = records(head, stride, 300, 20260985)
+    n = rec.shape[0]
+    pos = az.records_to_device(rec)
+    masks = torch.zeros((n, 30), dtype=torch.int64, device="cuda")
+    az.az_legal_masks(pos, stride, n, head, masks)
+    legal = torch.full((n, az.AZ_MAX_LEGAL), -1.0, device="cuda")
+    counts = torch.zeros(n, dtype=torch.int32, device="cuda")
+    value = torch.zeros(n, device="cuda")
+    az.az_standin_evaluate(pos, stride, masks, n, head, 77, legal, counts, value)
+    torch.cuda.synchronize()
+    legal, counts, value = legal.cpu().numpy(), counts.cpu().numpy(), value.cpu().numpy()
+    cur = cur_of(rec)
+    for i in range(n):
+        a, p, v = oracle.synth_eval(cur[i], head, 77)
+        assert counts[i] == len(a)
+        assert (legal[i, :len(a)].view(np.uint32) == p.view(np.uint32)).all() and (legal[i, len(a):] == -1.0).all()
+        assert np.float32(v).view(np.uint32) == value[i].view(np.uint32)
+
+
+def run_gpu_search(az, rec, head, stride, sims, leaves, groups, max_nodes, max_edges, seed, c_puct=1.5, runs=1):
+    cfg = az.make_search_config(rec.shape[0], head, stride, leaves=leaves, groups=groups, max_nodes=max_nodes,
+                                max_edges=max_edges, evaluator=az.AZ_SEARCH_EVAL_STANDIN, c_puct=c_puct, seed=seed)
+    s = az.az_search_create(None, cfg)
+    az.az_search_set_roots(s, rec)
+    for _ in range(runs):
+        az.az_search_run(s, sims // runs)
+    out = []
+    for g in range(rec.shape[0]):
+        a, n, w, p = az.az_search_root(s, g)
+        counts, nvis, wsum = az.az_search_tree(s, g)
+        out.append((a, n, w, p, counts, nvis, wsum))
+    az.az_search_destroy(s)
+    return out
+
+
+def compare_with_oracle(got, rec, head, sims, leaves, max_nodes, max_edges, seed, c_puct=1.5):
+    for g, (a, n, w, p, counts, nvis, wsum) in enumerate(got):
+        want = oracle.mcts_search(rec[g:g + 1], head, sims, leaves=leaves, c_puct=c_puct, seed=seed,
+                                  node_cap=max_nodes, edge_cap=max_edges)
+        where = f"game {g}"
+        assert (a == want["actions"]).all(), where
+        assert (p.view(np.uint32) == want["prior"].view(np.uint32)).all(), where
+        assert (n == want["visits"]).all(), (where, n, want["visits"])
+        assert (w.view(np.uint32) == want["w"].view(np.uint32)).all(), where
+        assert tuple(counts) == (want["n_nodes"], want["n_edges"], want["flags"], want["idle"]), where
+        assert (nvis == want["node_nvis"]).all(), where
+        assert (wsum.view(np.uint32) == want["node_wsum"].view(np.uint32)).all(), where
+
+
+@pytest.mark.parametrize("head,stride,leaves,groups", [(2, 128, 1, 1), (2, 128, 4, 2), (1, 104, 1, 2), (1, 104, 8, 1), (0, 784, 2, 2)])
+def test_trees_equal_the_oracles_node_by_node(head, stride, leaves, groups):
+    import paper_2609_37447_b200 as az
+    rec = records(head, stride, 29, 20260990 + leaves)               # 29 games: an odd split over two groups, a ragged last block
+    sims, nodes = 240, 240 * leaves + 2
+    got = run_gpu_search(az, rec, head, stride, sims, leaves, groups, nodes, 48 * nodes, seed=5)
+    compare_with_oracle(got, rec, head, sims, leaves, nodes, 48 * nodes, seed=5)
+
+
+def test_runs_add_up_and_other_constants():
+    import paper_2609_37447_b200 as az
+    rec = records(2, 128, 12, 20260995)
+    # three runs of 100 steps are one search of 300; the evaluation constants of App. B.1 (c = 1.0)
+    got = run_gpu_search(az, rec, 2, 128, 300, 2, 2, 700, 700 * 48, seed=9, c_puct=1.0, runs=3)
+    compare_with_oracle(got, rec, 2, 300, 2, 700, 700 * 48, seed=9, c_puct=1.0)
+
+
+def test_full_pools_are_reported_like_the_oracles():
+    import paper_2609_37447_b200 as az
+    rec = records(2, 128, 10, 20260996)
+    got = run_gpu_search(az, rec, 2, 128, 150, 2, 1, 60, 60 * 48, seed=3)
+    compare_with_oracle(got, rec, 2, 150, 2, 60, 60 * 48, seed=3)
+    assert any(c[4][2] & az.AZ_SEARCH_FLAG_NODES_FULL for c in got)
+    got = run_gpu_search(az, rec, 2, 128, 150, 1, 1, 200, 400, seed=3)
+    compare_with_oracle(got, rec, 2, 150, 1, 200, 400, seed=3)
+    assert any(c[4][2] & az.AZ_SEARCH_FLAG_EDGES_FULL for c in got)
+
+
+def test_many_games_at_the_papers_batch_shape():
+    """512 games in two groups of 256 (Sec. 5.1), 64 steps; sampled games against the oracle."""
+    import paper_2609_37447_b200 as az
+    rec = records(2, 128, 512, 20260997)
+    got = run_gpu_search(az, rec, 2, 128, 64, 1, 2, 80, 80 * 64, seed=11)
+    pick = [0, 1, 2, 3, 4, 5, 6, 7, 100, 255, 256, 257, 400, 511]
+    compare_with_oracle([got[g] for g in pick], rec[pick], 2, 64, 1, 80, 80 * 64, seed=11)
+    for a, n, w, p, counts, nvis, wsum in got:
+        assert n.sum() + counts[3] == 64 or len(a) == 0
+
+
+def test_root_visits_of_all_games_in_one_copy():
+    import paper_2609_37447_b200 as az
+    rec = records(2, 128, 33, 20260994)
+    s = az.az_search_create(None, az.make_search_config(33, 2, 128, leaves=2, max_nodes=300, evaluator=az.AZ_SEARCH_EVAL_STANDIN, seed=2))
+    az.az_search_set_roots(s, rec)
+    az.az_search_run(s, 120)
+    actions = np.full((33, az.AZ_MAX_LEGAL), -1, dtype=np.int32)
+    visits = np.full((33, az.AZ_MAX_LEGAL), -1, dtype=np.int32)
+    counts = np.zeros(33, dtype=np.int32)
+    az.az_search_root_visits(s, actions, visits, counts)
+    for g in range(33):
+        a, n, w, p = az.az_search_root(s, g)
+        assert counts[g] == len(a) and (actions[g, :len(a)] == a).all() and (visits[g, :len(a)] == n).all()
+    az.az_search_destroy(s)
+
+
+def test_search_with_the_network_as_evaluator():
+    import paper_2609_37447_b200 as az
+    cfg = pw.PNetConfig("ts", 2, 128, 64, 20260998, 4500)
+    blob = pw.make_blob(cfg, 0.1, 0.6)
+    arch = az.make_arch(52, cfg.blocks, cfg.channels, 2, 1, cfg.precision, 128)
+    net = az.az_load_net(arch, blob)
+    rec = records(2, 128, 40, 20260999)
+    n = rec.shape[0]
+    sc = az.make_search_config(n, 2, 128, leaves=2, groups=2, max_nodes=256, evaluator=az.AZ_SEARCH_EVAL_NET)
+    s = az.az_search_create(net, sc)
+    az.az_search_set_roots(s, rec)
+    ms = az.az_search_run(s, 100)
+    assert ms > 0 and az.az_search_launches_per_step(s) == 3 + az.az_launches_per_evaluate(net, 40)
+    # the root priors are the evaluator's own output for the root positions
+    pos = az.records_to_device(rec)
+    masks = torch.zeros((n, 30), dtype=torch.int64, device="cuda")
+    az.az_legal_masks(pos, 128, n, 2, masks)
+    legal = torch.zeros((n, az.AZ_MAX_LEGAL), device="cuda")
+    counts = torch.zeros(n, dtype=torch.int32, device="cuda")
+    value = torch.zeros((n, 3), device="cuda")
+    az.az_evaluate_legal(net, pos, masks, n, legal, counts, value)
+    torch.cuda.synchronize()
+    legal, counts, value = legal.cpu().numpy(), counts.cpu().numpy(), value.cpu().numpy()
+    want_masks = oracle.legal_masks(cur_of(rec), 2)
+    for g in range(n):
+        a, nv, w, p = az.az_search_root(s, g)
+        c, nvis, wsum = az.az_search_tree(s, g)
+        bits = np.flatnonzero(np.unpackbits(want_masks[g].view(np.uint8), bitorder="little")[:1880])
+        if len(bits) == 0 or rec[g]["cur"]["halfmove"] >= 100:
+            assert len(a) == 0 and c[0] == 1
+            continue
+        assert (a == bits).all() and c[2] == 0
+        assert (p.view(np.uint32) == legal[g, :counts[g]].view(np.uint32)).all()
+        assert nv.sum() + c[3] == 200 + 1 and c[0] <= 1 + nv.sum()       # the root's step idles its second row
+        assert nvis[0] == 1 + nv.sum() and (np.abs(w) <= nv + 1e-4).all()
+        # the root's value sum starts with its own evaluation: win minus loss
+        assert abs(float(wsum[0]) - float(w.sum()) - float(value[g, 0] - value[g, 2])) < 1e-3
+    az.az_search_destroy(s)
+    # a second search object on the same net, one group, gives the same trees as two groups (the order of the
+    # steps of different games does not matter)
+    s1 = az.az_search_create(net, az.make_search_config(n, 2, 128, leaves=2, groups=1, max_nodes=256))
+    s2 = az.az_search_create(net, az.make_search_config(n, 2, 128, leaves=2, groups=2, max_nodes=256))
+    for s in (s1, s2):
+        az.az_search_set_roots(s, rec)
+        az.az_search_run(s, 60)
+    for g in range(n):
+        r1, r2 = az.az_search_root(s1, g), az.az_search_root(s2, g)
+        assert all((x.view(np.uint32) == y.view(np.uint32)).all() for x, y in zip(r1, r2))
+    az.az_search_destroy(s1)
+    az.az_search_destroy(s2)
+    assert az.az_device_status(net) & ~1 == 0                            # only "a position had no legal move" may be set
+    az.az_free_net(net)
+
+
+def test_bad_arguments():
+    import paper_2609_37447_b200 as az
+    for kw in ({"leaves": 17}, {"groups": 3}, {"max_nodes": 1}):
+        with pytest.raises(az.AzError) as e:
+            az.az_search_create(None, az.make_search_config(4, 2, 128, evaluator=az.AZ_SEARCH_EVAL_STANDIN, **kw))
+        assert e.value.code == az.AZ_ERR_BAD_ARG
+    with pytest.raises(az.AzError) as e:
+        az.az_search_create(None, az.make_search_config(4, 2, 128))       # a network evaluator needs a network
+    assert e.value.code == az.AZ_ERR_BAD_ARG
+    with pytest.raises(az.AzError) as e:
+        az.az_search_create(None, az.make_search_config(4, 2, 100, evaluator=az.AZ_SEARCH_EVAL_STANDIN))
+    assert e.value.code == az.AZ_ERR_BAD_ARG
+    cfg = pw.PNetConfig("tb", 0, 128, 8, 20260998, 4501)
+    net = az.az_load_net(az.make_arch(52, 0, 128, 2, 1, cfg.precision, 8), pw.make_blob(cfg, 0.1, 0.6))
+    with pytest.raises(az.AzError) as e:
+        az.az_search_create(net, az.make_search_config(20, 2, 128, groups=2))    # 10 rows per step, the net takes 8
+    assert e.value.code == az.AZ_ERR_BATCH_TOO_LARGE
+    with pytest.raises(az.AzError) as e:
+        az.az_search_create(net, az.make_search_config(4, 1, 104))               # the net's action list is the 1,880 one
+    assert e.value.code == az.AZ_ERR_BAD_ARCH
+    az.az_free_net(net)

@@ -1,5 +1,6 @@
-"""The C-ABI library loads without a GPU and exports every function include/az_eval.h declares."""
+"""The C-ABI library loads without a GPU and exports every function the headers under include/ declare."""
 import ctypes
+import glob
 import os
 import re
 
@@ -9,9 +10,12 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def declared_functions():
-    with open(os.path.join(ROOT, "include", "az_eval.h")) as f:
-        text = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
-    return sorted(set(re.findall(r"\b(az_[a-z0-9_]+)\s*\(", text)))
+    names = set()
+    for header in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))):
+        with open(header) as f:
+            text = re.sub(r"/\*.*?\*/", "", f.read(), flags=re.S)
+        names |= set(re.findall(r"\b(az_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
 
 
 @pytest.fixture(scope="module")
@@ -22,7 +26,7 @@ def lib():
 
 def test_every_declared_entry_point_is_exported(lib):
     names = declared_functions()
-    assert {"az_load_net", "az_evaluate", "az_encode", "az_legal_masks", "az_free_net"} <= set(names)
+    assert {"az_load_net", "az_evaluate", "az_encode", "az_legal_masks", "az_free_net", "az_search_run", "az_apply_moves"} <= set(names)
     for name in names:
         assert hasattr(lib, name), name
 
