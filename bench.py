@@ -339,9 +339,9 @@ def run_search(args, name):
                          "flops_per_launch": flops},
         }
         if not args.no_cpu_baseline:
-            rate, dt = oracle_search_rate(recs, 400, 16)
+            rate, dt = oracle_search_rate(recs, 8000, 128)
             out["cpu_baseline"] = {"value": rate, "unit": SEARCH_UNIT, "cores": 1, "kind": "oracle",
-                                   "sample": f"16 games x 400 traversals, sequential, stand-in evaluator in place of the network "
+                                   "sample": f"128 games x 8,000 traversals, sequential, stand-in evaluator in place of the network "
                                              f"(the oracle has no network-backed search), {dt:.1f} s"}
         print(json.dumps(out))
     az.az_free_net(net)
