@@ -38,12 +38,14 @@ WORKLOADS = {
     "p12i": "p12i: p12 with the backbone's convolutions in int8 (pooled context and heads in floating point), batch 1024",
     "p14": "p14: the paper's own network at its reported size, 14x160 bf16, batch 320 as the paper serves it "
            "(App. D.3); --batch for other sizes",
+    "p14i": "p14i: p14 with the backbone's convolutions in int8, the precision the paper deploys; batch 320, --batch for other sizes",
+    "s14i": "s14i: the search of s14 over the int8 14x160 network",
     "s14": "s14: batched tree search (Eq. 1, c 1.5, first-play reduction 0.2, discount 0.99) over the paper's 14x160 "
            "network: two groups of games, each step one batch of leaf positions per group (320 rows as the paper "
            "serves, App. D.3; --batch for other sizes), one traversal per game and step",
     "s12": "s12: the same search over the 12x128 network",
 }
-SEARCH_NETS = {"s14": "p14", "s12": "p12"}
+SEARCH_NETS = {"s14": "p14", "s12": "p12", "s14i": "p14i"}
 SEARCH_METRIC = "searches/sec (tree traversals with their leaf evaluation)"
 SEARCH_UNIT = "searches/s"
 
@@ -250,6 +252,9 @@ def run_search(args, name):
     recs = make_records(cfg, games, first_index=sharding.rank_first_index(rank, games))
     blob = make_blob(cfg)
     net = az.az_load_net(az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, rows), blob)
+    if cfg.precision >= 2:      # 8-bit backbone: fix the activation ranges on the seeded calibration positions first
+        cal = positions.generate_moves(cfg.position_seed + configs.CALIBRATION_SEED_OFFSET, configs.CALIBRATION_COUNT, cfg.plies)[0]
+        az.az_calibrate(net, az.records_to_device(cal), cal.shape[0])
     nodes = (args.steps + args.warmup) * leaves + 2
 
     def new_search():
@@ -313,7 +318,7 @@ def run_search(args, name):
         total_s = ms_max * 1e-3
         achieved = flops * 2 * args.steps / total_s / 1e12
         sustained = total_s >= 1.0
-        peak_tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"]
+        peak_tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"] * (2.0 if cfg.precision >= 2 else 1.0)
         out = {
             "metric": SEARCH_METRIC, "value": world * searched / total_s, "unit": SEARCH_UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_max / args.steps,
@@ -332,7 +337,8 @@ def run_search(args, name):
             "clocks": clocks,
             "roofline": {"kernel": "tower_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
                          "frac": achieved / peak_tf, "traffic": None,
-                         "peak_source": f"of {peaks['source']} ({'sustained' if sustained else 'burst'} bf16 GEMM)",
+                         "peak_source": f"of {peaks['source']} ({'sustained' if sustained else 'burst'} bf16 GEMM"
+                                        + (" x 2, nominal 8-bit/bf16 ratio)" if cfg.precision >= 2 else ")"),
                          "note": "whole-loop figure: the tower's flops of all leaf batches over the search's elapsed time (the two "
                                  "groups' launches overlap, so a per-launch duration would count the shared time twice)",
                          "avg_launch_ms_overlapped": tower_ms / max(tower_passes, 1), "launches_timed": tower_passes,

@@ -56,6 +56,8 @@ PNET_CONFIGS = {
     "p14": PNetConfig("p14", 14, 160, 320, 20260962, 9371401),
     # p12 with the backbone's convolutions in int8, the precision the paper deploys (Sec. 4.3.6)
     "p12i": PNetConfig("p12i", 12, 128, 1024, 20260961, 9371201, precision=3, weights_like="p12"),
+    # the reported checkpoint's size in the precision the paper deploys it in (Sec. 4.3.6, App. B.1)
+    "p14i": PNetConfig("p14i", 14, 160, 320, 20260962, 9371401, precision=3, weights_like="p14"),
 }
 
 

@@ -274,7 +274,7 @@ int quantise_pnet(Net &n, const float *absmax) {
     if (!m) return AZ_ERR_UNSUPPORTED;
     const int C = (int)n.arch.channels, L = n.n_conv, P = C / 4, R = C - P;
     const float kTiny = 1e-30f;
-    constexpr int kStage = 9 * 128 * 32;              // bytes of one weight stage: 9 taps x 128 outputs x 32 bytes of K
+    const size_t kStage = (size_t)9 * C * 32;         // bytes of one weight stage: 9 taps x C outputs x 32 bytes of K
     std::vector<float> sa((size_t)L * C, 1.0f), ws((size_t)L * C, 1.0f);
     for (int l = 1; l < L; ++l)
         for (int c = 0; c < m->cin[l]; ++c) sa[(size_t)l * C + c] = fmaxf(absmax[(size_t)(l - 1) * C + c], kTiny) / 255.0f;

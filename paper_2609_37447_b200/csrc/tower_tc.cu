@@ -178,10 +178,10 @@ __global__ void __launch_bounds__(S::kThreads, 1)
 tower_tc_kernel(const TowerArgs args) {
     static_assert(!kInt8 || kFp8, "the int8 tower is a form of the 8-bit tower");
     static_assert(!kPnet || ((S::kC == 128 || S::kC == 160) && S::kSets == 1), "the paper's network runs on the one-set 128- and 160-channel shapes");
-    static_assert(!(kPnet && kFp8) || (kInt8 && S::kC == 128), "of the 8-bit towers the int8 one carries the paper's network, at 128 channels");
+    static_assert(!(kPnet && kFp8) || kInt8, "of the 8-bit towers the int8 one carries the paper's network");
     constexpr int kC = S::kC, kGroups = S::kGroups, kStages = S::kStages, kSlices = S::kSlices;
     constexpr int kFrameBytes = S::kFrameBytes, kStageBytes = S::kStageBytes, kThreads = S::kThreads;
-    static_assert(!kFp8 || kC == 128, "the FP8 tower exists for 128 channels");
+    static_assert(!kFp8 || kC == 128 || (kPnet && kC == 160), "the 8-bit towers exist for 128 channels and, for the paper's network, 160");
     extern __shared__ __align__(128) unsigned char smem[];
     // the warp index through a shuffle: the compiler then knows it is the same in all lanes, and role-
     // dependent address arithmetic can stay on the uniform datapath
@@ -1031,6 +1031,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape160, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape160, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
     const int sms = dev < 64 ? sm_count[dev] : 148;
@@ -1063,7 +1064,8 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     // one CTA per SM, or one per two-board group when there are fewer groups than SMs
     const int n_groups = (batch + kNB - 1) / kNB;
     const int grid = n_groups < sms ? n_groups : sms;
-    if (net.pnet && net.arch.channels == 160) tower_tc_kernel<false, Shape160, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(false, true), s>>>(a);
+    if (net.pnet && net.arch.channels == 160 && fp8) tower_tc_kernel<true, Shape160, true, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(true, true), s>>>(a);
+    else if (net.pnet && net.arch.channels == 160) tower_tc_kernel<false, Shape160, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(false, true), s>>>(a);
     else if (net.pnet && fp8) tower_tc_kernel<true, Shape128, true, true><<<grid, Shape128::kThreads, Shape128::smem_bytes(true, true), s>>>(a);
     else if (net.pnet) tower_tc_kernel<false, Shape128, true><<<grid, Shape128::kThreads, Shape128::smem_bytes(false, true), s>>>(a);
     else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);

@@ -152,6 +152,32 @@ def test_p12_with_an_int8_backbone():
     assert tg.min() >= 0.0 and tg.max() <= 6.0
 
 
+def test_p14_with_an_int8_backbone():
+    # the reported checkpoint's size in the deployed precision: 14 x 160, int8 convolutions, batch 320 and a ragged 299
+    import paper_2609_37447_b200 as az
+    cfg = pw.PNET_CONFIGS["p14i"]
+    blob = pw.make_blob(cfg)
+    cal, _ = positions.generate_moves(cfg.position_seed + 777_000_000, 512, cfg.plies)
+    net = load(az, cfg, blob, 512)
+    az.az_calibrate(net, az.records_to_device(cal), 512)
+    for batch in (320, 299):
+        rec, _ = positions.generate_moves(cfg.position_seed, batch, cfg.plies)
+        mg, pg, vg, tg = gpu_run(az, net, cfg, rec, tower=True)
+        rows = np.unique(np.concatenate([[0, 1, 147, 148, 149, 295, 296, batch - 2, batch - 1], np.arange(3, batch, 5)]))
+        mo, _, po, vo, extra = oracle.pnet_evaluate(blob, rec[rows], want_tower=True)
+        assert (mg[rows] == mo).all()
+        want = extra["tower"].reshape(rows.size, 160, 64).transpose(0, 2, 1)
+        rel = float(np.sqrt(((tg[rows] - want) ** 2).mean() / (want ** 2).mean()))
+        perr, verr = np.abs(pg[rows] - po).max(), np.abs(vg[rows] - vo).max()
+        agree = (pg[rows].argmax(axis=1) == po.argmax(axis=1)).mean()
+        print(f"p14i: n={rows.size} of {batch} policy max-abs {perr:.3e} value max-abs {verr:.3e} arg-max agreement {agree:.4f} backbone rms {rel:.3e}")
+        assert perr <= 5e-2 and verr <= 5e-2 and rel < 3e-2
+        assert tg.min() >= 0.0 and tg.max() <= 6.0
+        bits = np.unpackbits(mg.view(np.uint8), axis=1, bitorder="little")[:, :pw.ACTIONS].astype(bool)
+        assert np.isfinite(pg).all() and (pg[~bits] == 0.0).all() and np.abs(pg.sum(axis=1) - 1).max() < 1e-3
+    az.az_free_net(net)
+
+
 def test_other_entry_points_serve_the_papers_network_too():
     # legal-moves-only output, the pipelined host entry, CUDA-graph replay and the stand-alone encoder entry
     import paper_2609_37447_b200 as az
