@@ -41,8 +41,8 @@ WORKLOADS = {
     "p14i": "p14i: p14 with the backbone's convolutions in int8, the precision the paper deploys; batch 320, --batch for other sizes",
     "s14i": "s14i: the search of s14 over the int8 14x160 network",
     "s14": "s14: batched tree search (Eq. 1, c 1.5, first-play reduction 0.2, discount 0.99) over the paper's 14x160 "
-           "network: two groups of games, each step one batch of leaf positions per group (320 rows as the paper "
-           "serves, App. D.3; --batch for other sizes), one traversal per game and step",
+           "network: two groups of games, each step one batch of leaf positions per group (296 rows = one two-board "
+           "group per SM; the paper serves 320, App. D.3: --batch 320), one traversal per game and step",
     "s12": "s12: the same search over the 12x128 network",
 }
 SEARCH_NETS = {"s14": "p14", "s12": "p12", "s14i": "p14i"}
@@ -246,7 +246,7 @@ def run_search(args, name):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     cfg = get_config(name)
-    rows = args.batch if args.batch > 0 else 320
+    rows = args.batch if args.batch > 0 else 296     # one two-board group per SM and group of games (148 SMs)
     leaves = max(1, args.leaves)
     games = 2 * rows // leaves
     recs = make_records(cfg, games, first_index=sharding.rank_first_index(rank, games))

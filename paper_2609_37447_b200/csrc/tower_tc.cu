@@ -177,7 +177,7 @@ template <bool kFp8, class S, bool kPnet = false, bool kInt8 = false>
 __global__ void __launch_bounds__(S::kThreads, 1)
 tower_tc_kernel(const TowerArgs args) {
     static_assert(!kInt8 || kFp8, "the int8 tower is a form of the 8-bit tower");
-    static_assert(!kPnet || ((S::kC == 128 || S::kC == 160) && S::kSets == 1), "the paper's network runs on the one-set 128- and 160-channel shapes");
+    static_assert(!kPnet || S::kC == 128 || S::kC == 160, "the paper's network runs on the 128- and 160-channel shapes");
     static_assert(!(kPnet && kFp8) || kInt8, "of the 8-bit towers the int8 one carries the paper's network");
     constexpr int kC = S::kC, kGroups = S::kGroups, kStages = S::kStages, kSlices = S::kSlices;
     constexpr int kFrameBytes = S::kFrameBytes, kStageBytes = S::kStageBytes, kThreads = S::kThreads;
@@ -215,7 +215,7 @@ tower_tc_kernel(const TowerArgs args) {
         }
         for (int g = 0; g < kGroups; ++g) {
             ptx::mbar_init(bar_acc_full(g), 1);
-            ptx::mbar_init(bar_pool(g), 4);
+            ptx::mbar_init(bar_pool(g), 4 * S::kSets);
             for (int kc = 0; kc < kSlices; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4 * S::kSets);
         }
         ptx::mbar_init(bar_done, kGroups);
@@ -504,8 +504,9 @@ tower_tc_kernel(const TowerArgs args) {
                             const __nv_bfloat162 h2 = __floats2bfloat162_rn(pv[8 * j + 2 * i], pv[8 * j + 2 * i + 1]);
                             w[i] = *reinterpret_cast<const uint32_t *>(&h2);
                         }
-                        *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) =
-                            live ? make_uint4(w[0], w[1], w[2], w[3]) : make_uint4(0, 0, 0, 0);
+                        if (S::kSets == 1 || (j % S::kSets) == set)
+                            *reinterpret_cast<uint4 *>(frame + j * kPlaneBytes + slot * 16) =
+                                live ? make_uint4(w[0], w[1], w[2], w[3]) : make_uint4(0, 0, 0, 0);
                     }
                 } else {
                     const PosCur *rec = reinterpret_cast<const PosCur *>(args.positions + (size_t)(live ? board : 0) * args.position_stride);
@@ -571,8 +572,13 @@ tower_tc_kernel(const TowerArgs args) {
                     // half of its values that its partner keeps): 4 + 2 + 1 exchanges, after which every lane of
                     // the eight holds one channel; one more exchange joins the board's two row groups.  Sums and
                     // maxima travel together.
+                    // With two sets the eight-channel chunks go to the set that owns their 16-channel slice (whose
+                    // constants that set's warps hold).
 #pragma unroll
                     for (int pc = 0; pc < kPoolC / 8; ++pc) {
+                        const int pslice = (kRegC + pc * 8) / 16;                 // the slice this chunk lies in
+                        if (S::kSets > 1 && (pslice % S::kSets) != set) continue;
+                        const int cidx = (pslice / S::kSets) * 16 + (kRegC + pc * 8) % 16;   // in this warp's copy of the constants
                         uint32_t r8[8];
                         ptx::tmem_ld8(t_src + (uint32_t)(kRegC + pc * 8), r8);
                         ptx::tmem_ld_wait();
@@ -581,8 +587,8 @@ tower_tc_kernel(const TowerArgs args) {
                         for (int i = 0; i < 8; ++i) {
                             // (8-bit tower: int32 accumulator times the weight scale; these channels are not handed on,
                             // so their constants carry no activation scale and the value is in real units)
-                            const float pre = kFp8 ? fmaf(__int2float_rn((int)r8[i]), lc[kRegC + pc * 8 + i], bias[kRegC + pc * 8 + i])
-                                                   : __uint_as_float(r8[i]) + bias[kRegC + pc * 8 + i];
+                            const float pre = kFp8 ? fmaf(__int2float_rn((int)r8[i]), lc[cidx + i], bias[cidx + i])
+                                                   : __uint_as_float(r8[i]) + bias[cidx + i];
                             sm[i] = live ? fminf(fmaxf(pre, 0.0f), 6.0f) : 0.0f;
                             mx[i] = sm[i];
                         }
@@ -606,7 +612,9 @@ tower_tc_kernel(const TowerArgs args) {
                             pool_part[4 * 2 * kPoolC + (q * 2 + b) * kPoolC + c0] = mx[0];
                         }
                     }
-                    auto meet = [&]() -> bool {                                // the group's four warps, bounded
+                    constexpr int kGroupThreads = 128 * S::kSets;
+                    const int gt = (ew % (4 * S::kSets)) * 32 + lane;          // this thread among the group's epilogue threads
+                    auto meet = [&]() -> bool {                                // the group's epilogue warps, bounded
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(bar_pool(g));
                         const bool met = wait_bar(bar_pool(g), pool_phase, abort_flag, args.status);
@@ -616,7 +624,7 @@ tower_tc_kernel(const TowerArgs args) {
                     ok = meet();
                     if (!ok) break;
                     // (2) the four warps' partial results -> the pooled vector: one entry per thread
-                    for (int e = q * 32 + lane; e < 2 * 2 * kPoolC; e += 128) {   // e = board * 2 * kPoolC + entry
+                    for (int e = gt; e < 2 * 2 * kPoolC; e += kGroupThreads) {   // e = board * 2 * kPoolC + entry
                         const int pb = e / (2 * kPoolC), j = e % (2 * kPoolC), c = j % kPoolC;
                         const float *src = pool_part + (j >= kPoolC ? 4 * 2 * kPoolC : 0);
                         float acc = src[(0 * 2 + pb) * kPoolC + c];
@@ -629,7 +637,7 @@ tower_tc_kernel(const TowerArgs args) {
                     }
                     constexpr int kCtxPad = kCtxStride > kRegC ? kCtxStride - kRegC : 1;
                     if (kCtxStride > kRegC)                                    // the padding of the context stays zero
-                        for (int z = q * 32 + lane; z < 2 * kCtxPad; z += 128)
+                        for (int z = gt; z < 2 * kCtxPad; z += kGroupThreads)
                             pool_ctx[(z / kCtxPad) * kCtxStride + kRegC + z % kCtxPad] = 0.0f;
                     ok = meet();
                     if (!ok) break;
@@ -638,7 +646,7 @@ tower_tc_kernel(const TowerArgs args) {
                     // neighbouring words.
                     {
                         const float *gwt = args.gw + (size_t)((l - 3) >> 2) * kRegC * 2 * kPoolC;
-                        for (int e = q * 32 + lane; e < 2 * kRegC; e += 128) {
+                        for (int e = gt; e < 2 * kRegC; e += kGroupThreads) {
                             const int pb = e / kRegC, rr0 = e % kRegC;
                             const float *vec = pool_vec + pb * 2 * kPoolC;
                             float acc0 = 0.0f, acc1 = 0.0f;
@@ -654,14 +662,14 @@ tower_tc_kernel(const TowerArgs args) {
                     if (!ok) break;
                 }
                 const float *ctx = pool_ctx + b * kCtxStride;                  // this row's board
-                const int n_my = (kPnet && pooled) ? kShortSlices : kMySlices; // the pooled channels are not handed on
+                const int n_kc = (kPnet && pooled) ? kShortSlices : kSlices;   // the pooled channels are not handed on
                 ptx::tmem_ld16(t_src + (uint32_t)(set * 16), r[0]);
 #pragma unroll
                 for (int ks = 0; ks < kMySlices; ++ks) {
-                    if (kPnet && ks >= n_my) break;
                     const int kc = ks * S::kSets + set;             // the slice; ks indexes this warp's constants
+                    if (kPnet && kc >= n_kc) break;
                     ptx::tmem_ld_wait();
-                    if (ks + 1 < n_my) ptx::tmem_ld16(t_src + (uint32_t)((kc + S::kSets) * 16), r[(ks + 1) & 1]);
+                    if (kc + S::kSets < n_kc) ptx::tmem_ld16(t_src + (uint32_t)((kc + S::kSets) * 16), r[(ks + 1) & 1]);
                     uint32_t(&rr)[16] = r[ks & 1];
                     float v[16];
 #pragma unroll
@@ -688,7 +696,7 @@ tower_tc_kernel(const TowerArgs args) {
                     }
                     if (kPnet && pooled) {
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] += ctx[ks * 16 + i];
+                        for (int i = 0; i < 16; ++i) v[i] += ctx[kc * 16 + i];
                     }
                     // ReLU: a first convolution's output is only ever read as packed operands, and the
                     // conversion clamps; elsewhere the fp32 value itself goes on (residual stream, output)
@@ -850,7 +858,16 @@ typedef Shape<128, 2, 1> Shape128;
 #endif
 typedef Shape<128, 2, AZ_FP8_EPI_SETS> Shape128F8;
 typedef Shape<256, 1, 1> Shape256;
-typedef Shape<160, 1, 1> Shape160;
+// the paper's 160-channel network: one group, whose epilogue (not its MMAs) sets the pace with four warps;
+// two sets of four share each layer
+#ifndef AZ_P160_SETS
+#define AZ_P160_SETS 2
+#endif
+typedef Shape<160, 1, AZ_P160_SETS> Shape160;
+#ifndef AZ_P128_SETS
+#define AZ_P128_SETS 2
+#endif
+typedef Shape<128, 2, AZ_P128_SETS> Shape128P;           // the paper's 128-channel network
 constexpr int kStageBytes = Shape128::kStageBytes;       // host-side packing of the 128-channel stages
 
 }  // namespace
@@ -1028,9 +1045,9 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
-        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128P, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape160, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
-        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128P, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape160, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
@@ -1066,8 +1083,8 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     const int grid = n_groups < sms ? n_groups : sms;
     if (net.pnet && net.arch.channels == 160 && fp8) tower_tc_kernel<true, Shape160, true, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(true, true), s>>>(a);
     else if (net.pnet && net.arch.channels == 160) tower_tc_kernel<false, Shape160, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(false, true), s>>>(a);
-    else if (net.pnet && fp8) tower_tc_kernel<true, Shape128, true, true><<<grid, Shape128::kThreads, Shape128::smem_bytes(true, true), s>>>(a);
-    else if (net.pnet) tower_tc_kernel<false, Shape128, true><<<grid, Shape128::kThreads, Shape128::smem_bytes(false, true), s>>>(a);
+    else if (net.pnet && fp8) tower_tc_kernel<true, Shape128P, true, true><<<grid, Shape128P::kThreads, Shape128P::smem_bytes(true, true), s>>>(a);
+    else if (net.pnet) tower_tc_kernel<false, Shape128P, true><<<grid, Shape128P::kThreads, Shape128P::smem_bytes(false, true), s>>>(a);
     else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
     else if (fp8 && net.int8) tower_tc_kernel<true, Shape128F8, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else if (fp8) tower_tc_kernel<true, Shape128F8><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
