@@ -852,7 +852,10 @@ tower_tc_kernel(const TowerArgs args) {
     }
 }
 
-typedef Shape<128, 2, 1> Shape128;
+#ifndef AZ_C128_SETS
+#define AZ_C128_SETS 1
+#endif
+typedef Shape<128, 2, AZ_C128_SETS> Shape128;
 #ifndef AZ_FP8_EPI_SETS
 #define AZ_FP8_EPI_SETS 2
 #endif
