@@ -73,6 +73,16 @@ def _load():
         lib.orc_mcts_search.restype = ci
         lib.orc_mcts_search.argtypes = [vp, ci, ci, ci, ci, ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_uint64,
                                         ci, ci, vp, vp, vp, vp, vp, vp, vp]
+        lib.orc_mcts_new.restype = vp
+        lib.orc_mcts_new.argtypes = [vp, ci, ci, ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_uint64, ci, ci]
+        lib.orc_mcts_run.restype = ci
+        lib.orc_mcts_run.argtypes = [vp, ci, ci]
+        lib.orc_mcts_advance.restype = ci
+        lib.orc_mcts_advance.argtypes = [vp, ci]
+        lib.orc_mcts_read.restype = ci
+        lib.orc_mcts_read.argtypes = [vp] * 9
+        lib.orc_mcts_free.restype = None
+        lib.orc_mcts_free.argtypes = [vp]
         lib.orc_pnet_forward.restype = ci
         lib.orc_pnet_forward.argtypes = [vp, ctypes.c_size_t, vp, vp, ci, vp, vp, vp, vp]
         lib.orc_conv3x3.restype = None
@@ -182,6 +192,52 @@ def mcts_search(record, head: int, simulations: int, leaves: int = 1, c_puct: fl
     return {"actions": actions[:k].copy(), "visits": visits[:k].copy(), "w": w[:k].copy(), "prior": prior[:k].copy(),
             "n_nodes": int(counts[0]), "n_edges": int(counts[1]), "flags": int(counts[2]), "idle": int(counts[3]),
             "node_nvis": nvis[:counts[0]].copy(), "node_wsum": wsum[:counts[0]].copy()}
+
+
+class MctsTree:
+    """A search of one game that lives across played moves (the subtree under the played move is kept)."""
+
+    def __init__(self, record, head: int, leaves: int = 1, c_puct: float = 1.5, fpu_reduction: float = 0.2,
+                 discount: float = 0.99, seed: int = 0, node_cap: int = 1024, edge_cap: int | None = None):
+        rec, stride, n = _records(record)
+        assert n == 1
+        self.dtype, self.leaves, self.node_cap = rec.dtype, leaves, node_cap
+        self.handle = _load().orc_mcts_new(rec.ctypes.data, stride, head, c_puct, fpu_reduction, discount, seed,
+                                           node_cap, edge_cap or node_cap * 64)
+        if not self.handle:
+            raise ValueError("bad search arguments")
+
+    def run(self, simulations: int):
+        if _load().orc_mcts_run(self.handle, simulations, self.leaves) != 0:
+            raise ValueError("bad search arguments")
+
+    def advance(self, action: int):
+        """Plays `action` at the root; ValueError if the root has no such move."""
+        if _load().orc_mcts_advance(self.handle, int(action)) != 0:
+            raise ValueError("the root has no such move")
+
+    def read(self) -> dict:
+        actions = np.zeros(256, dtype=np.int32)
+        visits = np.zeros(256, dtype=np.int32)
+        w = np.zeros(256, dtype=np.float32)
+        prior = np.zeros(256, dtype=np.float32)
+        counts = np.zeros(4, dtype=np.int32)
+        nvis = np.zeros(self.node_cap, dtype=np.int32)
+        wsum = np.zeros(self.node_cap, dtype=np.float32)
+        root = np.zeros(1, dtype=self.dtype)
+        k = _load().orc_mcts_read(self.handle, actions.ctypes.data, visits.ctypes.data, w.ctypes.data, prior.ctypes.data,
+                                  counts.ctypes.data, nvis.ctypes.data, wsum.ctypes.data, root.ctypes.data)
+        return {"actions": actions[:k].copy(), "visits": visits[:k].copy(), "w": w[:k].copy(), "prior": prior[:k].copy(),
+                "n_nodes": int(counts[0]), "n_edges": int(counts[1]), "flags": int(counts[2]), "idle": int(counts[3]),
+                "node_nvis": nvis[:counts[0]].copy(), "node_wsum": wsum[:counts[0]].copy(), "root": root}
+
+    def close(self):
+        if self.handle:
+            _load().orc_mcts_free(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        self.close()
 
 
 def encode52(records) -> np.ndarray:

@@ -13,7 +13,12 @@
  *    node still waiting for its evaluation is given up (its reservations are removed, its slot idles);
  *  - a node is terminal if the mover has no legal move (value -1 in check, else 0) or the halfmove
  *    clock has reached 100 (value 0); repetitions are not tracked inside the tree;
- *  - the root's evaluation is a step of its own before the counted simulations.
+ *  - the root's evaluation is a step of its own before the counted simulations;
+ *  - when a move is played (Sec. 3.3: the relevant subtree becomes the next root) the subtree under the
+ *    root's edge of that action is kept with all its statistics and renumbered breadth-first (a node's
+ *    children in the order of its edges), everything else is dropped; if that edge has no child yet the
+ *    new tree is the bare successor position, waiting for its root evaluation.  Retaining only a share
+ *    of the visits (the paper's 60 %) belongs to self-play's recipe and is not applied.
  * Every decision (the arg-max of Eq. 1) is taken in float32 with one rounding per operation, in the
  * order written below, ties to the lower action index.
  *
@@ -180,6 +185,101 @@ static void finish(Tree *t, Slot *s) {
     }
 }
 
+static Tree *tree_new(const void *root_record, int stride, int head, float c_puct, float fpu_reduction, float discount,
+                      uint64_t seed, int node_cap, int edge_cap) {
+    Tree *t = (Tree *)calloc(1, sizeof(Tree));
+    t->nodes = (Node *)calloc((size_t)node_cap, sizeof(Node));
+    t->edges = (Edge *)calloc((size_t)edge_cap, sizeof(Edge));
+    t->node_cap = node_cap; t->edge_cap = edge_cap; t->stride = stride; t->head = head;
+    t->c_puct = c_puct; t->fpu_reduction = fpu_reduction; t->discount = discount; t->seed = seed;
+    memcpy(t->nodes[0].rec, root_record, (size_t)stride);
+    t->nodes[0].n_edges = -1;
+    t->n_nodes = 1;
+    return t;
+}
+
+static void tree_run(Tree *t, int simulations, int leaves) {
+    Slot *slots = (Slot *)calloc((size_t)leaves, sizeof(Slot));
+    const int steps = simulations + (t->root_submitted ? 0 : 1);      /* the root's own evaluation first */
+    for (int step = 0; step < steps; ++step) {
+        for (int j = 0; j < leaves; ++j) descend(t, &slots[j]);
+        for (int j = 0; j < leaves; ++j) finish(t, &slots[j]);
+    }
+    free(slots);
+}
+
+/* The move `action` is played at the root.  Returns 0, or -1 if the root has no such edge (nothing changes). */
+static int tree_advance(Tree *t, int action) {
+    const Node *root = &t->nodes[0];
+    int e0 = -1;
+    for (int i = 0; i < root->n_edges; ++i)
+        if (t->edges[root->edge_begin + i].action == action) e0 = root->edge_begin + i;
+    if (e0 < 0) return -1;
+    Node *nodes = (Node *)calloc((size_t)t->node_cap, sizeof(Node));
+    Edge *edges = (Edge *)calloc((size_t)t->edge_cap, sizeof(Edge));
+    int n_nodes = 1, n_edges = 0;
+    if (t->edges[e0].child < 0) {
+        int32_t a = action;
+        orc_apply_moves(root->rec, t->stride, 1, t->head, &a, nodes[0].rec);
+        nodes[0].n_edges = -1;
+        t->root_submitted = 0;
+    } else {
+        int *old_of = (int *)calloc((size_t)t->node_cap, sizeof(int));
+        old_of[0] = t->edges[e0].child;
+        for (int i = 0; i < n_nodes; ++i) {                           /* breadth-first: new node i was old node old_of[i] */
+            nodes[i] = t->nodes[old_of[i]];
+            const int begin = nodes[i].edge_begin;
+            nodes[i].edge_begin = n_edges;
+            for (int j = 0; j < nodes[i].n_edges; ++j) {
+                Edge e = t->edges[begin + j];
+                if (e.child >= 0) { old_of[n_nodes] = e.child; e.child = n_nodes++; }
+                edges[n_edges++] = e;
+            }
+        }
+        free(old_of);
+    }
+    free(t->nodes); free(t->edges);
+    t->nodes = nodes; t->edges = edges; t->n_nodes = n_nodes; t->n_edges = n_edges;
+    return 0;
+}
+
+static int tree_read(const Tree *t, int32_t *root_actions, int32_t *root_visits, float *root_w, float *root_prior,
+                     int32_t *counts, int32_t *node_nvis, float *node_wsum, void *root_record) {
+    const Node *root = &t->nodes[0];
+    const int k = root->n_edges > 0 ? root->n_edges : 0;
+    for (int i = 0; i < k && i < 256; ++i) {
+        const Edge *e = &t->edges[root->edge_begin + i];
+        root_actions[i] = e->action; root_visits[i] = e->n; root_w[i] = e->w; root_prior[i] = e->prior;
+    }
+    counts[0] = t->n_nodes; counts[1] = t->n_edges; counts[2] = (int32_t)t->flags; counts[3] = t->idle;
+    if (node_nvis && node_wsum)
+        for (int i = 0; i < t->n_nodes; ++i) { node_nvis[i] = t->nodes[i].nvis; node_wsum[i] = t->nodes[i].wsum; }
+    if (root_record) memcpy(root_record, root->rec, (size_t)t->stride);
+    return k;
+}
+
+/* A search that lives across calls (moves played, subtrees kept). */
+void *orc_mcts_new(const void *root_record, int stride, int head, float c_puct, float fpu_reduction, float discount,
+                   uint64_t seed, int node_cap, int edge_cap) {
+    if (stride > MAX_STRIDE || node_cap < 2 || edge_cap < 1) return NULL;
+    return tree_new(root_record, stride, head, c_puct, fpu_reduction, discount, seed, node_cap, edge_cap);
+}
+int orc_mcts_run(void *tree, int simulations, int leaves) {
+    if (!tree || leaves < 1 || leaves > 64) return -1;
+    tree_run((Tree *)tree, simulations, leaves);
+    return 0;
+}
+int orc_mcts_advance(void *tree, int action) { return tree ? tree_advance((Tree *)tree, action) : -1; }
+int orc_mcts_read(const void *tree, int32_t *root_actions, int32_t *root_visits, float *root_w, float *root_prior,
+                  int32_t *counts, int32_t *node_nvis, float *node_wsum, void *root_record) {
+    return tree_read((const Tree *)tree, root_actions, root_visits, root_w, root_prior, counts, node_nvis, node_wsum, root_record);
+}
+void orc_mcts_free(void *tree) {
+    Tree *t = (Tree *)tree;
+    if (!t) return;
+    free(t->nodes); free(t->edges); free(t);
+}
+
 /* One search from `root_record`: the root's evaluation, then `simulations` steps of `leaves` traversals each
  * (all traversals of a step choose their paths before any of the step's results arrive).
  * Out: the root's edges (action, visits, value sum, prior; at most 256), the counts of nodes and edges,
@@ -189,28 +289,9 @@ int orc_mcts_search(const void *root_record, int stride, int head, int simulatio
                     int32_t *root_actions, int32_t *root_visits, float *root_w, float *root_prior,
                     int32_t *counts /* n_nodes, n_edges, flags, idle */, int32_t *node_nvis, float *node_wsum) {
     if (stride > MAX_STRIDE || leaves < 1 || leaves > 64) return -1;
-    Tree t;
-    memset(&t, 0, sizeof t);
-    t.nodes = (Node *)calloc((size_t)node_cap, sizeof(Node));
-    t.edges = (Edge *)calloc((size_t)edge_cap, sizeof(Edge));
-    t.node_cap = node_cap; t.edge_cap = edge_cap; t.stride = stride; t.head = head;
-    t.c_puct = c_puct; t.fpu_reduction = fpu_reduction; t.discount = discount; t.seed = seed;
-    memcpy(t.nodes[0].rec, root_record, (size_t)stride);
-    t.nodes[0].n_edges = -1;
-    t.n_nodes = 1;
-    Slot *slots = (Slot *)calloc((size_t)leaves, sizeof(Slot));
-    for (int step = -1; step < simulations; ++step) {
-        for (int j = 0; j < leaves; ++j) descend(&t, &slots[j]);
-        for (int j = 0; j < leaves; ++j) finish(&t, &slots[j]);
-    }
-    const Node *root = &t.nodes[0];
-    for (int i = 0; i < root->n_edges && i < 256; ++i) {
-        const Edge *e = &t.edges[root->edge_begin + i];
-        root_actions[i] = e->action; root_visits[i] = e->n; root_w[i] = e->w; root_prior[i] = e->prior;
-    }
-    counts[0] = t.n_nodes; counts[1] = t.n_edges; counts[2] = (int32_t)t.flags; counts[3] = t.idle;
-    for (int i = 0; i < t.n_nodes; ++i) { node_nvis[i] = t.nodes[i].nvis; node_wsum[i] = t.nodes[i].wsum; }
-    const int k = root->n_edges;
-    free(slots); free(t.nodes); free(t.edges);
+    Tree *t = tree_new(root_record, stride, head, c_puct, fpu_reduction, discount, seed, node_cap, edge_cap);
+    tree_run(t, simulations, leaves);
+    const int k = tree_read(t, root_actions, root_visits, root_w, root_prior, counts, node_nvis, node_wsum, NULL);
+    orc_mcts_free(t);
     return k;
 }

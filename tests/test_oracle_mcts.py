@@ -131,3 +131,65 @@ def test_pools_that_fill_up_are_reported():
     assert r["flags"] & 1 and r["n_nodes"] == 40 and r["visits"].sum() + r["idle"] == 100
     r = oracle.mcts_search(rec, 2, 100, node_cap=128, edge_cap=300)
     assert r["flags"] & 2 and r["n_edges"] <= 300 and r["visits"].sum() == 100
+
+
+def test_played_moves_keep_their_subtree():
+    rec = positions.record_from_fen(START)
+    t = oracle.MctsTree(rec, 2, seed=4, node_cap=700)
+    t.run(300)
+    before = t.read()
+    best = int(np.argmax(before["visits"]))
+    action, n_child = int(before["actions"][best]), int(before["visits"][best])
+    t.advance(action)
+    after = t.read()
+    # the new root is the old child: its position is the successor, its visits are the old edge's, and every visit
+    # through it had opened exactly one node of its subtree (no terminal nodes this early in the game)
+    assert (after["root"].view(np.uint8) == oracle.apply_moves(rec, 2, [action]).view(np.uint8)).all()
+    assert after["node_nvis"][0] == n_child and after["n_nodes"] == n_child and after["visits"].sum() == n_child - 1
+    # the kept statistics are the old ones: every (visits, value sum) pair of the new tree occurs in the old one
+    old = {(int(n), np.float32(w).tobytes()) for n, w in zip(before["node_nvis"], before["node_wsum"])}
+    assert all((int(n), np.float32(w).tobytes()) in old for n, w in zip(after["node_nvis"], after["node_wsum"]))
+    # breadth-first renumbering: a node's visits never exceed its parent's, so the root comes first and the
+    # first level (the root's visited edges, in edge order) follows
+    level1 = after["visits"][after["visits"] > 0]
+    assert (after["node_nvis"][1:1 + len(level1)] == level1).all()
+    # the search goes on from the kept statistics
+    t.run(100)
+    more = t.read()
+    assert more["node_nvis"][0] == n_child + 100 and more["visits"].sum() == n_child - 1 + 100
+    with pytest.raises(ValueError):
+        t.advance(1879)                                                  # a promotion cannot be legal here
+    t.close()
+
+
+def test_a_move_without_a_subtree_starts_a_fresh_tree():
+    rec = positions.record_from_fen(START)
+    t = oracle.MctsTree(rec, 2, seed=6, node_cap=300)
+    t.run(5)
+    r = t.read()
+    unvisited = int(r["actions"][np.flatnonzero(r["visits"] == 0)[0]])
+    t.advance(unvisited)
+    assert t.read()["n_nodes"] == 1 and len(t.read()["actions"]) == 0      # waiting for its root evaluation
+    t.run(120)
+    got = t.read()
+    want = oracle.mcts_search(oracle.apply_moves(rec, 2, [unvisited]), 2, 120, seed=6, node_cap=300)
+    assert (got["visits"] == want["visits"]).all() and (got["w"].view(np.uint32) == want["w"].view(np.uint32)).all()
+    assert (got["node_nvis"] == want["node_nvis"]).all()
+    t.close()
+
+
+def test_a_game_played_by_the_search_follows_the_rules():
+    rec = positions.record_from_fen(START)
+    t = oracle.MctsTree(rec, 2, leaves=2, seed=8, node_cap=400)
+    cur = rec
+    for ply in range(30):
+        t.run(60)
+        r = t.read()
+        if len(r["actions"]) == 0:
+            break
+        a = int(r["actions"][int(np.argmax(r["visits"]))])
+        cur = oracle.apply_moves(cur, 2, [a])
+        t.advance(a)
+        assert (t.read()["root"].view(np.uint8) == cur.view(np.uint8)).all()
+    assert ply >= 10
+    t.close()
