@@ -135,6 +135,24 @@ int az_search_root(az_search *search, int game, int32_t *actions_host, int32_t *
 int az_search_root_visits(az_search *search, int32_t *actions_host, int32_t *visits_host, int32_t *counts_host);
 
 /*
+ * A move is played in every game (Sec. 3.3: "the relevant subtree becomes the next root").  actions_host holds
+ * one policy index per game, -1 for "no move in this game"; actions_host == NULL plays each game's most visited
+ * root move (ties to the lower policy index).  The subtree under the played move is kept with all its
+ * statistics and renumbered breadth-first (a node's children in the order of its edges); if that move has no
+ * subtree yet the game's tree becomes the bare successor position and the next az_search_run starts with a step
+ * in which such trees evaluate their roots while the others sit out.  A game whose root has no moves (the game
+ * is over, or the root was never evaluated), whose action is -1 or is not a move of its root (flag
+ * AZ_SEARCH_FLAG_BAD_ACTION) keeps its tree.  played_host (may be NULL) receives the action played per game,
+ * -1 where none was.  Keeping only a share of the old visits (the paper's 60 %) is self-play's recipe and is
+ * not applied.  The first call allocates a second set of tree pools (the kept subtrees are copied there).
+ * Errors: BAD_ARG, CUDA.
+ */
+int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *played_host);
+
+/* The current root records of all games, to a host buffer of games * position_bytes. */
+int az_search_root_positions(az_search *search, void *positions_host);
+
+/*
  * One game's tree: counts_out[4] = nodes, edges, AZ_SEARCH_FLAG_* bits, traversals given up;
  * node_visits_host / node_value_sum_host (max_nodes entries each, may be NULL) receive per node, in
  * the order the nodes were opened, the number of values backed up through it and their sum.

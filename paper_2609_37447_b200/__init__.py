@@ -28,7 +28,7 @@ EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_siz
            "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error",
            "az_apply_moves", "az_standin_evaluate", "az_search_create", "az_search_destroy", "az_search_set_roots",
-           "az_search_run", "az_search_root", "az_search_root_visits", "az_search_tree", "az_search_launches_per_step")
+           "az_search_run", "az_search_root", "az_search_root_visits", "az_search_advance", "az_search_root_positions", "az_search_tree", "az_search_launches_per_step")
 
 
 class az_arch(ctypes.Structure):
@@ -123,6 +123,10 @@ def _load_library():
     lib.az_search_root.argtypes = [vp, ci, vp, vp, vp, vp, ctypes.POINTER(ctypes.c_int32)]
     lib.az_search_root_visits.restype = ci
     lib.az_search_root_visits.argtypes = [vp, vp, vp, vp]
+    lib.az_search_advance.restype = ci
+    lib.az_search_advance.argtypes = [vp, vp, vp]
+    lib.az_search_root_positions.restype = ci
+    lib.az_search_root_positions.argtypes = [vp, vp]
     lib.az_search_tree.restype = ci
     lib.az_search_tree.argtypes = [vp, ci, vp, vp, vp]
     lib.az_search_launches_per_step.restype = ci
@@ -405,6 +409,28 @@ def az_search_root_visits(search: Search, actions_host: np.ndarray, visits_host:
             raise TypeError("int32 C-contiguous arrays of [games][AZ_MAX_LEGAL], [games][AZ_MAX_LEGAL], [games] expected")
     _check(_lib.az_search_root_visits(search.handle, actions_host.ctypes.data, visits_host.ctypes.data, counts_host.ctypes.data),
            "az_search_root_visits")
+
+
+def az_search_advance(search: Search, actions_host=None) -> np.ndarray:
+    """Plays one move per game (actions_host: int32 policy indices, -1 = none; None: the most visited root move).
+    Returns the actions played, -1 where a game's tree stayed as it was."""
+    played = np.zeros(search.config.games, dtype=np.int32)
+    act = None
+    if actions_host is not None:
+        act = np.ascontiguousarray(actions_host, dtype=np.int32)
+        if act.shape != (search.config.games,):
+            raise ValueError("one action per game expected")
+    _check(_lib.az_search_advance(search.handle, act.ctypes.data if act is not None else None, played.ctypes.data), "az_search_advance")
+    return played
+
+
+def az_search_root_positions(search: Search, dtype) -> np.ndarray:
+    """The current root records of all games as a numpy array of the given record dtype."""
+    out = np.zeros(search.config.games, dtype=dtype)
+    if out.dtype.itemsize != search.config.position_bytes:
+        raise ValueError("dtype does not match the search's position records")
+    _check(_lib.az_search_root_positions(search.handle, out.ctypes.data), "az_search_root_positions")
+    return out
 
 
 def az_search_tree(search: Search, game: int, nodes: bool = True):

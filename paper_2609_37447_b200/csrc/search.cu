@@ -14,6 +14,7 @@
 
 #include <mutex>
 #include <new>
+#include <utility>
 
 namespace az {
 namespace {
@@ -256,7 +257,7 @@ __device__ __forceinline__ void undo_path(const Trees &t, Edge *edges, Node *nod
 
 // select: one warp per game, `leaves` traversals one after the other
 __global__ void __launch_bounds__(32 * kWarps)
-search_select_kernel(Trees t, Batch b, int game0, int n_games) {
+search_select_kernel(Trees t, Batch b, int game0, int n_games, int root_step) {
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int gl = blockIdx.x * kWarps + w;
     if (gl >= n_games) return;
@@ -269,6 +270,12 @@ search_select_kernel(Trees t, Batch b, int game0, int n_games) {
         const int row = gl * t.leaves + j;
         int *pe = b.path_e + (size_t)row * kMaxDepth, *pn = b.path_n + (size_t)row * kMaxDepth;
         int kind = kSlotNone, leaf = -1, depth = 0;
+        if (root_step && gs->root_submitted && j == 0) {
+            // a step that exists only for the trees whose root still waits for its evaluation: this tree sits it out
+            for (int jj = lane; jj < t.leaves; jj += 32) b.kind[gl * t.leaves + jj] = kSlotNone;
+            __syncwarp();
+            break;
+        }
         if (!gs->root_submitted) {
             // the root's own evaluation, once; the step's other rows idle
             __syncwarp();
@@ -488,6 +495,11 @@ struct Search {
     cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
     unsigned char *roots_stage = nullptr;        // device copy of the root records
     int *out_actions = nullptr, *out_visits = nullptr, *out_counts = nullptr;   // read-out of all roots
+    bool need_root_step = true;                  // some tree's root still waits for its evaluation
+    // played moves: the kept subtrees are written to a second set of pools, which then becomes the first
+    Node *alt_nodes = nullptr; Edge *alt_edges = nullptr; unsigned char *alt_node_pos = nullptr;
+    int *remap = nullptr;                        // [games][max_nodes]: old index of every kept node
+    int *adv_actions = nullptr, *adv_played = nullptr, *adv_fresh = nullptr;
 };
 
 void free_search(Search *s) {
@@ -495,6 +507,8 @@ void free_search(Search *s) {
     cudaFree(s->trees.nodes); cudaFree(s->trees.edges); cudaFree(s->trees.node_pos); cudaFree(s->trees.games);
     cudaFree(s->roots_stage);
     cudaFree(s->out_actions); cudaFree(s->out_visits); cudaFree(s->out_counts);
+    cudaFree(s->alt_nodes); cudaFree(s->alt_edges); cudaFree(s->alt_node_pos); cudaFree(s->remap);
+    cudaFree(s->adv_actions); cudaFree(s->adv_played); cudaFree(s->adv_fresh);
     for (Group &g : s->groups) {
         cudaFree(g.batch.pos); cudaFree(g.batch.kind); cudaFree(g.batch.leaf); cudaFree(g.batch.depth);
         cudaFree(g.batch.path_e); cudaFree(g.batch.path_n);
@@ -523,6 +537,98 @@ __global__ void reset_trees_kernel(Trees t, const unsigned char *__restrict__ ro
     for (int i = threadIdx.x; i < t.stride / 8; i += blockDim.x) dst[i] = src[i];
 }
 
+// A move is played in every game (Sec. 3.3: the relevant subtree becomes the next root).  One warp per game:
+// the root's edge of the action (given, or the most visited one, ties to the lower action) is looked up; the
+// subtree under it is copied to the other pools breadth-first, a node's children in the order of its edges;
+// without a child the new tree is the bare successor position.  actions[g] == -1, a root without edges or an
+// action the root does not have leave the game's tree as it is (copied whole); played[g] tells which it was.
+__global__ void __launch_bounds__(32 * kWarps)
+search_advance_kernel(Trees t, Node *new_nodes, Edge *new_edges, unsigned char *new_pos, int games,
+                      const int *__restrict__ actions, int *__restrict__ played, int *__restrict__ remap_all, int *any_fresh) {
+    const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = blockIdx.x * kWarps + w;
+    if (g >= games) return;
+    const Node *nodes = t.nodes + (size_t)g * t.node_cap;
+    const Edge *edges = t.edges + (size_t)g * t.edge_cap;
+    const unsigned char *npos = t.node_pos + (size_t)g * t.node_cap * t.stride;
+    Node *nn = new_nodes + (size_t)g * t.node_cap;
+    Edge *ne = new_edges + (size_t)g * t.edge_cap;
+    unsigned char *np = new_pos + (size_t)g * t.node_cap * t.stride;
+    int *remap = remap_all + (size_t)g * t.node_cap;
+    GameState *gs = t.games + g;
+    const Node root = nodes[0];
+    const int want = actions ? actions[g] : -2;
+    // ---- the root's edge
+    int best = -1, best_n = -1;
+    for (int i = lane; i < root.n_edges; i += 32) {
+        const Edge e = edges[root.edge_begin + i];
+        if (want == -2 ? e.n > best_n : e.action == want) { best = i; best_n = e.n; }
+    }
+#pragma unroll
+    for (int d = 16; d; d >>= 1) {
+        const int on = __shfl_xor_sync(0xffffffffu, best_n, d), ob = __shfl_xor_sync(0xffffffffu, best, d);
+        if (ob >= 0 && (best < 0 || on > best_n || (on == best_n && ob < best))) { best = ob; best_n = on; }
+    }
+    const int words = t.stride / 8;
+    if (best < 0 || want == -1) {
+        // nothing is played: the tree moves to the other pools as it is
+        if (lane == 0) {
+            played[g] = -1;
+            if (want >= 0) gs->flags |= AZ_SEARCH_FLAG_BAD_ACTION;
+        }
+        const int n_nodes = gs->n_nodes, n_edges = gs->n_edges;
+        for (int i = lane; i < n_nodes; i += 32) nn[i] = nodes[i];
+        for (int i = lane; i < n_edges; i += 32) ne[i] = edges[i];
+        const u64 *src = reinterpret_cast<const u64 *>(npos);
+        u64 *dst = reinterpret_cast<u64 *>(np);
+        for (size_t i = lane; i < (size_t)n_nodes * words; i += 32) dst[i] = src[i];
+        return;
+    }
+    const Edge e0 = edges[root.edge_begin + best];
+    if (lane == 0) played[g] = e0.action;
+    if (e0.child < 0) {
+        apply_action_warp(npos, np, t.stride, t.head, e0.action, lane);
+        if (lane == 0) {
+            Node fresh{};
+            fresh.n_edges = -1;
+            nn[0] = fresh;
+            gs->n_nodes = 1; gs->n_edges = 0; gs->root_submitted = 0;
+            atomicOr(any_fresh, 1);
+        }
+        return;
+    }
+    // ---- breadth-first copy: new node i was old node remap[i]
+    if (lane == 0) remap[0] = e0.child;
+    __syncwarp();
+    int n_new = 1, e_new = 0;
+    for (int i = 0; i < n_new; ++i) {
+        const int o = remap[i];
+        Node nd = nodes[o];
+        const u64 *src = reinterpret_cast<const u64 *>(npos + (size_t)o * t.stride);
+        u64 *dst = reinterpret_cast<u64 *>(np + (size_t)i * t.stride);
+        for (int k = lane; k < words; k += 32) dst[k] = src[k];
+        const int begin = nd.edge_begin, cnt = nd.n_edges > 0 ? nd.n_edges : 0;
+        for (int base = 0; base < cnt; base += 32) {
+            const int j = base + lane;
+            Edge e{};
+            bool has = false;
+            if (j < cnt) { e = edges[begin + j]; has = e.child >= 0; }
+            const unsigned m = __ballot_sync(0xffffffffu, has);
+            if (has) {
+                const int id = n_new + __popc(m & ((1u << lane) - 1u));
+                remap[id] = e.child;
+                e.child = id;
+            }
+            if (j < cnt) ne[e_new + j] = e;
+            n_new += __popc(m);
+        }
+        if (lane == 0) { nd.edge_begin = e_new; nn[i] = nd; }
+        e_new += cnt;
+        __syncwarp();
+    }
+    if (lane == 0) { gs->n_nodes = n_new; gs->n_edges = e_new; }
+}
+
 // root actions and visit counts of every game, in rows of AZ_MAX_LEGAL
 __global__ void gather_roots_kernel(Trees t, int games, int *__restrict__ actions, int *__restrict__ visits, int *__restrict__ counts) {
     const int g = blockIdx.x;
@@ -539,10 +645,10 @@ __global__ void gather_roots_kernel(Trees t, int games, int *__restrict__ action
 
 // one step of one group: four launches (five with the paper's network or a tensor-core net: their
 // evaluation is two or three kernels)
-int queue_step(Search &s, int gi) {
+int queue_step(Search &s, int gi, bool root_step) {
     Group &g = s.groups[gi];
     const unsigned blocks = (unsigned)((g.n_games + kWarps - 1) / kWarps);
-    search_select_kernel<<<blocks, 32 * kWarps, 0, g.stream>>>(s.trees, g.batch, g.game0, g.n_games);
+    search_select_kernel<<<blocks, 32 * kWarps, 0, g.stream>>>(s.trees, g.batch, g.game0, g.n_games, root_step ? 1 : 0);
     AZ_LAUNCH_CHECK();
     int rc = launch_legal_masks(g.batch.pos, (size_t)s.trees.stride, g.rows, s.trees.head, g.masks, g.stream);
     if (rc != AZ_OK) return rc;
@@ -703,6 +809,7 @@ int az_search_set_roots(az_search *search, const void *positions_host) {
                                       (size_t)g.n_games, cudaMemcpyDeviceToDevice, st));
     }
     AZ_CUDA(cudaStreamSynchronize(st));
+    s->need_root_step = true;
     return AZ_OK;
 }
 
@@ -713,13 +820,11 @@ int az_search_run(az_search *search, int simulations, float *elapsed_ms_out) {
     cudaStream_t s1 = s->n_groups == 2 ? s->groups[1].stream : s0;
     AZ_CUDA(cudaEventRecord(s->ev_begin, s0));
     if (s1 != s0) AZ_CUDA(cudaStreamWaitEvent(s1, s->ev_begin, 0));
-    // a tree whose root has not been evaluated spends its first step on that; give every tree that step
-    az::GameState first{};
-    AZ_CUDA(cudaMemcpy(&first, s->trees.games, sizeof first, cudaMemcpyDeviceToHost));
-    const int steps = simulations + (first.root_submitted ? 0 : 1);
+    // a tree whose root has not been evaluated spends a step on that; the other trees sit that step out
+    const int steps = simulations + (s->need_root_step ? 1 : 0);
     for (int step = 0; step < steps; ++step)
         for (int gi = 0; gi < s->n_groups; ++gi) {
-            const int rc = az::queue_step(*s, gi);
+            const int rc = az::queue_step(*s, gi, s->need_root_step && step == 0);
             if (rc != AZ_OK) return rc;
         }
     if (s1 != s0) {
@@ -727,6 +832,7 @@ int az_search_run(az_search *search, int simulations, float *elapsed_ms_out) {
         AZ_CUDA(cudaStreamWaitEvent(s0, s->groups[1].done, 0));
     }
     AZ_CUDA(cudaEventRecord(s->ev_end, s0));
+    s->need_root_step = false;
     AZ_CUDA(cudaEventSynchronize(s->ev_end));
     if (elapsed_ms_out) AZ_CUDA(cudaEventElapsedTime(elapsed_ms_out, s->ev_begin, s->ev_end));
     if (s->net) {
@@ -764,6 +870,46 @@ int az_search_root_visits(az_search *search, int32_t *actions_host, int32_t *vis
     AZ_CUDA(cudaMemcpyAsync(actions_host, s->out_actions, G * AZ_MAX_LEGAL * sizeof(int), cudaMemcpyDeviceToHost, st));
     AZ_CUDA(cudaMemcpyAsync(visits_host, s->out_visits, G * AZ_MAX_LEGAL * sizeof(int), cudaMemcpyDeviceToHost, st));
     AZ_CUDA(cudaStreamSynchronize(st));
+    return AZ_OK;
+}
+
+int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *played_host) {
+    Search *s = reinterpret_cast<Search *>(search);
+    if (!s) return AZ_ERR_BAD_ARG;
+    az::Trees &t = s->trees;
+    const size_t G = s->cfg.games;
+    cudaStream_t st = s->groups[0].stream;
+    if (!s->alt_nodes) {
+        AZ_CUDA(cudaMalloc((void **)&s->alt_nodes, G * t.node_cap * sizeof(az::Node)));
+        AZ_CUDA(cudaMalloc((void **)&s->alt_edges, G * t.edge_cap * sizeof(az::Edge)));
+        AZ_CUDA(cudaMalloc((void **)&s->alt_node_pos, G * t.node_cap * (size_t)t.stride));
+        AZ_CUDA(cudaMalloc((void **)&s->remap, G * t.node_cap * sizeof(int)));
+        AZ_CUDA(cudaMalloc((void **)&s->adv_actions, G * sizeof(int)));
+        AZ_CUDA(cudaMalloc((void **)&s->adv_played, G * sizeof(int)));
+        AZ_CUDA(cudaMalloc((void **)&s->adv_fresh, sizeof(int)));
+    }
+    if (actions_host) AZ_CUDA(cudaMemcpyAsync(s->adv_actions, actions_host, G * sizeof(int), cudaMemcpyHostToDevice, st));
+    AZ_CUDA(cudaMemsetAsync(s->adv_fresh, 0, sizeof(int), st));
+    az::search_advance_kernel<<<(unsigned)((G + az::kWarps - 1) / az::kWarps), 32 * az::kWarps, 0, st>>>(
+        t, s->alt_nodes, s->alt_edges, s->alt_node_pos, (int)G, actions_host ? s->adv_actions : nullptr, s->adv_played, s->remap, s->adv_fresh);
+    AZ_LAUNCH_CHECK();
+    int fresh = 0;
+    if (played_host) AZ_CUDA(cudaMemcpyAsync(played_host, s->adv_played, G * sizeof(int), cudaMemcpyDeviceToHost, st));
+    AZ_CUDA(cudaMemcpyAsync(&fresh, s->adv_fresh, sizeof(int), cudaMemcpyDeviceToHost, st));
+    AZ_CUDA(cudaStreamSynchronize(st));
+    std::swap(t.nodes, s->alt_nodes);
+    std::swap(t.edges, s->alt_edges);
+    std::swap(t.node_pos, s->alt_node_pos);
+    if (fresh) s->need_root_step = true;
+    return AZ_OK;
+}
+
+int az_search_root_positions(az_search *search, void *positions_host) {
+    Search *s = reinterpret_cast<Search *>(search);
+    if (!s || !positions_host) return AZ_ERR_BAD_ARG;
+    const az::Trees &t = s->trees;
+    AZ_CUDA(cudaMemcpy2D(positions_host, (size_t)t.stride, t.node_pos, (size_t)t.node_cap * t.stride, (size_t)t.stride,
+                         (size_t)s->cfg.games, cudaMemcpyDeviceToHost));
     return AZ_OK;
 }
 

@@ -182,6 +182,99 @@ def test_root_visits_of_all_games_in_one_copy():
     az.az_search_destroy(s)
 
 
+def read_gpu_tree(az, s, g):
+    a, n, w, p = az.az_search_root(s, g)
+    counts, nvis, wsum = az.az_search_tree(s, g)
+    return a, n, w, p, counts, nvis, wsum
+
+
+def same_tree(got, want, where):
+    a, n, w, p, counts, nvis, wsum = got
+    assert (a == want["actions"]).all() and (n == want["visits"]).all(), where
+    assert (w.view(np.uint32) == want["w"].view(np.uint32)).all() and (p.view(np.uint32) == want["prior"].view(np.uint32)).all(), where
+    assert tuple(counts) == (want["n_nodes"], want["n_edges"], want["flags"], want["idle"]), (where, counts, want["n_nodes"], want["n_edges"])
+    assert (nvis == want["node_nvis"]).all() and (wsum.view(np.uint32) == want["node_wsum"].view(np.uint32)).all(), where
+
+
+@pytest.mark.parametrize("head,stride,leaves", [(2, 128, 1), (1, 784, 3)])
+def test_games_played_by_the_search_keep_their_subtrees_like_the_oracles(head, stride, leaves):
+    """Every game plays its most visited move after each search; trees, positions and moves equal the oracle's
+    at every ply (stand-in evaluator on both sides)."""
+    import paper_2609_37447_b200 as az
+    rec = records(head, stride, 21, 20261001)
+    n, sims, cap = rec.shape[0], 50, 50 * leaves * 14 + 2
+    s = az.az_search_create(None, az.make_search_config(n, head, stride, leaves=leaves, groups=2, max_nodes=cap, max_edges=cap * 48,
+                                                        evaluator=az.AZ_SEARCH_EVAL_STANDIN, seed=13))
+    az.az_search_set_roots(s, rec)
+    trees = [oracle.MctsTree(rec[g:g + 1], head, leaves=leaves, seed=13, node_cap=cap, edge_cap=cap * 48) for g in range(n)]
+    moved = 0
+    for ply in range(12):
+        az.az_search_run(s, sims)
+        want_play = []
+        for g in range(n):
+            trees[g].run(sims)
+            want = trees[g].read()
+            same_tree(read_gpu_tree(az, s, g), want, f"ply {ply} game {g}")
+            want_play.append(int(want["actions"][int(np.argmax(want["visits"]))]) if len(want["actions"]) else -1)
+        played = az.az_search_advance(s)
+        assert (played == np.array(want_play)).all()
+        roots = az.az_search_root_positions(s, rec.dtype)
+        for g in range(n):
+            if want_play[g] >= 0:
+                trees[g].advance(want_play[g])
+                moved += 1
+            want = trees[g].read()
+            assert (roots[g:g + 1].view(np.uint8) == want["root"].view(np.uint8)).all(), f"ply {ply} game {g}"
+            same_tree(read_gpu_tree(az, s, g), want, f"after the move of ply {ply}, game {g}")
+    assert moved > 10 * (n - 3)
+    az.az_search_destroy(s)
+    for t in trees:
+        t.close()
+
+
+def test_given_moves_none_unvisited_and_impossible_ones():
+    import paper_2609_37447_b200 as az
+    rec = records(2, 128, 12, 20261002)
+    n = rec.shape[0]
+    s = az.az_search_create(None, az.make_search_config(n, 2, 128, leaves=1, groups=1, max_nodes=400, evaluator=az.AZ_SEARCH_EVAL_STANDIN, seed=21))
+    az.az_search_set_roots(s, rec)
+    trees = [oracle.MctsTree(rec[g:g + 1], 2, seed=21, node_cap=400, edge_cap=400 * 64) for g in range(n)]
+    az.az_search_run(s, 12)
+    actions = np.full(n, -1, dtype=np.int32)
+    for g in range(n):
+        trees[g].run(12)
+        r = trees[g].read()
+        if len(r["actions"]) == 0:
+            continue
+        if g % 3 == 0:                                           # a move the search never tried: a fresh tree
+            actions[g] = int(r["actions"][np.flatnonzero(r["visits"] == 0)[0]])
+        elif g % 3 == 1:                                         # the least visited of the tried moves
+            tried = np.flatnonzero(r["visits"] > 0)
+            actions[g] = int(r["actions"][tried[np.argmin(r["visits"][tried])]])
+    bad = 9
+    actions[bad] = 1879 if not (trees[bad].read()["actions"] == 1879).any() else 1878      # not a move of that root
+    played = az.az_search_advance(s, actions)
+    for g in range(n):
+        if g == bad:
+            assert played[g] == -1 and az.az_search_tree(s, g, nodes=False)[0][2] & az.AZ_SEARCH_FLAG_BAD_ACTION
+            continue
+        assert played[g] == actions[g]
+        if actions[g] >= 0:
+            trees[g].advance(int(actions[g]))
+    # the next run: fresh trees evaluate their roots in a step of their own while the others sit it out
+    az.az_search_run(s, 40)
+    for g in range(n):
+        trees[g].run(40)
+        got = read_gpu_tree(az, s, g)
+        want = trees[g].read()
+        if g == bad:
+            want["flags"] |= az.AZ_SEARCH_FLAG_BAD_ACTION
+        same_tree(got, want, f"game {g}")
+    az.az_search_destroy(s)
+    for t in trees:
+        t.close()
+
+
 def test_search_with_the_network_as_evaluator():
     import paper_2609_37447_b200 as az
     cfg = pw.PNetConfig("ts", 2, 128, 64, 20260998, 4500)
