@@ -311,6 +311,36 @@ def run_search(args, name):
     az.az_search_destroy(s)
     status = az.az_device_status(net)
 
+    # ---- optional: games in progress.  Every game plays its most visited move after each K-step search and keeps
+    # the subtree under it (Sec. 3.3); wall clock over all moves, moves read back to the host
+    play = None
+    if args.moves > 0:
+        nodes_play = 6 * args.steps * leaves + 2
+        sc = az.make_search_config(games, 2, 128, leaves=leaves, groups=2, max_nodes=nodes_play, max_edges=48 * nodes_play)
+        s = az.az_search_create(net, sc)
+        az.az_search_set_roots(s, recs)
+        az.az_search_run(s, args.steps)
+        az.az_search_advance(s)
+        barrier()
+        t0 = time.perf_counter()
+        run_ms, moved = 0.0, 0
+        for _ in range(args.moves):
+            run_ms += az.az_search_run(s, args.steps)
+            moved += int((az.az_search_advance(s) >= 0).sum())
+        play_s = time.perf_counter() - t0
+        barrier()
+        flags_play, kept = 0, []
+        for g in range(0, games, max(1, games // 32)):
+            c = az.az_search_tree(s, g, nodes=False)[0]
+            flags_play |= int(c[2])
+            kept.append(int(c[0]))
+        az.az_search_destroy(s)
+        play = {"moves_per_game": args.moves, "moves_played": moved, "searches_per_s": games * leaves * args.steps * args.moves / play_s,
+                "moves_per_s": moved / play_s, "ms_per_move_all_games": 1e3 * play_s / args.moves,
+                "ms_in_search_per_move": run_ms / args.moves, "tree_flags": flags_play,
+                "kept_nodes_median": float(np.median(kept)),
+                "note": "wall clock over az_search_run + az_search_advance per move; every traversal of a step counted"}
+
     ms_max, e2e_ms = sharding.max_over_ranks([ms, e2e_s * 1e3], device="cuda")
     if rank == 0:
         peaks = load_peaks()
@@ -344,6 +374,8 @@ def run_search(args, name):
                          "avg_launch_ms_overlapped": tower_ms / max(tower_passes, 1), "launches_timed": tower_passes,
                          "flops_per_launch": flops},
         }
+        if play is not None:
+            out["games_in_progress"] = play
         if not args.no_cpu_baseline:
             rate, dt = oracle_search_rate(recs, 8000, 128)
             out["cpu_baseline"] = {"value": rate, "unit": SEARCH_UNIT, "cores": 1, "kind": "oracle",
@@ -365,6 +397,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures on a smaller case)")
     ap.add_argument("--leaves", type=int, default=1, help="search workloads: traversals per tree and step")
+    ap.add_argument("--moves", type=int, default=0, help="search workloads: also time this many played moves per game, each after "
+                                                         "a search of --steps steps (subtrees kept)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
