@@ -28,6 +28,11 @@
  *    (Q + ((c * P) * sqrt(max(1, N))) / (1 + n)), ties to the lower action index;
  *  - with a network whose value head is (win, draw, loss) the scalar is win - loss (Sec. 3.3).
  *
+ * Rows of a step that have nothing to evaluate (a traversal that ended in a known terminal node or was
+ * given up) are evaluated all the same (the batch keeps its shape) and their results ignored; leaves
+ * without a legal move go through the evaluator too, so the az_net's "a position had no legal move"
+ * status bit (az_device_status bit 0) may be set by a search and means nothing there.
+ *
  * Threading: one az_search is used by one host thread at a time; it uses the az_net's evaluation
  * workspace, so no other evaluation of that az_net may run during az_search_run.
  */
