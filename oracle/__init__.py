@@ -81,6 +81,8 @@ def _load():
         lib.orc_mcts_advance.argtypes = [vp, ci]
         lib.orc_mcts_read.restype = ci
         lib.orc_mcts_read.argtypes = [vp] * 9
+        lib.orc_mcts_node.restype = ci
+        lib.orc_mcts_node.argtypes = [vp, ci, vp, vp]
         lib.orc_mcts_free.restype = None
         lib.orc_mcts_free.argtypes = [vp]
         lib.orc_pnet_forward.restype = ci
@@ -230,6 +232,14 @@ class MctsTree:
         return {"actions": actions[:k].copy(), "visits": visits[:k].copy(), "w": w[:k].copy(), "prior": prior[:k].copy(),
                 "n_nodes": int(counts[0]), "n_edges": int(counts[1]), "flags": int(counts[2]), "idle": int(counts[3]),
                 "node_nvis": nvis[:counts[0]].copy(), "node_wsum": wsum[:counts[0]].copy(), "root": root}
+
+    def node(self, index: int):
+        """(record, parent index) of one node, for inspection."""
+        rec = np.zeros(1, dtype=self.dtype)
+        parent = np.zeros(1, dtype=np.int32)
+        if _load().orc_mcts_node(self.handle, index, rec.ctypes.data, parent.ctypes.data) != 0:
+            raise IndexError(index)
+        return rec, int(parent[0])
 
     def close(self):
         if self.handle:

@@ -11,8 +11,14 @@
  *  - a reservation (parallel leaves) counts on its edges as one visit that lost: N + m visits,
  *    W - m value; it is removed when the traversal's result arrives.  A traversal that runs into a
  *    node still waiting for its evaluation is given up (its reservations are removed, its slot idles);
- *  - a node is terminal if the mover has no legal move (value -1 in check, else 0) or the halfmove
- *    clock has reached 100 (value 0); repetitions are not tracked inside the tree;
+ *  - a new node's repetition count (the record's `repetitions` field, which the input planes show) is one
+ *    more than that of the most recent earlier occurrence of the same position (pieces, side to move,
+ *    castling rights, en-passant square) among its ancestors in the tree and the positions of the game
+ *    before the root, as far back as its halfmove clock reaches; 0 if there is none.  The game's earlier
+ *    positions are those the tree itself has seen as roots (played moves); the first root brings its own
+ *    count in its record;
+ *  - a node is terminal if the mover has no legal move (value -1 in check, else 0), if the halfmove
+ *    clock has reached 100 or if the position has occurred twice before (value 0);
  *  - the root's evaluation is a step of its own before the counted simulations;
  *  - when a move is played (Sec. 3.3: the relevant subtree becomes the next root) the subtree under the
  *    root's edge of that action is kept with all its statistics and renumbered breadth-first (a node's
@@ -47,8 +53,10 @@ typedef struct {
     int terminal; float tvalue;
     int nvis; float wsum;         /* values backed up through the node, its own first */
     int nsum;                     /* sum over edges of N + m */
+    int parent;                   /* -1 for the root */
     unsigned char rec[MAX_STRIDE];
 } Node;
+#define MAX_HISTORY 128
 
 static uint64_t mix64(uint64_t x) {
     x ^= x >> 30; x *= 0xbf58476d1ce4e5b9ULL;
@@ -97,7 +105,27 @@ typedef struct {
     uint64_t seed;
     uint32_t flags;               /* 1: node pool full, 2: edge pool full, 4: depth limit */
     int root_submitted, idle;     /* idle: traversals given up (collisions, full pools) */
+    Cur hist[MAX_HISTORY];        /* the game's positions before the root since the last irreversible move, oldest first */
+    int hist_n;
 } Tree;
+
+static int same_position(const Cur *a, const Cur *b) {
+    return memcmp(a->pieces, b->pieces, sizeof a->pieces) == 0 && a->stm == b->stm && a->castling == b->castling &&
+           a->ep_square == b->ep_square;
+}
+
+/* Repetition count of position `c`, reached from node `parent`: one more than the count of its most recent earlier
+ * occurrence within the last c->halfmove plies (ancestors first, then the game before the root), 0 without one. */
+static int repetition_count(const Tree *t, int parent, const Cur *c) {
+    int k = 1;
+    for (int n = parent; n >= 0 && k <= c->halfmove; n = t->nodes[n].parent, ++k) {
+        const Cur *p = (const Cur *)t->nodes[n].rec;
+        if (same_position(p, c)) return p->repetitions < 255 ? p->repetitions + 1 : 255;
+    }
+    for (int i = t->hist_n - 1; i >= 0 && k <= c->halfmove; --i, ++k)
+        if (same_position(&t->hist[i], c)) return t->hist[i].repetitions < 255 ? t->hist[i].repetitions + 1 : 255;
+    return 0;
+}
 
 typedef struct { int kind, leaf, depth; int path_e[MAX_DEPTH], path_n[MAX_DEPTH]; } Slot;
 enum { SLOT_NONE = 0, SLOT_EVAL = 1, SLOT_TERMINAL = 2 };
@@ -144,6 +172,8 @@ static void descend(Tree *t, Slot *s) {
             c->n_edges = -1;
             int32_t a = e->action;
             orc_apply_moves(nd->rec, t->stride, 1, t->head, &a, c->rec);
+            c->parent = node;
+            ((Cur *)c->rec)->repetitions = (uint8_t)repetition_count(t, node, (const Cur *)c->rec);
             e->child = child;
             s->kind = SLOT_EVAL; s->leaf = child;
             return;
@@ -162,7 +192,7 @@ static void finish(Tree *t, Slot *s) {
         const Cur *c = (const Cur *)nd->rec;
         nd->nsum = 0;
         if (k == 0) { nd->terminal = 1; nd->tvalue = orc_in_check(nd->rec) ? -1.0f : 0.0f; nd->n_edges = 0; }
-        else if (c->halfmove >= 100) { nd->terminal = 1; nd->tvalue = 0.0f; nd->n_edges = 0; }
+        else if (c->halfmove >= 100 || c->repetitions >= 2) { nd->terminal = 1; nd->tvalue = 0.0f; nd->n_edges = 0; }
         else if (t->n_edges + k > t->edge_cap) { t->flags |= 2; nd->terminal = 1; nd->tvalue = value; nd->n_edges = 0; }
         else {
             nd->edge_begin = t->n_edges; nd->n_edges = k; t->n_edges += k;
@@ -194,6 +224,7 @@ static Tree *tree_new(const void *root_record, int stride, int head, float c_puc
     t->c_puct = c_puct; t->fpu_reduction = fpu_reduction; t->discount = discount; t->seed = seed;
     memcpy(t->nodes[0].rec, root_record, (size_t)stride);
     t->nodes[0].n_edges = -1;
+    t->nodes[0].parent = -1;
     t->n_nodes = 1;
     return t;
 }
@@ -221,22 +252,32 @@ static int tree_advance(Tree *t, int action) {
     if (t->edges[e0].child < 0) {
         int32_t a = action;
         orc_apply_moves(root->rec, t->stride, 1, t->head, &a, nodes[0].rec);
+        ((Cur *)nodes[0].rec)->repetitions = (uint8_t)repetition_count(t, 0, (const Cur *)nodes[0].rec);
         nodes[0].n_edges = -1;
+        nodes[0].parent = -1;
         t->root_submitted = 0;
     } else {
         int *old_of = (int *)calloc((size_t)t->node_cap, sizeof(int));
         old_of[0] = t->edges[e0].child;
         for (int i = 0; i < n_nodes; ++i) {                           /* breadth-first: new node i was old node old_of[i] */
+            const int new_parent = nodes[i].parent;                   /* set when the node was queued */
             nodes[i] = t->nodes[old_of[i]];
+            nodes[i].parent = i == 0 ? -1 : new_parent;
             const int begin = nodes[i].edge_begin;
             nodes[i].edge_begin = n_edges;
             for (int j = 0; j < nodes[i].n_edges; ++j) {
                 Edge e = t->edges[begin + j];
-                if (e.child >= 0) { old_of[n_nodes] = e.child; e.child = n_nodes++; }
+                if (e.child >= 0) { old_of[n_nodes] = e.child; nodes[n_nodes].parent = i; e.child = n_nodes++; }
                 edges[n_edges++] = e;
             }
         }
         free(old_of);
+    }
+    /* the old root joins the game's earlier positions, unless the move was irreversible (then nothing before it can recur) */
+    if (((const Cur *)nodes[0].rec)->halfmove == 0) t->hist_n = 0;
+    else {
+        if (t->hist_n == MAX_HISTORY) { memmove(t->hist, t->hist + 1, sizeof(Cur) * (MAX_HISTORY - 1)); t->hist_n -= 1; }
+        memcpy(&t->hist[t->hist_n++], root->rec, sizeof(Cur));
     }
     free(t->nodes); free(t->edges);
     t->nodes = nodes; t->edges = edges; t->n_nodes = n_nodes; t->n_edges = n_edges;
@@ -273,6 +314,14 @@ int orc_mcts_advance(void *tree, int action) { return tree ? tree_advance((Tree 
 int orc_mcts_read(const void *tree, int32_t *root_actions, int32_t *root_visits, float *root_w, float *root_prior,
                   int32_t *counts, int32_t *node_nvis, float *node_wsum, void *root_record) {
     return tree_read((const Tree *)tree, root_actions, root_visits, root_w, root_prior, counts, node_nvis, node_wsum, root_record);
+}
+/* One node, for inspection: its record and its parent's index (-1 for the root).  Returns 0, -1 if there is no such node. */
+int orc_mcts_node(const void *tree, int index, void *record_out, int32_t *parent_out) {
+    const Tree *t = (const Tree *)tree;
+    if (!t || index < 0 || index >= t->n_nodes) return -1;
+    memcpy(record_out, t->nodes[index].rec, (size_t)t->stride);
+    *parent_out = t->nodes[index].parent;
+    return 0;
 }
 void orc_mcts_free(void *tree) {
     Tree *t = (Tree *)tree;

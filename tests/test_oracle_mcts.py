@@ -193,3 +193,61 @@ def test_a_game_played_by_the_search_follows_the_rules():
         assert (t.read()["root"].view(np.uint8) == cur.view(np.uint8)).all()
     assert ply >= 10
     t.close()
+
+
+def same_position(a, b):
+    return (a["pieces"] == b["pieces"]).all() and a["stm"] == b["stm"] and a["castling"] == b["castling"] and a["ep_square"] == b["ep_square"]
+
+
+def test_repetitions_across_played_moves():
+    # the knights go out and come back, twice: the start position has then occurred twice before
+    rec = positions.record_from_fen(START)
+    shuffle = [("g1", "f3", 0), ("g8", "f6", 1), ("f3", "g1", 0), ("f6", "g8", 1)]
+    # counts along the way: first round 0 0 0 1 (the start position again), second round 1 1 1 2
+    t2 = oracle.MctsTree(rec, 2, seed=1, node_cap=200)
+    seen = []
+    for rnd in range(2):
+        for frm, to, stm in shuffle:
+            t2.run(0)                                                  # the root's own evaluation: it learns its moves
+            t2.advance(oracle.policy_index(2, stm, sq(frm), sq(to)))
+            seen.append(int(t2.read()["root"]["repetitions"][0]))
+    assert seen == [0, 0, 0, 1, 1, 1, 1, 2]
+    # a position that has occurred twice before is a draw: its evaluation finds no moves to search
+    t2.run(5)
+    r = t2.read()
+    assert len(r["actions"]) == 0 and r["n_nodes"] == 1 and r["node_wsum"][0] == 0
+    # a pawn move in between cuts the history off
+    t3 = oracle.MctsTree(rec, 2, seed=1, node_cap=200)
+    for frm, to, stm in shuffle[:2] + [("e2", "e4", 0), ("f6", "g8", 1), ("f3", "g1", 0)]:
+        t3.run(0)
+        t3.advance(oracle.policy_index(2, stm, sq(frm), sq(to)))
+    assert int(t3.read()["root"]["repetitions"][0]) == 0
+    for tr in (t2, t3):
+        tr.close()
+
+
+def test_repetition_counts_inside_a_tree_against_a_brute_force_walk():
+    # few pieces: paths that return to an earlier position are common within a few plies
+    repeated = 0
+    for fen, seed in (("8/8/8/4k3/8/8/3QK3/8 w - - 10 40", 3), ("8/8/8/8/8/5k2/8/4K2R b - - 20 60", 5), ("8/8/8/4k3/8/8/3QK3/8 w - - 10 40", 9)):
+        rec = positions.record_from_fen(fen)
+        t = oracle.MctsTree(rec, 2, seed=seed, node_cap=3001)
+        t.run(3000)
+        n = t.read()["n_nodes"]
+        nodes = [t.node(i) for i in range(n)]
+        parents_with_children = {p for _, p in nodes}
+        for i, (r, parent) in enumerate(nodes):
+            cur = r[0]
+            want, k, p = 0, 1, parent
+            while p >= 0 and k <= int(cur["halfmove"]):
+                pr = nodes[p][0][0]
+                if same_position(pr, cur):
+                    want = int(pr["repetitions"]) + 1
+                    break
+                p, k = nodes[p][1], k + 1
+            assert int(cur["repetitions"]) == want, i
+            repeated += want >= 1
+            if want >= 2:
+                assert i not in parents_with_children                     # a drawn node is never expanded
+        t.close()
+    assert repeated >= 10
