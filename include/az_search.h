@@ -21,8 +21,14 @@
  *  - a reservation (a traversal whose result is still outstanding; `leaves` > 1) counts on its
  *    edges as one lost visit: N + m visits, W - m value; a traversal that reaches a node still
  *    waiting for its evaluation is given up and its batch row idles;
- *  - a node is terminal if the mover has no legal move (value -1 in check, else 0) or its
- *    halfmove clock has reached 100 (value 0); repetitions are not tracked inside a tree;
+ *  - a new node's repetition count (the `repetitions` field of its record, which the input planes
+ *    show) is one more than that of the most recent earlier occurrence of the same position (pieces,
+ *    side to move, castling rights, en-passant square; compared through a 64-bit hash) among its
+ *    ancestors in the tree and the game's positions before the root, as far back as its halfmove
+ *    clock reaches; 0 without one.  The game's earlier positions are the roots the search has seen
+ *    (az_search_advance); the first root brings its own count in its record;
+ *  - a node is terminal if the mover has no legal move (value -1 in check, else 0), if its
+ *    halfmove clock has reached 100 or if its position has occurred twice before (value 0);
  *  - the root's evaluation is a step of its own, queued by az_search_set_roots' first run;
  *  - the arg-max of Eq. 1 is taken in float32 with one rounding per operation
  *    (Q + ((c * P) * sqrt(max(1, N))) / (1 + n)), ties to the lower action index;

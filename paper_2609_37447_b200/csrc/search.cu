@@ -35,7 +35,9 @@ struct alignas(16) Node {                        // 32 bytes
     int nsum;                                    // sum over the edges of N + m
     int pad;
 };
-struct GameState { int n_nodes, n_edges, flags, idle, root_submitted, pad[3]; };
+struct GameState { int n_nodes, n_edges, flags, idle, root_submitted, hist_n, pad[2]; };
+constexpr int kMaxHistory = 128;                 // earlier positions of a game kept for the repetition test
+constexpr int kRepByte = 100;                    // offset of `repetitions` in a position record
 
 // inverse of the from-to numbering: pair number -> origin | destination << 6 (mover's orientation);
 // promotion combination -> origin file | destination file << 3
@@ -186,6 +188,29 @@ __device__ u64 position_key(const u64 *rec, u64 seed) {
     return mix64(h ^ (tail & 0xffffffull));                        // side to move | castling << 8 | en-passant square << 16
 }
 
+// Positions are compared through this hash (pieces, side to move, castling rights, en-passant square).
+constexpr u64 kRepSeed = 0x243f6a8885a308d3ull;
+
+// Repetition count of a position with hash h and halfmove clock `halfmove` that is reached from the path
+// pn[0 .. depth-1] (root first): one more than the count of its most recent earlier occurrence within the last
+// `halfmove` plies, ancestors first, then the game's positions before the root; 0 without one.  All lanes call
+// and get the same answer.
+__device__ int repetition_count_warp(const u64 *__restrict__ node_hash, const unsigned char *__restrict__ npos, int stride,
+                                     const int *pn, int depth, const u64 *__restrict__ hist_hash,
+                                     const unsigned char *__restrict__ hist_rep, int hist_n, u64 h, int halfmove, int lane) {
+    const int reach = min(halfmove, depth + hist_n);
+    int best_k = 0x7fffffff;
+    for (int k = lane + 1; k <= reach; k += 32) {
+        const u64 c = k <= depth ? node_hash[pn[depth - k]] : hist_hash[hist_n - (k - depth)];
+        if (c == h) { best_k = k; break; }
+    }
+#pragma unroll
+    for (int d = 16; d; d >>= 1) best_k = min(best_k, __shfl_xor_sync(0xffffffffu, best_k, d));
+    if (best_k == 0x7fffffff) return 0;
+    const int before = best_k <= depth ? npos[(size_t)pn[depth - best_k] * stride + kRepByte] : hist_rep[hist_n - (best_k - depth)];
+    return before < 255 ? before + 1 : 255;
+}
+
 // The set bits of a mask row in ascending order, dealt over the warp: lane L owns words L, L + 32, L + 64.
 // Calls f(action, rank) for every set bit, rank = the number of set bits before it; returns the total.
 template <typename F>
@@ -241,6 +266,8 @@ standin_eval_kernel(const unsigned char *__restrict__ positions, int stride, con
 // ---- the trees ------------------------------------------------------------------------------------
 struct Trees {
     Node *nodes; Edge *edges; unsigned char *node_pos; GameState *games;
+    u64 *node_hash;                              // [games][node_cap]: position hash of every node (repetition test)
+    u64 *hist_hash; unsigned char *hist_rep;     // [games][kMaxHistory]: the game's positions before the root, oldest first
     int node_cap, edge_cap, stride, head, leaves;
     float c_puct, fpu_reduction, discount;
 };
@@ -337,6 +364,17 @@ search_select_kernel(Trees t, Batch b, int game0, int n_games, int root_step) {
                     unsigned char *cpos = npos + (size_t)child * t.stride;
                     apply_action_warp(npos + (size_t)node * t.stride, cpos, t.stride, t.head, chosen.action, lane);
                     __syncwarp();
+                    {
+                        // the new position's repetition count (the input planes show it; twice before = a draw)
+                        const u64 *cw = reinterpret_cast<const u64 *>(cpos);
+                        const u64 h = position_key(cw, kRepSeed);
+                        const int halfmove = (int)((cw[12] >> 24) & 0xff);
+                        u64 *hashes = t.node_hash + (size_t)g * t.node_cap;
+                        const int reps = repetition_count_warp(hashes, npos, t.stride, pn, depth, t.hist_hash + (size_t)g * kMaxHistory,
+                                                               t.hist_rep + (size_t)g * kMaxHistory, gs->hist_n, h, halfmove, lane);
+                        if (lane == 0) { hashes[child] = h; cpos[kRepByte] = (unsigned char)reps; }
+                        __syncwarp();
+                    }
                     const u64 *src = reinterpret_cast<const u64 *>(cpos);
                     u64 *dst = reinterpret_cast<u64 *>(b.pos + (size_t)row * t.stride);
                     for (int i = lane; i < t.stride / 8; i += 32) dst[i] = src[i];
@@ -379,7 +417,7 @@ search_finish_kernel(Trees t, Batch b, int game0, int n_games, const u64 *__rest
             const int cnt = counts[row];
             const float net_v = vs == 3 ? __fsub_rn(value[(size_t)row * 3], value[(size_t)row * 3 + 2]) : value[row];
             const u64 *rec = reinterpret_cast<const u64 *>(b.pos + (size_t)row * t.stride);
-            const int halfmove = (int)((rec[12] >> 24) & 0xff);
+            const int halfmove = (int)((rec[12] >> 24) & 0xff), reps = (int)((rec[12] >> 32) & 0xff);
             Node nd = nodes[leaf];
             nd.nsum = 0; nd.n_edges = 0;
             if (cnt == 0) {
@@ -391,7 +429,7 @@ search_finish_kernel(Trees t, Batch b, int game0, int n_games, const u64 *__rest
                 const u64 king = rec[stm * 6 + 5];
                 const bool check = king && attacked(__ffsll((long long)king) - 1, stm ^ 1, opp, occ);
                 nd.terminal = 1; nd.tvalue = check ? -1.0f : 0.0f;
-            } else if (halfmove >= 100) {
+            } else if (halfmove >= 100 || reps >= 2) {
                 nd.terminal = 1; nd.tvalue = 0.0f;
             } else if (gs->n_edges + cnt > t.edge_cap) {
                 if (lane == 0) gs->flags |= AZ_SEARCH_FLAG_EDGES_FULL;
@@ -497,7 +535,7 @@ struct Search {
     int *out_actions = nullptr, *out_visits = nullptr, *out_counts = nullptr;   // read-out of all roots
     bool need_root_step = true;                  // some tree's root still waits for its evaluation
     // played moves: the kept subtrees are written to a second set of pools, which then becomes the first
-    Node *alt_nodes = nullptr; Edge *alt_edges = nullptr; unsigned char *alt_node_pos = nullptr;
+    Node *alt_nodes = nullptr; Edge *alt_edges = nullptr; unsigned char *alt_node_pos = nullptr; u64 *alt_node_hash = nullptr;
     int *remap = nullptr;                        // [games][max_nodes]: old index of every kept node
     int *adv_actions = nullptr, *adv_played = nullptr, *adv_fresh = nullptr;
 };
@@ -505,6 +543,7 @@ struct Search {
 void free_search(Search *s) {
     if (!s) return;
     cudaFree(s->trees.nodes); cudaFree(s->trees.edges); cudaFree(s->trees.node_pos); cudaFree(s->trees.games);
+    cudaFree(s->trees.node_hash); cudaFree(s->trees.hist_hash); cudaFree(s->trees.hist_rep); cudaFree(s->alt_node_hash);
     cudaFree(s->roots_stage);
     cudaFree(s->out_actions); cudaFree(s->out_visits); cudaFree(s->out_counts);
     cudaFree(s->alt_nodes); cudaFree(s->alt_edges); cudaFree(s->alt_node_pos); cudaFree(s->remap);
@@ -535,6 +574,7 @@ __global__ void reset_trees_kernel(Trees t, const unsigned char *__restrict__ ro
     const u64 *src = reinterpret_cast<const u64 *>(roots + (size_t)g * t.stride);
     u64 *dst = reinterpret_cast<u64 *>(t.node_pos + (size_t)g * t.node_cap * t.stride);
     for (int i = threadIdx.x; i < t.stride / 8; i += blockDim.x) dst[i] = src[i];
+    if (threadIdx.x == 0) t.node_hash[(size_t)g * t.node_cap] = position_key(src, kRepSeed);
 }
 
 // A move is played in every game (Sec. 3.3: the relevant subtree becomes the next root).  One warp per game:
@@ -543,7 +583,7 @@ __global__ void reset_trees_kernel(Trees t, const unsigned char *__restrict__ ro
 // without a child the new tree is the bare successor position.  actions[g] == -1, a root without edges or an
 // action the root does not have leave the game's tree as it is (copied whole); played[g] tells which it was.
 __global__ void __launch_bounds__(32 * kWarps)
-search_advance_kernel(Trees t, Node *new_nodes, Edge *new_edges, unsigned char *new_pos, int games,
+search_advance_kernel(Trees t, Node *new_nodes, Edge *new_edges, unsigned char *new_pos, u64 *new_hash, int games,
                       const int *__restrict__ actions, int *__restrict__ played, int *__restrict__ remap_all, int *any_fresh) {
     const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = blockIdx.x * kWarps + w;
@@ -556,6 +596,10 @@ search_advance_kernel(Trees t, Node *new_nodes, Edge *new_edges, unsigned char *
     unsigned char *np = new_pos + (size_t)g * t.node_cap * t.stride;
     int *remap = remap_all + (size_t)g * t.node_cap;
     GameState *gs = t.games + g;
+    const u64 *hashes = t.node_hash + (size_t)g * t.node_cap;
+    u64 *nh = new_hash + (size_t)g * t.node_cap;
+    u64 *hist_hash = t.hist_hash + (size_t)g * kMaxHistory;
+    unsigned char *hist_rep = t.hist_rep + (size_t)g * kMaxHistory;
     const Node root = nodes[0];
     const int want = actions ? actions[g] : -2;
     // ---- the root's edge
@@ -577,7 +621,7 @@ search_advance_kernel(Trees t, Node *new_nodes, Edge *new_edges, unsigned char *
             if (want >= 0) gs->flags |= AZ_SEARCH_FLAG_BAD_ACTION;
         }
         const int n_nodes = gs->n_nodes, n_edges = gs->n_edges;
-        for (int i = lane; i < n_nodes; i += 32) nn[i] = nodes[i];
+        for (int i = lane; i < n_nodes; i += 32) { nn[i] = nodes[i]; nh[i] = hashes[i]; }
         for (int i = lane; i < n_edges; i += 32) ne[i] = edges[i];
         const u64 *src = reinterpret_cast<const u64 *>(npos);
         u64 *dst = reinterpret_cast<u64 *>(np);
@@ -586,15 +630,50 @@ search_advance_kernel(Trees t, Node *new_nodes, Edge *new_edges, unsigned char *
     }
     const Edge e0 = edges[root.edge_begin + best];
     if (lane == 0) played[g] = e0.action;
+    const int hist_n = gs->hist_n;
+    const u64 old_root_hash = hashes[0];
+    const int old_root_reps = npos[kRepByte];
+    // the old root joins the game's earlier positions, unless the move is irreversible (then nothing before it can
+    // recur); called once the new root's record is in place
+    auto push_history = [&]() {
+        __syncwarp();
+        const int halfmove = (int)((reinterpret_cast<const u64 *>(np)[12] >> 24) & 0xff);
+        if (halfmove == 0) { if (lane == 0) gs->hist_n = 0; return; }
+        int n = hist_n;
+        if (n == kMaxHistory) {                                        // the oldest entry leaves
+            u64 hv[kMaxHistory / 32]; unsigned char rv[kMaxHistory / 32];
+#pragma unroll
+            for (int r = 0; r < kMaxHistory / 32; ++r) {
+                const int i = r * 32 + lane;
+                hv[r] = i + 1 < kMaxHistory ? hist_hash[i + 1] : 0ull;
+                rv[r] = i + 1 < kMaxHistory ? hist_rep[i + 1] : (unsigned char)0;
+            }
+            __syncwarp();
+#pragma unroll
+            for (int r = 0; r < kMaxHistory / 32; ++r) { hist_hash[r * 32 + lane] = hv[r]; hist_rep[r * 32 + lane] = rv[r]; }
+            __syncwarp();
+            n -= 1;
+        }
+        if (lane == 0) { hist_hash[n] = old_root_hash; hist_rep[n] = (unsigned char)old_root_reps; gs->hist_n = n + 1; }
+    };
     if (e0.child < 0) {
         apply_action_warp(npos, np, t.stride, t.head, e0.action, lane);
+        if (lane == 0) remap[0] = 0;                                   // the path to the new position: the old root alone
+        __syncwarp();
+        const u64 *cw = reinterpret_cast<const u64 *>(np);
+        const u64 h = position_key(cw, kRepSeed);
+        const int reps = repetition_count_warp(hashes, npos, t.stride, remap, 1, hist_hash, hist_rep, hist_n, h,
+                                               (int)((cw[12] >> 24) & 0xff), lane);
         if (lane == 0) {
+            np[kRepByte] = (unsigned char)reps;
+            nh[0] = h;
             Node fresh{};
             fresh.n_edges = -1;
             nn[0] = fresh;
             gs->n_nodes = 1; gs->n_edges = 0; gs->root_submitted = 0;
             atomicOr(any_fresh, 1);
         }
+        push_history();
         return;
     }
     // ---- breadth-first copy: new node i was old node remap[i]
@@ -622,11 +701,12 @@ search_advance_kernel(Trees t, Node *new_nodes, Edge *new_edges, unsigned char *
             if (j < cnt) ne[e_new + j] = e;
             n_new += __popc(m);
         }
-        if (lane == 0) { nd.edge_begin = e_new; nn[i] = nd; }
+        if (lane == 0) { nd.edge_begin = e_new; nn[i] = nd; nh[i] = hashes[o]; }
         e_new += cnt;
         __syncwarp();
     }
     if (lane == 0) { gs->n_nodes = n_new; gs->n_edges = e_new; }
+    push_history();
 }
 
 // root actions and visit counts of every game, in rows of AZ_MAX_LEGAL
@@ -750,6 +830,9 @@ int az_search_create(az_net *net, const az_search_config *c, az_search **out) {
     AZ_SEARCH_ALLOC(t.edges, G * t.edge_cap * sizeof(az::Edge));
     AZ_SEARCH_ALLOC(t.node_pos, G * t.node_cap * (size_t)t.stride);
     AZ_SEARCH_ALLOC(t.games, G * sizeof(az::GameState));
+    AZ_SEARCH_ALLOC(t.node_hash, G * t.node_cap * sizeof(az::u64));
+    AZ_SEARCH_ALLOC(t.hist_hash, G * az::kMaxHistory * sizeof(az::u64));
+    AZ_SEARCH_ALLOC(t.hist_rep, G * az::kMaxHistory);
     AZ_SEARCH_ALLOC(s->roots_stage, G * (size_t)t.stride);
     AZ_SEARCH_ALLOC(s->out_actions, G * AZ_MAX_LEGAL * sizeof(int));
     AZ_SEARCH_ALLOC(s->out_visits, G * AZ_MAX_LEGAL * sizeof(int));
@@ -883,6 +966,7 @@ int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *p
         AZ_CUDA(cudaMalloc((void **)&s->alt_nodes, G * t.node_cap * sizeof(az::Node)));
         AZ_CUDA(cudaMalloc((void **)&s->alt_edges, G * t.edge_cap * sizeof(az::Edge)));
         AZ_CUDA(cudaMalloc((void **)&s->alt_node_pos, G * t.node_cap * (size_t)t.stride));
+        AZ_CUDA(cudaMalloc((void **)&s->alt_node_hash, G * t.node_cap * sizeof(az::u64)));
         AZ_CUDA(cudaMalloc((void **)&s->remap, G * t.node_cap * sizeof(int)));
         AZ_CUDA(cudaMalloc((void **)&s->adv_actions, G * sizeof(int)));
         AZ_CUDA(cudaMalloc((void **)&s->adv_played, G * sizeof(int)));
@@ -891,7 +975,7 @@ int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *p
     if (actions_host) AZ_CUDA(cudaMemcpyAsync(s->adv_actions, actions_host, G * sizeof(int), cudaMemcpyHostToDevice, st));
     AZ_CUDA(cudaMemsetAsync(s->adv_fresh, 0, sizeof(int), st));
     az::search_advance_kernel<<<(unsigned)((G + az::kWarps - 1) / az::kWarps), 32 * az::kWarps, 0, st>>>(
-        t, s->alt_nodes, s->alt_edges, s->alt_node_pos, (int)G, actions_host ? s->adv_actions : nullptr, s->adv_played, s->remap, s->adv_fresh);
+        t, s->alt_nodes, s->alt_edges, s->alt_node_pos, s->alt_node_hash, (int)G, actions_host ? s->adv_actions : nullptr, s->adv_played, s->remap, s->adv_fresh);
     AZ_LAUNCH_CHECK();
     int fresh = 0;
     if (played_host) AZ_CUDA(cudaMemcpyAsync(played_host, s->adv_played, G * sizeof(int), cudaMemcpyDeviceToHost, st));
@@ -900,6 +984,7 @@ int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *p
     std::swap(t.nodes, s->alt_nodes);
     std::swap(t.edges, s->alt_edges);
     std::swap(t.node_pos, s->alt_node_pos);
+    std::swap(t.node_hash, s->alt_node_hash);
     if (fresh) s->need_root_step = true;
     return AZ_OK;
 }

@@ -232,6 +232,53 @@ def test_games_played_by_the_search_keep_their_subtrees_like_the_oracles(head, s
         t.close()
 
 
+def test_repetitions_inside_trees_and_across_played_moves():
+    """Endgames with few pieces, where paths return to earlier positions: repetition counts in the records, drawn
+    leaves and the history across played moves equal the oracle's (which a brute-force walk pins)."""
+    import paper_2609_37447_b200 as az
+    fens = ["8/8/8/4k3/8/8/3QK3/8 w - - 10 40", "8/8/8/8/8/5k2/8/4K2R b - - 20 60", "8/8/4k3/8/8/3K4/8/R7 w - - 30 70",
+            "8/5k2/8/8/8/8/2Q5/K7 b - - 4 50", "7k/8/8/8/8/8/R7/K7 w - - 0 1"]
+    rec, _ = positions.generate_moves(1, len(fens), (0, 2))
+    rec = rec.copy()
+    for i, fen in enumerate(fens):
+        rec[i] = np.zeros((), dtype=rec.dtype)
+        rec[i]["cur"] = positions.record_from_fen(fen)[0]
+    n, sims, cap = len(fens), 400, 2600
+    s = az.az_search_create(None, az.make_search_config(n, 2, 128, leaves=1, groups=2, max_nodes=cap, max_edges=cap * 32,
+                                                        evaluator=az.AZ_SEARCH_EVAL_STANDIN, seed=17))
+    az.az_search_set_roots(s, rec)
+    trees = [oracle.MctsTree(rec[g:g + 1], 2, seed=17, node_cap=cap, edge_cap=cap * 32) for g in range(n)]
+    repeated_nodes, repeated_roots = 0, 0
+    for ply in range(10):
+        az.az_search_run(s, sims)
+        for g in range(n):
+            trees[g].run(sims)
+            want = trees[g].read()
+            same_tree(read_gpu_tree(az, s, g), want, f"ply {ply} game {g}")
+            if ply == 0:
+                repeated_nodes += sum(int(trees[g].node(i)[0]["cur"]["repetitions"][0]) >= 1 for i in range(want["n_nodes"]))
+        # the least visited tried move: shuffles rather than progress
+        actions = np.full(n, -1, dtype=np.int32)
+        for g in range(n):
+            r = trees[g].read()
+            tried = np.flatnonzero(r["visits"] > 0)
+            if len(tried):
+                actions[g] = int(r["actions"][tried[np.argmin(r["visits"][tried])]])
+        played = az.az_search_advance(s, actions)
+        assert (played == actions).all()
+        roots = az.az_search_root_positions(s, rec.dtype)
+        for g in range(n):
+            if actions[g] >= 0:
+                trees[g].advance(int(actions[g]))
+            want = trees[g].read()
+            assert (roots[g:g + 1].view(np.uint8) == want["root"].view(np.uint8)).all(), f"ply {ply} game {g}"
+            repeated_roots += int(want["root"]["cur"]["repetitions"][0]) >= 1
+    assert repeated_nodes >= 5
+    az.az_search_destroy(s)
+    for t in trees:
+        t.close()
+
+
 def test_given_moves_none_unvisited_and_impossible_ones():
     import paper_2609_37447_b200 as az
     rec = records(2, 128, 12, 20261002)
