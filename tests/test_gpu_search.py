@@ -376,6 +376,48 @@ def test_search_with_the_network_as_evaluator():
     az.az_free_net(net)
 
 
+@pytest.mark.parametrize("in_planes,head,value_head,precision,channels", [(19, 1, 1, 1, 128), (112, 0, 0, 1, 128), (19, 0, 0, 0, 32)])
+def test_search_over_the_residual_tower_configs(in_planes, head, value_head, precision, channels):
+    """The classic networks as evaluators: tensor-core path with its second workspace (two groups side by side),
+    the 112-plane records with history, and the FP32-ALU path (one workspace: the groups take turns)."""
+    import paper_2609_37447_b200 as az
+    from inputs import configs, weights
+    cfg = configs.tiny_config(in_planes=in_planes, blocks=2, channels=channels, policy_head=head, value_head=value_head,
+                              precision=precision, batch=64)
+    blob = weights.make_blob(cfg, 0.02, 0.05)
+    net = az.az_load_net(az.make_arch(in_planes, 2, channels, head, value_head, precision, 64), blob)
+    stride = 784 if in_planes == 112 else 104
+    rec = records(head, stride, 31, 20261003)
+    n, size = rec.shape[0], SIZE[head]
+    results = []
+    for groups in (2, 1):
+        s = az.az_search_create(net, az.make_search_config(n, head, stride, leaves=2, groups=groups, max_nodes=200))
+        az.az_search_set_roots(s, rec)
+        az.az_search_run(s, 40)
+        played = az.az_search_advance(s)
+        az.az_search_run(s, 40)
+        out = []
+        for g in range(n):
+            a, nv, w, p = az.az_search_root(s, g)
+            c, nvis, wsum = az.az_search_tree(s, g)
+            out.append((a, nv, w, p, c, nvis, wsum, played[g]))
+            assert c[2] == 0 and (nvis[0] == 1 + nv.sum() or len(a) == 0)
+            assert (np.abs(w) <= nv + 1e-4).all() and (len(a) == 0 or abs(float(p.sum()) - 1) < 1e-3)
+        results.append(out)
+        az.az_search_destroy(s)
+    # one group and two groups: the same trees, bit for bit
+    for x, y in zip(*results):
+        assert all(np.atleast_1d(u).tobytes() == np.atleast_1d(v).tobytes() for u, v in zip(x, y))
+    # the moves played are legal moves of the roots
+    masks = oracle.legal_masks(cur_of(rec), head)
+    for g in range(n):
+        pl = int(results[0][g][7])
+        if pl >= 0:
+            assert (int(masks[g, pl >> 6]) >> (pl & 63)) & 1
+    assert az.az_device_status(net) & ~1 == 0
+    az.az_free_net(net)
+
+
 def test_bad_arguments():
     import paper_2609_37447_b200 as az
     for kw in ({"leaves": 17}, {"groups": 3}, {"max_nodes": 1}):
