@@ -601,7 +601,9 @@ def main():
                          "flops_per_launch": flops},
         }
         if not args.no_cpu_baseline:
-            sample = 256 if cfg.channels >= 128 else cfg.batch
+            # about twenty core-seconds of the oracle: 500 positions at 20 x 128 (it runs some 25 positions per
+            # second and core there), fewer in proportion to the tower's work for the larger networks
+            sample = max(16, int(500 * 757e6 / tower_flops_per_position(cfg))) if cfg.channels >= 128 else cfg.batch
             sample = min(sample, B)
             rate, dt, threads = oracle_rate(cfg, blob, recs, sample)
             out["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
