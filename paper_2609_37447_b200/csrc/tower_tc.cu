@@ -704,7 +704,10 @@ tower_tc_kernel(const TowerArgs args) {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] = fmaxf(v[i], 0.0f);
                     }
-                    if (kPnet) {                                     // activations capped at six (Sec. 4.3.6)
+                    // activations capped at six (Sec. 4.3.6).  A first convolution's output in the int8 form goes nowhere
+                    // but into the saturating conversion to unsigned 8-bit, whose 255 stands for the channel's calibrated
+                    // maximum, itself at most six: the cap is implied there.
+                    if (kPnet && !(kInt8 && from_acc)) {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] = fminf(v[i], kFp8 ? lc[3 * kMyC + ks * 16 + i] : 6.0f);   // six, in the layer's output units
                     }

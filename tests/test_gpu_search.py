@@ -155,12 +155,15 @@ def test_full_pools_are_reported_like_the_oracles():
     assert any(c[4][2] & az.AZ_SEARCH_FLAG_EDGES_FULL for c in got)
 
 
-def test_many_games_at_the_papers_batch_shape():
-    """512 games in two groups of 256 (Sec. 5.1), 64 steps; sampled games against the oracle."""
+@pytest.mark.parametrize("games", [592, 640])
+def test_many_games_in_the_benchmarks_launch_configuration(games):
+    """Two groups of 296 games (the benchmark's default: one two-board group per SM) and of 320 (the paper's batch,
+    Sec. 5.1), 64 steps; sampled games against the oracle."""
     import paper_2609_37447_b200 as az
-    rec = records(2, 128, 512, 20260997)
+    rec = records(2, 128, games, 20260997)
     got = run_gpu_search(az, rec, 2, 128, 64, 1, 2, 80, 80 * 64, seed=11)
-    pick = [0, 1, 2, 3, 4, 5, 6, 7, 100, 255, 256, 257, 400, 511]
+    half = games // 2
+    pick = [0, 1, 2, 3, 4, 5, 6, 7, 100, half - 1, half, half + 1, 400, games - 1]
     compare_with_oracle([got[g] for g in pick], rec[pick], 2, 64, 1, 80, 80 * 64, seed=11)
     for a, n, w, p, counts, nvis, wsum in got:
         assert n.sum() + counts[3] == 64 or len(a) == 0
