@@ -38,6 +38,7 @@ WORKLOADS = {
     "p12i": "p12i: p12 with the backbone's convolutions in int8 (pooled context and heads in floating point), batch 1024",
     "p14": "p14: the paper's own network at its reported size, 14x160 bf16, batch 320 as the paper serves it "
            "(App. D.3); --batch for other sizes",
+    "p19": "p19: the paper's own network at the largest size of its ladder, 19x176 bf16, batch 296 (one round); --batch for other sizes",
     "p14i": "p14i: p14 with the backbone's convolutions in int8, the precision the paper deploys; batch 320, --batch for other sizes",
     "s14i": "s14i: the search of s14 over the int8 14x160 network",
     "s14": "s14: batched tree search (Eq. 1, c 1.5, first-play reduction 0.2, discount 0.99) over the paper's 14x160 "

@@ -139,7 +139,8 @@ size_t az_plane_channels(const az_arch *arch);      /* channels of the encoded p
  * then in.w[C][52][3][3] in.scale in.bias; per block w1[C][C][3][3] scale1 bias1, (odd blocks)
  * gw[3C/4][C/2], w2[C][C or 3C/4][3][3] scale2 bias2; t.w[128][C] t.b; q.w[128][128] q.b; k.w k.b;
  * o.w[4][128] o.b; v.cw[2][C] v.cscale v.cbias; v.w1[48][128] v.b1; v.w2[3][48] v.b2.
- * Built for channels == 128 and 160 in bf16 (AZ_ERR_UNSUPPORTED otherwise).
+ * Built for the three sizes of the paper's ladder (App. D.3), channels == 128, 160 and 176, in bf16,
+ * and for 128 and 160 with an int8 backbone (AZ_PREC_INT8; AZ_ERR_UNSUPPORTED otherwise).
  * Errors: BAD_ARG, BAD_ARCH, BAD_WEIGHTS, UNSUPPORTED, CUDA.
  */
 int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az_net **out);

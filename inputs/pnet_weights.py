@@ -54,6 +54,8 @@ class PNetConfig:
 PNET_CONFIGS = {
     "p12": PNetConfig("p12", 12, 128, 1024, 20260961, 9371201),
     "p14": PNetConfig("p14", 14, 160, 320, 20260962, 9371401),
+    # the largest stage of the paper's ladder (App. D.3)
+    "p19": PNetConfig("p19", 19, 176, 296, 20260964, 9371901),
     # p12 with the backbone's convolutions in int8, the precision the paper deploys (Sec. 4.3.6)
     "p12i": PNetConfig("p12i", 12, 128, 1024, 20260961, 9371201, precision=3, weights_like="p12"),
     # the reported checkpoint's size in the precision the paper deploys it in (Sec. 4.3.6, App. B.1)

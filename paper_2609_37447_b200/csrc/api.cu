@@ -377,9 +377,10 @@ int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az
     *out = nullptr;
     if (!az::arch_ok(*arch)) return AZ_ERR_BAD_ARCH;
     const bool pnet = arch->in_planes == 52;
-    // of the paper's network ladder the 128- and 160-channel sizes are built, in bf16 and in int8
-    if (pnet && !((arch->precision == AZ_PREC_BF16 || arch->precision == AZ_PREC_INT8) &&
-                  (arch->channels == 128 || arch->channels == 160)))
+    // the paper's network ladder: 128, 160 and 176 channels in bf16; 128 and 160 also in int8 (its MMAs take 32
+    // channels at a time, which 176 is not a multiple of)
+    if (pnet && !((arch->precision == AZ_PREC_BF16 && (arch->channels == 128 || arch->channels == 160 || arch->channels == 176)) ||
+                  (arch->precision == AZ_PREC_INT8 && (arch->channels == 128 || arch->channels == 160))))
         return AZ_ERR_UNSUPPORTED;
     az::BlobView view;
     int rc = AZ_OK;

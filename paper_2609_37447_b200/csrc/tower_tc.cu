@@ -93,7 +93,8 @@ struct Shape {
     static constexpr int smem_bytes(bool fp8, bool pnet = false) {
         return kOffConst + kEpiWarps * (fp8 ? (pnet ? 4 : 3) : 1) * (kC / kSets) * 4 + 256 * 4 + (pnet ? kPoolFloats * 4 : 0);
     }
-    static_assert(kOffConst + kEpiWarps * 4 * (kC / kSets) * 4 + 1024 + kPoolFloats * 4 <= kMaxSmem || kC == 256, "shared memory budget");
+    // (four constant vectors per channel in the 8-bit forms, one in bf16; the 176-channel shape exists in bf16 only)
+    static_assert(kOffConst + kEpiWarps * (kC == 176 ? 1 : 4) * (kC / kSets) * 4 + 1024 + kPoolFloats * 4 <= kMaxSmem || kC == 256, "shared memory budget");
     static_assert(kGroups * 2 * kC <= (int)kTmemCols, "TMEM: per group C columns of residual stream and C of accumulator");
 };
 
@@ -165,9 +166,13 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
     return bounded_wait(bar, parity, abort_flag, status, kStatusWaitTimeout, kSpinLimit, waited);
 }
 
-// slices of the head projection's K that travel in one weight stage
+// slices of the head projection's K that travel in one weight stage (the last stage may carry fewer: eleven
+// slices of the 176-channel shape go as six and five)
 template <class S> __device__ __host__ constexpr int head_slices_per_stage(int head_n) {
-    return S::kC == 128 ? (head_n == 256 ? 4 : S::kSlices) : S::kC == 160 ? 5 : (head_n == 64 ? 8 : 4);
+    return S::kC == 128 ? (head_n == 256 ? 4 : S::kSlices) : S::kC == 160 ? 5 : S::kC == 176 ? 6 : (head_n == 64 ? 8 : 4);
+}
+template <class S> __device__ __host__ constexpr int head_stages(int head_n) {
+    return head_n ? (S::kSlices + head_slices_per_stage<S>(head_n) - 1) / head_slices_per_stage<S>(head_n) : 0;
 }
 
 // kFp8: the 8-bit tower (layers after the input layer read 8-bit operands, 32 channels per MMA); with
@@ -177,7 +182,8 @@ template <bool kFp8, class S, bool kPnet = false, bool kInt8 = false>
 __global__ void __launch_bounds__(S::kThreads, 1)
 tower_tc_kernel(const TowerArgs args) {
     static_assert(!kInt8 || kFp8, "the int8 tower is a form of the 8-bit tower");
-    static_assert(!kPnet || S::kC == 128 || S::kC == 160, "the paper's network runs on the 128- and 160-channel shapes");
+    static_assert(!kPnet || S::kC == 128 || S::kC == 160 || S::kC == 176, "the paper's network runs on the 128-, 160- and 176-channel shapes");
+    static_assert(S::kC != 176 || S::kSets == 1, "eleven slices do not split over two sets");
     static_assert(!(kPnet && kFp8) || kInt8, "of the 8-bit towers the int8 one carries the paper's network");
     constexpr int kC = S::kC, kGroups = S::kGroups, kStages = S::kStages, kSlices = S::kSlices;
     constexpr int kFrameBytes = S::kFrameBytes, kStageBytes = S::kStageBytes, kThreads = S::kThreads;
@@ -264,13 +270,14 @@ tower_tc_kernel(const TowerArgs args) {
             if (!rd.valid) break;
             int n_stages = 0;
             for (int l = 0; l < n_conv; ++l) n_stages += slices_of(l) * S::kStagesPerSlice;
-            const int n_head_stages = head_n ? kSlices / hsps : 0;
+            const int n_head_stages = head_stages<S>(head_n);
             for (int st = 0; st < n_stages + n_head_stages && ok; ++st) {
                 // tower stages are contiguous and equally sized; the head projections follow as small stages of their own
                 const bool head = st >= n_stages;
                 const unsigned char *src = head ? reinterpret_cast<const unsigned char *>(args.head_w) + (size_t)(st - n_stages) * hsps * head_n * 32
                                                 : reinterpret_cast<const unsigned char *>(args.weights) + (size_t)st * kStageBytes;
-                const uint32_t bytes = head ? (uint32_t)(hsps * head_n * 32) : (uint32_t)kStageBytes;
+                const int head_left = kSlices - (st - n_stages) * hsps;         // slices the head still has to fetch
+                const uint32_t bytes = head ? (uint32_t)((head_left < hsps ? head_left : hsps) * head_n * 32) : (uint32_t)kStageBytes;
                 ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 if (lane == 0) {
@@ -313,7 +320,7 @@ tower_tc_kernel(const TowerArgs args) {
             if ((g == 0 ? rd.group[0] : rd.group[1]) < 0) {
                 // a slot without a group this round still takes part in the ring protocol: it waits for
                 // every stage of the round and releases it without issuing anything
-                int n_stages = head_n ? kSlices / hsps : 0;
+                int n_stages = head_stages<S>(head_n);
                 for (int l = 0; l < n_conv; ++l) n_stages += slices_of(l) * S::kStagesPerSlice;
                 for (int st = 0; st < n_stages && ok; ++st) {
                     ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status);
@@ -413,7 +420,7 @@ tower_tc_kernel(const TowerArgs args) {
                         a_phase ^= 1u << kc;
                     }
                     ptx::tc_fence_after();
-                    const bool stage_done = (kc % hsps) == hsps - 1;
+                    const bool stage_done = (kc % hsps) == hsps - 1 || kc == kSlices - 1;
                     {
                         const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
                         const uint32_t b_lo = (((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) + (uint32_t)((kc % hsps) * head_n * 2)) |
@@ -575,7 +582,7 @@ tower_tc_kernel(const TowerArgs args) {
                     // With two sets the eight-channel chunks go to the set that owns their 16-channel slice (whose
                     // constants that set's warps hold).
 #pragma unroll
-                    for (int pc = 0; pc < kPoolC / 8; ++pc) {
+                    for (int pc = 0; pc < (kPoolC + 7) / 8; ++pc) {             // (176 channels: the last chunk is half a chunk)
                         const int pslice = (kRegC + pc * 8) / 16;                 // the slice this chunk lies in
                         if (S::kSets > 1 && (pslice % S::kSets) != set) continue;
                         const int cidx = (pslice / S::kSets) * 16 + (kRegC + pc * 8) % 16;   // in this warp's copy of the constants
@@ -589,7 +596,7 @@ tower_tc_kernel(const TowerArgs args) {
                             // so their constants carry no activation scale and the value is in real units)
                             const float pre = kFp8 ? fmaf(__int2float_rn((int)r8[i]), lc[cidx + i], bias[cidx + i])
                                                    : __uint_as_float(r8[i]) + bias[cidx + i];
-                            sm[i] = live ? fminf(fmaxf(pre, 0.0f), 6.0f) : 0.0f;
+                            sm[i] = (live && pc * 8 + i < kPoolC) ? fminf(fmaxf(pre, 0.0f), 6.0f) : 0.0f;
                             mx[i] = sm[i];
                         }
 #pragma unroll
@@ -608,8 +615,10 @@ tower_tc_kernel(const TowerArgs args) {
                         mx[0] = fmaxf(mx[0], __shfl_xor_sync(0xffffffffu, mx[0], 16));
                         if (lane < 16) {                                   // lanes 0-7 board 0, lanes 8-15 board 1
                             const int c0 = pc * 8 + 4 * (lane & 1) + 2 * ((lane >> 1) & 1) + ((lane >> 2) & 1);
-                            pool_part[(q * 2 + b) * kPoolC + c0] = sm[0];
-                            pool_part[4 * 2 * kPoolC + (q * 2 + b) * kPoolC + c0] = mx[0];
+                            if (c0 < kPoolC) {
+                                pool_part[(q * 2 + b) * kPoolC + c0] = sm[0];
+                                pool_part[4 * 2 * kPoolC + (q * 2 + b) * kPoolC + c0] = mx[0];
+                            }
                         }
                     }
                     constexpr int kGroupThreads = 128 * S::kSets;
@@ -874,6 +883,7 @@ typedef Shape<160, 1, AZ_P160_SETS> Shape160;
 #define AZ_P128_SETS 2
 #endif
 typedef Shape<128, 2, AZ_P128_SETS> Shape128P;           // the paper's 128-channel network
+typedef Shape<176, 1, 1> Shape176;                       // the ladder's largest size, 19 x 176 (eleven slices: one set)
 constexpr int kStageBytes = Shape128::kStageBytes;       // host-side packing of the 128-channel stages
 
 }  // namespace
@@ -1055,6 +1065,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape160, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128P, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape160, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape176, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
     const int sms = dev < 64 ? sm_count[dev] : 148;
@@ -1087,7 +1098,8 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     // one CTA per SM, or one per two-board group when there are fewer groups than SMs
     const int n_groups = (batch + kNB - 1) / kNB;
     const int grid = n_groups < sms ? n_groups : sms;
-    if (net.pnet && net.arch.channels == 160 && fp8) tower_tc_kernel<true, Shape160, true, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(true, true), s>>>(a);
+    if (net.pnet && net.arch.channels == 176) tower_tc_kernel<false, Shape176, true><<<grid, Shape176::kThreads, Shape176::smem_bytes(false, true), s>>>(a);
+    else if (net.pnet && net.arch.channels == 160 && fp8) tower_tc_kernel<true, Shape160, true, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(true, true), s>>>(a);
     else if (net.pnet && net.arch.channels == 160) tower_tc_kernel<false, Shape160, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(false, true), s>>>(a);
     else if (net.pnet && fp8) tower_tc_kernel<true, Shape128P, true, true><<<grid, Shape128P::kThreads, Shape128P::smem_bytes(true, true), s>>>(a);
     else if (net.pnet) tower_tc_kernel<false, Shape128P, true><<<grid, Shape128P::kThreads, Shape128P::smem_bytes(false, true), s>>>(a);

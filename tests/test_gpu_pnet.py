@@ -48,7 +48,7 @@ def test_masks_of_the_1880_action_list_are_bit_exact():
     assert bits[:, 1792:1880].sum() > 0 and not bits[:, 1880:].any()
 
 
-@pytest.mark.parametrize("channels", [128, 160])
+@pytest.mark.parametrize("channels", [128, 160, 176])
 @pytest.mark.parametrize("blocks,batch", [(0, 5), (1, 7), (2, 9), (4, 33)])
 def test_small_networks_layer_by_layer(blocks, batch, channels):
     import paper_2609_37447_b200 as az
@@ -115,6 +115,29 @@ def test_p14_the_reported_checkpoints_size_batch_320_and_a_ragged_multiple():
         agree = (pg[rows].argmax(axis=1) == po.argmax(axis=1)).mean()
         print(f"p14: n={rows.size} of {batch} policy max-abs {perr:.3e} value max-abs {verr:.3e} arg-max agreement {agree:.4f}")
         assert perr <= TOL and verr <= TOL and agree >= 0.95
+        bits = np.unpackbits(mg.view(np.uint8), axis=1, bitorder="little")[:, :pw.ACTIONS].astype(bool)
+        assert np.isfinite(pg).all() and (pg[~bits] == 0.0).all() and np.abs(pg.sum(axis=1) - 1).max() < 1e-3
+    az.az_free_net(net)
+
+
+def test_p19_the_ladders_largest_size():
+    # 19 x 176: eleven 16-channel slices, a pooled quarter of 44 channels that starts in the middle of a slice
+    import paper_2609_37447_b200 as az
+    cfg = pw.PNET_CONFIGS["p19"]
+    blob = pw.make_blob(cfg)
+    net = load(az, cfg, blob, 320)
+    for batch in (296, 311):
+        rec, _ = positions.generate_moves(cfg.position_seed, batch, cfg.plies)
+        mg, pg, vg, tg = gpu_run(az, net, cfg, rec, tower=True)
+        rows = np.unique(np.concatenate([[0, 1, 147, 148, 149, 295, batch - 2, batch - 1], np.arange(5, batch, 9)]))
+        mo, _, po, vo, extra = oracle.pnet_evaluate(blob, rec[rows], want_tower=True)
+        assert (mg[rows] == mo).all()
+        want = extra["tower"].reshape(rows.size, 176, 64).transpose(0, 2, 1)
+        rel = float(np.sqrt(((tg[rows] - want) ** 2).mean() / (want ** 2).mean()))
+        perr, verr = np.abs(pg[rows] - po).max(), np.abs(vg[rows] - vo).max()
+        agree = (pg[rows].argmax(axis=1) == po.argmax(axis=1)).mean()
+        print(f"p19: n={rows.size} of {batch} policy max-abs {perr:.3e} value max-abs {verr:.3e} arg-max agreement {agree:.4f} backbone rms {rel:.3e}")
+        assert perr <= TOL and verr <= TOL and rel < 1.5e-2 and agree >= 0.95
         bits = np.unpackbits(mg.view(np.uint8), axis=1, bitorder="little")[:, :pw.ACTIONS].astype(bool)
         assert np.isfinite(pg).all() and (pg[~bits] == 0.0).all() and np.abs(pg.sum(axis=1) - 1).max() < 1e-3
     az.az_free_net(net)
@@ -238,7 +261,11 @@ def test_other_entry_points_serve_the_papers_network_too():
 
 def test_unsupported_sizes_are_refused():
     import paper_2609_37447_b200 as az
-    cfg = pw.PNetConfig("p19", 2, 176, 16, 1, 1)                      # the ladder's 176-channel size is not built
+    cfg = pw.PNetConfig("p24", 2, 192, 16, 1, 1)                      # not a size of the paper's ladder
+    with pytest.raises(az.AzError) as e:
+        load(az, cfg, pw.make_blob(cfg, 1.0, 1.0), 16)
+    assert e.value.code == az.AZ_ERR_UNSUPPORTED
+    cfg = pw.PNetConfig("p19i", 2, 176, 16, 1, 1, precision=3)        # int8 MMAs take 32 channels at a time
     with pytest.raises(az.AzError) as e:
         load(az, cfg, pw.make_blob(cfg, 1.0, 1.0), 16)
     assert e.value.code == az.AZ_ERR_UNSUPPORTED
