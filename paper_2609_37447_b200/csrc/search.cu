@@ -24,10 +24,11 @@ constexpr int kMaxDepth = AZ_SEARCH_MAX_DEPTH;
 
 enum : int { kSlotNone = 0, kSlotEval = 1, kSlotTerminal = 2 };
 
-struct alignas(8) Edge {                         // 24 bytes
+struct alignas(16) Edge {                        // 32 bytes
     int action, child, n, m;
     float prior, w;
-};
+    int cbegin, ccnt;                            // the child's edge range once it has been expanded (a copy of its node's
+};                                               // fields): a descent fetches the child's node and edges side by side
 struct alignas(16) Node {                        // 32 bytes
     int edge_begin, n_edges;                     // n_edges < 0: waiting for its evaluation
     int terminal; float tvalue;
@@ -315,23 +316,29 @@ search_select_kernel(Trees t, Batch b, int game0, int n_games, int root_step) {
         } else {
             int node = 0;
             bool given_up = false;
+            // where the current node's edges lie, known before its node record arrives (from the edge that led here)
+            int ebegin = 0, ecnt = 0;
+            { const Node r0 = nodes[0]; ebegin = r0.edge_begin; ecnt = r0.n_edges; }
             for (;;) {
                 const Node nd = nodes[node];
+                Edge first{};                                           // this lane's first edge, fetched beside the node
+                if (lane < ecnt) first = edges[ebegin + lane];
                 if (nd.terminal) { kind = kSlotTerminal; leaf = node; break; }
                 if (nd.n_edges < 0) { given_up = true; break; }
                 if (depth == kMaxDepth) { if (lane == 0) gs->flags |= AZ_SEARCH_FLAG_DEPTH; given_up = true; break; }
                 const float sqrt_n = __fsqrt_rn((float)(nd.nsum > 1 ? nd.nsum : 1));
                 const float fpu = __fsub_rn(__fdiv_rn(nd.wsum, (float)nd.nvis), t.fpu_reduction);
                 float best_score = 0.0f; int best = -1;
+                Edge mine{};                                            // the edge behind this lane's best score
                 for (int i = lane; i < nd.n_edges; i += 32) {
-                    const Edge e = edges[nd.edge_begin + i];
+                    const Edge e = i == lane ? first : edges[nd.edge_begin + i];
                     const int n = e.n + e.m;
                     const float q = n > 0 ? __fdiv_rn(__fsub_rn(e.w, (float)e.m), (float)n) : fpu;
                     float u = __fmul_rn(t.c_puct, e.prior);
                     u = __fmul_rn(u, sqrt_n);
                     u = __fdiv_rn(u, (float)(1 + n));
                     const float score = __fadd_rn(q, u);
-                    if (best < 0 || score > best_score) { best = i; best_score = score; }
+                    if (best < 0 || score > best_score) { best = i; best_score = score; mine = e; }
                 }
 #pragma unroll
                 for (int d = 16; d; d >>= 1) {
@@ -341,7 +348,12 @@ search_select_kernel(Trees t, Batch b, int game0, int n_games, int root_step) {
                     if (ob >= 0 && (best < 0 || os > best_score || (os == best_score && ob < best))) { best = ob; best_score = os; }
                 }
                 const int ei = nd.edge_begin + best;
-                const Edge chosen = edges[ei];
+                Edge chosen;                                            // from the lane that scored it (edge i sits in lane i % 32)
+                chosen.action = __shfl_sync(0xffffffffu, mine.action, best & 31);
+                chosen.child = __shfl_sync(0xffffffffu, mine.child, best & 31);
+                chosen.m = __shfl_sync(0xffffffffu, mine.m, best & 31);
+                chosen.cbegin = __shfl_sync(0xffffffffu, mine.cbegin, best & 31);
+                chosen.ccnt = __shfl_sync(0xffffffffu, mine.ccnt, best & 31);
                 __syncwarp();
                 if (lane == 0) {
                     edges[ei].m = chosen.m + 1;
@@ -382,6 +394,7 @@ search_select_kernel(Trees t, Batch b, int game0, int n_games, int root_step) {
                     break;
                 }
                 node = chosen.child;
+                ebegin = chosen.cbegin; ecnt = chosen.ccnt;
             }
             if (given_up) {
                 __syncwarp();
@@ -442,11 +455,18 @@ search_finish_kernel(Trees t, Batch b, int game0, int n_games, const u64 *__rest
                     if (rank < cnt) {
                         Edge e;
                         e.action = action; e.child = -1; e.n = 0; e.m = 0; e.prior = pr[rank]; e.w = 0.0f;
+                        e.cbegin = 0; e.ccnt = 0;
                         edges[begin + rank] = e;
                     }
                 });
                 __syncwarp();
-                if (lane == 0) gs->n_edges = begin + cnt;
+                if (lane == 0) {
+                    gs->n_edges = begin + cnt;
+                    if (depth > 0) {                                    // the edge that leads here learns where the new edges lie
+                        Edge *up = edges + b.path_e[(size_t)row * kMaxDepth + depth - 1];
+                        up->cbegin = begin; up->ccnt = cnt;
+                    }
+                }
             }
             v = nd.terminal ? nd.tvalue : net_v;
             nd.nvis = 1; nd.wsum = v;
@@ -536,7 +556,7 @@ struct Search {
     bool need_root_step = true;                  // some tree's root still waits for its evaluation
     // played moves: the kept subtrees are written to a second set of pools, which then becomes the first
     Node *alt_nodes = nullptr; Edge *alt_edges = nullptr; unsigned char *alt_node_pos = nullptr; u64 *alt_node_hash = nullptr;
-    int *remap = nullptr;                        // [games][max_nodes]: old index of every kept node
+    int *remap = nullptr;                        // [games][2][max_nodes]: old index of every kept node, edge that leads to it
     int *adv_actions = nullptr, *adv_played = nullptr, *adv_fresh = nullptr;
 };
 
@@ -594,7 +614,8 @@ search_advance_kernel(Trees t, Node *new_nodes, Edge *new_edges, unsigned char *
     Node *nn = new_nodes + (size_t)g * t.node_cap;
     Edge *ne = new_edges + (size_t)g * t.edge_cap;
     unsigned char *np = new_pos + (size_t)g * t.node_cap * t.stride;
-    int *remap = remap_all + (size_t)g * t.node_cap;
+    int *remap = remap_all + (size_t)g * 2 * t.node_cap;            // [old index of kept node | index of the edge that leads to it]
+    int *up_edge = remap + t.node_cap;
     GameState *gs = t.games + g;
     const u64 *hashes = t.node_hash + (size_t)g * t.node_cap;
     u64 *nh = new_hash + (size_t)g * t.node_cap;
@@ -696,12 +717,16 @@ search_advance_kernel(Trees t, Node *new_nodes, Edge *new_edges, unsigned char *
             if (has) {
                 const int id = n_new + __popc(m & ((1u << lane) - 1u));
                 remap[id] = e.child;
+                up_edge[id] = e_new + j;                               // the kept node's edge range is filled in when its turn comes
                 e.child = id;
             }
             if (j < cnt) ne[e_new + j] = e;
             n_new += __popc(m);
         }
-        if (lane == 0) { nd.edge_begin = e_new; nn[i] = nd; nh[i] = hashes[o]; }
+        if (lane == 0) {
+            if (i > 0) { ne[up_edge[i]].cbegin = e_new; ne[up_edge[i]].ccnt = cnt; }
+            nd.edge_begin = e_new; nn[i] = nd; nh[i] = hashes[o];
+        }
         e_new += cnt;
         __syncwarp();
     }
@@ -967,7 +992,7 @@ int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *p
         AZ_CUDA(cudaMalloc((void **)&s->alt_edges, G * t.edge_cap * sizeof(az::Edge)));
         AZ_CUDA(cudaMalloc((void **)&s->alt_node_pos, G * t.node_cap * (size_t)t.stride));
         AZ_CUDA(cudaMalloc((void **)&s->alt_node_hash, G * t.node_cap * sizeof(az::u64)));
-        AZ_CUDA(cudaMalloc((void **)&s->remap, G * t.node_cap * sizeof(int)));
+        AZ_CUDA(cudaMalloc((void **)&s->remap, G * 2 * t.node_cap * sizeof(int)));
         AZ_CUDA(cudaMalloc((void **)&s->adv_actions, G * sizeof(int)));
         AZ_CUDA(cudaMalloc((void **)&s->adv_played, G * sizeof(int)));
         AZ_CUDA(cudaMalloc((void **)&s->adv_fresh, sizeof(int)));
