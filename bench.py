@@ -366,7 +366,7 @@ def run_search(args, name):
                            "(root visit counts to host memory); bytes are per step of the K-step search"},
             "gpu_launches": launches,
             "clocks": clocks,
-            "roofline": {"kernel": "tower_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
+            "roofline": {"kernel": roof_kernel, "bound": roof_bound, "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s",
                          "frac": achieved / peak_tf, "traffic": None,
                          "peak_source": f"of {peaks['source']} ({'sustained' if sustained else 'burst'} bf16 GEMM"
                                         + (" x 2, nominal 8-bit/bf16 ratio)" if cfg.precision >= 2 else ")"),
@@ -571,6 +571,12 @@ def main():
         peak_note = (f"of {peaks['source']} ({'sustained' if sustained else 'burst'} bf16 GEMM"
                      + (" x 2, nominal 8-bit/bf16 ratio" if cfg.precision >= 2 else "")
                      + "; sustained is used when a tower launch takes 2 ms or more)")
+        roof_kernel, roof_bound = "tower_tc_kernel", "tensor"
+        if cfg.precision == 0:
+            # the fp32 network runs on the FP32 FMA pipes: 148 SMs x 128 FMA per clock x 2 x the maximum SM clock
+            roof_kernel, roof_bound = "conv3x3_f32_tiled_kernel (13 launches)", "alu"
+            peak_tf = 148 * 128 * 2 * (clocks.get("sm_max_mhz") or 1965) * 1e6 / 1e12
+            peak_note = "derived: 148 SMs x 128 FP32 FMA per clock x 2 x the maximum SM clock"
         out = {
             "metric": METRIC, "value": evals / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
@@ -595,7 +601,7 @@ def main():
                                           "api": "az_evaluate_legal_host, pinned host buffers, one batch at a time"},
             "gpu_launches": args.steps * az.az_launches_per_evaluate(net, B),
             "clocks": clocks,
-            "roofline": {"kernel": "tower_tc_kernel", "bound": "tensor", "achieved": achieved, "peak": peak_tf,
+            "roofline": {"kernel": roof_kernel, "bound": roof_bound, "achieved": achieved, "peak": peak_tf,
                          "unit": "TFLOP/s", "frac": (achieved / peak_tf) if achieved else None,
                          "traffic": traffic, "peak_source": peak_note,
                          "avg_launch_ms": tower_avg_ms, "launches_timed": tower_passes,

@@ -9,7 +9,9 @@
 // One CTA per (board, 64 output channels).  The board's input is staged in shared memory as a
 // zero-bordered 10x10 frame in 32-channel chunks; a thread owns one output channel and 16
 // squares, reads its weights coalesced across the CTA ([tap][ci][co] layout) and the inputs as
-// shared-memory broadcasts.  Bound: FP32 FMA issue.
+// shared-memory broadcasts.  Bound: FP32 FMA issue.  This general form serves odd shapes and the
+// bf16 nets the tensor-core tower does not cover; fp32 nets with channel counts in multiples of
+// 32 / 64 (the fp32 config) take the tiled kernel further down.
 #include "common.cuh"
 
 namespace az {
@@ -85,12 +87,116 @@ conv3x3_simt_kernel(const T *__restrict__ in, const T *__restrict__ w, const flo
     }
 }
 
+// The same convolution for fp32 networks whose channel counts are multiples of 32 (in) and 64 (out), tiled
+// for the FMA pipes: one CTA per (half board, 64 output channels), 128 threads, a thread owns 4 output
+// channels x 4 neighbouring squares of one rank.  Per 32-channel chunk the half board's zero-bordered frame
+// (6 x 10 squares) and ALL the chunk's weights (9 taps x 32 x 64, 72 KB) are staged in shared memory, so the
+// inner loop is eight 16-byte shared-memory loads (four of weights, conflict-free across the 16 channel
+// groups of a warp; four of inputs, broadcasts) per 64 FMAs and touches no global memory.
+// 16-byte asynchronous copy global -> shared (all of a thread's copies are in flight together)
+__device__ __forceinline__ void cp_async16(float *smem_dst, const void *gmem_src) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+constexpr int kTileThreads = 128;
+constexpr int kTileFrame = 60 * kChunk;                   // floats
+constexpr int kTileWeights = 9 * kChunk * kCoutTile;      // floats
+constexpr int kTileSmem = (kTileFrame + kTileWeights) * 4;
+
+__global__ void __launch_bounds__(kTileThreads)
+conv3x3_f32_tiled_kernel(const float *__restrict__ in, const float *__restrict__ w, const float *__restrict__ scale,
+                         const float *__restrict__ bias, const float *__restrict__ residual, float *__restrict__ out,
+                         int cin, int cout) {
+    extern __shared__ __align__(16) float tile_smem[];
+    float *frame = tile_smem;                              // [6 ranks][10 files][32 channels]
+    float *wt = tile_smem + kTileFrame;                    // [9 taps][32 channels][64 outputs]
+    const int b = blockIdx.x, half = blockIdx.y, co0 = blockIdx.z * kCoutTile;
+    const int cog = threadIdx.x & 15, sqg = threadIdx.x >> 4;        // 16 groups of 4 outputs, 8 groups of 4 squares
+    const int ry = sqg >> 1, x0 = (sqg & 1) * 4;                      // rank within the half board, first file
+    float acc[4][4];                                                  // [square][output]
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+
+    for (int c0 = 0; c0 < cin; c0 += kChunk) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < 60 * (kChunk / 4); i += kTileThreads) {
+            const int p = i / (kChunk / 4), c4 = i % (kChunk / 4);
+            const int y = half * 4 + p / 10 - 1, x = p % 10 - 1;
+            if (y >= 0 && y < 8 && x >= 0 && x < 8)
+                cp_async16(frame + i * 4, reinterpret_cast<const float4 *>(in + ((size_t)b * 64 + y * 8 + x) * cin + c0) + c4);
+            else
+                reinterpret_cast<float4 *>(frame)[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        }
+        for (int i = threadIdx.x; i < 9 * kChunk * (kCoutTile / 4); i += kTileThreads) {
+            const int row = i / (kCoutTile / 4), c4 = i % (kCoutTile / 4);   // row = tap * 32 + channel of the chunk
+            const int tap = row / kChunk, ci = row % kChunk;
+            cp_async16(wt + i * 4, reinterpret_cast<const float4 *>(w + ((size_t)tap * cin + c0 + ci) * cout + co0) + c4);
+        }
+        cp_async_wait_all();                               // every copy of this thread has landed; the barrier publishes them
+        __syncthreads();
+#pragma unroll 1
+        for (int tap = 0; tap < 9; ++tap) {
+            const float *fr = frame + ((ry + tap / 3) * 10 + x0 + tap % 3) * kChunk;
+            const float *wr = wt + tap * kChunk * kCoutTile + cog * 4;
+#pragma unroll 2
+            for (int ci = 0; ci < kChunk; ci += 4) {
+                float4 wv[4], iv[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) wv[k] = *reinterpret_cast<const float4 *>(wr + (ci + k) * kCoutTile);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) iv[i] = *reinterpret_cast<const float4 *>(fr + i * kChunk + ci);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float a[4] = {iv[i].x, iv[i].y, iv[i].z, iv[i].w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        acc[i][0] = fmaf(a[k], wv[k].x, acc[i][0]);
+                        acc[i][1] = fmaf(a[k], wv[k].y, acc[i][1]);
+                        acc[i][2] = fmaf(a[k], wv[k].z, acc[i][2]);
+                        acc[i][3] = fmaf(a[k], wv[k].w, acc[i][3]);
+                    }
+                }
+            }
+        }
+    }
+    const float4 s4 = *reinterpret_cast<const float4 *>(scale + co0 + cog * 4);
+    const float4 b4 = *reinterpret_cast<const float4 *>(bias + co0 + cog * 4);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int sq = (half * 4 + ry) * 8 + x0 + i;
+        const size_t o = ((size_t)b * 64 + sq) * cout + co0 + cog * 4;
+        float4 v = make_float4(fmaf(s4.x, acc[i][0], b4.x), fmaf(s4.y, acc[i][1], b4.y), fmaf(s4.z, acc[i][2], b4.z), fmaf(s4.w, acc[i][3], b4.w));
+        if (residual) {
+            const float4 r = *reinterpret_cast<const float4 *>(residual + o);
+            v.x += r.x; v.y += r.y; v.z += r.z; v.w += r.w;
+        }
+        *reinterpret_cast<float4 *>(out + o) = make_float4(fmaxf(v.x, 0.0f), fmaxf(v.y, 0.0f), fmaxf(v.z, 0.0f), fmaxf(v.w, 0.0f));
+    }
+}
+
 }  // namespace
 
 int launch_conv3x3_simt(const void *in, const void *w, const float *scale, const float *bias,
                         const void *residual, void *out, int batch, int cin, int cout, bool bf16,
                         cudaStream_t s) {
     if (batch == 0) return AZ_OK;
+    if (!bf16 && cin % kChunk == 0 && cout % kCoutTile == 0) {
+        static bool configured[64] = {};
+        int dev = 0;
+        AZ_CUDA(cudaGetDevice(&dev));
+        if (dev < 64 && !configured[dev]) {
+            AZ_CUDA(cudaFuncSetAttribute(conv3x3_f32_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileSmem));
+            configured[dev] = true;
+        }
+        conv3x3_f32_tiled_kernel<<<dim3((unsigned)batch, 2, (unsigned)(cout / kCoutTile)), kTileThreads, kTileSmem, s>>>(
+            (const float *)in, (const float *)w, scale, bias, (const float *)residual, (float *)out, cin, cout);
+        AZ_LAUNCH_CHECK();
+        return AZ_OK;
+    }
     dim3 grid((unsigned)batch, (unsigned)((cout + kCoutTile - 1) / kCoutTile));
     if (bf16)
         conv3x3_simt_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>(

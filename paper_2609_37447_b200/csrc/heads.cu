@@ -105,6 +105,43 @@ fc_kernel(const TIN *__restrict__ a, const TIN *__restrict__ w, const float *__r
         }
 }
 
+// ---- fully-connected layer for few rows (the fp32 network's value head: 64 x 2048 -> 128): the tiled kernel above
+// would run on two CTAs.  Here a warp owns one output column and sixteen rows: its column of weights stays in
+// registers (K / 32 values per lane, K <= 2048), every row is one coalesced pass over K and a shuffle reduction.
+constexpr int kFcRows = 16;
+__global__ void __launch_bounds__(256)
+fc_fewrows_kernel(const float *__restrict__ a, const float *__restrict__ w, const float *__restrict__ bias,
+                  int m, int n, int k, int relu, float *__restrict__ out) {
+    const int lane = threadIdx.x & 31, col = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (col >= n) return;                                    // whole warps leave together
+    const int m0 = blockIdx.y * kFcRows;
+    const int k4 = k / 128;                                  // float4 per lane
+    float4 wv[16];
+    const float4 *wp = reinterpret_cast<const float4 *>(w + (size_t)col * k);
+#pragma unroll
+    for (int j = 0; j < 16; ++j) wv[j] = j < k4 ? __ldg(wp + j * 32 + lane) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    const float bv = bias[col];
+    for (int r = m0; r < m0 + kFcRows && r < m; ++r) {
+        const float4 *ap = reinterpret_cast<const float4 *>(a + (size_t)r * k);
+        float acc0 = 0.0f, acc1 = 0.0f;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            if (j < k4) {
+                const float4 av = __ldg(ap + j * 32 + lane);
+                acc0 = fmaf(av.x, wv[j].x, acc0); acc1 = fmaf(av.y, wv[j].y, acc1);
+                acc0 = fmaf(av.z, wv[j].z, acc0); acc1 = fmaf(av.w, wv[j].w, acc1);
+            }
+        }
+        float v = acc0 + acc1;
+#pragma unroll
+        for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) {
+            v += bv;
+            out[(size_t)r * n + col] = relu ? fmaxf(v, 0.0f) : v;
+        }
+    }
+}
+
 // ---- value tail: one warp per position ---------------------------------------------------------
 __global__ void __launch_bounds__(128)
 value_tail_kernel(const float *__restrict__ hidden, const float *__restrict__ w2, const float *__restrict__ b2,
@@ -290,6 +327,12 @@ int launch_fc(const void *a, const void *w, const float *bias, int m, int n, int
               bool bf16_in, void *out, bool out_f32, cudaStream_t s) {
     if (m == 0) return AZ_OK;
     typedef __nv_bfloat16 bf;
+    if (!bf16_in && out_f32 && m <= 256 && k % 128 == 0 && k <= 2048) {
+        fc_fewrows_kernel<<<dim3((unsigned)((n + 7) / 8), (unsigned)((m + kFcRows - 1) / kFcRows)), 256, 0, s>>>(
+            (const float *)a, (const float *)w, bias, m, n, k, relu, (float *)out);
+        AZ_LAUNCH_CHECK();
+        return AZ_OK;
+    }
     dim3 grid((unsigned)((n + 63) / 64), (unsigned)((m + 63) / 64));
     if (bf16_in && out_f32) fc_kernel<bf, float><<<grid, 256, 0, s>>>((const bf *)a, (const bf *)w, bias, m, n, k, relu, (float *)out);
     else if (bf16_in) fc_kernel<bf, bf><<<grid, 256, 0, s>>>((const bf *)a, (const bf *)w, bias, m, n, k, relu, (bf *)out);
