@@ -54,3 +54,19 @@ def test_host_only_helpers(lib):
     with pytest.raises(az.AzError) as e:
         az.az_load_net(az.make_arch(19, 1, 32, 0, 0, 0, 4), b"\0" * 128)
     assert e.value.code == az.AZ_ERR_BAD_WEIGHTS
+
+
+def test_search_arguments_are_checked_before_any_cuda_call(lib):
+    import paper_2609_37447_b200 as az
+    for kw in ({"leaves": 0}, {"leaves": 17}, {"groups": 0}, {"groups": 3}, {"max_nodes": 1}, {"c_puct": -1.0}, {"discount": 0.0}):
+        with pytest.raises(az.AzError) as e:
+            az.az_search_create(None, az.make_search_config(4, 2, 128, evaluator=az.AZ_SEARCH_EVAL_STANDIN, **kw))
+        assert e.value.code == az.AZ_ERR_BAD_ARG, kw
+    with pytest.raises(az.AzError) as e:
+        az.az_search_create(None, az.make_search_config(4, 2, 128))           # the network evaluator needs a network
+    assert e.value.code == az.AZ_ERR_BAD_ARG
+    with pytest.raises(az.AzError) as e:
+        az.az_search_create(None, az.make_search_config(4, 3, 128, evaluator=az.AZ_SEARCH_EVAL_STANDIN))   # no such action list
+    assert e.value.code == az.AZ_ERR_BAD_ARG
+    cfg = az.make_search_config(4, 2, 128)
+    assert (cfg.c_puct, cfg.fpu_reduction, cfg.discount) == (1.5, pytest.approx(0.2), pytest.approx(0.99))   # App. D.2

@@ -39,6 +39,16 @@ def _worker(rank, world, port, out_dir):
     whole = positions.for_config(cfg, B * world)
     expect = [hashlib.sha256(whole[r * B:(r + 1) * B].tobytes()).digest() for r in range(world)]
     assert gathered == expect                                  # disjoint, ordered, and covering
+    # the search workloads shard their games the same way: every rank's roots (records with the last eight moves)
+    # are its own stretch of the one seeded stream
+    from inputs import pnet_weights
+    pcfg = pnet_weights.PNET_CONFIGS["p14"]
+    games = 24
+    roots = positions.generate_moves(pcfg.position_seed, games, pcfg.plies, first_index=sharding.rank_first_index(rank, games))[0]
+    gathered = [None] * world
+    dist.all_gather_object(gathered, hashlib.sha256(roots.tobytes()).digest())
+    all_roots = positions.generate_moves(pcfg.position_seed, games * world, pcfg.plies)[0]
+    assert gathered == [hashlib.sha256(all_roots[r * games:(r + 1) * games].tobytes()).digest() for r in range(world)]
     # strong-scaling split: contiguous, disjoint, covering, sizes differ by at most one
     ranges = [sharding.split_batch(101, r, world) for r in range(world)]
     assert ranges[0][0] == 0 and ranges[-1][1] == 101
