@@ -275,7 +275,7 @@ def run_search(args, name):
 
     def done(s):
         az.az_search_root_visits(s, actions, visits, counts)
-        return int(sum(int(visits[g, :counts[g]].sum()) for g in range(games)))
+        return int(visits[np.arange(az.AZ_MAX_LEGAL)[None, :] < counts[:, None]].sum())
 
     # ---- device-timed: warm-up steps, then K steps queued in one call, timed by events on the search's stream
     s = new_search()
