@@ -325,6 +325,44 @@ def test_given_moves_none_unvisited_and_impossible_ones():
         t.close()
 
 
+def test_random_configurations_against_the_oracle():
+    """Thirty seeded configurations (games, leaves, groups, action list, record layout, pool sizes, constants),
+    each searched, moved and searched again on both sides."""
+    import paper_2609_37447_b200 as az
+    rng = np.random.default_rng(20261010)
+    for case in range(30):
+        head, stride = [(0, 104), (0, 784), (1, 104), (1, 784), (2, 128)][int(rng.integers(5))]
+        games, leaves, groups = int(rng.integers(1, 10)), int(rng.choice([1, 1, 2, 3, 5, 8, 16])), int(rng.integers(1, 3))
+        sims = int(rng.integers(5, 70))
+        cap = int(rng.choice([sims * leaves * 3 + 2, max(8, sims * leaves // 2)]))          # roomy, or a pool that fills up
+        ecap = int(rng.choice([cap * 48, cap * 12]))
+        c_puct, fpu, disc = float(rng.choice([1.5, 1.0, 3.0, 0.0])), float(rng.choice([0.2, 0.0, 0.5])), float(rng.choice([0.99, 1.0, 0.9]))
+        seed = int(rng.integers(1 << 30))
+        rec = records(head, stride, max(games, 9), 20261011 + case)[rng.permutation(max(games, 9))[:games]]
+        rec = np.ascontiguousarray(rec)
+        cfg = az.make_search_config(games, head, stride, leaves=leaves, groups=groups, max_nodes=cap, max_edges=ecap,
+                                    evaluator=az.AZ_SEARCH_EVAL_STANDIN, c_puct=c_puct, fpu_reduction=fpu, discount=disc, seed=seed)
+        s = az.az_search_create(None, cfg)
+        az.az_search_set_roots(s, rec)
+        trees = [oracle.MctsTree(rec[g:g + 1], head, leaves=leaves, c_puct=c_puct, fpu_reduction=fpu, discount=disc, seed=seed,
+                                 node_cap=cap, edge_cap=ecap) for g in range(games)]
+        for phase in range(3):
+            az.az_search_run(s, sims)
+            for g in range(games):
+                trees[g].run(sims)
+                same_tree(read_gpu_tree(az, s, g), trees[g].read(), f"case {case} phase {phase} game {g}")
+            played = az.az_search_advance(s)
+            for g in range(games):
+                r = trees[g].read()
+                want = int(r["actions"][int(np.argmax(r["visits"]))]) if len(r["actions"]) else -1
+                assert played[g] == want, f"case {case} phase {phase} game {g}"
+                if want >= 0:
+                    trees[g].advance(want)
+        az.az_search_destroy(s)
+        for t in trees:
+            t.close()
+
+
 def test_search_with_the_network_as_evaluator():
     import paper_2609_37447_b200 as az
     cfg = pw.PNetConfig("ts", 2, 128, 64, 20260998, 4500)
