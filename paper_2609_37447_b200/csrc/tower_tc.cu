@@ -338,6 +338,12 @@ tower_tc_kernel(const TowerArgs args) {
                 const bool conv2 = l >= 2 && (l & 1) == 0;             // accumulates onto the residual stream
                 const uint32_t d = d_h + (((l & 1) == 1) ? (uint32_t)kC : 0u);   // conv1 writes the ACC columns
                 for (int kc = 0; kc < nkc && ok; ++kc) {
+                    // one group per CTA: the slice's first weight stage is normally there long before its activations;
+                    // looking at it first leaves nothing between the activations' arrival and the first MMA
+                    if (kGroups == 1) {
+                        ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+                        if (!ok) break;
+                    }
                     ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
                     if (!ok) break;
                     a_phase ^= 1u << kc;
@@ -345,11 +351,13 @@ tower_tc_kernel(const TowerArgs args) {
                     const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
 #pragma unroll
                     for (int st = 0; st < S::kStagesPerSlice; ++st) {
-                        ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
-                        if (!ok) break;
-                        if (follow) {
-                            ok = wait_bar(bar_lead(stage), phase, abort_flag, args.status, tr ? &t_wait[2] : nullptr);
+                        if (kGroups > 1 || st > 0) {
+                            ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                             if (!ok) break;
+                            if (follow) {
+                                ok = wait_bar(bar_lead(stage), phase, abort_flag, args.status, tr ? &t_wait[2] : nullptr);
+                                if (!ok) break;
+                            }
                         }
                         ptx::tc_fence_after();
                         const long long ti0 = tr ? clock64() : 0;
@@ -670,6 +678,33 @@ tower_tc_kernel(const TowerArgs args) {
                     ok = meet();
                     if (!ok) break;
                 }
+                auto write_back_h = [&](int ks, int kc, const float (&v)[16]) {
+                    // fp32 copy back to H (FP8: pre-divided by the next conv2's weight scale, so that
+                    // conv2 can accumulate its raw products straight onto it).  With one group per CTA this
+                    // comes AFTER the slice's hand-off (the next layer's MMAs wait for the frame, not for H, and
+                    // nothing else covers the layer boundary); with two groups, whose boundaries cover each
+                    // other, before it (measured).  Its completion is awaited once, after the loop: the next
+                    // reader of H is the conv2 two layers on, whose MMAs are gated by barriers these same
+                    // threads arrive on only after that wait.
+                    uint32_t w[16];
+#pragma unroll
+                    for (int i = 0; i < 16; i += 4) {
+                        float4 hs = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
+                        if (kFp8) hs = *reinterpret_cast<const float4 *>(lc + 2 * kMyC + ks * 16 + i);
+                        if (kInt8) {    // the stream in the next second convolution's integer units, rounded
+                            w[i + 0] = (uint32_t)__float2int_rn(v[i + 0] * hs.x);
+                            w[i + 1] = (uint32_t)__float2int_rn(v[i + 1] * hs.y);
+                            w[i + 2] = (uint32_t)__float2int_rn(v[i + 2] * hs.z);
+                            w[i + 3] = (uint32_t)__float2int_rn(v[i + 3] * hs.w);
+                        } else {
+                            w[i + 0] = __float_as_uint(kFp8 ? v[i + 0] * hs.x : v[i + 0]);
+                            w[i + 1] = __float_as_uint(kFp8 ? v[i + 1] * hs.y : v[i + 1]);
+                            w[i + 2] = __float_as_uint(kFp8 ? v[i + 2] * hs.z : v[i + 2]);
+                            w[i + 3] = __float_as_uint(kFp8 ? v[i + 3] * hs.w : v[i + 3]);
+                        }
+                    }
+                    ptx::tmem_st16(t_lane + (uint32_t)(kc * 16), w);
+                };
                 const float *ctx = pool_ctx + b * kCtxStride;                  // this row's board
                 const int n_kc = (kPnet && pooled) ? kShortSlices : kSlices;   // the pooled channels are not handed on
                 ptx::tmem_ld16(t_src + (uint32_t)(set * 16), r[0]);
@@ -758,31 +793,7 @@ tower_tc_kernel(const TowerArgs args) {
                             *reinterpret_cast<uint4 *>(frame + (2 * kc) * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                             *reinterpret_cast<uint4 *>(frame + (2 * kc + 1) * kPlaneBytes + slot * 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                         }
-                        if (keep_h) {
-                            // fp32 copy back to H (FP8: pre-divided by the next conv2's weight scale, so that
-                            // conv2 can accumulate its raw products straight onto it).  Its completion is
-                            // awaited once, after the loop: the next reader of H is the conv2 two layers on,
-                            // whose MMAs are gated by barriers these same threads arrive on only after that wait.
-                            uint32_t w[16];
-#pragma unroll
-                            for (int i = 0; i < 16; i += 4) {
-                                float4 hs = make_float4(1.0f, 1.0f, 1.0f, 1.0f);
-                                if (kFp8) hs = *reinterpret_cast<const float4 *>(lc + 2 * kMyC + ks * 16 + i);
-                                if (kInt8) {    // the stream in the next second convolution's integer units, rounded
-                                    w[i + 0] = (uint32_t)__float2int_rn(v[i + 0] * hs.x);
-                                    w[i + 1] = (uint32_t)__float2int_rn(v[i + 1] * hs.y);
-                                    w[i + 2] = (uint32_t)__float2int_rn(v[i + 2] * hs.z);
-                                    w[i + 3] = (uint32_t)__float2int_rn(v[i + 3] * hs.w);
-                                } else {
-                                    w[i + 0] = __float_as_uint(kFp8 ? v[i + 0] * hs.x : v[i + 0]);
-                                    w[i + 1] = __float_as_uint(kFp8 ? v[i + 1] * hs.y : v[i + 1]);
-                                    w[i + 2] = __float_as_uint(kFp8 ? v[i + 2] * hs.z : v[i + 2]);
-                                    w[i + 3] = __float_as_uint(kFp8 ? v[i + 3] * hs.w : v[i + 3]);
-                                }
-                            }
-                            ptx::tmem_st16(t_lane + (uint32_t)(kc * 16), w);
-                            if (S::kSets > 1 && ks == kMySlices - 1) ptx::tmem_st_wait();
-                        }
+                        if (kGroups > 1 && keep_h) write_back_h(ks, kc, v);
                         // e4m3 layers consume 32 channels per MMA: one hand-off per two slices.  With two sets
                         // every barrier counts both sets' warps: a pair of slices is handed off by the four
                         // warps of each set, and where the next layer reads 16-channel slices (the bf16 head)
@@ -796,9 +807,10 @@ tower_tc_kernel(const TowerArgs args) {
                                 if (S::kSets == 2 && !next_e4m3) ptx::mbar_arrive(bar_a_ready(g, kc ^ 1));
                             }
                         }
+                        if (kGroups == 1 && keep_h) write_back_h(ks, kc, v);
                     }
                 }
-                if (S::kSets == 1 && keep_h) ptx::tmem_st_wait();
+                if (keep_h) ptx::tmem_st_wait();
             }
             if (head_n && ok) {
                 // ---- head projections out of the ACC columns
