@@ -44,9 +44,10 @@ WORKLOADS = {
     "s14": "s14: batched tree search (Eq. 1, c 1.5, first-play reduction 0.2, discount 0.99) over the paper's 14x160 "
            "network: two groups of games, each step one batch of leaf positions per group (296 rows = one two-board "
            "group per SM; the paper serves 320, App. D.3: --batch 320), one traversal per game and step",
-    "s12": "s12: the same search over the 12x128 network",
+    "s12": "s12: the same search over the 12x128 network (--batch 592: one round of two-group CTAs)",
+    "s12i": "s12i: the same search over the int8 12x128 network",
 }
-SEARCH_NETS = {"s14": "p14", "s12": "p12", "s14i": "p14i"}
+SEARCH_NETS = {"s14": "p14", "s12": "p12", "s14i": "p14i", "s12i": "p12i"}
 SEARCH_METRIC = "searches/sec (tree traversals with their leaf evaluation)"
 SEARCH_UNIT = "searches/s"
 
