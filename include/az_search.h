@@ -131,6 +131,16 @@ int az_search_set_roots(az_search *search, const void *positions_host);
 int az_search_run(az_search *search, int simulations, float *elapsed_ms_out);
 
 /*
+ * The same in two halves, for a host thread that has other work while the GPU searches (Sec. 3.3: the actor
+ * interleaves games and submits batches without waiting): az_search_run_async queues the steps and returns;
+ * az_search_wait blocks until they are done and reports like az_search_run.  Between the two every other
+ * call on this az_search answers AZ_ERR_BUSY (az_search_destroy excepted, which waits); a second
+ * az_search_run_async answers AZ_ERR_BUSY as well, az_search_wait without a pending run AZ_ERR_BAD_ARG.
+ */
+int az_search_run_async(az_search *search, int simulations);
+int az_search_wait(az_search *search, float *elapsed_ms_out);
+
+/*
  * Root statistics of one game, to host buffers of AZ_MAX_LEGAL entries each: the root's actions in
  * ascending order with their visit counts N, value sums W and priors P; *count_out their number.
  */

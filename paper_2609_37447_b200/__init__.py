@@ -28,7 +28,7 @@ EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_siz
            "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error",
            "az_apply_moves", "az_standin_evaluate", "az_search_create", "az_search_destroy", "az_search_set_roots",
-           "az_search_run", "az_search_root", "az_search_root_visits", "az_search_advance", "az_search_root_positions", "az_search_tree", "az_search_launches_per_step")
+           "az_search_run", "az_search_run_async", "az_search_wait", "az_search_root", "az_search_root_visits", "az_search_advance", "az_search_root_positions", "az_search_tree", "az_search_launches_per_step")
 
 
 class az_arch(ctypes.Structure):
@@ -119,6 +119,10 @@ def _load_library():
     lib.az_search_set_roots.argtypes = [vp, vp]
     lib.az_search_run.restype = ci
     lib.az_search_run.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_float)]
+    lib.az_search_run_async.restype = ci
+    lib.az_search_run_async.argtypes = [vp, ci]
+    lib.az_search_wait.restype = ci
+    lib.az_search_wait.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.az_search_root.restype = ci
     lib.az_search_root.argtypes = [vp, ci, vp, vp, vp, vp, ctypes.POINTER(ctypes.c_int32)]
     lib.az_search_root_visits.restype = ci
@@ -386,6 +390,17 @@ def az_search_run(search: Search, simulations: int) -> float:
     """Runs `simulations` steps on every tree; returns the device time in milliseconds."""
     ms = ctypes.c_float(0)
     _check(_lib.az_search_run(search.handle, simulations, ctypes.byref(ms)), "az_search_run")
+    return float(ms.value)
+
+
+def az_search_run_async(search: Search, simulations: int):
+    """Queues `simulations` steps on every tree and returns; az_search_wait collects them."""
+    _check(_lib.az_search_run_async(search.handle, simulations), "az_search_run_async")
+
+
+def az_search_wait(search: Search) -> float:
+    ms = ctypes.c_float(0)
+    _check(_lib.az_search_wait(search.handle, ctypes.byref(ms)), "az_search_wait")
     return float(ms.value)
 
 

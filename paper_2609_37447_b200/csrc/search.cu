@@ -554,6 +554,7 @@ struct Search {
     unsigned char *roots_stage = nullptr;        // device copy of the root records
     int *out_actions = nullptr, *out_visits = nullptr, *out_counts = nullptr;   // read-out of all roots
     bool need_root_step = true;                  // some tree's root still waits for its evaluation
+    bool pending = false;                        // az_search_run_async has queued steps that az_search_wait has not collected
     // played moves: the kept subtrees are written to a second set of pools, which then becomes the first
     Node *alt_nodes = nullptr; Edge *alt_edges = nullptr; unsigned char *alt_node_pos = nullptr; u64 *alt_node_hash = nullptr;
     int *remap = nullptr;                        // [games][2][max_nodes]: old index of every kept node, edge that leads to it
@@ -562,6 +563,7 @@ struct Search {
 
 void free_search(Search *s) {
     if (!s) return;
+    if (s->pending && s->ev_end) cudaEventSynchronize(s->ev_end);       // queued steps still use what is freed below
     cudaFree(s->trees.nodes); cudaFree(s->trees.edges); cudaFree(s->trees.node_pos); cudaFree(s->trees.games);
     cudaFree(s->trees.node_hash); cudaFree(s->trees.hist_hash); cudaFree(s->trees.hist_rep); cudaFree(s->alt_node_hash);
     cudaFree(s->roots_stage);
@@ -903,6 +905,7 @@ void az_search_destroy(az_search *search) { az::free_search(reinterpret_cast<Sea
 int az_search_set_roots(az_search *search, const void *positions_host) {
     Search *s = reinterpret_cast<Search *>(search);
     if (!s || !positions_host) return AZ_ERR_BAD_ARG;
+    if (s->pending) return AZ_ERR_BUSY;
     const az::Trees &t = s->trees;
     cudaStream_t st = s->groups[0].stream;
     AZ_CUDA(cudaMemcpyAsync(s->roots_stage, positions_host, (size_t)s->cfg.games * t.stride, cudaMemcpyHostToDevice, st));
@@ -921,9 +924,10 @@ int az_search_set_roots(az_search *search, const void *positions_host) {
     return AZ_OK;
 }
 
-int az_search_run(az_search *search, int simulations, float *elapsed_ms_out) {
+int az_search_run_async(az_search *search, int simulations) {
     Search *s = reinterpret_cast<Search *>(search);
     if (!s || simulations < 0) return AZ_ERR_BAD_ARG;
+    if (s->pending) return AZ_ERR_BUSY;
     cudaStream_t s0 = s->groups[0].stream;
     cudaStream_t s1 = s->n_groups == 2 ? s->groups[1].stream : s0;
     AZ_CUDA(cudaEventRecord(s->ev_begin, s0));
@@ -941,6 +945,14 @@ int az_search_run(az_search *search, int simulations, float *elapsed_ms_out) {
     }
     AZ_CUDA(cudaEventRecord(s->ev_end, s0));
     s->need_root_step = false;
+    s->pending = true;
+    return AZ_OK;
+}
+
+int az_search_wait(az_search *search, float *elapsed_ms_out) {
+    Search *s = reinterpret_cast<Search *>(search);
+    if (!s || !s->pending) return AZ_ERR_BAD_ARG;
+    s->pending = false;
     AZ_CUDA(cudaEventSynchronize(s->ev_end));
     if (elapsed_ms_out) AZ_CUDA(cudaEventElapsedTime(elapsed_ms_out, s->ev_begin, s->ev_end));
     if (s->net) {
@@ -951,11 +963,17 @@ int az_search_run(az_search *search, int simulations, float *elapsed_ms_out) {
     return AZ_OK;
 }
 
+int az_search_run(az_search *search, int simulations, float *elapsed_ms_out) {
+    const int rc = az_search_run_async(search, simulations);
+    return rc != AZ_OK ? rc : az_search_wait(search, elapsed_ms_out);
+}
+
 int az_search_root(az_search *search, int game, int32_t *actions_host, int32_t *visits_host, float *w_host,
                    float *prior_host, int32_t *count_out) {
     Search *s = reinterpret_cast<Search *>(search);
     if (!s || game < 0 || (uint32_t)game >= s->cfg.games || !actions_host || !visits_host || !w_host || !prior_host || !count_out)
         return AZ_ERR_BAD_ARG;
+    if (s->pending) return AZ_ERR_BUSY;
     az::Node root;
     AZ_CUDA(cudaMemcpy(&root, s->trees.nodes + (size_t)game * s->trees.node_cap, sizeof root, cudaMemcpyDeviceToHost));
     const int k = root.n_edges > 0 ? (root.n_edges < AZ_MAX_LEGAL ? root.n_edges : AZ_MAX_LEGAL) : 0;
@@ -970,6 +988,7 @@ int az_search_root(az_search *search, int game, int32_t *actions_host, int32_t *
 int az_search_root_visits(az_search *search, int32_t *actions_host, int32_t *visits_host, int32_t *counts_host) {
     Search *s = reinterpret_cast<Search *>(search);
     if (!s || !actions_host || !visits_host || !counts_host) return AZ_ERR_BAD_ARG;
+    if (s->pending) return AZ_ERR_BUSY;
     cudaStream_t st = s->groups[0].stream;
     const size_t G = s->cfg.games;
     az::gather_roots_kernel<<<(unsigned)G, 64, 0, st>>>(s->trees, (int)G, s->out_actions, s->out_visits, s->out_counts);
@@ -984,6 +1003,7 @@ int az_search_root_visits(az_search *search, int32_t *actions_host, int32_t *vis
 int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *played_host) {
     Search *s = reinterpret_cast<Search *>(search);
     if (!s) return AZ_ERR_BAD_ARG;
+    if (s->pending) return AZ_ERR_BUSY;
     az::Trees &t = s->trees;
     const size_t G = s->cfg.games;
     cudaStream_t st = s->groups[0].stream;
@@ -1017,6 +1037,7 @@ int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *p
 int az_search_root_positions(az_search *search, void *positions_host) {
     Search *s = reinterpret_cast<Search *>(search);
     if (!s || !positions_host) return AZ_ERR_BAD_ARG;
+    if (s->pending) return AZ_ERR_BUSY;
     const az::Trees &t = s->trees;
     AZ_CUDA(cudaMemcpy2D(positions_host, (size_t)t.stride, t.node_pos, (size_t)t.node_cap * t.stride, (size_t)t.stride,
                          (size_t)s->cfg.games, cudaMemcpyDeviceToHost));
@@ -1026,6 +1047,7 @@ int az_search_root_positions(az_search *search, void *positions_host) {
 int az_search_tree(az_search *search, int game, int32_t *counts_out, int32_t *node_visits_host, float *node_value_sum_host) {
     Search *s = reinterpret_cast<Search *>(search);
     if (!s || game < 0 || (uint32_t)game >= s->cfg.games || !counts_out) return AZ_ERR_BAD_ARG;
+    if (s->pending) return AZ_ERR_BUSY;
     az::GameState gs;
     AZ_CUDA(cudaMemcpy(&gs, s->trees.games + game, sizeof gs, cudaMemcpyDeviceToHost));
     counts_out[0] = gs.n_nodes; counts_out[1] = gs.n_edges; counts_out[2] = gs.flags; counts_out[3] = gs.idle;

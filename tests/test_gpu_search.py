@@ -459,6 +459,32 @@ def test_search_over_the_residual_tower_configs(in_planes, head, value_head, pre
     az.az_free_net(net)
 
 
+def test_run_in_two_halves():
+    import paper_2609_37447_b200 as az
+    rec = records(2, 128, 16, 20261020)
+    cfg = az.make_search_config(16, 2, 128, leaves=2, groups=2, max_nodes=500, evaluator=az.AZ_SEARCH_EVAL_STANDIN, seed=5)
+    a, b = az.az_search_create(None, cfg), az.az_search_create(None, cfg)
+    for s in (a, b):
+        az.az_search_set_roots(s, rec)
+    az.az_search_run(a, 200)
+    az.az_search_run_async(b, 200)
+    for call in (lambda: az.az_search_root(b, 0), lambda: az.az_search_advance(b), lambda: az.az_search_run_async(b, 1),
+                 lambda: az.az_search_set_roots(b, rec), lambda: az.az_search_tree(b, 0)):
+        with pytest.raises(az.AzError) as e:
+            call()
+        assert e.value.code == az.AZ_ERR_BUSY
+    assert az.az_search_wait(b) > 0
+    with pytest.raises(az.AzError) as e:
+        az.az_search_wait(b)
+    assert e.value.code == az.AZ_ERR_BAD_ARG
+    for g in range(16):
+        x, y = read_gpu_tree(az, a, g), read_gpu_tree(az, b, g)
+        assert all(np.atleast_1d(u).tobytes() == np.atleast_1d(v).tobytes() for u, v in zip(x, y))
+    az.az_search_run_async(b, 50)                     # destroying a search with a run pending waits for it
+    az.az_search_destroy(b)
+    az.az_search_destroy(a)
+
+
 def test_bad_arguments():
     import paper_2609_37447_b200 as az
     for kw in ({"leaves": 17}, {"groups": 3}, {"max_nodes": 1}):
