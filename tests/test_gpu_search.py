@@ -459,6 +459,33 @@ def test_search_over_the_residual_tower_configs(in_planes, head, value_head, pre
     az.az_free_net(net)
 
 
+def test_degenerate_runs():
+    """No steps at all (only the roots are evaluated), a single game with the maximum number of leaves, roots set anew."""
+    import paper_2609_37447_b200 as az
+    rec = records(2, 128, 9, 20261030)
+    s = az.az_search_create(None, az.make_search_config(9, 2, 128, leaves=az.AZ_SEARCH_MAX_LEAVES, groups=2, max_nodes=600,
+                                                        evaluator=az.AZ_SEARCH_EVAL_STANDIN, seed=4))
+    az.az_search_set_roots(s, rec)
+    az.az_search_run(s, 0)
+    for g in range(9):
+        want = oracle.mcts_search(rec[g:g + 1], 2, 0, leaves=16, seed=4, node_cap=600)
+        same_tree(read_gpu_tree(az, s, g), want, f"game {g}")
+        assert want["n_nodes"] == 1 and want["visits"].sum() == 0
+    az.az_search_run(s, 30)
+    az.az_search_set_roots(s, rec[::-1].copy())              # new roots: the old trees are gone
+    az.az_search_run(s, 20)
+    for g in range(9):
+        want = oracle.mcts_search(rec[8 - g:9 - g], 2, 20, leaves=16, seed=4, node_cap=600)
+        same_tree(read_gpu_tree(az, s, g), want, f"game {g} after the reset")
+    az.az_search_destroy(s)
+    one = az.az_search_create(None, az.make_search_config(1, 2, 128, leaves=16, groups=2, max_nodes=900,
+                                                          evaluator=az.AZ_SEARCH_EVAL_STANDIN, seed=4))
+    az.az_search_set_roots(one, rec[:1])
+    az.az_search_run(one, 50)
+    same_tree(read_gpu_tree(az, one, 0), oracle.mcts_search(rec[:1], 2, 50, leaves=16, seed=4, node_cap=900), "one game")
+    az.az_search_destroy(one)
+
+
 def test_run_in_two_halves():
     import paper_2609_37447_b200 as az
     rec = records(2, 128, 16, 20261020)
