@@ -817,7 +817,9 @@ tower_tc_kernel(const TowerArgs args) {
                 ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 acc_phase ^= 1u;
-                if (set != 0) continue;                               // the head's rows are few: set 0 writes them all
+                // the residual towers' head rows are few: set 0 writes them all; the paper network's sixteen slices of
+                // queries and keys are dealt out over the sets
+                if (!kPnet && set != 0) continue;
                 ptx::tc_fence_after();
                 const float *hb = head_bias_smem;
                 // this row's place in the GEMM A tiles: [tile of 128 boards][8-wide K chunk][board/8][board%8][8 k]
@@ -825,7 +827,7 @@ tower_tc_kernel(const TowerArgs args) {
                 const int n_slices = head_n / 16;
                 const int value_slice0 = n_slices - 2;               // the value projection is the last 32 columns
 #pragma unroll 1
-                for (int j = 0; j < n_slices; ++j) {
+                for (int j = kPnet ? set : 0; j < n_slices; j += kPnet ? S::kSets : 1) {
                     uint32_t rr[16];
                     ptx::tmem_ld16(t_lane + (kPnet ? 0u : (uint32_t)kC) + (uint32_t)(j * 16), rr);
                     ptx::tmem_ld_wait();
