@@ -325,10 +325,18 @@ def run_search(args, name):
         az.az_search_advance(s)
         barrier()
         t0 = time.perf_counter()
-        run_ms, moved = 0.0, 0
+        run_ms, moved, restarted, spare_at = 0.0, 0, 0, 0
+        spare = make_records(cfg, games, first_index=sharding.rank_first_index(rank, games) + world * games)
         for _ in range(args.moves):
             run_ms += az.az_search_run(s, args.steps)
-            moved += int((az.az_search_advance(s) >= 0).sum())
+            played = az.az_search_advance(s)
+            moved += int((played >= 0).sum())
+            over = np.flatnonzero(played < 0)                   # the game has ended: the next one starts in its place
+            if over.size:
+                pick = (spare_at + np.arange(over.size)) % games
+                az.az_search_replace_roots(s, over, np.ascontiguousarray(spare[pick]))
+                spare_at = int((spare_at + over.size) % games)
+                restarted += int(over.size)
         play_s = time.perf_counter() - t0
         barrier()
         flags_play, kept = 0, []
@@ -337,11 +345,12 @@ def run_search(args, name):
             flags_play |= int(c[2])
             kept.append(int(c[0]))
         az.az_search_destroy(s)
-        play = {"moves_per_game": args.moves, "moves_played": moved, "searches_per_s": games * leaves * args.steps * args.moves / play_s,
+        play = {"moves_per_game": args.moves, "moves_played": moved, "games_restarted": restarted, "searches_per_s": games * leaves * args.steps * args.moves / play_s,
                 "moves_per_s": moved / play_s, "ms_per_move_all_games": 1e3 * play_s / args.moves,
                 "ms_in_search_per_move": run_ms / args.moves, "tree_flags": flags_play,
                 "kept_nodes_median": float(np.median(kept)),
-                "note": "wall clock over az_search_run + az_search_advance per move; every traversal of a step counted"}
+                "note": "wall clock over az_search_run + az_search_advance (+ az_search_replace_roots for games that ended) per move; "
+                        "every traversal of a step counted"}
 
     ms_max, e2e_ms = sharding.max_over_ranks([ms, e2e_s * 1e3], device="cuda")
     if rank == 0:

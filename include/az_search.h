@@ -122,6 +122,15 @@ void az_search_destroy(az_search *search);
 int az_search_set_roots(az_search *search, const void *positions_host);
 
 /*
+ * New searches in some of the games only (a game is over, the next one starts in its place; Sec. 5.1: an actor
+ * keeps its games interleaved): games_host lists `count` game indices, positions_host holds their new root
+ * records in the same order.  Those trees are emptied and their histories of earlier positions forgotten; the
+ * other games are untouched.  A game listed twice takes one of its records.
+ * Errors: BAD_ARG (an index out of range, count above the number of games), BUSY, CUDA.  count == 0 is a no-op.
+ */
+int az_search_replace_roots(az_search *search, const int32_t *games_host, int count, const void *positions_host);
+
+/*
  * Runs `simulations` more steps on every tree (the first call after az_search_set_roots runs the
  * roots' own evaluation first) and waits for them.  One step of a tree is `leaves` traversals
  * that all choose their paths before any of the step's results are backed up.

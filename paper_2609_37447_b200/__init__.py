@@ -27,7 +27,7 @@ EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_siz
            "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_submit_host", "az_wait_host", "az_encode", "az_encode52", "az_tower", "az_tower_static", "az_legal_masks",
            "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error",
-           "az_apply_moves", "az_standin_evaluate", "az_search_create", "az_search_destroy", "az_search_set_roots",
+           "az_apply_moves", "az_standin_evaluate", "az_search_create", "az_search_destroy", "az_search_set_roots", "az_search_replace_roots",
            "az_search_run", "az_search_run_async", "az_search_wait", "az_search_root", "az_search_root_visits", "az_search_advance", "az_search_root_positions", "az_search_tree", "az_search_launches_per_step")
 
 
@@ -117,6 +117,8 @@ def _load_library():
     lib.az_search_destroy.argtypes = [vp]
     lib.az_search_set_roots.restype = ci
     lib.az_search_set_roots.argtypes = [vp, vp]
+    lib.az_search_replace_roots.restype = ci
+    lib.az_search_replace_roots.argtypes = [vp, vp, ci, vp]
     lib.az_search_run.restype = ci
     lib.az_search_run.argtypes = [vp, ci, ctypes.POINTER(ctypes.c_float)]
     lib.az_search_run_async.restype = ci
@@ -384,6 +386,15 @@ def az_search_set_roots(search: Search, positions_host: np.ndarray):
     if rec.nbytes != search.config.games * search.config.position_bytes:
         raise ValueError("positions_host must hold one record per game")
     _check(_lib.az_search_set_roots(search.handle, rec.ctypes.data), "az_search_set_roots")
+
+
+def az_search_replace_roots(search: Search, games, positions_host: np.ndarray):
+    """New root records for the listed games only (their trees are emptied); the other games go on."""
+    idx = np.ascontiguousarray(games, dtype=np.int32)
+    rec = np.ascontiguousarray(positions_host)
+    if rec.nbytes != idx.size * search.config.position_bytes:
+        raise ValueError("one record per listed game expected")
+    _check(_lib.az_search_replace_roots(search.handle, idx.ctypes.data, int(idx.size), rec.ctypes.data), "az_search_replace_roots")
 
 
 def az_search_run(search: Search, simulations: int) -> float:

@@ -582,9 +582,10 @@ void free_search(Search *s) {
     delete s;
 }
 
-__global__ void reset_trees_kernel(Trees t, const unsigned char *__restrict__ roots, int games) {
-    const int g = blockIdx.x;
-    if (g >= games) return;
+// New trees: block b empties game index[b] (game b without an index) and gives it root record b.
+__global__ void reset_trees_kernel(Trees t, const unsigned char *__restrict__ roots, int count, const int *__restrict__ index) {
+    if ((int)blockIdx.x >= count) return;
+    const int g = index ? index[blockIdx.x] : (int)blockIdx.x;
     if (threadIdx.x == 0) {
         GameState gs{};
         gs.n_nodes = 1;
@@ -593,7 +594,7 @@ __global__ void reset_trees_kernel(Trees t, const unsigned char *__restrict__ ro
         root.n_edges = -1;
         t.nodes[(size_t)g * t.node_cap] = root;
     }
-    const u64 *src = reinterpret_cast<const u64 *>(roots + (size_t)g * t.stride);
+    const u64 *src = reinterpret_cast<const u64 *>(roots + (size_t)blockIdx.x * t.stride);
     u64 *dst = reinterpret_cast<u64 *>(t.node_pos + (size_t)g * t.node_cap * t.stride);
     for (int i = threadIdx.x; i < t.stride / 8; i += blockDim.x) dst[i] = src[i];
     if (threadIdx.x == 0) t.node_hash[(size_t)g * t.node_cap] = position_key(src, kRepSeed);
@@ -909,7 +910,7 @@ int az_search_set_roots(az_search *search, const void *positions_host) {
     const az::Trees &t = s->trees;
     cudaStream_t st = s->groups[0].stream;
     AZ_CUDA(cudaMemcpyAsync(s->roots_stage, positions_host, (size_t)s->cfg.games * t.stride, cudaMemcpyHostToDevice, st));
-    az::reset_trees_kernel<<<s->cfg.games, 32, 0, st>>>(t, s->roots_stage, (int)s->cfg.games);
+    az::reset_trees_kernel<<<s->cfg.games, 32, 0, st>>>(t, s->roots_stage, (int)s->cfg.games, nullptr);
     AZ_LAUNCH_CHECK();
     // the rows of every group's batch must hold valid records from the first step on (rows that idle are still evaluated)
     for (int gi = 0; gi < s->n_groups; ++gi) {
@@ -919,6 +920,25 @@ int az_search_set_roots(az_search *search, const void *positions_host) {
                                       s->roots_stage + (size_t)g.game0 * t.stride, (size_t)t.stride, (size_t)t.stride,
                                       (size_t)g.n_games, cudaMemcpyDeviceToDevice, st));
     }
+    AZ_CUDA(cudaStreamSynchronize(st));
+    s->need_root_step = true;
+    return AZ_OK;
+}
+
+int az_search_replace_roots(az_search *search, const int32_t *games_host, int count, const void *positions_host) {
+    Search *s = reinterpret_cast<Search *>(search);
+    if (!s || count < 0 || (uint32_t)count > s->cfg.games) return AZ_ERR_BAD_ARG;
+    if (count == 0) return AZ_OK;
+    if (!games_host || !positions_host) return AZ_ERR_BAD_ARG;
+    if (s->pending) return AZ_ERR_BUSY;
+    for (int i = 0; i < count; ++i)
+        if (games_host[i] < 0 || (uint32_t)games_host[i] >= s->cfg.games) return AZ_ERR_BAD_ARG;
+    const az::Trees &t = s->trees;
+    cudaStream_t st = s->groups[0].stream;
+    AZ_CUDA(cudaMemcpyAsync(s->roots_stage, positions_host, (size_t)count * t.stride, cudaMemcpyHostToDevice, st));
+    AZ_CUDA(cudaMemcpyAsync(s->out_counts, games_host, (size_t)count * sizeof(int), cudaMemcpyHostToDevice, st));   // borrowed as the index list
+    az::reset_trees_kernel<<<(unsigned)count, 32, 0, st>>>(t, s->roots_stage, count, s->out_counts);
+    AZ_LAUNCH_CHECK();
     AZ_CUDA(cudaStreamSynchronize(st));
     s->need_root_step = true;
     return AZ_OK;

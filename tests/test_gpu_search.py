@@ -486,6 +486,41 @@ def test_degenerate_runs():
     az.az_search_destroy(one)
 
 
+def test_some_games_start_anew_while_the_others_go_on():
+    import paper_2609_37447_b200 as az
+    rec = records(2, 128, 14, 20261040)
+    fresh = records(2, 128, 12, 20261041)[9:12]
+    s = az.az_search_create(None, az.make_search_config(14, 2, 128, leaves=2, groups=2, max_nodes=500, evaluator=az.AZ_SEARCH_EVAL_STANDIN, seed=6))
+    az.az_search_set_roots(s, rec)
+    trees = [oracle.MctsTree(rec[g:g + 1], 2, leaves=2, seed=6, node_cap=500, edge_cap=500 * 64) for g in range(14)]
+    az.az_search_run(s, 60)
+    az.az_search_advance(s)
+    for g in range(14):
+        trees[g].run(60)
+        r = trees[g].read()
+        if len(r["actions"]):
+            trees[g].advance(int(r["actions"][int(np.argmax(r["visits"]))]))
+    picked = [11, 0, 6]
+    az.az_search_replace_roots(s, picked, fresh)
+    for i, g in enumerate(picked):
+        trees[g].close()
+        trees[g] = oracle.MctsTree(fresh[i:i + 1], 2, leaves=2, seed=6, node_cap=500, edge_cap=500 * 64)
+    az.az_search_run(s, 45)
+    roots = az.az_search_root_positions(s, rec.dtype)
+    for g in range(14):
+        trees[g].run(45)
+        want = trees[g].read()
+        same_tree(read_gpu_tree(az, s, g), want, f"game {g}")
+        assert (roots[g:g + 1].view(np.uint8) == want["root"].view(np.uint8)).all()
+    with pytest.raises(az.AzError) as e:
+        az.az_search_replace_roots(s, [14], fresh[:1])
+    assert e.value.code == az.AZ_ERR_BAD_ARG
+    az.az_search_replace_roots(s, [], fresh[:0])
+    az.az_search_destroy(s)
+    for t in trees:
+        t.close()
+
+
 def test_run_in_two_halves():
     import paper_2609_37447_b200 as az
     rec = records(2, 128, 16, 20261020)
