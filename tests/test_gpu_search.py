@@ -549,6 +549,28 @@ def test_run_in_two_halves():
 
 def test_bad_arguments():
     import paper_2609_37447_b200 as az
+    # az_apply_moves: empty batches are no-ops, in == out and unknown strides or lists are refused
+    rec = records(2, 128, 9, 20261050)
+    pos = az.records_to_device(rec)
+    out = torch.zeros_like(pos)
+    act = torch.zeros(9, dtype=torch.int32, device="cuda")
+    az.az_apply_moves(pos, 128, 0, 2, act, out)
+    for args in ((pos, 128, 9, 2, act, pos), (pos, 120, 9, 2, act, out), (pos, 128, 9, 3, act, out), (pos, 128, -1, 2, act, out)):
+        with pytest.raises(az.AzError) as e:
+            az.az_apply_moves(*args)
+        assert e.value.code == az.AZ_ERR_BAD_ARG
+    masks = torch.zeros((9, 30), dtype=torch.int64, device="cuda")
+    legal = torch.zeros((9, az.AZ_MAX_LEGAL), device="cuda")
+    counts = torch.zeros(9, dtype=torch.int32, device="cuda")
+    value = torch.zeros(9, device="cuda")
+    az.az_standin_evaluate(pos, 128, masks, 0, 2, 1, legal, counts, value)
+    with pytest.raises(az.AzError) as e:
+        az.az_standin_evaluate(pos, 100, masks, 9, 2, 1, legal, counts, value)
+    assert e.value.code == az.AZ_ERR_BAD_ARG
+    # an all-zero mask row is a position without moves: count 0, the value still comes
+    az.az_standin_evaluate(pos, 128, masks, 9, 2, 1, legal, counts, value)
+    torch.cuda.synchronize()
+    assert (counts.cpu().numpy() == 0).all() and (value.cpu().numpy() != 0).any()
     for kw in ({"leaves": 17}, {"groups": 3}, {"max_nodes": 1}):
         with pytest.raises(az.AzError) as e:
             az.az_search_create(None, az.make_search_config(4, 2, 128, evaluator=az.AZ_SEARCH_EVAL_STANDIN, **kw))
