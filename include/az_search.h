@@ -125,8 +125,9 @@ int az_search_set_roots(az_search *search, const void *positions_host);
  * New searches in some of the games only (a game is over, the next one starts in its place; Sec. 5.1: an actor
  * keeps its games interleaved): games_host lists `count` game indices, positions_host holds their new root
  * records in the same order.  Those trees are emptied and their histories of earlier positions forgotten; the
- * other games are untouched.  A game listed twice takes one of its records.
- * Errors: BAD_ARG (an index out of range, count above the number of games), BUSY, CUDA.  count == 0 is a no-op.
+ * other games are untouched.
+ * Errors: BAD_ARG (an index out of range or listed twice, count above the number of games), BUSY, CUDA.
+ * count == 0 is a no-op.
  */
 int az_search_replace_roots(az_search *search, const int32_t *games_host, int count, const void *positions_host);
 
@@ -175,7 +176,7 @@ int az_search_root_visits(az_search *search, int32_t *actions_host, int32_t *vis
  * AZ_SEARCH_FLAG_BAD_ACTION) keeps its tree.  played_host (may be NULL) receives the action played per game,
  * -1 where none was.  Keeping only a share of the old visits (the paper's 60 %) is self-play's recipe and is
  * not applied.  The first call allocates a second set of tree pools (the kept subtrees are copied there).
- * Errors: BAD_ARG, CUDA.
+ * Errors: BAD_ARG, BUSY, CUDA.
  */
 int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *played_host);
 

@@ -15,6 +15,7 @@
 #include <mutex>
 #include <new>
 #include <utility>
+#include <vector>
 
 namespace az {
 namespace {
@@ -931,8 +932,13 @@ int az_search_replace_roots(az_search *search, const int32_t *games_host, int co
     if (count == 0) return AZ_OK;
     if (!games_host || !positions_host) return AZ_ERR_BAD_ARG;
     if (s->pending) return AZ_ERR_BUSY;
-    for (int i = 0; i < count; ++i)
-        if (games_host[i] < 0 || (uint32_t)games_host[i] >= s->cfg.games) return AZ_ERR_BAD_ARG;
+    {
+        std::vector<bool> seen(s->cfg.games, false);
+        for (int i = 0; i < count; ++i) {
+            if (games_host[i] < 0 || (uint32_t)games_host[i] >= s->cfg.games || seen[games_host[i]]) return AZ_ERR_BAD_ARG;
+            seen[games_host[i]] = true;
+        }
+    }
     const az::Trees &t = s->trees;
     cudaStream_t st = s->groups[0].stream;
     AZ_CUDA(cudaMemcpyAsync(s->roots_stage, positions_host, (size_t)count * t.stride, cudaMemcpyHostToDevice, st));

@@ -515,6 +515,9 @@ def test_some_games_start_anew_while_the_others_go_on():
     with pytest.raises(az.AzError) as e:
         az.az_search_replace_roots(s, [14], fresh[:1])
     assert e.value.code == az.AZ_ERR_BAD_ARG
+    with pytest.raises(az.AzError) as e:
+        az.az_search_replace_roots(s, [3, 3], fresh[:2])
+    assert e.value.code == az.AZ_ERR_BAD_ARG
     az.az_search_replace_roots(s, [], fresh[:0])
     az.az_search_destroy(s)
     for t in trees:
