@@ -81,6 +81,8 @@ def _load():
         lib.orc_mcts_advance.argtypes = [vp, ci]
         lib.orc_mcts_read.restype = ci
         lib.orc_mcts_read.argtypes = [vp] * 9
+        lib.orc_mcts_root_noise.restype = ci
+        lib.orc_mcts_root_noise.argtypes = [vp, vp, ctypes.c_float]
         lib.orc_mcts_node.restype = ci
         lib.orc_mcts_node.argtypes = [vp, ci, vp, vp]
         lib.orc_mcts_free.restype = None
@@ -232,6 +234,12 @@ class MctsTree:
         return {"actions": actions[:k].copy(), "visits": visits[:k].copy(), "w": w[:k].copy(), "prior": prior[:k].copy(),
                 "n_nodes": int(counts[0]), "n_edges": int(counts[1]), "flags": int(counts[2]), "idle": int(counts[3]),
                 "node_nvis": nvis[:counts[0]].copy(), "node_wsum": wsum[:counts[0]].copy(), "root": root}
+
+    def root_noise(self, noise, epsilon: float) -> int:
+        """Mixes caller-drawn noise into the priors of the current root's edges; returns how many edges changed."""
+        eta = np.ascontiguousarray(noise, dtype=np.float32)
+        assert eta.size >= 256
+        return int(_load().orc_mcts_root_noise(self.handle, eta.ctypes.data, epsilon))
 
     def node(self, index: int):
         """(record, parent index) of one node, for inspection."""

@@ -20,6 +20,9 @@
  *  - a node is terminal if the mover has no legal move (value -1 in check, else 0), if the halfmove
  *    clock has reached 100 or if the position has occurred twice before (value 0);
  *  - the root's evaluation is a step of its own before the counted simulations;
+ *  - root noise, when the caller asks for it, replaces the priors of the root's edges by (1 - epsilon) P +
+ *    epsilon * noise with noise values the caller has drawn; it is applied to the current root as it stands
+ *    (a kept subtree's root included) and stays with those edges;
  *  - when a move is played (Sec. 3.3: the relevant subtree becomes the next root) the subtree under the
  *    root's edge of that action is kept with all its statistics and renumbered breadth-first (a node's
  *    children in the order of its edges), everything else is dropped; if that edge has no child yet the
@@ -315,6 +318,25 @@ int orc_mcts_read(const void *tree, int32_t *root_actions, int32_t *root_visits,
                   int32_t *counts, int32_t *node_nvis, float *node_wsum, void *root_record) {
     return tree_read((const Tree *)tree, root_actions, root_visits, root_w, root_prior, counts, node_nvis, node_wsum, root_record);
 }
+/* Root noise (Sec. 3.4: noise added to the root prior makes games consider different continuations; App. D.2:
+ * Dirichlet with epsilon 0.25, alpha 0.3).  The noise itself is drawn by the caller and passed in: the priors of
+ * the root's edges become (1 - epsilon) * P + epsilon * noise[i], i the edge's place among the root's edges,
+ * in float32 with one rounding per operation.  Returns the number of edges changed (0 if the root has not
+ * been evaluated yet or has no moves). */
+int orc_mcts_root_noise(void *tree, const float *noise, float epsilon) {
+    Tree *t = (Tree *)tree;
+    if (!t) return -1;
+    const Node *root = &t->nodes[0];
+    const float keep = 1.0f - epsilon;
+    for (int i = 0; i < root->n_edges; ++i) {
+        Edge *e = &t->edges[root->edge_begin + i];
+        const float a = keep * e->prior;
+        const float b = epsilon * noise[i];
+        e->prior = a + b;
+    }
+    return root->n_edges > 0 ? root->n_edges : 0;
+}
+
 /* One node, for inspection: its record and its parent's index (-1 for the root).  Returns 0, -1 if there is no such node. */
 int orc_mcts_node(const void *tree, int index, void *record_out, int32_t *parent_out) {
     const Tree *t = (const Tree *)tree;

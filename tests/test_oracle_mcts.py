@@ -251,3 +251,29 @@ def test_repetition_counts_inside_a_tree_against_a_brute_force_walk():
                 assert i not in parents_with_children                     # a drawn node is never expanded
         t.close()
     assert repeated >= 10
+
+
+def test_root_noise_mixes_into_the_root_priors_only():
+    rec = positions.record_from_fen(START)
+    t = oracle.MctsTree(rec, 2, seed=2, node_cap=400)
+    assert t.root_noise(np.zeros(256, dtype=np.float32), 0.25) == 0             # the root has not been evaluated yet
+    t.run(0)
+    before = t.read()["prior"]
+    eta = np.random.default_rng(5).dirichlet([0.3] * 20).astype(np.float32)     # App. D.2: alpha 0.3
+    noise = np.zeros(256, dtype=np.float32)
+    noise[:20] = eta
+    assert t.root_noise(noise, 0.25) == 20
+    after = t.read()["prior"]
+    want = (np.float32(0.75) * before).astype(np.float32) + (np.float32(0.25) * eta).astype(np.float32)
+    assert (after.view(np.uint32) == want.view(np.uint32)).all() and abs(float(after.sum()) - 1) < 1e-5
+    # the search follows the noisy priors: its first traversal takes the largest of them
+    t.run(1)
+    r = t.read()
+    assert r["visits"][int(np.argmax(after))] == 1
+    # epsilon 0 changes nothing; the noise stays at the root's edges and nowhere else
+    t2 = oracle.MctsTree(rec, 2, seed=2, node_cap=400)
+    t2.run(0)
+    t2.root_noise(noise, 0.0)
+    assert (t2.read()["prior"].view(np.uint32) == before.view(np.uint32)).all()
+    t.close()
+    t2.close()
