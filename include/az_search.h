@@ -180,6 +180,18 @@ int az_search_root_visits(az_search *search, int32_t *actions_host, int32_t *vis
  */
 int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *played_host);
 
+/*
+ * Root noise (Sec. 3.4: "noise added to the root prior makes games consider different continuations"; App. D.2:
+ * Dirichlet, epsilon 0.25, alpha 0.3).  The noise is the caller's (drawn on the host, any distribution):
+ * noise_host is [games][AZ_MAX_LEGAL] float32, entry i of row g belonging to the i-th move of game g's current
+ * root (ascending policy index); the priors of those edges become (1 - epsilon) P + epsilon * noise, in
+ * float32 with one rounding per operation, and stay with the edges.  Applies to the root as it stands, a kept
+ * subtree's root included; a root that has not been evaluated yet (run az_search_run(search, 0) first) or has
+ * no moves is left alone.  changed_host (may be NULL) receives per game the number of edges changed.
+ * Errors: BAD_ARG (epsilon outside [0, 1]), BUSY, CUDA.
+ */
+int az_search_root_noise(az_search *search, const float *noise_host, float epsilon, int32_t *changed_host);
+
 /* The current root records of all games, to a host buffer of games * position_bytes. */
 int az_search_root_positions(az_search *search, void *positions_host);
 

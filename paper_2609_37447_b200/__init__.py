@@ -28,7 +28,7 @@ EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_siz
            "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error",
            "az_apply_moves", "az_standin_evaluate", "az_search_create", "az_search_destroy", "az_search_set_roots", "az_search_replace_roots",
-           "az_search_run", "az_search_run_async", "az_search_wait", "az_search_root", "az_search_root_visits", "az_search_advance", "az_search_root_positions", "az_search_tree", "az_search_launches_per_step")
+           "az_search_run", "az_search_run_async", "az_search_wait", "az_search_root", "az_search_root_visits", "az_search_advance", "az_search_root_noise", "az_search_root_positions", "az_search_tree", "az_search_launches_per_step")
 
 
 class az_arch(ctypes.Structure):
@@ -131,6 +131,8 @@ def _load_library():
     lib.az_search_root_visits.argtypes = [vp, vp, vp, vp]
     lib.az_search_advance.restype = ci
     lib.az_search_advance.argtypes = [vp, vp, vp]
+    lib.az_search_root_noise.restype = ci
+    lib.az_search_root_noise.argtypes = [vp, vp, ctypes.c_float, vp]
     lib.az_search_root_positions.restype = ci
     lib.az_search_root_positions.argtypes = [vp, vp]
     lib.az_search_tree.restype = ci
@@ -448,6 +450,17 @@ def az_search_advance(search: Search, actions_host=None) -> np.ndarray:
             raise ValueError("one action per game expected")
     _check(_lib.az_search_advance(search.handle, act.ctypes.data if act is not None else None, played.ctypes.data), "az_search_advance")
     return played
+
+
+def az_search_root_noise(search: Search, noise_host: np.ndarray, epsilon: float) -> np.ndarray:
+    """Mixes caller-drawn noise ([games][AZ_MAX_LEGAL] float32) into the priors of every game's current root;
+    returns the number of edges changed per game."""
+    eta = np.ascontiguousarray(noise_host, dtype=np.float32)
+    if eta.shape != (search.config.games, AZ_MAX_LEGAL):
+        raise ValueError("noise must be [games][AZ_MAX_LEGAL]")
+    changed = np.zeros(search.config.games, dtype=np.int32)
+    _check(_lib.az_search_root_noise(search.handle, eta.ctypes.data, epsilon, changed.ctypes.data), "az_search_root_noise")
+    return changed
 
 
 def az_search_root_positions(search: Search, dtype) -> np.ndarray:

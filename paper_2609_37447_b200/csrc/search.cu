@@ -738,6 +738,21 @@ search_advance_kernel(Trees t, Node *new_nodes, Edge *new_edges, unsigned char *
     push_history();
 }
 
+// Root noise (Sec. 3.4; App. D.2): P <- (1 - epsilon) P + epsilon * noise on the edges of every game's current
+// root, noise[g][i] belonging to the root's i-th edge; one rounding per operation.  Roots that have not been
+// evaluated yet, or have no moves, are left alone; changed[g] tells how many edges were touched.
+__global__ void root_noise_kernel(Trees t, int games, const float *__restrict__ noise, float epsilon, int *__restrict__ changed) {
+    const int g = blockIdx.x;
+    if (g >= games) return;
+    const Node root = t.nodes[(size_t)g * t.node_cap];
+    const int k = root.n_edges > 0 ? (root.n_edges < AZ_MAX_LEGAL ? root.n_edges : AZ_MAX_LEGAL) : 0;
+    Edge *e = t.edges + (size_t)g * t.edge_cap + root.edge_begin;
+    const float keep = __fsub_rn(1.0f, epsilon);
+    for (int i = threadIdx.x; i < k; i += blockDim.x)
+        e[i].prior = __fadd_rn(__fmul_rn(keep, e[i].prior), __fmul_rn(epsilon, noise[(size_t)g * AZ_MAX_LEGAL + i]));
+    if (threadIdx.x == 0) changed[g] = k;
+}
+
 // root actions and visit counts of every game, in rows of AZ_MAX_LEGAL
 __global__ void gather_roots_kernel(Trees t, int games, int *__restrict__ actions, int *__restrict__ visits, int *__restrict__ counts) {
     const int g = blockIdx.x;
@@ -1057,6 +1072,22 @@ int az_search_advance(az_search *search, const int32_t *actions_host, int32_t *p
     std::swap(t.node_pos, s->alt_node_pos);
     std::swap(t.node_hash, s->alt_node_hash);
     if (fresh) s->need_root_step = true;
+    return AZ_OK;
+}
+
+int az_search_root_noise(az_search *search, const float *noise_host, float epsilon, int32_t *changed_host) {
+    Search *s = reinterpret_cast<Search *>(search);
+    if (!s || !noise_host || !(epsilon >= 0.0f && epsilon <= 1.0f)) return AZ_ERR_BAD_ARG;
+    if (s->pending) return AZ_ERR_BUSY;
+    const size_t G = s->cfg.games;
+    cudaStream_t st = s->groups[0].stream;
+    // the read-out buffers double as staging: visits (int32 [games][AZ_MAX_LEGAL]) holds the noise, counts the answer
+    float *noise_dev = reinterpret_cast<float *>(s->out_visits);
+    AZ_CUDA(cudaMemcpyAsync(noise_dev, noise_host, G * AZ_MAX_LEGAL * sizeof(float), cudaMemcpyHostToDevice, st));
+    az::root_noise_kernel<<<(unsigned)G, 64, 0, st>>>(s->trees, (int)G, noise_dev, epsilon, s->out_counts);
+    AZ_LAUNCH_CHECK();
+    if (changed_host) AZ_CUDA(cudaMemcpyAsync(changed_host, s->out_counts, G * sizeof(int), cudaMemcpyDeviceToHost, st));
+    AZ_CUDA(cudaStreamSynchronize(st));
     return AZ_OK;
 }
 

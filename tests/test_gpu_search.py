@@ -524,6 +524,45 @@ def test_some_games_start_anew_while_the_others_go_on():
         t.close()
 
 
+def test_root_noise_like_the_oracles():
+    """A self-play style loop: evaluate the roots, mix Dirichlet noise (drawn here) into their priors, search, play,
+    and again on the kept subtrees' roots; trees equal the oracle's throughout."""
+    import paper_2609_37447_b200 as az
+    rec = records(2, 128, 11, 20261060)
+    n = rec.shape[0]
+    s = az.az_search_create(None, az.make_search_config(n, 2, 128, leaves=2, groups=2, max_nodes=700, evaluator=az.AZ_SEARCH_EVAL_STANDIN, seed=8))
+    az.az_search_set_roots(s, rec)
+    trees = [oracle.MctsTree(rec[g:g + 1], 2, leaves=2, seed=8, node_cap=700, edge_cap=700 * 64) for g in range(n)]
+    rng = np.random.default_rng(77)
+    early = az.az_search_root_noise(s, np.zeros((n, az.AZ_MAX_LEGAL), dtype=np.float32), 0.25)
+    assert (early == 0).all()                                            # no root has been evaluated yet
+    for move in range(4):
+        az.az_search_run(s, 0)                                           # roots that are new evaluate themselves
+        noise = np.zeros((n, az.AZ_MAX_LEGAL), dtype=np.float32)
+        for g in range(n):
+            trees[g].run(0)
+            k = len(trees[g].read()["actions"])
+            if k:
+                noise[g, :k] = rng.dirichlet([0.3] * k).astype(np.float32)
+        changed = az.az_search_root_noise(s, noise, 0.25)
+        for g in range(n):
+            assert changed[g] == trees[g].root_noise(noise[g], 0.25)
+        az.az_search_run(s, 50)
+        for g in range(n):
+            trees[g].run(50)
+            same_tree(read_gpu_tree(az, s, g), trees[g].read(), f"move {move} game {g}")
+        played = az.az_search_advance(s)
+        for g in range(n):
+            if played[g] >= 0:
+                trees[g].advance(int(played[g]))
+    with pytest.raises(az.AzError) as e:
+        az.az_search_root_noise(s, np.zeros((n, az.AZ_MAX_LEGAL), dtype=np.float32), 1.5)
+    assert e.value.code == az.AZ_ERR_BAD_ARG
+    az.az_search_destroy(s)
+    for t in trees:
+        t.close()
+
+
 def test_run_in_two_halves():
     import paper_2609_37447_b200 as az
     rec = records(2, 128, 16, 20261020)
