@@ -32,6 +32,7 @@ WORKLOADS = {
     "c5": "c5: 40x256 bf16, 112 history planes, flat-1858 policy + WDL value (batch sweep via --batch)",
     "c4": "c4: 20x128 FP8-e4m3 tower (bf16 heads) batch 4096, 73-plane policy + tanh value",
     "c4b": "c4b: c4 with residual branches scaled by 1/sqrt(20)",
+    "c4p": "c4p: c4 as specified (plain weights) with the tower in int8, batch 4096",
     "c4i": "c4i: c4b with the tower in int8 (u8 activations x s8 weights, int32 accumulation), batch 4096",
     "p12": "p12: the paper's own network, 12x128 bf16 batch 1024 (52 planes, capped scaled blocks, pooled context, "
            "query-key policy over 1,880 actions, WDL value)",

@@ -62,6 +62,8 @@ CONFIGS = {
     # precision the paper deploys (Sec. 4.3.6); precision code 3
     "c4i": Config("c4i", 19, 20, 128, 0, 0, 3, 4096, (0, 80), (0, 80), 20260941, 9370002, weights_like="c4b",
                   branch_scale=20 ** -0.5),
+    # c4 as specified (the plain weights of c2) with the tower in int8 instead of e4m3
+    "c4p": Config("c4p", 19, 20, 128, 0, 0, 3, 4096, (0, 80), (0, 80), 20260941, 9370002, weights_like="c2"),
     "c5": Config("c5", 112, 40, 256, 1, 1, 1, 1024, (0, 80), (0, 80), 20260942, 9370005,
                  sweep=(16, 64, 256, 1024, 4096, 8192)),
 }

@@ -681,22 +681,36 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const int C = (int)n->arch.channels, L = n->n_conv;
     const size_t pb = az_position_bytes(&n->arch);
-    // 1. bf16 tower over the calibration positions, recording every layer's per-channel output maximum
+    // 1. bf16 tower over the calibration positions, recording every layer's per-channel output maximum and the sum
+    //    of its pre-activation values (for the bias correction of step 3)
     unsigned int *absmax_dev = nullptr;
+    float *presum_dev = nullptr;
     AZ_CUDA(cudaMalloc((void **)&absmax_dev, (size_t)L * C * sizeof(unsigned int)));
+    if (cudaMalloc((void **)&presum_dev, (size_t)L * C * sizeof(float)) != cudaSuccess) { cudaFree(absmax_dev); return AZ_ERR_CUDA; }
     cudaError_t e = cudaMemsetAsync(absmax_dev, 0, (size_t)L * C * sizeof(unsigned int), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(presum_dev, 0, (size_t)L * C * sizeof(float), s);
     int rc = AZ_OK;
-    for (int first = 0; first < count && rc == AZ_OK && e == cudaSuccess; first += (int)n->arch.max_batch) {
-        const int chunk = count - first < (int)n->arch.max_batch ? count - first : (int)n->arch.max_batch;
-        const unsigned char *p = static_cast<const unsigned char *>(positions_dev) + (size_t)first * pb;
-        rc = az::launch_tower_tc(*n, nullptr, p, chunk, nullptr, false, absmax_dev, s);
-    }
-    std::vector<float> absmax((size_t)L * C);
+    // one pass of the tower (whichever form is ready) over all calibration positions
+    auto tower_pass = [&](unsigned int *absmax_hook) {
+        for (int first = 0; first < count && rc == AZ_OK && e == cudaSuccess; first += (int)n->arch.max_batch) {
+            const int chunk = count - first < (int)n->arch.max_batch ? count - first : (int)n->arch.max_batch;
+            const unsigned char *p = static_cast<const unsigned char *>(positions_dev) + (size_t)first * pb;
+            rc = az::launch_tower_tc(*n, nullptr, p, chunk, nullptr, false, absmax_hook, s);
+        }
+    };
+    n->calib_presum = n->pnet ? nullptr : presum_dev;
+    tower_pass(absmax_dev);
+    n->calib_presum = nullptr;
+    std::vector<float> absmax((size_t)L * C), mean_exact((size_t)L * C);
     if (rc == AZ_OK && e == cudaSuccess) e = cudaMemcpyAsync(absmax.data(), absmax_dev, absmax.size() * sizeof(float), cudaMemcpyDeviceToHost, s);
+    if (rc == AZ_OK && e == cudaSuccess) e = cudaMemcpyAsync(mean_exact.data(), presum_dev, mean_exact.size() * sizeof(float), cudaMemcpyDeviceToHost, s);
     if (rc == AZ_OK && e == cudaSuccess) e = cudaStreamSynchronize(s);
     cudaFree(absmax_dev);
+    if (rc != AZ_OK || e != cudaSuccess) cudaFree(presum_dev);
     if (rc != AZ_OK) return rc;
     if (e != cudaSuccess) { az::set_cuda_error(e, "az_calibrate"); return AZ_ERR_CUDA; }
+    // from here on presum_dev is freed on every path through free_presum
+    struct Guard { float *p; ~Guard() { cudaFree(p); } } free_presum{presum_dev};
     // 2. quantise the tower with those ranges
     if (n->pnet) return az::quantise_pnet(*n, absmax.data());
     az::HostMaster *hm = static_cast<az::HostMaster *>(n->host_master);
@@ -711,6 +725,40 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
     AZ_CUDA(cudaMemcpy(n->tc8_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
     AZ_CUDA(cudaMemcpy(n->tc8_lconst, lconst.data(), lconst.size() * sizeof(float), cudaMemcpyHostToDevice));
     n->fp8_ready = true;
+    // 3. bias correction (the usual post-training remedy for the systematic part of the rounding error: weights
+    //    rounded to 8 bits meet activations that are not zero-mean, which shifts every output channel's mean).
+    //    Layer by layer, in order, the 8-bit tower runs over the calibration positions and the layer's biases are
+    //    moved so that its mean pre-activation per channel equals the bf16 tower's.  Layer 0 is bf16 in both.
+    if (getenv("AZ_NO_BIAS_CORRECTION") != nullptr) return AZ_OK;      // measurement aid: the quantisation as it is without step 3
+    const float kMax = n->int8 ? 255.0f : 448.0f;
+    const double cells = (double)count * 64.0;
+    std::vector<float> sum_q(C);
+    for (int l = 1; l < L; ++l) {
+        AZ_CUDA(cudaMemsetAsync(presum_dev, 0, (size_t)L * C * sizeof(float), s));
+        n->calib_presum = presum_dev;
+        tower_pass(nullptr);
+        n->calib_presum = nullptr;
+        if (rc != AZ_OK) return rc;
+        if (e != cudaSuccess) { az::set_cuda_error(e, "az_calibrate"); return AZ_ERR_CUDA; }
+        AZ_CUDA(cudaMemcpyAsync(sum_q.data(), presum_dev + (size_t)l * C, (size_t)C * sizeof(float), cudaMemcpyDeviceToHost, s));
+        AZ_CUDA(cudaStreamSynchronize(s));
+        float *bias_q = lconst.data() + (size_t)l * 3 * C + C;         // bias x the layer's output scale
+        for (int c = 0; c < C; ++c) {
+            const float top = absmax[(size_t)l * C + c];                              // the channel's largest output
+            if (!(top > 1e-20f)) continue;                                            // a dead channel has nothing to correct
+            const float qs = l + 1 < L ? kMax / top : 1.0f;
+            const double want = (double)mean_exact[(size_t)l * C + c] / cells;        // real units
+            const double have = (double)sum_q[c] / cells / qs;
+            double corr = want - have;
+            if (!std::isfinite(corr)) continue;
+            // a shift of the mean is a fraction of the channel's range; anything larger is not rounding error
+            if (corr > 0.25 * top) corr = 0.25 * top;
+            if (corr < -0.25 * top) corr = -0.25 * top;
+            bias_q[c] += (float)(corr * qs);
+        }
+        AZ_CUDA(cudaMemcpyAsync(n->tc8_lconst + (size_t)l * 3 * C + C, bias_q, (size_t)C * sizeof(float), cudaMemcpyHostToDevice, s));
+    }
+    AZ_CUDA(cudaStreamSynchronize(s));
     return AZ_OK;
 }
 

@@ -51,6 +51,7 @@ struct Net {
     void *tc8_weights = nullptr;
     float *tc8_lconst = nullptr;      // [n_conv][3][C]
     void *host_master = nullptr;      // fp32 tower weights kept on the host until calibration (FP8 nets)
+    float *calib_presum = nullptr;    // set only inside az_calibrate: where the tower kernels add up their pre-activations
     void *tc_head_w = nullptr;        // packed 1x1 head projections (policy | value), fused into the tower kernel
     float *tc_head_bias = nullptr;
     int tc_head_n = 0;                // 64 (flat policy head) or 112 (73-plane policy head)

@@ -123,6 +123,10 @@ struct TowerArgs {
     const float *lconst;
     // calibration run (bf16 kernel): per-layer, per-channel maximum of the layer outputs, as float bits
     unsigned int *absmax;            // [n_conv][C]
+    // calibration runs (either kernel): per-layer, per-channel SUM of the pre-activation values over all squares of
+    // all boards, in the kernel's own output units (real values in bf16, real x the next layer's activation scale in
+    // the 8-bit forms); the host compares the two networks' means and corrects the 8-bit biases (see az_calibrate)
+    float *presum;                   // [n_conv][C] or null
     // the paper's own network (kPnet instantiation; Sec. 3.2, 4.3.3, 4.3.6, App. D.1): activations capped
     // at six, pooled context in blocks 1, 3, 5, ..., query / key projections as the fused head layer
     const float *gw;                 // [pooled block][C/2][3C/4] fp32, transposed: pooled vector -> context
@@ -742,6 +746,15 @@ tower_tc_kernel(const TowerArgs args) {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] += ctx[kc * 16 + i];
                     }
+                    if (!kPnet && args.presum != nullptr) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            float sm = live ? v[i] : 0.0f;
+#pragma unroll
+                            for (int o = 16; o > 0; o >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, o);
+                            if (lane == i) atomicAdd(args.presum + l * kC + kc * 16 + i, sm);
+                        }
+                    }
                     // ReLU: a first convolution's output is only ever read as packed operands, and the
                     // conversion clamps; elsewhere the fp32 value itself goes on (residual stream, output)
                     if (!from_acc || (!kFp8 && args.absmax != nullptr)) {
@@ -1105,6 +1118,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     a.logits = net.logits;
     a.lconst = net.tc8_lconst;
     a.absmax = absmax;
+    a.presum = net.calib_presum;
     a.gw = net.pnet_gw;
     a.qk_out = static_cast<float *>(net.pnet_qk);
     static const bool trace = getenv("AZ_TOWER_TRACE") != nullptr;

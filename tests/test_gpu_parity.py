@@ -269,13 +269,13 @@ def fp8_run(az, name, batch, oracle_rows):
 def test_c4_fp8_tower_batch_4096_does_what_e4m3_arithmetic_gives(az):
     # Full-size launch (4096), oracle on 256 sampled rows.  An emulation of the same quantisation with
     # EXACT accumulation (e4m3-rounded weights and activations, per-channel scales from the same kind
-    # of calibration) puts this network's tower 8.8 % rms off the fp64 tower; the kernel must land
-    # there, not above.  Whether that is inside the 5e-2 output bar is a property of the arithmetic
-    # and of this plain residual block, tested separately below.
+    # of calibration) puts this network's tower 8.8 % rms off the fp64 tower, 7.2 % with the bias
+    # correction az_calibrate applies; the kernel must land there, not above.  Whether that is inside the
+    # 5e-2 output bar is a property of the arithmetic and of this plain residual block, tested separately below.
     rows = np.arange(0, 4096, 16)
     perr, verr, agree, tower_err = fp8_run(az, "c4", 4096, rows)
-    assert 0.03 < tower_err < 0.11
-    assert perr < 0.2 and verr < 0.2 and agree > 0.85
+    assert 0.03 < tower_err < 0.09
+    assert perr < 0.15 and verr < 0.15 and agree > 0.85
 
 
 @pytest.mark.xfail(strict=False, reason="post-training FP8 of the plain residual tower: e4m3 weights and activations "
@@ -288,11 +288,12 @@ def test_c4_fp8_meets_the_5e_2_bar(az):
 
 def test_c4b_fp8_with_scaled_residual_branches(az):
     # the paper's remedy (Sec. 4.3.6): residual branches scaled by 1/sqrt(depth), folded into the second
-    # convolution.  Same kernels, different weights.  Emulated floor: tower 4.7 % rms, value well
-    # inside the bar, policy at its edge.
+    # convolution.  Same kernels, different weights.  Emulated floor without bias correction: tower 4.7 % rms,
+    # value well inside the bar, policy at its edge (0.04-0.07); with the bias correction of az_calibrate the
+    # kernel measures tower 4.0 %, policy 4.6e-2, value 1.8e-2: inside the bar.
     perr, verr, agree, tower_err = fp8_run(az, "c4b", 512, np.arange(256))
-    assert 0.02 < tower_err < 0.06
-    assert verr <= TOL[2] and perr < 0.1
+    assert 0.02 < tower_err < 0.05
+    assert verr <= TOL[2] and perr <= TOL[2]
 
 
 def test_c4i_int8_tower_meets_the_bar_of_the_quantised_configs(az):
@@ -301,6 +302,15 @@ def test_c4i_int8_tower_meets_the_bar_of_the_quantised_configs(az):
     rows = np.arange(0, 4096, 16)
     perr, verr, agree, tower_err = fp8_run(az, "c4i", 4096, rows)
     assert tower_err < 2.5e-2
+    assert perr <= TOL[2] and verr <= TOL[2]
+
+
+def test_c4p_int8_tower_on_the_plain_weights_of_c4(az):
+    # c4 exactly as specified (plain residual blocks, the weights of c2), quantised to int8 instead of e4m3, with
+    # the bias correction of az_calibrate: inside the 5e-2 bar that e4m3 cannot reach on this network
+    rows = np.arange(0, 4096, 16)
+    perr, verr, agree, tower_err = fp8_run(az, "c4p", 4096, rows)
+    assert tower_err < 3e-2
     assert perr <= TOL[2] and verr <= TOL[2]
 
 
