@@ -684,11 +684,11 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
     // 1. bf16 tower over the calibration positions, recording every layer's per-channel output maximum and the sum
     //    of its pre-activation values (for the bias correction of step 3)
     unsigned int *absmax_dev = nullptr;
-    float *presum_dev = nullptr;
+    double *presum_dev = nullptr;
     AZ_CUDA(cudaMalloc((void **)&absmax_dev, (size_t)L * C * sizeof(unsigned int)));
-    if (cudaMalloc((void **)&presum_dev, (size_t)L * C * sizeof(float)) != cudaSuccess) { cudaFree(absmax_dev); return AZ_ERR_CUDA; }
+    if (cudaMalloc((void **)&presum_dev, (size_t)L * C * sizeof(double)) != cudaSuccess) { cudaFree(absmax_dev); return AZ_ERR_CUDA; }
     cudaError_t e = cudaMemsetAsync(absmax_dev, 0, (size_t)L * C * sizeof(unsigned int), s);
-    if (e == cudaSuccess) e = cudaMemsetAsync(presum_dev, 0, (size_t)L * C * sizeof(float), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(presum_dev, 0, (size_t)L * C * sizeof(double), s);
     int rc = AZ_OK;
     // one pass of the tower (whichever form is ready) over all calibration positions
     auto tower_pass = [&](unsigned int *absmax_hook) {
@@ -698,57 +698,71 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
             rc = az::launch_tower_tc(*n, nullptr, p, chunk, nullptr, false, absmax_hook, s);
         }
     };
-    n->calib_presum = n->pnet ? nullptr : presum_dev;
+    n->calib_presum = presum_dev;
     tower_pass(absmax_dev);
     n->calib_presum = nullptr;
-    std::vector<float> absmax((size_t)L * C), mean_exact((size_t)L * C);
+    std::vector<float> absmax((size_t)L * C);
+    std::vector<double> mean_exact((size_t)L * C);
     if (rc == AZ_OK && e == cudaSuccess) e = cudaMemcpyAsync(absmax.data(), absmax_dev, absmax.size() * sizeof(float), cudaMemcpyDeviceToHost, s);
-    if (rc == AZ_OK && e == cudaSuccess) e = cudaMemcpyAsync(mean_exact.data(), presum_dev, mean_exact.size() * sizeof(float), cudaMemcpyDeviceToHost, s);
+    if (rc == AZ_OK && e == cudaSuccess) e = cudaMemcpyAsync(mean_exact.data(), presum_dev, mean_exact.size() * sizeof(double), cudaMemcpyDeviceToHost, s);
     if (rc == AZ_OK && e == cudaSuccess) e = cudaStreamSynchronize(s);
     cudaFree(absmax_dev);
     if (rc != AZ_OK || e != cudaSuccess) cudaFree(presum_dev);
     if (rc != AZ_OK) return rc;
     if (e != cudaSuccess) { az::set_cuda_error(e, "az_calibrate"); return AZ_ERR_CUDA; }
     // from here on presum_dev is freed on every path through free_presum
-    struct Guard { float *p; ~Guard() { cudaFree(p); } } free_presum{presum_dev};
+    struct Guard { double *p; ~Guard() { cudaFree(p); } } free_presum{presum_dev};
     // 2. quantise the tower with those ranges
-    if (n->pnet) return az::quantise_pnet(*n, absmax.data());
-    az::HostMaster *hm = static_cast<az::HostMaster *>(n->host_master);
-    std::vector<const float *> w, sc, bi;
-    for (int l = 0; l < L; ++l) { w.push_back(hm->w[l].data()); sc.push_back(hm->scale[l].data()); bi.push_back(hm->bias[l].data()); }
-    const size_t bytes = az::tc8_packed_weight_bytes(n->in_pad, C, L);
-    std::vector<unsigned char> packed(bytes);
-    std::vector<float> lconst((size_t)L * 3 * C);
-    az::tc8_pack(w.data(), sc.data(), bi.data(), absmax.data(), (int)n->arch.in_planes, n->in_pad, C, L, n->int8, packed.data(), lconst.data());
-    if (!n->tc8_weights) AZ_CUDA(cudaMalloc(&n->tc8_weights, bytes));
-    if (!n->tc8_lconst) AZ_CUDA(cudaMalloc((void **)&n->tc8_lconst, lconst.size() * sizeof(float)));
-    AZ_CUDA(cudaMemcpy(n->tc8_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
-    AZ_CUDA(cudaMemcpy(n->tc8_lconst, lconst.data(), lconst.size() * sizeof(float), cudaMemcpyHostToDevice));
-    n->fp8_ready = true;
+    std::vector<float> lconst;
+    std::vector<int> next_cin(L, C);                  // output channels of layer l that the next layer reads as 8-bit activations
+    next_cin[L - 1] = 0;
+    int vecs = 3;                                     // constant vectors per layer: scale, bias, residual ratio (+ cap)
+    if (n->pnet) {
+        rc = az::quantise_pnet(*n, absmax.data(), &lconst, &next_cin);
+        if (rc != AZ_OK) return rc;
+        vecs = 4;
+    } else {
+        az::HostMaster *hm = static_cast<az::HostMaster *>(n->host_master);
+        std::vector<const float *> w, sc, bi;
+        for (int l = 0; l < L; ++l) { w.push_back(hm->w[l].data()); sc.push_back(hm->scale[l].data()); bi.push_back(hm->bias[l].data()); }
+        const size_t bytes = az::tc8_packed_weight_bytes(n->in_pad, C, L);
+        std::vector<unsigned char> packed(bytes);
+        lconst.resize((size_t)L * 3 * C);
+        az::tc8_pack(w.data(), sc.data(), bi.data(), absmax.data(), (int)n->arch.in_planes, n->in_pad, C, L, n->int8, packed.data(), lconst.data());
+        if (!n->tc8_weights) AZ_CUDA(cudaMalloc(&n->tc8_weights, bytes));
+        if (!n->tc8_lconst) AZ_CUDA(cudaMalloc((void **)&n->tc8_lconst, lconst.size() * sizeof(float)));
+        AZ_CUDA(cudaMemcpy(n->tc8_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
+        AZ_CUDA(cudaMemcpy(n->tc8_lconst, lconst.data(), lconst.size() * sizeof(float), cudaMemcpyHostToDevice));
+        n->fp8_ready = true;
+    }
     // 3. bias correction (the usual post-training remedy for the systematic part of the rounding error: weights
     //    rounded to 8 bits meet activations that are not zero-mean, which shifts every output channel's mean).
     //    Layer by layer, in order, the 8-bit tower runs over the calibration positions and the layer's biases are
-    //    moved so that its mean pre-activation per channel equals the bf16 tower's.  Layer 0 is bf16 in both.
+    //    moved so that its mean pre-activation per channel equals the bf16 tower's.  Layer 0 is bf16 in both.  In
+    //    the paper's network the pooled quarter of a pooled block's first convolution stays as it is (those
+    //    channels are not handed on as 8-bit activations and take another path through the kernel).
     if (getenv("AZ_NO_BIAS_CORRECTION") != nullptr) return AZ_OK;      // measurement aid: the quantisation as it is without step 3
     const float kMax = n->int8 ? 255.0f : 448.0f;
     const double cells = (double)count * 64.0;
-    std::vector<float> sum_q(C);
+    std::vector<double> sum_q(C);
     for (int l = 1; l < L; ++l) {
-        AZ_CUDA(cudaMemsetAsync(presum_dev, 0, (size_t)L * C * sizeof(float), s));
+        AZ_CUDA(cudaMemsetAsync(presum_dev, 0, (size_t)L * C * sizeof(double), s));
         n->calib_presum = presum_dev;
         tower_pass(nullptr);
         n->calib_presum = nullptr;
         if (rc != AZ_OK) return rc;
         if (e != cudaSuccess) { az::set_cuda_error(e, "az_calibrate"); return AZ_ERR_CUDA; }
-        AZ_CUDA(cudaMemcpyAsync(sum_q.data(), presum_dev + (size_t)l * C, (size_t)C * sizeof(float), cudaMemcpyDeviceToHost, s));
+        AZ_CUDA(cudaMemcpyAsync(sum_q.data(), presum_dev + (size_t)l * C, (size_t)C * sizeof(double), cudaMemcpyDeviceToHost, s));
         AZ_CUDA(cudaStreamSynchronize(s));
-        float *bias_q = lconst.data() + (size_t)l * 3 * C + C;         // bias x the layer's output scale
-        for (int c = 0; c < C; ++c) {
+        float *bias_q = lconst.data() + ((size_t)l * vecs + 1) * C;    // bias x the layer's output scale
+        const bool pooled_layer = n->pnet && (l & 3) == 3;
+        const int correct = pooled_layer ? C - C / 4 : C;
+        for (int c = 0; c < correct; ++c) {
             const float top = absmax[(size_t)l * C + c];                              // the channel's largest output
             if (!(top > 1e-20f)) continue;                                            // a dead channel has nothing to correct
-            const float qs = l + 1 < L ? kMax / top : 1.0f;
-            const double want = (double)mean_exact[(size_t)l * C + c] / cells;        // real units
-            const double have = (double)sum_q[c] / cells / qs;
+            const float qs = c < next_cin[l] ? kMax / top : 1.0f;
+            const double want = mean_exact[(size_t)l * C + c] / cells;                // real units
+            const double have = sum_q[c] / cells / qs;
             double corr = want - have;
             if (!std::isfinite(corr)) continue;
             // a shift of the mean is a fraction of the channel's range; anything larger is not rounding error
@@ -756,7 +770,7 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
             if (corr < -0.25 * top) corr = -0.25 * top;
             bias_q[c] += (float)(corr * qs);
         }
-        AZ_CUDA(cudaMemcpyAsync(n->tc8_lconst + (size_t)l * 3 * C + C, bias_q, (size_t)C * sizeof(float), cudaMemcpyHostToDevice, s));
+        AZ_CUDA(cudaMemcpyAsync(n->tc8_lconst + ((size_t)l * vecs + 1) * C, bias_q, (size_t)C * sizeof(float), cudaMemcpyHostToDevice, s));
     }
     AZ_CUDA(cudaStreamSynchronize(s));
     return AZ_OK;

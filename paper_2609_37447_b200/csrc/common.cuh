@@ -6,6 +6,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <vector>
 
 #include "az_eval.h"
 
@@ -51,7 +52,7 @@ struct Net {
     void *tc8_weights = nullptr;
     float *tc8_lconst = nullptr;      // [n_conv][3][C]
     void *host_master = nullptr;      // fp32 tower weights kept on the host until calibration (FP8 nets)
-    float *calib_presum = nullptr;    // set only inside az_calibrate: where the tower kernels add up their pre-activations
+    double *calib_presum = nullptr;    // set only inside az_calibrate: where the tower kernels add up their pre-activations
     void *tc_head_w = nullptr;        // packed 1x1 head projections (policy | value), fused into the tower kernel
     float *tc_head_bias = nullptr;
     int tc_head_n = 0;                // 64 (flat policy head) or 112 (73-plane policy head)
@@ -154,7 +155,9 @@ void swap_workspace(Net &n);
 // ---- kernels' launch functions (each returns AZ_OK or AZ_ERR_CUDA) ---------------------------
 int launch_encode52(const void *positions, int batch, bool bf16, void *planes, cudaStream_t s);
 int build_pnet(Net &n, const unsigned char *blob, size_t nbytes);
-int quantise_pnet(Net &n, const float *absmax);      // int8 form, after the calibration pass ([n_conv][C] output maxima)
+// int8 form, after the calibration pass ([n_conv][C] output maxima); hands back the per-layer constants it uploaded
+// ([n_conv][4][C]) and, per layer, how many of its output channels the next layer reads as 8-bit activations
+int quantise_pnet(Net &n, const float *absmax, std::vector<float> *lconst_out, std::vector<int> *next_cin_out);
 void free_pnet_master(void *master);
 int launch_pnet_finish(const Net &n, const uint64_t *masks, int batch, float *policy, float *legal, int *counts,
                        float *value, cudaStream_t s);

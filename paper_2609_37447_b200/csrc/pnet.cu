@@ -269,7 +269,7 @@ void free_pnet_master(void *master) { delete static_cast<PnetMaster *>(master); 
 // their values stay in real units), hs = 1 / ws of the next second convolution on the residual
 // stream.  The context map's rows are multiplied by the same qs, since the context is added to
 // values that are already in those units.
-int quantise_pnet(Net &n, const float *absmax) {
+int quantise_pnet(Net &n, const float *absmax, std::vector<float> *lconst_out, std::vector<int> *next_cin_out) {
     const PnetMaster *m = static_cast<const PnetMaster *>(n.pnet_master);
     if (!m) return AZ_ERR_UNSUPPORTED;
     const int C = (int)n.arch.channels, L = n.n_conv, P = C / 4, R = C - P;
@@ -339,6 +339,11 @@ int quantise_pnet(Net &n, const float *absmax) {
     // the scaled context maps replace the plain ones (the calibration pass, which needed those, is over)
     AZ_CUDA(cudaMemcpy(n.pnet_gw, gwt.data(), gwt.size() * sizeof(float), cudaMemcpyHostToDevice));
     n.fp8_ready = true;
+    if (next_cin_out) {
+        next_cin_out->assign(L, 0);
+        for (int l = 0; l + 1 < L; ++l) (*next_cin_out)[l] = m->cin[l + 1];
+    }
+    if (lconst_out) *lconst_out = std::move(lconst);
     return AZ_OK;
 }
 

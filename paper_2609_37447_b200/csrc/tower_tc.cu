@@ -126,7 +126,7 @@ struct TowerArgs {
     // calibration runs (either kernel): per-layer, per-channel SUM of the pre-activation values over all squares of
     // all boards, in the kernel's own output units (real values in bf16, real x the next layer's activation scale in
     // the 8-bit forms); the host compares the two networks' means and corrects the 8-bit biases (see az_calibrate)
-    float *presum;                   // [n_conv][C] or null
+    double *presum;                  // [n_conv][C] or null (double: the host subtracts two nearly equal means)
     // the paper's own network (kPnet instantiation; Sec. 3.2, 4.3.3, 4.3.6, App. D.1): activations capped
     // at six, pooled context in blocks 1, 3, 5, ..., query / key projections as the fused head layer
     const float *gw;                 // [pooled block][C/2][3C/4] fp32, transposed: pooled vector -> context
@@ -746,13 +746,13 @@ tower_tc_kernel(const TowerArgs args) {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] += ctx[kc * 16 + i];
                     }
-                    if (!kPnet && args.presum != nullptr) {
+                    if (args.presum != nullptr) {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) {
                             float sm = live ? v[i] : 0.0f;
 #pragma unroll
                             for (int o = 16; o > 0; o >>= 1) sm += __shfl_xor_sync(0xffffffffu, sm, o);
-                            if (lane == i) atomicAdd(args.presum + l * kC + kc * 16 + i, sm);
+                            if (lane == i) atomicAdd(args.presum + l * kC + kc * 16 + i, (double)sm);
                         }
                     }
                     // ReLU: a first convolution's output is only ever read as packed operands, and the
