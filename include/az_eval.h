@@ -306,11 +306,14 @@ int az_legal_masks(const void *positions_dev, size_t position_stride, int batch,
  * deploys: unsigned 8-bit activations (range / 255; they are never negative), signed 8-bit weights
  * (max / 127 per output channel), int32 accumulation, the residual stream kept as int32 in the
  * second convolution's units; input layer and heads in bf16 in both.
- * Then, for the residual-tower nets, a bias correction (the usual post-training remedy for the
+ * Then a bias correction (the usual post-training remedy for the
  * systematic part of rounding error: rounded weights meet activations that are not zero-mean, which
  * shifts every output channel's mean): layer by layer the 8-bit tower runs over the same positions
  * and the layer's biases are moved so that each channel's mean pre-activation equals the bf16
- * tower's (one tower pass per layer; shifts are limited to a quarter of the channel's range).
+ * tower's (one tower pass per layer; shifts are limited to a quarter of the channel's range; the
+ * sums behind the means are accumulated in double, so the result is repeatable).  In the paper's
+ * network the pooled quarter of a pooled block's first convolution is left as it is.  With the
+ * environment variable AZ_NO_BIAS_CORRECTION set the correction is skipped (a measurement aid).
  * Synchronises the stream.  Errors: BAD_ARG, BATCH_TOO_LARGE, CUDA, UNSUPPORTED (not an 8-bit net).
  */
 int az_calibrate(az_net *net, const void *positions_dev, int n, void *cuda_stream);
