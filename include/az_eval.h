@@ -267,10 +267,13 @@ int az_tower(az_net *net, const void *positions_dev, int batch, void *tower_dev,
  * device (every GPU that loads the library holds it until the process exits).  Results are the
  * same as az_tower's: tower_dev receives [batch][64][channels] bfloat16.
  *   - Limits: batch <= 256 (AZ_ERR_BATCH_TOO_LARGE beyond, and beyond arch.max_batch); networks
- *     with the tensor-core tower only, i.e. bf16, 128 channels, 19 input planes
- *     (AZ_ERR_UNSUPPORTED otherwise).
- *   - The first call on a device looks up the array's device address (one-time set-up, no
- *     allocation); make that first call outside any stream capture.
+ *     with the bf16 tensor-core tower only, i.e. AZ_PREC_BF16, 128 channels, 19 input planes
+ *     (AZ_ERR_UNSUPPORTED otherwise: fp32 networks, the 8-bit towers whether calibrated or not,
+ *     other widths, the 112- and 52-plane networks).
+ *   - The current device must be the one the network was loaded on (AZ_ERR_BAD_ARG otherwise):
+ *     every device has its own copy of the array, and the call uses the current device's.
+ *   - The first call on a device looks up the array's device address (one-time set-up under a
+ *     lock, no allocation); make that first call outside any stream capture.
  *   - All calls, from every az_net and every stream, share the one array, and it keeps whatever
  *     the previous call left in it.  Nothing in it needs clearing (each call overwrites all it
  *     reads), but two calls that overlap on the GPU race on it: serialise them on one stream or
@@ -312,11 +315,22 @@ int az_legal_masks(const void *positions_dev, size_t position_stride, int batch,
  * and the layer's biases are moved so that each channel's mean pre-activation equals the bf16
  * tower's (one tower pass per layer; shifts are limited to a quarter of the channel's range; the
  * sums behind the means are accumulated in double, so the result is repeatable).  In the paper's
- * network the pooled quarter of a pooled block's first convolution is left as it is.  With the
- * environment variable AZ_NO_BIAS_CORRECTION set the correction is skipped (a measurement aid).
+ * network the pooled quarter of a pooled block's first convolution is left as it is.
+ * If a CUDA error interrupts the correction, the call returns it and the network counts as not
+ * calibrated again (AZ_ERR_NOT_CALIBRATED from the evaluation calls) rather than running with biases
+ * corrected in part; the residual networks may then be calibrated anew, the paper's network has to
+ * be loaded again (its first calibration rescales its context maps; a second one is refused with
+ * AZ_ERR_UNSUPPORTED).
  * Synchronises the stream.  Errors: BAD_ARG, BATCH_TOO_LARGE, CUDA, UNSUPPORTED (not an 8-bit net).
+ *
+ * az_calibrate_ex is the same call with options (az_calibrate passes 0):
+ *   AZ_CALIBRATE_NO_BIAS_CORRECTION  stop after the ranges and scales are fixed.  For reports that
+ *     separate the rounding error of the 8-bit operands from what the correction removes.
+ * Unknown bits: BAD_ARG.
  */
+#define AZ_CALIBRATE_NO_BIAS_CORRECTION 1u
 int az_calibrate(az_net *net, const void *positions_dev, int n, void *cuda_stream);
+int az_calibrate_ex(az_net *net, const void *positions_dev, int n, uint32_t flags, void *cuda_stream);
 
 /* Device-side status word of the last kernels (0 = clean).  Synchronises the given stream. */
 int az_device_status(az_net *net, void *cuda_stream, uint32_t *status_out);

@@ -25,7 +25,7 @@ AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3, AZ_PREC_INT8 = 0, 1, 2, 3
 
 EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
            "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_submit_host", "az_wait_host", "az_encode", "az_encode52", "az_tower", "az_tower_static", "az_legal_masks",
-           "az_calibrate", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
+           "az_calibrate", "az_calibrate_ex", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error",
            "az_apply_moves", "az_standin_evaluate", "az_search_create", "az_search_destroy", "az_search_set_roots", "az_search_replace_roots",
            "az_search_run", "az_search_run_async", "az_search_wait", "az_search_root", "az_search_root_visits", "az_search_advance", "az_search_root_noise", "az_search_root_positions", "az_search_tree", "az_search_launches_per_step")
@@ -97,6 +97,8 @@ def _load_library():
     lib.az_legal_masks.argtypes = [vp, sz, ci, ci, vp, vp]
     lib.az_calibrate.restype = ci
     lib.az_calibrate.argtypes = [vp, vp, ci, vp]
+    lib.az_calibrate_ex.restype = ci
+    lib.az_calibrate_ex.argtypes = [vp, vp, ci, ctypes.c_uint32, vp]
     lib.az_device_status.restype = ci
     lib.az_device_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.az_selftest_wait_timeout.restype = ci
@@ -314,6 +316,13 @@ def az_legal_masks(positions_dev, position_stride, batch, policy_head, masks_dev
 
 def az_calibrate(net: Net, positions_dev, n, stream=None):
     _check(_lib.az_calibrate(net.handle, _dev_ptr(positions_dev, "positions"), n, _stream_ptr(stream)), "az_calibrate")
+
+
+AZ_CALIBRATE_NO_BIAS_CORRECTION = 1
+
+
+def az_calibrate_ex(net: Net, positions_dev, n, flags=0, stream=None):
+    _check(_lib.az_calibrate_ex(net.handle, _dev_ptr(positions_dev, "positions"), n, flags, _stream_ptr(stream)), "az_calibrate_ex")
 
 
 def az_device_status(net: Net, stream=None) -> int:

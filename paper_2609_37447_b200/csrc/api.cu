@@ -121,11 +121,6 @@ int alloc_simt_buffers(Net &n) {
     return AZ_OK;
 }
 
-bool want_simt_tower() {
-    const char *e = getenv("AZ_EVAL_TOWER");
-    return e && strcmp(e, "simt") == 0;
-}
-
 int build_net(Net &n, const BlobView &v) {
     const az_arch &a = n.arch;
     const int C = (int)a.channels, L = (int)a.blocks;
@@ -140,7 +135,7 @@ int build_net(Net &n, const BlobView &v) {
     // tensor-core tower: bf16 with 128 or 256 channels; the FP8 tower exists for 128 channels
     const bool tc_shape = a.precision != AZ_PREC_FP32 && (C == 128 || (C == 256 && !n.fp8));
     if (n.fp8 && !tc_shape) return AZ_ERR_UNSUPPORTED;
-    if (tc_shape && (n.fp8 || !want_simt_tower())) {
+    if (tc_shape) {
         std::vector<const float *> w, s, b;
         w.push_back(v.in_w); s.push_back(v.in_s); b.push_back(v.in_b);
         for (int i = 0; i < L; ++i) {
@@ -674,10 +669,16 @@ int az_legal_masks(const void *positions_dev, size_t position_stride, int batch,
 }
 
 int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_stream) {
+    return az_calibrate_ex(net, positions_dev, count, 0u, cuda_stream);
+}
+
+int az_calibrate_ex(az_net *net, const void *positions_dev, int count, uint32_t flags, void *cuda_stream) {
     Net *n = reinterpret_cast<Net *>(net);
     if (!n || count <= 0 || !positions_dev || (reinterpret_cast<uintptr_t>(positions_dev) & 7)) return AZ_ERR_BAD_ARG;
+    if (flags & ~(uint32_t)AZ_CALIBRATE_NO_BIAS_CORRECTION) return AZ_ERR_BAD_ARG;
     if (!n->fp8 || (!n->host_master && !n->pnet_master)) return AZ_ERR_UNSUPPORTED;
-    if (n->pnet && n->fp8_ready) return AZ_ERR_UNSUPPORTED;   // its context maps were rescaled by the first calibration
+    // the paper network's context maps are rescaled by its first calibration, finished or not
+    if (n->pnet && (n->fp8_ready || n->calib_broken)) return AZ_ERR_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const int C = (int)n->arch.channels, L = n->n_conv;
     const size_t pb = az_position_bytes(&n->arch);
@@ -734,6 +735,7 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
         AZ_CUDA(cudaMemcpy(n->tc8_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
         AZ_CUDA(cudaMemcpy(n->tc8_lconst, lconst.data(), lconst.size() * sizeof(float), cudaMemcpyHostToDevice));
         n->fp8_ready = true;
+        n->calib_broken = false;
     }
     // 3. bias correction (the usual post-training remedy for the systematic part of the rounding error: weights
     //    rounded to 8 bits meet activations that are not zero-mean, which shifts every output channel's mean).
@@ -741,7 +743,9 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
     //    moved so that its mean pre-activation per channel equals the bf16 tower's.  Layer 0 is bf16 in both.  In
     //    the paper's network the pooled quarter of a pooled block's first convolution stays as it is (those
     //    channels are not handed on as 8-bit activations and take another path through the kernel).
-    if (getenv("AZ_NO_BIAS_CORRECTION") != nullptr) return AZ_OK;      // measurement aid: the quantisation as it is without step 3
+    if (flags & AZ_CALIBRATE_NO_BIAS_CORRECTION) return AZ_OK;
+    // a failure from here on leaves the biases partly corrected: the net then counts as not calibrated
+    struct Unready { Net *n; bool armed; ~Unready() { if (armed) { n->fp8_ready = false; n->calib_broken = true; } } } unready{n, true};
     const float kMax = n->int8 ? 255.0f : 448.0f;
     const double cells = (double)count * 64.0;
     std::vector<double> sum_q(C);
@@ -773,6 +777,7 @@ int az_calibrate(az_net *net, const void *positions_dev, int count, void *cuda_s
         AZ_CUDA(cudaMemcpyAsync(n->tc8_lconst + ((size_t)l * vecs + 1) * C, bias_q, (size_t)C * sizeof(float), cudaMemcpyHostToDevice, s));
     }
     AZ_CUDA(cudaStreamSynchronize(s));
+    unready.armed = false;
     return AZ_OK;
 }
 

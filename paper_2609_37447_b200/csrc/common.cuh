@@ -49,6 +49,7 @@ struct Net {
     // FP8-e4m3 tower (weights and per-layer constants exist once az_calibrate has run)
     bool fp8 = false, fp8_ready = false;   // 8-bit tower (FP8-e4m3 or int8) and whether it has been calibrated
     bool int8 = false;                      // the 8-bit tower's operands are u8 activations x s8 weights
+    bool calib_broken = false;              // az_calibrate failed half-way through its bias correction
     void *tc8_weights = nullptr;
     float *tc8_lconst = nullptr;      // [n_conv][3][C]
     void *host_master = nullptr;      // fp32 tower weights kept on the host until calibration (FP8 nets)

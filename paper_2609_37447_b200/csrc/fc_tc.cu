@@ -15,6 +15,8 @@
 #include "common.cuh"
 #include "ptx.cuh"
 
+#include <mutex>
+
 namespace az {
 namespace {
 
@@ -223,11 +225,15 @@ void fc_tc_pack_weights(const float *w, int n, __nv_bfloat16 *packed) {
 int launch_fc_tc(const Net &net, int batch, float *value_out, cudaStream_t s) {
     if (batch == 0) return AZ_OK;
     static bool configured[64] = {};
+    static std::mutex configured_lock;                  // any thread may make a device's first launch
     int dev = 0;
     AZ_CUDA(cudaGetDevice(&dev));
-    if (dev < 64 && !configured[dev]) {
-        AZ_CUDA(cudaFuncSetAttribute(fc_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-        configured[dev] = true;
+    {
+        std::lock_guard<std::mutex> hold(configured_lock);
+        if (dev >= 0 && dev < 64 && !configured[dev]) {
+            AZ_CUDA(cudaFuncSetAttribute(fc_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+            configured[dev] = true;
+        }
     }
     const bool flat = net.arch.policy_head == AZ_POLICY_FLAT1858;
     FcArgs a;

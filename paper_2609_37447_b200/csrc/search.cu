@@ -850,7 +850,16 @@ int az_search_create(az_net *net, const az_search_config *c, az_search **out) {
     const int n_groups = c->games >= 2 ? (int)c->groups : 1;
     const int per_group = (int)((c->games + n_groups - 1) / n_groups);
     if (c->evaluator == AZ_SEARCH_EVAL_NET && (uint64_t)per_group * c->leaves > n->arch.max_batch) return AZ_ERR_BATCH_TOO_LARGE;
-    if (n) AZ_CUDA(cudaSetDevice(n->device));
+    // everything below is allocated on the network's device; the caller's current device is put back on return
+    struct DeviceGuard {
+        int prev = -1;
+        ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+    } device_guard;
+    if (n) {
+        int cur = 0;
+        AZ_CUDA(cudaGetDevice(&cur));
+        if (cur != n->device) { AZ_CUDA(cudaSetDevice(n->device)); device_guard.prev = cur; }
+    }
     int rc = az::ensure_inverse_tables();
     if (rc != AZ_OK) return rc;
     Search *s = new (std::nothrow) Search();
@@ -978,7 +987,13 @@ int az_search_run_async(az_search *search, int simulations) {
     for (int step = 0; step < steps; ++step)
         for (int gi = 0; gi < s->n_groups; ++gi) {
             const int rc = az::queue_step(*s, gi, s->need_root_step && step == 0);
-            if (rc != AZ_OK) return rc;
+            if (rc != AZ_OK) {
+                // kernels of earlier steps may already be queued on both streams and still use the trees: let them
+                // finish before the caller gets the error (and may destroy the search or set new roots)
+                cudaStreamSynchronize(s0);
+                if (s1 != s0) cudaStreamSynchronize(s1);
+                return rc;
+            }
         }
     if (s1 != s0) {
         AZ_CUDA(cudaEventRecord(s->groups[1].done, s1));

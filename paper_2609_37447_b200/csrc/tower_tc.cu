@@ -39,6 +39,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
+#include <mutex>
 #include <vector>
 
 namespace az {
@@ -110,7 +111,9 @@ struct TowerArgs {
     int batch;
     int n_conv;                      // 1 + 2*blocks
     int in_pad;                      // channels of the plane tensor (32 or 128)
-    int trace;                       // CTA 0 prints how long each role waited (debugging aid)
+#ifdef AZ_TRACE
+    int trace;                       // diagnostic builds only: CTA 0 prints how long each role waited
+#endif
     // fused 1x1 head projections (one extra MMA layer on the final activations); head_n == 0: none
     int head_n;                      // 64: flat policy proj (32) | value proj (32); 112: 73 policy planes (+7 pad) | value proj (32)
     const __nv_bfloat16 *head_w;     // packed [slice][k8 2][n-group head_n/8][8][8]
@@ -257,10 +260,15 @@ tower_tc_kernel(const TowerArgs args) {
     auto slices_of = [&](int l) {                                                               // K per MMA: 16 bf16 or 32 e4m3
         return l == 0 ? in_slices : short_layer(l) ? (kFp8 ? kShortSlices / 2 : kShortSlices) : (kFp8 ? kC / 32 : kC / 16);
     };
+    // role tracing (clocks spent waiting, printed by CTA 0) exists in diagnostic builds only (-DAZ_TRACE)
+#ifdef AZ_TRACE
     const bool tr = args.trace && blockIdx.x == 0;
+#else
+    constexpr bool tr = false;
+#endif
     long long t_wait[3] = {0, 0, 0};
     long long t_issue = 0;
-    const long long t_begin = clock64();
+    const long long t_begin = tr ? clock64() : 0;
 
     if (warp == 0) {
         // ================= weight producer =================
@@ -315,7 +323,7 @@ tower_tc_kernel(const TowerArgs args) {
         // only after group 0 has issued its own (bar_lead).  While one issuer sits in its barrier round
         // trips the other's MMAs keep the tensor pipe busy, and the groups reach their layer boundaries
         // one stage apart instead of together.
-        const bool follow = kGroups == 2 && g == 1 && !(args.trace & 2);
+        const bool follow = kGroups == 2 && g == 1;
         const bool lead = kGroups == 2 && g == 0;
         const uint32_t elected = ptx::elect_one();              // the lane that issues; the warp stays converged
         for (int r = 0; ok; ++r) {
@@ -1079,9 +1087,11 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
                     bool with_heads, unsigned int *absmax, cudaStream_t s) {
     if (batch == 0) return AZ_OK;
     static int sm_count[64] = {};
+    static std::mutex sm_count_lock;                    // any thread may make a device's first launch
     int dev = 0;
     AZ_CUDA(cudaGetDevice(&dev));
-    if (dev < 64 && sm_count[dev] == 0) {
+    std::unique_lock<std::mutex> hold(sm_count_lock);
+    if (dev >= 0 && dev < 64 && sm_count[dev] == 0) {
         int n = 0;
         AZ_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
@@ -1095,7 +1105,8 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape176, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         sm_count[dev] = n;
     }
-    const int sms = dev < 64 ? sm_count[dev] : 148;
+    const int sms = (dev >= 0 && dev < 64) ? sm_count[dev] : 148;
+    hold.unlock();
     const bool fp8 = net.fp8_ready && absmax == nullptr;      // the calibration pass itself runs in bf16
     const bool wide = net.arch.channels == 256;
     TowerArgs a;
@@ -1121,8 +1132,10 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     a.presum = net.calib_presum;
     a.gw = net.pnet_gw;
     a.qk_out = static_cast<float *>(net.pnet_qk);
+#ifdef AZ_TRACE
     static const bool trace = getenv("AZ_TOWER_TRACE") != nullptr;
     a.trace = trace ? atoi(getenv("AZ_TOWER_TRACE")) : 0;
+#endif
     // one CTA per SM, or one per two-board group when there are fewer groups than SMs
     const int n_groups = (batch + kNB - 1) / kNB;
     const int grid = n_groups < sms ? n_groups : sms;

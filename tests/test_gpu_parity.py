@@ -85,6 +85,34 @@ def test_encoding_is_bit_exact(az, in_planes, precision):
     az.az_free_net(net)
 
 
+@pytest.mark.parametrize("in_planes,channels,batch", [(19, 128, 1301), (112, 256, 701), (112, 128, 1301)])
+def test_encoder_fused_into_the_tower_kernel_is_bit_exact(az, in_planes, channels, batch):
+    # az_evaluate never runs the stand-alone encoder on the tensor-core path: the tower kernel's epilogue
+    # warps encode each board straight into the shared-memory frame.  A network without blocks whose
+    # input convolution is the centre-tap identity (scale one, bias zero) makes the tower's output the
+    # planes themselves (they are never negative, so the ReLU is the identity), which shows that copy
+    # bit for bit.  The batch spans more than two rounds of the persistent kernel and ends in a lone board.
+    cfg = configs.tiny_config(in_planes=in_planes, blocks=0, channels=channels, policy_head=1, value_head=1,
+                              precision=1, batch=batch)
+    t = weights.draw_tensors(cfg, 1.0, 1.0)
+    w = np.zeros((channels, in_planes, 3, 3), dtype=np.float32)
+    w[np.arange(in_planes), np.arange(in_planes), 1, 1] = 1.0
+    t["in.w"], t["in.scale"], t["in.bias"] = w, np.ones(channels, np.float32), np.zeros(channels, np.float32)
+    net, _ = load(az, cfg, blob=weights.pack_blob(cfg, t))
+    rec, _ = positions.generate(271828, batch, (0, 40), (40, 160))
+    recs = positions.records_for_planes(in_planes, rec)
+    ref = oracle.encode(recs, in_planes)                                  # [n][P][8][8] float64
+    tower = torch.full((batch, 64, channels), 9.0, dtype=torch.bfloat16, device="cuda")
+    az.az_tower(net, az.records_to_device(recs), batch, tower)
+    torch.cuda.synchronize()
+    want = torch.zeros((batch, 64, channels), dtype=torch.float32)
+    want[:, :, :in_planes] = torch.from_numpy(ref.reshape(batch, in_planes, 64).transpose(0, 2, 1).astype(np.float32))
+    want = want.to(torch.bfloat16)                                        # the planes' own rounding decision (halfmove / 100)
+    assert torch.equal(tower.cpu().view(torch.int16), want.view(torch.int16))
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
 @pytest.mark.parametrize("head", [0, 1])
 def test_legal_masks_are_bit_exact(az, head):
     rec, _ = positions.generate(4242 + head, 6000, (0, 60), (40, 200))

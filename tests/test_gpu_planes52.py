@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import oracle
-from inputs import positions
+from inputs import pnet_weights, positions
 
 pytestmark = pytest.mark.gpu
 
@@ -51,3 +51,30 @@ def test_encoding52_hand_built_and_degenerate_sizes():
     with pytest.raises(az.AzError) as e:
         az._check(az._lib.az_encode52(None, 1, 0, None, None), "az_encode52")
     assert e.value.code == az.AZ_ERR_BAD_ARG
+
+
+def test_encoder52_fused_into_the_tower_kernel_is_bit_exact():
+    # Inside az_evaluate the 52 planes are written by the tower kernel's epilogue warps straight into the
+    # shared-memory frame, not by the stand-alone encoder.  A network of the paper's kind without blocks
+    # whose input convolution passes plane c to channel c as +x/32 and to channel 64 + c as -x/32
+    # (centre tap, scale one, bias zero) shows them: the activation keeps max(., 0) of each (and 100/32
+    # stays under its cap of six), x = 32 * (channel c - channel 64 + c), every value exact in bf16.
+    import paper_2609_37447_b200 as az
+    n = 1301                                                               # more than two rounds, a lone last board
+    cfg = pnet_weights.PNetConfig("pid", 0, 128, n, 20260965, 77)
+    t = pnet_weights.draw_tensors(cfg, 1.0, 1.0)
+    w = np.zeros((128, 52, 3, 3), dtype=np.float32)
+    w[np.arange(52), np.arange(52), 1, 1] = 1.0 / 32
+    w[64 + np.arange(52), np.arange(52), 1, 1] = -1.0 / 32
+    t["in.w"], t["in.scale"], t["in.bias"] = w, np.ones(128, np.float32), np.zeros(128, np.float32)
+    net = az.az_load_net(az.make_arch(52, 0, 128, 2, 1, 1, n), pnet_weights.pack_blob(cfg, t))
+    rec, _ = positions.generate_moves(20260966, n, (0, 200))
+    tower = torch.full((n, 64, 128), 9.0, dtype=torch.bfloat16, device="cuda")
+    az.az_tower(net, az.records_to_device(rec), n, tower)
+    torch.cuda.synchronize()
+    got = tower.float().cpu().numpy()
+    want = oracle.encode52(rec).reshape(-1, 52, 64).transpose(0, 2, 1)   # [n][square][channel]
+    assert (32.0 * (got[:, :, :52] - got[:, :, 64:116]) == want).all()
+    assert (got[:, :, 52:64] == 0).all() and (got[:, :, 116:] == 0).all()
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)

@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from inputs import configs, positions, weights
 
 pytestmark = pytest.mark.gpu
@@ -36,6 +37,11 @@ def test_static_scratch_tower_matches_az_tower_on_two_calls_in_a_row():
         # same kernels, same inputs: identical bits expected; the bound is the suite's bf16 bar
         assert np.abs(a - b).max() <= 2e-2 * max(1.0, np.abs(a).max())
         assert (a == b).all()
+        # and not merely equal to each other: rows spread over the call against the CPU oracle's tower
+        rows = np.unique(np.array([0, 1, n // 2, n - 2, n - 1]))
+        ref = oracle.evaluate(blob, recs[rows], 19, cfg.policy_head, want_tower=True)[4]["tower"]    # [rows][C][8][8]
+        mine = b[rows].transpose(0, 2, 1).reshape(len(rows), 128, 8, 8)
+        assert np.abs(mine - ref).max() <= 2e-2 * 3 ** 0.5 * np.abs(ref).max()
     assert az.az_device_status(net) == 0
     # beyond the fixed scratch the call refuses instead of overrunning it
     pos = az.records_to_device(cur[:257])
@@ -43,7 +49,26 @@ def test_static_scratch_tower_matches_az_tower_on_two_calls_in_a_row():
     with pytest.raises(az.AzError) as e:
         az.az_tower_static(net, pos, 257, out)
     assert e.value.code == az.AZ_ERR_BATCH_TOO_LARGE
+    # a caller that has switched to another GPU since az_load_net is refused: that GPU's copy of the array is not
+    # the one this network's kernels can use (needs a second GPU; a one-GPU machine has no other device to switch to)
+    if torch.cuda.device_count() > 1:
+        with torch.cuda.device(1):
+            with pytest.raises(az.AzError) as e:
+                az.az_tower_static(net, az.records_to_device(cur[:4]), 4, out)
+        assert e.value.code == az.AZ_ERR_BAD_ARG
     az.az_free_net(net)
+    # the 8-bit towers are refused whether calibrated or not: this entry point is the bf16 tower's
+    cfg8 = configs.tiny_config(blocks=1, channels=128, precision=2, batch=16, weight_seed=322)
+    net8 = az.az_load_net(az.make_arch(19, 1, 128, 0, 0, 2, 16), weights.make_blob(cfg8, 1.0, 1.0))
+    pos8 = az.records_to_device(cur[:16])
+    out8 = torch.zeros((16, 64, 128), dtype=torch.bfloat16, device="cuda")
+    for calibrated in (False, True):
+        if calibrated:
+            az.az_calibrate(net8, pos8, 16)
+        with pytest.raises(az.AzError) as e:
+            az.az_tower_static(net8, pos8, 16, out8)
+        assert e.value.code == az.AZ_ERR_UNSUPPORTED
+    az.az_free_net(net8)
     # networks without the tensor-core tower are refused, not silently routed elsewhere
     cfg32 = configs.tiny_config(blocks=1, channels=32, precision=0, batch=4)
     net32 = az.az_load_net(az.make_arch(19, 1, 32, 0, 0, 0, 4), weights.make_blob(cfg32))
