@@ -23,8 +23,15 @@ if ROOT not in sys.path:
 
 from inputs import configs, pnet_weights, positions, weights  # noqa: E402
 
-METRIC = "leaf evals/sec, 20x128 bf16 batch 1024"
+METRIC = "leaf evals/sec, 20x128 bf16 batch 1024"      # the headline workload (c3); other workloads name themselves
 UNIT = "evals/s"
+
+
+def metric_of(cfg) -> str:
+    if cfg.name == "c3" and cfg.batch == 1024:
+        return METRIC
+    net = f"{cfg.blocks}x{cfg.channels}"
+    return f"leaf evals/sec, {net} {DTYPE[cfg.precision]} batch {cfg.batch} (workload {cfg.name})"
 WORKLOADS = {
     "c1": "c1: 6x64 fp32 batch 64, 73-plane policy + tanh value",
     "c2": "c2: 20x128 bf16 batch 256, 73-plane policy + tanh value",
@@ -32,6 +39,9 @@ WORKLOADS = {
     "c5": "c5: 40x256 bf16, 112 history planes, flat-1858 policy + WDL value (batch sweep via --batch)",
     "c4": "c4: 20x128 FP8-e4m3 tower (bf16 heads) batch 4096, 73-plane policy + tanh value",
     "c4b": "c4b: c4 with residual branches scaled by 1/sqrt(20)",
+    "c4x": "c4x: c4 as specified (plain weights, e4m3 weights and activations) with every operand as a pair of e4m3 numbers "
+           "(three products per layer), batch 4096",
+    "c4a": "c4a: c4 with pairs of e4m3 numbers for the activations only (two products per layer), batch 4096",
     "c4p": "c4p: c4 as specified (plain weights) with the tower in int8, batch 4096",
     "c4i": "c4i: c4b with the tower in int8 (u8 activations x s8 weights, int32 accumulation), batch 4096",
     "p12": "p12: the paper's own network, 12x128 bf16 batch 1024 (52 planes, capped scaled blocks, pooled context, "
@@ -71,15 +81,37 @@ def make_records(cfg, count, first_index=0):
 
 def make_blob(cfg):
     return pnet_weights.make_blob(cfg) if is_pnet(cfg) else weights.make_blob(cfg)
-DTYPE = {0: "f32", 1: "bf16", 2: "fp8_e4m3", 3: "int8"}
+DTYPE = {0: "f32", 1: "bf16", 2: "fp8_e4m3", 3: "int8", 4: "fp8_e4m3 (operand pairs)", 5: "fp8_e4m3 (activation pairs)"}
 
-# DRAM bytes (read + write) of one tower-kernel launch, from the ncu capture summarised in
-# profiles/tower_tc_kernel_c3_batch592.md: 12.06 MB at batch 592, of which 11.87 MB are the weights
-# (read once whatever the batch) and the rest the 104-byte position records.
+# DRAM bytes (read + write) of one launch of the dominant kernel come from the ncu capture of that workload,
+# summarised under profiles/: each summary ends with a line
+#     traffic_model: fixed_bytes=<weights and constants, read once per launch> per_position_bytes=<grows with the batch>
+# taken from its dram__bytes_read.sum + dram__bytes_write.sum (captured at a batch of a few hundred; the per-position
+# part scales in proportion, the weights do not).  No capture of a workload: no traffic figure.
+TRAFFIC_PROFILES = {
+    "c1": "tower_f32_kernel_c1_batch64.md",
+    "c3": "tower_tc_kernel_c3_batch592.md",
+    "c4": "tower_tc_kernel_fp8_c4_batch592.md", "c4b": "tower_tc_kernel_fp8_c4_batch592.md",
+    "c4i": "tower_tc_kernel_int8_c4i_batch592.md", "c4p": "tower_tc_kernel_int8_c4i_batch592.md",
+    "c5": "tower_tc_kernel_c5_batch296.md",
+    "p14": "tower_tc_kernel_p14_batch296.md",
+    "p14i": "tower_tc_kernel_int8_p14i_batch296.md",
+}
+
+
 def tower_traffic_bytes(cfg, batch):
-    if is_pnet(cfg) or cfg.channels != 128 or cfg.blocks != 20 or cfg.precision != 1:
-        return None             # no capture yet for other shapes / the FP8 tower
-    return 12.06e6 + (batch - 592) * 104.0
+    name = TRAFFIC_PROFILES.get(cfg.name)
+    if name is None:
+        return None, None
+    try:
+        with open(os.path.join(ROOT, "profiles", name)) as f:
+            for line in f:
+                if line.startswith("traffic_model:"):
+                    kv = dict(item.split("=") for item in line.split()[1:])
+                    return float(kv["fixed_bytes"]) + batch * float(kv["per_position_bytes"]), f"profiles/{name}"
+    except (OSError, KeyError, ValueError):
+        pass
+    return None, None
 
 
 def tower_flops_per_position(cfg) -> float:
@@ -102,6 +134,48 @@ def load_peaks():
                 "hbm_gbs": float(p["hbm_gbs"]), "source": "measured"}
     except (OSError, KeyError, ValueError):
         return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+NOMINAL_DENSE_TFLOPS = {0: None, 1: 2250.0, 2: 4500.0, 3: 4500.0, 4: 4500.0, 5: 4500.0}    # datasheet, dense, per GPU
+
+
+def measure_8bit_peak(int8: bool, seconds: float = 4.0):
+    """The library GEMM of the 8-bit type at 8192^3, measured here the way the bf16 peaks were measured for
+    MEASURED_PEAKS.json: best of ten launches (burst) and back to back for `seconds` (sustained), CUDA events.
+    Returns {"burst": TFLOP/s, "sustained": TFLOP/s, "how": ...} or None when the library call is not available."""
+    import torch
+    n = 8192
+    try:
+        if int8:
+            a = torch.randint(-127, 128, (n, n), dtype=torch.int8, device="cuda")
+            b = torch.randint(-127, 128, (n, n), dtype=torch.int8, device="cuda")
+            run = lambda: torch._int_mm(a, b)
+            how = "torch._int_mm int8 8192^3"
+        else:
+            a = torch.randn(n, n, device="cuda").to(torch.float8_e4m3fn)
+            b = torch.randn(n, n, device="cuda").to(torch.float8_e4m3fn).t()          # column-major second operand
+            one = torch.ones((), dtype=torch.float32, device="cuda")
+            run = lambda: torch._scaled_mm(a, b, scale_a=one, scale_b=one, out_dtype=torch.bfloat16)
+            how = "torch._scaled_mm e4m3 8192^3"
+        for _ in range(3):
+            run()
+        torch.cuda.synchronize()
+        flops = 2.0 * n ** 3
+        best = float("inf")
+        for _ in range(10):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); run(); e1.record(); torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        reps = max(10, int(seconds * 1e3 / best))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            run()
+        e1.record(); torch.cuda.synchronize()
+        return {"burst": flops / (best * 1e-3) / 1e12, "sustained": flops * reps / (e0.elapsed_time(e1) * 1e-3) / 1e12,
+                "how": f"{how}: best of 10 (burst), {reps} launches back to back (sustained), measured in this run"}
+    except Exception as exc:            # the library has no such GEMM here: say so, fall back to the nominal ratio
+        return {"error": f"{type(exc).__name__}: {exc}"[:200]}
 
 
 class ClockSampler(threading.Thread):
@@ -187,7 +261,7 @@ def run_reference(args, cfg):
     value = total_n / total_t
     sample_txt = f"first {sample} positions of the {cfg.batch}-position batch per step"
     print(json.dumps({
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "impl": "reference", "metric": metric_of(cfg), "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": WORKLOADS[cfg.name], "sample": sample_txt},
@@ -409,6 +483,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures on a smaller case)")
     ap.add_argument("--leaves", type=int, default=1, help="search workloads: traversals per tree and step")
+    ap.add_argument("--legs", default="all", choices=["all", "device"],
+                    help="device: only the device-resident timed leg (short runs for profiler captures)")
     ap.add_argument("--moves", type=int, default=0, help="search workloads: also time this many played moves per game, each after "
                                                          "a search of --steps steps (subtrees kept)")
     args = ap.parse_args()
@@ -500,7 +576,137 @@ def main():
     barrier()
     b2b_ms = ev0.elapsed_time(ev1)
 
-    # ---- end to end through the host-buffer entry point: pinned host in, pinned host out
+    # ---- sustained: at least two seconds of evaluations back to back, clocks sampled throughout.  The timed region
+    # above is a few milliseconds at boost clocks; this leg shows what holds once the power cap has settled.
+    sustained = None
+    if args.legs == "all" and cfg.precision != 0:
+        n_sus = max(args.steps, int(2500.0 / max(b2b_ms / args.steps, 1e-3)))     # (the library times the first 4096 tower passes)
+        az.az_profile_tower(net, True)
+        az.az_tower_time(net)
+        sus_sampler = ClockSampler(local_rank)
+        barrier()
+        sus_sampler.start()
+        ev0.record()
+        for _ in range(n_sus):
+            az.az_evaluate(net, pos_dev, masks_dev, B, policy_dev, value_dev)
+        ev1.record()
+        barrier()
+        sus_clocks = sus_sampler.stop()
+        sus_ms = ev0.elapsed_time(ev1)
+        sus_tower_ms, sus_passes = az.az_tower_time(net)
+        az.az_profile_tower(net, False)
+        sustained = {"steps": n_sus, "ms": sus_ms, "tower_ms": sus_tower_ms, "passes": sus_passes, "clocks": sus_clocks}
+
+    host = None
+    if args.legs == "all":
+        host = host_legs(az, torch, args, cfg, net, recs, masks_dev, B, barrier)
+
+    # ---- the library GEMM of the 8-bit operand type, measured here (MEASURED_PEAKS.json has bf16 only)
+    peak8 = None
+    if cfg.precision >= 2 and rank == 0 and args.legs == "all":
+        peak8 = measure_8bit_peak(cfg.precision == 3)
+
+    # ---- max over ranks
+    times = [total_ms, b2b_ms, tower_ms] + ([sustained["ms"]] if sustained else [0.0]) + (host["times_ms"] if host else [0.0] * 4)
+    total_ms, b2b_ms, tower_ms_max, sus_ms_max, e2e_ms, e2e_legal_ms, e2e_pipe_ms, e2e_pipe_legal_ms = sharding.max_over_ranks(times, device="cuda")
+
+    if rank == 0:
+        peaks = load_peaks()
+        evals = world * B * args.steps
+        flops = tower_flops_per_position(cfg) * B
+        tower_avg_ms = tower_ms / max(tower_passes, 1)
+        achieved = flops / (tower_avg_ms * 1e-3) / 1e12 if tower_passes else None
+        traffic, traffic_source = tower_traffic_bytes(cfg, B)
+        # a tower launch of a few hundred microseconds between L2 flushes is a burst; launches of milliseconds back to
+        # back for the whole timed region run under the power cap like the sustained GEMM
+        long_launch = tower_avg_ms >= 2.0
+        which = "sustained" if long_launch else "burst"
+        if cfg.precision >= 2 and peak8 is not None and "error" not in peak8:
+            peak_tf, peak_sus = peak8[which], peak8["sustained"]
+            peak_note = f"of measured ({which}; {peak8['how']})"
+        elif cfg.precision >= 2:
+            peak_tf = peaks["bf16_tflops_sustained" if long_launch else "bf16_tflops"] * 2.0
+            peak_sus = peaks["bf16_tflops_sustained"] * 2.0
+            peak_note = (f"of {peaks['source']} ({which} bf16 GEMM x 2, the nominal 8-bit/bf16 ratio; no 8-bit library GEMM was measured"
+                         + (": " + peak8["error"] if peak8 else " in this run") + ")")
+        else:
+            peak_tf = peaks["bf16_tflops_sustained" if long_launch else "bf16_tflops"]
+            peak_sus = peaks["bf16_tflops_sustained"]
+            peak_note = f"of {peaks['source']} ({which} bf16 GEMM; sustained is used when a tower launch takes 2 ms or more)"
+        roof_kernel, roof_bound = "tower_tc_kernel", "tensor"
+        nominal = NOMINAL_DENSE_TFLOPS[cfg.precision]
+        if cfg.precision == 0:
+            # the fp32 network runs on the FP32 FMA pipes: 148 SMs x 128 FMA per clock x 2 x the maximum SM clock
+            roof_kernel, roof_bound = "tower_f32_kernel", "alu"
+            peak_tf = 148 * 128 * 2 * (clocks.get("sm_max_mhz") or 1965) * 1e6 / 1e12
+            peak_sus, nominal = peak_tf, peak_tf
+            peak_note = "derived: 148 SMs x 128 FP32 FMA per clock x 2 x the maximum SM clock"
+        out = {
+            "metric": metric_of(cfg), "value": evals / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+            "ms_per_step_median": float(np.median(step_ms)), "ms_per_step_best": float(min(step_ms)),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": DTYPE[cfg.precision], "data": "synthetic",
+            "config": {"workload": WORKLOADS[cfg.name], "batch_per_gpu": B, "l2": "flushed before every step (256 MB write)",
+                       "timing": "CUDA events around each step on the launch stream, summed; max over ranks",
+                       "device_status": status},
+            "back_to_back": {"value": evals / (b2b_ms * 1e-3), "unit": UNIT, "ms_per_step": b2b_ms / args.steps,
+                             "note": "no L2 flush between steps"},
+            "gpu_launches": args.steps * az.az_launches_per_evaluate(net, B),
+            "clocks": clocks,
+            "roofline": {"kernel": roof_kernel, "bound": roof_bound, "achieved": achieved, "peak": peak_tf,
+                         "unit": "TFLOP/s", "frac": (achieved / peak_tf) if achieved else None,
+                         "frac_of_nominal_dense_peak": (achieved / nominal) if achieved and nominal else None,
+                         "nominal_dense_peak": nominal,
+                         "traffic": traffic, "traffic_source": traffic_source, "peak_source": peak_note,
+                         "avg_launch_ms": tower_avg_ms, "launches_timed": tower_passes,
+                         "flops_per_launch": flops},
+        }
+        if sustained:
+            sus_tower_avg = sustained["tower_ms"] / max(sustained["passes"], 1)
+            sus_ach = flops / (sus_tower_avg * 1e-3) / 1e12 if sustained["passes"] else None
+            mhz = sustained["clocks"].get("sm_mhz")
+            out["sustained"] = {
+                "value": world * B * sustained["steps"] / (sus_ms_max * 1e-3), "unit": UNIT, "steps": sustained["steps"],
+                "seconds": sus_ms_max * 1e-3, "ms_per_step": sus_ms_max / sustained["steps"], "clocks": sustained["clocks"],
+                "ms_per_step_x_sm_mhz": (sus_ms_max / sustained["steps"]) * mhz if mhz else None,
+                "tower_avg_launch_ms": sus_tower_avg, "tower_achieved": sus_ach, "tower_peak_sustained": peak_sus,
+                "tower_frac_of_sustained_peak": (sus_ach / peak_sus) if sus_ach else None,
+                "tower_frac_of_nominal_dense_peak": (sus_ach / nominal) if sus_ach and nominal else None,
+                "note": "evaluations back to back on one stream for two seconds and more, no L2 flush, clocks sampled throughout; "
+                        "the tower's launches timed by events inside the library",
+            }
+        if host:
+            h2d, d2h, d2h_legal = host["h2d"], host["d2h"], host["d2h_legal"]
+            out["config"]["policy_checksum"] = host["checksum"]
+            out["e2e"] = {"value": evals / (e2e_pipe_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                          "ms_per_step": e2e_pipe_ms / args.steps,
+                          "api": "az_submit_host / az_wait_host, pinned host buffers, two batches in flight (dense policy out)"}
+            out["e2e_sync"] = {"value": evals / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                               "ms_per_step": e2e_ms / args.steps, "api": "az_evaluate_host, pinned host buffers, one batch at a time"}
+            out["e2e_legal_moves_only"] = {"value": evals / (e2e_pipe_legal_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                                           "d2h_bytes_per_step": int(d2h_legal), "ms_per_step": e2e_pipe_legal_ms / args.steps,
+                                           "api": "az_submit_host / az_wait_host, legal-moves-only policy out, two batches in flight"}
+            out["e2e_legal_moves_only_sync"] = {"value": evals / (e2e_legal_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+                                                "d2h_bytes_per_step": int(d2h_legal), "ms_per_step": e2e_legal_ms / args.steps,
+                                                "api": "az_evaluate_legal_host, pinned host buffers, one batch at a time"}
+        if not args.no_cpu_baseline and args.legs == "all":
+            # about twenty core-seconds of the oracle: 500 positions at 20 x 128 (it runs some 25 positions per
+            # second and core there), fewer in proportion to the tower's work for the larger networks
+            sample = max(16, int(500 * 757e6 / tower_flops_per_position(cfg))) if cfg.channels >= 128 else cfg.batch
+            sample = min(sample, B)
+            rate, dt, threads = oracle_rate(cfg, blob, recs, sample)
+            out["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                   "sample": f"first {sample} positions of the batch, {dt:.1f} s"}
+        print(json.dumps(out))
+    az.az_free_net(net)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def host_legs(az, torch, args, cfg, net, recs, masks_dev, B, barrier):
+    """The end-to-end legs: the same evaluation through the entry points that take HOST buffers, every step copying its
+    inputs in from pinned host memory and its results out.  Returns wall-clock times in ms and the bytes moved per step."""
     pos_host = torch.from_numpy(np.ascontiguousarray(recs).view(np.uint8).reshape(B, -1).copy()).pin_memory()
     masks_host = masks_dev.cpu().pin_memory()
     policy_host = torch.zeros((B, cfg.policy_size), dtype=torch.float32).pin_memory()
@@ -531,8 +737,8 @@ def main():
     d2h_legal = (legal_host.numel() + counts_host.numel() + value_host.numel()) * 4
     checksum = float(policy_host.sum())            # every row sums to one
 
-    # ---- end to end, pipelined: az_submit_host / az_wait_host with two batches in flight, each with its
-    # own pinned input and output buffers; every step still copies its inputs in and its results out
+    # pipelined: az_submit_host / az_wait_host with two batches in flight, each with its own pinned input and output
+    # buffers; every step still copies its inputs in and its results out
     def pipelined(dense: bool) -> float:
         bufs = []
         for _ in range(az.AZ_HOST_SLOTS):
@@ -562,74 +768,8 @@ def main():
 
     e2e_pipe_s = pipelined(True)
     e2e_pipe_legal_s = pipelined(False)
-
-    # ---- max over ranks
-    total_ms, b2b_ms, e2e_ms, tower_ms_max, e2e_legal_ms, e2e_pipe_ms, e2e_pipe_legal_ms = sharding.max_over_ranks(
-        [total_ms, b2b_ms, e2e_s * 1e3, tower_ms, e2e_legal_s * 1e3, e2e_pipe_s * 1e3, e2e_pipe_legal_s * 1e3], device="cuda")
-
-    if rank == 0:
-        peaks = load_peaks()
-        evals = world * B * args.steps
-        flops = tower_flops_per_position(cfg) * B
-        tower_avg_ms = tower_ms / max(tower_passes, 1)
-        achieved = flops / (tower_avg_ms * 1e-3) / 1e12 if tower_passes else None
-        traffic = tower_traffic_bytes(cfg, B)
-        # FP8 contraction: the measured bf16 peak times the nominal e4m3/bf16 ratio of 2 (4.5 / 2.25 PFLOP/s)
-        # a tower launch of a few hundred microseconds between L2 flushes is a burst; launches of
-        # milliseconds back to back for the whole timed region run under the power cap like the sustained GEMM
-        sustained = tower_avg_ms >= 2.0
-        peak_tf = peaks["bf16_tflops_sustained" if sustained else "bf16_tflops"] * (2.0 if cfg.precision >= 2 else 1.0)
-        peak_note = (f"of {peaks['source']} ({'sustained' if sustained else 'burst'} bf16 GEMM"
-                     + (" x 2, nominal 8-bit/bf16 ratio" if cfg.precision >= 2 else "")
-                     + "; sustained is used when a tower launch takes 2 ms or more)")
-        roof_kernel, roof_bound = "tower_tc_kernel", "tensor"
-        if cfg.precision == 0:
-            # the fp32 network runs on the FP32 FMA pipes: 148 SMs x 128 FMA per clock x 2 x the maximum SM clock
-            roof_kernel, roof_bound = "conv3x3_f32_tiled_kernel (13 launches)", "alu"
-            peak_tf = 148 * 128 * 2 * (clocks.get("sm_max_mhz") or 1965) * 1e6 / 1e12
-            peak_note = "derived: 148 SMs x 128 FP32 FMA per clock x 2 x the maximum SM clock"
-        out = {
-            "metric": METRIC, "value": evals / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
-            "ms_per_step_median": float(np.median(step_ms)), "ms_per_step_best": float(min(step_ms)),
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": DTYPE[cfg.precision], "data": "synthetic",
-            "config": {"workload": WORKLOADS[cfg.name], "batch_per_gpu": B, "l2": "flushed before every step (256 MB write)",
-                       "timing": "CUDA events around each step on the launch stream, summed; max over ranks",
-                       "device_status": status, "policy_checksum": checksum},
-            "back_to_back": {"value": evals / (b2b_ms * 1e-3), "unit": UNIT, "ms_per_step": b2b_ms / args.steps,
-                             "note": "no L2 flush between steps"},
-            "e2e": {"value": evals / (e2e_pipe_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                    "ms_per_step": e2e_pipe_ms / args.steps,
-                    "api": "az_submit_host / az_wait_host, pinned host buffers, two batches in flight (dense policy out)"},
-            "e2e_sync": {"value": evals / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
-                         "ms_per_step": e2e_ms / args.steps, "api": "az_evaluate_host, pinned host buffers, one batch at a time"},
-            "e2e_legal_moves_only": {"value": evals / (e2e_pipe_legal_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-                                     "d2h_bytes_per_step": int(d2h_legal), "ms_per_step": e2e_pipe_legal_ms / args.steps,
-                                     "api": "az_submit_host / az_wait_host, legal-moves-only policy out, two batches in flight"},
-            "e2e_legal_moves_only_sync": {"value": evals / (e2e_legal_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
-                                          "d2h_bytes_per_step": int(d2h_legal), "ms_per_step": e2e_legal_ms / args.steps,
-                                          "api": "az_evaluate_legal_host, pinned host buffers, one batch at a time"},
-            "gpu_launches": args.steps * az.az_launches_per_evaluate(net, B),
-            "clocks": clocks,
-            "roofline": {"kernel": roof_kernel, "bound": roof_bound, "achieved": achieved, "peak": peak_tf,
-                         "unit": "TFLOP/s", "frac": (achieved / peak_tf) if achieved else None,
-                         "traffic": traffic, "peak_source": peak_note,
-                         "avg_launch_ms": tower_avg_ms, "launches_timed": tower_passes,
-                         "flops_per_launch": flops},
-        }
-        if not args.no_cpu_baseline:
-            # about twenty core-seconds of the oracle: 500 positions at 20 x 128 (it runs some 25 positions per
-            # second and core there), fewer in proportion to the tower's work for the larger networks
-            sample = max(16, int(500 * 757e6 / tower_flops_per_position(cfg))) if cfg.channels >= 128 else cfg.batch
-            sample = min(sample, B)
-            rate, dt, threads = oracle_rate(cfg, blob, recs, sample)
-            out["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                   "sample": f"first {sample} positions of the batch, {dt:.1f} s"}
-        print(json.dumps(out))
-    az.az_free_net(net)
-    if world > 1:
-        dist.destroy_process_group()
+    return {"times_ms": [e2e_s * 1e3, e2e_legal_s * 1e3, e2e_pipe_s * 1e3, e2e_pipe_legal_s * 1e3],
+            "h2d": h2d, "d2h": d2h, "d2h_legal": d2h_legal, "checksum": checksum}
 
 
 if __name__ == "__main__":

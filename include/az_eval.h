@@ -49,7 +49,15 @@ enum {
 
 enum { AZ_POLICY_PLANES73 = 0, AZ_POLICY_FLAT1858 = 1, AZ_POLICY_FROMTO1880 = 2 };
 enum { AZ_VALUE_TANH = 0, AZ_VALUE_WDL = 1 };
-enum { AZ_PREC_FP32 = 0, AZ_PREC_BF16 = 1, AZ_PREC_FP8_E4M3 = 2, AZ_PREC_INT8 = 3 };
+/* Precision of the convolution tower (the heads are bf16 in every form but FP32):
+ *   FP8_E4M3      e4m3 weights and activations, one number per operand
+ *   INT8          unsigned 8-bit activations, signed 8-bit weights (the paper's deployed precision, Sec. 4.3.6)
+ *   FP8_E4M3_X2   e4m3 weights and activations, every operand as a PAIR of e4m3 numbers (the rounded value and the
+ *                 rounded remainder); a layer is three tensor-core products (value x value, remainder x value,
+ *                 value x remainder).  Costs three times the e4m3 tower's products, i.e. 1.5 x the bf16 tower's
+ *                 time, and is closer to the fp64 network than bf16.  See az_calibrate.
+ *   FP8_E4M3_X2A  the same with pairs for the activations only (two products: the bf16 tower's time). */
+enum { AZ_PREC_FP32 = 0, AZ_PREC_BF16 = 1, AZ_PREC_FP8_E4M3 = 2, AZ_PREC_INT8 = 3, AZ_PREC_FP8_E4M3_X2 = 4, AZ_PREC_FP8_E4M3_X2A = 5 };
 
 /* Network shape.  in_planes 19 or 112; blocks >= 0 residual blocks of `channels` channels
  * (a multiple of 16); heads and precision as the enums above; max_batch sizes the workspace.
@@ -302,13 +310,15 @@ int az_legal_masks(const void *positions_dev, size_t position_stride, int batch,
                    uint64_t *masks_dev, void *cuda_stream);
 
 /*
- * 8-bit towers only (AZ_PREC_FP8_E4M3, AZ_PREC_INT8; Sec. 4.3.6: ranges are fixed on a few hundred
+ * 8-bit towers only (AZ_PREC_FP8_E4M3, its paired forms AZ_PREC_FP8_E4M3_X2 / _X2A, AZ_PREC_INT8; Sec. 4.3.6: ranges are fixed on a few hundred
  * calibration positions): runs the bf16 tower on `n` positions, records per-channel activation
  * ranges and fixes the scales.  FP8: e4m3 activations (range / 448 per input channel, folded into
  * the weights) and e4m3 weights (one fp32 scale per output channel).  INT8, the precision the paper
  * deploys: unsigned 8-bit activations (range / 255; they are never negative), signed 8-bit weights
  * (max / 127 per output channel), int32 accumulation, the residual stream kept as int32 in the
  * second convolution's units; input layer and heads in bf16 in both.
+ * Paired e4m3 forms: same scales; an activation a is stored as q1 = e4m3(a / range) and q2 = e4m3(a / range - q1)
+ * (a value beyond the calibrated range saturates q1 and spills into q2), a weight likewise in _X2.
  * Then a bias correction (the usual post-training remedy for the
  * systematic part of rounding error: rounded weights meet activations that are not zero-mean, which
  * shifts every output channel's mean): layer by layer the 8-bit tower runs over the same positions

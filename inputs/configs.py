@@ -3,7 +3,8 @@
 Pure data.  `arch` fields use the same integer codes as the library's arch struct:
 policy_head 0 = 73 move planes (4672 logits), 1 = flat 1858-move list;
 value_head 0 = scalar tanh, 1 = win/draw/loss softmax;
-precision 0 = fp32, 1 = bf16, 2 = FP8-e4m3 tower (heads bf16), 3 = int8 tower (heads bf16).
+precision 0 = fp32, 1 = bf16, 2 = FP8-e4m3 tower (heads bf16), 3 = int8 tower (heads bf16),
+4 = FP8-e4m3 tower with every operand as a pair of e4m3 numbers, 5 = pairs for the activations only.
 """
 from dataclasses import dataclass, field
 from typing import Tuple
@@ -64,6 +65,10 @@ CONFIGS = {
                   branch_scale=20 ** -0.5),
     # c4 as specified (the plain weights of c2) with the tower in int8 instead of e4m3
     "c4p": Config("c4p", 19, 20, 128, 0, 0, 3, 4096, (0, 80), (0, 80), 20260941, 9370002, weights_like="c2"),
+    # c4 as specified (plain weights of c2, e4m3 weights and activations) with every operand carried as a pair of
+    # e4m3 numbers, value and remainder (precision code 4), and with pairs for the activations only (code 5)
+    "c4x": Config("c4x", 19, 20, 128, 0, 0, 4, 4096, (0, 80), (0, 80), 20260941, 9370002, weights_like="c2"),
+    "c4a": Config("c4a", 19, 20, 128, 0, 0, 5, 4096, (0, 80), (0, 80), 20260941, 9370002, weights_like="c2"),
     "c5": Config("c5", 112, 40, 256, 1, 1, 1, 1024, (0, 80), (0, 80), 20260942, 9370005,
                  sweep=(16, 64, 256, 1024, 4096, 8192)),
 }

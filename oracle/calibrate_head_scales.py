@@ -6,16 +6,18 @@ vacuous.  Following the paper's own bootstrap (a small final policy projection, 
 set on a few hundred encoded positions, no chess targets: Sec. 4.3.5), the LAST linear layer of
 each head is multiplied by a scalar chosen on 512 seeded calibration positions so that
   * the standard deviation of a position's legal-move logits averages 1.0, and
-  * the value head's pre-activation has standard deviation 0.2 for the three win/draw/loss
-    logits and 0.03 for the scalar tanh head.  Why so small: an emulation with bf16-rounded
-    operands but EXACT accumulation (the floor of any bf16 kernel) leaves the towers' activations
-    0.6-0.7 % (rms) off, and the value heads turn that into a pre-activation error of a quarter
-    to a third of the head's spread over positions.  At a spread of 0.5 that floor alone is
-    0.03-0.05 in the tanh output of the 20x128 net and 0.03 in the win/draw/loss probabilities
-    of the 40x256 net, outside the 2e-2 bar for every possible bf16 implementation.  The tanh
-    head has unit slope near the origin and no softmax to cancel an error common to its logits,
-    hence the smaller figure.  A value head with a small final projection is also what an
-    untrained bootstrap network looks like.
+  * the value head's pre-activation has standard deviation 0.5 over positions (for the three
+    win/draw/loss logits: of the centred logits) wherever the arithmetic allows it: the fp32 network
+    (c1) and the headline network (c3).  Two weight sets get less, VALUE_SPREAD below, and the
+    reason is measured, not assumed: `oracle/quant_emul.py` evaluates each network with
+    bf16-rounded operands and EXACT accumulation, the floor of any bf16 kernel, and
+    tests/golden/quant_floors.json keeps the result.  For c3 that floor is 0.8 % of the value
+    head's spread (4e-3 in the probabilities at spread 0.5).  For the c2 weights (scalar tanh head)
+    and the c5 weights it is 9-10 % of the spread: at 0.5 the floor alone is 0.03 in the output,
+    outside the 2e-2 bar for every possible bf16 implementation, so c2 is scaled to 0.03 and c5
+    to 0.14 for the test that gates on 2e-2, and a second test evaluates them at 0.5 and gates on
+    the error RELATIVE to the spread.  (The draw of the value head's weights decides this: c2's
+    and c5's heads cancel large hidden contributions, c3's does not.)
 The scalars become part of the weights, so the oracle and the CUDA library see the same network.
 
 Calls only the oracle and the input generators.  Usage:  python -m oracle.calibrate_head_scales
@@ -28,6 +30,10 @@ import numpy as np
 
 import oracle
 from inputs import configs, positions, weights
+
+
+# standard deviation of the value head's pre-activation over the calibration positions, per weight set
+VALUE_SPREAD = {"c1": 0.5, "c2": 0.03, "c3": 0.5, "c4b": 0.03, "c5": 0.14}
 
 
 def scales_for(cfg) -> dict:
@@ -43,9 +49,11 @@ def scales_for(cfg) -> dict:
         if legal.size >= 2:
             stds.append(float(np.std(legal)))
     policy = 1.0 / float(np.mean(stds))
-    value = (0.2 if cfg.value_head == 1 else 0.03) / float(np.std(raw["value_pre"]))
-    return {"policy": policy, "value": value, "positions": int(recs.shape[0]),
-            "raw_legal_logit_std": float(np.mean(stds)), "raw_value_std": float(np.std(raw["value_pre"]))}
+    zv = raw["value_pre"]
+    zv = zv - zv.mean(axis=1, keepdims=True) if zv.shape[1] > 1 else zv
+    value = VALUE_SPREAD[cfg.name] / float(np.std(zv))
+    return {"policy": policy, "value": value, "value_spread": VALUE_SPREAD[cfg.name], "positions": int(recs.shape[0]),
+            "raw_legal_logit_std": float(np.mean(stds)), "raw_value_std": float(np.std(zv))}
 
 
 def main(names):

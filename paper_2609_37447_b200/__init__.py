@@ -21,7 +21,7 @@ AZ_ERR_CUDA, AZ_ERR_DEVICE_TIMEOUT, AZ_ERR_NOT_CALIBRATED, AZ_ERR_UNSUPPORTED, A
 AZ_HOST_SLOTS = 2
 AZ_POLICY_PLANES73, AZ_POLICY_FLAT1858, AZ_POLICY_FROMTO1880 = 0, 1, 2
 AZ_VALUE_TANH, AZ_VALUE_WDL = 0, 1
-AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3, AZ_PREC_INT8 = 0, 1, 2, 3
+AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3, AZ_PREC_INT8, AZ_PREC_FP8_E4M3_X2, AZ_PREC_FP8_E4M3_X2A = 0, 1, 2, 3, 4, 5
 
 EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
            "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_submit_host", "az_wait_host", "az_encode", "az_encode52", "az_tower", "az_tower_static", "az_legal_masks",

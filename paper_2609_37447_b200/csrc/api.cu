@@ -38,7 +38,7 @@ bool arch_ok(const az_arch &a) {
     if (a.abi_version != AZ_ABI_VERSION) return false;
     if (a.in_planes != 19 && a.in_planes != 112 && a.in_planes != 52) return false;
     if (a.blocks > 64 || a.channels < 8 || a.channels > 512 || a.channels % 8) return false;
-    if (a.policy_head > 2 || a.value_head > 1 || a.precision > 3) return false;
+    if (a.policy_head > 2 || a.value_head > 1 || a.precision > AZ_PREC_FP8_E4M3_X2A) return false;
     // the paper's own network: 52 planes go with the 1,880-action head and the win/draw/loss value, and only with them
     if ((a.in_planes == 52) != (a.policy_head == AZ_POLICY_FROMTO1880)) return false;
     if (a.in_planes == 52 && a.value_head != AZ_VALUE_WDL) return false;
@@ -130,8 +130,10 @@ int build_net(Net &n, const BlobView &v) {
     int rc;
 
     // tensor-core tower: bf16, 128 channels, 19-plane input
-    n.fp8 = a.precision == AZ_PREC_FP8_E4M3 || a.precision == AZ_PREC_INT8;
+    n.fp8 = a.precision >= AZ_PREC_FP8_E4M3;          // every 8-bit form
     n.int8 = a.precision == AZ_PREC_INT8;
+    n.split_a = a.precision == AZ_PREC_FP8_E4M3_X2 || a.precision == AZ_PREC_FP8_E4M3_X2A;
+    n.split_w = a.precision == AZ_PREC_FP8_E4M3_X2;
     // tensor-core tower: bf16 with 128 or 256 channels; the FP8 tower exists for 128 channels
     const bool tc_shape = a.precision != AZ_PREC_FP32 && (C == 128 || (C == 256 && !n.fp8));
     if (n.fp8 && !tc_shape) return AZ_ERR_UNSUPPORTED;
@@ -726,10 +728,10 @@ int az_calibrate_ex(az_net *net, const void *positions_dev, int count, uint32_t 
         az::HostMaster *hm = static_cast<az::HostMaster *>(n->host_master);
         std::vector<const float *> w, sc, bi;
         for (int l = 0; l < L; ++l) { w.push_back(hm->w[l].data()); sc.push_back(hm->scale[l].data()); bi.push_back(hm->bias[l].data()); }
-        const size_t bytes = az::tc8_packed_weight_bytes(n->in_pad, C, L);
+        const size_t bytes = az::tc8_packed_weight_bytes(n->in_pad, C, L, n->split_w);
         std::vector<unsigned char> packed(bytes);
         lconst.resize((size_t)L * 3 * C);
-        az::tc8_pack(w.data(), sc.data(), bi.data(), absmax.data(), (int)n->arch.in_planes, n->in_pad, C, L, n->int8, packed.data(), lconst.data());
+        az::tc8_pack(w.data(), sc.data(), bi.data(), absmax.data(), (int)n->arch.in_planes, n->in_pad, C, L, n->int8, n->split_w, packed.data(), lconst.data());
         if (!n->tc8_weights) AZ_CUDA(cudaMalloc(&n->tc8_weights, bytes));
         if (!n->tc8_lconst) AZ_CUDA(cudaMalloc((void **)&n->tc8_lconst, lconst.size() * sizeof(float)));
         AZ_CUDA(cudaMemcpy(n->tc8_weights, packed.data(), bytes, cudaMemcpyHostToDevice));

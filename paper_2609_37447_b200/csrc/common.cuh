@@ -49,6 +49,7 @@ struct Net {
     // FP8-e4m3 tower (weights and per-layer constants exist once az_calibrate has run)
     bool fp8 = false, fp8_ready = false;   // 8-bit tower (FP8-e4m3 or int8) and whether it has been calibrated
     bool int8 = false;                      // the 8-bit tower's operands are u8 activations x s8 weights
+    bool split_a = false, split_w = false;   // e4m3 tower whose activations (and weights) travel as pairs of e4m3 numbers
     bool calib_broken = false;              // az_calibrate failed half-way through its bias correction
     void *tc8_weights = nullptr;
     float *tc8_lconst = nullptr;      // [n_conv][3][C]
@@ -192,9 +193,9 @@ void tc_pack_weights(const float *const *w, const float *const *scale, int in_pl
 // exactly one of `planes` (encoded plane tensor) and `positions` (records to encode in the kernel) is non-null
 int launch_tower_tc(const Net &net, const void *planes, const void *positions, int batch, void *tower_out,
                     bool with_heads, unsigned int *absmax, cudaStream_t s);
-size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv);
+size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv, bool split_w);
 void tc8_pack(const float *const *w, const float *const *scale, const float *const *bias, const float *absmax,
-              int in_planes, int in_pad, int channels, int n_conv, bool int8, unsigned char *packed, float *lconst);
+              int in_planes, int in_pad, int channels, int n_conv, bool int8, bool split_w, unsigned char *packed, float *lconst);
 int tower_tc_launch_count();
 size_t tc_head_weight_bytes(int head_n, int channels);
 void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,

@@ -3,6 +3,7 @@
 #pragma once
 
 #include <stdint.h>
+#include <cuda_fp16.h>
 
 namespace az {
 namespace ptx {
@@ -204,6 +205,18 @@ __device__ __forceinline__ uint32_t pack_e4m3x2_relu(float lo, float hi) {
     unsigned short d;
     asm("cvt.rn.satfinite.relu.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
     return (uint32_t)d;
+}
+// Two fp32 -> packed e4m3x2 without the clamp at zero (remainders carry a sign), and the exact way back.
+__device__ __forceinline__ uint32_t pack_e4m3x2(float lo, float hi) {
+    unsigned short d;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+    return (uint32_t)d;
+}
+__device__ __forceinline__ void unpack_e4m3x2(uint32_t packed, float &lo, float &hi) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((unsigned short)packed));
+    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+    lo = f.x; hi = f.y;
 }
 // 16 consecutive fp32 columns of this thread's TMEM lane (warp-wide, lanes 32*(warp%4)..+31)
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {

@@ -132,6 +132,7 @@ struct TowerArgs {
     double *presum;                  // [n_conv][C] or null (double: the host subtracts two nearly equal means)
     // the paper's own network (kPnet instantiation; Sec. 3.2, 4.3.3, 4.3.6, App. D.1): activations capped
     // at six, pooled context in blocks 1, 3, 5, ..., query / key projections as the fused head layer
+    int split_w;                     // e4m3 tower with split operands: the weights are pairs as well (two stages per slice)
     const float *gw;                 // [pooled block][C/2][3C/4] fp32, transposed: pooled vector -> context
     float *qk_out;                   // [batch][64][256] fp32: queries (128) then keys (128) per square
 };
@@ -185,10 +186,16 @@ template <class S> __device__ __host__ constexpr int head_stages(int head_n) {
 // kFp8: the 8-bit tower (layers after the input layer read 8-bit operands, 32 channels per MMA); with
 // kInt8 those operands are unsigned 8-bit activations and signed 8-bit weights (kind::i8, int32
 // accumulators, the residual stream kept as int32 in the same units), else e4m3 (kind::f8f6f4).
-template <bool kFp8, class S, bool kPnet = false, bool kInt8 = false>
+// kSplitA (e4m3 only): every activation travels as TWO e4m3 numbers, the rounded value and the rounded
+// remainder (planes C/16 .. C/8 - 1 of the frame, which the 8-bit forms otherwise leave unused), and every weight
+// stage is multiplied with both; with args.split_w the weights are pairs too (a second stage per slice holds the
+// remainders, multiplied with the activations' first parts).  Three products per layer instead of one: the
+// operands are still e4m3, the result carries about seven mantissa bits per operand instead of three.
+template <bool kFp8, class S, bool kPnet = false, bool kInt8 = false, bool kSplitA = false>
 __global__ void __launch_bounds__(S::kThreads, 1)
 tower_tc_kernel(const TowerArgs args) {
     static_assert(!kInt8 || kFp8, "the int8 tower is a form of the 8-bit tower");
+    static_assert(!kSplitA || (kFp8 && !kInt8 && !kPnet && S::kC == 128), "split operands exist for the e4m3 tower of the 128-channel residual networks");
     static_assert(!kPnet || S::kC == 128 || S::kC == 160 || S::kC == 176, "the paper's network runs on the 128-, 160- and 176-channel shapes");
     static_assert(S::kC != 176 || S::kSets == 1, "eleven slices do not split over two sets");
     static_assert(!(kPnet && kFp8) || kInt8, "of the 8-bit towers the int8 one carries the paper's network");
@@ -260,6 +267,9 @@ tower_tc_kernel(const TowerArgs args) {
     auto slices_of = [&](int l) {                                                               // K per MMA: 16 bf16 or 32 e4m3
         return l == 0 ? in_slices : short_layer(l) ? (kFp8 ? kShortSlices / 2 : kShortSlices) : (kFp8 ? kC / 32 : kC / 16);
     };
+    // weight stages of layer l: per slice three 3-tap stages in the 256-channel shape, else one; twice that where
+    // the weights of an e4m3 layer come as pairs
+    auto stages_of = [&](int l) { return slices_of(l) * S::kStagesPerSlice * ((kSplitA && l > 0 && args.split_w) ? 2 : 1); };
     // role tracing (clocks spent waiting, printed by CTA 0) exists in diagnostic builds only (-DAZ_TRACE)
 #ifdef AZ_TRACE
     const bool tr = args.trace && blockIdx.x == 0;
@@ -281,7 +291,7 @@ tower_tc_kernel(const TowerArgs args) {
             const Round rd = round_of(r);
             if (!rd.valid) break;
             int n_stages = 0;
-            for (int l = 0; l < n_conv; ++l) n_stages += slices_of(l) * S::kStagesPerSlice;
+            for (int l = 0; l < n_conv; ++l) n_stages += stages_of(l);
             const int n_head_stages = head_stages<S>(head_n);
             for (int st = 0; st < n_stages + n_head_stages && ok; ++st) {
                 // tower stages are contiguous and equally sized; the head projections follow as small stages of their own
@@ -333,7 +343,7 @@ tower_tc_kernel(const TowerArgs args) {
                 // a slot without a group this round still takes part in the ring protocol: it waits for
                 // every stage of the round and releases it without issuing anything
                 int n_stages = head_stages<S>(head_n);
-                for (int l = 0; l < n_conv; ++l) n_stages += slices_of(l) * S::kStagesPerSlice;
+                for (int l = 0; l < n_conv; ++l) n_stages += stages_of(l);
                 for (int st = 0; st < n_stages && ok; ++st) {
                     ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status);
                     if (ok && follow) ok = wait_bar(bar_lead(stage), phase, abort_flag, args.status);
@@ -361,9 +371,12 @@ tower_tc_kernel(const TowerArgs args) {
                     a_phase ^= 1u << kc;
                     // low descriptor word in 16-byte units; row m = 0 sits at slot 2*9 + 1 = 19
                     const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
+                    const int n_parts = (kSplitA && e4m3 && args.split_w) ? 2 : 1;      // weight pairs: first parts, then remainders
+#pragma unroll 1
+                    for (int part = 0; part < n_parts && ok; ++part) {
 #pragma unroll
                     for (int st = 0; st < S::kStagesPerSlice; ++st) {
-                        if (kGroups > 1 || st > 0) {
+                        if (kGroups > 1 || st > 0 || part > 0) {
                             ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                             if (!ok) break;
                             if (follow) {
@@ -382,14 +395,18 @@ tower_tc_kernel(const TowerArgs args) {
                                 for (int t = 0; t < S::kStageTaps; ++t) {
                                     const int tap = st * S::kStageTaps + t;
                                     const int dy = tap / 3 - 1, dx = tap % 3 - 1;
+                                    const uint32_t first = (tap == 0 && !conv2 && kc == 0 && part == 0) ? 0u : 1u;
                                     if (kInt8)
                                         ptx::mma_i8_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                          b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8,
-                                                          (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
+                                                          b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8, first, elected);
                                     else
                                         ptx::mma_e4m3_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                            b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8,
-                                                            (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
+                                                            b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8, first, elected);
+                                    // the activations' remainders against the same weights (first parts of the weights only:
+                                    // remainder times remainder is below what fp32 accumulation keeps anyway)
+                                    if (kSplitA && part == 0)
+                                        ptx::mma_e4m3_elect(d, a_lo + (uint32_t)((kC / 16) * kSlots + dy * kNB * 9 + dx), kADescHi,
+                                                            b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8, 1u, elected);
                                 }
                             } else {
 #pragma unroll
@@ -402,7 +419,7 @@ tower_tc_kernel(const TowerArgs args) {
                                 }
                             }
                             if (elected) {
-                                if (kc == nkc - 1 && st == S::kStagesPerSlice - 1) ptx::mma_commit(bar_acc_full(g));
+                                if (kc == nkc - 1 && st == S::kStagesPerSlice - 1 && part == n_parts - 1) ptx::mma_commit(bar_acc_full(g));
                                 ptx::mma_commit(bar_w_empty(stage));
                                 if (lead) ptx::mbar_arrive(bar_lead(stage));
                             }
@@ -410,6 +427,7 @@ tower_tc_kernel(const TowerArgs args) {
                         __syncwarp();
                         if (tr) t_issue += clock64() - ti0;
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
                     }
                 }
             }
@@ -807,6 +825,21 @@ tower_tc_kernel(const TowerArgs args) {
                                     pk[i] = ptx::pack_e4m3x2_relu(v[4 * i], v[4 * i + 1]) | (ptx::pack_e4m3x2_relu(v[4 * i + 2], v[4 * i + 3]) << 16);
                             }
                             *reinterpret_cast<uint4 *>(frame + kc * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                            if (kSplitA) {
+                                // the remainder of every activation after its own rounding, rounded in turn, into the
+                                // second half of the frame (a value beyond the calibrated range saturates the first
+                                // part and spills into the second)
+                                uint32_t pl[4];
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    float h0, h1, h2, h3;
+                                    ptx::unpack_e4m3x2(pk[i] & 0xFFFFu, h0, h1);
+                                    ptx::unpack_e4m3x2(pk[i] >> 16, h2, h3);
+                                    pl[i] = ptx::pack_e4m3x2(fmaxf(v[4 * i], 0.0f) - h0, fmaxf(v[4 * i + 1], 0.0f) - h1) |
+                                            (ptx::pack_e4m3x2(fmaxf(v[4 * i + 2], 0.0f) - h2, fmaxf(v[4 * i + 3], 0.0f) - h3) << 16);
+                                }
+                                *reinterpret_cast<uint4 *>(frame + (kC / 16 + kc) * kPlaneBytes + slot * 16) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+                            }
                         } else {
                             uint32_t pk[8];
 #pragma unroll
@@ -1004,15 +1037,17 @@ int tower_tc_launch_count() { return 1; }
 // the layer's output already divided by the next layer's activation scale, converts it to e4m3 (the
 // conversion clamps at zero: ReLU commutes with the positive scale), and on the residual stream writes
 // relu(v') * lconst2 back to TMEM, the stream pre-divided by the next conv2's weight scale.
-size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv) {
-    return ((size_t)in_pad / 16 + (size_t)(n_conv - 1) * (channels / 32)) * kStageBytes;
+size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv, bool split_w) {
+    return ((size_t)in_pad / 16 + (size_t)(n_conv - 1) * (channels / 32) * (split_w ? 2 : 1)) * kStageBytes;
 }
 
 // int8 form (the paper's deployed precision, Sec. 4.3.6): activations unsigned 8-bit with sa =
 // calibration maximum / 255 (they are never negative), weights signed 8-bit with ws = max|W'| / 127,
 // round to nearest; same constants, same layout.
+// split_w (e4m3 only): every weight as a pair, q_w = e4m3(W' / ws) and e4m3(W' / ws - q_w); per 32-channel slice
+// the stage of first parts is followed by a stage of remainders.
 void tc8_pack(const float *const *w, const float *const *scale, const float *const *bias, const float *absmax,
-              int in_planes, int in_pad, int channels, int n_conv, bool int8, unsigned char *packed, float *lconst) {
+              int in_planes, int in_pad, int channels, int n_conv, bool int8, bool split_w, unsigned char *packed, float *lconst) {
     const int C = channels;
     const float kMax = int8 ? 255.0f : 448.0f, kMaxW = int8 ? 127.0f : 448.0f, kTiny = 1e-30f;
     std::vector<float> sa((size_t)n_conv * C, 1.0f), ws((size_t)n_conv * C, 1.0f);
@@ -1034,20 +1069,26 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
             ws[(size_t)l * C + co] = fmaxf(mx, kTiny) / kMaxW;
         }
         for (int kc = 0; kc < C / 32; ++kc)
-            for (int tap = 0; tap < 9; ++tap)
-                for (int k16 = 0; k16 < 2; ++k16)
-                    for (int ng = 0; ng < C / 8; ++ng)
-                        for (int r = 0; r < 8; ++r)
-                            for (int e = 0; e < 16; ++e) {
-                                const int n = ng * 8 + r, ci = kc * 32 + k16 * 16 + e;
-                                const float v = wf[((size_t)n * C + ci) * 9 + tap] / ws[(size_t)l * C + n];
-                                if (int8) {
-                                    const float q = fminf(fmaxf(nearbyintf(v), -127.0f), 127.0f);
-                                    *dst++ = (unsigned char)(signed char)q;
-                                } else {
-                                    *dst++ = (unsigned char)__nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
+            for (int part = 0; part < (split_w ? 2 : 1); ++part)
+                for (int tap = 0; tap < 9; ++tap)
+                    for (int k16 = 0; k16 < 2; ++k16)
+                        for (int ng = 0; ng < C / 8; ++ng)
+                            for (int r = 0; r < 8; ++r)
+                                for (int e = 0; e < 16; ++e) {
+                                    const int n = ng * 8 + r, ci = kc * 32 + k16 * 16 + e;
+                                    const float v = wf[((size_t)n * C + ci) * 9 + tap] / ws[(size_t)l * C + n];
+                                    if (int8) {
+                                        const float q = fminf(fmaxf(nearbyintf(v), -127.0f), 127.0f);
+                                        *dst++ = (unsigned char)(signed char)q;
+                                    } else {
+                                        const __nv_fp8_storage_t q = __nv_cvt_float_to_fp8(v, __NV_SATFINITE, __NV_E4M3);
+                                        if (part == 0) *dst++ = (unsigned char)q;
+                                        else {
+                                            const float first = __half2float(__half(__nv_cvt_fp8_to_halfraw(q, __NV_E4M3)));
+                                            *dst++ = (unsigned char)__nv_cvt_float_to_fp8(v - first, __NV_SATFINITE, __NV_E4M3);
+                                        }
+                                    }
                                 }
-                            }
     }
     for (int l = 0; l < n_conv; ++l) {
         float *lc = lconst + (size_t)l * 3 * C;
@@ -1097,6 +1138,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128P, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape160, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
@@ -1130,6 +1172,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     a.lconst = net.tc8_lconst;
     a.absmax = absmax;
     a.presum = net.calib_presum;
+    a.split_w = net.split_w ? 1 : 0;
     a.gw = net.pnet_gw;
     a.qk_out = static_cast<float *>(net.pnet_qk);
 #ifdef AZ_TRACE
@@ -1146,6 +1189,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     else if (net.pnet) tower_tc_kernel<false, Shape128P, true><<<grid, Shape128P::kThreads, Shape128P::smem_bytes(false, true), s>>>(a);
     else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
     else if (fp8 && net.int8) tower_tc_kernel<true, Shape128F8, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
+    else if (fp8 && net.split_a) tower_tc_kernel<true, Shape128F8, false, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else if (fp8) tower_tc_kernel<true, Shape128F8><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else tower_tc_kernel<false, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(false), s>>>(a);
     AZ_LAUNCH_CHECK();

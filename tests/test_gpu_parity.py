@@ -56,10 +56,39 @@ def compare(cfg, masks_g, pol_g, val_g, masks_o, pol_o, val_o, tol):
     print(f"{cfg.name}: n={pol_g.shape[0]} policy max-abs {perr:.3e} value max-abs {verr:.3e} arg-max agreement {agree:.4f}")
     assert perr <= tol and verr <= tol
     if pol_g.shape[0] >= 32:
-        # scale-free guard: the value must follow the oracle's ups and downs, not merely sit near it
+        # scale-free guard: the value must follow the oracle's ups and downs, not merely sit near it.  Every output
+        # component's correlation with the oracle's must reach 0.9, or what bf16 operands with exact accumulation
+        # leave of it for this weight set where that is less (tests/golden/quant_floors.json).
+        need = 0.9
+        if cfg.name in ("c2", "c3", "c5") and cfg.precision == 1:
+            need = min(0.9, stored_floor(cfg.name)["value_min_component_corr"] - 0.03)
         for k in range(val_o.shape[1]):
-            assert np.corrcoef(val_g[:, k], val_o[:, k])[0, 1] > 0.7
+            assert np.corrcoef(val_g[:, k], val_o[:, k])[0, 1] > need
+        zg, zo = value_pre(val_g), value_pre(val_o)
+        assert np.corrcoef(zg.ravel(), zo.ravel())[0, 1] > 0.9
     return agree
+
+
+def value_pre(val):
+    """The value head's pre-activation recovered from its output: atanh of the scalar, the centred logits of
+    (win, draw, loss)."""
+    val = np.asarray(val, dtype=np.float64)
+    if val.shape[1] == 1:
+        return np.arctanh(np.clip(val, -1 + 1e-9, 1 - 1e-9))
+    lg = np.log(np.clip(val, 1e-300, None))
+    return lg - lg.mean(axis=1, keepdims=True)
+
+
+def value_error_over_spread(val_g, val_o):
+    zg, zo = value_pre(val_g), value_pre(val_o)
+    return float(np.sqrt(((zg - zo) ** 2).mean()) / zo.std()), float(zo.std())
+
+
+def stored_floor(name, label="bf16"):
+    import json
+    from oracle import quant_emul
+    with open(quant_emul.GOLDEN) as f:
+        return json.load(f)[name][label]
 
 
 # ---- encoder and masks: bit-exact ------------------------------------------------------------------
@@ -205,6 +234,38 @@ def test_c2_bf16_batch_256(az):
     az.az_free_net(net)
 
 
+@pytest.mark.parametrize("name,batch", [("c2", 256), ("c3", 1024), ("c5", 48)])
+def test_value_head_error_relative_to_its_spread(az, name, batch):
+    # The max-abs bar says little about a value head whose outputs barely move: this check is free of the head's
+    # scale.  The error of the head's pre-activation (recovered from the outputs), as a fraction of its spread over
+    # positions, must stay within 1.5 x the fraction that bf16 operands with exact accumulation leave
+    # (oracle/quant_emul.py; tests/golden/quant_floors.json), at the stored head scale and, for the two weight
+    # sets whose stored spread is small, again with the value head rescaled to a spread of 0.5.
+    import dataclasses
+    cfg = dataclasses.replace(configs.CONFIGS[name], batch=batch)
+    recs = positions.records_for_planes(cfg.in_planes, positions.for_config(cfg, batch))
+    for spread in ((None,) if name == "c3" else (None, 0.5)):
+        tensors = weights.draw_tensors(cfg)
+        floor = stored_floor(name if spread is None else f"{name}@{spread}")
+        if spread is not None:
+            for k in ("v.w2", "v.b2"):
+                tensors[k] = (tensors[k] * np.float32(spread / floor_spread)).astype(np.float32)
+        blob = weights.pack_blob(cfg, tensors)
+        net, _ = load(az, cfg, blob=blob)
+        mg, pg, vg = gpu_evaluate(az, net, cfg, recs)
+        az.az_free_net(net)
+        mo, _, po, vo = oracle.evaluate(blob, recs, cfg.in_planes, cfg.policy_head)
+        frac, got_spread = value_error_over_spread(vg, vo)
+        print(f"{name} value head at spread {got_spread:.3f}: pre-activation error {frac:.4f} of the spread "
+              f"(bf16 floor {floor['value_pre_rms_over_spread']:.4f}), output max-abs {np.abs(vg - vo).max():.3e}")
+        assert frac <= 1.5 * floor["value_pre_rms_over_spread"] + 2e-3
+        for k in range(vo.shape[1]):
+            assert np.corrcoef(vg[:, k], vo[:, k])[0, 1] > min(0.9, floor["value_min_component_corr"] - 0.03)
+        assert np.corrcoef(value_pre(vg).ravel(), value_pre(vo).ravel())[0, 1] > 0.9
+        if spread is None:
+            floor_spread = got_spread          # what the stored head scale gives on these positions
+
+
 def test_c3_bf16_batch_1024_full_launch(az):
     # the launch configuration the benchmark times (batch 1024); the oracle evaluates every row
     # (a few seconds on the host cores), so the arg-max agreement is taken over 1024 positions
@@ -257,9 +318,10 @@ def test_c5_large_batches_on_sampled_rows(az, batch):
     assert np.abs(pg.sum(axis=1) - 1.0).max() < 1e-3 and np.abs(vg.sum(axis=1) - 1.0).max() < 1e-5
 
 
-def fp8_run(az, name, batch, oracle_rows):
+def fp8_run(az, name, batch, oracle_rows, calibrate_flags=0, oracle_blob=None):
     """Load the FP8 net, calibrate it on the 512 seeded calibration positions, evaluate `batch`
-    positions, and return GPU and oracle results on `oracle_rows` of them, plus tower outputs."""
+    positions, and return GPU and oracle results on `oracle_rows` of them, plus tower outputs.
+    oracle_blob: compare against the oracle's evaluation of THIS network instead of the one loaded."""
     import dataclasses
     cfg = dataclasses.replace(configs.CONFIGS[name], batch=batch)
     net, blob = load(az, cfg)
@@ -273,14 +335,15 @@ def fp8_run(az, name, batch, oracle_rows):
         az.az_evaluate(net, pos, masks, batch, policy, value)
     assert e.value.code == az.AZ_ERR_NOT_CALIBRATED
     cal = positions.cur_records(positions.for_config(cfg, calibration=True))
-    az.az_calibrate(net, az.records_to_device(cal), cal.shape[0])
+    az.az_calibrate_ex(net, az.records_to_device(cal), cal.shape[0], calibrate_flags)
     az.az_evaluate(net, pos, masks, batch, policy, value)
     tower = torch.zeros((len(oracle_rows), 64, 128), dtype=torch.bfloat16, device="cuda")
     az.az_tower(net, az.records_to_device(recs[oracle_rows]), len(oracle_rows), tower)
     torch.cuda.synchronize()
     assert az.az_device_status(net) == 0
     az.az_free_net(net)
-    mo, _, po, vo, raw = oracle.evaluate(blob, recs[oracle_rows], 19, cfg.policy_head, want_tower=True)
+    mo, _, po, vo, raw = oracle.evaluate(blob if oracle_blob is None else oracle_blob, recs[oracle_rows], 19, cfg.policy_head,
+                                         want_tower=True)
     assert (az.masks_to_numpy(masks)[oracle_rows] == mo).all()
     pg, vg = policy.cpu().numpy(), value.cpu().numpy()
     assert np.isfinite(pg).all() and np.isfinite(vg).all() and np.abs(pg.sum(axis=1) - 1).max() < 1e-3
@@ -295,33 +358,80 @@ def fp8_run(az, name, batch, oracle_rows):
 
 
 def test_c4_fp8_tower_batch_4096_does_what_e4m3_arithmetic_gives(az):
-    # Full-size launch (4096), oracle on 256 sampled rows.  An emulation of the same quantisation with
-    # EXACT accumulation (e4m3-rounded weights and activations, per-channel scales from the same kind
-    # of calibration) puts this network's tower 8.8 % rms off the fp64 tower, 7.2 % with the bias
-    # correction az_calibrate applies; the kernel must land there, not above.  Whether that is inside the
-    # 5e-2 output bar is a property of the arithmetic and of this plain residual block, tested separately below.
+    # Full-size launch (4096), oracle on 256 sampled rows.  With one e4m3 number per weight and per activation the
+    # arithmetic itself, emulated with EXACT accumulation (oracle/quant_emul.py, tests/golden/quant_floors.json,
+    # asserted in tests/test_quant_emul.py), leaves this plain residual tower 7.2 % rms off the fp64 tower after the
+    # bias correction (9.0 % before) and the policy 0.06-0.10 off: outside the 5e-2 bar before any kernel is
+    # involved (Sec. 4.3.6 reports the same failure of post-training quantisation on an ordinary tower).  The kernel
+    # must do what that arithmetic gives, not worse.
     rows = np.arange(0, 4096, 16)
+    floor = stored_floor("c4", "e4m3, bias correction")
     perr, verr, agree, tower_err = fp8_run(az, "c4", 4096, rows)
-    assert 0.03 < tower_err < 0.09
-    assert perr < 0.15 and verr < 0.15 and agree > 0.85
+    assert 0.8 * floor["tower_rms"] < tower_err < 1.15 * floor["tower_rms"]
+    assert perr < 0.13 and verr < 0.13 and agree > 0.85
 
 
-@pytest.mark.xfail(strict=False, reason="post-training FP8 of the plain residual tower: e4m3 weights and activations "
-                   "with exact accumulation already leave policy max-abs 0.05-0.12 (Sec. 4.3.6 reports the same "
-                   "failure of an ordinary tower); the 5e-2 bar is not reachable by any kernel on this network")
-def test_c4_fp8_meets_the_5e_2_bar(az):
+def test_c4_single_e4m3_operands_are_outside_the_5e_2_bar_as_their_arithmetic_is(az):
+    # kept visible: config 4 read as ONE e4m3 number per operand does not meet its bar, on the GPU as in the
+    # exact-accumulation emulation (policy floor 0.06 on 128 positions).  The forms that do meet it follow.
     perr, verr, _, _ = fp8_run(az, "c4", 512, np.arange(256))
+    floor = stored_floor("c4", "e4m3, bias correction")
+    assert floor["policy_max_abs"] > TOL[2]
+    assert perr > TOL[2] and perr < 2.5 * floor["policy_max_abs"]
+
+
+def test_c4x_e4m3_operand_pairs_meet_the_5e_2_bar(az):
+    # config 4 with e4m3 weights and activations, every operand carried as a pair of e4m3 numbers (value and
+    # remainder), three tensor-core products per layer, fp32 accumulation, per-channel scales from the 512
+    # calibration positions: inside the 5e-2 bar with room, and closer to the fp64 tower than bf16 operands get.
+    rows = np.arange(0, 4096, 16)
+    perr, verr, agree, tower_err = fp8_run(az, "c4x", 4096, rows)
+    assert tower_err < 6e-3
+    assert perr <= 2e-2 and verr <= 2e-2 and agree >= 0.97
+
+
+def test_c4a_e4m3_activation_pairs_are_inside_the_bar_with_little_room(az):
+    # pairs for the activations only (two products per layer, the bf16 tower's time): the weights' rounding is what
+    # remains; the emulation gives tower 3.9 % rms, policy 0.03, value 0.04 on 128 positions
+    rows = np.arange(0, 4096, 16)
+    floor = stored_floor("c4", "e4m3, split activations, bias correction")
+    perr, verr, agree, tower_err = fp8_run(az, "c4a", 4096, rows)
+    assert tower_err < 1.15 * floor["tower_rms"]
     assert perr <= TOL[2] and verr <= TOL[2]
+
+
+def test_c4_error_split_into_weights_and_activations(az):
+    # The decomposition: the e4m3 tower against the fp64 oracle fed the DEQUANTISED weights (what the 8-bit weight
+    # codes stand for, computed oracle-side from the oracle's own calibration pass) isolates the share of the
+    # activations' rounding; against the original weights it is the whole error.  No bias correction on either side.
+    from oracle import quant_emul as qe
+    cfg = configs.CONFIGS["c4"]
+    tensors = weights.draw_tensors(cfg)
+    net_e = qe.ResidualTower(cfg, tensors)
+    cal = positions.cur_records(positions.for_config(cfg, calibration=True))
+    sa, _ = net_e.calibrate(torch.from_numpy(oracle.encode(cal, 19)), qe.Spec("e4m3"))
+    deq_blob = weights.pack_blob(cfg, net_e.dequantised_tensors(tensors, sa, "e4m3"))
+    rows = np.arange(128)
+    whole = fp8_run(az, "c4", 512, rows, calibrate_flags=az.AZ_CALIBRATE_NO_BIAS_CORRECTION)
+    acts = fp8_run(az, "c4", 512, rows, calibrate_flags=az.AZ_CALIBRATE_NO_BIAS_CORRECTION, oracle_blob=deq_blob)
+    print(f"c4 e4m3, no bias correction: tower rms vs the fp64 network {whole[3]:.4f}, vs the fp64 network with the "
+          f"dequantised weights {acts[3]:.4f} (activations' share); policy max-abs {whole[0]:.3f} / {acts[0]:.3f}")
+    floor_all = stored_floor("c4", "e4m3")["tower_rms"]
+    floor_w = stored_floor("c4", "e4m3, weights only")["tower_rms"]
+    assert 0.85 * floor_all < whole[3] < 1.15 * floor_all
+    assert acts[3] < whole[3]                                          # the weights' rounding is part of the whole
+    # the two shares add in quadrature to the whole, within a quarter
+    assert 0.75 * whole[3] ** 2 < acts[3] ** 2 + floor_w ** 2 < 1.35 * whole[3] ** 2
 
 
 def test_c4b_fp8_with_scaled_residual_branches(az):
     # the paper's remedy (Sec. 4.3.6): residual branches scaled by 1/sqrt(depth), folded into the second
-    # convolution.  Same kernels, different weights.  Emulated floor without bias correction: tower 4.7 % rms,
-    # value well inside the bar, policy at its edge (0.04-0.07); with the bias correction of az_calibrate the
-    # kernel measures tower 4.0 %, policy 5.7e-2 (7.3e-2 without), value 1.4e-2.
+    # convolution.  Same kernels, different weights.  One e4m3 number per operand: the emulated floor with the bias
+    # correction is at the bar's edge, and so is the kernel (asserted against the floor, not against the bar).
+    floor = stored_floor("c4b", "e4m3, bias correction")
     perr, verr, agree, tower_err = fp8_run(az, "c4b", 512, np.arange(256))
-    assert 0.02 < tower_err < 0.05
-    assert verr <= TOL[2] and perr < 0.08
+    assert tower_err < 1.15 * floor["tower_rms"]
+    assert verr <= TOL[2] and perr < max(6.5e-2, 1.5 * floor["policy_max_abs"])
 
 
 def test_c4i_int8_tower_meets_the_bar_of_the_quantised_configs(az):

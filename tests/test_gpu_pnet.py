@@ -88,14 +88,21 @@ def test_p12_batch_1024():
     print(f"p12: n={cfg.batch} policy max-abs {perr:.3e} value max-abs {verr:.3e} arg-max agreement {agree:.4f}")
     # arg-max agreement: measured 0.986.  The misses are near-ties: with some 35 legal actions at a logit
     # spread of 1 about one position in sixty has its two best actions closer than the bf16 backbone's
-    # error; wherever the oracle's two best probabilities differ by more than the tolerance, the choice agrees
+    # error; wherever the oracle's two best probabilities differ by more than the tolerance, the choice agrees.
+    # The bar is what bf16 operands with EXACT accumulation leave of it (oracle/quant_emul.py: 0.977 on the first
+    # 256 of these positions, stored in tests/golden/quant_floors.json): no bf16 kernel can be asked for more.
+    import json
+    from oracle import quant_emul
+    with open(quant_emul.GOLDEN) as f:
+        floor = json.load(f)["p12"]["bf16"]
+    assert floor["argmax_agreement_clear_gap"] == 1.0
     top2 = np.sort(po, axis=1)[:, -2:]
     clear = (top2[:, 1] - top2[:, 0]) > TOL
     agree_clear = (pg.argmax(axis=1) == po.argmax(axis=1))[clear].mean()
     print(f"p12: {clear.mean():.3f} of the positions have a clear best action; agreement there {agree_clear:.4f}")
-    assert perr <= TOL and verr <= TOL and agree >= 0.975 and agree_clear == 1.0
+    assert perr <= TOL and verr <= TOL and agree >= floor["argmax_agreement"] and agree_clear == 1.0
     for k in range(3):
-        assert np.corrcoef(vg[:, k], vo[:, k])[0, 1] > 0.7
+        assert np.corrcoef(vg[:, k], vo[:, k])[0, 1] > 0.9
 
 
 def test_p14_the_reported_checkpoints_size_batch_320_and_a_ragged_multiple():
