@@ -24,7 +24,7 @@ AZ_VALUE_TANH, AZ_VALUE_WDL = 0, 1
 AZ_PREC_FP32, AZ_PREC_BF16, AZ_PREC_FP8_E4M3, AZ_PREC_INT8, AZ_PREC_FP8_E4M3_X2, AZ_PREC_FP8_E4M3_X2A = 0, 1, 2, 3, 4, 5
 
 EXPORTS = ("az_position_bytes", "az_policy_size", "az_mask_words", "az_value_size", "az_plane_channels",
-           "az_load_net", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_submit_host", "az_wait_host", "az_encode", "az_encode52", "az_tower", "az_tower_static", "az_legal_masks",
+           "az_load_net", "az_load_net_ex", "az_free_net", "az_evaluate", "az_evaluate_legal", "az_evaluate_legal_host", "az_evaluate_host", "az_submit_host", "az_wait_host", "az_encode", "az_encode52", "az_tower", "az_tower_static", "az_legal_masks",
            "az_calibrate", "az_calibrate_ex", "az_device_status", "az_profile_tower", "az_tower_time", "az_selftest_wait_timeout", "az_launches_per_evaluate", "az_strerror",
            "az_last_cuda_error",
            "az_apply_moves", "az_standin_evaluate", "az_search_create", "az_search_destroy", "az_search_set_roots", "az_search_replace_roots",
@@ -67,6 +67,8 @@ def _load_library():
         getattr(lib, name).argtypes = [ap]
     lib.az_load_net.restype = ci
     lib.az_load_net.argtypes = [ap, vp, sz, ctypes.POINTER(vp)]
+    lib.az_load_net_ex.restype = ci
+    lib.az_load_net_ex.argtypes = [ap, vp, sz, ctypes.c_uint32, ctypes.POINTER(vp)]
     lib.az_free_net.restype = None
     lib.az_free_net.argtypes = [vp]
     lib.az_evaluate.restype = ci
@@ -205,6 +207,18 @@ def az_load_net(arch: az_arch, weights_host) -> Net:
                                 else weights_host, dtype=np.uint8)
     out = ctypes.c_void_p()
     _check(_lib.az_load_net(ctypes.byref(arch), blob.ctypes.data, blob.nbytes, ctypes.byref(out)), "az_load_net")
+    return Net(out.value, arch)
+
+
+AZ_LOAD_TOWER_CTA_PAIRS = 1
+
+
+def az_load_net_ex(arch: az_arch, weights_host, flags=0) -> Net:
+    """az_load_net with options (AZ_LOAD_TOWER_CTA_PAIRS: the tower kernel as clusters of two CTAs)."""
+    blob = np.ascontiguousarray(np.frombuffer(weights_host, dtype=np.uint8) if isinstance(weights_host, (bytes, bytearray))
+                                else weights_host, dtype=np.uint8)
+    out = ctypes.c_void_p()
+    _check(_lib.az_load_net_ex(ctypes.byref(arch), blob.ctypes.data, blob.nbytes, flags, ctypes.byref(out)), "az_load_net_ex")
     return Net(out.value, arch)
 
 

@@ -146,7 +146,9 @@ int build_net(Net &n, const BlobView &v) {
         }
         const size_t bytes = tc_packed_weight_bytes(n.in_pad, C, n.n_conv);
         std::vector<__nv_bfloat16> packed(bytes / sizeof(__nv_bfloat16));
-        tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, packed.data());
+        n.tc_pair = n.want_pair && tc_pair_shape(C, (int)a.precision, false);
+        const int halves = n.tc_pair ? 2 : 1;
+        tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, halves, packed.data());
         AZ_CUDA(cudaMalloc(&n.tc_weights, bytes));
         AZ_CUDA(cudaMemcpy(n.tc_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
         std::vector<float> bias((size_t)n.n_conv * C);
@@ -168,7 +170,7 @@ int build_net(Net &n, const BlobView &v) {
         const int n_policy = flat ? kHeadChannels : kPlanes73, n_policy_pad = flat ? kHeadChannels : 80;
         n.tc_head_n = n_policy_pad + kHeadChannels;
         std::vector<__nv_bfloat16> hw(tc_head_weight_bytes(n.tc_head_n, C) / sizeof(__nv_bfloat16));
-        tc_pack_head(v.p_w, flat ? v.p_s : nullptr, n_policy, n_policy_pad, v.v_cw, v.v_cs, C, hw.data());
+        tc_pack_head(v.p_w, flat ? v.p_s : nullptr, n_policy, n_policy_pad, v.v_cw, v.v_cs, C, halves, hw.data());
         AZ_CUDA(cudaMalloc(&n.tc_head_w, hw.size() * sizeof(__nv_bfloat16)));
         AZ_CUDA(cudaMemcpy(n.tc_head_w, hw.data(), hw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
         std::vector<float> hb(n.tc_head_n, 0.0f);
@@ -369,11 +371,17 @@ size_t az_value_size(const az_arch *a) { return a && a->value_head == AZ_VALUE_W
 size_t az_plane_channels(const az_arch *a) { return a && a->in_planes == 112 ? 128 : a && a->in_planes == 52 ? 64 : 32; }
 
 int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az_net **out) {
+    return az_load_net_ex(arch, weights_host, nbytes, 0u, out);
+}
+
+int az_load_net_ex(const az_arch *arch, const void *weights_host, size_t nbytes, uint32_t flags, az_net **out) {
     static_assert(sizeof(az_position) == 104 && sizeof(az_position_h8) == 784 && sizeof(az_position_m8) == 128, "record layout");
     if (!arch || !weights_host || !out) return AZ_ERR_BAD_ARG;
     *out = nullptr;
+    if (flags & ~(uint32_t)AZ_LOAD_TOWER_CTA_PAIRS) return AZ_ERR_BAD_ARG;
     if (!az::arch_ok(*arch)) return AZ_ERR_BAD_ARCH;
     const bool pnet = arch->in_planes == 52;
+    if ((flags & AZ_LOAD_TOWER_CTA_PAIRS) && !az::tc_pair_shape((int)arch->channels, (int)arch->precision, pnet)) return AZ_ERR_UNSUPPORTED;
     // the paper's network ladder: 128, 160 and 176 channels in bf16; 128 and 160 also in int8 (its MMAs take 32
     // channels at a time, which 176 is not a multiple of)
     if (pnet && !((arch->precision == AZ_PREC_BF16 && (arch->channels == 128 || arch->channels == 160 || arch->channels == 176)) ||
@@ -386,6 +394,7 @@ int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az
     Net *n = new (std::nothrow) Net();
     if (!n) return AZ_ERR_BAD_ARG;
     n->arch = *arch;
+    n->want_pair = (flags & AZ_LOAD_TOWER_CTA_PAIRS) != 0;
     cudaError_t e = cudaGetDevice(&n->device);
     if (e != cudaSuccess) { az::set_cuda_error(e, "cudaGetDevice"); delete n; return AZ_ERR_CUDA; }
     rc = pnet ? az::build_pnet(*n, static_cast<const unsigned char *>(weights_host), nbytes) : az::build_net(*n, view);

@@ -46,6 +46,8 @@ struct Net {
     void *tc_weights = nullptr;       // packed UMMA B-operand tiles, all layers
     float *tc_bias = nullptr;         // [n_conv][C] folded bias (scales are folded into the weights)
     bool tc_ready = false;
+    bool want_pair = false;           // az_load_net_ex was asked for the CTA-pair form of the tower
+    bool tc_pair = false;             // the bf16 128-channel tower runs on CTA pairs (tcgen05 .cta_group::2)
     // FP8-e4m3 tower (weights and per-layer constants exist once az_calibrate has run)
     bool fp8 = false, fp8_ready = false;   // 8-bit tower (FP8-e4m3 or int8) and whether it has been calibrated
     bool int8 = false;                      // the 8-bit tower's operands are u8 activations x s8 weights
@@ -189,7 +191,8 @@ int launch_masked_softmax(const float *logits, const uint64_t *masks, int batch,
 // tensor-core tower (tower_tc.cu)
 size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv);
 void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
-                     int channels, int n_conv, __nv_bfloat16 *packed_host);
+                     int channels, int n_conv, int halves, __nv_bfloat16 *packed_host);
+bool tc_pair_shape(int channels, int precision, bool pnet);     // the tower runs on CTA pairs (weights packed in halves)
 // exactly one of `planes` (encoded plane tensor) and `positions` (records to encode in the kernel) is non-null
 int launch_tower_tc(const Net &net, const void *planes, const void *positions, int batch, void *tower_out,
                     bool with_heads, unsigned int *absmax, cudaStream_t s);
@@ -199,7 +202,7 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
 int tower_tc_launch_count();
 size_t tc_head_weight_bytes(int head_n, int channels);
 void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,
-                  int channels, __nv_bfloat16 *packed);
+                  int channels, int halves, __nv_bfloat16 *packed);
 
 // tensor-core fully-connected layers of the heads (fc_tc.cu)
 size_t fc_tc_weight_bytes(int n);

@@ -182,6 +182,71 @@ __device__ __forceinline__ uint32_t cvt_u8_sat(float v) {
     asm("cvt.rni.sat.u8.f32 %0, %1;" : "=r"(d) : "f"(v));
     return d;
 }
+// ---- CTA pairs (a cluster of two CTAs on neighbouring SMs working on one 256-row MMA tile) --------------------
+// tcgen05 with .cta_group::2: the MMA is issued by one thread of the pair's first CTA; each CTA supplies its own 128
+// rows of A and its own HALF of the B tile (N/2 rows) from its own shared memory, at the same offsets in both, and
+// receives its 128 rows of D in its own TMEM.  Every B byte is read from shared memory once per pair instead of
+// once per CTA.  Nothing here is a multicast: each CTA bulk-copies its own half of every weight stage, and
+// completion is signalled to each CTA's barrier by a commit of its own.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// the shared::cluster address of `addr` (a shared::cta address of this CTA) in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {     // acquire at cluster scope
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+// TMEM allocation for a pair: the same warp of BOTH CTAs executes these, with the same arguments
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void mma_bf16_elect_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                    uint32_t idesc, uint32_t accumulate, uint32_t elected) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 p, %6, 0;\n"
+        "setp.ne.b32 q, %7, 0;\n"
+        "mov.b64 da, {%1, %2};\n"
+        "mov.b64 db, {%3, %4};\n"
+        "@q tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elected));
+}
+// the barrier at shared-memory offset `bar` in BOTH CTAs of the pair arrives once all MMAs issued so far by this
+// thread have completed: two plain commits, one per CTA's barrier (shared::cluster addresses)
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
+    const uint32_t b0 = map_to_cta(bar, 0), b1 = map_to_cta(bar, 1);
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(b0) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(b1) : "memory");
+}
 // mbarrier arrives once all MMAs issued so far by this thread have completed
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
@@ -251,12 +316,13 @@ __device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontr
 // Returns false (to every lane alike) if the CTA has been aborted or this wait ran out; the latter
 // raises the CTA's abort flag and ORs `timeout_bit` into the status word the host reads.  Callers
 // stop issuing work, drain what is in flight and leave through their normal teardown.
+template <bool kClusterScope = false>
 __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
                                              uint32_t timeout_bit, uint32_t limit, long long *waited = nullptr) {
     const long long t0 = waited ? clock64() : 0;
     bool done = false;
     for (uint32_t i = 0; i < limit; ++i) {
-        if (ptx::mbar_try_wait(bar, parity)) { done = true; break; }
+        if (kClusterScope ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity)) { done = true; break; }
         if ((i & 63u) == 63u && *abort_flag) break;
     }
     if (!done && !*abort_flag) {

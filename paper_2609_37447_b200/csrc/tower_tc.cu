@@ -65,24 +65,32 @@ constexpr uint32_t kSpinLimit = 1u << 24;
 // one group as well (two would need 640 TMEM columns), stages of 9 taps.
 // SETS: how many sets of four epilogue warps share a group's layer (each set takes a contiguous run of
 // the 16-channel slices).  Two sets for the FP8 tower, whose MMAs are twice as fast as its epilogue needs.
-template <int C, int GROUPS, int SETS>
+// PAIR: two CTAs on neighbouring SMs (a cluster of two) share every MMA: M = 256 rows, 128 from each CTA's own
+// frame, N = C with each CTA holding HALF of every weight tile in its own shared memory (tcgen05 .cta_group::2).
+// The shared-memory pipe that bounds the 128-channel shape then carries 6 KB of operands per MMA instead of 8.
+template <int C, int GROUPS, int SETS, bool PAIR = false>
 struct Shape {
     static constexpr int kC = C, kGroups = GROUPS, kSets = SETS;
+    static constexpr bool kPair = PAIR;
+    static constexpr int kHalves = PAIR ? 2 : 1;
     static constexpr int kSlices = kC / 16;                          // 16-channel slices of a layer's output
     static constexpr int kFrameBytes = kPlaneBytes * (kC / 8);       // 46336 / 92672 per group
-    static constexpr int kTileBytes = kC * 32;                       // one tap: N = C rows x 32 bytes of K
+    static constexpr int kTileBytes = kC * 32 / kHalves;             // one tap: N = C (pair: C / 2) rows x 32 bytes of K
     static constexpr int kStageTaps = kC == 256 ? 3 : 9;
     static constexpr int kStagesPerSlice = 9 / kStageTaps;
-    static constexpr int kStageBytes = kStageTaps * kTileBytes;      // 36864 / 24576
-    static constexpr int kStages = kC == 256 ? 5 : 3;
+    static constexpr int kStageBytes = kStageTaps * kTileBytes;      // 36864 / 24576; pair: 18432
+    static constexpr int kStages = kC == 256 ? 5 : PAIR ? 7 : 3;
+    // pair: the second group's issuer runs this many weight stages behind the first's (half a layer), so that each
+    // group's layer hand-over falls into the middle of the other's layer; the halved stages make the ring deep enough
+    static constexpr int kLag = PAIR ? 4 : 0;
     static constexpr int kEpiWarps = 4 * kGroups * kSets;
     static constexpr int kThreads = 32 * (1 + kGroups + kEpiWarps);  // producer, one issuer per group, 4 epilogue warps per group and set
-    static constexpr uint32_t kBDescLbo = (uint32_t)kC << 16;        // K core matrices C*16 bytes apart
+    static constexpr uint32_t kBDescLbo = (uint32_t)(kC / kHalves) << 16;   // K core matrices (rows of this CTA's tile)*16 bytes apart
     static constexpr int kOffFrames = 0;
     static constexpr int kOffWeights = kGroups * kFrameBytes;
     static constexpr int kOffBars = kOffWeights + kStages * kStageBytes;
-    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done, lead[S], pool[G]
-    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1 + kStages + kGroups;
+    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done, lead[S], pool[G], peer_full[S]
+    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1 + kStages + kGroups + kStages;
     static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
     static constexpr int kOffAbort = kOffTmemPtr + 4;
     static constexpr int kOffConst = (kOffAbort + 4 + 15) & ~15;     // per-warp copies of the current layer's channel constants
@@ -95,7 +103,7 @@ struct Shape {
         return kOffConst + kEpiWarps * (fp8 ? (pnet ? 4 : 3) : 1) * (kC / kSets) * 4 + 256 * 4 + (pnet ? kPoolFloats * 4 : 0);
     }
     // (four constant vectors per channel in the 8-bit forms, one in bf16; the 176-channel shape exists in bf16 only)
-    static_assert(kOffConst + kEpiWarps * (kC == 176 ? 1 : 4) * (kC / kSets) * 4 + 1024 + kPoolFloats * 4 <= kMaxSmem || kC == 256, "shared memory budget");
+    static_assert(kOffConst + kEpiWarps * ((kC == 176 || PAIR) ? 1 : 4) * (kC / kSets) * 4 + 1024 + (PAIR ? 0 : kPoolFloats * 4) <= kMaxSmem || kC == 256, "shared memory budget");
     static_assert(kGroups * 2 * kC <= (int)kTmemCols, "TMEM: per group C columns of residual stream and C of accumulator");
 };
 
@@ -173,6 +181,11 @@ __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile
                                          long long *waited = nullptr) {
     return bounded_wait(bar, parity, abort_flag, status, kStatusWaitTimeout, kSpinLimit, waited);
 }
+// the same for a barrier that threads of the pair's other CTA arrive on (acquire at cluster scope)
+__device__ __forceinline__ bool wait_bar_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
+                                                 long long *waited = nullptr) {
+    return bounded_wait<true>(bar, parity, abort_flag, status, kStatusWaitTimeout, kSpinLimit, waited);
+}
 
 // slices of the head projection's K that travel in one weight stage (the last stage may carry fewer: eleven
 // slices of the 176-channel shape go as six and five)
@@ -215,6 +228,12 @@ tower_tc_kernel(const TowerArgs args) {
     const uint32_t bar_done = bars + 8u * (2 * kStages + kGroups + kGroups * kSlices);
     auto bar_lead = [&](int s) { return bar_done + 8u * (1 + s); };   // group 0 has issued its MMAs on stage s
     auto bar_pool = [&](int g) { return bar_done + 8u * (1 + kStages + g); };   // the four epilogue warps of group g meet here
+    auto bar_peer = [&](int s) { return bar_done + 8u * (1 + kStages + kGroups + s); };   // pair: the other CTA's half of stage s has landed
+    // CTA pair: rank 0 issues every MMA of the pair; rank 1 supplies its rows, its half of the weights, its epilogue
+    constexpr bool kPair = S::kPair;
+    static_assert(!kPair || (!kFp8 && !kPnet && kGroups == 2), "CTA pairs exist for the two-group bf16 shape of the residual networks");
+    const uint32_t cta_rank = kPair ? ptx::cluster_ctarank() : 0u;
+    const bool leader = cta_rank == 0;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + S::kOffAbort);
     uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + S::kOffTmemPtr);
     constexpr int kVecs = kFp8 ? (kPnet ? 4 : 3) : 1;           // per layer: (scale, bias, h ratio[, cap]) or bias
@@ -232,11 +251,13 @@ tower_tc_kernel(const TowerArgs args) {
             ptx::mbar_init(bar_w_full(s), 1);
             ptx::mbar_init(bar_w_empty(s), kGroups);
             ptx::mbar_init(bar_lead(s), 1);
+            ptx::mbar_init(bar_peer(s), 1);
         }
         for (int g = 0; g < kGroups; ++g) {
             ptx::mbar_init(bar_acc_full(g), 1);
             ptx::mbar_init(bar_pool(g), 4 * S::kSets);
-            for (int kc = 0; kc < kSlices; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4 * S::kSets);
+            // (pair: the first CTA's barriers also count the other CTA's epilogue warps)
+            for (int kc = 0; kc < kSlices; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4 * S::kSets * S::kHalves);
         }
         ptx::mbar_init(bar_done, kGroups);
         *abort_flag = 0;
@@ -244,16 +265,24 @@ tower_tc_kernel(const TowerArgs args) {
     }
     ptx::fence_proxy_async_smem();
     if (warp == 0) {
-        ptx::tmem_alloc(ptx::smem_addr(tmem_ptr_smem), kTmemCols);
-        ptx::tmem_relinquish();
+        if (kPair) { ptx::tmem_alloc_pair(ptx::smem_addr(tmem_ptr_smem), kTmemCols); ptx::tmem_relinquish_pair(); }
+        else { ptx::tmem_alloc(ptx::smem_addr(tmem_ptr_smem), kTmemCols); ptx::tmem_relinquish(); }
     }
     ptx::tc_fence_before();
     __syncthreads();
+    if (kPair) {
+        // nothing may reach into the other CTA (remote arrivals, commits, MMAs reading its shared memory) before its
+        // barriers and frames are initialised
+        ptx::cluster_arrive();
+        ptx::cluster_wait();
+    }
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_smem;
     ptx::launch_dependents();        // the head GEMM kernel may set itself up on idle SMs; it waits for this grid before reading
 
-    const int n_groups = (args.batch + kNB - 1) / kNB;
+    // pair: the schedule deals out PAIRS of groups (four boards) to pairs of CTAs; the CTA of rank r takes the r-th
+    // group of each (a group beyond the batch runs on dead boards and writes nothing)
+    const int n_groups = kPair ? ((args.batch + kNB - 1) / kNB + 1) / 2 : (args.batch + kNB - 1) / kNB;
     const int n_conv = args.n_conv;
     const int head_n = args.head_n;
     const int in_slices = args.in_pad / 16;
@@ -263,7 +292,8 @@ tower_tc_kernel(const TowerArgs args) {
     auto pool_layer = [&](int l) { return kPnet && (l & 3) == 3; };
     auto short_layer = [&](int l) { return kPnet && l >= 4 && (l & 3) == 0; };
     constexpr int kShortSlices = (3 * kC / 4 + 15) / 16;      // slices that hold the 3C/4 channels a pooled block hands on
-    auto round_of = [&](int r) { return get_round<S>(r, (int)blockIdx.x, (int)gridDim.x, n_groups); };
+    auto round_of = [&](int r) { return get_round<S>(r, (int)blockIdx.x / S::kHalves, (int)gridDim.x / S::kHalves, n_groups); };
+    auto my_group = [&](const Round &rd, int g) { return kPair ? 2 * rd.group[g] + (int)cta_rank : rd.group[g]; };   // valid when rd.group[g] >= 0
     auto slices_of = [&](int l) {                                                               // K per MMA: 16 bf16 or 32 e4m3
         return l == 0 ? in_slices : short_layer(l) ? (kFp8 ? kShortSlices / 2 : kShortSlices) : (kFp8 ? kC / 32 : kC / 16);
     };
@@ -296,10 +326,11 @@ tower_tc_kernel(const TowerArgs args) {
             for (int st = 0; st < n_stages + n_head_stages && ok; ++st) {
                 // tower stages are contiguous and equally sized; the head projections follow as small stages of their own
                 const bool head = st >= n_stages;
-                const unsigned char *src = head ? reinterpret_cast<const unsigned char *>(args.head_w) + (size_t)(st - n_stages) * hsps * head_n * 32
-                                                : reinterpret_cast<const unsigned char *>(args.weights) + (size_t)st * kStageBytes;
+                // (pair: every stage is stored as this CTA's half, then the other's)
                 const int head_left = kSlices - (st - n_stages) * hsps;         // slices the head still has to fetch
-                const uint32_t bytes = head ? (uint32_t)((head_left < hsps ? head_left : hsps) * head_n * 32) : (uint32_t)kStageBytes;
+                const uint32_t bytes = head ? (uint32_t)((head_left < hsps ? head_left : hsps) * head_n * 32 / S::kHalves) : (uint32_t)kStageBytes;
+                const unsigned char *src = head ? reinterpret_cast<const unsigned char *>(args.head_w) + (size_t)(st - n_stages) * hsps * head_n * 32 + (size_t)cta_rank * bytes
+                                                : reinterpret_cast<const unsigned char *>(args.weights) + ((size_t)st * S::kHalves + cta_rank) * kStageBytes;
                 ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 if (lane == 0) {
@@ -319,9 +350,43 @@ tower_tc_kernel(const TowerArgs args) {
                         if (ptx::mbar_try_wait(bar_w_full(s), last_parity[s])) break;
         }
     } else if (warp <= kGroups) {
+        if (kPair && !leader) {
+            // ================= pair, second CTA: no MMAs are issued here =================
+            // Warp 1 tells the first CTA's issuers when this CTA's half of a weight stage has landed (its bulk copies
+            // signal a barrier of this CTA; a barrier can only be waited on by its own CTA).  Then it waits for the
+            // pair's last MMAs, which also write this CTA's TMEM.
+            if (warp == 1) {
+                int stage = 0;
+                uint32_t phase = 0;
+                bool ok = true;
+                for (int r = 0; ok; ++r) {
+                    const Round rd = round_of(r);
+                    if (!rd.valid) break;
+                    int n_stages = head_stages<S>(head_n);
+                    for (int l = 0; l < n_conv; ++l) n_stages += stages_of(l);
+                    for (int st = 0; st < n_stages && ok; ++st) {
+                        ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status);
+                        if (!ok) break;
+                        if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_peer(stage), 0));
+                        __syncwarp();
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+                for (uint32_t i = 0; i < (1u << 22); ++i)
+                    if (ptx::mbar_try_wait_cluster(bar_done, 0)) break;
+            }
+        } else {
         // ================= MMA issuer of group g =================
         const int g = warp - 1;
-        constexpr uint32_t idesc = ptx::idesc_bf16_f32(128, kC);
+        constexpr uint32_t idesc = ptx::idesc_bf16_f32(128 * S::kHalves, kC);
+        // a weight stage is ready when this CTA's copy has landed and, in a pair, the other CTA's half as well
+        auto wait_stage = [&](int st_, uint32_t ph_, long long *w_) -> bool {
+            bool k_ = wait_bar(bar_w_full(st_), ph_, abort_flag, args.status, w_);
+            if (kPair && k_) k_ = wait_bar_cluster(bar_peer(st_), ph_, abort_flag, args.status, w_);
+            return k_;
+        };
+        // barrier(s) that arrive when the MMAs issued so far have completed: this CTA's, in a pair both CTAs'
+        auto commit = [&](uint32_t bar_) { if (kPair) ptx::mma_commit_pair(bar_); else ptx::mma_commit(bar_); };
         constexpr uint32_t idesc8 = kInt8 ? ptx::idesc_u8s8_s32(128, kC) : ptx::idesc_e4m3_f32(128, kC);
         int stage = 0;
         uint32_t phase = 0;
@@ -336,6 +401,15 @@ tower_tc_kernel(const TowerArgs args) {
         const bool follow = kGroups == 2 && g == 1;
         const bool lead = kGroups == 2 && g == 0;
         const uint32_t elected = ptx::elect_one();              // the lane that issues; the warp stays converged
+        // group 1 issues on stage number i (counted over the whole launch) once group 0 has issued on stage
+        // min(i + kLag, last stage of i's layer): it trails by kLag stages through the first part of a layer and catches
+        // up to the layer's end while group 0 sits in its layer hand-over, so that each group's hand-over is covered by
+        // the other's MMAs (kLag == 0: strict turns on every stage)
+        int gi = 0, layer_last = 0;
+        auto wait_lead = [&](long long *w_) -> bool {
+            const int j = gi + S::kLag < layer_last ? gi + S::kLag : (gi > layer_last ? gi : layer_last);
+            return wait_bar(bar_lead(j % kStages), (uint32_t)(j / kStages) & 1u, abort_flag, args.status, w_);
+        };
         for (int r = 0; ok; ++r) {
             const Round rd = round_of(r);
             if (!rd.valid) break;
@@ -345,11 +419,19 @@ tower_tc_kernel(const TowerArgs args) {
                 int n_stages = head_stages<S>(head_n);
                 for (int l = 0; l < n_conv; ++l) n_stages += stages_of(l);
                 for (int st = 0; st < n_stages && ok; ++st) {
-                    ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status);
-                    if (ok && follow) ok = wait_bar(bar_lead(stage), phase, abort_flag, args.status);
+                    layer_last = gi;
+                    ok = wait_stage(stage, phase, nullptr);
+                    if (ok && follow) ok = wait_lead(nullptr);
                     if (!ok) break;
-                    if (lane == 0) { ptx::mbar_arrive(bar_w_empty(stage)); if (lead) ptx::mbar_arrive(bar_lead(stage)); }
+                    if (lane == 0) {
+                        if (kPair) {
+                            ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_w_empty(stage), 0));
+                            ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_w_empty(stage), 1));
+                        } else ptx::mbar_arrive(bar_w_empty(stage));
+                        if (lead) ptx::mbar_arrive(bar_lead(stage));
+                    }
                     __syncwarp();
+                    ++gi;
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
                 continue;
@@ -359,6 +441,7 @@ tower_tc_kernel(const TowerArgs args) {
                 const bool e4m3 = kFp8 && l > 0;                       // the input layer stays bf16
                 const bool conv2 = l >= 2 && (l & 1) == 0;             // accumulates onto the residual stream
                 const uint32_t d = d_h + (((l & 1) == 1) ? (uint32_t)kC : 0u);   // conv1 writes the ACC columns
+                layer_last = gi + stages_of(l) - 1;
                 for (int kc = 0; kc < nkc && ok; ++kc) {
                     // one group per CTA: the slice's first weight stage is normally there long before its activations;
                     // looking at it first leaves nothing between the activations' arrival and the first MMA
@@ -366,7 +449,8 @@ tower_tc_kernel(const TowerArgs args) {
                         ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                         if (!ok) break;
                     }
-                    ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
+                    ok = kPair ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
+                               : wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
                     if (!ok) break;
                     a_phase ^= 1u << kc;
                     // low descriptor word in 16-byte units; row m = 0 sits at slot 2*9 + 1 = 19
@@ -377,10 +461,10 @@ tower_tc_kernel(const TowerArgs args) {
 #pragma unroll
                     for (int st = 0; st < S::kStagesPerSlice; ++st) {
                         if (kGroups > 1 || st > 0 || part > 0) {
-                            ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+                            ok = wait_stage(stage, phase, tr ? &t_wait[0] : nullptr);
                             if (!ok) break;
                             if (follow) {
-                                ok = wait_bar(bar_lead(stage), phase, abort_flag, args.status, tr ? &t_wait[2] : nullptr);
+                                ok = wait_lead(tr ? &t_wait[2] : nullptr);
                                 if (!ok) break;
                             }
                         }
@@ -413,19 +497,25 @@ tower_tc_kernel(const TowerArgs args) {
                                 for (int t = 0; t < S::kStageTaps; ++t) {
                                     const int tap = st * S::kStageTaps + t;
                                     const int dy = tap / 3 - 1, dx = tap % 3 - 1;
-                                    ptx::mma_bf16_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                        b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc,
-                                                        (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
+                                    if (kPair)
+                                        ptx::mma_bf16_elect_pair(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                                                 b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc,
+                                                                 (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
+                                    else
+                                        ptx::mma_bf16_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
+                                                            b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc,
+                                                            (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
                                 }
                             }
                             if (elected) {
-                                if (kc == nkc - 1 && st == S::kStagesPerSlice - 1 && part == n_parts - 1) ptx::mma_commit(bar_acc_full(g));
-                                ptx::mma_commit(bar_w_empty(stage));
+                                if (kc == nkc - 1 && st == S::kStagesPerSlice - 1 && part == n_parts - 1) commit(bar_acc_full(g));
+                                commit(bar_w_empty(stage));
                                 if (lead) ptx::mbar_arrive(bar_lead(stage));
                             }
                         }
                         __syncwarp();
                         if (tr) t_issue += clock64() - ti0;
+                        ++gi;
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
                     }
@@ -433,7 +523,8 @@ tower_tc_kernel(const TowerArgs args) {
             }
             if (head_n && ok) {
                 // head projections: a 1x1 convolution = the centre tap only, N = head_n, into the ACC columns
-                const uint32_t idesc_h = ptx::idesc_bf16_f32(128, head_n);
+                const uint32_t idesc_h = ptx::idesc_bf16_f32(128 * S::kHalves, head_n);
+                layer_last = gi + head_stages<S>(head_n) - 1;
                 if (kPnet) {
                     // 256 output columns = the residual stream's columns and the accumulator's: the last
                     // layer's epilogue must have read all of them before the first MMA overwrites any
@@ -445,15 +536,16 @@ tower_tc_kernel(const TowerArgs args) {
                 }
                 for (int kc = 0; kc < kSlices && ok; ++kc) {
                     if (kc % hsps == 0) {
-                        ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+                        ok = wait_stage(stage, phase, tr ? &t_wait[0] : nullptr);
                         if (!ok) break;
                         if (follow) {
-                            ok = wait_bar(bar_lead(stage), phase, abort_flag, args.status, tr ? &t_wait[2] : nullptr);
+                            ok = wait_lead(tr ? &t_wait[2] : nullptr);
                             if (!ok) break;
                         }
                     }
                     if (!kPnet) {
-                        ok = wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
+                        ok = kPair ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
+                                   : wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
                         if (!ok) break;
                         a_phase ^= 1u << kc;
                     }
@@ -461,27 +553,33 @@ tower_tc_kernel(const TowerArgs args) {
                     const bool stage_done = (kc % hsps) == hsps - 1 || kc == kSlices - 1;
                     {
                         const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
-                        const uint32_t b_lo = (((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) + (uint32_t)((kc % hsps) * head_n * 2)) |
-                                              ((uint32_t)head_n << 16);          // K core matrices head_n*16 bytes apart
-                        ptx::mma_bf16_elect(d_h + (kPnet ? 0u : (uint32_t)kC), a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u, elected);
+                        // (pair: this CTA's half of the head tile, head_n / 2 rows)
+                        const uint32_t b_lo = (((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) + (uint32_t)((kc % hsps) * head_n * 2 / S::kHalves)) |
+                                              ((uint32_t)(head_n / S::kHalves) << 16);          // K core matrices rows*16 bytes apart
+                        if (kPair) ptx::mma_bf16_elect_pair(d_h + (uint32_t)kC, a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u, elected);
+                        else ptx::mma_bf16_elect(d_h + (kPnet ? 0u : (uint32_t)kC), a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u, elected);
                     }
                     if (elected) {
-                        if (kc == kSlices - 1) ptx::mma_commit(bar_acc_full(g));
+                        if (kc == kSlices - 1) commit(bar_acc_full(g));
                         if (stage_done) {
-                            ptx::mma_commit(bar_w_empty(stage));
+                            commit(bar_w_empty(stage));
                             if (lead) ptx::mbar_arrive(bar_lead(stage));
                         }
                     }
                     __syncwarp();
-                    if (stage_done && ++stage == kStages) { stage = 0; phase ^= 1u; }
+                    if (stage_done) {
+                        ++gi;
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
                 }
             }
         }
         // all issued MMAs must have completed before TMEM is freed
-        if (elected) ptx::mma_commit(bar_done);
+        if (elected) commit(bar_done);
         __syncwarp();
         for (uint32_t i = 0; i < (1u << 22); ++i)
             if (ptx::mbar_try_wait(bar_done, 0)) break;
+        }
     } else {
         // ================= epilogue: 4 warps per group and set =================
         // A set's last hand-off of a layer comes after its TMEM loads and stores of that layer have
@@ -509,6 +607,11 @@ tower_tc_kernel(const TowerArgs args) {
         uint32_t pool_phase = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
+        // hand-off of a slice to the issuer: a barrier of this CTA, in a pair the first CTA's (which counts both CTAs' warps)
+        auto ready = [&](int kc_) {
+            if (kPair) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_a_ready(g, kc_), 0));
+            else ptx::mbar_arrive(bar_a_ready(g, kc_));
+        };
         if (kPnet) {
             // the pooled-context maps are read in the middle of a layer's hand-over, where a miss to DRAM would
             // sit on the critical path: ask for all of them now (148 CTAs ask for the same lines; L2 merges them)
@@ -522,7 +625,7 @@ tower_tc_kernel(const TowerArgs args) {
             const Round rd = round_of(r);
             if (!rd.valid) break;
             if ((g == 0 ? rd.group[0] : rd.group[1]) < 0) continue;                     // this slot sits the round out
-            const int board = (g == 0 ? rd.group[0] : rd.group[1]) * kNB + b;
+            const int board = my_group(rd, g) * kNB + b;
             const bool live = board < args.batch;
             const int sq = y * 8 + x;
             // ---- the group's input planes -> the first in_pad/8 planes of the frame, either copied from an
@@ -576,7 +679,7 @@ tower_tc_kernel(const TowerArgs args) {
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0)
-                    for (int kc = 0; kc < in_slices; ++kc) ptx::mbar_arrive(bar_a_ready(g, kc));
+                    for (int kc = 0; kc < in_slices; ++kc) ready(kc);
             }
             for (int l = 0; l < n_conv && ok; ++l) {
                 const bool from_acc = (l & 1) == 1;
@@ -857,8 +960,8 @@ tower_tc_kernel(const TowerArgs args) {
                             ptx::tc_fence_before();
                             __syncwarp();
                             if (lane == 0) {
-                                ptx::mbar_arrive(bar_a_ready(g, next_e4m3 ? (kc >> 1) : kc));
-                                if (S::kSets == 2 && !next_e4m3) ptx::mbar_arrive(bar_a_ready(g, kc ^ 1));
+                                ready(next_e4m3 ? (kc >> 1) : kc);
+                                if (S::kSets == 2 && !next_e4m3) ready(kc ^ 1);
                             }
                         }
                         if (kGroups == 1 && keep_h) write_back_h(ks, kc, v);
@@ -926,9 +1029,16 @@ tower_tc_kernel(const TowerArgs args) {
     // ---- teardown
     ptx::tc_fence_before();
     __syncthreads();
+    if (kPair) {
+        // neither CTA may leave (and release shared memory and TMEM that the other's arrivals, commits and MMAs
+        // address) before both are through
+        ptx::cluster_arrive();
+        ptx::cluster_wait();
+    }
     if (warp == 0) {
         ptx::tc_fence_after();
-        ptx::tmem_dealloc(tmem_base, kTmemCols);
+        if (kPair) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+        else ptx::tmem_dealloc(tmem_base, kTmemCols);
     }
 }
 
@@ -936,6 +1046,7 @@ tower_tc_kernel(const TowerArgs args) {
 #define AZ_C128_SETS 1
 #endif
 typedef Shape<128, 2, AZ_C128_SETS> Shape128;
+typedef Shape<128, 2, AZ_C128_SETS, true> Shape128Pair;    // the bf16 residual networks: CTA pairs on 256-row tiles
 #ifndef AZ_FP8_EPI_SETS
 #define AZ_FP8_EPI_SETS 2
 #endif
@@ -963,25 +1074,30 @@ size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv) {
     return slices * 9 * (size_t)channels * 32;             // per slice and tap: N = channels rows x 32 bytes of K
 }
 
+// halves == 2 (CTA pairs): every stage (layer, slice) is stored as two halves of N, rows [0, C/2) of all nine taps for
+// the pair's first CTA, then rows [C/2, C) for the second.
 void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
-                     int channels, int n_conv, __nv_bfloat16 *packed) {
+                     int channels, int n_conv, int halves, __nv_bfloat16 *packed) {
     __nv_bfloat16 *dst = packed;
+    const int groups_per_half = channels / 8 / halves;
     for (int l = 0; l < n_conv; ++l) {
         const int cin = l == 0 ? in_planes : channels;
         const int nkc = (l == 0 ? in_pad : channels) / 16;
         for (int kc = 0; kc < nkc; ++kc)
-            for (int tap = 0; tap < 9; ++tap)
-                for (int k8 = 0; k8 < 2; ++k8)
-                    for (int ng = 0; ng < channels / 8; ++ng)
-                        for (int r = 0; r < 8; ++r)
-                            for (int e = 0; e < 8; ++e) {
-                                const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
-                                float v = 0.0f;
-                                if (ci < cin) v = scale[l][n] * w[l][((size_t)n * cin + ci) * 9 + tap];
-                                *dst++ = __float2bfloat16_rn(v);
-                            }
+            for (int h = 0; h < halves; ++h)
+                for (int tap = 0; tap < 9; ++tap)
+                    for (int k8 = 0; k8 < 2; ++k8)
+                        for (int ng = h * groups_per_half; ng < (h + 1) * groups_per_half; ++ng)
+                            for (int r = 0; r < 8; ++r)
+                                for (int e = 0; e < 8; ++e) {
+                                    const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
+                                    float v = 0.0f;
+                                    if (ci < cin) v = scale[l][n] * w[l][((size_t)n * cin + ci) * 9 + tap];
+                                    *dst++ = __float2bfloat16_rn(v);
+                                }
     }
 }
+bool tc_pair_shape(int channels, int precision, bool pnet) { return channels == 128 && precision == AZ_PREC_BF16 && !pnet; }
 
 // The same tiles for a tower whose layers read different numbers of input channels (the paper's
 // network: 52 planes padded to 64 into the input layer, 3C/4 channels into the second convolution
@@ -1054,7 +1170,7 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
     for (int l = 1; l < n_conv; ++l)
         for (int c = 0; c < C; ++c) sa[(size_t)l * C + c] = fmaxf(absmax[(size_t)(l - 1) * C + c], kTiny) / kMax;
     // layer 0: bf16 tiles exactly as in the bf16 tower
-    tc_pack_weights(w, scale, in_planes, in_pad, C, 1, reinterpret_cast<__nv_bfloat16 *>(packed));
+    tc_pack_weights(w, scale, in_planes, in_pad, C, 1, 1, reinterpret_cast<__nv_bfloat16 *>(packed));
     unsigned char *dst = packed + (size_t)(in_pad / 16) * kStageBytes;
     std::vector<float> wf((size_t)C * C * 9);
     for (int l = 1; l < n_conv; ++l) {
@@ -1107,21 +1223,25 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
 // rows of the value projection.  Same core-matrix order as the tower's weight tiles.
 size_t tc_head_weight_bytes(int head_n, int channels) { return (size_t)head_n * channels * 2; }
 
+// halves == 2 (CTA pairs, 128 channels: all eight slices travel in one stage): the stage as rows [0, head_n/2) of every
+// slice, then rows [head_n/2, head_n).
 void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,
-                  int channels, __nv_bfloat16 *packed) {
+                  int channels, int halves, __nv_bfloat16 *packed) {
     const int head_n = n_policy_pad + kHeadChannels;
+    const int groups_per_half = head_n / 8 / halves;
     __nv_bfloat16 *dst = packed;
-    for (int kc = 0; kc < channels / 16; ++kc)
-        for (int k8 = 0; k8 < 2; ++k8)
-            for (int ng = 0; ng < head_n / 8; ++ng)
-                for (int r = 0; r < 8; ++r)
-                    for (int e = 0; e < 8; ++e) {
-                        const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
-                        float v = 0.0f;
-                        if (n < n_policy) v = (sp ? sp[n] : 1.0f) * wp[(size_t)n * channels + ci];
-                        else if (n >= n_policy_pad) v = sv[n - n_policy_pad] * wv[(size_t)(n - n_policy_pad) * channels + ci];
-                        *dst++ = __float2bfloat16_rn(v);
-                    }
+    for (int h = 0; h < halves; ++h)
+        for (int kc = 0; kc < channels / 16; ++kc)
+            for (int k8 = 0; k8 < 2; ++k8)
+                for (int ng = h * groups_per_half; ng < (h + 1) * groups_per_half; ++ng)
+                    for (int r = 0; r < 8; ++r)
+                        for (int e = 0; e < 8; ++e) {
+                            const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
+                            float v = 0.0f;
+                            if (n < n_policy) v = (sp ? sp[n] : 1.0f) * wp[(size_t)n * channels + ci];
+                            else if (n >= n_policy_pad) v = sv[n - n_policy_pad] * wv[(size_t)(n - n_policy_pad) * channels + ci];
+                            *dst++ = __float2bfloat16_rn(v);
+                        }
 }
 
 int launch_tower_tc(const Net &net, const void *planes, const void *positions, int batch, void *tower_out,
@@ -1136,6 +1256,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         int n = 0;
         AZ_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128Pair>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
@@ -1191,6 +1312,19 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     else if (fp8 && net.int8) tower_tc_kernel<true, Shape128F8, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else if (fp8 && net.split_a) tower_tc_kernel<true, Shape128F8, false, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else if (fp8) tower_tc_kernel<true, Shape128F8><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
+    else if (net.tc_pair) {
+        // clusters of two CTAs; a pair takes pairs of groups
+        const int n_super = (n_groups + 1) / 2, pairs = n_super < sms / 2 ? n_super : sms / 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(Shape128Pair::kThreads);
+        cfg.dynamicSmemBytes = Shape128Pair::smem_bytes(false); cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<false, Shape128Pair>, a));
+        return AZ_OK;
+    }
     else tower_tc_kernel<false, Shape128><<<grid, Shape128::kThreads, Shape128::smem_bytes(false), s>>>(a);
     AZ_LAUNCH_CHECK();
     return AZ_OK;

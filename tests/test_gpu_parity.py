@@ -499,6 +499,43 @@ def test_work_schedule_is_invisible_in_the_results(az, channels, in_planes):
     az.az_free_net(net)
 
 
+@pytest.mark.parametrize("name,batches", [("c3", (1024, 301, 5)), ("c2", (256, 3))])
+def test_tower_on_cta_pairs_gives_the_default_kernels_bits(az, name, batches):
+    # az_load_net_ex(AZ_LOAD_TOWER_CTA_PAIRS): the same arithmetic on 256-row tiles shared by two CTAs (each holds
+    # half of every weight tile).  Same products, same accumulation order: outputs equal the default kernel's bit for
+    # bit, through several rounds of the persistent kernel, a ragged last pair and a lone board; the default kernel
+    # is checked against the oracle above, and the first batch here once more.
+    cfg = configs.CONFIGS[name]
+    blob = weights.make_blob(cfg)
+    arch = az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, max(batches))
+    net_d, net_p = az.az_load_net(arch, blob), az.az_load_net_ex(arch, blob, az.AZ_LOAD_TOWER_CTA_PAIRS)
+    recs = positions.cur_records(positions.for_config(cfg, max(batches)))
+    for n in batches:
+        md, pd, vd = gpu_evaluate(az, net_d, cfg, recs[:n])
+        mp, pp, vp = gpu_evaluate(az, net_p, cfg, recs[:n])
+        assert np.array_equal(pd, pp) and np.array_equal(vd, vp), n
+        if n == batches[0]:
+            rows = np.arange(0, n, 8)
+            mo, _, po, vo = oracle.evaluate(blob, recs[rows], cfg.in_planes, cfg.policy_head)
+            assert np.abs(pp[rows] - po).max() <= TOL[1] and np.abs(vp[rows] - vo).max() <= TOL[1]
+    tower_d = torch.zeros((301, 64, 128), dtype=torch.bfloat16, device="cuda")
+    tower_p = torch.zeros((301, 64, 128), dtype=torch.bfloat16, device="cuda")
+    if max(batches) >= 301:
+        pos = az.records_to_device(recs[:301])
+        az.az_tower(net_d, pos, 301, tower_d)
+        az.az_tower(net_p, pos, 301, tower_p)
+        torch.cuda.synchronize()
+        assert torch.equal(tower_d, tower_p)
+    assert az.az_device_status(net_d) == 0 and az.az_device_status(net_p) == 0
+    az.az_free_net(net_d)
+    az.az_free_net(net_p)
+    # other shapes refuse the option instead of ignoring it
+    with pytest.raises(az.AzError) as e:
+        az.az_load_net_ex(az.make_arch(19, 1, 32, 0, 0, 0, 4), weights.make_blob(configs.tiny_config(blocks=1, channels=32, batch=4)),
+                          az.AZ_LOAD_TOWER_CTA_PAIRS)
+    assert e.value.code == az.AZ_ERR_UNSUPPORTED
+
+
 def test_empty_mask_row_gives_zero_policy_and_a_status_flag(az):
     cfg = configs.tiny_config(blocks=1, channels=32, batch=4)
     net, blob = load(az, cfg, max_batch=8)
