@@ -68,29 +68,36 @@ constexpr uint32_t kSpinLimit = 1u << 24;
 // PAIR: two CTAs on neighbouring SMs (a cluster of two) share every MMA: M = 256 rows, 128 from each CTA's own
 // frame, N = C with each CTA holding HALF of every weight tile in its own shared memory (tcgen05 .cta_group::2).
 // The shared-memory pipe that bounds the 128-channel shape then carries 6 KB of operands per MMA instead of 8.
-template <int C, int GROUPS, int SETS, bool PAIR = false>
+// NSPLIT > 1 (small batches of the 256-channel shape): a cluster of NSPLIT CTAs carries ONE group; each CTA computes
+// C / NSPLIT of every layer's output channels from the whole input (its own copy of the frame) and writes its slices
+// into every CTA's frame through distributed shared memory, so a layer takes 1 / NSPLIT of the tensor time.
+template <int C, int GROUPS, int SETS, bool PAIR = false, int NSPLIT = 1>
 struct Shape {
     static constexpr int kC = C, kGroups = GROUPS, kSets = SETS;
     static constexpr bool kPair = PAIR;
     static constexpr int kHalves = PAIR ? 2 : 1;
+    static constexpr int kNSplit = NSPLIT;
+    static constexpr int kN = C / NSPLIT;                            // output channels this CTA computes (TMEM columns per region)
+    static constexpr int kParts = kHalves * kNSplit;                 // CTAs of a cluster that each hold one part of every weight tile
+    static_assert(!(PAIR && NSPLIT > 1), "one or the other");
     static constexpr int kSlices = kC / 16;                          // 16-channel slices of a layer's output
     static constexpr int kFrameBytes = kPlaneBytes * (kC / 8);       // 46336 / 92672 per group
-    static constexpr int kTileBytes = kC * 32 / kHalves;             // one tap: N = C (pair: C / 2) rows x 32 bytes of K
+    static constexpr int kTileBytes = kC * 32 / kParts;              // one tap: this CTA's rows of the N = C tile x 32 bytes of K
     static constexpr int kStageTaps = kC == 256 ? 3 : 9;
     static constexpr int kStagesPerSlice = 9 / kStageTaps;
     static constexpr int kStageBytes = kStageTaps * kTileBytes;      // 36864 / 24576; pair: 18432
-    static constexpr int kStages = kC == 256 ? 5 : PAIR ? 7 : 3;
+    static constexpr int kStages = NSPLIT > 1 ? 10 : kC == 256 ? 5 : PAIR ? 7 : 3;
     // pair: the second group's issuer runs this many weight stages behind the first's (half a layer), so that each
     // group's layer hand-over falls into the middle of the other's layer; the halved stages make the ring deep enough
     static constexpr int kLag = PAIR ? 4 : 0;
     static constexpr int kEpiWarps = 4 * kGroups * kSets;
     static constexpr int kThreads = 32 * (1 + kGroups + kEpiWarps);  // producer, one issuer per group, 4 epilogue warps per group and set
-    static constexpr uint32_t kBDescLbo = (uint32_t)(kC / kHalves) << 16;   // K core matrices (rows of this CTA's tile)*16 bytes apart
+    static constexpr uint32_t kBDescLbo = (uint32_t)(kC / kParts) << 16;    // K core matrices (rows of this CTA's tile)*16 bytes apart
     static constexpr int kOffFrames = 0;
     static constexpr int kOffWeights = kGroups * kFrameBytes;
     static constexpr int kOffBars = kOffWeights + kStages * kStageBytes;
-    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done, lead[S], pool[G], peer_full[S]
-    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1 + kStages + kGroups + kStages;
+    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done, lead[S], pool[G], peer_full[S], peers_done[G]
+    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1 + kStages + kGroups + kStages + kGroups;
     static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
     static constexpr int kOffAbort = kOffTmemPtr + 4;
     static constexpr int kOffConst = (kOffAbort + 4 + 15) & ~15;     // per-warp copies of the current layer's channel constants
@@ -104,7 +111,7 @@ struct Shape {
     }
     // (four constant vectors per channel in the 8-bit forms, one in bf16; the 176-channel shape exists in bf16 only)
     static_assert(kOffConst + kEpiWarps * ((kC == 176 || PAIR) ? 1 : 4) * (kC / kSets) * 4 + 1024 + (PAIR ? 0 : kPoolFloats * 4) <= kMaxSmem || kC == 256, "shared memory budget");
-    static_assert(kGroups * 2 * kC <= (int)kTmemCols, "TMEM: per group C columns of residual stream and C of accumulator");
+    static_assert(kGroups * 2 * kN <= (int)kTmemCols, "TMEM: per group N columns of residual stream and N of accumulator");
 };
 
 struct TowerArgs {
@@ -190,7 +197,7 @@ __device__ __forceinline__ bool wait_bar_cluster(uint32_t bar, uint32_t parity, 
 // slices of the head projection's K that travel in one weight stage (the last stage may carry fewer: eleven
 // slices of the 176-channel shape go as six and five)
 template <class S> __device__ __host__ constexpr int head_slices_per_stage(int head_n) {
-    return S::kC == 128 ? (head_n == 256 ? 4 : S::kSlices) : S::kC == 160 ? 5 : S::kC == 176 ? 6 : (head_n == 64 ? 8 : 4);
+    return S::kC == 128 ? (head_n == 256 ? 4 : S::kSlices) : S::kC == 160 ? 5 : S::kC == 176 ? 6 : (S::kNSplit > 1 ? (head_n == 64 ? 4 : 2) : head_n == 64 ? 8 : 4);    // (split: stages of 12 KB)
 }
 template <class S> __device__ __host__ constexpr int head_stages(int head_n) {
     return head_n ? (S::kSlices + head_slices_per_stage<S>(head_n) - 1) / head_slices_per_stage<S>(head_n) : 0;
@@ -220,6 +227,10 @@ tower_tc_kernel(const TowerArgs args) {
     // dependent address arithmetic can stay on the uniform datapath
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const uint32_t smem_base = ptx::smem_addr(smem);
+    // start-address field of a shared-memory matrix descriptor: 14 bits, in 16-byte units, an offset within THIS CTA's
+    // shared memory.  (Inside a cluster a CTA's shared addresses carry its rank above bit 23; left in, those bits
+    // would run into the descriptor's stride field.)
+    const uint32_t desc_base = (smem_base >> 4) & 0x3FFFu;
     const uint32_t bars = smem_base + S::kOffBars;
     auto bar_w_full = [&](int s) { return bars + 8u * s; };
     auto bar_w_empty = [&](int s) { return bars + 8u * (kStages + s); };
@@ -230,15 +241,21 @@ tower_tc_kernel(const TowerArgs args) {
     auto bar_pool = [&](int g) { return bar_done + 8u * (1 + kStages + g); };   // the four epilogue warps of group g meet here
     auto bar_peer = [&](int s) { return bar_done + 8u * (1 + kStages + kGroups + s); };   // pair: the other CTA's half of stage s has landed
     // CTA pair: rank 0 issues every MMA of the pair; rank 1 supplies its rows, its half of the weights, its epilogue
+    auto bar_pdone = [&](int g) { return bar_done + 8u * (1 + kStages + kGroups + kStages + g); };   // N-split: the other CTAs' MMAs of this layer are complete
     constexpr bool kPair = S::kPair;
     static_assert(!kPair || (!kFp8 && !kPnet && kGroups == 2), "CTA pairs exist for the two-group bf16 shape of the residual networks");
-    const uint32_t cta_rank = kPair ? ptx::cluster_ctarank() : 0u;
+    constexpr int kNSplit = S::kNSplit, kN = S::kN;
+    constexpr bool kCluster = kPair || kNSplit > 1;
+    static_assert(kNSplit == 1 || (!kFp8 && !kPnet && kGroups == 1 && S::kSets == 1), "the N-split exists for the one-group bf16 shape of the residual networks");
+    const uint32_t cta_rank = kCluster ? ptx::cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
+    constexpr int kOutSlices = kN / 16;                          // 16-channel slices of a layer's output that this CTA produces
+    const int out0 = kNSplit > 1 ? (int)cta_rank * kOutSlices : 0;   // the first of them
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + S::kOffAbort);
     uint32_t *tmem_ptr_smem = reinterpret_cast<uint32_t *>(smem + S::kOffTmemPtr);
     constexpr int kVecs = kFp8 ? (kPnet ? 4 : 3) : 1;           // per layer: (scale, bias, h ratio[, cap]) or bias
     constexpr int kConstFloats = kVecs * kC;
-    constexpr int kMyC = kC / S::kSets;                         // channels an epilogue warp is responsible for
+    constexpr int kMyC = kN / S::kSets;                         // channels an epilogue warp is responsible for
     constexpr int kMyConstFloats = kVecs * kMyC;
     float *head_bias_smem = reinterpret_cast<float *>(smem + S::kOffConst) + S::kEpiWarps * kMyConstFloats;
 
@@ -255,6 +272,7 @@ tower_tc_kernel(const TowerArgs args) {
         }
         for (int g = 0; g < kGroups; ++g) {
             ptx::mbar_init(bar_acc_full(g), 1);
+            ptx::mbar_init(bar_pdone(g), kNSplit > 1 ? kNSplit - 1 : 1);
             ptx::mbar_init(bar_pool(g), 4 * S::kSets);
             // (pair: the first CTA's barriers also count the other CTA's epilogue warps)
             for (int kc = 0; kc < kSlices; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4 * S::kSets * S::kHalves);
@@ -270,9 +288,9 @@ tower_tc_kernel(const TowerArgs args) {
     }
     ptx::tc_fence_before();
     __syncthreads();
-    if (kPair) {
-        // nothing may reach into the other CTA (remote arrivals, commits, MMAs reading its shared memory) before its
-        // barriers and frames are initialised
+    if (kCluster) {
+        // nothing may reach into the other CTA (remote arrivals, commits, stores, MMAs reading its shared memory) before
+        // its barriers and frames are initialised
         ptx::cluster_arrive();
         ptx::cluster_wait();
     }
@@ -292,7 +310,7 @@ tower_tc_kernel(const TowerArgs args) {
     auto pool_layer = [&](int l) { return kPnet && (l & 3) == 3; };
     auto short_layer = [&](int l) { return kPnet && l >= 4 && (l & 3) == 0; };
     constexpr int kShortSlices = (3 * kC / 4 + 15) / 16;      // slices that hold the 3C/4 channels a pooled block hands on
-    auto round_of = [&](int r) { return get_round<S>(r, (int)blockIdx.x / S::kHalves, (int)gridDim.x / S::kHalves, n_groups); };
+    auto round_of = [&](int r) { return get_round<S>(r, (int)blockIdx.x / S::kParts, (int)gridDim.x / S::kParts, n_groups); };
     auto my_group = [&](const Round &rd, int g) { return kPair ? 2 * rd.group[g] + (int)cta_rank : rd.group[g]; };   // valid when rd.group[g] >= 0
     auto slices_of = [&](int l) {                                                               // K per MMA: 16 bf16 or 32 e4m3
         return l == 0 ? in_slices : short_layer(l) ? (kFp8 ? kShortSlices / 2 : kShortSlices) : (kFp8 ? kC / 32 : kC / 16);
@@ -329,8 +347,8 @@ tower_tc_kernel(const TowerArgs args) {
                 // (pair: every stage is stored as this CTA's half, then the other's)
                 const int head_left = kSlices - (st - n_stages) * hsps;         // slices the head still has to fetch
                 const uint32_t bytes = head ? (uint32_t)((head_left < hsps ? head_left : hsps) * head_n * 32 / S::kHalves) : (uint32_t)kStageBytes;
-                const unsigned char *src = head ? reinterpret_cast<const unsigned char *>(args.head_w) + (size_t)(st - n_stages) * hsps * head_n * 32 + (size_t)cta_rank * bytes
-                                                : reinterpret_cast<const unsigned char *>(args.weights) + ((size_t)st * S::kHalves + cta_rank) * kStageBytes;
+                const unsigned char *src = head ? reinterpret_cast<const unsigned char *>(args.head_w) + (size_t)(st - n_stages) * hsps * head_n * 32 + (S::kHalves > 1 ? (size_t)cta_rank * bytes : (size_t)0)
+                                                : reinterpret_cast<const unsigned char *>(args.weights) + ((size_t)st * S::kParts + cta_rank) * kStageBytes;
                 ok = wait_bar(bar_w_empty(stage), phase ^ 1u, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 if (lane == 0) {
@@ -378,7 +396,7 @@ tower_tc_kernel(const TowerArgs args) {
         } else {
         // ================= MMA issuer of group g =================
         const int g = warp - 1;
-        constexpr uint32_t idesc = ptx::idesc_bf16_f32(128 * S::kHalves, kC);
+        constexpr uint32_t idesc = ptx::idesc_bf16_f32(128 * S::kHalves, kN);
         // a weight stage is ready when this CTA's copy has landed and, in a pair, the other CTA's half as well
         auto wait_stage = [&](int st_, uint32_t ph_, long long *w_) -> bool {
             bool k_ = wait_bar(bar_w_full(st_), ph_, abort_flag, args.status, w_);
@@ -392,8 +410,8 @@ tower_tc_kernel(const TowerArgs args) {
         uint32_t phase = 0;
         uint32_t a_phase = 0;
         bool ok = true;
-        const uint32_t d_h = tmem_base + (uint32_t)(g * 2 * kC);
-        const uint32_t frame_lo = (((smem_base + S::kOffFrames + g * kFrameBytes) >> 4) + (uint32_t)(kNB * 9 + 1)) | kADescLbo;
+        const uint32_t d_h = tmem_base + (uint32_t)(g * 2 * kN);
+        const uint32_t frame_lo = (desc_base + (uint32_t)((S::kOffFrames + g * kFrameBytes) >> 4) + (uint32_t)(kNB * 9 + 1)) | kADescLbo;
         // The two issuers take strict turns on every weight stage: group 1 issues its MMAs on a stage
         // only after group 0 has issued its own (bar_lead).  While one issuer sits in its barrier round
         // trips the other's MMAs keep the tensor pipe busy, and the groups reach their layer boundaries
@@ -440,7 +458,7 @@ tower_tc_kernel(const TowerArgs args) {
                 const int nkc = slices_of(l);
                 const bool e4m3 = kFp8 && l > 0;                       // the input layer stays bf16
                 const bool conv2 = l >= 2 && (l & 1) == 0;             // accumulates onto the residual stream
-                const uint32_t d = d_h + (((l & 1) == 1) ? (uint32_t)kC : 0u);   // conv1 writes the ACC columns
+                const uint32_t d = d_h + (((l & 1) == 1) ? (uint32_t)kN : 0u);   // conv1 writes the ACC columns
                 layer_last = gi + stages_of(l) - 1;
                 for (int kc = 0; kc < nkc && ok; ++kc) {
                     // one group per CTA: the slice's first weight stage is normally there long before its activations;
@@ -449,8 +467,8 @@ tower_tc_kernel(const TowerArgs args) {
                         ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                         if (!ok) break;
                     }
-                    ok = kPair ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
-                               : wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
+                    ok = kCluster ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
+                                  : wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
                     if (!ok) break;
                     a_phase ^= 1u << kc;
                     // low descriptor word in 16-byte units; row m = 0 sits at slot 2*9 + 1 = 19
@@ -471,7 +489,7 @@ tower_tc_kernel(const TowerArgs args) {
                         ptx::tc_fence_after();
                         const long long ti0 = tr ? clock64() : 0;
                         {
-                            const uint32_t b_lo = ((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) | S::kBDescLbo;
+                            const uint32_t b_lo = (desc_base + (uint32_t)((S::kOffWeights + stage * kStageBytes) >> 4)) | S::kBDescLbo;
                             // the operand type is chosen once per stage: a branch between consecutive MMAs
                             // costs more than the MMA itself takes on the tensor pipe
                             if (e4m3) {
@@ -544,8 +562,8 @@ tower_tc_kernel(const TowerArgs args) {
                         }
                     }
                     if (!kPnet) {
-                        ok = kPair ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
-                                   : wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
+                        ok = kCluster ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
+                                      : wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
                         if (!ok) break;
                         a_phase ^= 1u << kc;
                     }
@@ -554,10 +572,10 @@ tower_tc_kernel(const TowerArgs args) {
                     {
                         const uint32_t a_lo = frame_lo + (uint32_t)(2 * kc * kSlots);
                         // (pair: this CTA's half of the head tile, head_n / 2 rows)
-                        const uint32_t b_lo = (((smem_base + S::kOffWeights + stage * kStageBytes) >> 4) + (uint32_t)((kc % hsps) * head_n * 2 / S::kHalves)) |
+                        const uint32_t b_lo = (desc_base + (uint32_t)((S::kOffWeights + stage * kStageBytes) >> 4) + (uint32_t)((kc % hsps) * head_n * 2 / S::kHalves)) |
                                               ((uint32_t)(head_n / S::kHalves) << 16);          // K core matrices rows*16 bytes apart
                         if (kPair) ptx::mma_bf16_elect_pair(d_h + (uint32_t)kC, a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u, elected);
-                        else ptx::mma_bf16_elect(d_h + (kPnet ? 0u : (uint32_t)kC), a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u, elected);
+                        else ptx::mma_bf16_elect(d_h + (kPnet ? 0u : (uint32_t)kN), a_lo, kADescHi, b_lo, kBDescHi, idesc_h, kc > 0 ? 1u : 0u, elected);
                     }
                     if (elected) {
                         if (kc == kSlices - 1) commit(bar_acc_full(g));
@@ -590,13 +608,13 @@ tower_tc_kernel(const TowerArgs args) {
         // this warp's share of every layer: the slices kc = ks * sets + set.  Interleaved, so that with two
         // sets the two slices of the next layer's first 32-channel e4m3 step are produced side by side.
         const int set = (ew >> 2) % S::kSets;
-        constexpr int kMySlices = kSlices / S::kSets;
+        constexpr int kMySlices = kOutSlices / S::kSets;
         const int q = warp & 3;                               // TMEM lane quarter this warp may access
         const int m = q * 32 + lane;                          // GEMM row = TMEM lane
         const int g8 = m >> 3, y = g8 >> 1, b = g8 & 1, x = m & 7;
         const int slot = (g8 + kNB) * 9 + x + 1;
         unsigned char *frame = smem + S::kOffFrames + g * kFrameBytes;
-        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 2 * kC);
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(g * 2 * kN);
         float *lc = reinterpret_cast<float *>(smem + S::kOffConst) + ew * kMyConstFloats;   // this warp's copy of the layer constants
         // pooled-context scratch of this group (paper's network only)
         constexpr int kPoolC = kC / 4, kRegC = kC - kC / 4;
@@ -607,11 +625,22 @@ tower_tc_kernel(const TowerArgs args) {
         uint32_t pool_phase = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
-        // hand-off of a slice to the issuer: a barrier of this CTA, in a pair the first CTA's (which counts both CTAs' warps)
+        // hand-off of a slice to the issuer: a barrier of this CTA; in a pair the first CTA's (which counts both CTAs'
+        // warps); with the N-split the barrier of EVERY CTA of the cluster (the slice has been written into every frame)
         auto ready = [&](int kc_) {
             if (kPair) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_a_ready(g, kc_), 0));
-            else ptx::mbar_arrive(bar_a_ready(g, kc_));
+            else if (kNSplit > 1) {
+                // own frame: written with ordinary stores, handed off as always; the other CTAs' frames: written with
+                // asynchronous stores that count as transaction bytes on THEIR barrier (1 KB per warp and slice: 32
+                // rows x 32 bytes), announced with this warp's arrival; nothing here waits for the remote traffic
+                ptx::mbar_arrive(bar_a_ready(g, kc_));
+#pragma unroll
+                for (int p = 0; p < kNSplit; ++p)
+                    if (p != (int)cta_rank) ptx::mbar_arrive_expect_tx_cluster(ptx::map_to_cta(bar_a_ready(g, kc_), (uint32_t)p), 1024u);
+            } else ptx::mbar_arrive(bar_a_ready(g, kc_));
         };
+        uint32_t pdone_phase = 0;
+        const uint32_t frame_addr = ptx::smem_addr(frame);
         if (kPnet) {
             // the pooled-context maps are read in the middle of a layer's hand-over, where a miss to DRAM would
             // sit on the critical path: ask for all of them now (148 CTAs ask for the same lines; L2 merges them)
@@ -679,7 +708,10 @@ tower_tc_kernel(const TowerArgs args) {
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0)
-                    for (int kc = 0; kc < in_slices; ++kc) ready(kc);
+                    for (int kc = 0; kc < in_slices; ++kc) {
+                        if (kNSplit > 1) ptx::mbar_arrive(bar_a_ready(g, kc));      // every CTA encodes its own copy of the input
+                        else ready(kc);
+                    }
             }
             for (int l = 0; l < n_conv && ok; ++l) {
                 const bool from_acc = (l & 1) == 1;
@@ -696,7 +728,7 @@ tower_tc_kernel(const TowerArgs args) {
                     for (int idx = lane; idx < kMyConstFloats / 4; idx += 32) {
                         // own copy: [vector][own slice ks][16 channels]
                         const int vec = idx / (kMyC / 4), within = idx % (kMyC / 4);
-                        const int kc = (within >> 2) * S::kSets + set;
+                        const int kc = out0 + (within >> 2) * S::kSets + set;
                         reinterpret_cast<float4 *>(lc)[idx] = __ldg(reinterpret_cast<const float4 *>(src) + vec * (kC / 4) + kc * 4 + (within & 3));
                     }
                     __syncwarp();
@@ -705,9 +737,20 @@ tower_tc_kernel(const TowerArgs args) {
                 if (!ok) break;
                 acc_phase ^= 1u;
                 ptx::tc_fence_after();
+                if (kNSplit > 1) {
+                    // this CTA's MMAs of the layer are complete, so the other CTAs may overwrite its frame: tell them
+                    // (their own completion is awaited below, just before the first store into their frames)
+                    if (q == 0 && lane == 0) {
+#pragma unroll
+                        for (int p = 0; p < kNSplit; ++p)
+                            if (p != (int)cta_rank) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_pdone(g), (uint32_t)p));
+                    }
+                    __syncwarp();
+                }
+                bool peers_done = kNSplit == 1;
                 const float *bias = kFp8 ? lc + kMyC : lc;
                 __nv_bfloat16 *dst = args.out + ((size_t)board * 64 + sq) * kC;
-                const uint32_t t_src = t_lane + (uint32_t)(from_acc ? kC : 0);
+                const uint32_t t_src = t_lane + (uint32_t)(from_acc ? kN : 0);
                 const bool keep_h = !from_acc && l != n_conv - 1;   // the residual stream stays in TMEM as fp32
                 uint32_t r[2][16];
                 const bool pooled = pool_layer(l);
@@ -811,7 +854,7 @@ tower_tc_kernel(const TowerArgs args) {
                     ok = meet();
                     if (!ok) break;
                 }
-                auto write_back_h = [&](int ks, int kc, const float (&v)[16]) {
+                auto write_back_h = [&](int ks, int kl_, const float (&v)[16]) {
                     // fp32 copy back to H (FP8: pre-divided by the next conv2's weight scale, so that
                     // conv2 can accumulate its raw products straight onto it).  With one group per CTA this
                     // comes AFTER the slice's hand-off (the next layer's MMAs wait for the frame, not for H, and
@@ -836,17 +879,18 @@ tower_tc_kernel(const TowerArgs args) {
                             w[i + 3] = __float_as_uint(kFp8 ? v[i + 3] * hs.w : v[i + 3]);
                         }
                     }
-                    ptx::tmem_st16(t_lane + (uint32_t)(kc * 16), w);
+                    ptx::tmem_st16(t_lane + (uint32_t)(kl_ * 16), w);
                 };
                 const float *ctx = pool_ctx + b * kCtxStride;                  // this row's board
-                const int n_kc = (kPnet && pooled) ? kShortSlices : kSlices;   // the pooled channels are not handed on
+                const int n_kc = (kPnet && pooled) ? kShortSlices : kOutSlices;   // the pooled channels are not handed on
                 ptx::tmem_ld16(t_src + (uint32_t)(set * 16), r[0]);
 #pragma unroll
                 for (int ks = 0; ks < kMySlices; ++ks) {
-                    const int kc = ks * S::kSets + set;             // the slice; ks indexes this warp's constants
-                    if (kPnet && kc >= n_kc) break;
+                    const int kl = ks * S::kSets + set;             // the slice among this CTA's output slices (its TMEM columns); ks indexes this warp's constants
+                    const int kc = out0 + kl;                       // the slice among the layer's output channels (frame planes, global memory)
+                    if (kPnet && kl >= n_kc) break;
                     ptx::tmem_ld_wait();
-                    if (kc + S::kSets < n_kc) ptx::tmem_ld16(t_src + (uint32_t)((kc + S::kSets) * 16), r[(ks + 1) & 1]);
+                    if (kl + S::kSets < n_kc) ptx::tmem_ld16(t_src + (uint32_t)((kl + S::kSets) * 16), r[(ks + 1) & 1]);
                     uint32_t(&rr)[16] = r[ks & 1];
                     float v[16];
 #pragma unroll
@@ -949,8 +993,26 @@ tower_tc_kernel(const TowerArgs args) {
                             for (int i = 0; i < 8; ++i) pk[i] = ptx::pack_bf16x2_relu(v[2 * i], v[2 * i + 1]);
                             *reinterpret_cast<uint4 *>(frame + (2 * kc) * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                             *reinterpret_cast<uint4 *>(frame + (2 * kc + 1) * kPlaneBytes + slot * 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                            if (kNSplit > 1) {
+                                // the same slice into the other CTAs' frames, once their MMAs of this layer (which read
+                                // those frames) are complete
+                                if (!peers_done) {
+                                    ok = wait_bar_cluster(bar_pdone(g), pdone_phase, abort_flag, args.status);
+                                    pdone_phase ^= 1u;
+                                    peers_done = true;
+                                    if (!ok) break;
+                                }
+#pragma unroll
+                                for (int p = 0; p < kNSplit; ++p)
+                                    if (p != (int)cta_rank) {
+                                        const uint32_t dst0 = ptx::map_to_cta(frame_addr + (uint32_t)((2 * kc) * kPlaneBytes + slot * 16), (uint32_t)p);
+                                        const uint32_t rbar = ptx::map_to_cta(bar_a_ready(g, kc), (uint32_t)p);
+                                        ptx::st_async_cluster_v4(dst0, pk[0], pk[1], pk[2], pk[3], rbar);
+                                        ptx::st_async_cluster_v4(dst0 + (uint32_t)kPlaneBytes, pk[4], pk[5], pk[6], pk[7], rbar);
+                                    }
+                            }
                         }
-                        if (kGroups > 1 && keep_h) write_back_h(ks, kc, v);
+                        if (kGroups > 1 && keep_h) write_back_h(ks, kl, v);
                         // e4m3 layers consume 32 channels per MMA: one hand-off per two slices.  With two sets
                         // every barrier counts both sets' warps: a pair of slices is handed off by the four
                         // warps of each set, and where the next layer reads 16-channel slices (the bf16 head)
@@ -964,10 +1026,14 @@ tower_tc_kernel(const TowerArgs args) {
                                 if (S::kSets == 2 && !next_e4m3) ready(kc ^ 1);
                             }
                         }
-                        if (kGroups == 1 && keep_h) write_back_h(ks, kc, v);
+                        if (kGroups == 1 && keep_h) write_back_h(ks, kl, v);
                     }
                 }
                 if (keep_h) ptx::tmem_st_wait();
+                if (kNSplit > 1 && !peers_done && ok) {            // a layer that wrote no frame still takes the other CTAs' signal
+                    ok = wait_bar_cluster(bar_pdone(g), pdone_phase, abort_flag, args.status);
+                    pdone_phase ^= 1u;
+                }
             }
             if (head_n && ok) {
                 // ---- head projections out of the ACC columns
@@ -986,13 +1052,14 @@ tower_tc_kernel(const TowerArgs args) {
 #pragma unroll 1
                 for (int j = kPnet ? set : 0; j < n_slices; j += kPnet ? S::kSets : 1) {
                     uint32_t rr[16];
-                    ptx::tmem_ld16(t_lane + (kPnet ? 0u : (uint32_t)kC) + (uint32_t)(j * 16), rr);
+                    ptx::tmem_ld16(t_lane + (kPnet ? 0u : (uint32_t)kN) + (uint32_t)(j * 16), rr);
                     ptx::tmem_ld_wait();
                     float v[16];
 #pragma unroll
                     for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(rr[i]) + hb[j * 16 + i];
-                    if (!live) {
-                        // rows past the end of the batch produce nothing
+                    if (!live || (kNSplit > 1 && cta_rank != 0)) {
+                        // rows past the end of the batch produce nothing; with the N-split every CTA computes the (small)
+                        // head projections from its own copy of the frame and the first one writes them
                     } else if (kPnet) {
                         // queries (columns 0..127) and keys (128..255) of this square, fp32 as accumulated, row-major
                         float4 *qk = reinterpret_cast<float4 *>(args.qk_out + ((size_t)board * 64 + sq) * 256 + j * 16);
@@ -1029,8 +1096,8 @@ tower_tc_kernel(const TowerArgs args) {
     // ---- teardown
     ptx::tc_fence_before();
     __syncthreads();
-    if (kPair) {
-        // neither CTA may leave (and release shared memory and TMEM that the other's arrivals, commits and MMAs
+    if (kCluster) {
+        // neither CTA may leave (and release shared memory and TMEM that the other's arrivals, commits, stores and MMAs
         // address) before both are through
         ptx::cluster_arrive();
         ptx::cluster_wait();
@@ -1052,6 +1119,7 @@ typedef Shape<128, 2, AZ_C128_SETS, true> Shape128Pair;    // the bf16 residual 
 #endif
 typedef Shape<128, 2, AZ_FP8_EPI_SETS> Shape128F8;
 typedef Shape<256, 1, 1> Shape256;
+typedef Shape<256, 1, 1, false, 2> Shape256Split2;      // small batches: two CTAs per group, 128 output channels each
 // the paper's 160-channel network: one group, whose epilogue (not its MMAs) sets the pace with four warps;
 // two sets of four share each layer
 #ifndef AZ_P160_SETS
@@ -1074,27 +1142,30 @@ size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv) {
     return slices * 9 * (size_t)channels * 32;             // per slice and tap: N = channels rows x 32 bytes of K
 }
 
-// halves == 2 (CTA pairs): every stage (layer, slice) is stored as two halves of N, rows [0, C/2) of all nine taps for
-// the pair's first CTA, then rows [C/2, C) for the second.
+// halves == 2 (CTA pairs, or two CTAs splitting the output channels): every weight stage (layer, slice, stage_taps
+// taps: nine, or three in the 256-channel shape) is stored as two halves of N, rows [0, C/2) of the stage's taps for
+// the cluster's first CTA, then rows [C/2, C) for the second.
 void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
-                     int channels, int n_conv, int halves, __nv_bfloat16 *packed) {
+                     int channels, int n_conv, int halves, int stage_taps, __nv_bfloat16 *packed) {
     __nv_bfloat16 *dst = packed;
     const int groups_per_half = channels / 8 / halves;
     for (int l = 0; l < n_conv; ++l) {
         const int cin = l == 0 ? in_planes : channels;
         const int nkc = (l == 0 ? in_pad : channels) / 16;
         for (int kc = 0; kc < nkc; ++kc)
-            for (int h = 0; h < halves; ++h)
-                for (int tap = 0; tap < 9; ++tap)
-                    for (int k8 = 0; k8 < 2; ++k8)
-                        for (int ng = h * groups_per_half; ng < (h + 1) * groups_per_half; ++ng)
-                            for (int r = 0; r < 8; ++r)
-                                for (int e = 0; e < 8; ++e) {
-                                    const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
-                                    float v = 0.0f;
-                                    if (ci < cin) v = scale[l][n] * w[l][((size_t)n * cin + ci) * 9 + tap];
-                                    *dst++ = __float2bfloat16_rn(v);
-                                }
+            for (int st = 0; st < 9 / stage_taps; ++st)
+                for (int h = 0; h < halves; ++h)
+                    for (int t = 0; t < stage_taps; ++t)
+                        for (int k8 = 0; k8 < 2; ++k8)
+                            for (int ng = h * groups_per_half; ng < (h + 1) * groups_per_half; ++ng)
+                                for (int r = 0; r < 8; ++r)
+                                    for (int e = 0; e < 8; ++e) {
+                                        const int tap = st * stage_taps + t;
+                                        const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
+                                        float v = 0.0f;
+                                        if (ci < cin) v = scale[l][n] * w[l][((size_t)n * cin + ci) * 9 + tap];
+                                        *dst++ = __float2bfloat16_rn(v);
+                                    }
     }
 }
 bool tc_pair_shape(int channels, int precision, bool pnet) { return channels == 128 && precision == AZ_PREC_BF16 && !pnet; }
@@ -1170,7 +1241,7 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
     for (int l = 1; l < n_conv; ++l)
         for (int c = 0; c < C; ++c) sa[(size_t)l * C + c] = fmaxf(absmax[(size_t)(l - 1) * C + c], kTiny) / kMax;
     // layer 0: bf16 tiles exactly as in the bf16 tower
-    tc_pack_weights(w, scale, in_planes, in_pad, C, 1, 1, reinterpret_cast<__nv_bfloat16 *>(packed));
+    tc_pack_weights(w, scale, in_planes, in_pad, C, 1, 1, 9, reinterpret_cast<__nv_bfloat16 *>(packed));
     unsigned char *dst = packed + (size_t)(in_pad / 16) * kStageBytes;
     std::vector<float> wf((size_t)C * C * 9);
     for (int l = 1; l < n_conv; ++l) {
@@ -1261,6 +1332,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256Split2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128P, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape160, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128P, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
@@ -1308,6 +1380,20 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     else if (net.pnet && net.arch.channels == 160) tower_tc_kernel<false, Shape160, true><<<grid, Shape160::kThreads, Shape160::smem_bytes(false, true), s>>>(a);
     else if (net.pnet && fp8) tower_tc_kernel<true, Shape128P, true, true><<<grid, Shape128P::kThreads, Shape128P::smem_bytes(true, true), s>>>(a);
     else if (net.pnet) tower_tc_kernel<false, Shape128P, true><<<grid, Shape128P::kThreads, Shape128P::smem_bytes(false, true), s>>>(a);
+    else if (wide && n_groups * 2 <= sms) {
+        // few boards: two CTAs (a cluster) per group, each computing half of every layer's output channels from a
+        // second copy of the weights packed for that split
+        a.weights = net.tc_weights_split;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * n_groups); cfg.blockDim = dim3(Shape256Split2::kThreads);
+        cfg.dynamicSmemBytes = Shape256Split2::smem_bytes(false); cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<false, Shape256Split2>, a));
+        return AZ_OK;
+    }
     else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
     else if (fp8 && net.int8) tower_tc_kernel<true, Shape128F8, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else if (fp8 && net.split_a) tower_tc_kernel<true, Shape128F8, false, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
