@@ -214,6 +214,13 @@ int build_net(Net &n, const BlobView &v) {
             if ((rc = upload_f32(v.b2[i], C, &n.conv_bias[l2])) != AZ_OK) return rc;
         }
         if ((rc = alloc_simt_buffers(n)) != AZ_OK) return rc;
+        if (tower_f32_shape(a)) {
+            std::vector<F32Layer> table(n.n_conv);
+            for (int l = 0; l < n.n_conv; ++l)
+                table[l] = F32Layer{static_cast<const float *>(n.conv_w[l]), n.conv_scale[l], n.conv_bias[l]};
+            AZ_CUDA(cudaMalloc((void **)&n.f32_layers, table.size() * sizeof(F32Layer)));
+            AZ_CUDA(cudaMemcpy(n.f32_layers, table.data(), table.size() * sizeof(F32Layer), cudaMemcpyHostToDevice));
+        }
     }
 
     // heads
@@ -253,6 +260,7 @@ int build_net(Net &n, const BlobView &v) {
 void free_net(Net *n) {
     if (!n) return;
     for (int i = 0; i < 1 + 2 * 64; ++i) { cudaFree(n->conv_w[i]); cudaFree(n->conv_scale[i]); cudaFree(n->conv_bias[i]); }
+    cudaFree(n->f32_layers);
     cudaFree(n->tc_weights); cudaFree(n->tc_weights_split); cudaFree(n->tc_bias); cudaFree(n->tc_head_w); cudaFree(n->tc_head_bias);
     cudaFree(n->tc8_weights); cudaFree(n->tc8_lconst);
     delete static_cast<HostMaster *>(n->host_master);
@@ -302,6 +310,14 @@ int run_tower(Net &n, const void *positions, int batch, void **tower_out, bool f
         if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
         *tower_out = fused_heads ? nullptr : n.act[0];
         rc = launch_tower_tc(n, nullptr, positions, batch, *tower_out, fused_heads, nullptr, s);
+        if (rc == AZ_OK && timed) AZ_CUDA(cudaEventRecord(n.ev_end[n.n_events++], s));
+        return rc;
+    }
+    if (n.f32_layers) {
+        // 64-channel fp32 networks: encoder and every convolution in one launch, activations resident in shared memory
+        if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
+        *tower_out = n.act[0];
+        rc = launch_tower_f32(n, positions, batch, static_cast<float *>(n.act[0]), s);
         if (rc == AZ_OK && timed) AZ_CUDA(cudaEventRecord(n.ev_end[n.n_events++], s));
         return rc;
     }
@@ -475,6 +491,8 @@ static int evaluate_impl(az_net *net, const void *positions_dev, const uint64_t 
         return az::launch_masked_softmax(n->logits, legal_masks_dev, batch, (int)az_policy_size(&a), (int)az_mask_words(&a),
                                          policy_dev, n->status_dev, true, s);
     }
+    if (n->f32_layers && a.policy_head == AZ_POLICY_PLANES73)      // 64-channel fp32 networks: both heads and the softmax in one launch
+        return az::launch_heads_f32(*n, h, legal_masks_dev, batch, policy_dev, legal_dev, counts_dev, value_dev, s);
     if (a.policy_head == AZ_POLICY_PLANES73) {
         rc = az::launch_conv1x1(h, n->p_w, nullptr, n->p_bias, batch, C, az::kPlanes73, false, n->bf16, n->logits, true, s);
         if (rc != AZ_OK) return rc;
@@ -814,6 +832,8 @@ int az_launches_per_evaluate(const az_net *net, int batch) {
     if (n->pnet) return az::tower_tc_launch_count() /*encoder + tower + query/key maps*/ + 1 /*scores, softmax, value head*/;
     if (n->tc_ready) return az::tower_tc_launch_count() /*encoder + tower + head projections*/ + 1 /*head GEMMs*/ + 1 /*softmax*/;
     const int policy = n->arch.policy_head == AZ_POLICY_PLANES73 ? 1 : 2;
+    if (n->f32_layers && n->arch.policy_head == AZ_POLICY_PLANES73) return 1 /*encoder + tower*/ + 1 /*heads + softmax*/;
+    if (n->f32_layers) return 1 /*encoder + tower*/ + policy + 3 /*value*/ + 1 /*softmax*/;
     return 1 /*encode*/ + n->n_conv + policy + 3 /*value*/ + 1 /*softmax*/;
 }
 

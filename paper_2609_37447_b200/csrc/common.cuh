@@ -30,6 +30,11 @@ struct ConvLayerF32 {                 // fp32 path: weights [tap][cin][cout], fo
     int cin = 0, cout = 0;
 };
 
+struct F32Layer {                    // one convolution of the fused fp32 tower: device pointers
+    const float *w;                   // [tap][cin][cout]
+    const float *scale, *bias;        // folded batch-norm
+};
+
 struct Net {
     az_arch arch{};
     int device = 0;
@@ -41,6 +46,8 @@ struct Net {
     void *conv_w[1 + 2 * 64] = {};    // element type = activation type
     float *conv_scale[1 + 2 * 64] = {};
     float *conv_bias[1 + 2 * 64] = {};
+
+    F32Layer *f32_layers = nullptr;   // device table [n_conv] for the fused fp32 tower (64 channels, 19 planes); null otherwise
 
     // ---- tensor-core tower (bf16, channels == 128) ----
     void *tc_weights = nullptr;       // packed UMMA B-operand tiles, all layers
@@ -188,6 +195,13 @@ int launch_masked_softmax_compact(const float *logits, const uint64_t *masks, in
                                   float *out, int *counts, uint32_t *status, bool pdl, cudaStream_t s);
 int launch_masked_softmax(const float *logits, const uint64_t *masks, int batch, int n, int words,
                           float *policy, uint32_t *status, bool pdl, cudaStream_t s);
+
+// fused fp32 tower (tower_f32.cu): encoder + all convolutions of a 64-channel, 19-plane fp32 network in one launch
+bool tower_f32_shape(const az_arch &a);
+int launch_tower_f32(const Net &net, const void *positions, int batch, float *out, cudaStream_t s);
+// policy (dense, or legal moves only with counts) and value of those networks with the 73-plane head, one launch
+int launch_heads_f32(const Net &n, const void *tower, const uint64_t *masks, int batch, float *policy, float *legal,
+                     int *counts, float *value, cudaStream_t s);
 
 // tensor-core tower (tower_tc.cu)
 size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv);

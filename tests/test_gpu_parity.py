@@ -201,6 +201,45 @@ def test_small_and_ragged_batches(az, batch, precision):
     az.az_free_net(net)
 
 
+@pytest.mark.parametrize("blocks,value_head,batch", [(0, 0, 3), (1, 1, 1), (2, 0, 7), (3, 1, 65), (6, 0, 150)])
+def test_fp32_64_channel_networks_on_the_fused_kernels(az, blocks, value_head, batch):
+    # 64-channel fp32 networks with the 73-plane head run as two launches: encoder + whole tower (a cluster of two
+    # CTAs per board, activations resident in shared memory, the rank between the two halves exchanged through
+    # distributed shared memory after every layer), then both heads with the masked softmax.  Against the oracle at
+    # the fp32 bar, for depths from no block at all to config 1's six, both value heads, odd batch sizes and more
+    # boards than half the SMs; the tower's activations themselves at 1e-5 of their largest; the legal-moves-only
+    # output against the dense one.
+    cfg = configs.tiny_config(blocks=blocks, channels=64, policy_head=0, value_head=value_head, precision=0, batch=batch,
+                              weight_seed=600 + blocks)
+    blob = weights.make_blob(cfg, 0.2 / (1 + blocks), 0.3 / (1 + blocks))
+    net, _ = load(az, cfg, blob=blob)
+    recs = positions.cur_records(positions.generate(4600 + blocks, batch, (0, 120))[0])
+    mo, _, po, vo, raw = oracle.evaluate(blob, recs, 19, 0, want_tower=True)
+    mg, pg, vg = gpu_evaluate(az, net, cfg, recs)
+    compare(cfg, mg, pg, vg, mo, po, vo, TOL[0])
+    assert (pg.argmax(axis=1) == po.argmax(axis=1)).all()
+    tower = torch.zeros((batch, 64, 64), dtype=torch.float32, device="cuda")
+    pos = az.records_to_device(recs)
+    az.az_tower(net, pos, batch, tower)
+    masks = torch.from_numpy(mo.view(np.int64)).cuda()
+    legal = torch.full((batch, az.AZ_MAX_LEGAL), -1.0, dtype=torch.float32, device="cuda")
+    counts = torch.zeros((batch,), dtype=torch.int32, device="cuda")
+    val2 = torch.zeros((batch, cfg.value_size), dtype=torch.float32, device="cuda")
+    az.az_evaluate_legal(net, pos, masks, batch, legal, counts, val2)
+    torch.cuda.synchronize()
+    got = tower.cpu().numpy().transpose(0, 2, 1).reshape(batch, 64, 8, 8)
+    assert np.abs(got - raw["tower"]).max() <= 1e-5 * max(1.0, np.abs(raw["tower"]).max())
+    bits = np.unpackbits(mo.view(np.uint8), axis=1, bitorder="little")[:, : cfg.policy_size].astype(bool)
+    lg, cn = legal.cpu().numpy(), counts.cpu().numpy()
+    for i in range(batch):
+        assert cn[i] == bits[i].sum()
+        assert np.array_equal(lg[i, : cn[i]], pg[i][bits[i]])
+        assert (lg[i, cn[i]:] == -1.0).all()
+    assert np.array_equal(val2.cpu().numpy(), vg)
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
 @pytest.mark.parametrize("blocks", [0, 1, 3])
 def test_tower_activations_bf16_128_channels(az, blocks):
     # layer-level check of the convolution tower against the oracle's tower output
