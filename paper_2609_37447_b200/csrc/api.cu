@@ -148,14 +148,17 @@ int build_net(Net &n, const BlobView &v) {
         std::vector<__nv_bfloat16> packed(bytes / sizeof(__nv_bfloat16));
         n.tc_pair = n.want_pair && tc_pair_shape(C, (int)a.precision, false);
         const int halves = n.tc_pair ? 2 : 1;
-        tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, halves, 9, packed.data());
+        tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, halves, 9, false, packed.data());
         AZ_CUDA(cudaMalloc(&n.tc_weights, bytes));
         AZ_CUDA(cudaMemcpy(n.tc_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
         if (C == 256) {
             // small batches run two CTAs per group, each on half of the output channels: the same tiles, packed per half
-            tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, 2, 3, packed.data());
+            tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, 2, 9, true, packed.data());
             AZ_CUDA(cudaMalloc(&n.tc_weights_split, bytes));
             AZ_CUDA(cudaMemcpy(n.tc_weights_split, packed.data(), bytes, cudaMemcpyHostToDevice));
+            tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, 4, 9, true, packed.data());
+            AZ_CUDA(cudaMalloc(&n.tc_weights_split4, bytes));
+            AZ_CUDA(cudaMemcpy(n.tc_weights_split4, packed.data(), bytes, cudaMemcpyHostToDevice));
         }
         std::vector<float> bias((size_t)n.n_conv * C);
         for (int l = 0; l < n.n_conv; ++l) memcpy(&bias[(size_t)l * C], b[l], sizeof(float) * C);
@@ -261,7 +264,7 @@ void free_net(Net *n) {
     if (!n) return;
     for (int i = 0; i < 1 + 2 * 64; ++i) { cudaFree(n->conv_w[i]); cudaFree(n->conv_scale[i]); cudaFree(n->conv_bias[i]); }
     cudaFree(n->f32_layers);
-    cudaFree(n->tc_weights); cudaFree(n->tc_weights_split); cudaFree(n->tc_bias); cudaFree(n->tc_head_w); cudaFree(n->tc_head_bias);
+    cudaFree(n->tc_weights); cudaFree(n->tc_weights_split); cudaFree(n->tc_weights_split4); cudaFree(n->tc_bias); cudaFree(n->tc_head_w); cudaFree(n->tc_head_bias);
     cudaFree(n->tc8_weights); cudaFree(n->tc8_lconst);
     delete static_cast<HostMaster *>(n->host_master);
     cudaFree(n->fc_policy_w); cudaFree(n->fc_value_w); cudaFree(n->u_policy); cudaFree(n->u_value);

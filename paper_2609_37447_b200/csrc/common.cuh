@@ -52,6 +52,7 @@ struct Net {
     // ---- tensor-core tower (bf16, channels == 128) ----
     void *tc_weights = nullptr;       // packed UMMA B-operand tiles, all layers
     void *tc_weights_split = nullptr; // 256 channels: the same tiles packed in halves of N for the small-batch kernel (two CTAs per group)
+    void *tc_weights_split4 = nullptr;// and in quarters (four CTAs per group)
     float *tc_bias = nullptr;         // [n_conv][C] folded bias (scales are folded into the weights)
     bool tc_ready = false;
     bool want_pair = false;           // az_load_net_ex was asked for the CTA-pair form of the tower
@@ -206,7 +207,7 @@ int launch_heads_f32(const Net &n, const void *tower, const uint64_t *masks, int
 // tensor-core tower (tower_tc.cu)
 size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv);
 void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
-                     int channels, int n_conv, int halves, int stage_taps, __nv_bfloat16 *packed_host);
+                     int channels, int n_conv, int halves, int stage_taps, bool rotate, __nv_bfloat16 *packed_host);
 bool tc_pair_shape(int channels, int precision, bool pnet);     // the tower runs on CTA pairs (weights packed in halves)
 // exactly one of `planes` (encoded plane tensor) and `positions` (records to encode in the kernel) is non-null
 int launch_tower_tc(const Net &net, const void *planes, const void *positions, int batch, void *tower_out,

@@ -51,6 +51,18 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void *src
                  : "memory");
 }
 
+// the same from this CTA's shared memory into the shared memory of a CTA of the cluster (dst and bar: shared::cluster
+// addresses of that CTA, from map_to_cta); completion counts as transaction bytes on THAT CTA's mbarrier
+__device__ __forceinline__ void bulk_copy_s2s(uint32_t dst_cluster, uint32_t src_smem, uint32_t bytes, uint32_t cluster_bar) {
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_cluster), "r"(src_smem), "r"(bytes), "r"(cluster_bar)
+                 : "memory");
+}
+// asks L2 for a range of global memory that a later bulk copy will read (16-byte aligned, a multiple of 16 bytes)
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src_gmem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src_gmem), "r"(bytes) : "memory");
+}
+
 // ---- tcgen05 -----------------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {   // whole warp
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
@@ -201,6 +213,12 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// the same without release semantics: for signals that publish no writes of this thread ("the tensor core is done
+// reading", "the copies have landed").  A releasing arrival at cluster scope costs its thread on the order of a
+// thousand cycles (measured), which matters on a layer's critical path.
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ uint32_t mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {     // acquire at cluster scope
     uint32_t ok;

@@ -69,8 +69,12 @@ constexpr uint32_t kSpinLimit = 1u << 24;
 // frame, N = C with each CTA holding HALF of every weight tile in its own shared memory (tcgen05 .cta_group::2).
 // The shared-memory pipe that bounds the 128-channel shape then carries 6 KB of operands per MMA instead of 8.
 // NSPLIT > 1 (small batches of the 256-channel shape): a cluster of NSPLIT CTAs carries ONE group; each CTA computes
-// C / NSPLIT of every layer's output channels from the whole input (its own copy of the frame) and writes its slices
-// into every CTA's frame through distributed shared memory, so a layer takes 1 / NSPLIT of the tensor time.
+// C / NSPLIT of every layer's output channels from the whole input (its own copy of the frame).  Its epilogue writes the
+// slices into its own frame; a warp of its own sends each finished slice on to the other CTAs' frames as one bulk copy
+// through distributed shared memory, counted on the receiver's hand-off barrier; another acknowledges the slices
+// received.  Each CTA walks a layer's K starting at its own slices, so the exchange overlaps its first MMAs.  A layer
+// then takes 1/2 (two CTAs) or 3/8 (four: MMAs of 64 columns are bound by the operand reads, 48 cycles, not 32) of the
+// tensor time.
 template <int C, int GROUPS, int SETS, bool PAIR = false, int NSPLIT = 1>
 struct Shape {
     static constexpr int kC = C, kGroups = GROUPS, kSets = SETS;
@@ -83,21 +87,21 @@ struct Shape {
     static constexpr int kSlices = kC / 16;                          // 16-channel slices of a layer's output
     static constexpr int kFrameBytes = kPlaneBytes * (kC / 8);       // 46336 / 92672 per group
     static constexpr int kTileBytes = kC * 32 / kParts;              // one tap: this CTA's rows of the N = C tile x 32 bytes of K
-    static constexpr int kStageTaps = kC == 256 ? 3 : 9;
+    static constexpr int kStageTaps = (kC == 256 && NSPLIT == 1) ? 3 : 9;
     static constexpr int kStagesPerSlice = 9 / kStageTaps;
     static constexpr int kStageBytes = kStageTaps * kTileBytes;      // 36864 / 24576; pair: 18432
-    static constexpr int kStages = NSPLIT > 1 ? 10 : kC == 256 ? 5 : PAIR ? 7 : 3;
+    static constexpr int kStages = NSPLIT == 4 ? 6 : NSPLIT > 1 ? 3 : kC == 256 ? 5 : PAIR ? 7 : 3;     // (N-split: 108 KB of 18 / 36 KB stages)
     // pair: the second group's issuer runs this many weight stages behind the first's (half a layer), so that each
     // group's layer hand-over falls into the middle of the other's layer; the halved stages make the ring deep enough
     static constexpr int kLag = PAIR ? 4 : 0;
     static constexpr int kEpiWarps = 4 * kGroups * kSets;
-    static constexpr int kThreads = 32 * (1 + kGroups + kEpiWarps);  // producer, one issuer per group, 4 epilogue warps per group and set
+    static constexpr int kThreads = 32 * (1 + kGroups + kEpiWarps + (NSPLIT > 1 ? 2 : 0));  // producer, one issuer per group, 4 epilogue warps per group and set; N-split: a warp that sends the finished slices to the other CTAs and one that acknowledges theirs
     static constexpr uint32_t kBDescLbo = (uint32_t)(kC / kParts) << 16;    // K core matrices (rows of this CTA's tile)*16 bytes apart
     static constexpr int kOffFrames = 0;
     static constexpr int kOffWeights = kGroups * kFrameBytes;
     static constexpr int kOffBars = kOffWeights + kStages * kStageBytes;
-    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done, lead[S], pool[G], peer_full[S], peers_done[G]
-    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1 + kStages + kGroups + kStages + kGroups;
+    // barriers: w_full[S], w_empty[S], acc_full[G], a_ready[G][slices], done, lead[S], pool[G], peer_full[S], peers_done[G], ack[G]
+    static constexpr int kNumBars = 2 * kStages + kGroups + kGroups * kSlices + 1 + kStages + kGroups + kStages + 2 * kGroups;
     static constexpr int kOffTmemPtr = kOffBars + kNumBars * 8;
     static constexpr int kOffAbort = kOffTmemPtr + 4;
     static constexpr int kOffConst = (kOffAbort + 4 + 15) & ~15;     // per-warp copies of the current layer's channel constants
@@ -184,6 +188,15 @@ __device__ __forceinline__ Round get_round(int r, int cta, int P, int G) {
     return rd;
 }
 
+// N-split: the order in which the CTA of rank `rank` walks the K slices of a layer after the input layer: first the
+// out_slices slices it produced itself (they are in its frame first), then the other CTAs', their first slices, then their
+// second ones, and so on, which is the order in which they arrive.  The weights are packed in the same order.
+__host__ __device__ inline int nsplit_k_slice(int nsplit, int out_slices, int rank, int ki) {
+    if (ki < out_slices) return rank * out_slices + ki;
+    const int j = ki - out_slices, i = j / (nsplit - 1), p = (rank + 1 + j % (nsplit - 1)) % nsplit;
+    return p * out_slices + i;
+}
+
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status,
                                          long long *waited = nullptr) {
     return bounded_wait(bar, parity, abort_flag, status, kStatusWaitTimeout, kSpinLimit, waited);
@@ -197,7 +210,7 @@ __device__ __forceinline__ bool wait_bar_cluster(uint32_t bar, uint32_t parity, 
 // slices of the head projection's K that travel in one weight stage (the last stage may carry fewer: eleven
 // slices of the 176-channel shape go as six and five)
 template <class S> __device__ __host__ constexpr int head_slices_per_stage(int head_n) {
-    return S::kC == 128 ? (head_n == 256 ? 4 : S::kSlices) : S::kC == 160 ? 5 : S::kC == 176 ? 6 : (S::kNSplit > 1 ? (head_n == 64 ? 4 : 2) : head_n == 64 ? 8 : 4);    // (split: stages of 12 KB)
+    return S::kC == 128 ? (head_n == 256 ? 4 : S::kSlices) : S::kC == 160 ? 5 : S::kC == 176 ? 6 : (S::kNSplit == 4 ? (head_n == 64 ? 8 : 4) : S::kNSplit > 1 ? (head_n == 64 ? 16 : 8) : head_n == 64 ? 8 : 4);    // (split: stages of 18 / 36 KB)
 }
 template <class S> __device__ __host__ constexpr int head_stages(int head_n) {
     return head_n ? (S::kSlices + head_slices_per_stage<S>(head_n) - 1) / head_slices_per_stage<S>(head_n) : 0;
@@ -242,6 +255,7 @@ tower_tc_kernel(const TowerArgs args) {
     auto bar_peer = [&](int s) { return bar_done + 8u * (1 + kStages + kGroups + s); };   // pair: the other CTA's half of stage s has landed
     // CTA pair: rank 0 issues every MMA of the pair; rank 1 supplies its rows, its half of the weights, its epilogue
     auto bar_pdone = [&](int g) { return bar_done + 8u * (1 + kStages + kGroups + kStages + g); };   // N-split: the other CTAs' MMAs of this layer are complete
+    auto bar_ack = [&](int g) { return bar_done + 8u * (1 + kStages + kGroups + kStages + kGroups + g); };   // N-split: the other CTAs hold this CTA's slices of the layer
     constexpr bool kPair = S::kPair;
     static_assert(!kPair || (!kFp8 && !kPnet && kGroups == 2), "CTA pairs exist for the two-group bf16 shape of the residual networks");
     constexpr int kNSplit = S::kNSplit, kN = S::kN;
@@ -273,6 +287,7 @@ tower_tc_kernel(const TowerArgs args) {
         for (int g = 0; g < kGroups; ++g) {
             ptx::mbar_init(bar_acc_full(g), 1);
             ptx::mbar_init(bar_pdone(g), kNSplit > 1 ? kNSplit - 1 : 1);
+            ptx::mbar_init(bar_ack(g), kNSplit > 1 ? kNSplit - 1 : 1);
             ptx::mbar_init(bar_pool(g), 4 * S::kSets);
             // (pair: the first CTA's barriers also count the other CTA's epilogue warps)
             for (int kc = 0; kc < kSlices; ++kc) ptx::mbar_init(bar_a_ready(g, kc), 4 * S::kSets * S::kHalves);
@@ -341,7 +356,14 @@ tower_tc_kernel(const TowerArgs args) {
             int n_stages = 0;
             for (int l = 0; l < n_conv; ++l) n_stages += stages_of(l);
             const int n_head_stages = head_stages<S>(head_n);
+            // N-split (few CTAs, each waiting on its own stream of weights): ask L2 for every stage one layer before it
+            // is copied, so that the copy's latency is L2's, not DRAM's
+            constexpr int kAhead = kSlices * S::kStagesPerSlice;
+            auto stage_src = [&](int st_) { return reinterpret_cast<const unsigned char *>(args.weights) + ((size_t)st_ * S::kParts + cta_rank) * kStageBytes; };
+            if (kNSplit > 1 && lane == 0)
+                for (int st = 0; st < kAhead && st < n_stages; ++st) ptx::bulk_prefetch_l2(stage_src(st), (uint32_t)kStageBytes);
             for (int st = 0; st < n_stages + n_head_stages && ok; ++st) {
+                if (kNSplit > 1 && lane == 0 && st + kAhead < n_stages) ptx::bulk_prefetch_l2(stage_src(st + kAhead), (uint32_t)kStageBytes);
                 // tower stages are contiguous and equally sized; the head projections follow as small stages of their own
                 const bool head = st >= n_stages;
                 // (pair: every stage is stored as this CTA's half, then the other's)
@@ -460,14 +482,17 @@ tower_tc_kernel(const TowerArgs args) {
                 const bool conv2 = l >= 2 && (l & 1) == 0;             // accumulates onto the residual stream
                 const uint32_t d = d_h + (((l & 1) == 1) ? (uint32_t)kN : 0u);   // conv1 writes the ACC columns
                 layer_last = gi + stages_of(l) - 1;
-                for (int kc = 0; kc < nkc && ok; ++kc) {
+                for (int ki = 0; ki < nkc && ok; ++ki) {
+                    // N-split: a CTA walks a layer's K starting at the slices it produced itself (the other CTAs' arrive
+                    // while these are being multiplied); its weights are packed in that order
+                    const int kc = (kNSplit > 1 && l > 0) ? nsplit_k_slice(kNSplit, kOutSlices, (int)cta_rank, ki) : ki;
                     // one group per CTA: the slice's first weight stage is normally there long before its activations;
                     // looking at it first leaves nothing between the activations' arrival and the first MMA
                     if (kGroups == 1) {
                         ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                         if (!ok) break;
                     }
-                    ok = kCluster ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
+                    ok = kPair ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
                                   : wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
                     if (!ok) break;
                     a_phase ^= 1u << kc;
@@ -497,7 +522,7 @@ tower_tc_kernel(const TowerArgs args) {
                                 for (int t = 0; t < S::kStageTaps; ++t) {
                                     const int tap = st * S::kStageTaps + t;
                                     const int dy = tap / 3 - 1, dx = tap % 3 - 1;
-                                    const uint32_t first = (tap == 0 && !conv2 && kc == 0 && part == 0) ? 0u : 1u;
+                                    const uint32_t first = (tap == 0 && !conv2 && ki == 0 && part == 0) ? 0u : 1u;
                                     if (kInt8)
                                         ptx::mma_i8_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
                                                           b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8, first, elected);
@@ -518,15 +543,15 @@ tower_tc_kernel(const TowerArgs args) {
                                     if (kPair)
                                         ptx::mma_bf16_elect_pair(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
                                                                  b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc,
-                                                                 (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
+                                                                 (tap == 0 && !conv2 && ki == 0) ? 0u : 1u, elected);
                                     else
                                         ptx::mma_bf16_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
                                                             b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc,
-                                                            (tap == 0 && !conv2 && kc == 0) ? 0u : 1u, elected);
+                                                            (tap == 0 && !conv2 && ki == 0) ? 0u : 1u, elected);
                                 }
                             }
                             if (elected) {
-                                if (kc == nkc - 1 && st == S::kStagesPerSlice - 1 && part == n_parts - 1) commit(bar_acc_full(g));
+                                if (ki == nkc - 1 && st == S::kStagesPerSlice - 1 && part == n_parts - 1) commit(bar_acc_full(g));
                                 commit(bar_w_empty(stage));
                                 if (lead) ptx::mbar_arrive(bar_lead(stage));
                             }
@@ -562,7 +587,7 @@ tower_tc_kernel(const TowerArgs args) {
                         }
                     }
                     if (!kPnet) {
-                        ok = kCluster ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
+                        ok = kPair ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
                                       : wait_bar(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
                         if (!ok) break;
                         a_phase ^= 1u << kc;
@@ -598,6 +623,86 @@ tower_tc_kernel(const TowerArgs args) {
         for (uint32_t i = 0; i < (1u << 22); ++i)
             if (ptx::mbar_try_wait(bar_done, 0)) break;
         }
+    } else if (kNSplit > 1 && warp == 1 + kGroups + S::kEpiWarps) {
+        // ================= N-split: the finished slices of this CTA -> the other CTAs' frames =================
+        // A slice (two planes of the frame, 5792 contiguous bytes, borders included: they are zero everywhere) goes out as
+        // one bulk copy per receiving CTA once the four epilogue warps have handed it off here; its bytes count on the
+        // RECEIVER's hand-off barrier of the slice, on which four lanes arrive for the four warps that barrier expects.
+        // A layer's slices go out only after every receiver's MMAs of that layer, which read the frames the copies land
+        // in, are complete (bar_pdone: each CTA's epilogue announces its own completion to the others).
+        constexpr uint32_t kSliceBytes = 2 * kPlaneBytes;
+        const uint32_t frame_addr = smem_base + S::kOffFrames;
+        uint32_t s_phase = 0, pdone_phase = 0, acc_phase = 0;
+        bool ok = true;
+        for (int r = 0; ok; ++r) {
+            const Round rd = round_of(r);
+            if (!rd.valid) break;
+            // hand-offs of a round: the input planes (not sent: every CTA encodes its own copy), then every layer
+            for (int h = 0; h <= n_conv && ok; ++h) {
+                if (h > 0) {
+                    // this CTA's MMAs of the layer are complete: the other CTAs may send their slices into its frame.  (Said
+                    // from here, not from the epilogue, whose warps are on the layer's critical path.)
+                    ok = wait_bar(bar_acc_full(0), acc_phase, abort_flag, args.status);
+                    acc_phase ^= 1u;
+                    if (!ok) break;
+                    if (lane == 0) {
+#pragma unroll
+                        for (int p = 0; p < kNSplit; ++p)
+                            if (p != (int)cta_rank) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(bar_pdone(0), (uint32_t)p));
+                    }
+                    __syncwarp();
+                    ok = wait_bar_cluster(bar_pdone(0), pdone_phase, abort_flag, args.status);
+                    pdone_phase ^= 1u;
+                    if (!ok || (h == n_conv && head_n == 0)) break;         // the last layer's output is read again only by the heads
+                }
+                for (int kl = 0; kl < kOutSlices && ok; ++kl) {
+                    const int kc = out0 + kl;
+                    if (h == 0 && kc >= in_slices) continue;                // the input planes fill the first in_slices slices only
+                    ok = wait_bar(bar_a_ready(0, kc), (s_phase >> kl) & 1u, abort_flag, args.status);
+                    if (!ok) break;
+                    s_phase ^= 1u << kl;
+                    if (h == 0) continue;
+#pragma unroll
+                    for (int p = 0; p < kNSplit; ++p)
+                        if (p != (int)cta_rank) {
+                            const uint32_t rbar = ptx::map_to_cta(bar_a_ready(0, kc), (uint32_t)p);
+                            if (lane < 4) ptx::mbar_arrive_expect_tx_cluster(rbar, kSliceBytes / 4);
+                            if (lane == 0)
+                                ptx::bulk_copy_s2s(ptx::map_to_cta(frame_addr + (uint32_t)(2 * kc) * kPlaneBytes, (uint32_t)p),
+                                                   frame_addr + (uint32_t)(2 * kc) * kPlaneBytes, kSliceBytes, rbar);
+                        }
+                    __syncwarp();
+                }
+            }
+            if (ok && head_n != 0) {                                        // (the head projections complete a phase of their own)
+                ok = wait_bar(bar_acc_full(0), acc_phase, abort_flag, args.status);
+                acc_phase ^= 1u;
+            }
+        }
+    } else if (kNSplit > 1 && warp == 2 + kGroups + S::kEpiWarps) {
+        // ================= N-split: acknowledge the other CTAs' slices =================
+        // The copies that bring a slice here read the SENDER's frame asynchronously; the sender may overwrite those planes
+        // (its epilogue of the next layer) only when the copies are done.  Their completion is visible here, on the slice's
+        // hand-off barrier: once all slices of a sender's layer have landed, tell the sender (bar_ack there).
+        uint32_t k_phase = 0;
+        bool ok = true;
+        for (int r = 0; ok; ++r) {
+            const Round rd = round_of(r);
+            if (!rd.valid) break;
+            const int n_sent = head_n != 0 ? n_conv : n_conv - 1;
+            for (int h = 0; h <= n_sent && ok; ++h)
+                for (int pi = 1; pi < kNSplit && ok; ++pi) {
+                    const int p = ((int)cta_rank + pi) % kNSplit;
+                    for (int kl = 0; kl < kOutSlices && ok; ++kl) {
+                        const int kc = p * kOutSlices + kl;
+                        if (h == 0 && kc >= in_slices) continue;
+                        ok = wait_bar(bar_a_ready(0, kc), (k_phase >> kc) & 1u, abort_flag, args.status);
+                        k_phase ^= 1u << kc;
+                    }
+                    if (ok && h > 0 && lane == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(bar_ack(0), (uint32_t)p));
+                    __syncwarp();
+                }
+        }
     } else {
         // ================= epilogue: 4 warps per group and set =================
         // A set's last hand-off of a layer comes after its TMEM loads and stores of that layer have
@@ -626,21 +731,13 @@ tower_tc_kernel(const TowerArgs args) {
         uint32_t acc_phase = 0;
         bool ok = true;
         // hand-off of a slice to the issuer: a barrier of this CTA; in a pair the first CTA's (which counts both CTAs'
-        // warps); with the N-split the barrier of EVERY CTA of the cluster (the slice has been written into every frame)
+        // warps).  With the N-split this hands off the CTA's OWN copy of the slice, to its issuer and to the warp that
+        // sends it on to the other CTAs.
         auto ready = [&](int kc_) {
             if (kPair) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_a_ready(g, kc_), 0));
-            else if (kNSplit > 1) {
-                // own frame: written with ordinary stores, handed off as always; the other CTAs' frames: written with
-                // asynchronous stores that count as transaction bytes on THEIR barrier (1 KB per warp and slice: 32
-                // rows x 32 bytes), announced with this warp's arrival; nothing here waits for the remote traffic
-                ptx::mbar_arrive(bar_a_ready(g, kc_));
-#pragma unroll
-                for (int p = 0; p < kNSplit; ++p)
-                    if (p != (int)cta_rank) ptx::mbar_arrive_expect_tx_cluster(ptx::map_to_cta(bar_a_ready(g, kc_), (uint32_t)p), 1024u);
-            } else ptx::mbar_arrive(bar_a_ready(g, kc_));
+            else ptx::mbar_arrive(bar_a_ready(g, kc_));
         };
-        uint32_t pdone_phase = 0;
-        const uint32_t frame_addr = ptx::smem_addr(frame);
+        uint32_t ack_phase = 0;
         if (kPnet) {
             // the pooled-context maps are read in the middle of a layer's hand-over, where a miss to DRAM would
             // sit on the critical path: ask for all of them now (148 CTAs ask for the same lines; L2 merges them)
@@ -708,10 +805,7 @@ tower_tc_kernel(const TowerArgs args) {
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0)
-                    for (int kc = 0; kc < in_slices; ++kc) {
-                        if (kNSplit > 1) ptx::mbar_arrive(bar_a_ready(g, kc));      // every CTA encodes its own copy of the input
-                        else ready(kc);
-                    }
+                    for (int kc = 0; kc < in_slices; ++kc) ready(kc);      // (N-split: every CTA encodes its own copy of the input)
             }
             for (int l = 0; l < n_conv && ok; ++l) {
                 const bool from_acc = (l & 1) == 1;
@@ -737,17 +831,13 @@ tower_tc_kernel(const TowerArgs args) {
                 if (!ok) break;
                 acc_phase ^= 1u;
                 ptx::tc_fence_after();
-                if (kNSplit > 1) {
-                    // this CTA's MMAs of the layer are complete, so the other CTAs may overwrite its frame: tell them
-                    // (their own completion is awaited below, just before the first store into their frames)
-                    if (q == 0 && lane == 0) {
-#pragma unroll
-                        for (int p = 0; p < kNSplit; ++p)
-                            if (p != (int)cta_rank) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_pdone(g), (uint32_t)p));
-                    }
-                    __syncwarp();
+                if (kNSplit > 1 && l > 0) {
+                    // before this layer's slices overwrite the last layer's in this frame, the copies that carry those to the
+                    // other CTAs must be done reading them: the receivers have said so (bar_ack; long ago, as a rule)
+                    ok = wait_bar_cluster(bar_ack(g), ack_phase, abort_flag, args.status, tr ? &t_wait[1] : nullptr);
+                    ack_phase ^= 1u;
+                    if (!ok) break;
                 }
-                bool peers_done = kNSplit == 1;
                 const float *bias = kFp8 ? lc + kMyC : lc;
                 __nv_bfloat16 *dst = args.out + ((size_t)board * 64 + sq) * kC;
                 const uint32_t t_src = t_lane + (uint32_t)(from_acc ? kN : 0);
@@ -993,24 +1083,6 @@ tower_tc_kernel(const TowerArgs args) {
                             for (int i = 0; i < 8; ++i) pk[i] = ptx::pack_bf16x2_relu(v[2 * i], v[2 * i + 1]);
                             *reinterpret_cast<uint4 *>(frame + (2 * kc) * kPlaneBytes + slot * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                             *reinterpret_cast<uint4 *>(frame + (2 * kc + 1) * kPlaneBytes + slot * 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-                            if (kNSplit > 1) {
-                                // the same slice into the other CTAs' frames, once their MMAs of this layer (which read
-                                // those frames) are complete
-                                if (!peers_done) {
-                                    ok = wait_bar_cluster(bar_pdone(g), pdone_phase, abort_flag, args.status);
-                                    pdone_phase ^= 1u;
-                                    peers_done = true;
-                                    if (!ok) break;
-                                }
-#pragma unroll
-                                for (int p = 0; p < kNSplit; ++p)
-                                    if (p != (int)cta_rank) {
-                                        const uint32_t dst0 = ptx::map_to_cta(frame_addr + (uint32_t)((2 * kc) * kPlaneBytes + slot * 16), (uint32_t)p);
-                                        const uint32_t rbar = ptx::map_to_cta(bar_a_ready(g, kc), (uint32_t)p);
-                                        ptx::st_async_cluster_v4(dst0, pk[0], pk[1], pk[2], pk[3], rbar);
-                                        ptx::st_async_cluster_v4(dst0 + (uint32_t)kPlaneBytes, pk[4], pk[5], pk[6], pk[7], rbar);
-                                    }
-                            }
                         }
                         if (kGroups > 1 && keep_h) write_back_h(ks, kl, v);
                         // e4m3 layers consume 32 channels per MMA: one hand-off per two slices.  With two sets
@@ -1030,16 +1102,17 @@ tower_tc_kernel(const TowerArgs args) {
                     }
                 }
                 if (keep_h) ptx::tmem_st_wait();
-                if (kNSplit > 1 && !peers_done && ok) {            // a layer that wrote no frame still takes the other CTAs' signal
-                    ok = wait_bar_cluster(bar_pdone(g), pdone_phase, abort_flag, args.status);
-                    pdone_phase ^= 1u;
-                }
             }
             if (head_n && ok) {
                 // ---- head projections out of the ACC columns
                 ok = wait_bar(bar_acc_full(g), acc_phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
                 if (!ok) break;
                 acc_phase ^= 1u;
+                if (kNSplit > 1) {                                 // (the last layer's slices were sent as well)
+                    ok = wait_bar_cluster(bar_ack(g), ack_phase, abort_flag, args.status);
+                    ack_phase ^= 1u;
+                    if (!ok) break;
+                }
                 // the residual towers' head rows are few: set 0 writes them all; the paper network's sixteen slices of
                 // queries and keys are dealt out over the sets
                 if (!kPnet && set != 0) continue;
@@ -1109,6 +1182,9 @@ tower_tc_kernel(const TowerArgs args) {
     }
 }
 
+#ifndef AZ_NSPLIT_MAX
+#define AZ_NSPLIT_MAX 4                  // the widest split of a group over CTAs that the launches use
+#endif
 #ifndef AZ_C128_SETS
 #define AZ_C128_SETS 1
 #endif
@@ -1120,6 +1196,7 @@ typedef Shape<128, 2, AZ_C128_SETS, true> Shape128Pair;    // the bf16 residual 
 typedef Shape<128, 2, AZ_FP8_EPI_SETS> Shape128F8;
 typedef Shape<256, 1, 1> Shape256;
 typedef Shape<256, 1, 1, false, 2> Shape256Split2;      // small batches: two CTAs per group, 128 output channels each
+typedef Shape<256, 1, 1, false, 4> Shape256Split4;      // smaller still: four CTAs per group, 64 output channels each
 // the paper's 160-channel network: one group, whose epilogue (not its MMAs) sets the pace with four warps;
 // two sets of four share each layer
 #ifndef AZ_P160_SETS
@@ -1142,17 +1219,18 @@ size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv) {
     return slices * 9 * (size_t)channels * 32;             // per slice and tap: N = channels rows x 32 bytes of K
 }
 
-// halves == 2 (CTA pairs, or two CTAs splitting the output channels): every weight stage (layer, slice, stage_taps
-// taps: nine, or three in the 256-channel shape) is stored as two halves of N, rows [0, C/2) of the stage's taps for
-// the cluster's first CTA, then rows [C/2, C) for the second.
+// halves > 1 (CTA pairs, or 2 / 4 CTAs splitting the output channels): every weight stage (layer, slice, stage_taps
+// taps: nine, or three in the 256-channel shape) is stored as `halves` parts of N, rows [0, C/halves) of the stage's
+// taps for the cluster's first CTA, then the next CTA's rows, and so on.  rotate (the N-split): after the input
+// layer, part h walks K in the order nsplit_k_slice gives, its own output slices of the layer before first.
 void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
-                     int channels, int n_conv, int halves, int stage_taps, __nv_bfloat16 *packed) {
+                     int channels, int n_conv, int halves, int stage_taps, bool rotate, __nv_bfloat16 *packed) {
     __nv_bfloat16 *dst = packed;
     const int groups_per_half = channels / 8 / halves;
     for (int l = 0; l < n_conv; ++l) {
         const int cin = l == 0 ? in_planes : channels;
         const int nkc = (l == 0 ? in_pad : channels) / 16;
-        for (int kc = 0; kc < nkc; ++kc)
+        for (int kp = 0; kp < nkc; ++kp)
             for (int st = 0; st < 9 / stage_taps; ++st)
                 for (int h = 0; h < halves; ++h)
                     for (int t = 0; t < stage_taps; ++t)
@@ -1160,6 +1238,7 @@ void tc_pack_weights(const float *const *w, const float *const *scale, int in_pl
                             for (int ng = h * groups_per_half; ng < (h + 1) * groups_per_half; ++ng)
                                 for (int r = 0; r < 8; ++r)
                                     for (int e = 0; e < 8; ++e) {
+                                        const int kc = (rotate && l > 0) ? nsplit_k_slice(halves, nkc / halves, h, kp) : kp;
                                         const int tap = st * stage_taps + t;
                                         const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
                                         float v = 0.0f;
@@ -1241,7 +1320,7 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
     for (int l = 1; l < n_conv; ++l)
         for (int c = 0; c < C; ++c) sa[(size_t)l * C + c] = fmaxf(absmax[(size_t)(l - 1) * C + c], kTiny) / kMax;
     // layer 0: bf16 tiles exactly as in the bf16 tower
-    tc_pack_weights(w, scale, in_planes, in_pad, C, 1, 1, 9, reinterpret_cast<__nv_bfloat16 *>(packed));
+    tc_pack_weights(w, scale, in_planes, in_pad, C, 1, 1, 9, false, reinterpret_cast<__nv_bfloat16 *>(packed));
     unsigned char *dst = packed + (size_t)(in_pad / 16) * kStageBytes;
     std::vector<float> wf((size_t)C * C * 9);
     for (int l = 1; l < n_conv; ++l) {
@@ -1333,6 +1412,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256Split2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256Split4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128P, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape160, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128P, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
@@ -1381,17 +1461,19 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
     else if (net.pnet && fp8) tower_tc_kernel<true, Shape128P, true, true><<<grid, Shape128P::kThreads, Shape128P::smem_bytes(true, true), s>>>(a);
     else if (net.pnet) tower_tc_kernel<false, Shape128P, true><<<grid, Shape128P::kThreads, Shape128P::smem_bytes(false, true), s>>>(a);
     else if (wide && n_groups * 2 <= sms) {
-        // few boards: two CTAs (a cluster) per group, each computing half of every layer's output channels from a
-        // second copy of the weights packed for that split
-        a.weights = net.tc_weights_split;
+        // few boards: a cluster of four or two CTAs per group, each computing a quarter or half of every layer's output
+        // channels from a copy of the weights packed for that split
+        const int split = (net.tc_weights_split4 != nullptr && n_groups * 4 <= sms && AZ_NSPLIT_MAX >= 4) ? 4 : 2;
+        a.weights = split == 4 ? net.tc_weights_split4 : net.tc_weights_split;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(2 * n_groups); cfg.blockDim = dim3(Shape256Split2::kThreads);
-        cfg.dynamicSmemBytes = Shape256Split2::smem_bytes(false); cfg.stream = s;
+        cfg.gridDim = dim3(split * n_groups); cfg.blockDim = dim3(Shape256Split2::kThreads);
+        cfg.dynamicSmemBytes = split == 4 ? Shape256Split4::smem_bytes(false) : Shape256Split2::smem_bytes(false); cfg.stream = s;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        attr[0].val.clusterDim.x = split; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
         cfg.attrs = attr; cfg.numAttrs = 1;
-        AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<false, Shape256Split2>, a));
+        if (split == 4) AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<false, Shape256Split4>, a));
+        else AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<false, Shape256Split2>, a));
         return AZ_OK;
     }
     else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);

@@ -44,6 +44,14 @@ def gpu_evaluate(az, net, cfg, recs, masks_np=None):
     return az.masks_to_numpy(masks), policy.cpu().numpy(), value.cpu().numpy()
 
 
+def corr_bar(floor_corr, n):
+    # What a correlation with the oracle must reach over n positions when bf16 operands with exact accumulation leave
+    # floor_corr of it: 0.9 where the floor allows; else the floor less three standard errors of a sample correlation
+    # coefficient, (1 - r^2) / sqrt(n).  (The kernel's rounding errors are one draw, the emulation's another: any change
+    # in the order of the fp32 accumulation redraws them.  48 positions at r = 0.89: 0.09; 1024 positions: 0.02.)
+    return min(0.9, floor_corr - 3.0 * (1.0 - floor_corr ** 2) / np.sqrt(n))
+
+
 def compare(cfg, masks_g, pol_g, val_g, masks_o, pol_o, val_o, tol):
     assert (masks_g == masks_o).all(), "legal masks differ"
     assert np.isfinite(pol_g).all() and np.isfinite(val_g).all()
@@ -61,7 +69,7 @@ def compare(cfg, masks_g, pol_g, val_g, masks_o, pol_o, val_o, tol):
         # leave of it for this weight set where that is less (tests/golden/quant_floors.json).
         need = 0.9
         if cfg.name in ("c2", "c3", "c5") and cfg.precision == 1:
-            need = min(0.9, stored_floor(cfg.name)["value_min_component_corr"] - 0.03)
+            need = corr_bar(stored_floor(cfg.name)["value_min_component_corr"], pol_g.shape[0])
         for k in range(val_o.shape[1]):
             assert np.corrcoef(val_g[:, k], val_o[:, k])[0, 1] > need
         zg, zo = value_pre(val_g), value_pre(val_o)
@@ -299,7 +307,7 @@ def test_value_head_error_relative_to_its_spread(az, name, batch):
               f"(bf16 floor {floor['value_pre_rms_over_spread']:.4f}), output max-abs {np.abs(vg - vo).max():.3e}")
         assert frac <= 1.5 * floor["value_pre_rms_over_spread"] + 2e-3
         for k in range(vo.shape[1]):
-            assert np.corrcoef(vg[:, k], vo[:, k])[0, 1] > min(0.9, floor["value_min_component_corr"] - 0.03)
+            assert np.corrcoef(vg[:, k], vo[:, k])[0, 1] > corr_bar(floor["value_min_component_corr"], batch)
         assert np.corrcoef(value_pre(vg).ravel(), value_pre(vo).ravel())[0, 1] > 0.9
         if spread is None:
             floor_spread = got_spread          # what the stored head scale gives on these positions
@@ -522,13 +530,30 @@ def test_work_schedule_is_invisible_in_the_results(az, channels, in_planes):
     _, p_all, v_all = gpu_evaluate(az, net, cfg, recs, masks_np=masks)
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     per_round = sms * (4 if channels == 128 else 2)           # positions one full round of all CTAs takes
-    sizes = sorted({1, 2, 3, 5, 2 * sms - 1, 2 * sms, 2 * sms + 1, per_round - 3, per_round, per_round + 2,
-                    per_round + 2 * sms, per_round + 2 * sms + 2, per_round + 3 * sms + 1, 2 * per_round - 2, 1199})
-    for n in sizes:
+    sizes = {1, 2, 3, 5, 2 * sms - 1, 2 * sms, 2 * sms + 1, per_round - 3, per_round, per_round + 2,
+             per_round + 2 * sms, per_round + 2 * sms + 2, per_round + 3 * sms + 1, 2 * per_round - 2, 1199}
+    # The 256-channel tower has three forms: up to sms/4 two-board groups run on clusters of four CTAs per group, up
+    # to sms/2 on clusters of two, more on one CTA per group.  The forms add up a layer's products in different
+    # orders (each CTA of a cluster starts with the slices it produced itself), so between forms a row agrees to
+    # rounding; within a form every prefix reproduces bit for bit.
+    def form(n):
+        groups = (n + 1) // 2
+        return 0 if channels != 256 else 2 if 4 * groups <= sms else 1 if 2 * groups <= sms else 0
+    edges = [2 * (sms // 4), 2 * (sms // 2)] if channels == 256 else []
+    for e in edges:
+        sizes |= {e - 1, e, e + 1}
+    whole = {0: (p_all, v_all)}
+    for f, e in zip((2, 1), edges):
+        _, pe, ve = gpu_evaluate(az, net, cfg, recs[:e], masks_np=masks[:e])
+        whole[f] = (pe, ve)
+        assert np.abs(pe - p_all[:e]).max() <= 1e-3 and np.abs(ve - v_all[:e]).max() <= 1e-3     # between forms
+        assert not np.array_equal(pe, p_all[:e])              # (they do differ: the forms are really in use)
+    for n in sorted(sizes):
         if n > 1200:
             continue
         _, p, v = gpu_evaluate(az, net, cfg, recs[:n], masks_np=masks[:n])
-        assert np.array_equal(p, p_all[:n]) and np.array_equal(v, v_all[:n]), n
+        pw, vw = whole[form(n)]
+        assert np.array_equal(p, pw[:n]) and np.array_equal(v, vw[:n]), n
     # oracle spot check on rows that sit at the seams of the schedule
     rows = np.array([0, 1, 2 * sms - 1, 2 * sms, per_round - 1, per_round, min(per_round + 2 * sms, 1199), 1199])
     rows = rows[rows < 1200]
