@@ -192,7 +192,7 @@ masked_softmax_kernel(const float *__restrict__ logits, const unsigned long long
     for (int j = 0; j < ITEMS; ++j) {
         const int i = tid + 128 * j;
         const bool legal = i < n && ((mw[i >> 6] >> (i & 63)) & 1ull);
-        v[j] = legal ? row[i] : -INFINITY;
+        v[j] = legal ? __ldcg(row + i) : -INFINITY;      // (written by the kernel before: not through the read-only path)
         mx = fmaxf(mx, v[j]);
     }
 #pragma unroll
@@ -271,7 +271,7 @@ masked_softmax_compact_kernel(const float *__restrict__ logits, const unsigned l
             const int bit = __ffsll((long long)bits) - 1;
             bits &= bits - 1;
             if (j < kMaxLegal) {
-                const float l = row[(lane + 32 * k) * 64 + bit];
+                const float l = __ldcg(row + (lane + 32 * k) * 64 + bit);
                 v[j] = l;
                 mx = fmaxf(mx, l);
             }

@@ -108,6 +108,7 @@ tower_f32_kernel(const F32Args args) {
     // nothing may reach into the other CTA before its barriers and frames are initialised
     ptx::cluster_arrive();
     ptx::cluster_wait();
+    ptx::launch_dependents();        // the heads kernel may start its set-up; it waits for this grid before reading its output
 
     const int n_conv = args.n_conv;
     auto chunks_of = [&](int l) { return (l == 0 ? kInPad : kC) / kChunkCi; };
@@ -337,13 +338,28 @@ heads_f32_kernel(const HeadsF32Args a) {
     __shared__ float part[kValueHidden * 8];                     // the hidden layer's per-warp partial sums
     __shared__ float red[kHeadThreads / 32];
     __shared__ int rank_base[kPlanes73 + 1];
-    const int pos = blockIdx.x, tid = threadIdx.x, sq = tid & 63, pg = tid >> 6, lane = tid & 31, warp = tid >> 5;
+    // two CTAs per position, on two SMs: the even one computes the policy, the odd one the value (both need nothing but
+    // the position's tower output, and one after the other they were a chain of load latencies on one SM)
+    const int pos = blockIdx.x >> 1, tid = threadIdx.x, sq = tid & 63, pg = tid >> 6, lane = tid & 31, warp = tid >> 5;
+    const bool policy_cta = (blockIdx.x & 1) == 0;
+    // before the tower's output exists: ask L2 for this CTA's share of the weights (the hidden layer's megabyte is split
+    // over the value CTAs, the policy map over the policy CTAs)
+    {
+        const char *wb = reinterpret_cast<const char *>(policy_cta ? a.p_w : a.v_w1);
+        const size_t bytes = policy_cta ? sizeof(float) * kPlanes73 * kC : sizeof(float) * (size_t)kValueHidden * kHeadChannels * 64;
+        const size_t n_cta = gridDim.x >> 1, share = (bytes / n_cta + 127) & ~(size_t)127;
+        const size_t off = (size_t)pos * share + (size_t)tid * 128;
+        if ((size_t)tid * 128 < share && off < bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(wb + off));
+    }
+    ptx::grid_dependency_wait();
     float hr[kC];
     {
         const float4 *src = reinterpret_cast<const float4 *>(a.h + ((size_t)pos * 64 + sq) * kC);
 #pragma unroll
-        for (int i = 0; i < kC / 4; ++i) { const float4 v = __ldg(src + i); hr[4 * i] = v.x; hr[4 * i + 1] = v.y; hr[4 * i + 2] = v.z; hr[4 * i + 3] = v.w; }
+        // (not through the read-only path: this kernel may have started before the tower kernel wrote these lines)
+        for (int i = 0; i < kC / 4; ++i) { const float4 v = __ldcg(src + i); hr[4 * i] = v.x; hr[4 * i + 1] = v.y; hr[4 * i + 2] = v.z; hr[4 * i + 3] = v.w; }
     }
+    if (policy_cta) {
     // ---- policy logits of this square: planes pg, pg + 4, ...
     float lg[kPolicyPerThread];
     float mx = -INFINITY;
@@ -365,22 +381,8 @@ heads_f32_kernel(const HeadsF32Args a) {
         }
         mx = fmaxf(mx, lg[j]);
     }
-    // ---- value projection of this square: channels pg, pg + 4, ...
-#pragma unroll
-    for (int j = 0; j < kHeadChannels / 4; ++j) {
-        const int c = pg + 4 * j;
-        const float4 *wr = reinterpret_cast<const float4 *>(a.v_cw + (size_t)c * kC);
-        float acc0 = 0.0f, acc1 = 0.0f;
-#pragma unroll
-        for (int i = 0; i < kC / 4; ++i) {
-            const float4 w = __ldg(wr + i);
-            acc0 = fmaf(w.x, hr[4 * i], acc0); acc1 = fmaf(w.y, hr[4 * i + 1], acc1);
-            acc0 = fmaf(w.z, hr[4 * i + 2], acc0); acc1 = fmaf(w.w, hr[4 * i + 3], acc1);
-        }
-        u[c * 64 + sq] = fmaxf(fmaf(__ldg(a.v_cs + c), acc0 + acc1, __ldg(a.v_cb + c)), 0.0f);
-    }
     // ---- masked softmax over the position's legal logits
-    mx = block_reduce(mx, true, red);                           // (its barriers also publish u[])
+    mx = block_reduce(mx, true, red);
     const bool any = mx > -INFINITY;
     float sum = 0.0f;
 #pragma unroll
@@ -421,6 +423,23 @@ heads_f32_kernel(const HeadsF32Args a) {
         if (tid == 0) a.counts[pos] = rank_base[kPlanes73] < kMaxLegal ? rank_base[kPlanes73] : kMaxLegal;
     }
     if (!any && tid == 0) atomicOr(a.status, kStatusEmptyMask);
+    return;
+    }
+    // ---- value projection of this square: channels pg, pg + 4, ...
+#pragma unroll
+    for (int j = 0; j < kHeadChannels / 4; ++j) {
+        const int c = pg + 4 * j;
+        const float4 *wr = reinterpret_cast<const float4 *>(a.v_cw + (size_t)c * kC);
+        float acc0 = 0.0f, acc1 = 0.0f;
+#pragma unroll
+        for (int i = 0; i < kC / 4; ++i) {
+            const float4 w = __ldg(wr + i);
+            acc0 = fmaf(w.x, hr[4 * i], acc0); acc1 = fmaf(w.y, hr[4 * i + 1], acc1);
+            acc0 = fmaf(w.z, hr[4 * i + 2], acc0); acc1 = fmaf(w.w, hr[4 * i + 3], acc1);
+        }
+        u[c * 64 + sq] = fmaxf(fmaf(__ldg(a.v_cs + c), acc0 + acc1, __ldg(a.v_cb + c)), 0.0f);
+    }
+    __syncthreads();
     // ---- hidden layer: all eight warps share every row (a thread holds eight of the 2,048 inputs in registers and
     // reads the matching eight weights of sixteen rows at a time, 32 independent 16-byte loads in flight), the warps'
     // partial sums meet in shared memory
@@ -492,8 +511,7 @@ int launch_heads_f32(const Net &n, const void *tower, const uint64_t *masks, int
     a.policy = policy; a.legal = legal; a.counts = counts; a.value = value;
     a.status = n.status_dev;
     a.wdl = n.arch.value_head == AZ_VALUE_WDL;
-    heads_f32_kernel<<<batch, kHeadThreads, 0, s>>>(a);
-    AZ_LAUNCH_CHECK();
+    AZ_CUDA(launch_dependent(heads_f32_kernel, dim3(2 * batch), dim3(kHeadThreads), 0, s, a));
     return AZ_OK;
 }
 

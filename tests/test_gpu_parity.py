@@ -248,6 +248,34 @@ def test_fp32_64_channel_networks_on_the_fused_kernels(az, blocks, value_head, b
     az.az_free_net(net)
 
 
+@pytest.mark.parametrize("channels,in_planes,policy_head,precision", [(64, 19, 0, 0), (128, 19, 0, 1), (128, 19, 1, 1), (256, 112, 1, 1)])
+def test_alternating_batches_each_see_their_own_tower_output(az, channels, in_planes, policy_head, precision):
+    # The head kernels start before the tower kernel has finished (programmatic dependent launch) and wait for it before
+    # they read what it wrote.  A read that slipped ahead of that wait would see the tower output of the evaluation
+    # BEFORE, which no test that evaluates one batch per network can notice.  Two different batches, alternately, through
+    # the same network and the same workspace: every evaluation must reproduce its batch's own result bit for bit and
+    # match the oracle.
+    cfg = configs.tiny_config(in_planes=in_planes, blocks=2, channels=channels, policy_head=policy_head, value_head=1,
+                              precision=precision, batch=40, weight_seed=77)
+    blob = weights.make_blob(cfg, 0.3, 0.3)
+    net, _ = load(az, cfg, blob=blob)
+    rec_a = positions.records_for_planes(in_planes, positions.generate(9100, 40, (0, 30))[0])
+    rec_b = positions.records_for_planes(in_planes, positions.generate(9200, 40, (60, 140))[0])
+    ma, pa, va = gpu_evaluate(az, net, cfg, rec_a)
+    mb, pb, vb = gpu_evaluate(az, net, cfg, rec_b)
+    assert not np.array_equal(pa, pb)
+    for _ in range(3):
+        _, p2, v2 = gpu_evaluate(az, net, cfg, rec_a)
+        assert np.array_equal(p2, pa) and np.array_equal(v2, va)
+        _, p2, v2 = gpu_evaluate(az, net, cfg, rec_b)
+        assert np.array_equal(p2, pb) and np.array_equal(v2, vb)
+    for m, p, v, rec in ((ma, pa, va, rec_a), (mb, pb, vb, rec_b)):
+        mo, _, po, vo = oracle.evaluate(blob, rec, in_planes, policy_head)
+        compare(cfg, m, p, v, mo, po, vo, TOL[precision])
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
 @pytest.mark.parametrize("blocks", [0, 1, 3])
 def test_tower_activations_bf16_128_channels(az, blocks):
     # layer-level check of the convolution tower against the oracle's tower output

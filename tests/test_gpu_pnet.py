@@ -70,6 +70,29 @@ def test_small_networks_layer_by_layer(blocks, batch, channels):
     assert np.abs(pg - po).max() <= TOL and np.abs(vg - vo).max() <= TOL
 
 
+def test_alternating_batches_each_see_their_own_tower_output():
+    # the finishing kernel starts before the tower kernel has ended and must not read the tower's output (features,
+    # queries, keys) before its dependency wait: two different batches, alternately, through one network
+    import paper_2609_37447_b200 as az
+    cfg = pw.PNetConfig("alt", 2, 128, 40, 20260972, 4490)
+    blob = pw.make_blob(cfg, 0.1, 0.6)
+    net = load(az, cfg, blob, 64)
+    rec_a, _ = positions.generate_moves(9300, 40, (0, 30))
+    rec_b, _ = positions.generate_moves(9400, 40, (60, 160))
+    _, pa, va, _ = gpu_run(az, net, cfg, rec_a)
+    _, pb, vb, _ = gpu_run(az, net, cfg, rec_b)
+    assert not np.array_equal(pa, pb)
+    for _ in range(3):
+        _, p2, v2, _ = gpu_run(az, net, cfg, rec_a)
+        assert np.array_equal(p2, pa) and np.array_equal(v2, va)
+        _, p2, v2, _ = gpu_run(az, net, cfg, rec_b)
+        assert np.array_equal(p2, pb) and np.array_equal(v2, vb)
+    az.az_free_net(net)
+    for p, v, rec in ((pa, va, rec_a), (pb, vb, rec_b)):
+        _, _, po, vo = oracle.pnet_evaluate(blob, rec)
+        assert np.abs(p - po).max() <= TOL and np.abs(v - vo).max() <= TOL
+
+
 def test_p12_batch_1024():
     import paper_2609_37447_b200 as az
     cfg = pw.PNET_CONFIGS["p12"]
