@@ -14,6 +14,8 @@
 // 32 / 64 (the fp32 config) take the tiled kernel further down.
 #include "common.cuh"
 
+#include <mutex>
+
 namespace az {
 namespace {
 
@@ -186,11 +188,15 @@ int launch_conv3x3_simt(const void *in, const void *w, const float *scale, const
     if (batch == 0) return AZ_OK;
     if (!bf16 && cin % kChunk == 0 && cout % kCoutTile == 0) {
         static bool configured[64] = {};
+        static std::mutex configured_lock;                  // any thread may make a device's first launch
         int dev = 0;
         AZ_CUDA(cudaGetDevice(&dev));
-        if (dev < 64 && !configured[dev]) {
-            AZ_CUDA(cudaFuncSetAttribute(conv3x3_f32_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileSmem));
-            configured[dev] = true;
+        {
+            std::lock_guard<std::mutex> hold(configured_lock);
+            if (dev >= 0 && dev < 64 && !configured[dev]) {
+                AZ_CUDA(cudaFuncSetAttribute(conv3x3_f32_tiled_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTileSmem));
+                configured[dev] = true;
+            }
         }
         conv3x3_f32_tiled_kernel<<<dim3((unsigned)batch, 2, (unsigned)(cout / kCoutTile)), kTileThreads, kTileSmem, s>>>(
             (const float *)in, (const float *)w, scale, bias, (const float *)residual, (float *)out, cin, cout);

@@ -122,13 +122,14 @@ def test_encoding_is_bit_exact(az, in_planes, precision):
     az.az_free_net(net)
 
 
-@pytest.mark.parametrize("in_planes,channels,batch", [(19, 128, 1301), (112, 256, 701), (112, 128, 1301)])
+@pytest.mark.parametrize("in_planes,channels,batch", [(19, 128, 1301), (112, 256, 701), (112, 128, 1301), (112, 256, 7), (112, 256, 99)])
 def test_encoder_fused_into_the_tower_kernel_is_bit_exact(az, in_planes, channels, batch):
     # az_evaluate never runs the stand-alone encoder on the tensor-core path: the tower kernel's epilogue
     # warps encode each board straight into the shared-memory frame.  A network without blocks whose
     # input convolution is the centre-tap identity (scale one, bias zero) makes the tower's output the
     # planes themselves (they are never negative, so the ReLU is the identity), which shows that copy
-    # bit for bit.  The batch spans more than two rounds of the persistent kernel and ends in a lone board.
+    # bit for bit.  The batch spans more than two rounds of the persistent kernel and ends in a lone board; the two small
+    # batches of the 256-channel shape run on its cluster forms (four and two CTAs per board pair).
     cfg = configs.tiny_config(in_planes=in_planes, blocks=0, channels=channels, policy_head=1, value_head=1,
                               precision=1, batch=batch)
     t = weights.draw_tensors(cfg, 1.0, 1.0)
@@ -293,6 +294,33 @@ def test_tower_activations_bf16_128_channels(az, blocks):
     err = np.abs(got - ref).max() / np.abs(ref).max()
     print(f"tower blocks={blocks}: max-abs error relative to the largest activation {err:.3e}")
     assert err < 2e-2 * (1 + blocks) ** 0.5
+    assert az.az_device_status(net) == 0
+    az.az_free_net(net)
+
+
+@pytest.mark.parametrize("batch", [5, 74, 100, 148, 151])
+@pytest.mark.parametrize("blocks", [0, 2])
+def test_the_three_forms_of_the_256_channel_tower(az, blocks, batch):
+    # up to 74 positions: four CTAs per board pair; up to 148: two; beyond: one.  Each form against the oracle, both
+    # through az_tower (no head layer follows the last convolution: its slices go nowhere but out) and through
+    # az_evaluate (the head projections read the last layer's slices from every CTA's own frame); batches at the edges
+    # of the forms and a lone last board
+    cfg = configs.tiny_config(in_planes=112, blocks=blocks, channels=256, policy_head=1, value_head=1, precision=1,
+                              batch=batch, weight_seed=31 + blocks)
+    blob = weights.make_blob(cfg, 0.5, 0.5)
+    net, _ = load(az, cfg, max_batch=160, blob=blob)
+    rec, _ = positions.generate(777 + batch, batch, (0, 120))
+    recs = positions.records_for_planes(112, rec)
+    mo, _, po, vo, raw = oracle.evaluate(blob, recs, 112, 1, want_tower=True)
+    tower = torch.zeros((batch, 64, 256), dtype=torch.bfloat16, device="cuda")
+    az.az_tower(net, az.records_to_device(recs), batch, tower)
+    torch.cuda.synchronize()
+    got = tower.float().cpu().numpy().transpose(0, 2, 1).reshape(batch, 256, 8, 8)
+    err = np.abs(got - raw["tower"]).max() / np.abs(raw["tower"]).max()
+    print(f"256 channels, blocks={blocks}, batch {batch}: tower max-abs error relative to the largest activation {err:.3e}")
+    assert err < 2e-2 * (1 + blocks) ** 0.5
+    mg, pg, vg = gpu_evaluate(az, net, cfg, recs)
+    compare(cfg, mg, pg, vg, mo, po, vo, TOL[1])
     assert az.az_device_status(net) == 0
     az.az_free_net(net)
 
