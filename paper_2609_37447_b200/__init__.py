@@ -282,8 +282,9 @@ def az_wait_host(net: Net, ticket: int):
     _check(_lib.az_wait_host(net.handle, ticket), "az_wait_host")
 
 
-def az_profile_tower(net: Net, enable: bool):
-    _check(_lib.az_profile_tower(net.handle, 1 if enable else 0), "az_profile_tower")
+def az_profile_tower(net: Net, enable, every: int = 1):
+    """enable False / 0: off; True: every `every`-th evaluation's tower pass is bracketed with events."""
+    _check(_lib.az_profile_tower(net.handle, int(every) if enable else 0), "az_profile_tower")
 
 
 def az_tower_time(net: Net):

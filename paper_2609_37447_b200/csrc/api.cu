@@ -299,7 +299,7 @@ void free_net(Net *n) {
 int run_tower(Net &n, const void *positions, int batch, void **tower_out, bool fused_heads, cudaStream_t s) {
     int rc = AZ_OK;
     const int C = (int)n.arch.channels;
-    const bool timed = n.profile && n.n_events < kMaxProfiledPasses;
+    const bool timed = n.profile > 0 && n.n_events < kMaxProfiledPasses && (++n.profile_count % (unsigned)n.profile) == 0;
     if (n.pnet) {
         // the paper's network: the tower encodes the 52 planes itself, as the other tensor-core towers do
         if (timed) AZ_CUDA(cudaEventRecord(n.ev_begin[n.n_events], s));
@@ -676,7 +676,9 @@ int az_profile_tower(az_net *net, int enable) {
             AZ_CUDA(cudaEventCreate(&n->ev_end[i]));
         }
     }
-    n->profile = enable != 0;
+    if (enable < 0) return AZ_ERR_BAD_ARG;
+    n->profile = enable;
+    n->profile_count = 0;
     return AZ_OK;
 }
 

@@ -129,7 +129,8 @@ struct Net {
     void *pnet_master = nullptr;      // int8 form: the fp32 tower parameters, kept until az_calibrate has quantised them
 
     // ---- optional event timing of the tower ----
-    bool profile = false;
+    int profile = 0;                  // 0: off; k: every k-th tower pass is bracketed with events
+    unsigned profile_count = 0;
     int n_events = 0;                 // pairs recorded since the last read
     cudaEvent_t *ev_begin = nullptr, *ev_end = nullptr;
 };

@@ -145,6 +145,17 @@ def test_tower_event_timing_counts_passes(setup):
     az.az_evaluate(net, pos, masks, 96, pol, val)
     assert az.az_tower_time(net) == (0.0, 0)
     assert az.az_launches_per_evaluate(net, 96) == 3
+    # every third evaluation only (the third, sixth, ... after the call): 7 evaluations, 2 timed; results unchanged
+    az.az_profile_tower(net, True, every=3)
+    for _ in range(7):
+        az.az_evaluate(net, pos, masks, 96, pol, val)
+    ms, passes = az.az_tower_time(net)
+    az.az_profile_tower(net, False)
+    assert passes == 2 and 0.0 < ms < 50.0
+    torch.cuda.synchronize()
+    assert torch.equal(pol, policy) and torch.equal(val, value)
+    with pytest.raises(az.AzError):
+        az.az_profile_tower(net, True, every=-2)
 
 
 def test_a_wait_that_runs_out_is_reported_and_leaves_the_context_usable(setup):
