@@ -483,8 +483,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures on a smaller case)")
     ap.add_argument("--leaves", type=int, default=1, help="search workloads: traversals per tree and step")
-    ap.add_argument("--cta-pairs", action="store_true",
-                    help="load the network with AZ_LOAD_TOWER_CTA_PAIRS (bf16 128-channel residual networks): the tower on clusters of two CTAs")
+    ap.add_argument("--single-ctas", action="store_true",
+                    help="load the network with AZ_LOAD_TOWER_SINGLE_CTAS: the one-CTA tower kernel instead of clusters of two CTAs "
+                         "(the default for bf16 128-channel residual networks), for comparisons")
     ap.add_argument("--legs", default="all", choices=["all", "device"],
                     help="device: only the device-resident timed leg (short runs for profiler captures)")
     ap.add_argument("--moves", type=int, default=0, help="search workloads: also time this many played moves per game, each after "
@@ -524,7 +525,7 @@ def main():
     recs = make_records(cfg, B, first_index=sharding.rank_first_index(rank, B))
     blob = make_blob(cfg)
     arch = az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, B)
-    net = az.az_load_net_ex(arch, blob, az.AZ_LOAD_TOWER_CTA_PAIRS) if args.cta_pairs else az.az_load_net(arch, blob)
+    net = az.az_load_net_ex(arch, blob, az.AZ_LOAD_TOWER_SINGLE_CTAS) if args.single_ctas else az.az_load_net(arch, blob)
     if cfg.precision >= 2:      # 8-bit tower: fix the activation ranges on the seeded calibration positions first
         if is_pnet(cfg):
             cal = positions.generate_moves(cfg.position_seed + configs.CALIBRATION_SEED_OFFSET, configs.CALIBRATION_COUNT, cfg.plies)[0]
@@ -654,7 +655,7 @@ def main():
             "dtype": DTYPE[cfg.precision], "data": "synthetic",
             "config": {"workload": WORKLOADS[cfg.name], "batch_per_gpu": B, "l2": "flushed before every step (256 MB write)",
                        "timing": "CUDA events around each step on the launch stream, summed; max over ranks",
-                       "device_status": status, "tower_cta_pairs": bool(args.cta_pairs)},
+                       "device_status": status, "tower_cta_pairs": bool(not args.single_ctas and cfg.channels == 128 and cfg.precision == 1)},
             "back_to_back": {"value": evals / (b2b_ms * 1e-3), "unit": UNIT, "ms_per_step": b2b_ms / args.steps,
                              "note": "no L2 flush between steps"},
             "gpu_launches": args.steps * az.az_launches_per_evaluate(net, B),

@@ -154,19 +154,20 @@ size_t az_plane_channels(const az_arch *arch);      /* channels of the encoded p
 int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az_net **out);
 
 /*
- * az_load_net with options (az_load_net passes 0):
- *   AZ_LOAD_TOWER_CTA_PAIRS  bf16 residual networks of 128 channels only (AZ_ERR_UNSUPPORTED otherwise): the
- *     tower kernel runs as clusters of two CTAs on neighbouring SMs that share every tensor-core product
- *     (tcgen05 .cta_group::2: 256 rows, 128 from each CTA; each CTA keeps HALF of every weight tile in its own
- *     shared memory and bulk-copies only that half, so the operand traffic of the shared-memory pipe drops from
- *     8 to 6 KB per product and the weight traffic from L2 halves).  The arithmetic and the results are those of
- *     the default kernel, bit for bit.  Measured on B200 (same box, batches of one to four rounds): the same time
- *     per round as the default kernel, which is power-limited, not shared-memory-limited, at this operating
- *     point, and 10 us more per launch; one group per CTA (batch <= 296) runs at half the default's speed.  It is
- *     therefore an option, not the default.
- * Unknown bits: BAD_ARG.
+ * az_load_net with options (az_load_net passes 0).
+ * CTA pairs: the bf16 residual networks of 128 channels run their tower kernel as clusters of two CTAs on
+ * neighbouring SMs that share every tensor-core product (tcgen05 .cta_group::2: 256 rows, 128 from each CTA; each
+ * CTA keeps HALF of every weight tile in its own shared memory and bulk-copies only that half, so the operand
+ * traffic of the shared-memory pipe drops from 8 to 6 KB per product and the weight traffic from L2 halves).  The
+ * arithmetic and the results are those of the one-CTA kernel, bit for bit.  Measured on B200 (same box): 9 to 12 %
+ * less time per evaluation at every batch size from 256 to 4096 (batch 1024: 0.527 -> 0.480 ms), which is why it is
+ * the default for that shape.
+ *   AZ_LOAD_TOWER_CTA_PAIRS    insist on it: AZ_ERR_UNSUPPORTED for a shape that has no such form
+ *   AZ_LOAD_TOWER_SINGLE_CTAS  never: the one-CTA kernel (comparisons, tests)
+ * Both, or unknown bits: BAD_ARG.
  */
 #define AZ_LOAD_TOWER_CTA_PAIRS 1u
+#define AZ_LOAD_TOWER_SINGLE_CTAS 2u
 int az_load_net_ex(const az_arch *arch, const void *weights_host, size_t nbytes, uint32_t flags, az_net **out);
 
 /* Frees the network's device memory.  Null is allowed. */

@@ -211,10 +211,12 @@ def az_load_net(arch: az_arch, weights_host) -> Net:
 
 
 AZ_LOAD_TOWER_CTA_PAIRS = 1
+AZ_LOAD_TOWER_SINGLE_CTAS = 2
 
 
 def az_load_net_ex(arch: az_arch, weights_host, flags=0) -> Net:
-    """az_load_net with options (AZ_LOAD_TOWER_CTA_PAIRS: the tower kernel as clusters of two CTAs)."""
+    """az_load_net with options (AZ_LOAD_TOWER_CTA_PAIRS: insist on the tower kernel as clusters of two CTAs, the
+    default where the shape has that form; AZ_LOAD_TOWER_SINGLE_CTAS: never)."""
     blob = np.ascontiguousarray(np.frombuffer(weights_host, dtype=np.uint8) if isinstance(weights_host, (bytes, bytearray))
                                 else weights_host, dtype=np.uint8)
     out = ctypes.c_void_p()

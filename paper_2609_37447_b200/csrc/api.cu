@@ -403,7 +403,8 @@ int az_load_net_ex(const az_arch *arch, const void *weights_host, size_t nbytes,
     static_assert(sizeof(az_position) == 104 && sizeof(az_position_h8) == 784 && sizeof(az_position_m8) == 128, "record layout");
     if (!arch || !weights_host || !out) return AZ_ERR_BAD_ARG;
     *out = nullptr;
-    if (flags & ~(uint32_t)AZ_LOAD_TOWER_CTA_PAIRS) return AZ_ERR_BAD_ARG;
+    if (flags & ~(uint32_t)(AZ_LOAD_TOWER_CTA_PAIRS | AZ_LOAD_TOWER_SINGLE_CTAS)) return AZ_ERR_BAD_ARG;
+    if ((flags & AZ_LOAD_TOWER_CTA_PAIRS) && (flags & AZ_LOAD_TOWER_SINGLE_CTAS)) return AZ_ERR_BAD_ARG;
     if (!az::arch_ok(*arch)) return AZ_ERR_BAD_ARCH;
     const bool pnet = arch->in_planes == 52;
     if ((flags & AZ_LOAD_TOWER_CTA_PAIRS) && !az::tc_pair_shape((int)arch->channels, (int)arch->precision, pnet)) return AZ_ERR_UNSUPPORTED;
@@ -419,7 +420,7 @@ int az_load_net_ex(const az_arch *arch, const void *weights_host, size_t nbytes,
     Net *n = new (std::nothrow) Net();
     if (!n) return AZ_ERR_BAD_ARG;
     n->arch = *arch;
-    n->want_pair = (flags & AZ_LOAD_TOWER_CTA_PAIRS) != 0;
+    n->want_pair = (flags & AZ_LOAD_TOWER_SINGLE_CTAS) == 0;
     cudaError_t e = cudaGetDevice(&n->device);
     if (e != cudaSuccess) { az::set_cuda_error(e, "cudaGetDevice"); delete n; return AZ_ERR_CUDA; }
     rc = pnet ? az::build_pnet(*n, static_cast<const unsigned char *>(weights_host), nbytes) : az::build_net(*n, view);

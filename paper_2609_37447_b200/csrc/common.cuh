@@ -55,7 +55,7 @@ struct Net {
     void *tc_weights_split4 = nullptr;// and in quarters (four CTAs per group)
     float *tc_bias = nullptr;         // [n_conv][C] folded bias (scales are folded into the weights)
     bool tc_ready = false;
-    bool want_pair = false;           // az_load_net_ex was asked for the CTA-pair form of the tower
+    bool want_pair = true;            // the CTA-pair form of the tower where the shape has one (az_load_net_ex can turn it off)
     bool tc_pair = false;             // the bf16 128-channel tower runs on CTA pairs (tcgen05 .cta_group::2)
     // FP8-e4m3 tower (weights and per-layer constants exist once az_calibrate has run)
     bool fp8 = false, fp8_ready = false;   // 8-bit tower (FP8-e4m3 or int8) and whether it has been calibrated

@@ -407,7 +407,7 @@ tower_tc_kernel(const TowerArgs args) {
                     for (int st = 0; st < n_stages && ok; ++st) {
                         ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status);
                         if (!ok) break;
-                        if (lane == 0) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_peer(stage), 0));
+                        if (lane == 0) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(bar_peer(stage), 0));   // (the copies were written by the bulk-copy engine; this thread publishes nothing of its own)
                         __syncwarp();
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
@@ -464,9 +464,9 @@ tower_tc_kernel(const TowerArgs args) {
                     if (ok && follow) ok = wait_lead(nullptr);
                     if (!ok) break;
                     if (lane == 0) {
-                        if (kPair) {
-                            ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_w_empty(stage), 0));
-                            ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_w_empty(stage), 1));
+                        if (kPair) {      // (relaxed: nothing is published, the slot merely does not need the stage)
+                            ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(bar_w_empty(stage), 0));
+                            ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(bar_w_empty(stage), 1));
                         } else ptx::mbar_arrive(bar_w_empty(stage));
                         if (lead) ptx::mbar_arrive(bar_lead(stage));
                     }
@@ -734,7 +734,10 @@ tower_tc_kernel(const TowerArgs args) {
         // warps).  With the N-split this hands off the CTA's OWN copy of the slice, to its issuer and to the warp that
         // sends it on to the other CTAs.
         auto ready = [&](int kc_) {
-            if (kPair) ptx::mbar_arrive_cluster(ptx::map_to_cta(bar_a_ready(g, kc_), 0));
+            // (pair, second CTA: a relaxed arrival.  Its slice sits in its OWN shared memory, made visible to the async
+            // proxy by the fence before this call, and is read by its own tensor core when the first CTA's product
+            // arrives; a releasing cluster-scope arrival costs the warp about a thousand cycles, eight times a layer.)
+            if (kPair && !leader) ptx::mbar_arrive_cluster_relaxed(ptx::map_to_cta(bar_a_ready(g, kc_), 0));
             else ptx::mbar_arrive(bar_a_ready(g, kc_));
         };
         uint32_t ack_phase = 0;

@@ -621,14 +621,14 @@ def test_work_schedule_is_invisible_in_the_results(az, channels, in_planes):
 
 @pytest.mark.parametrize("name,batches", [("c3", (1024, 301, 5)), ("c2", (256, 3))])
 def test_tower_on_cta_pairs_gives_the_default_kernels_bits(az, name, batches):
-    # az_load_net_ex(AZ_LOAD_TOWER_CTA_PAIRS): the same arithmetic on 256-row tiles shared by two CTAs (each holds
-    # half of every weight tile).  Same products, same accumulation order: outputs equal the default kernel's bit for
-    # bit, through several rounds of the persistent kernel, a ragged last pair and a lone board; the default kernel
-    # is checked against the oracle above, and the first batch here once more.
+    # The default for these networks: the tower on 256-row tiles shared by two CTAs (each holds half of every weight
+    # tile); az_load_net_ex(AZ_LOAD_TOWER_SINGLE_CTAS) gives the one-CTA kernel.  Same products, same accumulation
+    # order: the outputs of the two are equal bit for bit, through several rounds of the persistent kernel, a ragged
+    # last pair and a lone board; both against the oracle on the first batch.
     cfg = configs.CONFIGS[name]
     blob = weights.make_blob(cfg)
     arch = az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, max(batches))
-    net_d, net_p = az.az_load_net(arch, blob), az.az_load_net_ex(arch, blob, az.AZ_LOAD_TOWER_CTA_PAIRS)
+    net_d, net_p = az.az_load_net_ex(arch, blob, az.AZ_LOAD_TOWER_SINGLE_CTAS), az.az_load_net_ex(arch, blob, az.AZ_LOAD_TOWER_CTA_PAIRS)
     recs = positions.cur_records(positions.for_config(cfg, max(batches)))
     for n in batches:
         md, pd, vd = gpu_evaluate(az, net_d, cfg, recs[:n])
@@ -649,11 +649,20 @@ def test_tower_on_cta_pairs_gives_the_default_kernels_bits(az, name, batches):
     assert az.az_device_status(net_d) == 0 and az.az_device_status(net_p) == 0
     az.az_free_net(net_d)
     az.az_free_net(net_p)
-    # other shapes refuse the option instead of ignoring it
+    # the default IS the pair form
+    net_0 = az.az_load_net(arch, blob)
+    _, p0, v0 = gpu_evaluate(az, net_0, cfg, recs[:batches[-1]])
+    assert np.array_equal(p0, pp) and np.array_equal(v0, vp)
+    az.az_free_net(net_0)
+    # other shapes refuse the demand instead of ignoring it; both flags at once make no sense
+    small = weights.make_blob(configs.tiny_config(blocks=1, channels=32, batch=4))
     with pytest.raises(az.AzError) as e:
-        az.az_load_net_ex(az.make_arch(19, 1, 32, 0, 0, 0, 4), weights.make_blob(configs.tiny_config(blocks=1, channels=32, batch=4)),
-                          az.AZ_LOAD_TOWER_CTA_PAIRS)
+        az.az_load_net_ex(az.make_arch(19, 1, 32, 0, 0, 0, 4), small, az.AZ_LOAD_TOWER_CTA_PAIRS)
     assert e.value.code == az.AZ_ERR_UNSUPPORTED
+    with pytest.raises(az.AzError) as e:
+        az.az_load_net_ex(arch, blob, az.AZ_LOAD_TOWER_CTA_PAIRS | az.AZ_LOAD_TOWER_SINGLE_CTAS)
+    assert e.value.code == az.AZ_ERR_BAD_ARG
+    az.az_free_net(az.az_load_net_ex(az.make_arch(19, 1, 32, 0, 0, 0, 4), small, az.AZ_LOAD_TOWER_SINGLE_CTAS))
 
 
 def test_empty_mask_row_gives_zero_policy_and_a_status_flag(az):
