@@ -146,7 +146,11 @@ int build_net(Net &n, const BlobView &v) {
         }
         const size_t bytes = tc_packed_weight_bytes(n.in_pad, C, n.n_conv);
         std::vector<__nv_bfloat16> packed(bytes / sizeof(__nv_bfloat16));
-        n.tc_pair = n.want_pair && tc_pair_shape(C, (int)a.precision, false);
+        // CTA pairs: the bf16 tower of a bf16 network, or the 8-bit tower of an 8-bit one (whose bf16 passes, the
+        // calibration's, stay on single CTAs: their weights are packed whole)
+        const bool pair_shape = n.want_pair && tc_pair_shape(C, (int)a.precision, false);
+        n.tc_pair = pair_shape && a.precision == AZ_PREC_BF16;
+        n.tc_pair8 = pair_shape && a.precision != AZ_PREC_BF16;
         const int halves = n.tc_pair ? 2 : 1;
         tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, halves, 9, false, packed.data());
         AZ_CUDA(cudaMalloc(&n.tc_weights, bytes));
@@ -179,7 +183,7 @@ int build_net(Net &n, const BlobView &v) {
         const int n_policy = flat ? kHeadChannels : kPlanes73, n_policy_pad = flat ? kHeadChannels : 80;
         n.tc_head_n = n_policy_pad + kHeadChannels;
         std::vector<__nv_bfloat16> hw(tc_head_weight_bytes(n.tc_head_n, C) / sizeof(__nv_bfloat16));
-        tc_pack_head(v.p_w, flat ? v.p_s : nullptr, n_policy, n_policy_pad, v.v_cw, v.v_cs, C, halves, hw.data());
+        tc_pack_head(v.p_w, flat ? v.p_s : nullptr, n_policy, n_policy_pad, v.v_cw, v.v_cs, C, (n.tc_pair || n.tc_pair8) ? 2 : 1, hw.data());
         AZ_CUDA(cudaMalloc(&n.tc_head_w, hw.size() * sizeof(__nv_bfloat16)));
         AZ_CUDA(cudaMemcpy(n.tc_head_w, hw.data(), hw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
         std::vector<float> hb(n.tc_head_n, 0.0f);
@@ -770,7 +774,7 @@ int az_calibrate_ex(az_net *net, const void *positions_dev, int count, uint32_t 
         const size_t bytes = az::tc8_packed_weight_bytes(n->in_pad, C, L, n->split_w);
         std::vector<unsigned char> packed(bytes);
         lconst.resize((size_t)L * 3 * C);
-        az::tc8_pack(w.data(), sc.data(), bi.data(), absmax.data(), (int)n->arch.in_planes, n->in_pad, C, L, n->int8, n->split_w, packed.data(), lconst.data());
+        az::tc8_pack(w.data(), sc.data(), bi.data(), absmax.data(), (int)n->arch.in_planes, n->in_pad, C, L, n->int8, n->split_w, n->tc_pair8 ? 2 : 1, packed.data(), lconst.data());
         if (!n->tc8_weights) AZ_CUDA(cudaMalloc(&n->tc8_weights, bytes));
         if (!n->tc8_lconst) AZ_CUDA(cudaMalloc((void **)&n->tc8_lconst, lconst.size() * sizeof(float)));
         AZ_CUDA(cudaMemcpy(n->tc8_weights, packed.data(), bytes, cudaMemcpyHostToDevice));

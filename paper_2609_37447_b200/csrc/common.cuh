@@ -57,6 +57,7 @@ struct Net {
     bool tc_ready = false;
     bool want_pair = true;            // the CTA-pair form of the tower where the shape has one (az_load_net_ex can turn it off)
     bool tc_pair = false;             // the bf16 128-channel tower runs on CTA pairs (tcgen05 .cta_group::2)
+    bool tc_pair8 = false;            // the 8-bit tower of a 128-channel residual network runs on CTA pairs (its bf16 passes, calibration, do not)
     // FP8-e4m3 tower (weights and per-layer constants exist once az_calibrate has run)
     bool fp8 = false, fp8_ready = false;   // 8-bit tower (FP8-e4m3 or int8) and whether it has been calibrated
     bool int8 = false;                      // the 8-bit tower's operands are u8 activations x s8 weights
@@ -215,7 +216,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
                     bool with_heads, unsigned int *absmax, cudaStream_t s);
 size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv, bool split_w);
 void tc8_pack(const float *const *w, const float *const *scale, const float *const *bias, const float *absmax,
-              int in_planes, int in_pad, int channels, int n_conv, bool int8, bool split_w, unsigned char *packed, float *lconst);
+              int in_planes, int in_pad, int channels, int n_conv, bool int8, bool split_w, int halves, unsigned char *packed, float *lconst);
 int tower_tc_launch_count();
 size_t tc_head_weight_bytes(int head_n, int channels);
 void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,

@@ -277,6 +277,33 @@ __device__ __forceinline__ void mma_bf16_elect_pair(uint32_t d_tmem, uint32_t a_
 }
 // the barrier at shared-memory offset `bar` in BOTH CTAs of the pair arrives once all MMAs issued so far by this
 // thread have completed: two plain commits, one per CTA's barrier (shared::cluster addresses)
+// the same for e4m3 operands (kind::f8f6f4) and for unsigned x signed 8-bit integers (kind::i8), K = 32
+__device__ __forceinline__ void mma_e4m3_elect_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                    uint32_t idesc, uint32_t accumulate, uint32_t elected) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 p, %6, 0;\n"
+        "setp.ne.b32 q, %7, 0;\n"
+        "mov.b64 da, {%1, %2};\n"
+        "mov.b64 db, {%3, %4};\n"
+        "@q tcgen05.mma.cta_group::2.kind::f8f6f4 [%0], da, db, %5, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elected));
+}
+__device__ __forceinline__ void mma_i8_elect_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                  uint32_t idesc, uint32_t accumulate, uint32_t elected) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        ".reg .b64 da, db;\n"
+        "setp.ne.b32 p, %6, 0;\n"
+        "setp.ne.b32 q, %7, 0;\n"
+        "mov.b64 da, {%1, %2};\n"
+        "mov.b64 db, {%3, %4};\n"
+        "@q tcgen05.mma.cta_group::2.kind::i8 [%0], da, db, %5, p;\n"
+        "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(elected));
+}
 __device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
     const uint32_t b0 = map_to_cta(bar, 0), b1 = map_to_cta(bar, 1);
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(b0) : "memory");

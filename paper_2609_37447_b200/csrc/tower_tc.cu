@@ -90,7 +90,7 @@ struct Shape {
     static constexpr int kStageTaps = (kC == 256 && NSPLIT == 1) ? 3 : 9;
     static constexpr int kStagesPerSlice = 9 / kStageTaps;
     static constexpr int kStageBytes = kStageTaps * kTileBytes;      // 36864 / 24576; pair: 18432
-    static constexpr int kStages = NSPLIT == 4 ? 6 : NSPLIT > 1 ? 3 : kC == 256 ? 5 : PAIR ? 7 : 3;     // (N-split: 108 KB of 18 / 36 KB stages)
+    static constexpr int kStages = NSPLIT == 4 ? 6 : NSPLIT > 1 ? 3 : kC == 256 ? 5 : PAIR ? (SETS == 2 ? 6 : 7) : 3;     // (N-split: 108 KB of 18 / 36 KB stages)
     // pair: the second group's issuer runs this many weight stages behind the first's (half a layer), so that each
     // group's layer hand-over falls into the middle of the other's layer; the halved stages make the ring deep enough
     static constexpr int kLag = PAIR ? 4 : 0;
@@ -114,7 +114,7 @@ struct Shape {
         return kOffConst + kEpiWarps * (fp8 ? (pnet ? 4 : 3) : 1) * (kC / kSets) * 4 + 256 * 4 + (pnet ? kPoolFloats * 4 : 0);
     }
     // (four constant vectors per channel in the 8-bit forms, one in bf16; the 176-channel shape exists in bf16 only)
-    static_assert(kOffConst + kEpiWarps * ((kC == 176 || PAIR) ? 1 : 4) * (kC / kSets) * 4 + 1024 + (PAIR ? 0 : kPoolFloats * 4) <= kMaxSmem || kC == 256, "shared memory budget");
+    static_assert(kOffConst + kEpiWarps * ((kC == 176 || (PAIR && SETS == 1)) ? 1 : 4) * (kC / kSets) * 4 + 1024 + (PAIR ? 0 : kPoolFloats * 4) <= kMaxSmem || kC == 256, "shared memory budget");
     static_assert(kGroups * 2 * kN <= (int)kTmemCols, "TMEM: per group N columns of residual stream and N of accumulator");
 };
 
@@ -257,7 +257,7 @@ tower_tc_kernel(const TowerArgs args) {
     auto bar_pdone = [&](int g) { return bar_done + 8u * (1 + kStages + kGroups + kStages + g); };   // N-split: the other CTAs' MMAs of this layer are complete
     auto bar_ack = [&](int g) { return bar_done + 8u * (1 + kStages + kGroups + kStages + kGroups + g); };   // N-split: the other CTAs hold this CTA's slices of the layer
     constexpr bool kPair = S::kPair;
-    static_assert(!kPair || (!kFp8 && !kPnet && kGroups == 2), "CTA pairs exist for the two-group bf16 shape of the residual networks");
+    static_assert(!kPair || (!kPnet && kGroups == 2), "CTA pairs exist for the two-group shapes of the residual networks");
     constexpr int kNSplit = S::kNSplit, kN = S::kN;
     constexpr bool kCluster = kPair || kNSplit > 1;
     static_assert(kNSplit == 1 || (!kFp8 && !kPnet && kGroups == 1 && S::kSets == 1), "the N-split exists for the one-group bf16 shape of the residual networks");
@@ -427,7 +427,7 @@ tower_tc_kernel(const TowerArgs args) {
         };
         // barrier(s) that arrive when the MMAs issued so far have completed: this CTA's, in a pair both CTAs'
         auto commit = [&](uint32_t bar_) { if (kPair) ptx::mma_commit_pair(bar_); else ptx::mma_commit(bar_); };
-        constexpr uint32_t idesc8 = kInt8 ? ptx::idesc_u8s8_s32(128, kC) : ptx::idesc_e4m3_f32(128, kC);
+        constexpr uint32_t idesc8 = kInt8 ? ptx::idesc_u8s8_s32(128 * S::kHalves, kN) : ptx::idesc_e4m3_f32(128 * S::kHalves, kN);
         int stage = 0;
         uint32_t phase = 0;
         uint32_t a_phase = 0;
@@ -523,17 +523,20 @@ tower_tc_kernel(const TowerArgs args) {
                                     const int tap = st * S::kStageTaps + t;
                                     const int dy = tap / 3 - 1, dx = tap % 3 - 1;
                                     const uint32_t first = (tap == 0 && !conv2 && ki == 0 && part == 0) ? 0u : 1u;
-                                    if (kInt8)
-                                        ptx::mma_i8_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                          b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8, first, elected);
-                                    else
-                                        ptx::mma_e4m3_elect(d, a_lo + (uint32_t)(dy * kNB * 9 + dx), kADescHi,
-                                                            b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8, first, elected);
+                                    const uint32_t a_t = a_lo + (uint32_t)(dy * kNB * 9 + dx), b_t = b_lo + (uint32_t)(t * (S::kTileBytes / 16));
+                                    if (kInt8) {
+                                        if (kPair) ptx::mma_i8_elect_pair(d, a_t, kADescHi, b_t, kBDescHi, idesc8, first, elected);
+                                        else ptx::mma_i8_elect(d, a_t, kADescHi, b_t, kBDescHi, idesc8, first, elected);
+                                    } else {
+                                        if (kPair) ptx::mma_e4m3_elect_pair(d, a_t, kADescHi, b_t, kBDescHi, idesc8, first, elected);
+                                        else ptx::mma_e4m3_elect(d, a_t, kADescHi, b_t, kBDescHi, idesc8, first, elected);
+                                    }
                                     // the activations' remainders against the same weights (first parts of the weights only:
                                     // remainder times remainder is below what fp32 accumulation keeps anyway)
-                                    if (kSplitA && part == 0)
-                                        ptx::mma_e4m3_elect(d, a_lo + (uint32_t)((kC / 16) * kSlots + dy * kNB * 9 + dx), kADescHi,
-                                                            b_lo + (uint32_t)(t * (S::kTileBytes / 16)), kBDescHi, idesc8, 1u, elected);
+                                    if (kSplitA && part == 0) {
+                                        if (kPair) ptx::mma_e4m3_elect_pair(d, a_t + (uint32_t)((kC / 16) * kSlots), kADescHi, b_t, kBDescHi, idesc8, 1u, elected);
+                                        else ptx::mma_e4m3_elect(d, a_t + (uint32_t)((kC / 16) * kSlots), kADescHi, b_t, kBDescHi, idesc8, 1u, elected);
+                                    }
                                 }
                             } else {
 #pragma unroll
@@ -1197,6 +1200,7 @@ typedef Shape<128, 2, AZ_C128_SETS, true> Shape128Pair;    // the bf16 residual 
 #define AZ_FP8_EPI_SETS 2
 #endif
 typedef Shape<128, 2, AZ_FP8_EPI_SETS> Shape128F8;
+typedef Shape<128, 2, AZ_FP8_EPI_SETS, true> Shape128F8Pair;   // the 8-bit towers on CTA pairs
 typedef Shape<256, 1, 1> Shape256;
 typedef Shape<256, 1, 1, false, 2> Shape256Split2;      // small batches: two CTAs per group, 128 output channels each
 typedef Shape<256, 1, 1, false, 4> Shape256Split4;      // smaller still: four CTAs per group, 64 output channels each
@@ -1250,7 +1254,7 @@ void tc_pack_weights(const float *const *w, const float *const *scale, int in_pl
                                     }
     }
 }
-bool tc_pair_shape(int channels, int precision, bool pnet) { return channels == 128 && precision == AZ_PREC_BF16 && !pnet; }
+bool tc_pair_shape(int channels, int precision, bool pnet) { return channels == 128 && precision != AZ_PREC_FP32 && !pnet; }
 
 // The same tiles for a tower whose layers read different numbers of input channels (the paper's
 // network: 52 planes padded to 64 into the input layer, 3C/4 channels into the second convolution
@@ -1315,15 +1319,16 @@ size_t tc8_packed_weight_bytes(int in_pad, int channels, int n_conv, bool split_
 // round to nearest; same constants, same layout.
 // split_w (e4m3 only): every weight as a pair, q_w = e4m3(W' / ws) and e4m3(W' / ws - q_w); per 32-channel slice
 // the stage of first parts is followed by a stage of remainders.
+// halves == 2 (CTA pairs): every stage as rows [0, C/2) of its nine taps, then rows [C/2, C), as in tc_pack_weights.
 void tc8_pack(const float *const *w, const float *const *scale, const float *const *bias, const float *absmax,
-              int in_planes, int in_pad, int channels, int n_conv, bool int8, bool split_w, unsigned char *packed, float *lconst) {
+              int in_planes, int in_pad, int channels, int n_conv, bool int8, bool split_w, int halves, unsigned char *packed, float *lconst) {
     const int C = channels;
     const float kMax = int8 ? 255.0f : 448.0f, kMaxW = int8 ? 127.0f : 448.0f, kTiny = 1e-30f;
     std::vector<float> sa((size_t)n_conv * C, 1.0f), ws((size_t)n_conv * C, 1.0f);
     for (int l = 1; l < n_conv; ++l)
         for (int c = 0; c < C; ++c) sa[(size_t)l * C + c] = fmaxf(absmax[(size_t)(l - 1) * C + c], kTiny) / kMax;
     // layer 0: bf16 tiles exactly as in the bf16 tower
-    tc_pack_weights(w, scale, in_planes, in_pad, C, 1, 1, 9, false, reinterpret_cast<__nv_bfloat16 *>(packed));
+    tc_pack_weights(w, scale, in_planes, in_pad, C, 1, halves, 9, false, reinterpret_cast<__nv_bfloat16 *>(packed));
     unsigned char *dst = packed + (size_t)(in_pad / 16) * kStageBytes;
     std::vector<float> wf((size_t)C * C * 9);
     for (int l = 1; l < n_conv; ++l) {
@@ -1339,9 +1344,10 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
         }
         for (int kc = 0; kc < C / 32; ++kc)
             for (int part = 0; part < (split_w ? 2 : 1); ++part)
+              for (int h = 0; h < halves; ++h)
                 for (int tap = 0; tap < 9; ++tap)
                     for (int k16 = 0; k16 < 2; ++k16)
-                        for (int ng = 0; ng < C / 8; ++ng)
+                        for (int ng = h * (C / 8 / halves); ng < (h + 1) * (C / 8 / halves); ++ng)
                             for (int r = 0; r < 8; ++r)
                                 for (int e = 0; e < 16; ++e) {
                                     const int n = ng * 8 + r, ci = kc * 32 + k16 * 16 + e;
@@ -1413,6 +1419,9 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8Pair>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8Pair, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8Pair, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256Split2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256Split4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
@@ -1480,6 +1489,21 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         return AZ_OK;
     }
     else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);
+    else if (fp8 && net.tc_pair8) {
+        // the 8-bit towers on clusters of two CTAs; a pair takes pairs of groups
+        const int n_super = (n_groups + 1) / 2, pairs = n_super < sms / 2 ? n_super : sms / 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(Shape128F8Pair::kThreads);
+        cfg.dynamicSmemBytes = Shape128F8Pair::smem_bytes(true); cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        if (net.int8) AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<true, Shape128F8Pair, false, true>, a));
+        else if (net.split_a) AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<true, Shape128F8Pair, false, false, true>, a));
+        else AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<true, Shape128F8Pair>, a));
+        return AZ_OK;
+    }
     else if (fp8 && net.int8) tower_tc_kernel<true, Shape128F8, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else if (fp8 && net.split_a) tower_tc_kernel<true, Shape128F8, false, false, true><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);
     else if (fp8) tower_tc_kernel<true, Shape128F8><<<grid, Shape128F8::kThreads, Shape128F8::smem_bytes(true), s>>>(a);

@@ -665,6 +665,29 @@ def test_tower_on_cta_pairs_gives_the_default_kernels_bits(az, name, batches):
     az.az_free_net(az.az_load_net_ex(az.make_arch(19, 1, 32, 0, 0, 0, 4), small, az.AZ_LOAD_TOWER_SINGLE_CTAS))
 
 
+@pytest.mark.parametrize("name", ["c4", "c4i", "c4x"])
+def test_8_bit_towers_on_cta_pairs_give_the_single_cta_kernels_bits(az, name):
+    # the e4m3, int8 and e4m3-operand-pair towers run on CTA pairs by default as well; same products in the same
+    # order, same calibration: results equal the one-CTA kernels' bit for bit (several rounds, a ragged end)
+    cfg = configs.CONFIGS[name]
+    blob = weights.make_blob(cfg)
+    batch = 1203
+    arch = az.make_arch(cfg.in_planes, cfg.blocks, cfg.channels, cfg.policy_head, cfg.value_head, cfg.precision, batch)
+    recs = positions.cur_records(positions.for_config(cfg, batch))
+    cal = positions.cur_records(positions.for_config(cfg, calibration=True))
+    results = []
+    for flags in (az.AZ_LOAD_TOWER_SINGLE_CTAS, az.AZ_LOAD_TOWER_CTA_PAIRS, 0):
+        net = az.az_load_net_ex(arch, blob, flags)
+        az.az_calibrate(net, az.records_to_device(cal), cal.shape[0])
+        out = [gpu_evaluate(az, net, cfg, recs[:n])[1:] for n in (batch, 7)]
+        assert az.az_device_status(net) == 0
+        az.az_free_net(net)
+        results.append(out)
+    for other in results[1:]:
+        for (p0, v0), (p1, v1) in zip(results[0], other):
+            assert np.array_equal(p0, p1) and np.array_equal(v0, v1)
+
+
 def test_empty_mask_row_gives_zero_policy_and_a_status_flag(az):
     cfg = configs.tiny_config(blocks=1, channels=32, batch=4)
     net, blob = load(az, cfg, max_batch=8)
