@@ -46,14 +46,14 @@ struct Small {
 };
 
 // (Both operands of these two products come from the tower kernel, which may still be running when this kernel starts
-// (programmatic dependent launch): they are read after the dependency wait and NOT through the read-only path, whose
-// loads the compiler may move ahead of the wait.)
+// (programmatic dependent launch): they are read after the dependency wait with ordinary cached loads, NOT through the
+// read-only path, whose loads the compiler may move ahead of the wait.  Cached in L1: a row is read once per move.)
 __device__ __forceinline__ float dot128_f32(const float *a, const float *b) {
     const float4 *pa = reinterpret_cast<const float4 *>(a), *pb = reinterpret_cast<const float4 *>(b);
     float acc = 0.0f;
 #pragma unroll 8
     for (int i = 0; i < 32; ++i) {
-        const float4 x = __ldcg(pa + i), y = __ldcg(pb + i);
+        const float4 x = __ldca(pa + i), y = __ldca(pb + i);
         acc = fmaf(x.x, y.x, acc); acc = fmaf(x.y, y.y, acc);
         acc = fmaf(x.z, y.z, acc); acc = fmaf(x.w, y.w, acc);
     }
@@ -65,7 +65,7 @@ __device__ __forceinline__ float dot_f32_bf16(const float *w, const __nv_bfloat1
     float acc = 0.0f;
 #pragma unroll 4
     for (int i = 0; i < n / 8; ++i) {
-        const uint4 y = __ldcg(ph + i);
+        const uint4 y = __ldca(ph + i);
         const uint32_t ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
