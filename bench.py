@@ -483,6 +483,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (profiling captures on a smaller case)")
     ap.add_argument("--leaves", type=int, default=1, help="search workloads: traversals per tree and step")
+    ap.add_argument("--tower-timing-every", type=int, default=4,
+                    help="the library's events around the tower kernel (roofline) on every n-th timed step (they cost the step its "
+                         "dependent launch's overlap); 1 with fewer than 8 steps")
     ap.add_argument("--single-ctas", action="store_true",
                     help="load the network with AZ_LOAD_TOWER_SINGLE_CTAS: the one-CTA tower kernel instead of clusters of two CTAs "
                          "(the default for bf16 128-channel residual networks), for comparisons")
@@ -551,7 +554,7 @@ def main():
     torch.cuda.synchronize()
     # the tower's own duration (roofline) is taken on every fourth step: the library's events between the tower's
     # launch and the head kernel's cost an evaluation the overlap of its dependent launch (about 9 us at batch 1024)
-    timed_every = 4 if args.steps >= 8 else 1
+    timed_every = max(1, args.tower_timing_every) if args.steps >= 8 else 1
     az.az_profile_tower(net, True, every=timed_every)
     az.az_tower_time(net)
     starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]

@@ -46,14 +46,15 @@ struct Small {
 };
 
 // (Both operands of these two products come from the tower kernel, which may still be running when this kernel starts
-// (programmatic dependent launch): they are read after the dependency wait with ordinary cached loads, NOT through the
-// read-only path, whose loads the compiler may move ahead of the wait.  Cached in L1: a row is read once per move.)
+// (programmatic dependent launch).  They are read through the read-only path, whose hit rate these products need (a
+// row is read once per legal move), but such loads the compiler may move ahead of the dependency wait: the kernel
+// therefore takes their base pointers through an opaque assembly statement placed AFTER the wait.)
 __device__ __forceinline__ float dot128_f32(const float *a, const float *b) {
     const float4 *pa = reinterpret_cast<const float4 *>(a), *pb = reinterpret_cast<const float4 *>(b);
     float acc = 0.0f;
 #pragma unroll 8
     for (int i = 0; i < 32; ++i) {
-        const float4 x = __ldca(pa + i), y = __ldca(pb + i);
+        const float4 x = __ldg(pa + i), y = __ldg(pb + i);
         acc = fmaf(x.x, y.x, acc); acc = fmaf(x.y, y.y, acc);
         acc = fmaf(x.z, y.z, acc); acc = fmaf(x.w, y.w, acc);
     }
@@ -65,7 +66,7 @@ __device__ __forceinline__ float dot_f32_bf16(const float *w, const __nv_bfloat1
     float acc = 0.0f;
 #pragma unroll 4
     for (int i = 0; i < n / 8; ++i) {
-        const uint4 y = __ldca(ph + i);
+        const uint4 y = __ldg(ph + i);
         const uint32_t ys[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -125,9 +126,10 @@ pnet_finish_kernel(const __nv_bfloat16 *__restrict__ h, const float *__restrict_
             bits &= bits - 1;
         }
     }
-    ptx::grid_dependency_wait();                     // from here on the tower's outputs are read
+    ptx::grid_dependency_wait();                     // (no effect in an ordinary launch; kept should the launch become a dependent one)
     const __nv_bfloat16 *hp = h + (size_t)pos * 64 * C;
     const float *qkp = qk + (size_t)pos * 64 * 256;
+    asm volatile("" : "+l"(hp), "+l"(qkp) : : "memory");   // no load through these pointers can be scheduled above the wait
 
     // ---- value head
     {
@@ -474,10 +476,13 @@ int build_pnet(Net &n, const unsigned char *blob, size_t nbytes) {
 int launch_pnet_finish(const Net &n, const uint64_t *masks, int batch, float *policy, float *legal, int *counts,
                        float *value, cudaStream_t s) {
     if (batch == 0) return AZ_OK;
-    AZ_CUDA(launch_dependent(pnet_finish_kernel, dim3((unsigned)batch), dim3(kFinishThreads), 0, s,
-                             static_cast<const __nv_bfloat16 *>(n.act[0]), static_cast<const float *>(n.pnet_qk), masks,
-                             static_cast<const float *>(n.pnet_small), reinterpret_cast<const uchar4 *>(n.pnet_actions), batch,
-                             (int)n.arch.channels, policy, legal, counts, value, n.status_dev));
+    // an ordinary launch, not a dependent one: started early, this kernel's many small CTAs pile onto the SMs that the
+    // tower's last round leaves idle first and then do all their work from there (batch 1024: 10 us slower, measured)
+    pnet_finish_kernel<<<dim3((unsigned)batch), dim3(kFinishThreads), 0, s>>>(
+        static_cast<const __nv_bfloat16 *>(n.act[0]), static_cast<const float *>(n.pnet_qk), masks,
+        static_cast<const float *>(n.pnet_small), reinterpret_cast<const uchar4 *>(n.pnet_actions), batch,
+        (int)n.arch.channels, policy, legal, counts, value, n.status_dev);
+    AZ_LAUNCH_CHECK();
     return AZ_OK;
 }
 
