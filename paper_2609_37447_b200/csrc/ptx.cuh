@@ -198,8 +198,8 @@ __device__ __forceinline__ uint32_t cvt_u8_sat(float v) {
 // tcgen05 with .cta_group::2: the MMA is issued by one thread of the pair's first CTA; each CTA supplies its own 128
 // rows of A and its own HALF of the B tile (N/2 rows) from its own shared memory, at the same offsets in both, and
 // receives its 128 rows of D in its own TMEM.  Every B byte is read from shared memory once per pair instead of
-// once per CTA.  Nothing here is a multicast: each CTA bulk-copies its own half of every weight stage, and
-// completion is signalled to each CTA's barrier by a commit of its own.
+// once per CTA.  No copy and no commit here addresses more than one CTA: each CTA bulk-copies its own half of every
+// weight stage, and completion is signalled to each CTA's barrier by a commit of its own.
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
