@@ -311,9 +311,8 @@ tower_tc_kernel(const TowerArgs args) {
     }
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_ptr_smem;
-    // the head GEMM kernel may set itself up on idle SMs; it waits for this grid before reading.  (The finishing kernel
-    // of the paper's network is an ordinary launch.)
-    if (!kPnet) ptx::launch_dependents();
+    // the head kernel that follows may set itself up on idle SMs; it waits for this grid before reading
+    ptx::launch_dependents();
 
     // pair: the schedule deals out PAIRS of groups (four boards) to pairs of CTAs; the CTA of rank r takes the r-th
     // group of each (a group beyond the batch runs on dead boards and writes nothing)
