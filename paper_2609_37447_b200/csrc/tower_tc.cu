@@ -93,7 +93,10 @@ struct Shape {
     static constexpr int kStages = NSPLIT == 4 ? 6 : NSPLIT > 1 ? 3 : kC == 256 ? 5 : PAIR ? (SETS == 2 ? 6 : 7) : 3;     // (N-split: 108 KB of 18 / 36 KB stages)
     // pair: the second group's issuer runs this many weight stages behind the first's (half a layer), so that each
     // group's layer hand-over falls into the middle of the other's layer; the halved stages make the ring deep enough
-    static constexpr int kLag = PAIR ? 4 : 0;
+#ifndef AZ_PAIR_LAG
+#define AZ_PAIR_LAG 4
+#endif
+    static constexpr int kLag = PAIR ? AZ_PAIR_LAG : 0;
     static constexpr int kEpiWarps = 4 * kGroups * kSets;
     static constexpr int kThreads = 32 * (1 + kGroups + kEpiWarps + (NSPLIT > 1 ? 2 : 0));  // producer, one issuer per group, 4 epilogue warps per group and set; N-split: a warp that sends the finished slices to the other CTAs and one that acknowledges theirs
     static constexpr uint32_t kBDescLbo = (uint32_t)(kC / kParts) << 16;    // K core matrices (rows of this CTA's tile)*16 bytes apart
