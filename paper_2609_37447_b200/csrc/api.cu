@@ -191,14 +191,14 @@ int build_net(Net &n, const BlobView &v) {
         for (int i = 0; i < kHeadChannels; ++i) hb[n_policy_pad + i] = v.v_cb[i];
         if ((rc = upload_f32(hb.data(), hb.size(), &n.tc_head_bias)) != AZ_OK) return rc;
         {
-            std::vector<__nv_bfloat16> fw(fc_tc_weight_bytes(kValueHidden) / sizeof(__nv_bfloat16));
-            fc_tc_pack_weights(v.v_w1, kValueHidden, fw.data());
+            std::vector<__nv_bfloat16> fw(fc_tc_weight_bytes(kValueHidden, false) / sizeof(__nv_bfloat16));
+            fc_tc_pack_weights(v.v_w1, kValueHidden, false, fw.data());
             AZ_CUDA(cudaMalloc(&n.fc_value_w, fw.size() * sizeof(__nv_bfloat16)));
             AZ_CUDA(cudaMemcpy(n.fc_value_w, fw.data(), fw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
         }
         if (flat) {
-            std::vector<__nv_bfloat16> fw(fc_tc_weight_bytes(kFlatMoves) / sizeof(__nv_bfloat16));
-            fc_tc_pack_weights(v.p_fw, kFlatMoves, fw.data());
+            std::vector<__nv_bfloat16> fw(fc_tc_weight_bytes(kFlatMoves, true) / sizeof(__nv_bfloat16));
+            fc_tc_pack_weights(v.p_fw, kFlatMoves, true, fw.data());
             AZ_CUDA(cudaMalloc(&n.fc_policy_w, fw.size() * sizeof(__nv_bfloat16)));
             AZ_CUDA(cudaMemcpy(n.fc_policy_w, fw.data(), fw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
         }

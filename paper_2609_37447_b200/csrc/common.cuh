@@ -223,8 +223,8 @@ void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_p
                   int channels, int halves, __nv_bfloat16 *packed);
 
 // tensor-core fully-connected layers of the heads (fc_tc.cu)
-size_t fc_tc_weight_bytes(int n);
-void fc_tc_pack_weights(const float *w, int n, __nv_bfloat16 *packed);     // w[n][32*64], K permuted to square*32 + channel
+size_t fc_tc_weight_bytes(int n, bool policy);
+void fc_tc_pack_weights(const float *w, int n, bool policy, __nv_bfloat16 *packed);     // w[n][32*64], K permuted to square*32 + channel; policy: the tile height of the head GEMM's CTA pairs
 int launch_fc_tc(const Net &net, int batch, float *value_out, cudaStream_t s);
 
 }  // namespace az

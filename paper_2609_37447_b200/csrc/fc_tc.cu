@@ -35,9 +35,15 @@ constexpr int kNumKStages = kK / kStageK;      // 32
 constexpr int kOperandStageBytes = 128 * kStageK * 2;   // 16384
 constexpr int kStages = 5;
 constexpr int kThreads = 32 * 6;               // producer, issuer, 4 epilogue warps
+#ifndef AZ_FC_PAIR_COLS
+#define AZ_FC_PAIR_COLS 256
+#endif
+constexpr int kPairCols = AZ_FC_PAIR_COLS;       // columns of a pair's output tile (256 or 128)
+constexpr int kPairRows = kPairCols / 2;        // weight rows a CTA of a pair holds per stage
+constexpr int kPairBStageBytes = kPairRows * kStageK * 2;
 constexpr uint32_t kTmemCols = 256;
 constexpr uint32_t kSpinLimit = 1u << 24;
-constexpr int kLogitPitch = 257;                // floats per row of the logits tile staged in shared memory
+constexpr int kLogitPitch = kPairCols + 1;       // floats per row of the logits tile staged in shared memory
 
 static_assert(128 * kLogitPitch * 4 <= 2 * kStages * kOperandStageBytes, "the logits tile is staged in the operand stages");
 constexpr int kOffA = 0;
@@ -56,7 +62,7 @@ struct FcArgs {
     float *logits;                              // [batch][1858]
     float *value;                               // [batch][V]
     uint32_t *status;
-    int batch, n_policy, n_policy_tiles, wdl;   // n_policy_tiles: tiles of 256 columns
+    int batch, n_policy, n_policy_tiles, wdl;   // n_policy_tiles: tiles of kPairCols columns
 };
 
 __device__ __forceinline__ bool wait_bar(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t *status) {
@@ -121,11 +127,12 @@ fc_tc_kernel(const FcArgs args) {
         // ---- producer: two 16 KB bulk copies per stage: this CTA's 128 rows of A, and 128 rows of B (pair: the weight
         // rows of this CTA's half of the 256 columns)
         const int a_tile = tile_live ? m_tile : 0;
-        const int b_tile = is_value ? 0 : 2 * (int)blockIdx.y + (int)rank;
+        const int b_tile = is_value ? 0 : 2 * (int)blockIdx.y + (int)rank;      // (the policy's tiles: kPairRows rows each)
+        const uint32_t b_bytes = is_value ? (uint32_t)kOperandStageBytes : (uint32_t)kPairBStageBytes;
         const unsigned char *a_src = reinterpret_cast<const unsigned char *>(is_value ? args.u_value : args.u_policy) +
                                      (size_t)a_tile * (kK * 128 * 2);
         const unsigned char *b_src = reinterpret_cast<const unsigned char *>(is_value ? args.w_value : args.w_policy) +
-                                     (size_t)b_tile * (kK * 128 * 2);
+                                     (size_t)b_tile * ((size_t)kK * (is_value ? 128 : kPairRows) * 2);
         bool ok = true;
         int issued = 0;
         for (int ks = 0; ks < kNumKStages; ++ks) {
@@ -133,9 +140,9 @@ fc_tc_kernel(const FcArgs args) {
             ok = wait_bar(bar_empty(s), ((ks / kStages) & 1) ^ 1u, abort_flag, args.status);
             if (!ok) break;
             if (lane == 0) {
-                ptx::mbar_arrive_expect_tx(bar_full(s), 2 * kOperandStageBytes);
+                ptx::mbar_arrive_expect_tx(bar_full(s), (uint32_t)kOperandStageBytes + b_bytes);
                 ptx::bulk_copy_g2s(smem_base + kOffA + s * kOperandStageBytes, a_src + (size_t)ks * kOperandStageBytes, kOperandStageBytes, bar_full(s));
-                ptx::bulk_copy_g2s(smem_base + kOffB + s * kOperandStageBytes, b_src + (size_t)ks * kOperandStageBytes, kOperandStageBytes, bar_full(s));
+                ptx::bulk_copy_g2s(smem_base + kOffB + s * kOperandStageBytes, b_src + (size_t)ks * b_bytes, b_bytes, bar_full(s));
             }
             issued = ks + 1;
             __syncwarp();
@@ -159,7 +166,8 @@ fc_tc_kernel(const FcArgs args) {
         }
     } else if (warp == 1) {
         // ---- MMA issuer: four K=16 steps per stage
-        constexpr uint32_t idesc_solo = ptx::idesc_bf16_f32(128, 128), idesc_pair = ptx::idesc_bf16_f32(256, 256);
+        constexpr uint32_t idesc_solo = ptx::idesc_bf16_f32(128, 128), idesc_pair = ptx::idesc_bf16_f32(256, kPairCols);
+        constexpr uint32_t lbo_pair = (uint32_t)(kPairRows * 16 >> 4) << 16;   // the pair's B: K core matrices kPairRows x 16 bytes apart
         constexpr uint32_t desc_hi = (uint32_t)(128 >> 4) | (1u << 14);        // 8-row groups 128 B apart
         constexpr uint32_t lbo = (uint32_t)(2048 >> 4) << 16;                  // K core matrices 2048 B apart
         const uint32_t elected = ptx::elect_one();
@@ -171,11 +179,11 @@ fc_tc_kernel(const FcArgs args) {
             if (!ok) break;
             ptx::tc_fence_after();
             const uint32_t a_lo = (desc_base + (uint32_t)((kOffA + s * kOperandStageBytes) >> 4)) | lbo;
-            const uint32_t b_lo = (desc_base + (uint32_t)((kOffB + s * kOperandStageBytes) >> 4)) | lbo;
+            const uint32_t b_lo = (desc_base + (uint32_t)((kOffB + s * kOperandStageBytes) >> 4)) | (pair ? lbo_pair : lbo);
             if (pair) {
 #pragma unroll
                 for (int j = 0; j < kStageK / 16; ++j)
-                    ptx::mma_bf16_elect_pair(tmem_base, a_lo + (uint32_t)(j * 256), desc_hi, b_lo + (uint32_t)(j * 256), desc_hi, idesc_pair,
+                    ptx::mma_bf16_elect_pair(tmem_base, a_lo + (uint32_t)(j * 256), desc_hi, b_lo + (uint32_t)(j * 2 * kPairRows), desc_hi, idesc_pair,
                                              (ks > 0 || j > 0) ? 1u : 0u, elected);
             } else {
 #pragma unroll
@@ -202,7 +210,7 @@ fc_tc_kernel(const FcArgs args) {
         ptx::tc_fence_after();
         float z[3] = {0.0f, 0.0f, 0.0f};
         if (ok) {
-            const int n_chunks = is_value ? 8 : 16;
+            const int n_chunks = is_value ? 8 : kPairCols / 16;
 #pragma unroll 1
             for (int j = 0; j < n_chunks; ++j) {
                 uint32_t r[16];
@@ -232,17 +240,17 @@ fc_tc_kernel(const FcArgs args) {
         if (ok) {
             if (!is_value) {
                 const float *stage = reinterpret_cast<const float *>(smem);
-                const int n0 = (int)blockIdx.y * 256 + lane;
-                float bias[8];
+                const int n0 = (int)blockIdx.y * kPairCols + lane;
+                float bias[kPairCols / 32];
 #pragma unroll
-                for (int k = 0; k < 8; ++k) bias[k] = n0 + 32 * k < args.n_policy ? __ldg(args.b_policy + n0 + 32 * k) : 0.0f;
+                for (int k = 0; k < kPairCols / 32; ++k) bias[k] = n0 + 32 * k < args.n_policy ? __ldg(args.b_policy + n0 + 32 * k) : 0.0f;
                 // warp q writes rows q, q + 4, ...: a store instruction covers 32 consecutive logits of one row
                 for (int rr = q; rr < 128; rr += 4) {
                     const int mm = m_tile * 128 + rr;
                     if (!tile_live || mm >= args.batch) break;
                     float *dst = args.logits + (size_t)mm * args.n_policy;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k)
+                    for (int k = 0; k < kPairCols / 32; ++k)
                         if (n0 + 32 * k < args.n_policy) dst[n0 + 32 * k] = stage[rr * kLogitPitch + lane + 32 * k] + bias[k];
                 }
             }
@@ -276,25 +284,25 @@ fc_tc_kernel(const FcArgs args) {
 
 }  // namespace
 
-// bytes of the packed weight tiles of an n-row matrix; the policy's tiles come in pairs (a 256-column tile is two), so
-// an odd count is rounded up with a tile of zeros
-size_t fc_tc_weight_bytes(int n) {
-    int tiles = (n + 127) / 128;
-    if (tiles > 1) tiles = (tiles + 1) & ~1;
-    return (size_t)tiles * kK * 128 * 2;
+// bytes of the packed weight tiles of an n-row matrix.  The value head's hidden layer is one tile of 128 rows; the
+// policy's tiles have kPairRows rows (what one CTA of a pair holds of a kPairCols-column tile), an even number of them
+size_t fc_tc_weight_bytes(int n, bool policy) {
+    if (!policy) return (size_t)((n + 127) / 128) * kK * 128 * 2;
+    return (size_t)(2 * ((n + kPairCols - 1) / kPairCols)) * kK * kPairRows * 2;
 }
 
-// w[n][2048] with the input flattened channel-major (channel*64 + square)  ->  128-row tiles
-// [tile][8-wide K chunk (256)][row group (16)][row (8)][k (8)] with K = square*32 + channel.
-void fc_tc_pack_weights(const float *w, int n, __nv_bfloat16 *packed) {
-    const int tiles = (int)(fc_tc_weight_bytes(n) / ((size_t)kK * 128 * 2));
+// w[n][2048] with the input flattened channel-major (channel*64 + square)  ->  tiles of `rows` rows
+// [tile][8-wide K chunk (256)][row group (rows/8)][row (8)][k (8)] with K = square*32 + channel.
+void fc_tc_pack_weights(const float *w, int n, bool policy, __nv_bfloat16 *packed) {
+    const int rows = policy ? kPairRows : 128;
+    const int tiles = (int)(fc_tc_weight_bytes(n, policy) / ((size_t)kK * rows * 2));
     __nv_bfloat16 *dst = packed;
     for (int t = 0; t < tiles; ++t)
         for (int kc8 = 0; kc8 < kK / 8; ++kc8)
-            for (int ng = 0; ng < 16; ++ng)
+            for (int ng = 0; ng < rows / 8; ++ng)
                 for (int r = 0; r < 8; ++r)
                     for (int e = 0; e < 8; ++e) {
-                        const int row = t * 128 + ng * 8 + r, k = kc8 * 8 + e;
+                        const int row = t * rows + ng * 8 + r, k = kc8 * 8 + e;
                         const int sq = k / kHeadChannels, c = k % kHeadChannels;
                         *dst++ = __float2bfloat16_rn(row < n ? w[(size_t)row * kK + c * 64 + sq] : 0.0f);
                     }
@@ -328,7 +336,7 @@ int launch_fc_tc(const Net &net, int batch, float *value_out, cudaStream_t s) {
     a.status = net.status_dev;
     a.batch = batch;
     a.n_policy = kFlatMoves;
-    a.n_policy_tiles = flat ? (kFlatMoves + 255) / 256 : 0;
+    a.n_policy_tiles = flat ? (kFlatMoves + kPairCols - 1) / kPairCols : 0;
     a.wdl = net.arch.value_head == AZ_VALUE_WDL;
     const int m_tiles = (batch + 127) / 128;
     // clusters of two CTAs along x (the kernel's own attribute); started as soon as the tower kernel lets its dependents go
