@@ -152,7 +152,7 @@ int build_net(Net &n, const BlobView &v) {
         n.tc_pair = pair_shape && a.precision == AZ_PREC_BF16;
         n.tc_pair8 = pair_shape && a.precision != AZ_PREC_BF16;
         const int halves = n.tc_pair ? 2 : 1;
-        tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, halves, 9, false, packed.data());
+        tc_pack_weights(w.data(), s.data(), (int)a.in_planes, n.in_pad, C, n.n_conv, halves, C == 256 ? 3 : 9, false, packed.data());
         AZ_CUDA(cudaMalloc(&n.tc_weights, bytes));
         AZ_CUDA(cudaMemcpy(n.tc_weights, packed.data(), bytes, cudaMemcpyHostToDevice));
         if (C == 256) {
@@ -183,9 +183,17 @@ int build_net(Net &n, const BlobView &v) {
         const int n_policy = flat ? kHeadChannels : kPlanes73, n_policy_pad = flat ? kHeadChannels : 80;
         n.tc_head_n = n_policy_pad + kHeadChannels;
         std::vector<__nv_bfloat16> hw(tc_head_weight_bytes(n.tc_head_n, C) / sizeof(__nv_bfloat16));
-        tc_pack_head(v.p_w, flat ? v.p_s : nullptr, n_policy, n_policy_pad, v.v_cw, v.v_cs, C, (n.tc_pair || n.tc_pair8) ? 2 : 1, hw.data());
+        const int head_halves = (n.tc_pair || n.tc_pair8) ? 2 : 1;
+        tc_pack_head(v.p_w, flat ? v.p_s : nullptr, n_policy, n_policy_pad, v.v_cw, v.v_cs, C, head_halves,
+                     tc_head_stage_slices(C, n.tc_head_n), hw.data());
         AZ_CUDA(cudaMalloc(&n.tc_head_w, hw.size() * sizeof(__nv_bfloat16)));
         AZ_CUDA(cudaMemcpy(n.tc_head_w, hw.data(), hw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
+        if (C == 256 && head_halves == 2) {
+            // the small-batch cluster kernels read the head projections whole, in plain slice order
+            tc_pack_head(v.p_w, flat ? v.p_s : nullptr, n_policy, n_policy_pad, v.v_cw, v.v_cs, C, 1, C / 16, hw.data());
+            AZ_CUDA(cudaMalloc(&n.tc_head_w_plain, hw.size() * sizeof(__nv_bfloat16)));
+            AZ_CUDA(cudaMemcpy(n.tc_head_w_plain, hw.data(), hw.size() * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice));
+        }
         std::vector<float> hb(n.tc_head_n, 0.0f);
         for (int i = 0; i < n_policy; ++i) hb[i] = v.p_b[i];
         for (int i = 0; i < kHeadChannels; ++i) hb[n_policy_pad + i] = v.v_cb[i];
@@ -268,7 +276,7 @@ void free_net(Net *n) {
     if (!n) return;
     for (int i = 0; i < 1 + 2 * 64; ++i) { cudaFree(n->conv_w[i]); cudaFree(n->conv_scale[i]); cudaFree(n->conv_bias[i]); }
     cudaFree(n->f32_layers);
-    cudaFree(n->tc_weights); cudaFree(n->tc_weights_split); cudaFree(n->tc_weights_split4); cudaFree(n->tc_bias); cudaFree(n->tc_head_w); cudaFree(n->tc_head_bias);
+    cudaFree(n->tc_weights); cudaFree(n->tc_weights_split); cudaFree(n->tc_weights_split4); cudaFree(n->tc_bias); cudaFree(n->tc_head_w); cudaFree(n->tc_head_w_plain); cudaFree(n->tc_head_bias);
     cudaFree(n->tc8_weights); cudaFree(n->tc8_lconst);
     delete static_cast<HostMaster *>(n->host_master);
     cudaFree(n->fc_policy_w); cudaFree(n->fc_value_w); cudaFree(n->u_policy); cudaFree(n->u_value);

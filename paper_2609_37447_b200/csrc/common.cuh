@@ -68,6 +68,7 @@ struct Net {
     void *host_master = nullptr;      // fp32 tower weights kept on the host until calibration (FP8 nets)
     double *calib_presum = nullptr;    // set only inside az_calibrate: where the tower kernels add up their pre-activations
     void *tc_head_w = nullptr;        // packed 1x1 head projections (policy | value), fused into the tower kernel
+    void *tc_head_w_plain = nullptr;  // 256 channels on CTA pairs: the same in plain slice order for the small-batch cluster kernels
     float *tc_head_bias = nullptr;
     int tc_head_n = 0;                // 64 (flat policy head) or 112 (73-plane policy head)
     void *fc_policy_w = nullptr;      // flat policy FC as GEMM B tiles (K permuted to square*32 + channel)
@@ -211,6 +212,7 @@ size_t tc_packed_weight_bytes(int in_pad, int channels, int n_conv);
 void tc_pack_weights(const float *const *w, const float *const *scale, int in_planes, int in_pad,
                      int channels, int n_conv, int halves, int stage_taps, bool rotate, __nv_bfloat16 *packed_host);
 bool tc_pair_shape(int channels, int precision, bool pnet);     // the tower runs on CTA pairs (weights packed in halves)
+int tc_head_stage_slices(int channels, int head_n);
 // exactly one of `planes` (encoded plane tensor) and `positions` (records to encode in the kernel) is non-null
 int launch_tower_tc(const Net &net, const void *planes, const void *positions, int batch, void *tower_out,
                     bool with_heads, unsigned int *absmax, cudaStream_t s);
@@ -220,7 +222,7 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
 int tower_tc_launch_count();
 size_t tc_head_weight_bytes(int head_n, int channels);
 void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,
-                  int channels, int halves, __nv_bfloat16 *packed);
+                  int channels, int halves, int stage_slices, __nv_bfloat16 *packed);
 
 // tensor-core fully-connected layers of the heads (fc_tc.cu)
 size_t fc_tc_weight_bytes(int n, bool policy);

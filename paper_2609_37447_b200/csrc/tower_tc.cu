@@ -90,7 +90,7 @@ struct Shape {
     static constexpr int kStageTaps = (kC == 256 && NSPLIT == 1) ? 3 : 9;
     static constexpr int kStagesPerSlice = 9 / kStageTaps;
     static constexpr int kStageBytes = kStageTaps * kTileBytes;      // 36864 / 24576; pair: 18432
-    static constexpr int kStages = NSPLIT == 4 ? 6 : NSPLIT > 1 ? 3 : kC == 256 ? 5 : PAIR ? (SETS == 2 ? 6 : 7) : 3;     // (N-split: 108 KB of 18 / 36 KB stages)
+    static constexpr int kStages = NSPLIT == 4 ? 6 : NSPLIT > 1 ? 3 : kC == 256 ? (PAIR ? 10 : 5) : PAIR ? (SETS == 2 ? 6 : 7) : 3;     // (N-split: 108 KB of 18 / 36 KB stages)
     // pair: the second group's issuer runs this many weight stages behind the first's (half a layer), so that each
     // group's layer hand-over falls into the middle of the other's layer; the halved stages make the ring deep enough
 #ifndef AZ_PAIR_LAG
@@ -260,7 +260,7 @@ tower_tc_kernel(const TowerArgs args) {
     auto bar_pdone = [&](int g) { return bar_done + 8u * (1 + kStages + kGroups + kStages + g); };   // N-split: the other CTAs' MMAs of this layer are complete
     auto bar_ack = [&](int g) { return bar_done + 8u * (1 + kStages + kGroups + kStages + kGroups + g); };   // N-split: the other CTAs hold this CTA's slices of the layer
     constexpr bool kPair = S::kPair;
-    static_assert(!kPair || (!kPnet && kGroups == 2), "CTA pairs exist for the two-group shapes of the residual networks");
+    static_assert(!kPair || !kPnet, "CTA pairs exist for the residual networks");
     constexpr int kNSplit = S::kNSplit, kN = S::kN;
     constexpr bool kCluster = kPair || kNSplit > 1;
     static_assert(kNSplit == 1 || (!kFp8 && !kPnet && kGroups == 1 && S::kSets == 1), "the N-split exists for the one-group bf16 shape of the residual networks");
@@ -493,7 +493,7 @@ tower_tc_kernel(const TowerArgs args) {
                     // one group per CTA: the slice's first weight stage is normally there long before its activations;
                     // looking at it first leaves nothing between the activations' arrival and the first MMA
                     if (kGroups == 1) {
-                        ok = wait_bar(bar_w_full(stage), phase, abort_flag, args.status, tr ? &t_wait[0] : nullptr);
+                        ok = wait_stage(stage, phase, tr ? &t_wait[0] : nullptr);
                         if (!ok) break;
                     }
                     ok = kPair ? wait_bar_cluster(bar_a_ready(g, kc), (a_phase >> kc) & 1u, abort_flag, args.status, tr ? &t_wait[1] : nullptr)
@@ -1206,6 +1206,7 @@ typedef Shape<128, 2, AZ_C128_SETS, true> Shape128Pair;    // the bf16 residual 
 typedef Shape<128, 2, AZ_FP8_EPI_SETS> Shape128F8;
 typedef Shape<128, 2, AZ_FP8_EPI_SETS, true> Shape128F8Pair;   // the 8-bit towers on CTA pairs
 typedef Shape<256, 1, 1> Shape256;
+typedef Shape<256, 1, 1, true> Shape256Pair;              // CTA pairs: each CTA its own group and half of every weight tile
 typedef Shape<256, 1, 1, false, 2> Shape256Split2;      // small batches: two CTAs per group, 128 output channels each
 typedef Shape<256, 1, 1, false, 4> Shape256Split4;      // smaller still: four CTAs per group, 64 output channels each
 // the paper's 160-channel network: one group, whose epilogue (not its MMAs) sets the pace with four warps;
@@ -1258,7 +1259,13 @@ void tc_pack_weights(const float *const *w, const float *const *scale, int in_pl
                                     }
     }
 }
-bool tc_pair_shape(int channels, int precision, bool pnet) { return channels == 128 && precision != AZ_PREC_FP32 && !pnet; }
+bool tc_pair_shape(int channels, int precision, bool pnet) {
+    return !pnet && ((channels == 128 && precision != AZ_PREC_FP32) || (channels == 256 && precision == AZ_PREC_BF16));
+}
+// 16-channel slices of the head projection's K that travel in one weight stage of the network's main tower kernel
+int tc_head_stage_slices(int channels, int head_n) {
+    return channels == 256 ? head_slices_per_stage<Shape256>(head_n) : head_slices_per_stage<Shape128>(head_n);
+}
 
 // The same tiles for a tower whose layers read different numbers of input channels (the paper's
 // network: 52 planes padded to 64 into the input layer, 3C/4 channels into the second convolution
@@ -1386,25 +1393,27 @@ void tc8_pack(const float *const *w, const float *const *scale, const float *con
 // rows of the value projection.  Same core-matrix order as the tower's weight tiles.
 size_t tc_head_weight_bytes(int head_n, int channels) { return (size_t)head_n * channels * 2; }
 
-// halves == 2 (CTA pairs, 128 channels: all eight slices travel in one stage): the stage as rows [0, head_n/2) of every
-// slice, then rows [head_n/2, head_n).
+// halves == 2 (CTA pairs): per weight stage of `stage_slices` slices, rows [0, head_n/2) of the stage's slices, then rows
+// [head_n/2, head_n) (128 channels: all eight slices are one stage).  halves == 1: plain slice order.
 void tc_pack_head(const float *wp, const float *sp, int n_policy, int n_policy_pad, const float *wv, const float *sv,
-                  int channels, int halves, __nv_bfloat16 *packed) {
+                  int channels, int halves, int stage_slices, __nv_bfloat16 *packed) {
     const int head_n = n_policy_pad + kHeadChannels;
     const int groups_per_half = head_n / 8 / halves;
+    const int n_slices = channels / 16;
     __nv_bfloat16 *dst = packed;
-    for (int h = 0; h < halves; ++h)
-        for (int kc = 0; kc < channels / 16; ++kc)
-            for (int k8 = 0; k8 < 2; ++k8)
-                for (int ng = h * groups_per_half; ng < (h + 1) * groups_per_half; ++ng)
-                    for (int r = 0; r < 8; ++r)
-                        for (int e = 0; e < 8; ++e) {
-                            const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
-                            float v = 0.0f;
-                            if (n < n_policy) v = (sp ? sp[n] : 1.0f) * wp[(size_t)n * channels + ci];
-                            else if (n >= n_policy_pad) v = sv[n - n_policy_pad] * wv[(size_t)(n - n_policy_pad) * channels + ci];
-                            *dst++ = __float2bfloat16_rn(v);
-                        }
+    for (int s0 = 0; s0 < n_slices; s0 += stage_slices)
+        for (int h = 0; h < halves; ++h)
+            for (int kc = s0; kc < s0 + stage_slices && kc < n_slices; ++kc)
+                for (int k8 = 0; k8 < 2; ++k8)
+                    for (int ng = h * groups_per_half; ng < (h + 1) * groups_per_half; ++ng)
+                        for (int r = 0; r < 8; ++r)
+                            for (int e = 0; e < 8; ++e) {
+                                const int n = ng * 8 + r, ci = kc * 16 + k8 * 8 + e;
+                                float v = 0.0f;
+                                if (n < n_policy) v = (sp ? sp[n] : 1.0f) * wp[(size_t)n * channels + ci];
+                                else if (n >= n_policy_pad) v = sv[n - n_policy_pad] * wv[(size_t)(n - n_policy_pad) * channels + ci];
+                                *dst++ = __float2bfloat16_rn(v);
+                            }
 }
 
 int launch_tower_tc(const Net &net, const void *planes, const void *positions, int batch, void *tower_out,
@@ -1427,6 +1436,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8Pair, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<true, Shape128F8Pair, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
+        AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256Pair>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256Split2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape256Split4>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
         AZ_CUDA(cudaFuncSetAttribute(tower_tc_kernel<false, Shape128P, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem));
@@ -1481,6 +1491,7 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         // channels from a copy of the weights packed for that split
         const int split = (net.tc_weights_split4 != nullptr && n_groups * 4 <= sms && AZ_NSPLIT_MAX >= 4) ? 4 : 2;
         a.weights = split == 4 ? net.tc_weights_split4 : net.tc_weights_split;
+        a.head_w = static_cast<const __nv_bfloat16 *>(net.tc_head_w_plain ? net.tc_head_w_plain : net.tc_head_w);
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(split * n_groups); cfg.blockDim = dim3(Shape256Split2::kThreads);
         cfg.dynamicSmemBytes = split == 4 ? Shape256Split4::smem_bytes(false) : Shape256Split2::smem_bytes(false); cfg.stream = s;
@@ -1490,6 +1501,19 @@ int launch_tower_tc(const Net &net, const void *planes, const void *positions, i
         cfg.attrs = attr; cfg.numAttrs = 1;
         if (split == 4) AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<false, Shape256Split4>, a));
         else AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<false, Shape256Split2>, a));
+        return AZ_OK;
+    }
+    else if (wide && net.tc_pair) {
+        // clusters of two CTAs, one group each
+        const int n_super = (n_groups + 1) / 2, pairs = n_super < sms / 2 ? n_super : sms / 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * pairs); cfg.blockDim = dim3(Shape256Pair::kThreads);
+        cfg.dynamicSmemBytes = Shape256Pair::smem_bytes(false); cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        AZ_CUDA(cudaLaunchKernelEx(&cfg, tower_tc_kernel<false, Shape256Pair>, a));
         return AZ_OK;
     }
     else if (wide) tower_tc_kernel<false, Shape256><<<grid, Shape256::kThreads, Shape256::smem_bytes(false), s>>>(a);

@@ -665,6 +665,36 @@ def test_tower_on_cta_pairs_gives_the_default_kernels_bits(az, name, batches):
     az.az_free_net(az.az_load_net_ex(az.make_arch(19, 1, 32, 0, 0, 0, 4), small, az.AZ_LOAD_TOWER_SINGLE_CTAS))
 
 
+def test_256_channel_tower_on_cta_pairs_gives_the_single_cta_kernels_bits(az):
+    # beyond 148 positions the 256-channel tower runs on CTA pairs as well (one group per CTA, each CTA half of every
+    # weight tile): same products in the same order as the one-CTA kernel, so the same bits; through more than two
+    # rounds, a ragged last pair and a lone last board; the head projections travel in several weight stages here
+    cfg = configs.tiny_config(in_planes=112, blocks=2, channels=256, policy_head=1, value_head=1, precision=1,
+                              batch=701, weight_seed=58)
+    blob = weights.make_blob(cfg, 0.5, 0.5)
+    arch = az.make_arch(112, 2, 256, 1, 1, 1, 701)
+    rec, _ = positions.generate(8123, 701, (0, 120))
+    recs = positions.records_for_planes(112, rec)
+    outs = []
+    for flags in (az.AZ_LOAD_TOWER_SINGLE_CTAS, az.AZ_LOAD_TOWER_CTA_PAIRS, 0):
+        net = az.az_load_net_ex(arch, blob, flags)
+        res = [gpu_evaluate(az, net, cfg, recs[:n])[1:] for n in (701, 301, 151)]
+        tower = torch.zeros((301, 64, 256), dtype=torch.bfloat16, device="cuda")
+        az.az_tower(net, az.records_to_device(recs[:301]), 301, tower)
+        torch.cuda.synchronize()
+        assert az.az_device_status(net) == 0
+        az.az_free_net(net)
+        outs.append((res, tower.cpu()))
+    for res, tower in outs[1:]:
+        for (p0, v0), (p1, v1) in zip(outs[0][0], res):
+            assert np.array_equal(p0, p1) and np.array_equal(v0, v1)
+        assert torch.equal(outs[0][1], tower)
+    rows = np.arange(0, 701, 25)
+    mo, _, po, vo = oracle.evaluate(blob, recs[rows], 112, 1)
+    p, v = outs[2][0][0]
+    assert np.abs(p[rows] - po).max() <= TOL[1] and np.abs(v[rows] - vo).max() <= TOL[1]
+
+
 @pytest.mark.parametrize("name", ["c4", "c4i", "c4x"])
 def test_8_bit_towers_on_cta_pairs_give_the_single_cta_kernels_bits(az, name):
     # the e4m3, int8 and e4m3-operand-pair towers run on CTA pairs by default as well; same products in the same
