@@ -155,13 +155,14 @@ int az_load_net(const az_arch *arch, const void *weights_host, size_t nbytes, az
 
 /*
  * az_load_net with options (az_load_net passes 0).
- * CTA pairs: the bf16 residual networks of 128 channels run their tower kernel as clusters of two CTAs on
- * neighbouring SMs that share every tensor-core product (tcgen05 .cta_group::2: 256 rows, 128 from each CTA; each
- * CTA keeps HALF of every weight tile in its own shared memory and bulk-copies only that half, so the operand
- * traffic of the shared-memory pipe drops from 8 to 6 KB per product and the weight traffic from L2 halves).  The
- * arithmetic and the results are those of the one-CTA kernel, bit for bit.  Measured on B200 (same box): 9 to 12 %
- * less time per evaluation at every batch size from 256 to 4096 (batch 1024: 0.527 -> 0.480 ms), which is why it is
- * the default for that shape.
+ * CTA pairs: the residual networks of 128 channels (bf16 and the 8-bit forms) and of 256 channels (bf16, more than
+ * 148 positions) run their tower kernel as clusters of two CTAs on neighbouring SMs that share every tensor-core
+ * product (tcgen05 .cta_group::2: 256 rows, 128 from each CTA; each CTA keeps HALF of every weight tile in its own
+ * shared memory and bulk-copies only that half, so the operand traffic of the shared-memory pipe drops, for 128
+ * channels from 8 to 6 KB per product, and the weight traffic from L2 halves).  The arithmetic and the results are
+ * those of the one-CTA kernel, bit for bit.  Measured on B200 (same box): 128 channels bf16 9 to 12 % less time per
+ * evaluation at every batch size from 256 to 4096 (batch 1024: 0.527 -> 0.480 ms), 256 channels 4 to 6 %, the 8-bit
+ * forms 3 to 7 %, which is why it is the default for those shapes.
  *   AZ_LOAD_TOWER_CTA_PAIRS    insist on it: AZ_ERR_UNSUPPORTED for a shape that has no such form
  *   AZ_LOAD_TOWER_SINGLE_CTAS  never: the one-CTA kernel (comparisons, tests)
  * Both, or unknown bits: BAD_ARG.
