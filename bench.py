@@ -658,7 +658,7 @@ def main():
             "dtype": DTYPE[cfg.precision], "data": "synthetic",
             "config": {"workload": WORKLOADS[cfg.name], "batch_per_gpu": B, "l2": "flushed before every step (256 MB write)",
                        "timing": "CUDA events around each step on the launch stream, summed; max over ranks",
-                       "device_status": status, "tower_cta_pairs": bool(not args.single_ctas and cfg.channels == 128 and cfg.precision == 1)},
+                       "device_status": status, "tower_cta_pairs": bool(not args.single_ctas and cfg.precision != 0 and (cfg.channels == 128 or (cfg.channels == 256 and cfg.precision == 1 and B > 148)))},
             "back_to_back": {"value": evals / (b2b_ms * 1e-3), "unit": UNIT, "ms_per_step": b2b_ms / args.steps,
                              "note": "no L2 flush between steps"},
             "gpu_launches": args.steps * az.az_launches_per_evaluate(net, B),
