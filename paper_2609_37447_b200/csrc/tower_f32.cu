@@ -58,6 +58,11 @@ __device__ __forceinline__ void cp_async16(float *smem_dst, const void *gmem_src
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+#ifndef AZ_F32_UNROLL
+#define AZ_F32_UNROLL 8
+#endif
+constexpr int kCiUnroll = AZ_F32_UNROLL;      // input channels of a chunk unrolled together in the inner loop
+
 __device__ __forceinline__ void st_async_cluster_f32(uint32_t cluster_addr, float v, uint32_t cluster_bar) {
     asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.b32 [%0], %1, [%2];"
                  ::"r"(cluster_addr), "r"(__float_as_uint(v)), "r"(cluster_bar) : "memory");
@@ -166,7 +171,7 @@ tower_f32_kernel(const F32Args args) {
         {
             const float *wb = wbuf + (idx & 1) * kChunkFloats + co;
             const float *fb = frame + cur * kFrameFloats + ((k * kChunkCi) * kRows + 2 * row_pair) * kCols;
-#pragma unroll 2
+#pragma unroll kCiUnroll
             for (int c2 = 0; c2 < kChunkCi / kSets; ++c2) {
                 const int ci = kSets * c2 + ci_set;
                 float a[4][10];
