@@ -36,7 +36,10 @@ constexpr int kSets = 2;                         // sets of four warps that shar
 constexpr int kThreads = 128 * kSets;
 constexpr int kRows = 6, kCols = 12;           // frame geometry per channel
 constexpr int kFrameFloats = kC * kRows * kCols;               // 4608 floats = 18 KB per buffer
-constexpr int kChunkCi = 16;
+#ifndef AZ_F32_CHUNK
+#define AZ_F32_CHUNK 16
+#endif
+constexpr int kChunkCi = AZ_F32_CHUNK;
 constexpr int kChunkFloats = 9 * kChunkCi * kC;                // 9216 floats = 36 KB per buffer
 constexpr int kHaloBytes = kC * 8 * 4;                          // one rank of all channels
 constexpr uint32_t kSpinLimit = 1u << 22;
